@@ -1,0 +1,251 @@
+/* ipkv.h — C ABI of the sequence-split decode-attention path over a write-time-partitioned KV cache.
+ *
+ * The library implements, for one NVIDIA B200 (sm_100a), the hot path of the InplaceKVCache /
+ * WriteScope method:
+ *
+ *   1. write-time routing of every new K/V token into the four-region layout
+ *      (device affinity x access pattern; Sec. 4.1, Sec. 4.2 of the paper),
+ *   2. attention of one decode query per sequence over the GPU-side share of the sequence,
+ *      producing a partial (O, LSE) per query head (Sec. 5.1),
+ *   3. the exact log-sum-exp join of that partial with the partial of the CPU-side share
+ *      (Sec. 4.2, Sec. 5.1).
+ *
+ * Conventions
+ *   - Every function returns an ipkv_status; nothing throws, aborts, traps the device or keeps
+ *     process-global state.  ipkv_last_error() gives the text of the last failure on a handle.
+ *   - "dev" pointers are device memory of the handle's device, "host" pointers are host memory.
+ *   - All bf16 tensors are raw 16-bit patterns.  Scores are softmax_scale * <q, k>; LSE is the
+ *     NATURAL log of the sum of exp(scores); partial outputs O are normalised (divided by their own
+ *     softmax denominator).  An empty token set gives O = 0, LSE = -inf.
+ *   - Query head h reads KV head floor(h / (n_q_heads / n_kv_heads)).
+ *   - Calls are asynchronous on the CUDA stream they are given (a cudaStream_t passed as void*;
+ *     NULL is the legacy default stream).  Host-visible results (U / P contents, statistics) are
+ *     valid after that stream has been synchronised.  One host thread per handle at a time, and the
+ *     calls on one handle must be ordered on the device: use one stream, or order streams with events
+ *     (the handle's scratch memory and staging buffers are shared by consecutive calls).
+ *   - No CPU fallback exists: without a usable CUDA device every compute entry point fails with
+ *     IPKV_ECUDA.
+ *
+ * Regions (Sec. 4.1).  U: host, unpinned, read by a CPU attention engine.  P: host, pinned, source of
+ * host-to-device loads.  W: device, the D-window that stages the newest decode tokens.  PP: device,
+ * overwrite-reused slots that P chunks are streamed through ("ping-pong").  On a GPU whose memory can
+ * hold part of the GPU-side share, `resident_tokens_per_seq` keeps the newest P blocks of each
+ * sequence in a device-side ring (a cache of P; P stays the authoritative copy) so that they need no
+ * per-step load; with 0 the layout is exactly the paper's (W + PP only).
+ *
+ * Block layouts.  A block holds `block_tokens` consecutive tokens of one (layer, sequence).
+ *   PLAIN (region U): for each KV head g: K[block_tokens][dim_qk] then V[block_tokens][dim_v],
+ *     row-major bf16.
+ *   TILE (regions P, W, PP and the resident ring): for each KV head g: the K plane then the V plane.
+ *     A plane of width d is d/64 panels; a panel is block_tokens rows of 128 bytes (64 bf16 columns);
+ *     inside a row the 16-byte chunk c (0..7) of token offset t sits at chunk position c ^ (t & 7).
+ *     Byte offset of column x of token offset t in a plane:
+ *       (x/64)*block_tokens*128 + t*128 + ((((x%64)/8) ^ (t&7))*16) + (x%8)*2.
+ *     This is the bank-conflict-free shared-memory operand layout of the attention kernel, so a
+ *     block travels host -> device -> shared memory as plain contiguous copies.
+ *   The compressed-latent kind (IPKV_MLA) stores only the K plane (dim_qk = latent + rope columns);
+ *   its V is the first dim_v columns of the same row (Sec. 6.1) and no V plane exists.
+ */
+#ifndef IPKV_H
+#define IPKV_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ipkv ipkv_t; /* opaque; owned by the library */
+
+typedef enum {
+  IPKV_OK = 0,
+  IPKV_EINVAL = 1,    /* bad argument                                            */
+  IPKV_ENOMEM = 2,    /* an allocation failed or a caller buffer is too small    */
+  IPKV_ERANGE = 3,    /* a region or the sequence capacity would be exceeded     */
+  IPKV_ESTATE = 4,    /* call not legal in the current state                     */
+  IPKV_ECUDA = 5,     /* a CUDA call failed (or no device)                       */
+  IPKV_ETIMEOUT = 6,  /* a bounded wait inside a kernel gave up                  */
+  IPKV_EINTERNAL = 7
+} ipkv_status;
+
+typedef enum { IPKV_GQA = 0, IPKV_MLA = 1 } ipkv_kind;
+typedef enum { IPKV_REGION_U = 0, IPKV_REGION_P = 1, IPKV_REGION_W = 2 } ipkv_region;
+typedef enum { IPKV_LAYOUT_PLAIN = 0, IPKV_LAYOUT_TILE = 1 } ipkv_layout;
+
+/* flags */
+#define IPKV_FLAG_NO_HOST_U 1u /* U contents are not kept (routing indices still are): for callers whose
+                                  CPU engine keeps its own copy, and for benchmarks                       */
+#define IPKV_FLAG_NO_HOST_P 2u /* no host copy of P: every P block must stay device-resident, otherwise
+                                  an append fails with IPKV_ERANGE                                        */
+
+/* The paper's PartitionSpec (Sec. 4.3): the four regions, block granularity, eviction batch size, and
+ * the share that the roofline policy of Sec. 5.3 would supply, here as an exact rational. */
+typedef struct {
+  uint32_t struct_size;           /* = sizeof(ipkv_config)                                             */
+  int32_t kind;                   /* ipkv_kind                                                         */
+  int32_t n_layers, max_seqs;
+  int32_t n_q_heads, n_kv_heads;  /* IPKV_MLA: n_kv_heads = 1                                          */
+  int32_t dim_qk, dim_v;          /* multiples of 64. GQA kernels: 64 or 128, equal; MLA: 576 / 512    */
+  int32_t block_tokens;           /* 16, 32 or a multiple of 64 (paper: "fixed-size blocks", Sec. 4.1) */
+  int32_t window_tokens;          /* D, multiple of block_tokens (Sec. 4.2; 256 in the paper)          */
+  int32_t chunk_tokens;           /* tokens per sequence in one PP slot, multiple of block_tokens       */
+  int32_t n_slots;                /* >= 2; 2 is the paper's ping-pong                                  */
+  int64_t max_u_tokens_per_seq;   /* capacity of U per (layer, sequence)                               */
+  int64_t max_p_tokens_per_seq;   /* capacity of P per (layer, sequence)                               */
+  int64_t resident_tokens_per_seq;/* device ring for the newest P blocks; 0 = stream everything        */
+  float softmax_scale;            /* 0 => 1/sqrt(dim_qk)                                               */
+  int32_t share_num, share_den;   /* marginal CPU share p = num/den of decode eviction batches         */
+  int32_t device;                 /* CUDA device ordinal                                               */
+  uint32_t flags;
+  /* Optional caller-provided memory (e.g. torch tensors); NULL => the library allocates.
+     Sizes come from ipkv_query_sizes; a smaller buffer fails with IPKV_ENOMEM. The caller keeps
+     ownership and must keep the memory alive until ipkv_destroy. Device buffers are zeroed by create. */
+  void* u_host;        size_t u_bytes;
+  void* p_host_pinned; size_t p_bytes;
+  void* w_dev;         size_t w_bytes;
+  void* resident_dev;  size_t resident_bytes;
+  void* pp_dev;        size_t pp_bytes;
+} ipkv_config;
+
+/* out_bytes[0..4] = U, P, W, resident ring, PP slots.  (Table 2 of the paper is these sizes.) */
+ipkv_status ipkv_query_sizes(const ipkv_config* cfg, size_t out_bytes[5]);
+
+/* The paper's `init` (Sec. 4.3): sizes the regions and pre-allocates them. */
+ipkv_status ipkv_create(const ipkv_config* cfg, ipkv_t** out);
+ipkv_status ipkv_destroy(ipkv_t* h);
+
+/* Marginal CPU share for later eviction batches (Sec. 5.3); same denominator as at creation. */
+ipkv_status ipkv_set_share(ipkv_t* h, int32_t num);
+
+/* Forget one sequence (seq >= 0) or all (seq = -1): its blocks are reused in place (Sec. 4.2). */
+ipkv_status ipkv_reset(ipkv_t* h, int32_t seq);
+
+/* Prefill routing in one shot (Sec. 4.2): legal only on an empty (layer, sequence).
+ * k_dev [n_tokens][n_kv_heads][dim_qk], v_dev [n_tokens][n_kv_heads][dim_v] bf16 on the device
+ * (v_dev = NULL for IPKV_MLA).  The oldest n_cpu = block_tokens * floor(floor(n_tokens/block_tokens)
+ * * num0/den0) tokens go to U, the rest to P (and into the resident ring as far as it reaches).
+ * The inputs may be reused once work queued on `stream` so far has completed. */
+ipkv_status ipkv_append_bulk(ipkv_t* h, int32_t layer, int32_t seq, const void* k_dev, const void* v_dev,
+                             int64_t n_tokens, int32_t num0, int32_t den0, void* stream);
+
+/* The paper's `append` for decode (Sec. 4.2): one new token for each listed sequence goes into its
+ * D-window; a window that is already full is flushed first, so the newest token is always GPU-side.
+ * seq_ids: host, n_seq distinct ids.  k_dev [n_seq][n_kv_heads][dim_qk], v_dev [n_seq][n_kv_heads][dim_v]. */
+ipkv_status ipkv_append(ipkv_t* h, int32_t layer, const int32_t* seq_ids, int32_t n_seq,
+                        const void* k_dev, const void* v_dev, void* stream);
+
+/* The paper's `flush` (Sec. 4.2, 4.3): evict the window of (layer, seq) as one whole batch to U or P;
+ * the side follows the integer error-diffusion rule  acc += num; if (acc >= den) { acc -= den; U } else P
+ * with acc starting at den/2, which holds the running fraction of CPU-placed batches at num/den
+ * (Sec. 5.3).  layer = -1 / seq = -1 mean all.  A placed batch never moves again.  No-op on an empty window. */
+ipkv_status ipkv_flush(ipkv_t* h, int32_t layer, int32_t seq, void* stream);
+
+typedef struct {
+  int32_t kv_splits;   /* 0 = automatic; otherwise the number of sequence chunks per (sequence, KV head) */
+  int32_t reserved;
+  void* side_stream;   /* stream for host-to-device chunk copies; NULL = the handle's own             */
+} ipkv_attend_opts;
+
+/* Attention over the GPU-side share (Sec. 5.1): the D-window plus every P token, device-resident ones
+ * read in place and the others streamed through the PP slots on the side stream while the resident part
+ * is being computed.  Which tokens are attended is fixed by the format at write time, never an argument.
+ * q_dev [n_seq][n_q_heads][dim_qk] bf16.  Outputs (fp32, device): o_part [n_seq][n_q_heads][dim_v],
+ * lse_part [n_seq][n_q_heads].  opts may be NULL. */
+ipkv_status ipkv_attend_gpu(ipkv_t* h, int32_t layer, const int32_t* seq_ids, int32_t n_seq,
+                            const void* q_dev, const ipkv_attend_opts* opts,
+                            float* o_part_dev, float* lse_part_dev, void* stream);
+
+/* Exact n-way log-sum-exp join (Sec. 4.2, 5.1) of row-aligned partials over disjoint token sets:
+ *   LSE = m + ln sum_i exp(LSE_i - m), m = max_i LSE_i;  O = sum_i exp(LSE_i - LSE) * O_i.
+ * o_parts[i] [n_rows][dim_v] fp32, lse_parts[i] [n_rows] fp32; the pointer arrays are host memory;
+ * each part may be device memory or host memory (host parts are copied on `stream` first; pinned host
+ * memory keeps that copy asynchronous).  1 <= n_parts <= 8.  o_out_dev is fp32, or bf16 (round to
+ * nearest even) when o_out_is_bf16 != 0.  lse_out_dev may be NULL.  h may be NULL only if every part is
+ * device memory. */
+ipkv_status ipkv_merge(ipkv_t* h, int32_t n_rows, int32_t dim_v, int32_t n_parts,
+                       const float* const* o_parts, const float* const* lse_parts,
+                       void* o_out_dev, int32_t o_out_is_bf16, float* lse_out_dev, void* stream);
+
+/* The paper's `views` (Sec. 4.3): zero-copy description of where a (layer, sequence) lives.
+ * One extent per placed run (prefill share, each eviction batch) plus one for the window, in token order. */
+typedef struct {
+  int32_t region;        /* ipkv_region                                                        */
+  int32_t layout;        /* ipkv_layout of the blocks                                          */
+  int64_t first_token;   /* first token index of the run in the sequence                       */
+  int64_t n_tokens;
+  int64_t region_block;  /* ordinal of the run's first block inside its region (W: 0)          */
+  const void* host_ptr;  /* first block in U or P host memory, NULL if none                    */
+  const void* dev_ptr;   /* first block on the device (W, or a fully resident P run), else NULL */
+  int64_t block_bytes;   /* consecutive blocks of a run are contiguous at this pitch           */
+} ipkv_extent;
+
+ipkv_status ipkv_views(ipkv_t* h, int32_t layer, int32_t seq, ipkv_extent* out, int32_t cap, int32_t* n_out);
+
+/* Where one token lives: region, block ordinal in the region, offset in the block (W: slot index). */
+ipkv_status ipkv_locate(ipkv_t* h, int32_t layer, int32_t seq, int64_t token,
+                        int32_t* region, int64_t* region_block, int32_t* offset_in_block);
+
+/* Token counts of (layer, seq): counts[0..2] = tokens in U, P, W; counts[3] = P tokens that are
+ * device-resident; counts[4..5] = eviction batches so far, of which CPU-placed. */
+ipkv_status ipkv_counts(ipkv_t* h, int32_t layer, int32_t seq, int64_t counts[6]);
+
+/* Copy the K (and V) row of one token, de-swizzled to plain [n_kv_heads][dim] order, into host buffers
+ * (synchronises the device; for tests and debugging).  v_out may be NULL. */
+ipkv_status ipkv_read_token(ipkv_t* h, int32_t layer, int32_t seq, int64_t token, void* k_out, void* v_out);
+
+typedef struct {
+  uint64_t attend_calls, attend_kernels, reduce_kernels, merge_kernels, append_kernels, pack_kernels;
+  uint64_t kv_bytes_attended;   /* tokens * bytes per token, summed over attend calls            */
+  uint64_t h2d_bytes, d2h_bytes, d2d_bytes;
+  uint64_t flushes, flushes_to_u;
+  uint32_t device_status;       /* nonzero after a kernel's bounded wait gave up (synchronises)  */
+} ipkv_stats;
+ipkv_status ipkv_get_stats(ipkv_t* h, ipkv_stats* out);
+
+/* ---- stateless kernel entry points (no handle) ------------------------------------------------- */
+
+typedef struct {
+  int32_t kind;                   /* ipkv_kind */
+  int32_t n_q_heads, n_kv_heads, dim_qk, dim_v, block_tokens;
+  float softmax_scale;            /* 0 => 1/sqrt(dim_qk) */
+} ipkv_attn_shape;
+
+typedef struct {
+  const void* blocks_dev;  /* first block of a run of contiguous TILE-layout blocks on the device; every
+                              block of the run must be fully allocated and hold finite values           */
+  int64_t n_tokens;        /* valid tokens in the run (the last block may be partly filled)           */
+} ipkv_run;
+
+/* Scratch needed by ipkv_attend_runs for n_rows rows, n_runs runs in total holding total_tokens tokens. */
+ipkv_status ipkv_attend_scratch_bytes(const ipkv_attn_shape* shape, int32_t n_rows, int32_t n_runs,
+                                      int64_t total_tokens, int32_t kv_splits, size_t* out_bytes);
+
+/* Split-K decode attention (Sec. 5.1, GPU side) of n_rows queries, row r over the union of the runs
+ * runs[row_run_start[r] .. row_run_start[r+1]).  runs and row_run_start are host arrays.
+ * scratch_dev: device memory of at least ipkv_attend_scratch_bytes (256-byte aligned), private to this
+ * call until the work queued on `stream` has completed.  Outputs as in ipkv_attend_gpu.
+ * status_dev: optional device uint32 that receives a nonzero value if a bounded wait gave up. */
+ipkv_status ipkv_attend_runs(const ipkv_attn_shape* shape, int32_t n_rows,
+                             const ipkv_run* runs, const int32_t* row_run_start,
+                             const void* q_dev, int32_t kv_splits,
+                             void* scratch_dev, size_t scratch_bytes,
+                             float* o_part_dev, float* lse_part_dev, uint32_t* status_dev, void* stream);
+
+/* Re-lay token-major K/V ([n_tokens][n_kv_heads][dim]) into consecutive blocks of the given layout
+ * starting at token offset 0 of dst_dev (device to device; used by tests and by callers that build
+ * blocks themselves).  v_dev = NULL for IPKV_MLA. */
+ipkv_status ipkv_pack_blocks(const ipkv_attn_shape* shape, int32_t layout, const void* k_dev, const void* v_dev,
+                             int64_t n_tokens, void* dst_dev, void* stream);
+
+/* Bytes of one block for a shape. */
+int64_t ipkv_block_bytes(const ipkv_attn_shape* shape);
+
+const char* ipkv_status_str(ipkv_status s);
+const char* ipkv_last_error(const ipkv_t* h);
+const char* ipkv_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* IPKV_H */

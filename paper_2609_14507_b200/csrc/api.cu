@@ -1,0 +1,937 @@
+// C ABI of the library (include/ipkv.h): the handle, the host-side scheduler that turns the routing
+// state into kernel launches and copies, and the stateless entry points.
+//
+// Decode step of one layer (Sec. 4.2, Sec. 5.1):
+//   ipkv_append      router -> append kernel (new token into the D-window); a full window is evicted first
+//                    (whole batch, device -> host on the idle D2H direction, TILE -> PLAIN for U)
+//   ipkv_attend_gpu  split-K attention over the resident ring and the D-window; P chunks that are not
+//                    device-resident are copied H2D into PP slots on a side stream, each slot attended as
+//                    soon as its copy has landed and folded into the running partial
+//   ipkv_merge       LSE join with the CPU-side partial
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "../../include/ipkv.h"
+#include "kernels.h"
+#include "plan.hpp"
+#include "router.hpp"
+
+namespace ipkvi {
+cudaError_t launch_attend_gqa(const AttnLaunch& a, cudaStream_t s);
+cudaError_t launch_attend_mla(const AttnLaunch& a, cudaStream_t s);
+
+cudaError_t launch_attend(const AttnLaunch& a, cudaStream_t s) {
+    return a.kind == IPKV_MLA ? launch_attend_mla(a, s) : launch_attend_gqa(a, s);
+}
+}  // namespace ipkvi
+
+using namespace ipkvi;
+
+namespace {
+
+
+struct PRun {            // maximal run of P blocks that the attention kernel can walk as one segment
+    int64_t first_block;
+    int64_t n_tokens;
+};
+
+struct SeqState {
+    SeqRouter router;
+    std::vector<PRun> p_runs;
+};
+
+size_t partial_bytes(size_t n_items, int Hq, int dv) {
+    return align_up(n_items * size_t(Hq) * dv * sizeof(float), 256) + align_up(n_items * size_t(Hq) * sizeof(float), 256);
+}
+
+int64_t max_items_bound(int n_rows, int n_runs, int64_t total_tokens, int kv_splits) {
+    const int64_t tiles = (total_tokens + kTileTokens - 1) / kTileTokens + n_runs;
+    if (kv_splits > 0) return int64_t(n_runs) * (kv_splits + 1) + n_rows;
+    return std::max<int64_t>(int64_t(kSmCount) * kCtasPerSm, tiles / 8) + n_runs + n_rows;
+}
+
+bool shape_ok(int kind, int Hq, int Hkv, int dqk, int dv, int bt, std::string* why) {
+    auto fail = [&](const char* m) { if (why) *why = m; return false; };
+    if (Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0) return fail("n_q_heads must be a positive multiple of n_kv_heads");
+    if (!(bt == 16 || bt == 32 || (bt > 0 && bt % 64 == 0))) return fail("block_tokens must be 16, 32 or a multiple of 64");
+    if (kind == IPKV_GQA) {
+        if (!((dqk == 128 && dv == 128) || (dqk == 64 && dv == 64))) return fail("GQA kernels support dim_qk = dim_v in {64, 128}");
+    } else if (kind == IPKV_MLA) {
+        if (Hkv != 1) return fail("the compressed-latent kind has one shared KV head");
+        if (dqk != 576 || dv != 512) return fail("the compressed-latent kernel supports dim_qk 576 / dim_v 512");
+        if (Hq > 128) return fail("the compressed-latent kernel supports at most 128 query heads");
+    } else {
+        return fail("unknown kind");
+    }
+    return true;
+}
+
+BlockGeom make_geom(int kind, int Hkv, int dqk, int dv, int bt) {
+    BlockGeom g;
+    g.n_kv_heads = Hkv; g.dim_qk = dqk; g.dim_v_stored = (kind == IPKV_MLA) ? 0 : dv; g.bt = bt;
+    return g;
+}
+
+}  // namespace
+
+// ---- the handle ---------------------------------------------------------------------------------
+struct ipkv {
+    ipkv_config cfg;
+    BlockGeom geom;
+    float scale = 0.f;
+    int64_t bb = 0;                 // block bytes
+    int64_t u_cap = 0, p_cap = 0;   // blocks per (layer, seq)
+    int64_t ring = 0;               // resident blocks per (layer, seq)
+    int64_t w_blocks = 0, chunk_blocks = 0;
+    size_t sizes[5] = {0, 0, 0, 0, 0};
+    char *u_host = nullptr, *p_host = nullptr, *w_dev = nullptr, *res_dev = nullptr, *pp_dev = nullptr;
+    bool own[5] = {false, false, false, false, false};
+    std::vector<SeqState> st;
+    // staging for layout conversion on the way to host memory
+    char* staging = nullptr;
+    size_t staging_bytes = 0;
+    // split-K scratch: descriptor tables + partials
+    char* scratch = nullptr;
+    size_t scratch_bytes = 0;
+    char* table_pinned = nullptr;   // ring of pinned table images, mirrored at the same offsets on the device
+    char* table_dev = nullptr;
+    size_t table_cap = 0, table_head = 0;
+    static constexpr int kTableParts = 8;
+    cudaEvent_t table_ev[kTableParts] = {};
+    bool table_ev_set[kTableParts] = {};
+    int table_part = 0;
+    std::vector<char> last_table;
+    size_t last_table_off = 0;
+    cudaStream_t last_table_stream = nullptr;
+    bool last_table_valid = false;
+    // merge staging for host-side partials
+    char* merge_stage = nullptr;
+    size_t merge_stage_bytes = 0;
+    uint32_t* status_dev = nullptr;
+    cudaStream_t side = nullptr;
+    std::vector<cudaEvent_t> slot_ready, slot_free;
+    std::vector<char> slot_free_set;
+    cudaEvent_t ev_main = nullptr;
+    ipkv_stats stats;
+    std::string err;
+
+    SeqState& state(int layer, int seq) { return st[size_t(layer) * cfg.max_seqs + seq]; }
+    int64_t seq_index(int layer, int seq) const { return int64_t(layer) * cfg.max_seqs + seq; }
+    char* u_ptr(int layer, int seq, int64_t blk) { return u_host + (seq_index(layer, seq) * u_cap + blk) * bb; }
+    char* p_ptr(int layer, int seq, int64_t blk) { return p_host + (seq_index(layer, seq) * p_cap + blk) * bb; }
+    int64_t w_off(int seq) const { return int64_t(seq) * w_blocks * bb; }                       // inside a layer
+    char* w_layer(int layer) { return w_dev + int64_t(layer) * cfg.max_seqs * w_blocks * bb; }
+    int64_t ring_off(int seq) const { return int64_t(seq) * ring * bb; }                        // inside a layer
+    char* ring_layer(int layer) { return res_dev + int64_t(layer) * cfg.max_seqs * ring * bb; }
+    int64_t slot_bytes() const { return int64_t(cfg.max_seqs) * chunk_blocks * bb; }
+};
+
+namespace {
+
+ipkv_status fail(ipkv* h, ipkv_status s, const std::string& msg) {
+    if (h) h->err = msg;
+    return s;
+}
+ipkv_status fail_cuda(ipkv* h, cudaError_t e, const char* what) {
+    return fail(h, IPKV_ECUDA, std::string(what) + ": " + cudaGetErrorString(e));
+}
+#define CU(h, call)                                                  \
+    do {                                                             \
+        cudaError_t e__ = (call);                                    \
+        if (e__ != cudaSuccess) return fail_cuda((h), e__, #call);   \
+    } while (0)
+
+ipkv_status validate(const ipkv_config* c, std::string* why) {
+    auto bad = [&](const char* m) { *why = m; return IPKV_EINVAL; };
+    if (!c) return bad("config is NULL");
+    if (c->struct_size != sizeof(ipkv_config)) return bad("struct_size does not match this library's ipkv_config");
+    if (c->n_layers <= 0 || c->max_seqs <= 0) return bad("n_layers and max_seqs must be positive");
+    if (!shape_ok(c->kind, c->n_q_heads, c->n_kv_heads, c->dim_qk, c->dim_v, c->block_tokens, why)) return IPKV_EINVAL;
+    if (c->window_tokens <= 0 || c->window_tokens % c->block_tokens != 0) return bad("window_tokens must be a positive multiple of block_tokens");
+    if (c->chunk_tokens <= 0 || c->chunk_tokens % c->block_tokens != 0) return bad("chunk_tokens must be a positive multiple of block_tokens");
+    if (c->n_slots < 2) return bad("n_slots must be at least 2");
+    if (c->max_u_tokens_per_seq < 0 || c->max_p_tokens_per_seq < 0 || c->resident_tokens_per_seq < 0) return bad("negative capacity");
+    if (c->share_den <= 0 || c->share_num < 0 || c->share_num > c->share_den) return bad("share must satisfy 0 <= num <= den, den > 0");
+    if (!(c->softmax_scale >= 0.f) || std::isinf(c->softmax_scale)) return bad("softmax_scale must be finite and non-negative");
+    return IPKV_OK;
+}
+
+void compute_sizes(const ipkv_config* c, int64_t* bb, int64_t* u_cap, int64_t* p_cap, int64_t* ring, size_t sizes[5]) {
+    const BlockGeom g = make_geom(c->kind, c->n_kv_heads, c->dim_qk, c->dim_v, c->block_tokens);
+    *bb = g.block_bytes();
+    const int64_t bt = c->block_tokens;
+    // +1 block: a run always starts on a block boundary, so an explicit partial eviction can waste one
+    *u_cap = (c->max_u_tokens_per_seq + bt - 1) / bt + (c->max_u_tokens_per_seq > 0 ? 1 : 0);
+    *p_cap = (c->max_p_tokens_per_seq + bt - 1) / bt + (c->max_p_tokens_per_seq > 0 ? 1 : 0);
+    *ring = (c->resident_tokens_per_seq + bt - 1) / bt;
+    const int64_t seqs = int64_t(c->n_layers) * c->max_seqs;
+    sizes[0] = (c->flags & IPKV_FLAG_NO_HOST_U) ? 0 : size_t(seqs * *u_cap * *bb);
+    sizes[1] = (c->flags & IPKV_FLAG_NO_HOST_P) ? 0 : size_t(seqs * *p_cap * *bb);
+    sizes[2] = size_t(seqs * (c->window_tokens / bt) * *bb);
+    sizes[3] = size_t(seqs * *ring * *bb);
+    sizes[4] = size_t(int64_t(c->n_slots) * c->max_seqs * (c->chunk_tokens / bt) * *bb);
+}
+
+ipkv_status check_ls(ipkv* h, int layer, int seq) {
+    if (!h) return IPKV_EINVAL;
+    if (layer < 0 || layer >= h->cfg.n_layers) return fail(h, IPKV_EINVAL, "layer out of range");
+    if (seq < 0 || seq >= h->cfg.max_seqs) return fail(h, IPKV_EINVAL, "sequence id out of range");
+    return IPKV_OK;
+}
+
+// Record a P run for the attention scheduler: consecutive whole blocks extend the previous run.
+void note_p_run(SeqState& s, const Run& r, int64_t bt) {
+    if (!s.p_runs.empty()) {
+        PRun& last = s.p_runs.back();
+        if (last.n_tokens % bt == 0 && last.first_block + last.n_tokens / bt == r.first_block) {
+            last.n_tokens += r.n_tokens;
+            return;
+        }
+    }
+    s.p_runs.push_back(PRun{r.first_block, r.n_tokens});
+}
+
+// Copy blocks [j0, j1) of a P run from `src` (contiguous, block j0 first) into the resident ring.
+ipkv_status ring_store(ipkv* h, int layer, int seq, int64_t j0, int64_t j1, const char* src, cudaStream_t s) {
+    if (h->ring == 0) return IPKV_OK;
+    if (j1 - j0 > h->ring) { src += (j1 - j0 - h->ring) * h->bb; j0 = j1 - h->ring; }   // only the newest fit
+    char* base = h->ring_layer(layer) + h->ring_off(seq);
+    while (j0 < j1) {
+        const int64_t pos = j0 % h->ring;
+        const int64_t n = std::min(j1 - j0, h->ring - pos);
+        CU(h, cudaMemcpyAsync(base + pos * h->bb, src, size_t(n * h->bb), cudaMemcpyDeviceToDevice, s));
+        h->stats.d2d_bytes += uint64_t(n * h->bb);
+        src += n * h->bb; j0 += n;
+    }
+    return IPKV_OK;
+}
+
+ipkv_status ensure_staging(ipkv* h, size_t bytes) {
+    if (h->staging_bytes >= bytes) return IPKV_OK;
+    CU(h, cudaDeviceSynchronize());
+    if (h->staging) cudaFree(h->staging);
+    h->staging = nullptr; h->staging_bytes = 0;
+    CU(h, cudaMalloc(&h->staging, bytes));
+    h->staging_bytes = bytes;
+    return IPKV_OK;
+}
+
+ipkv_status do_flush(ipkv* h, int layer, int seq, cudaStream_t s) {
+    SeqState& st = h->state(layer, seq);
+    const int64_t fill = st.router.window_fill();
+    if (fill == 0) return IPKV_OK;
+    const int64_t nb = st.router.blocks_for(fill);
+    const int side = st.router.peek_eviction_side();
+    const bool no_u = h->cfg.flags & IPKV_FLAG_NO_HOST_U, no_p = h->cfg.flags & IPKV_FLAG_NO_HOST_P;
+    if (side == REGION_U) {
+        if (st.router.blocks_used(REGION_U) + nb > h->u_cap) return fail(h, IPKV_ERANGE, "eviction would exceed the capacity of U");
+    } else {
+        if (st.router.blocks_used(REGION_P) + nb > h->p_cap) return fail(h, IPKV_ERANGE, "eviction would exceed the capacity of P");
+        if (no_p && st.router.blocks_used(REGION_P) + nb > h->ring)
+            return fail(h, IPKV_ERANGE, "eviction would push P blocks out of the resident ring, and no host copy of P exists");
+    }
+    const Run r = st.router.evict();
+    const char* src = h->w_layer(layer) + h->w_off(seq);
+    h->stats.flushes += 1;
+    if (r.region == REGION_U) {
+        h->stats.flushes_to_u += 1;
+        if (!no_u) {
+            ipkv_status rc = ensure_staging(h, size_t(nb * h->bb));
+            if (rc != IPKV_OK) return rc;
+            CU(h, launch_tile_to_plain(h->geom, src, h->staging, nb, s));
+            h->stats.pack_kernels += 1;
+            CU(h, cudaMemcpyAsync(h->u_ptr(layer, seq, r.first_block), h->staging, size_t(nb * h->bb), cudaMemcpyDeviceToHost, s));
+            h->stats.d2h_bytes += uint64_t(nb * h->bb);
+        }
+    } else {
+        if (!no_p) {
+            CU(h, cudaMemcpyAsync(h->p_ptr(layer, seq, r.first_block), src, size_t(nb * h->bb), cudaMemcpyDeviceToHost, s));
+            h->stats.d2h_bytes += uint64_t(nb * h->bb);
+        }
+        ipkv_status rc = ring_store(h, layer, seq, r.first_block, r.first_block + nb, src, s);
+        if (rc != IPKV_OK) return rc;
+        note_p_run(st, r, h->cfg.block_tokens);
+    }
+    return IPKV_OK;
+}
+
+// Upload a table image; returns its device address. Identical consecutive images are uploaded once.
+ipkv_status upload_table(ipkv* h, const Plan& plan, cudaStream_t s, const char** dev_out) {
+    const size_t bytes = align_up(plan.table_bytes(), 256);
+    std::vector<char> img(bytes, 0);
+    plan.serialize(img.data());
+    if (h->last_table_valid && h->last_table_stream == s && h->last_table.size() == bytes &&
+        std::memcmp(h->last_table.data(), img.data(), bytes) == 0) {
+        *dev_out = h->table_dev + h->last_table_off;
+        return IPKV_OK;
+    }
+    const size_t part_cap = h->table_cap / ipkv::kTableParts;
+    if (bytes > part_cap) {
+        // grow the rings (rare: very large batches)
+        CU(h, cudaDeviceSynchronize());
+        const size_t cap = align_up(bytes * ipkv::kTableParts * 2, 4096);
+        if (h->table_pinned) cudaFreeHost(h->table_pinned);
+        if (h->table_dev) cudaFree(h->table_dev);
+        h->table_pinned = nullptr; h->table_dev = nullptr; h->table_cap = 0;
+        CU(h, cudaMallocHost(&h->table_pinned, cap));
+        CU(h, cudaMalloc(&h->table_dev, cap));
+        h->table_cap = cap; h->table_head = 0; h->table_part = 0;
+        for (int i = 0; i < ipkv::kTableParts; ++i) h->table_ev_set[i] = false;
+        h->last_table_valid = false;
+    }
+    const size_t pc = h->table_cap / ipkv::kTableParts;
+    size_t part_begin = size_t(h->table_part) * pc;
+    if (h->table_head + bytes > part_begin + pc || (h->last_table_valid && h->last_table_stream != s)) {
+        // leave this part: mark it with an event on the stream that used it, enter the next one when it is free
+        if (h->last_table_valid) {
+            CU(h, cudaEventRecord(h->table_ev[h->table_part], h->last_table_stream));
+            h->table_ev_set[h->table_part] = true;
+        }
+        h->table_part = (h->table_part + 1) % ipkv::kTableParts;
+        if (h->table_ev_set[h->table_part]) CU(h, cudaEventSynchronize(h->table_ev[h->table_part]));
+        part_begin = size_t(h->table_part) * pc;
+        h->table_head = part_begin;
+    }
+    const size_t off = h->table_head;
+    std::memcpy(h->table_pinned + off, img.data(), bytes);
+    CU(h, cudaMemcpyAsync(h->table_dev + off, h->table_pinned + off, bytes, cudaMemcpyHostToDevice, s));
+    h->stats.h2d_bytes += bytes;
+    h->table_head += bytes;
+    h->last_table.swap(img);
+    h->last_table_off = off; h->last_table_stream = s; h->last_table_valid = true;
+    *dev_out = h->table_dev + off;
+    return IPKV_OK;
+}
+
+ipkv_status ensure_scratch(ipkv* h, size_t bytes) {
+    if (h->scratch_bytes >= bytes) return IPKV_OK;
+    CU(h, cudaDeviceSynchronize());
+    if (h->scratch) cudaFree(h->scratch);
+    h->scratch = nullptr; h->scratch_bytes = 0;
+    const size_t want = align_up(bytes + bytes / 4, 1 << 20);
+    CU(h, cudaMalloc(&h->scratch, want));
+    h->scratch_bytes = want;
+    return IPKV_OK;
+}
+
+void fill_launch(AttnLaunch* a, int kind, int Hq, int Hkv, int dqk, int dv, int bt, float scale, const Plan& plan,
+                 const char* table_dev, char* partials, const void* q, int n_rows) {
+    a->kind = kind; a->n_q_heads = Hq; a->n_kv_heads = Hkv; a->dim_qk = dqk; a->dim_v = dv; a->bt = bt; a->scale = scale;
+    a->q = q;
+    size_t o = 0;
+    a->segs = reinterpret_cast<const Seg*>(table_dev + o);
+    o += align_up(plan.segs.size() * sizeof(Seg), 16);
+    a->items = reinterpret_cast<const Item*>(table_dev + o);
+    o += align_up(plan.items.size() * sizeof(Item), 16);
+    a->row_item_start = reinterpret_cast<const int32_t*>(table_dev + o);
+    a->n_items = int(plan.items.size());
+    a->n_rows = n_rows;
+    a->part_o = reinterpret_cast<float*>(partials);
+    a->part_lse = reinterpret_cast<float*>(partials + align_up(plan.items.size() * size_t(Hq) * dv * sizeof(float), 256));
+}
+
+int heads_per_tile(int kind, int Hq, int Hkv) {
+    if (kind == IPKV_MLA) return 1;
+    const int G = Hq / Hkv;
+    return Hkv * ((G + 15) / 16);
+}
+
+// One group of segments for all rows: attention + split reduce, folding into (out_o, out_lse) when `fold`.
+ipkv_status run_group(ipkv* h, const std::vector<std::vector<PlanSeg>>& rows, const char* const bases[kMaxBases],
+                      const void* q, int kv_splits, bool fold, float* out_o, float* out_lse, cudaStream_t s) {
+    const ipkv_config& c = h->cfg;
+    Plan plan;
+    build_plan(rows, heads_per_tile(c.kind, c.n_q_heads, c.n_kv_heads), kv_splits, &plan);
+    ipkv_status rc = ensure_scratch(h, partial_bytes(plan.items.size(), c.n_q_heads, c.dim_v));
+    if (rc != IPKV_OK) return rc;
+    const char* table = nullptr;
+    rc = upload_table(h, plan, s, &table);
+    if (rc != IPKV_OK) return rc;
+    AttnLaunch a{};
+    fill_launch(&a, c.kind, c.n_q_heads, c.n_kv_heads, c.dim_qk, c.dim_v, c.block_tokens, h->scale, plan, table, h->scratch, q,
+                int(rows.size()));
+    for (int i = 0; i < kMaxBases; ++i) a.bases[i] = bases[i];
+    a.acc_o = fold ? out_o : nullptr;
+    a.acc_lse = fold ? out_lse : nullptr;
+    a.out_o = out_o; a.out_lse = out_lse;
+    a.status = h->status_dev;
+    if (a.n_items > 0) {
+        CU(h, launch_attend(a, s));
+        h->stats.attend_kernels += 1;
+    }
+    CU(h, launch_split_reduce(a, s));
+    h->stats.reduce_kernels += 1;
+    h->stats.kv_bytes_attended += uint64_t(plan.total_tokens) * uint64_t(h->bb / c.block_tokens);
+    return IPKV_OK;
+}
+
+}  // namespace
+
+// ---- C ABI --------------------------------------------------------------------------------------
+extern "C" {
+
+const char* ipkv_version(void) { return "ipkv 0.1 (sm_100a)"; }
+
+const char* ipkv_status_str(ipkv_status s) {
+    switch (s) {
+        case IPKV_OK: return "ok";
+        case IPKV_EINVAL: return "invalid argument";
+        case IPKV_ENOMEM: return "out of memory";
+        case IPKV_ERANGE: return "capacity exceeded";
+        case IPKV_ESTATE: return "illegal in this state";
+        case IPKV_ECUDA: return "CUDA error";
+        case IPKV_ETIMEOUT: return "device wait timed out";
+        case IPKV_EINTERNAL: return "internal error";
+    }
+    return "unknown status";
+}
+
+const char* ipkv_last_error(const ipkv_t* h) { return h ? h->err.c_str() : "no handle"; }
+
+ipkv_status ipkv_query_sizes(const ipkv_config* cfg, size_t out_bytes[5]) {
+    std::string why;
+    ipkv_status rc = validate(cfg, &why);
+    if (rc != IPKV_OK || !out_bytes) return IPKV_EINVAL;
+    int64_t bb, u_cap, p_cap, ring;
+    compute_sizes(cfg, &bb, &u_cap, &p_cap, &ring, out_bytes);
+    return IPKV_OK;
+}
+
+ipkv_status ipkv_destroy(ipkv_t* h) {
+    if (!h) return IPKV_OK;
+    cudaSetDevice(h->cfg.device);
+    cudaDeviceSynchronize();
+    if (h->own[0] && h->u_host) std::free(h->u_host);
+    if (h->own[1] && h->p_host) cudaFreeHost(h->p_host);
+    if (h->own[2] && h->w_dev) cudaFree(h->w_dev);
+    if (h->own[3] && h->res_dev) cudaFree(h->res_dev);
+    if (h->own[4] && h->pp_dev) cudaFree(h->pp_dev);
+    if (h->staging) cudaFree(h->staging);
+    if (h->scratch) cudaFree(h->scratch);
+    if (h->table_pinned) cudaFreeHost(h->table_pinned);
+    if (h->table_dev) cudaFree(h->table_dev);
+    if (h->merge_stage) cudaFree(h->merge_stage);
+    if (h->status_dev) cudaFree(h->status_dev);
+    for (int i = 0; i < ipkv::kTableParts; ++i) if (h->table_ev[i]) cudaEventDestroy(h->table_ev[i]);
+    for (auto e : h->slot_ready) cudaEventDestroy(e);
+    for (auto e : h->slot_free) cudaEventDestroy(e);
+    if (h->ev_main) cudaEventDestroy(h->ev_main);
+    if (h->side) cudaStreamDestroy(h->side);
+    delete h;
+    return IPKV_OK;
+}
+
+ipkv_status ipkv_create(const ipkv_config* cfg, ipkv_t** out) {
+    if (!out) return IPKV_EINVAL;
+    *out = nullptr;
+    std::string why;
+    ipkv_status rc = validate(cfg, &why);
+    if (rc != IPKV_OK) return rc;
+    int n_dev = 0;
+    if (cudaGetDeviceCount(&n_dev) != cudaSuccess || cfg->device < 0 || cfg->device >= n_dev) return IPKV_ECUDA;
+    if (cudaSetDevice(cfg->device) != cudaSuccess) return IPKV_ECUDA;
+    ipkv* h = new (std::nothrow) ipkv();
+    if (!h) return IPKV_ENOMEM;
+    h->cfg = *cfg;
+    std::memset(&h->stats, 0, sizeof h->stats);
+    h->geom = make_geom(cfg->kind, cfg->n_kv_heads, cfg->dim_qk, cfg->dim_v, cfg->block_tokens);
+    h->scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / std::sqrt(float(cfg->dim_qk));
+    compute_sizes(cfg, &h->bb, &h->u_cap, &h->p_cap, &h->ring, h->sizes);
+    h->w_blocks = cfg->window_tokens / cfg->block_tokens;
+    h->chunk_blocks = cfg->chunk_tokens / cfg->block_tokens;
+
+    auto bail = [&](ipkv_status s) { ipkv_destroy(h); return s; };
+    struct Prov { void* p; size_t n; } prov[5] = {{cfg->u_host, cfg->u_bytes}, {cfg->p_host_pinned, cfg->p_bytes},
+                                                  {cfg->w_dev, cfg->w_bytes}, {cfg->resident_dev, cfg->resident_bytes},
+                                                  {cfg->pp_dev, cfg->pp_bytes}};
+    char** dst[5] = {&h->u_host, &h->p_host, &h->w_dev, &h->res_dev, &h->pp_dev};
+    for (int i = 0; i < 5; ++i) {
+        if (h->sizes[i] == 0) continue;
+        if (prov[i].p) {
+            if (prov[i].n < h->sizes[i]) return bail(IPKV_ENOMEM);
+            *dst[i] = static_cast<char*>(prov[i].p);
+        } else {
+            void* p = nullptr;
+            if (i == 0) { p = std::malloc(h->sizes[i]); if (!p) return bail(IPKV_ENOMEM); }
+            else if (i == 1) { if (cudaMallocHost(&p, h->sizes[i]) != cudaSuccess) return bail(IPKV_ENOMEM); }
+            else { if (cudaMalloc(&p, h->sizes[i]) != cudaSuccess) return bail(IPKV_ENOMEM); }
+            *dst[i] = static_cast<char*>(p);
+            h->own[i] = true;
+        }
+        if (i >= 2 && cudaMemset(*dst[i], 0, h->sizes[i]) != cudaSuccess) return bail(IPKV_ECUDA);
+    }
+    h->st.resize(size_t(cfg->n_layers) * cfg->max_seqs);
+    for (auto& s : h->st) s.router.init(cfg->block_tokens, cfg->window_tokens, cfg->share_num, cfg->share_den);
+
+    if (cudaMalloc(&h->status_dev, 256) != cudaSuccess) return bail(IPKV_ENOMEM);
+    if (cudaMemset(h->status_dev, 0, 256) != cudaSuccess) return bail(IPKV_ECUDA);
+    h->table_cap = 1 << 20;
+    if (cudaMallocHost(&h->table_pinned, h->table_cap) != cudaSuccess) return bail(IPKV_ENOMEM);
+    if (cudaMalloc(&h->table_dev, h->table_cap) != cudaSuccess) return bail(IPKV_ENOMEM);
+    for (int i = 0; i < ipkv::kTableParts; ++i)
+        if (cudaEventCreateWithFlags(&h->table_ev[i], cudaEventDisableTiming) != cudaSuccess) return bail(IPKV_ECUDA);
+    if (cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking) != cudaSuccess) return bail(IPKV_ECUDA);
+    h->slot_ready.resize(cfg->n_slots); h->slot_free.resize(cfg->n_slots); h->slot_free_set.assign(cfg->n_slots, 0);
+    for (int i = 0; i < cfg->n_slots; ++i) {
+        if (cudaEventCreateWithFlags(&h->slot_ready[i], cudaEventDisableTiming) != cudaSuccess) return bail(IPKV_ECUDA);
+        if (cudaEventCreateWithFlags(&h->slot_free[i], cudaEventDisableTiming) != cudaSuccess) return bail(IPKV_ECUDA);
+    }
+    if (cudaEventCreateWithFlags(&h->ev_main, cudaEventDisableTiming) != cudaSuccess) return bail(IPKV_ECUDA);
+    if (cudaDeviceSynchronize() != cudaSuccess) return bail(IPKV_ECUDA);
+    *out = h;
+    return IPKV_OK;
+}
+
+ipkv_status ipkv_set_share(ipkv_t* h, int32_t num) {
+    if (!h) return IPKV_EINVAL;
+    if (num < 0 || num > h->cfg.share_den) return fail(h, IPKV_EINVAL, "share numerator out of range");
+    h->cfg.share_num = num;
+    for (auto& s : h->st) s.router.set_share(num);
+    return IPKV_OK;
+}
+
+ipkv_status ipkv_reset(ipkv_t* h, int32_t seq) {
+    if (!h) return IPKV_EINVAL;
+    if (seq < -1 || seq >= h->cfg.max_seqs) return fail(h, IPKV_EINVAL, "sequence id out of range");
+    for (int l = 0; l < h->cfg.n_layers; ++l)
+        for (int s = 0; s < h->cfg.max_seqs; ++s)
+            if (seq < 0 || s == seq) { h->state(l, s).router.clear(); h->state(l, s).p_runs.clear(); }
+    h->last_table_valid = false;
+    return IPKV_OK;
+}
+
+ipkv_status ipkv_append_bulk(ipkv_t* h, int32_t layer, int32_t seq, const void* k_dev, const void* v_dev,
+                             int64_t n_tokens, int32_t num0, int32_t den0, void* stream) {
+    ipkv_status rc = check_ls(h, layer, seq);
+    if (rc != IPKV_OK) return rc;
+    const ipkv_config& c = h->cfg;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (n_tokens < 0 || den0 <= 0 || num0 < 0 || num0 > den0) return fail(h, IPKV_EINVAL, "bad token count or prefill share");
+    if (n_tokens > 0 && (!k_dev || (c.kind == IPKV_GQA && !v_dev))) return fail(h, IPKV_EINVAL, "K/V pointer is NULL");
+    SeqState& st = h->state(layer, seq);
+    if (st.router.length() != 0) return fail(h, IPKV_ESTATE, "bulk append is only legal on an empty sequence");
+    const int64_t bt = c.block_tokens;
+    const int64_t n_cpu = st.router.prefill_cpu_tokens(n_tokens, num0, den0);
+    const int64_t n_gpu = n_tokens - n_cpu;
+    const bool no_u = c.flags & IPKV_FLAG_NO_HOST_U, no_p = c.flags & IPKV_FLAG_NO_HOST_P;
+    if (st.router.blocks_for(n_cpu) > h->u_cap) return fail(h, IPKV_ERANGE, "prefill exceeds the capacity of U");
+    if (st.router.blocks_for(n_gpu) > h->p_cap) return fail(h, IPKV_ERANGE, "prefill exceeds the capacity of P");
+    if (no_p && st.router.blocks_for(n_gpu) > h->ring) return fail(h, IPKV_ERANGE, "prefill exceeds the resident ring and no host copy of P exists");
+    CU(h, cudaSetDevice(c.device));
+    Run placed[2];
+    const int n_runs = st.router.bulk(n_tokens, num0, den0, placed);
+    const int64_t k_row = int64_t(c.n_kv_heads) * c.dim_qk * 2, v_row = int64_t(c.n_kv_heads) * c.dim_v * 2;
+    const size_t stage_cap = size_t(std::max<int64_t>(h->bb, (int64_t(32) << 20) / h->bb * h->bb));
+    for (int i = 0; i < n_runs; ++i) {
+        const Run& r = placed[i];
+        const int64_t nb = st.router.blocks_for(r.n_tokens);
+        const bool to_u = r.region == REGION_U;
+        if (!to_u) note_p_run(st, r, bt);
+        if (to_u && no_u) continue;
+        const int64_t first_resident = to_u ? nb : std::max<int64_t>(0, nb - h->ring);   // relative block index
+        int64_t j = 0;
+        while (j < nb) {
+            const bool resident = !to_u && j >= first_resident;
+            int64_t j_end;
+            char* dst;
+            if (resident) {
+                const int64_t pos = (r.first_block + j) % h->ring;
+                j_end = std::min(nb, j + (h->ring - pos));
+                dst = h->ring_layer(layer) + h->ring_off(seq) + pos * h->bb;
+            } else {
+                if (!to_u && no_p) { j = first_resident; continue; }
+                rc = ensure_staging(h, stage_cap);
+                if (rc != IPKV_OK) return rc;
+                j_end = std::min<int64_t>(to_u ? nb : first_resident, j + int64_t(stage_cap / h->bb));
+                dst = h->staging;
+            }
+            const int64_t tok0 = j * bt, tok1 = std::min(r.n_tokens, j_end * bt);
+            const char* ks = static_cast<const char*>(k_dev) + (r.first_token + tok0) * k_row;
+            const char* vs = v_dev ? static_cast<const char*>(v_dev) + (r.first_token + tok0) * v_row : nullptr;
+            CU(h, launch_pack(h->geom, to_u ? 0 : 1, ks, vs, tok1 - tok0, dst, 0, s));
+            h->stats.pack_kernels += 1;
+            char* host = to_u ? h->u_ptr(layer, seq, r.first_block + j) : (no_p ? nullptr : h->p_ptr(layer, seq, r.first_block + j));
+            if (host) {
+                CU(h, cudaMemcpyAsync(host, dst, size_t((j_end - j) * h->bb), cudaMemcpyDeviceToHost, s));
+                h->stats.d2h_bytes += uint64_t((j_end - j) * h->bb);
+            }
+            j = j_end;
+        }
+    }
+    return IPKV_OK;
+}
+
+ipkv_status ipkv_flush(ipkv_t* h, int32_t layer, int32_t seq, void* stream) {
+    if (!h) return IPKV_EINVAL;
+    if (layer < -1 || layer >= h->cfg.n_layers) return fail(h, IPKV_EINVAL, "layer out of range");
+    if (seq < -1 || seq >= h->cfg.max_seqs) return fail(h, IPKV_EINVAL, "sequence id out of range");
+    CU(h, cudaSetDevice(h->cfg.device));
+    for (int l = 0; l < h->cfg.n_layers; ++l)
+        for (int s = 0; s < h->cfg.max_seqs; ++s)
+            if ((layer < 0 || l == layer) && (seq < 0 || s == seq)) {
+                ipkv_status rc = do_flush(h, l, s, static_cast<cudaStream_t>(stream));
+                if (rc != IPKV_OK) return rc;
+            }
+    return IPKV_OK;
+}
+
+ipkv_status ipkv_append(ipkv_t* h, int32_t layer, const int32_t* seq_ids, int32_t n_seq,
+                        const void* k_dev, const void* v_dev, void* stream) {
+    if (!h) return IPKV_EINVAL;
+    const ipkv_config& c = h->cfg;
+    if (layer < 0 || layer >= c.n_layers) return fail(h, IPKV_EINVAL, "layer out of range");
+    if (n_seq < 0 || (n_seq > 0 && (!seq_ids || !k_dev || (c.kind == IPKV_GQA && !v_dev)))) return fail(h, IPKV_EINVAL, "bad arguments");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    for (int i = 0; i < n_seq; ++i) {
+        if (seq_ids[i] < 0 || seq_ids[i] >= c.max_seqs) return fail(h, IPKV_EINVAL, "sequence id out of range");
+        for (int j = 0; j < i; ++j) if (seq_ids[j] == seq_ids[i]) return fail(h, IPKV_EINVAL, "duplicate sequence id");
+    }
+    CU(h, cudaSetDevice(c.device));
+    // evict full windows first, so that the newest token is always GPU-side
+    for (int i = 0; i < n_seq; ++i)
+        if (h->state(layer, seq_ids[i]).router.window_full()) {
+            ipkv_status rc = do_flush(h, layer, seq_ids[i], s);
+            if (rc != IPKV_OK) return rc;
+        }
+    const int64_t k_row = int64_t(c.n_kv_heads) * c.dim_qk * 2, v_row = int64_t(c.n_kv_heads) * c.dim_v * 2;
+    for (int base = 0; base < n_seq; base += kAppendRowsPerLaunch) {
+        const int n = std::min(kAppendRowsPerLaunch, n_seq - base);
+        AppendRows rows;
+        for (int i = 0; i < n; ++i) {
+            SeqState& st = h->state(layer, seq_ids[base + i]);
+            rows.dst_off[i] = h->w_off(seq_ids[base + i]);
+            rows.slot[i] = int32_t(st.router.stage());
+        }
+        const char* ks = static_cast<const char*>(k_dev) + base * k_row;
+        const char* vs = v_dev ? static_cast<const char*>(v_dev) + base * v_row : nullptr;
+        CU(h, launch_append(h->geom, ks, vs, c.dim_v, h->w_layer(layer), rows, n, s));
+        h->stats.append_kernels += 1;
+    }
+    return IPKV_OK;
+}
+
+ipkv_status ipkv_attend_gpu(ipkv_t* h, int32_t layer, const int32_t* seq_ids, int32_t n_seq,
+                            const void* q_dev, const ipkv_attend_opts* opts,
+                            float* o_part_dev, float* lse_part_dev, void* stream) {
+    if (!h) return IPKV_EINVAL;
+    const ipkv_config& c = h->cfg;
+    if (layer < 0 || layer >= c.n_layers) return fail(h, IPKV_EINVAL, "layer out of range");
+    if (n_seq <= 0 || !seq_ids || !q_dev || !o_part_dev || !lse_part_dev) return fail(h, IPKV_EINVAL, "bad arguments");
+    if (n_seq > c.max_seqs) return fail(h, IPKV_EINVAL, "more rows than max_seqs");
+    for (int i = 0; i < n_seq; ++i)
+        if (seq_ids[i] < 0 || seq_ids[i] >= c.max_seqs) return fail(h, IPKV_EINVAL, "sequence id out of range");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int kv_splits = opts ? opts->kv_splits : 0;
+    if (kv_splits < 0) return fail(h, IPKV_EINVAL, "kv_splits must be >= 0");
+    cudaStream_t side = (opts && opts->side_stream) ? static_cast<cudaStream_t>(opts->side_stream) : h->side;
+    CU(h, cudaSetDevice(c.device));
+    h->stats.attend_calls += 1;
+    const int64_t bt = c.block_tokens;
+
+    // group 0: everything already on the device (resident ring + D-window)
+    std::vector<std::vector<PlanSeg>> rows(n_seq);
+    int64_t max_stream_chunks = 0;
+    for (int i = 0; i < n_seq; ++i) {
+        const int seq = seq_ids[i];
+        SeqState& st = h->state(layer, seq);
+        const int64_t used = st.router.blocks_used(REGION_P);
+        const int64_t nr = std::max<int64_t>(0, used - h->ring);      // blocks [0, nr) are host-only
+        if (nr > 0 && (c.flags & IPKV_FLAG_NO_HOST_P)) return fail(h, IPKV_EINTERNAL, "host-only P blocks without a host copy");
+        max_stream_chunks = std::max(max_stream_chunks, (nr + h->chunk_blocks - 1) / h->chunk_blocks);
+        for (const PRun& r : st.p_runs) {
+            const int64_t nb = (r.n_tokens + bt - 1) / bt;
+            int64_t j = std::max(r.first_block, nr);
+            const int64_t end = r.first_block + nb;
+            while (j < end) {
+                const int64_t pos = j % h->ring;
+                const int64_t n = std::min(end - j, h->ring - pos);
+                const int64_t tok = std::min(r.n_tokens - (j - r.first_block) * bt, n * bt);
+                rows[i].push_back(PlanSeg{0, h->ring_off(seq) + pos * h->bb, tok});
+                j += n;
+            }
+        }
+        if (st.router.window_fill() > 0) rows[i].push_back(PlanSeg{1, h->w_off(seq), st.router.window_fill()});
+    }
+    const char* bases[kMaxBases] = {h->ring ? h->ring_layer(layer) : nullptr, h->w_layer(layer), h->pp_dev, nullptr};
+    ipkv_status rc = run_group(h, rows, bases, q_dev, kv_splits, false, o_part_dev, lse_part_dev, s);
+    if (rc != IPKV_OK) return rc;
+    if (max_stream_chunks == 0) return IPKV_OK;
+
+    // groups 1..: host-only P chunks, streamed through the PP slots in overwrite-reuse order (Sec. 4.2)
+    CU(h, cudaEventRecord(h->ev_main, s));                 // P's host bytes were written by work on `s`
+    CU(h, cudaStreamWaitEvent(side, h->ev_main, 0));
+    const int64_t chunk_bytes = h->chunk_blocks * h->bb;
+    for (int64_t ch = 0; ch < max_stream_chunks; ++ch) {
+        const int slot = int(ch % c.n_slots);
+        if (h->slot_free_set[slot]) CU(h, cudaStreamWaitEvent(side, h->slot_free[slot], 0));
+        for (int i = 0; i < n_seq; ++i) {
+            rows[i].clear();
+            const int seq = seq_ids[i];
+            SeqState& st = h->state(layer, seq);
+            const int64_t nr = std::max<int64_t>(0, st.router.blocks_used(REGION_P) - h->ring);
+            const int64_t lo = ch * h->chunk_blocks, hi = std::min(nr, lo + h->chunk_blocks);
+            if (lo >= hi) continue;
+            char* dst = h->pp_dev + slot * h->slot_bytes() + int64_t(i) * chunk_bytes;
+            CU(h, cudaMemcpyAsync(dst, h->p_ptr(layer, seq, lo), size_t((hi - lo) * h->bb), cudaMemcpyHostToDevice, side));
+            h->stats.h2d_bytes += uint64_t((hi - lo) * h->bb);
+            for (const PRun& r : st.p_runs) {
+                const int64_t nb = (r.n_tokens + bt - 1) / bt;
+                const int64_t a = std::max(lo, r.first_block), b = std::min(hi, r.first_block + nb);
+                if (a >= b) continue;
+                const int64_t tok = std::min(r.n_tokens - (a - r.first_block) * bt, (b - a) * bt);
+                rows[i].push_back(PlanSeg{2, slot * h->slot_bytes() + int64_t(i) * chunk_bytes + (a - lo) * h->bb, tok});
+            }
+        }
+        CU(h, cudaEventRecord(h->slot_ready[slot], side));
+        CU(h, cudaStreamWaitEvent(s, h->slot_ready[slot], 0));
+        rc = run_group(h, rows, bases, q_dev, kv_splits, true, o_part_dev, lse_part_dev, s);
+        if (rc != IPKV_OK) return rc;
+        CU(h, cudaEventRecord(h->slot_free[slot], s));
+        h->slot_free_set[slot] = 1;
+    }
+    return IPKV_OK;
+}
+
+ipkv_status ipkv_merge(ipkv_t* h, int32_t n_rows, int32_t dim_v, int32_t n_parts,
+                       const float* const* o_parts, const float* const* lse_parts,
+                       void* o_out_dev, int32_t o_out_is_bf16, float* lse_out_dev, void* stream) {
+    if (n_rows < 0 || dim_v <= 0 || dim_v % 4 != 0 || n_parts < 1 || n_parts > kMaxMergeParts || !o_parts || !lse_parts || !o_out_dev)
+        return fail(h, IPKV_EINVAL, "bad merge arguments");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (h) CU(h, cudaSetDevice(h->cfg.device));
+    MergeLaunch m{};
+    m.n_parts = n_parts; m.n_rows = n_rows; m.dim_v = dim_v;
+    m.out_o = o_out_dev; m.out_is_bf16 = o_out_is_bf16; m.out_lse = lse_out_dev;
+    const size_t o_bytes = size_t(n_rows) * dim_v * sizeof(float), l_bytes = size_t(n_rows) * sizeof(float);
+    const size_t per_part = align_up(o_bytes, 256) + align_up(l_bytes, 256);
+    int n_host = 0;
+    for (int i = 0; i < n_parts; ++i) {
+        if (!o_parts[i] || !lse_parts[i]) return fail(h, IPKV_EINVAL, "NULL partial");
+        cudaPointerAttributes at{};
+        const cudaError_t e = cudaPointerGetAttributes(&at, o_parts[i]);
+        const bool on_dev = (e == cudaSuccess) && (at.type == cudaMemoryTypeDevice || at.type == cudaMemoryTypeManaged);
+        if (e != cudaSuccess) cudaGetLastError();
+        if (on_dev) { m.o[i] = o_parts[i]; m.lse[i] = lse_parts[i]; continue; }
+        if (!h) return fail(h, IPKV_EINVAL, "host partials need a handle for staging");
+        const size_t need = per_part * kMaxMergeParts;
+        if (h->merge_stage_bytes < need) {
+            CU(h, cudaDeviceSynchronize());
+            if (h->merge_stage) cudaFree(h->merge_stage);
+            h->merge_stage = nullptr; h->merge_stage_bytes = 0;
+            CU(h, cudaMalloc(&h->merge_stage, need));
+            h->merge_stage_bytes = need;
+        }
+        char* dst = h->merge_stage + size_t(n_host) * per_part;
+        CU(h, cudaMemcpyAsync(dst, o_parts[i], o_bytes, cudaMemcpyHostToDevice, s));
+        CU(h, cudaMemcpyAsync(dst + align_up(o_bytes, 256), lse_parts[i], l_bytes, cudaMemcpyHostToDevice, s));
+        h->stats.h2d_bytes += o_bytes + l_bytes;
+        m.o[i] = reinterpret_cast<const float*>(dst);
+        m.lse[i] = reinterpret_cast<const float*>(dst + align_up(o_bytes, 256));
+        ++n_host;
+    }
+    CU(h, launch_merge(m, s));
+    if (h) h->stats.merge_kernels += 1;
+    return IPKV_OK;
+}
+
+ipkv_status ipkv_views(ipkv_t* h, int32_t layer, int32_t seq, ipkv_extent* out, int32_t cap, int32_t* n_out) {
+    ipkv_status rc = check_ls(h, layer, seq);
+    if (rc != IPKV_OK) return rc;
+    if (!n_out || (cap > 0 && !out)) return fail(h, IPKV_EINVAL, "bad arguments");
+    SeqState& st = h->state(layer, seq);
+    const auto& runs = st.router.runs();
+    const int total = int(runs.size()) + (st.router.window_fill() > 0 ? 1 : 0);
+    *n_out = total;
+    if (cap < total) return cap == 0 ? IPKV_OK : fail(h, IPKV_ERANGE, "extent array too small");
+    const int64_t bt = h->cfg.block_tokens;
+    const int64_t used_p = st.router.blocks_used(REGION_P);
+    const int64_t nr = std::max<int64_t>(0, used_p - h->ring);
+    int k = 0;
+    for (const Run& r : runs) {
+        ipkv_extent& e = out[k++];
+        e.region = r.region; e.first_token = r.first_token; e.n_tokens = r.n_tokens; e.region_block = r.first_block;
+        e.block_bytes = h->bb; e.host_ptr = nullptr; e.dev_ptr = nullptr;
+        const int64_t nb = (r.n_tokens + bt - 1) / bt;
+        if (r.region == REGION_U) {
+            e.layout = IPKV_LAYOUT_PLAIN;
+            if (h->u_host) e.host_ptr = h->u_ptr(layer, seq, r.first_block);
+        } else {
+            e.layout = IPKV_LAYOUT_TILE;
+            if (h->p_host) e.host_ptr = h->p_ptr(layer, seq, r.first_block);
+            if (h->ring > 0 && r.first_block >= nr && (r.first_block % h->ring) + nb <= h->ring)
+                e.dev_ptr = h->ring_layer(layer) + h->ring_off(seq) + (r.first_block % h->ring) * h->bb;
+        }
+    }
+    if (st.router.window_fill() > 0) {
+        ipkv_extent& e = out[k++];
+        e.region = IPKV_REGION_W; e.layout = IPKV_LAYOUT_TILE; e.first_token = st.router.window_first();
+        e.n_tokens = st.router.window_fill(); e.region_block = 0; e.block_bytes = h->bb;
+        e.host_ptr = nullptr; e.dev_ptr = h->w_layer(layer) + h->w_off(seq);
+    }
+    return IPKV_OK;
+}
+
+ipkv_status ipkv_locate(ipkv_t* h, int32_t layer, int32_t seq, int64_t token,
+                        int32_t* region, int64_t* region_block, int32_t* offset_in_block) {
+    ipkv_status rc = check_ls(h, layer, seq);
+    if (rc != IPKV_OK) return rc;
+    if (!region || !region_block || !offset_in_block) return fail(h, IPKV_EINVAL, "NULL output");
+    if (!h->state(layer, seq).router.locate(token, region, region_block, offset_in_block))
+        return fail(h, IPKV_ERANGE, "token index out of range");
+    return IPKV_OK;
+}
+
+ipkv_status ipkv_counts(ipkv_t* h, int32_t layer, int32_t seq, int64_t counts[6]) {
+    ipkv_status rc = check_ls(h, layer, seq);
+    if (rc != IPKV_OK) return rc;
+    if (!counts) return fail(h, IPKV_EINVAL, "NULL output");
+    SeqState& st = h->state(layer, seq);
+    counts[0] = st.router.tokens_in(REGION_U);
+    counts[1] = st.router.tokens_in(REGION_P);
+    counts[2] = st.router.tokens_in(REGION_W);
+    const int64_t nr = std::max<int64_t>(0, st.router.blocks_used(REGION_P) - h->ring);
+    int64_t res = 0;
+    const int64_t bt = h->cfg.block_tokens;
+    for (const PRun& r : st.p_runs) {
+        const int64_t nb = (r.n_tokens + bt - 1) / bt;
+        const int64_t j = std::max(r.first_block, nr);
+        if (j < r.first_block + nb) res += r.n_tokens - (j - r.first_block) * bt;
+    }
+    counts[3] = res;
+    counts[4] = st.router.evictions();
+    counts[5] = st.router.evictions_cpu();
+    return IPKV_OK;
+}
+
+ipkv_status ipkv_read_token(ipkv_t* h, int32_t layer, int32_t seq, int64_t token, void* k_out, void* v_out) {
+    ipkv_status rc = check_ls(h, layer, seq);
+    if (rc != IPKV_OK) return rc;
+    if (!k_out) return fail(h, IPKV_EINVAL, "NULL output");
+    int32_t region, off;
+    int64_t blk;
+    SeqState& st = h->state(layer, seq);
+    if (!st.router.locate(token, &region, &blk, &off)) return fail(h, IPKV_ERANGE, "token index out of range");
+    CU(h, cudaSetDevice(h->cfg.device));
+    CU(h, cudaDeviceSynchronize());
+    std::vector<char> buf(size_t(h->bb));
+    bool tile = true;
+    const int64_t bt = h->cfg.block_tokens;
+    if (region == REGION_U) {
+        if (!h->u_host) return fail(h, IPKV_ESTATE, "U contents are not kept (IPKV_FLAG_NO_HOST_U)");
+        std::memcpy(buf.data(), h->u_ptr(layer, seq, blk), size_t(h->bb));
+        tile = false;
+    } else if (region == REGION_P) {
+        if (h->p_host) {
+            std::memcpy(buf.data(), h->p_ptr(layer, seq, blk), size_t(h->bb));
+        } else {
+            CU(h, cudaMemcpy(buf.data(), h->ring_layer(layer) + h->ring_off(seq) + (blk % h->ring) * h->bb, size_t(h->bb), cudaMemcpyDeviceToHost));
+        }
+    } else {
+        const int64_t wb = off / bt;
+        off = int32_t(off - wb * bt);
+        CU(h, cudaMemcpy(buf.data(), h->w_layer(layer) + h->w_off(seq) + wb * h->bb, size_t(h->bb), cudaMemcpyDeviceToHost));
+    }
+    const BlockGeom& g = h->geom;
+    for (int head = 0; head < g.n_kv_heads; ++head) {
+        const char* hp = buf.data() + int64_t(head) * g.head_bytes();
+        for (int ch = 0; ch < g.dim_qk / 8; ++ch) {
+            const int64_t o = tile ? tile_chunk_offset(g.bt, off, ch) : plain_chunk_offset(g.dim_qk, off, ch);
+            std::memcpy(static_cast<char*>(k_out) + (int64_t(head) * g.dim_qk + ch * 8) * 2, hp + o, 16);
+        }
+        if (v_out && g.dim_v_stored > 0)
+            for (int ch = 0; ch < g.dim_v_stored / 8; ++ch) {
+                const int64_t o = g.k_plane_bytes() + (tile ? tile_chunk_offset(g.bt, off, ch) : plain_chunk_offset(g.dim_v_stored, off, ch));
+                std::memcpy(static_cast<char*>(v_out) + (int64_t(head) * g.dim_v_stored + ch * 8) * 2, hp + o, 16);
+            }
+    }
+    return IPKV_OK;
+}
+
+ipkv_status ipkv_get_stats(ipkv_t* h, ipkv_stats* out) {
+    if (!h || !out) return IPKV_EINVAL;
+    CU(h, cudaSetDevice(h->cfg.device));
+    CU(h, cudaDeviceSynchronize());
+    CU(h, cudaMemcpy(&h->stats.device_status, h->status_dev, sizeof(uint32_t), cudaMemcpyDeviceToHost));
+    *out = h->stats;
+    return h->stats.device_status ? fail(h, IPKV_ETIMEOUT, "a kernel's bounded wait gave up; results of that call are invalid") : IPKV_OK;
+}
+
+// ---- stateless entry points ---------------------------------------------------------------------
+
+int64_t ipkv_block_bytes(const ipkv_attn_shape* sh) {
+    if (!sh || !shape_ok(sh->kind, sh->n_q_heads, sh->n_kv_heads, sh->dim_qk, sh->dim_v, sh->block_tokens, nullptr)) return -1;
+    return make_geom(sh->kind, sh->n_kv_heads, sh->dim_qk, sh->dim_v, sh->block_tokens).block_bytes();
+}
+
+ipkv_status ipkv_attend_scratch_bytes(const ipkv_attn_shape* sh, int32_t n_rows, int32_t n_runs,
+                                      int64_t total_tokens, int32_t kv_splits, size_t* out_bytes) {
+    if (!sh || !out_bytes || n_rows < 0 || n_runs < 0 || total_tokens < 0 || kv_splits < 0) return IPKV_EINVAL;
+    if (!shape_ok(sh->kind, sh->n_q_heads, sh->n_kv_heads, sh->dim_qk, sh->dim_v, sh->block_tokens, nullptr)) return IPKV_EINVAL;
+    const int64_t items = max_items_bound(n_rows, n_runs, total_tokens, kv_splits);
+    const size_t table = align_up(size_t(n_runs) * sizeof(Seg), 16) + align_up(size_t(items) * sizeof(Item), 16) +
+                         align_up(size_t(n_rows + 1) * sizeof(int32_t), 16);
+    *out_bytes = align_up(table, 256) + 256 + partial_bytes(size_t(items), sh->n_q_heads, sh->dim_v);
+    return IPKV_OK;
+}
+
+ipkv_status ipkv_attend_runs(const ipkv_attn_shape* sh, int32_t n_rows,
+                             const ipkv_run* runs, const int32_t* row_run_start,
+                             const void* q_dev, int32_t kv_splits,
+                             void* scratch_dev, size_t scratch_bytes,
+                             float* o_part_dev, float* lse_part_dev, uint32_t* status_dev, void* stream) {
+    if (!sh || n_rows <= 0 || !row_run_start || !q_dev || !scratch_dev || !o_part_dev || !lse_part_dev || kv_splits < 0) return IPKV_EINVAL;
+    if (!shape_ok(sh->kind, sh->n_q_heads, sh->n_kv_heads, sh->dim_qk, sh->dim_v, sh->block_tokens, nullptr)) return IPKV_EINVAL;
+    if ((reinterpret_cast<uintptr_t>(scratch_dev) & 255u) != 0) return IPKV_EINVAL;
+    const int n_runs = row_run_start[n_rows];
+    if (n_runs < 0 || (n_runs > 0 && !runs)) return IPKV_EINVAL;
+    std::vector<std::vector<PlanSeg>> rows(n_rows);
+    for (int r = 0; r < n_rows; ++r) {
+        if (row_run_start[r] > row_run_start[r + 1] || row_run_start[r] < 0) return IPKV_EINVAL;
+        for (int k = row_run_start[r]; k < row_run_start[r + 1]; ++k) {
+            if (runs[k].n_tokens < 0 || (runs[k].n_tokens > 0 && !runs[k].blocks_dev)) return IPKV_EINVAL;
+            if (reinterpret_cast<uintptr_t>(runs[k].blocks_dev) & 15u) return IPKV_EINVAL;
+            rows[r].push_back(PlanSeg{0, int64_t(reinterpret_cast<intptr_t>(runs[k].blocks_dev)), runs[k].n_tokens});
+        }
+    }
+    Plan plan;
+    build_plan(rows, heads_per_tile(sh->kind, sh->n_q_heads, sh->n_kv_heads), kv_splits, &plan);
+    const size_t table = align_up(plan.table_bytes(), 256);
+    if (table + 256 + partial_bytes(plan.items.size(), sh->n_q_heads, sh->dim_v) > scratch_bytes) return IPKV_ENOMEM;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    std::vector<char> img(table, 0);
+    plan.serialize(img.data());
+    // pageable source: the runtime stages it before returning, so `img` may go out of scope
+    if (cudaMemcpyAsync(scratch_dev, img.data(), table, cudaMemcpyHostToDevice, s) != cudaSuccess) return IPKV_ECUDA;
+    AttnLaunch a{};
+    const float scale = sh->softmax_scale > 0.f ? sh->softmax_scale : 1.0f / std::sqrt(float(sh->dim_qk));
+    fill_launch(&a, sh->kind, sh->n_q_heads, sh->n_kv_heads, sh->dim_qk, sh->dim_v, sh->block_tokens, scale, plan,
+                static_cast<const char*>(scratch_dev), static_cast<char*>(scratch_dev) + table + 256, q_dev, n_rows);
+    a.bases[0] = nullptr;
+    a.out_o = o_part_dev; a.out_lse = lse_part_dev;
+    a.status = status_dev ? status_dev : reinterpret_cast<uint32_t*>(static_cast<char*>(scratch_dev) + table);
+    if (a.n_items > 0 && launch_attend(a, s) != cudaSuccess) return IPKV_ECUDA;
+    if (launch_split_reduce(a, s) != cudaSuccess) return IPKV_ECUDA;
+    return IPKV_OK;
+}
+
+ipkv_status ipkv_pack_blocks(const ipkv_attn_shape* sh, int32_t layout, const void* k_dev, const void* v_dev,
+                             int64_t n_tokens, void* dst_dev, void* stream) {
+    if (!sh || n_tokens < 0 || (n_tokens > 0 && (!k_dev || !dst_dev))) return IPKV_EINVAL;
+    if (!shape_ok(sh->kind, sh->n_q_heads, sh->n_kv_heads, sh->dim_qk, sh->dim_v, sh->block_tokens, nullptr)) return IPKV_EINVAL;
+    if (sh->kind == IPKV_GQA && n_tokens > 0 && !v_dev) return IPKV_EINVAL;
+    if (layout != IPKV_LAYOUT_PLAIN && layout != IPKV_LAYOUT_TILE) return IPKV_EINVAL;
+    const BlockGeom g = make_geom(sh->kind, sh->n_kv_heads, sh->dim_qk, sh->dim_v, sh->block_tokens);
+    if (launch_pack(g, layout == IPKV_LAYOUT_TILE, k_dev, v_dev, n_tokens, dst_dev, 0, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return IPKV_ECUDA;
+    return IPKV_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,74 @@
+// Internal launch interface between the host scheduler (api.cu) and the CUDA kernels.
+#pragma once
+#include <cuda_runtime.h>
+#include <cstdint>
+
+#include "layout.cuh"
+
+namespace ipkvi {
+
+// One run of contiguous TILE-layout blocks that a row attends to; address = bases[base_id] + off.
+struct Seg {
+    int64_t off;
+    int32_t n_tokens;
+    int32_t base_id;
+};
+// One unit of split-K work: tiles [tile0, tile0 + ntiles) of segment `seg` for query row `row`.
+// The partial it produces has the item's own index.
+struct Item {
+    int32_t row, seg, tile0, ntiles;
+};
+
+constexpr int kMaxBases = 4;
+
+struct AttnLaunch {
+    int kind;                       // 0 = GQA, 1 = compressed latent (MLA)
+    int n_q_heads, n_kv_heads, dim_qk, dim_v, bt;
+    float scale;                    // softmax scale applied to fp32 scores
+    const void* q;                  // [n_rows][Hq][dqk] bf16
+    const char* bases[kMaxBases];
+    const Seg* segs;                // device
+    const Item* items;              // device
+    const int32_t* row_item_start;  // device, [n_rows + 1]
+    int n_items, n_rows;
+    float* part_o;                  // [n_items][Hq][dv]
+    float* part_lse;                // [n_items][Hq]
+    const float* acc_o;             // optional earlier partial to fold in, [n_rows][Hq][dv]
+    const float* acc_lse;
+    float* out_o;                   // [n_rows][Hq][dv]
+    float* out_lse;                 // [n_rows][Hq]
+    uint32_t* status;               // device word, OR-ed with an error bit if a bounded wait gives up
+};
+
+// Split-K attention: one partial (O, LSE) per (item, query head).
+cudaError_t launch_attend(const AttnLaunch& a, cudaStream_t s);
+// Second pass: per (row, head) LSE-reduce the row's item partials (and acc_*, if given) into out_*.
+cudaError_t launch_split_reduce(const AttnLaunch& a, cudaStream_t s);
+
+constexpr int kMaxMergeParts = 8;
+struct MergeLaunch {
+    const float* o[kMaxMergeParts];
+    const float* lse[kMaxMergeParts];
+    int n_parts, n_rows, dim_v;
+    void* out_o;
+    int out_is_bf16;
+    float* out_lse;                 // may be null
+};
+cudaError_t launch_merge(const MergeLaunch& m, cudaStream_t s);
+
+// Token-major K/V -> blocks. dst_token0 = token offset (in the destination's block space) of src token 0.
+cudaError_t launch_pack(const BlockGeom& g, int layout_tile, const void* k, const void* v, int64_t n_tokens,
+                        void* dst, int64_t dst_token0, cudaStream_t s);
+// TILE-layout blocks -> PLAIN-layout blocks (eviction of a window batch to the CPU-compute region).
+cudaError_t launch_tile_to_plain(const BlockGeom& g, const void* src, void* dst, int64_t n_blocks, cudaStream_t s);
+
+constexpr int kAppendRowsPerLaunch = 64;
+struct AppendRows {
+    int64_t dst_off[kAppendRowsPerLaunch];   // byte offset of the row's window (first block) from w_base
+    int32_t slot[kAppendRowsPerLaunch];      // token slot inside the window
+};
+// One new token per row into its D-window (TILE layout). k/v point at the first row of this launch.
+cudaError_t launch_append(const BlockGeom& g, const void* k, const void* v, int dim_v_src, char* w_base,
+                          const AppendRows& rows, int n_rows, cudaStream_t s);
+
+}  // namespace ipkvi

@@ -1,0 +1,74 @@
+// Test-only C shim over the product's host-side headers (router.hpp, plan.hpp, layout.cuh) so that
+// the routing state machine, the split-K planner and the block-layout arithmetic can be exercised on
+// a machine without a GPU.  Compiled by tests/host_shim.py with g++; not part of the library.
+#include <cstdint>
+#include <cstring>
+#include <vector>
+
+#include "../paper_2609_14507_b200/csrc/plan.hpp"
+#include "../paper_2609_14507_b200/csrc/router.hpp"
+
+using namespace ipkvi;
+
+extern "C" {
+
+void* shim_router_new(int64_t block, int64_t window, int64_t num, int64_t den) { return new SeqRouter(block, window, num, den); }
+void shim_router_free(void* r) { delete static_cast<SeqRouter*>(r); }
+void shim_router_set_share(void* r, int64_t num) { static_cast<SeqRouter*>(r)->set_share(num); }
+void shim_router_bulk(void* r, int64_t n, int64_t num0, int64_t den0) {
+    Run out[2];
+    static_cast<SeqRouter*>(r)->bulk(n, num0, den0, out);
+}
+void shim_router_flush(void* r) { static_cast<SeqRouter*>(r)->evict(); }
+// the library's append: evict a full window first, then stage
+void shim_router_append(void* r) {
+    SeqRouter* s = static_cast<SeqRouter*>(r);
+    if (s->window_full()) s->evict();
+    s->stage();
+}
+int64_t shim_router_len(void* r) { return static_cast<SeqRouter*>(r)->length(); }
+void shim_router_counts(void* r, int64_t* c) {
+    SeqRouter* s = static_cast<SeqRouter*>(r);
+    c[0] = s->tokens_in(REGION_U); c[1] = s->tokens_in(REGION_P); c[2] = s->tokens_in(REGION_W);
+    c[3] = s->blocks_used(REGION_U); c[4] = s->blocks_used(REGION_P);
+    c[5] = s->evictions(); c[6] = s->evictions_cpu();
+}
+void shim_router_dump(void* r, int8_t* region, int64_t* blk, int32_t* off) {
+    SeqRouter* s = static_cast<SeqRouter*>(r);
+    for (int64_t t = 0; t < s->length(); ++t) {
+        int32_t g, o;
+        int64_t b;
+        s->locate(t, &g, &b, &o);
+        region[t] = int8_t(g); blk[t] = b; off[t] = o;
+    }
+}
+
+// plan: rows given as flat (row_start[n_rows+1], n_tokens[n_segs]); returns counts, fills arrays up to cap
+int shim_plan(int n_rows, const int32_t* row_start, const int64_t* seg_tokens, int heads_per_tile, int kv_splits,
+              int cap_items, int32_t* item_row, int32_t* item_seg, int32_t* item_tile0, int32_t* item_ntiles,
+              int32_t* row_item_start, int32_t* seg_tokens_out, int* n_segs_out) {
+    std::vector<std::vector<PlanSeg>> rows(n_rows);
+    for (int r = 0; r < n_rows; ++r)
+        for (int k = row_start[r]; k < row_start[r + 1]; ++k) rows[r].push_back(PlanSeg{0, int64_t(k) * 4096, seg_tokens[k]});
+    Plan plan;
+    build_plan(rows, heads_per_tile, kv_splits, &plan);
+    const int n = int(plan.items.size());
+    if (n > cap_items) return -n;
+    for (int i = 0; i < n; ++i) {
+        item_row[i] = plan.items[i].row; item_seg[i] = plan.items[i].seg;
+        item_tile0[i] = plan.items[i].tile0; item_ntiles[i] = plan.items[i].ntiles;
+    }
+    for (int r = 0; r <= n_rows; ++r) row_item_start[r] = plan.row_item_start[r];
+    *n_segs_out = int(plan.segs.size());
+    for (size_t k = 0; k < plan.segs.size(); ++k) seg_tokens_out[k] = plan.segs[k].n_tokens;
+    return n;
+}
+
+int64_t shim_tile_chunk_offset(int32_t bt, int32_t t, int32_t chunk) { return tile_chunk_offset(bt, t, chunk); }
+int64_t shim_plain_chunk_offset(int32_t d, int32_t t, int32_t chunk) { return plain_chunk_offset(d, t, chunk); }
+int64_t shim_block_bytes(int32_t hkv, int32_t dqk, int32_t dv_stored, int32_t bt) {
+    BlockGeom g{hkv, dqk, dv_stored, bt};
+    return g.block_bytes();
+}
+
+}  // extern "C"

@@ -1,0 +1,242 @@
+"""GPU parity of the handle-based path (create / append / flush / attend_gpu / merge / views) against the
+oracle: routing indices and region contents bit-exact, partial and merged outputs within tolerance."""
+import ctypes as C
+
+import numpy as np
+import pytest
+
+from oracle import c_oracle
+from paper_2609_14507_b200 import binding, synth
+from tests import layouts
+from tests.gpu_util import check_partial
+
+pytestmark = pytest.mark.gpu
+torch = pytest.importorskip("torch")
+DEV = "cuda:0"
+
+
+class RefSeq:
+    """Everything appended to one (layer, sequence) plus the oracle's routing of it."""
+
+    def __init__(self, shape, block, D, num, den):
+        self.shape, self.route = shape, c_oracle.Route(block, D, num, den)
+        self.k = np.zeros((0, shape.n_kv_heads, shape.dim_qk), np.uint16)
+        self.v = None if shape.kind == "mla" else np.zeros((0, shape.n_kv_heads, shape.dim_v), np.uint16)
+
+    def bulk(self, k, v, num0, den0):
+        self.route.bulk(k.shape[0], num0, den0)
+        self._push(k, v)
+
+    def append(self, k, v):
+        self.route.append()
+        self._push(k, v)
+
+    def _push(self, k, v):
+        self.k = np.concatenate([self.k, k])
+        if self.v is not None:
+            self.v = np.concatenate([self.v, v])
+
+    def attend(self, q, which, scale):
+        region, _, _ = self.route.dump()
+        idx = np.nonzero(region == 0)[0] if which == "cpu" else (np.nonzero(region != 0)[0] if which == "gpu" else np.arange(len(region)))
+        v = self.shape.dim_v if self.v is None else self.v
+        return c_oracle.attend(q, self.k, v, idx, scale)
+
+
+def make_cache(shape, n_layers, max_seqs, **kw):
+    kind = binding.MLA if shape.kind == "mla" else binding.GQA
+    cfg = binding.make_config(kind, n_layers, max_seqs, shape.n_q_heads, shape.n_kv_heads, shape.dim_qk, shape.dim_v,
+                              softmax_scale=shape.scale, **kw)
+    return binding.Cache(cfg)
+
+
+def check_routing(cache, layer, seq, ref, sample=None):
+    region, blk, off = ref.route.dump()
+    n = len(region)
+    c = cache.counts(layer, seq)
+    rc = ref.route.counts()
+    assert (c["n_u"], c["n_p"], c["n_w"], c["n_flush"], c["n_flush_cpu"]) == (rc["n_u"], rc["n_p"], rc["n_w"], rc["n_flush"], rc["n_flush_cpu"])
+    tokens = range(n) if sample is None else sample
+    for t in tokens:
+        assert cache.locate(layer, seq, t) == (int(region[t]), int(blk[t]), int(off[t])), t
+
+
+def check_contents(cache, layer, seq, ref, tokens):
+    for t in tokens:
+        k, v = cache.read_token(layer, seq, int(t))
+        np.testing.assert_array_equal(k, ref.k[t])
+        if ref.v is not None:
+            np.testing.assert_array_equal(v, ref.v[t])
+
+
+def host_bytes(ptr, n):
+    return np.ctypeslib.as_array(C.cast(ptr, C.POINTER(C.c_uint16)), shape=(n // 2,)).copy()
+
+
+def test_config1_append_attend_merge():
+    """Single layer, batch 1, GQA 32/4, head_dim 128, 4096 tokens, CPU share = first half; append one token,
+    attend the GPU share, merge with the CPU partial: equals unsplit attention over all 4097 tokens."""
+    sh = synth.SMALL_GQA
+    L = 4096
+    k, v = synth.host_kv(sh, L + 1, seed=1000)
+    q = synth.host_q(sh, 1, seed=1001)
+    with make_cache(sh, 1, 1, block_tokens=64, window_tokens=256, chunk_tokens=512, max_u_tokens_per_seq=L,
+                    max_p_tokens_per_seq=L, resident_tokens_per_seq=L) as cache:
+        ref = RefSeq(sh, 64, 256, 0, 1)
+        cache.append_bulk(0, 0, synth.bits_to_torch(k[:L], DEV), synth.bits_to_torch(v[:L], DEV), L, 1, 2)
+        ref.bulk(k[:L], v[:L], 1, 2)
+        cache.append(0, [0], synth.bits_to_torch(k[L:], DEV), synth.bits_to_torch(v[L:], DEV))
+        ref.append(k[L:], v[L:])
+        torch.cuda.synchronize()
+        check_routing(cache, 0, 0, ref)
+        assert cache.counts(0, 0)["n_u"] == 2048 and cache.counts(0, 0)["n_p"] == 2048 and cache.counts(0, 0)["n_w"] == 1
+        check_contents(cache, 0, 0, ref, [0, 1, 63, 64, 2047, 2048, 2049, 3000, 4095, 4096])
+        # whole regions, byte for byte: U is PLAIN, P is TILE
+        ext = cache.views(0, 0)
+        assert [(e.region, e.first_token, e.n_tokens) for e in ext] == [(0, 0, 2048), (1, 2048, 2048), (2, 4096, 1)]
+        bb = ext[0].block_bytes
+        np.testing.assert_array_equal(host_bytes(ext[0].host_ptr, 32 * bb), layouts.blocks_image(k[:2048], v[:2048], 64, False))
+        np.testing.assert_array_equal(host_bytes(ext[1].host_ptr, 32 * bb), layouts.blocks_image(k[2048:4096], v[2048:4096], 64, True))
+        qd = synth.bits_to_torch(q, DEV)
+        o = torch.zeros((1, 32, 128), device=DEV); lse = torch.zeros((1, 32), device=DEV)
+        cache.attend_gpu(0, [0], qd, o, lse)
+        torch.cuda.synchronize()
+        scale = float(np.float32(sh.scale))
+        o_gpu, l_gpu = ref.attend(q[0], "gpu", scale)
+        check_partial(o.cpu().numpy()[0], lse.cpu().numpy()[0], o_gpu, l_gpu, "gpu share")
+        # CPU partial from the oracle (float32, pinned host memory), merged on the GPU
+        o_cpu, l_cpu = ref.attend(q[0], "cpu", scale)
+        o_cpu_t = torch.from_numpy(o_cpu.astype(np.float32)).pin_memory()
+        l_cpu_t = torch.from_numpy(l_cpu.astype(np.float32)).pin_memory()
+        out = torch.zeros((32, 128), device=DEV); out_lse = torch.zeros(32, device=DEV)
+        cache.merge(32, 128, [o.view(32, 128), o_cpu_t], [lse.view(32), l_cpu_t], out, out_lse)
+        torch.cuda.synchronize()
+        o_all, l_all = ref.attend(q[0], "all", scale)
+        check_partial(out.cpu().numpy(), out_lse.cpu().numpy(), o_all, l_all, "merged")
+        st = cache.get_stats()
+        assert st["device_status"] == 0 and st["attend_kernels"] == 1 and st["merge_kernels"] == 1
+
+
+def test_merge_at_many_split_points_equals_unsplit():
+    sh = synth.SMALL_GQA
+    L = 1024
+    k, v = synth.host_kv(sh, L + 1, seed=1100)
+    q = synth.host_q(sh, 1, seed=1101)
+    scale = float(np.float32(sh.scale))
+    kd, vd, qd = synth.bits_to_torch(k, DEV), synth.bits_to_torch(v, DEV), synth.bits_to_torch(q, DEV)
+    o_all, l_all = c_oracle.attend(q[0], k, v, np.arange(L + 1), scale)
+    with make_cache(sh, 1, 1, block_tokens=64, window_tokens=256, max_u_tokens_per_seq=L, max_p_tokens_per_seq=L,
+                    resident_tokens_per_seq=L) as cache:
+        for num in range(0, 17):                      # CPU share num/16 of 16 blocks: every block boundary
+            cache.reset()
+            cache.append_bulk(0, 0, kd, vd, L, num, 16)
+            cache.append(0, [0], kd[L:], vd[L:])
+            assert cache.counts(0, 0)["n_u"] == num * 64
+            o = torch.zeros((1, 32, 128), device=DEV); lse = torch.zeros((1, 32), device=DEV)
+            cache.attend_gpu(0, [0], qd, o, lse)
+            o_cpu, l_cpu = c_oracle.attend(q[0], k, v, np.arange(num * 64), scale)
+            o_cpu_t = torch.from_numpy(o_cpu.astype(np.float32)).to(DEV)
+            l_cpu_t = torch.from_numpy(l_cpu.astype(np.float32)).to(DEV)
+            out = torch.zeros((32, 128), device=DEV); out_lse = torch.zeros(32, device=DEV)
+            cache.merge(32, 128, [o_cpu_t, o.view(32, 128)], [l_cpu_t, lse.view(32)], out, out_lse)
+            torch.cuda.synchronize()
+            check_partial(out.cpu().numpy(), out_lse.cpu().numpy(), o_all, l_all, f"split {num}/16")
+
+
+@pytest.mark.parametrize("resident,chunk,bt,D", [(4096, 128, 16, 64), (0, 64, 16, 32), (96, 32, 16, 32), (128, 64, 64, 64)])
+def test_decode_steps_with_evictions(resident, chunk, bt, D):
+    """Several layers and ragged sequences through prefill and many decode steps; every few steps the GPU
+    partial and the merged output are checked, at the end all routing indices and contents.
+    resident = 0 is the paper's exact layout (W + PP only: every P chunk is streamed each step);
+    a small resident ring wraps and pushes old blocks out to the streamed path."""
+    sh = synth.Shape("tiny", "gqa", 2, 8, 2, 128, 128, 128 ** -0.5)
+    n_layers, seqs, steps = 2, [0, 2, 3], 150
+    lens = {0: 100, 2: 0, 3: 257}
+    rng = np.random.default_rng(50)
+    scale = float(np.float32(sh.scale))
+    with make_cache(sh, n_layers, 4, block_tokens=bt, window_tokens=D, chunk_tokens=chunk, n_slots=2, max_u_tokens_per_seq=600,
+                    max_p_tokens_per_seq=600, resident_tokens_per_seq=resident, share_num=1, share_den=3) as cache:
+        refs = {}
+        for layer in range(n_layers):
+            for s in seqs:
+                r = RefSeq(sh, bt, D, 1, 3)
+                k, v = synth.host_kv(sh, lens[s], seed=5000 + 10 * layer + s)
+                cache.append_bulk(layer, s, synth.bits_to_torch(k, DEV) if lens[s] else None,
+                                  synth.bits_to_torch(v, DEV) if lens[s] else None, lens[s], 2, 5)
+                r.bulk(k, v, 2, 5)
+                refs[(layer, s)] = r
+        for step in range(steps):
+            if step == 70:
+                cache.set_share(2)                     # the policy retunes p: later batches follow 2/3
+                for r in refs.values():
+                    r.route.set_share(2)
+            for layer in range(n_layers):
+                k = synth.normal_bf16(rng, (len(seqs), 2, 128)); v = synth.normal_bf16(rng, (len(seqs), 2, 128))
+                cache.append(layer, seqs, synth.bits_to_torch(k, DEV), synth.bits_to_torch(v, DEV))
+                for i, s in enumerate(seqs):
+                    refs[(layer, s)].append(k[i:i + 1], v[i:i + 1])
+                if step % 13 == 0 or step == steps - 1:
+                    q = synth.normal_bf16(rng, (len(seqs), 8, 128))
+                    o = torch.zeros((len(seqs), 8, 128), device=DEV); lse = torch.zeros((len(seqs), 8), device=DEV)
+                    cache.attend_gpu(layer, seqs, synth.bits_to_torch(q, DEV), o, lse)
+                    parts = [refs[(layer, s)].attend(q[i], "gpu", scale) for i, s in enumerate(seqs)]
+                    torch.cuda.synchronize()
+                    check_partial(o.cpu().numpy(), lse.cpu().numpy(), np.stack([p[0] for p in parts]), np.stack([p[1] for p in parts]),
+                                  f"step {step} layer {layer}")
+                    cpu = [refs[(layer, s)].attend(q[i], "cpu", scale) for i, s in enumerate(seqs)]
+                    oc = torch.from_numpy(np.stack([p[0] for p in cpu]).astype(np.float32)).to(DEV)
+                    lc = torch.from_numpy(np.stack([p[1] for p in cpu]).astype(np.float32)).to(DEV)
+                    out = torch.zeros((len(seqs) * 8, 128), device=DEV); out_lse = torch.zeros(len(seqs) * 8, device=DEV)
+                    cache.merge(len(seqs) * 8, 128, [o.view(-1, 128), oc.view(-1, 128)], [lse.view(-1), lc.view(-1)], out, out_lse)
+                    torch.cuda.synchronize()
+                    full = [refs[(layer, s)].attend(q[i], "all", scale) for i, s in enumerate(seqs)]
+                    check_partial(out.cpu().numpy().reshape(len(seqs), 8, 128), out_lse.cpu().numpy().reshape(len(seqs), 8),
+                                  np.stack([p[0] for p in full]), np.stack([p[1] for p in full]), f"merged step {step}")
+        torch.cuda.synchronize()
+        for (layer, s), r in refs.items():
+            check_routing(cache, layer, s, r)
+            check_contents(cache, layer, s, r, range(0, len(r.route), 7))
+        st = cache.get_stats()
+        assert st["device_status"] == 0 and st["flushes"] > 0 and 0 < st["flushes_to_u"] < st["flushes"]
+
+
+def test_explicit_partial_flush_and_errors():
+    sh = synth.Shape("tiny", "gqa", 1, 8, 2, 128, 128, 128 ** -0.5)
+    rng = np.random.default_rng(60)
+    with make_cache(sh, 1, 2, block_tokens=16, window_tokens=32, chunk_tokens=32, max_u_tokens_per_seq=64,
+                    max_p_tokens_per_seq=64, resident_tokens_per_seq=64, share_num=1, share_den=2) as cache:
+        ref = RefSeq(sh, 16, 32, 1, 2)
+        ref.route.bulk(0, 0, 1)
+        for i in range(5):
+            k = synth.normal_bf16(rng, (1, 2, 128)); v = synth.normal_bf16(rng, (1, 2, 128))
+            cache.append(0, [1], synth.bits_to_torch(k, DEV), synth.bits_to_torch(v, DEV)); ref.append(k, v)
+        cache.flush(0, 1); ref.route.flush()          # a 5-token batch occupies one block
+        for i in range(3):
+            k = synth.normal_bf16(rng, (1, 2, 128)); v = synth.normal_bf16(rng, (1, 2, 128))
+            cache.append(0, [1], synth.bits_to_torch(k, DEV), synth.bits_to_torch(v, DEV)); ref.append(k, v)
+        cache.flush(); ref.route.flush()
+        torch.cuda.synchronize()
+        check_routing(cache, 0, 1, ref)
+        check_contents(cache, 0, 1, ref, range(8))
+        q = synth.normal_bf16(rng, (1, 8, 128))
+        o = torch.zeros((1, 8, 128), device=DEV); lse = torch.zeros((1, 8), device=DEV)
+        cache.attend_gpu(0, [1], synth.bits_to_torch(q, DEV), o, lse)
+        torch.cuda.synchronize()
+        og, lg = ref.attend(q[0], "gpu", float(np.float32(sh.scale)))
+        check_partial(o.cpu().numpy()[0], lse.cpu().numpy()[0], og, lg, "after partial flushes")
+        # a sequence with nothing on the GPU side: (0, -inf)
+        cache.attend_gpu(0, [0], synth.bits_to_torch(q, DEV), o, lse)
+        torch.cuda.synchronize()
+        assert torch.all(o == 0) and torch.all(torch.isneginf(lse))
+        kk = synth.bits_to_torch(synth.normal_bf16(rng, (200, 2, 128)), DEV)
+        with pytest.raises(binding.IpkvError) as e:
+            cache.append_bulk(0, 1, kk, kk, 10, 0, 1)
+        assert e.value.status == 4                     # not an empty sequence
+        with pytest.raises(binding.IpkvError) as e:
+            cache.append_bulk(0, 0, kk, kk, 200, 0, 1)
+        assert e.value.status == 3                     # exceeds the capacity of P
+        with pytest.raises(binding.IpkvError) as e:
+            cache.append(0, [1, 1], kk, kk)
+        assert e.value.status == 1
+        with pytest.raises(binding.IpkvError):
+            cache.locate(0, 1, 99)

@@ -1,0 +1,163 @@
+"""The library's host-side logic, run without a GPU: its router against the oracle's routing simulator
+(bit-exact indices), its split-K planner (every tile of every run covered exactly once), its layout
+arithmetic against the header's formula, and the C-ABI surface."""
+import ctypes as C
+import os
+import re
+import subprocess
+
+import numpy as np
+import pytest
+
+from oracle import c_oracle, np_oracle
+from paper_2609_14507_b200 import binding
+from tests import host_shim
+from tests.conftest import ROOT
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    from paper_2609_14507_b200 import build
+    build.build()
+
+
+def test_router_matches_oracle_on_random_programs():
+    rng = np.random.default_rng(31)
+    for trial in range(60):
+        block = int(rng.choice([1, 4, 16, 64]))
+        D = block * int(rng.integers(1, 5))
+        den = int(rng.integers(1, 16)); num = int(rng.integers(0, den + 1))
+        ours, ref = host_shim.Router(block, D, num, den), c_oracle.Route(block, D, num, den)
+        n0 = int(rng.integers(0, 400)); den0 = int(rng.integers(1, 11)); num0 = int(rng.integers(0, den0 + 1))
+        ours.bulk(n0, num0, den0); ref.bulk(n0, num0, den0)
+        for _ in range(int(rng.integers(0, 600))):
+            op = rng.integers(0, 40)
+            if op == 0:
+                ours.flush(); ref.flush()
+            elif op == 1:
+                s = int(rng.integers(0, den + 1)); ours.set_share(s); ref.set_share(s)
+            else:
+                ours.append(); ref.append()
+        for a, b in zip(ours.dump(), ref.dump()):
+            np.testing.assert_array_equal(a, b)
+        assert ours.counts() == ref.counts()
+
+
+def test_router_matches_oracle_on_paper_shaped_runs():
+    # D = 256, block 64, prefill 2048 (the paper's 2K prompt), decode to 8K at the shares of Table 3
+    for num, den, num0, den0 in [(15, 32, 15, 32), (35, 64, 1, 2), (5, 8, 0, 1), (0, 1, 1, 4), (1, 1, 1, 1)]:
+        ours, ref = host_shim.Router(64, 256, num, den), np_oracle.Route(64, 256, num, den)
+        ours.bulk(2048, num0, den0); ref.bulk(2048, num0, den0)
+        for _ in range(6144 + 1):
+            ours.append(); ref.append()
+        for a, b in zip(ours.dump(), ref.dump()):
+            np.testing.assert_array_equal(a, b)
+        assert ours.counts() == ref.counts()
+
+
+def test_plan_covers_every_tile_exactly_once():
+    rng = np.random.default_rng(32)
+    for trial in range(40):
+        n_rows = int(rng.integers(1, 20))
+        rows = [[int(x) for x in rng.integers(0, 5000, size=rng.integers(0, 4))] for _ in range(n_rows)]
+        heads = int(rng.choice([1, 4, 8]))
+        splits = int(rng.choice([0, 0, 1, 3, 16]))
+        p = host_shim.plan(rows, heads, splits)
+        live = [[n for n in row if n > 0] for row in rows]
+        assert list(p["seg_tokens"]) == [n for row in live for n in row]
+        assert p["row_item_start"][0] == 0 and p["row_item_start"][-1] == len(p["row"])
+        seg_id = 0
+        for r, row in enumerate(live):
+            i0, i1 = p["row_item_start"][r], p["row_item_start"][r + 1]
+            assert np.all(p["row"][i0:i1] == r)
+            covered = {}
+            for i in range(i0, i1):
+                assert p["ntiles"][i] >= 1
+                covered.setdefault(int(p["seg"][i]), []).append((int(p["tile0"][i]), int(p["ntiles"][i])))
+            for n in row:
+                pieces = sorted(covered.pop(seg_id))
+                t = 0
+                for t0, cnt in pieces:
+                    assert t0 == t
+                    t += cnt
+                assert t == -(-n // 64)
+                sizes = [c for _, c in pieces]
+                assert max(sizes) - min(sizes) <= 1          # balanced pieces
+                seg_id += 1
+            assert not covered
+
+
+def test_plan_fills_the_machine_in_whole_waves():
+    # Qwen3-shaped step: 16 rows x 32769 tokens, 4 KV heads -> CTAs = items * 4 close to a multiple of 296
+    p = host_shim.plan([[32768 - 256, 257]] * 16, 4)
+    ctas = len(p["row"]) * 4
+    assert 296 * 4 <= ctas <= 296 * 8
+    assert p["ntiles"].max() <= 32
+
+
+def test_layout_arithmetic_matches_header_formula():
+    L = host_shim.lib()
+    for bt in (16, 64, 256):
+        for t in range(bt):
+            for chunk in range(72):
+                x = chunk * 8
+                want = (x // 64) * bt * 128 + t * 128 + ((((x % 64) // 8) ^ (t & 7)) * 16)
+                assert L.shim_tile_chunk_offset(bt, t, chunk) == want
+                assert L.shim_plain_chunk_offset(576, t, chunk) == (t * 576 + x) * 2
+    # bytes per token per layer: the sizes behind Tables 1 and 2
+    assert L.shim_block_bytes(4, 128, 128, 64) == 64 * 2048
+    assert L.shim_block_bytes(8, 128, 128, 64) == 64 * 4096
+    assert L.shim_block_bytes(1, 576, 0, 64) == 64 * 1152
+
+
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(ROOT, "include", "ipkv.h")).read()
+    declared = sorted(set(re.findall(r"\b(ipkv_[a-z_]+)\s*\(", header)))
+    assert declared and set(declared) == set(binding.EXPORTS)
+    L = binding.lib()
+    for name in declared:
+        assert hasattr(L, name), name
+
+
+def test_struct_sizes_match_the_c_header(tmp_path):
+    src = tmp_path / "sz.c"
+    src.write_text('#include <stdio.h>\n#include "ipkv.h"\nint main(void){printf("%zu %zu %zu %zu %zu %zu\\n", sizeof(ipkv_config),'
+                   'sizeof(ipkv_attend_opts), sizeof(ipkv_extent), sizeof(ipkv_stats), sizeof(ipkv_attn_shape), sizeof(ipkv_run));return 0;}\n')
+    exe = tmp_path / "sz"
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)], check=True)
+    sizes = [int(x) for x in subprocess.run([str(exe)], capture_output=True, text=True, check=True).stdout.split()]
+    assert sizes == [C.sizeof(binding.Config), C.sizeof(binding.AttendOpts), C.sizeof(binding.Extent),
+                     C.sizeof(binding.Stats), C.sizeof(binding.AttnShape), C.sizeof(binding.Run)]
+
+
+def test_query_sizes_reproduce_table2(golden):
+    # The library's own sizing of W and PP (no GPU needed) against Table 2: bs=32, D=256, two
+    # ping-pong slots of 512 tokens per sequence.
+    shapes = {"ds2": (binding.MLA, 27, 16, 1, 576, 512), "qwen3": (binding.GQA, 48, 32, 4, 128, 128),
+              "mixtral": (binding.GQA, 32, 32, 8, 128, 128)}
+    for name, (kind, nl, hq, hkv, dqk, dv) in shapes.items():
+        cfg = binding.make_config(kind, nl, 32, hq, hkv, dqk, dv, block_tokens=64, window_tokens=256, chunk_tokens=512,
+                                  n_slots=2, max_u_tokens_per_seq=0, max_p_tokens_per_seq=0)
+        s = binding.ipkv_query_sizes(cfg)
+        assert abs(s["w"] / 1e6 - golden[f"table2.dwindow_mb.{name}"]) < 0.5
+        assert abs(s["pp"] / 1e6 - golden[f"table2.pingpong_mb.{name}"]) < 0.06
+        assert s["resident"] == 0 and s["u"] == 0 and s["p"] == 0
+
+
+def test_bad_configs_are_rejected_and_no_gpu_fails_loudly():
+    good = dict(block_tokens=64, window_tokens=256, chunk_tokens=512)
+    for kw in (dict(block_tokens=48), dict(window_tokens=100), dict(chunk_tokens=96), dict(n_slots=1),
+               dict(share_num=3, share_den=2), dict(share_den=0)):
+        cfg = binding.make_config(binding.GQA, 1, 1, 32, 4, 128, 128, **{**good, **kw})
+        with pytest.raises(binding.IpkvError):
+            binding.ipkv_query_sizes(cfg)
+    for dims in ((32, 5, 128, 128), (32, 4, 96, 96), (32, 4, 128, 64)):
+        cfg = binding.make_config(binding.GQA, 1, 1, *dims, **good)
+        with pytest.raises(binding.IpkvError):
+            binding.ipkv_query_sizes(cfg)
+    import torch
+    if not torch.cuda.is_available():
+        cfg = binding.make_config(binding.GQA, 1, 1, 32, 4, 128, 128, **good)
+        with pytest.raises(binding.IpkvError) as e:
+            binding.Cache(cfg)
+        assert e.value.status == 5          # IPKV_ECUDA: no silent CPU path
