@@ -1,0 +1,366 @@
+#!/usr/bin/env python
+"""Benchmark of the sequence-split decode-attention path (one JSON line on stdout, printed by rank 0).
+
+A "step" is one decode step of the whole path over one batch: for every layer, append one new K/V token
+per sequence (write-time routing into the D-window), attend the GPU-side share (split-K attention kernel +
+LSE reduce), and merge with the CPU-side partial (LSE merge kernel).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+Metric: KV-tokens/s of GPU-share decode attention, where one KV-token is one token of one layer's cache
+(all KV heads) attended by all query heads; bytes = KV-tokens x bytes per token per layer.
+With N > 1 every rank runs an independent replica on its own GPU (the path has no exchange step);
+`value` is the sum over ranks divided by the slowest rank's time.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from paper_2609_14507_b200 import synth  # noqa: E402
+
+METRIC = "gpu_share_decode_attn_kv_tokens_per_s"
+UNIT = "KV-tokens/s"
+
+WORKLOADS = {
+    # BASELINE config 2: Mixtral-8x7B-shaped attention, 32 layers, batch 16, 32K context, CPU share 25 %
+    "mixtral-8x7b-bs16-32k-cpu25": dict(shape=synth.MIXTRAL, batch=16, ctx=32768, share=(1, 4), cfg_id=2),
+    # BASELINE config 3 at CPU share 0: Qwen3-30B-A3B-shaped attention, 48 layers, batch 16, 32K context
+    "qwen3-30b-a3b-bs16-32k-cpu0": dict(shape=synth.QWEN3, batch=16, ctx=32768, share=(0, 1), cfg_id=3),
+    "qwen3-30b-a3b-bs16-32k-cpu50": dict(shape=synth.QWEN3, batch=16, ctx=32768, share=(1, 2), cfg_id=3),
+    # BASELINE config 1 (single layer, batch 1, 4K): latency-bound, for quick checks
+    "small-gqa-bs1-4k-cpu50": dict(shape=synth.SMALL_GQA, batch=1, ctx=4096, share=(1, 2), cfg_id=1),
+}
+DEFAULT_WORKLOAD = "mixtral-8x7b-bs16-32k-cpu25"
+BLOCK, WINDOW = 64, 256
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu_index, self.rows, self.proc, self.thread, self.t_mark = gpu_index, [], None, None, 0.0
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + self.FIELDS,
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), [x.strip() for x in line.split(",")]))
+
+    def mark(self):
+        """Start of the timed region: earlier samples are dropped."""
+        self.t_mark = time.time()
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        if self.thread:
+            self.thread.join(timeout=2)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ts, r in self.rows:
+            if len(r) < 7 or ts < self.t_mark:
+                continue
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, r[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_sample(wl, seconds_target=15.0, threads=None):
+    """Time the float64 oracle, as it stands, on a bounded sample of the workload: the GPU-side share of whole
+    sequences of layer 0 (all KV heads, all query heads), as many sequences as fit the time target."""
+    import torch
+    from oracle import c_oracle
+    sh = wl["shape"]
+    num0, den0 = wl["share"]
+    n_cpu = BLOCK * ((wl["ctx"] // BLOCK) * num0 // den0)
+    if threads:
+        c_oracle.set_threads(threads)
+    dev = "cuda:0" if torch.cuda.is_available() else None
+    done_tokens, t_total, n_seq = 0, 0.0, 0
+    while True:
+        seed = 1000 * wl["cfg_id"] + n_seq
+        if dev:
+            kd, vd = synth.device_kv(sh, wl["ctx"], seed, dev)
+            k, v = synth.torch_bits(kd), (synth.torch_bits(vd) if vd is not None else None)
+            q = synth.torch_bits(synth.device_q(sh, 1, seed + 500000, dev))[0]
+        else:
+            k, v = synth.host_kv(sh, wl["ctx"], seed)
+            q = synth.host_q(sh, 1, seed + 500000)[0]
+        idx = np.arange(n_cpu, wl["ctx"])
+        t0 = time.perf_counter()
+        c_oracle.attend(q, k, sh.dim_v if v is None else v, idx, float(np.float32(sh.scale)))
+        dt = time.perf_counter() - t0
+        done_tokens += idx.size
+        t_total += dt
+        n_seq += 1
+        if t_total >= seconds_target or n_seq >= sh.n_layers * wl["batch"]:
+            break
+    return dict(value=done_tokens / t_total, unit=UNIT, cores=c_oracle.num_threads(), kind="oracle",
+                sample=f"{n_seq} of {sh.n_layers * wl['batch']} (layer, sequence) pairs, GPU-side share ({idx.size} tokens each), "
+                       f"all heads; {t_total:.1f} s of float64 C++ (OpenMP over query heads)")
+
+
+def run_reference(args, wl, name):
+    """--impl reference: the oracle on the host cores, on the same workload and metric; each step is a bounded sample."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    per_step = []
+    for _ in range(args.warmup):
+        oracle_sample(wl, seconds_target=1.0)
+    info = None
+    for _ in range(args.steps):
+        info = oracle_sample(wl, seconds_target=max(2.0, min(15.0, 120.0 / max(1, args.steps))))
+        per_step.append(info["value"])
+    value = float(np.mean(per_step))
+    info["value"] = value
+    sh = wl["shape"]
+    n_tok = sh.n_layers * wl["batch"] * (wl["ctx"] - BLOCK * ((wl["ctx"] // BLOCK) * wl["share"][0] // wl["share"][1]) + 1)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * n_tok / value, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": {"workload": name},
+        "cpu_baseline": info, "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--kv-splits", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    wl = WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, wl, args.workload)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2609_14507_b200 import binding, build
+    build.build()                      # no-op when libipkv.so is up to date; raises if it cannot be built
+    binding.lib()                      # fail loudly if the CUDA library is missing
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    sh, B, ctx = wl["shape"], wl["batch"], wl["ctx"]
+    num0, den0 = wl["share"]
+    NL, Hq, Hkv, dqk, dv = sh.n_layers, sh.n_q_heads, sh.n_kv_heads, sh.dim_qk, sh.dim_v
+    n_cpu = BLOCK * ((ctx // BLOCK) * num0 // den0)
+    n_gpu0 = ctx - n_cpu
+    total_steps = 2 * (args.warmup + args.steps) + 8
+    p_cap = n_gpu0 + WINDOW * (total_steps // WINDOW + 2)
+    kind = binding.MLA if sh.kind == "mla" else binding.GQA
+    cfg = binding.make_config(kind, NL, B, Hq, Hkv, dqk, dv, block_tokens=BLOCK, window_tokens=WINDOW, chunk_tokens=512,
+                              n_slots=2, max_u_tokens_per_seq=n_cpu + WINDOW * (total_steps // WINDOW + 2),
+                              max_p_tokens_per_seq=p_cap, resident_tokens_per_seq=p_cap, softmax_scale=sh.scale,
+                              share_num=num0, share_den=den0, device=local_rank,
+                              flags=binding.FLAG_NO_HOST_U | binding.FLAG_NO_HOST_P)
+    cache = binding.Cache(cfg)
+    seq_ids = list(range(B))
+    # ---- populate: prefill routed in one shot, the GPU-side share lands in the resident ring -------------
+    for layer in range(NL):
+        for s in range(B):
+            k, v = synth.device_kv(sh, ctx, 1000 * wl["cfg_id"] + (layer * B + s) + 100 * rank, dev)
+            cache.append_bulk(layer, s, k, v, ctx, num0, den0)
+        torch.cuda.synchronize()
+    g = torch.Generator(device=dev); g.manual_seed(77 + rank)
+    bf = torch.bfloat16
+    q = torch.randn((NL, B, Hq, dqk), generator=g, device=dev).to(bf)
+    k_new = torch.randn((NL, B, Hkv, dqk), generator=g, device=dev).to(bf)
+    v_new = None if sh.kind == "mla" else torch.randn((NL, B, Hkv, dv), generator=g, device=dev).to(bf)
+    # CPU-side partial: synthetic values of the right shape and scale (the CPU engine is outside this path)
+    o_cpu = (torch.randn((NL, B * Hq, dv), generator=g, device=dev) / max(1.0, float(n_cpu)) ** 0.5).contiguous()
+    lse_cpu = (torch.randn((NL, B * Hq), generator=g, device=dev) * 0.1 + float(np.log(max(1, n_cpu)))).contiguous()
+    if n_cpu == 0:
+        o_cpu.zero_(); lse_cpu.fill_(float("-inf"))
+    o_part = torch.zeros((B, Hq, dv), device=dev)
+    lse_part = torch.zeros((B, Hq), device=dev)
+    out = torch.zeros((NL, B * Hq, dv), device=dev, dtype=bf)
+    out_lse = torch.zeros((B * Hq,), device=dev)
+    bpt = sh.bytes_per_token
+
+    def step():
+        for layer in range(NL):
+            cache.append(layer, seq_ids, k_new[layer], None if v_new is None else v_new[layer])
+            cache.attend_gpu(layer, seq_ids, q[layer], o_part, lse_part, kv_splits=args.kv_splits)
+            cache.merge(B * Hq, dv, [o_part.view(B * Hq, dv), o_cpu[layer]], [lse_part.view(-1), lse_cpu[layer]],
+                        out[layer], out_lse, out_is_bf16=True)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x):
+        if world == 1:
+            return x
+        t = torch.tensor([x], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    st0 = cache.get_stats()
+    cache.profile_enable(True)
+    cache.profile_read()
+    sampler.mark()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    ms = max_over_ranks(e0.elapsed_time(e1))
+    kern_ms, n_timed, n_launch = cache.profile_read()
+    cache.profile_enable(False)
+    st1 = cache.get_stats()
+    bytes_attended = st1["kv_bytes_attended"] - st0["kv_bytes_attended"]
+    tokens = bytes_attended // bpt
+    launches = sum(st1[k] - st0[k] for k in ("attend_kernels", "reduce_kernels", "merge_kernels", "append_kernels", "pack_kernels"))
+    value = world * tokens / (ms * 1e-3)
+    peak, peak_kind = measured_peaks()
+    ach = (bytes_attended * (n_timed / max(1, n_launch))) / (kern_ms * 1e-3) / 1e9 if kern_ms > 0 else 0.0
+    roofline = {"bound": "hbm", "kernel": "attn_gqa_kernel" if sh.kind == "gqa" else "attn_mla_kernel", "achieved": ach,
+                "peak": peak, "peak_kind": peak_kind + " copy bandwidth (MEASURED_PEAKS.json hbm_gbs)" if peak_kind == "measured"
+                else "fallback 6650 GB/s", "unit": "GB/s", "frac": ach / peak, "frac_of_8000_nominal": ach / 8000.0,
+                "avg_launch_us": 1e3 * kern_ms / max(1, n_timed), "bytes_per_launch": bytes_attended / max(1, n_launch),
+                "traffic": None, "whole_step_gbs": world * bytes_attended / (ms * 1e-3) / 1e9}
+    traffic_path = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(traffic_path):
+        try:
+            with open(traffic_path) as f:
+                tj = json.load(f).get(args.workload)
+            if tj:
+                roofline["traffic"] = tj["dram_bytes_per_launch"]
+        except (OSError, ValueError, KeyError):
+            pass
+
+    # ---- end to end: host buffers in, host buffer out, through the same calls ---------------------------------
+    e2e = None
+    if not args.no_e2e:
+        hq = q.cpu().pin_memory(); hk = k_new.cpu().pin_memory()
+        hv = None if v_new is None else v_new.cpu().pin_memory()
+        hoc = o_cpu.cpu().pin_memory(); hlc = lse_cpu.cpu().pin_memory()
+        hout = torch.zeros((NL, B * Hq, dv), dtype=bf).pin_memory()
+        dq = torch.empty_like(q[0]); dk = torch.empty_like(k_new[0]); dvn = None if v_new is None else torch.empty_like(v_new[0])
+
+        def step_e2e():
+            for layer in range(NL):
+                dq.copy_(hq[layer], non_blocking=True)
+                dk.copy_(hk[layer], non_blocking=True)
+                if dvn is not None:
+                    dvn.copy_(hv[layer], non_blocking=True)
+                cache.append(layer, seq_ids, dk, dvn)
+                cache.attend_gpu(layer, seq_ids, dq, o_part, lse_part, kv_splits=args.kv_splits)
+                # the CPU-side partial is handed over in pinned host memory; ipkv_merge copies it in
+                cache.merge(B * Hq, dv, [o_part.view(B * Hq, dv), hoc[layer]], [lse_part.view(-1), hlc[layer]],
+                            out[layer], out_lse, out_is_bf16=True)
+                hout[layer].copy_(out[layer], non_blocking=True)
+            torch.cuda.synchronize()
+
+        for _ in range(args.warmup):
+            step_e2e()
+        barrier()
+        s0 = cache.get_stats()
+        t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+        t0.record()
+        for _ in range(args.steps):
+            step_e2e()
+        t1.record()
+        barrier()
+        ms2 = max_over_ranks(t0.elapsed_time(t1))
+        s1 = cache.get_stats()
+        tok2 = (s1["kv_bytes_attended"] - s0["kv_bytes_attended"]) // bpt
+        h2d = NL * (hq[0].numel() * 2 + hk[0].numel() * 2 + (0 if hv is None else hv[0].numel() * 2) + hoc[0].numel() * 4 + hlc[0].numel() * 4)
+        e2e = {"value": world * tok2 / (ms2 * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": NL * hout[0].numel() * 2, "ms_per_step": ms2 / args.steps}
+    status = cache.get_stats()["device_status"]
+    if status != 0:
+        raise RuntimeError("a kernel reported a timed-out wait; the numbers are invalid")
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cache.close()
+        torch.cuda.empty_cache()
+        cpu = oracle_sample(wl)
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": args.workload, "layers": NL, "batch": B, "context": ctx, "cpu_share": f"{num0}/{den0}",
+                       "gpu_share_tokens_per_seq": n_gpu0 + 1, "bytes_per_kv_token": bpt, "block_tokens": BLOCK, "window_tokens": WINDOW,
+                       "gpu_share": "HBM-resident", "host_copies_of_U_and_P": "off (benchmark)", "cpu_partial": "synthetic values",
+                       "l2": "inputs larger than L2 (each layer reads its own %.2f GB)" % (bytes_attended / max(1, n_launch) / 1e9),
+                       "multi_gpu": "replicas only", "kv_splits": args.kv_splits},
+            "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu,
+            "step_gbs": world * bytes_attended / (ms * 1e-3) / 1e9,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -203,6 +203,13 @@ typedef struct {
 } ipkv_stats;
 ipkv_status ipkv_get_stats(ipkv_t* h, ipkv_stats* out);
 
+/* Kernel timing for benchmarks.  While enabled, every attention-kernel launch of ipkv_attend_gpu is
+ * bracketed by a pair of CUDA events on the launching stream.  ipkv_profile_read synchronises the device,
+ * returns the summed kernel time (milliseconds) and the number of launches since the last read, and resets
+ * both.  At most 8192 launches are kept between two reads; later ones are counted but not timed. */
+ipkv_status ipkv_profile_enable(ipkv_t* h, int32_t on);
+ipkv_status ipkv_profile_read(ipkv_t* h, double* attend_kernel_ms, int64_t* n_timed, int64_t* n_launches);
+
 /* ---- stateless kernel entry points (no handle) ------------------------------------------------- */
 
 typedef struct {

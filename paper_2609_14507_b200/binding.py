@@ -22,7 +22,7 @@ STATUS_NAMES = {0: "OK", 1: "EINVAL", 2: "ENOMEM", 3: "ERANGE", 4: "ESTATE", 5: 
 EXPORTS = [
     "ipkv_query_sizes", "ipkv_create", "ipkv_destroy", "ipkv_set_share", "ipkv_reset", "ipkv_append_bulk",
     "ipkv_append", "ipkv_flush", "ipkv_attend_gpu", "ipkv_merge", "ipkv_views", "ipkv_locate", "ipkv_counts",
-    "ipkv_read_token", "ipkv_get_stats", "ipkv_attend_scratch_bytes", "ipkv_attend_runs", "ipkv_pack_blocks",
+    "ipkv_read_token", "ipkv_get_stats", "ipkv_profile_enable", "ipkv_profile_read", "ipkv_attend_scratch_bytes", "ipkv_attend_runs", "ipkv_pack_blocks",
     "ipkv_block_bytes", "ipkv_status_str", "ipkv_last_error", "ipkv_version",
 ]
 
@@ -100,6 +100,8 @@ def lib():
         "ipkv_counts": [vp, i32, i32, C.POINTER(i64)],
         "ipkv_read_token": [vp, i32, i32, i64, vp, vp],
         "ipkv_get_stats": [vp, C.POINTER(Stats)],
+        "ipkv_profile_enable": [vp, i32],
+        "ipkv_profile_read": [vp, C.POINTER(C.c_double), C.POINTER(i64), C.POINTER(i64)],
         "ipkv_attend_scratch_bytes": [C.POINTER(AttnShape), i32, i32, i64, i32, C.POINTER(C.c_size_t)],
         "ipkv_attend_runs": [C.POINTER(AttnShape), i32, C.POINTER(Run), C.POINTER(i32), vp, i32, vp, C.c_size_t, vp, vp, vp, vp],
         "ipkv_pack_blocks": [C.POINTER(AttnShape), i32, vp, vp, i64, vp, vp],
@@ -249,6 +251,15 @@ class Cache:
         self._check(lib().ipkv_read_token(self._h, layer, seq, token, k.ctypes.data, v.ctypes.data if v is not None else None),
                     "ipkv_read_token")
         return k, v
+
+    def profile_enable(self, on=True):
+        self._check(lib().ipkv_profile_enable(self._h, 1 if on else 0), "ipkv_profile_enable")
+
+    def profile_read(self):
+        """(summed attention-kernel milliseconds, launches timed, launches seen) since the last read."""
+        ms, nt, nl = C.c_double(), C.c_int64(), C.c_int64()
+        self._check(lib().ipkv_profile_read(self._h, C.byref(ms), C.byref(nt), C.byref(nl)), "ipkv_profile_read")
+        return ms.value, nt.value, nl.value
 
     def get_stats(self):
         s = Stats()

@@ -122,6 +122,11 @@ struct ipkv {
     cudaEvent_t ev_main = nullptr;
     ipkv_stats stats;
     std::string err;
+    // optional kernel timing
+    bool prof_on = false;
+    std::vector<cudaEvent_t> prof_ev;      // pairs
+    size_t prof_used = 0;                  // events used
+    int64_t prof_launches = 0;
 
     SeqState& state(int layer, int seq) { return st[size_t(layer) * cfg.max_seqs + seq]; }
     int64_t seq_index(int layer, int seq) const { return int64_t(layer) * cfg.max_seqs + seq; }
@@ -364,7 +369,11 @@ ipkv_status run_group(ipkv* h, const std::vector<std::vector<PlanSeg>>& rows, co
     a.out_o = out_o; a.out_lse = out_lse;
     a.status = h->status_dev;
     if (a.n_items > 0) {
+        const bool timed = h->prof_on && h->prof_used + 2 <= h->prof_ev.size();
+        if (timed) CU(h, cudaEventRecord(h->prof_ev[h->prof_used], s));
         CU(h, launch_attend(a, s));
+        if (timed) { CU(h, cudaEventRecord(h->prof_ev[h->prof_used + 1], s)); h->prof_used += 2; }
+        if (h->prof_on) h->prof_launches += 1;
         h->stats.attend_kernels += 1;
     }
     CU(h, launch_split_reduce(a, s));
@@ -421,6 +430,7 @@ ipkv_status ipkv_destroy(ipkv_t* h) {
     if (h->merge_stage) cudaFree(h->merge_stage);
     if (h->status_dev) cudaFree(h->status_dev);
     for (int i = 0; i < ipkv::kTableParts; ++i) if (h->table_ev[i]) cudaEventDestroy(h->table_ev[i]);
+    for (auto e : h->prof_ev) cudaEventDestroy(e);
     for (auto e : h->slot_ready) cudaEventDestroy(e);
     for (auto e : h->slot_free) cudaEventDestroy(e);
     if (h->ev_main) cudaEventDestroy(h->ev_main);
@@ -862,6 +872,35 @@ ipkv_status ipkv_get_stats(ipkv_t* h, ipkv_stats* out) {
     CU(h, cudaMemcpy(&h->stats.device_status, h->status_dev, sizeof(uint32_t), cudaMemcpyDeviceToHost));
     *out = h->stats;
     return h->stats.device_status ? fail(h, IPKV_ETIMEOUT, "a kernel's bounded wait gave up; results of that call are invalid") : IPKV_OK;
+}
+
+ipkv_status ipkv_profile_enable(ipkv_t* h, int32_t on) {
+    if (!h) return IPKV_EINVAL;
+    CU(h, cudaSetDevice(h->cfg.device));
+    if (on && h->prof_ev.empty()) {
+        h->prof_ev.resize(2 * 8192);
+        for (auto& e : h->prof_ev) e = nullptr;
+        for (auto& e : h->prof_ev) CU(h, cudaEventCreate(&e));
+    }
+    h->prof_on = on != 0;
+    return IPKV_OK;
+}
+
+ipkv_status ipkv_profile_read(ipkv_t* h, double* attend_kernel_ms, int64_t* n_timed, int64_t* n_launches) {
+    if (!h || !attend_kernel_ms || !n_timed || !n_launches) return IPKV_EINVAL;
+    CU(h, cudaSetDevice(h->cfg.device));
+    CU(h, cudaDeviceSynchronize());
+    double total = 0.0;
+    for (size_t i = 0; i + 1 < h->prof_used; i += 2) {
+        float ms = 0.f;
+        CU(h, cudaEventElapsedTime(&ms, h->prof_ev[i], h->prof_ev[i + 1]));
+        total += ms;
+    }
+    *attend_kernel_ms = total;
+    *n_timed = int64_t(h->prof_used / 2);
+    *n_launches = h->prof_launches;
+    h->prof_used = 0; h->prof_launches = 0;
+    return IPKV_OK;
 }
 
 // ---- stateless entry points ---------------------------------------------------------------------

@@ -60,7 +60,7 @@ struct SmemPlan {
     static_assert(kMergeL + kConsumerWarps * 16 * 4 <= kStagesBytes + 16 * kQPitch, "merge area must fit");
 };
 
-template <int D, int STAGES>
+template <int D, int STAGES, bool DUP>
 __global__ void __launch_bounds__(kThreads) attn_gqa_kernel(const GqaParams p) {
     using SP = SmemPlan<D, STAGES>;
     extern __shared__ unsigned char smem_dyn[];
@@ -89,8 +89,9 @@ __global__ void __launch_bounds__(kThreads) attn_gqa_kernel(const GqaParams p) {
     for (int c = tid; c < 16 * (D / 8); c += kThreads) {
         const int r = c / (D / 8), ch = c - r * (D / 8);
         uint4 val = make_uint4(0, 0, 0, 0);
-        if (r < n_heads)
-            val = *reinterpret_cast<const uint4*>(p.q + (int64_t(item.row) * p.Hq + head0 + r) * D + ch * 8);
+        const int hr = DUP ? (r & 7) : r;                  // DUP: rows 8..15 repeat rows 0..7
+        if (hr < n_heads)
+            val = *reinterpret_cast<const uint4*>(p.q + (int64_t(item.row) * p.Hq + head0 + hr) * D + ch * 8);
         *reinterpret_cast<uint4*>(smem + SP::kQOff + r * SP::kQPitch + ch * 16) = val;
     }
     if (p.bt < kTileTokens) {
@@ -160,6 +161,11 @@ __global__ void __launch_bounds__(kThreads) attn_gqa_kernel(const GqaParams p) {
     }
 
     // ---------------- consumers ----------------
+    // The softmax weights are split into a bf16 head and a bf16 remainder (p = p_hi + p_lo, about 16
+    // significant bits) before the P.V product, so that the output error stays at fp32-accumulation level.
+    //   DUP (at most 8 query heads in the CTA): query rows 8..15 duplicate rows 0..7; MMA rows 0..7 carry
+    //   p_hi and rows 8..15 carry p_lo, so the remainder costs no extra tensor-core work.
+    //   otherwise: two P.V products per tile.
     uint32_t qa[D / 16][4];
     {
         const int mi = lane >> 3, r = lane & 7;
@@ -202,39 +208,59 @@ __global__ void __launch_bounds__(kThreads) attn_gqa_kernel(const GqaParams p) {
 #pragma unroll
             for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
+                for (int j = 0; j < (DUP ? 2 : 4); ++j) {
                     const int t = tcol + nt * 8 + (j & 1);
                     s[nt][j] = (t < n_valid) ? s[nt][j] * p.scale_log2 : -INFINITY;
                 }
             float mx0 = fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1]));
-            float mx1 = fmaxf(fmaxf(s[0][2], s[0][3]), fmaxf(s[1][2], s[1][3]));
             mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
             mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
-            mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
-            mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-            const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
-            const float ms0 = (mn0 == -INFINITY) ? 0.f : mn0, ms1 = (mn1 == -INFINITY) ? 0.f : mn1;
-            const float a0 = ptx::ex2(m0 - ms0), a1 = ptx::ex2(m1 - ms1);
-            m0 = mn0; m1 = mn1;
+            const float mn0 = fmaxf(m0, mx0);
+            const float ms0 = (mn0 == -INFINITY) ? 0.f : mn0;
+            const float a0 = ptx::ex2(m0 - ms0);
+            m0 = mn0;
+            float a1 = a0, ms1 = ms0;
+            if (!DUP) {
+                float mx1 = fmaxf(fmaxf(s[0][2], s[0][3]), fmaxf(s[1][2], s[1][3]));
+                mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+                mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+                const float mn1 = fmaxf(m1, mx1);
+                ms1 = (mn1 == -INFINITY) ? 0.f : mn1;
+                a1 = ptx::ex2(m1 - ms1);
+                m1 = mn1;
+            }
             float pr[2][4];
 #pragma unroll
             for (int nt = 0; nt < 2; ++nt) {
                 pr[nt][0] = ptx::ex2(s[nt][0] - ms0);
                 pr[nt][1] = ptx::ex2(s[nt][1] - ms0);
-                pr[nt][2] = ptx::ex2(s[nt][2] - ms1);
-                pr[nt][3] = ptx::ex2(s[nt][3] - ms1);
+                if (!DUP) {
+                    pr[nt][2] = ptx::ex2(s[nt][2] - ms1);
+                    pr[nt][3] = ptx::ex2(s[nt][3] - ms1);
+                }
             }
             l0 = l0 * a0 + (pr[0][0] + pr[0][1] + pr[1][0] + pr[1][1]);
-            l1 = l1 * a1 + (pr[0][2] + pr[0][3] + pr[1][2] + pr[1][3]);
+            if (!DUP) l1 = l1 * a1 + (pr[0][2] + pr[0][3] + pr[1][2] + pr[1][3]);
             if (__any_sync(0xffffffffu, (a0 != 1.f) | (a1 != 1.f))) {
 #pragma unroll
                 for (int nt = 0; nt < D / 8; ++nt) { o[nt][0] *= a0; o[nt][1] *= a0; o[nt][2] *= a1; o[nt][3] *= a1; }
             }
-            uint32_t pa[4];
-            pa[0] = ptx::pack_bf16(pr[0][0], pr[0][1]);
-            pa[1] = ptx::pack_bf16(pr[0][2], pr[0][3]);
-            pa[2] = ptx::pack_bf16(pr[1][0], pr[1][1]);
-            pa[3] = ptx::pack_bf16(pr[1][2], pr[1][3]);
+            uint32_t pa[4], pb[4];
+            if (DUP) {
+                pa[0] = ptx::pack_bf16(pr[0][0], pr[0][1]);
+                pa[2] = ptx::pack_bf16(pr[1][0], pr[1][1]);
+                pa[1] = ptx::pack_bf16(pr[0][0] - ptx::bf16_lo(pa[0]), pr[0][1] - ptx::bf16_hi(pa[0]));
+                pa[3] = ptx::pack_bf16(pr[1][0] - ptx::bf16_lo(pa[2]), pr[1][1] - ptx::bf16_hi(pa[2]));
+            } else {
+                pa[0] = ptx::pack_bf16(pr[0][0], pr[0][1]);
+                pa[1] = ptx::pack_bf16(pr[0][2], pr[0][3]);
+                pa[2] = ptx::pack_bf16(pr[1][0], pr[1][1]);
+                pa[3] = ptx::pack_bf16(pr[1][2], pr[1][3]);
+                pb[0] = ptx::pack_bf16(pr[0][0] - ptx::bf16_lo(pa[0]), pr[0][1] - ptx::bf16_hi(pa[0]));
+                pb[1] = ptx::pack_bf16(pr[0][2] - ptx::bf16_lo(pa[1]), pr[0][3] - ptx::bf16_hi(pa[1]));
+                pb[2] = ptx::pack_bf16(pr[1][0] - ptx::bf16_lo(pa[2]), pr[1][1] - ptx::bf16_hi(pa[2]));
+                pb[3] = ptx::pack_bf16(pr[1][2] - ptx::bf16_lo(pa[3]), pr[1][3] - ptx::bf16_hi(pa[3]));
+            }
 #pragma unroll
             for (int jj = 0; jj < D / 16; ++jj) {
                 const int chunk = 2 * jj + (mi >> 1);
@@ -242,6 +268,10 @@ __global__ void __launch_bounds__(kThreads) attn_gqa_kernel(const GqaParams p) {
                 ptx::ldmatrix_x4_trans(vb + (chunk >> 3) * 8192 + tokV * 128 + (((chunk & 7) ^ r8) << 4), b0, b1, b2, b3);
                 ptx::mma_bf16(o[2 * jj], pa, b0, b1);
                 ptx::mma_bf16(o[2 * jj + 1], pa, b2, b3);
+                if (!DUP) {
+                    ptx::mma_bf16(o[2 * jj], pb, b0, b1);
+                    ptx::mma_bf16(o[2 * jj + 1], pb, b2, b3);
+                }
             }
         }
         __syncwarp();
@@ -264,12 +294,16 @@ __global__ void __launch_bounds__(kThreads) attn_gqa_kernel(const GqaParams p) {
         float* w = mo + warp * 16 * D;
 #pragma unroll
         for (int nt = 0; nt < D / 8; ++nt) {
-            *reinterpret_cast<float2*>(w + r0 * D + nt * 8 + c0) = make_float2(o[nt][0], o[nt][1]);
-            *reinterpret_cast<float2*>(w + (r0 + 8) * D + nt * 8 + c0) = make_float2(o[nt][2], o[nt][3]);
+            if (DUP) {
+                *reinterpret_cast<float2*>(w + r0 * D + nt * 8 + c0) = make_float2(o[nt][0] + o[nt][2], o[nt][1] + o[nt][3]);
+            } else {
+                *reinterpret_cast<float2*>(w + r0 * D + nt * 8 + c0) = make_float2(o[nt][0], o[nt][1]);
+                *reinterpret_cast<float2*>(w + (r0 + 8) * D + nt * 8 + c0) = make_float2(o[nt][2], o[nt][3]);
+            }
         }
         if ((lane & 3) == 0) {
-            mm[warp * 16 + r0] = m0; mm[warp * 16 + r0 + 8] = m1;
-            ml[warp * 16 + r0] = l0; ml[warp * 16 + r0 + 8] = l1;
+            mm[warp * 16 + r0] = m0; ml[warp * 16 + r0] = l0;
+            if (!DUP) { mm[warp * 16 + r0 + 8] = m1; ml[warp * 16 + r0 + 8] = l1; }
         }
     }
     __syncthreads();
@@ -294,7 +328,7 @@ __global__ void __launch_bounds__(kThreads) attn_gqa_kernel(const GqaParams p) {
     }
 }
 
-template <int D, int STAGES>
+template <int D, int STAGES, bool DUP>
 cudaError_t launch_gqa(const AttnLaunch& a, cudaStream_t s) {
     using SP = SmemPlan<D, STAGES>;
     GqaParams p;
@@ -313,12 +347,12 @@ cudaError_t launch_gqa(const AttnLaunch& a, cudaStream_t s) {
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64 || !configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(attn_gqa_kernel<D, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        cudaError_t e = cudaFuncSetAttribute(attn_gqa_kernel<D, STAGES, DUP>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
     dim3 grid(a.n_items, a.n_kv_heads * p.n_hg);
-    attn_gqa_kernel<D, STAGES><<<grid, kThreads, smem, s>>>(p);
+    attn_gqa_kernel<D, STAGES, DUP><<<grid, kThreads, smem, s>>>(p);
     return cudaGetLastError();
 }
 
@@ -326,8 +360,9 @@ cudaError_t launch_gqa(const AttnLaunch& a, cudaStream_t s) {
 
 cudaError_t launch_attend_gqa(const AttnLaunch& a, cudaStream_t s) {
     if (a.n_items <= 0) return cudaSuccess;
-    if (a.dim_qk == 128 && a.dim_v == 128) return launch_gqa<128, 3>(a, s);
-    if (a.dim_qk == 64 && a.dim_v == 64) return launch_gqa<64, 4>(a, s);
+    const bool dup = a.n_q_heads / a.n_kv_heads <= 8;
+    if (a.dim_qk == 128 && a.dim_v == 128) return dup ? launch_gqa<128, 3, true>(a, s) : launch_gqa<128, 3, false>(a, s);
+    if (a.dim_qk == 64 && a.dim_v == 64) return dup ? launch_gqa<64, 4, true>(a, s) : launch_gqa<64, 4, false>(a, s);
     return cudaErrorInvalidValue;
 }
 
