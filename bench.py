@@ -38,6 +38,11 @@ WORKLOADS = {
     # BASELINE config 3 at CPU share 0: Qwen3-30B-A3B-shaped attention, 48 layers, batch 16, 32K context
     "qwen3-30b-a3b-bs16-32k-cpu0": dict(shape=synth.QWEN3, batch=16, ctx=32768, share=(0, 1), cfg_id=3),
     "qwen3-30b-a3b-bs16-32k-cpu50": dict(shape=synth.QWEN3, batch=16, ctx=32768, share=(1, 2), cfg_id=3),
+    # two layers of config 2: a few GB on the device, still far larger than L2 -- the size used for ncu captures
+    "mixtral-2layers-bs16-32k-cpu25": dict(shape=synth.Shape("mixtral-2l", "gqa", 2, 32, 8, 128, 128, 128 ** -0.5), batch=16,
+                                           ctx=32768, share=(1, 4), cfg_id=2),
+    "qwen3-2layers-bs16-32k-cpu0": dict(shape=synth.Shape("qwen3-2l", "gqa", 2, 32, 4, 128, 128, 128 ** -0.5), batch=16,
+                                        ctx=32768, share=(0, 1), cfg_id=3),
     # BASELINE config 1 (single layer, batch 1, 4K): latency-bound, for quick checks
     "small-gqa-bs1-4k-cpu50": dict(shape=synth.SMALL_GQA, batch=1, ctx=4096, share=(1, 2), cfg_id=1),
 }
