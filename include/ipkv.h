@@ -239,6 +239,28 @@ ipkv_status ipkv_attend_runs(const ipkv_attn_shape* shape, int32_t n_rows,
                              void* scratch_dev, size_t scratch_bytes,
                              float* o_part_dev, float* lse_part_dev, uint32_t* status_dev, void* stream);
 
+/* Same computation and arguments as ipkv_attend_runs, but without a scratch argument: the scratch lives in a
+ * fixed 16 MiB array inside the library's device image.  (The paper has no counterpart; this exists for hosts
+ * that must not allocate device memory where they call attention: servers that give all memory to their own
+ * pool at start-up, latency-critical loops that cannot afford cudaMalloc's device-wide synchronisation,
+ * plug-ins whose contract forbids allocation.)  The call allocates nothing on the device: no cudaMalloc,
+ * no cudaFree, no allocating library routine.
+ *   - Limit: the call needs ipkv_attend_scratch_bytes(shape, n_rows, n_runs, total tokens, kv_splits) bytes;
+ *     if that exceeds ipkv_noalloc_scratch_limit() (16 MiB) it returns IPKV_ERANGE and does nothing.
+ *     A larger kv_splits or batch needs more; use ipkv_attend_runs with your own scratch then.
+ *   - The array is one per GPU and is held from library load to process exit by every GPU that runs it.
+ *   - The first call on a device resolves the array's device address (cudaGetSymbolAddress, with that device
+ *     current).  Make that first call outside any stream capture.
+ *   - All calls on a device share the array and each finds the previous call's bytes in it; nothing needs
+ *     clearing between calls, but two calls whose work overlaps on the GPU (different streams without an
+ *     ordering event, or another host thread) race on it.  Order them.
+ * status_dev as in ipkv_attend_runs. */
+ipkv_status ipkv_attend_runs_noalloc(const ipkv_attn_shape* shape, int32_t n_rows,
+                                     const ipkv_run* runs, const int32_t* row_run_start,
+                                     const void* q_dev, int32_t kv_splits,
+                                     float* o_part_dev, float* lse_part_dev, uint32_t* status_dev, void* stream);
+size_t ipkv_noalloc_scratch_limit(void);
+
 /* Re-lay token-major K/V ([n_tokens][n_kv_heads][dim]) into consecutive blocks of the given layout
  * starting at token offset 0 of dst_dev (device to device; used by tests and by callers that build
  * blocks themselves).  v_dev = NULL for IPKV_MLA. */

@@ -23,6 +23,7 @@ EXPORTS = [
     "ipkv_query_sizes", "ipkv_create", "ipkv_destroy", "ipkv_set_share", "ipkv_reset", "ipkv_append_bulk",
     "ipkv_append", "ipkv_flush", "ipkv_attend_gpu", "ipkv_merge", "ipkv_views", "ipkv_locate", "ipkv_counts",
     "ipkv_read_token", "ipkv_get_stats", "ipkv_profile_enable", "ipkv_profile_read", "ipkv_attend_scratch_bytes", "ipkv_attend_runs", "ipkv_pack_blocks",
+    "ipkv_attend_runs_noalloc", "ipkv_noalloc_scratch_limit",
     "ipkv_block_bytes", "ipkv_status_str", "ipkv_last_error", "ipkv_version",
 ]
 
@@ -105,6 +106,7 @@ def lib():
         "ipkv_attend_scratch_bytes": [C.POINTER(AttnShape), i32, i32, i64, i32, C.POINTER(C.c_size_t)],
         "ipkv_attend_runs": [C.POINTER(AttnShape), i32, C.POINTER(Run), C.POINTER(i32), vp, i32, vp, C.c_size_t, vp, vp, vp, vp],
         "ipkv_pack_blocks": [C.POINTER(AttnShape), i32, vp, vp, i64, vp, vp],
+        "ipkv_attend_runs_noalloc": [C.POINTER(AttnShape), i32, C.POINTER(Run), C.POINTER(i32), vp, i32, vp, vp, vp, vp],
     }
     for name, args in sig.items():
         f = getattr(L, name)
@@ -112,6 +114,8 @@ def lib():
         f.restype = C.c_int
     L.ipkv_block_bytes.argtypes = [C.POINTER(AttnShape)]
     L.ipkv_block_bytes.restype = C.c_int64
+    L.ipkv_noalloc_scratch_limit.argtypes = []
+    L.ipkv_noalloc_scratch_limit.restype = C.c_size_t
     L.ipkv_status_str.argtypes = [C.c_int]
     L.ipkv_status_str.restype = C.c_char_p
     L.ipkv_last_error.argtypes = [vp]
@@ -307,6 +311,30 @@ def ipkv_attend_runs(shape, runs_per_row, q, scratch, o_part, lse_part, kv_split
                                 _stream(stream))
     if rc != OK:
         raise IpkvError(rc, "ipkv_attend_runs")
+
+
+def _marshal_runs(runs_per_row):
+    flat, start = [], [0]
+    for row in runs_per_row:
+        for ptr, n in row:
+            flat.append(Run(_ptr(ptr), int(n)))
+        start.append(len(flat))
+    return (Run * max(1, len(flat)))(*flat), (C.c_int32 * len(start))(*start)
+
+
+def ipkv_noalloc_scratch_limit():
+    return int(lib().ipkv_noalloc_scratch_limit())
+
+
+def ipkv_attend_runs_noalloc(shape, runs_per_row, q, o_part, lse_part, kv_splits=0, status=None, stream=None):
+    """ipkv_attend_runs for callers that cannot allocate device memory at the call site: same arguments minus the
+    scratch buffer, which is a fixed 16 MiB array inside the library (shared by all calls on a device; calls that
+    overlap on the GPU race on it).  Raises IpkvError(ERANGE) when the call would need more than that."""
+    runs, starts = _marshal_runs(runs_per_row)
+    rc = lib().ipkv_attend_runs_noalloc(C.byref(shape), len(runs_per_row), runs, starts, _ptr(q), kv_splits,
+                                        _ptr(o_part), _ptr(lse_part), _ptr(status), _stream(stream))
+    if rc != OK:
+        raise IpkvError(rc, "ipkv_attend_runs_noalloc")
 
 
 def ipkv_pack_blocks(shape, layout, k, v, n_tokens, dst, stream=None):

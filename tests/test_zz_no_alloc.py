@@ -1,0 +1,78 @@
+"""The allocation-free attention entry point against the ordinary one.
+
+ipkv_attend_runs_noalloc is for callers that cannot allocate device memory where they call attention (a server
+whose pool owns all memory, a latency-critical loop, a plug-in that may not allocate): its scratch is a fixed
+array inside the library. This file is collected last, so a run that stops at the first failure has already
+run every other test. It must pass on its own in a fresh process and after the rest of the suite.
+"""
+import numpy as np
+import pytest
+
+from paper_2609_14507_b200 import binding, synth
+from tests.gpu_util import pack_run, shape_of
+
+pytestmark = pytest.mark.gpu
+torch = pytest.importorskip("torch")
+
+
+def _case(seed, rows, hq=32, hkv=4, d=128, bt=64):
+    shape = shape_of(binding.GQA, hq, hkv, d, d, bt)
+    rng = np.random.default_rng(seed)
+    q = synth.bits_to_torch(synth.normal_bf16(rng, (len(rows), hq, d)), "cuda:0")
+    bufs, runs = [], []
+    for row in rows:
+        rr = []
+        for n in row:
+            buf = pack_run(shape, synth.normal_bf16(rng, (n, hkv, d)), synth.normal_bf16(rng, (n, hkv, d)))
+            bufs.append(buf); rr.append((buf, n))
+        runs.append(rr)
+    return shape, q, runs, bufs
+
+
+def _both(shape, q, runs, kv_splits):
+    n_rows = len(runs)
+    total = sum(n for row in runs for _, n in row)
+    n_runs = sum(len(row) for row in runs)
+    scratch = torch.zeros(binding.ipkv_attend_scratch_bytes(shape, n_rows, n_runs, total, kv_splits), dtype=torch.uint8, device="cuda:0")
+    outs = []
+    for use_static in (False, True):
+        o = torch.full((n_rows, shape.n_q_heads, shape.dim_v), float("nan"), device="cuda:0")
+        lse = torch.full((n_rows, shape.n_q_heads), float("nan"), device="cuda:0")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda:0")
+        if use_static:
+            binding.ipkv_attend_runs_noalloc(shape, runs, q, o, lse, kv_splits, status)
+        else:
+            binding.ipkv_attend_runs(shape, runs, q, scratch, o, lse, kv_splits, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        outs.append((o.cpu().numpy(), lse.cpu().numpy()))
+    return outs
+
+
+def test_noalloc_matches_scratch_variant_on_two_calls_in_a_row():
+    # Two different problems back to back: the second call finds the first call's tables and partials in the
+    # shared array and must not be affected by them.
+    for seed, rows, splits in [(71, [[3000, 130], [64], []], 0), (72, [[900], [2500, 1], [77]], 4)]:
+        shape, q, runs, _keep = _case(seed, rows)
+        (o_ref, l_ref), (o, l) = _both(shape, q, runs, splits)
+        assert np.array_equal(np.isneginf(l), np.isneginf(l_ref))
+        fin = np.isfinite(l_ref)
+        np.testing.assert_allclose(o, o_ref, atol=2e-3, rtol=0)
+        np.testing.assert_allclose(l[fin], l_ref[fin], atol=1e-3, rtol=0)
+        # same kernels, same plan: in fact identical
+        np.testing.assert_array_equal(o, o_ref)
+
+
+def test_noalloc_rejects_problems_beyond_its_array():
+    shape = shape_of(binding.GQA, 32, 4, 128, 128, 64)
+    limit = binding.ipkv_noalloc_scratch_limit()
+    assert limit == 16 << 20
+    # many splits of a large batch need more partial storage than the array holds; nothing is launched
+    rows = [[(1 << 20, 70000)] for _ in range(64)]            # pointers are never dereferenced: the call is refused first
+    assert binding.ipkv_attend_scratch_bytes(shape, 64, 64, 64 * 70000, 64) > limit
+    q = torch.zeros((64, 32, 128), dtype=torch.bfloat16, device="cuda:0")
+    o = torch.zeros((64, 32, 128), device="cuda:0"); lse = torch.zeros((64, 32), device="cuda:0")
+    with pytest.raises(binding.IpkvError) as e:
+        binding.ipkv_attend_runs_noalloc(shape, rows, q, o, lse, kv_splits=64)
+    assert e.value.status == 3
+    torch.cuda.synchronize()
