@@ -43,6 +43,10 @@ WORKLOADS = {
                                            ctx=32768, share=(1, 4), cfg_id=2),
     "qwen3-2layers-bs16-32k-cpu0": dict(shape=synth.Shape("qwen3-2l", "gqa", 2, 32, 4, 128, 128, 128 ** -0.5), batch=16,
                                         ctx=32768, share=(0, 1), cfg_id=3),
+    # BASELINE config 4: DeepSeek-V2-Lite-shaped MLA decode, 27 layers, batch 8, 128K context, CPU share 40 %
+    "deepseek-v2-lite-mla-bs8-128k-cpu40": dict(shape=synth.DSV2_LITE, batch=8, ctx=131072, share=(2, 5), cfg_id=4),
+    "deepseek-v2-lite-mla-2layers-bs8-128k-cpu40": dict(shape=synth.Shape("dsv2-2l", "mla", 2, 16, 1, 576, 512, 192 ** -0.5),
+                                                        batch=8, ctx=131072, share=(2, 5), cfg_id=4),
     # BASELINE config 1 (single layer, batch 1, 4K): latency-bound, for quick checks
     "small-gqa-bs1-4k-cpu50": dict(shape=synth.SMALL_GQA, batch=1, ctx=4096, share=(1, 2), cfg_id=1),
 }

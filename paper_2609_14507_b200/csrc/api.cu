@@ -55,7 +55,7 @@ size_t partial_bytes(size_t n_items, int Hq, int dv) {
 int64_t max_items_bound(int n_rows, int n_runs, int64_t total_tokens, int kv_splits) {
     const int64_t tiles = (total_tokens + kTileTokens - 1) / kTileTokens + n_runs;
     if (kv_splits > 0) return int64_t(n_runs) * (kv_splits + 1) + n_rows;
-    return std::max<int64_t>(int64_t(kSmCount) * kCtasPerSm, tiles / 8) + n_runs + n_rows;
+    return tiles + n_runs + n_rows;   // the planner never makes items smaller than one tile
 }
 
 bool shape_ok(int kind, int Hq, int Hkv, int dqk, int dv, int bt, std::string* why) {
@@ -343,8 +343,10 @@ void fill_launch(AttnLaunch* a, int kind, int Hq, int Hkv, int dqk, int dv, int 
     a->part_lse = reinterpret_cast<float*>(partials + align_up(plan.items.size() * size_t(Hq) * dv * sizeof(float), 256));
 }
 
+int ctas_per_sm(int kind) { return kind == IPKV_MLA ? 1 : 2; }
+
 int heads_per_tile(int kind, int Hq, int Hkv) {
-    if (kind == IPKV_MLA) return 1;
+    if (kind == IPKV_MLA) return (Hq + 15) / 16;
     const int G = Hq / Hkv;
     return Hkv * ((G + 15) / 16);
 }
@@ -354,7 +356,7 @@ ipkv_status run_group(ipkv* h, const std::vector<std::vector<PlanSeg>>& rows, co
                       const void* q, int kv_splits, bool fold, float* out_o, float* out_lse, cudaStream_t s) {
     const ipkv_config& c = h->cfg;
     Plan plan;
-    build_plan(rows, heads_per_tile(c.kind, c.n_q_heads, c.n_kv_heads), kv_splits, &plan);
+    build_plan(rows, heads_per_tile(c.kind, c.n_q_heads, c.n_kv_heads), kv_splits, ctas_per_sm(c.kind), &plan);
     ipkv_status rc = ensure_scratch(h, partial_bytes(plan.items.size(), c.n_q_heads, c.dim_v));
     if (rc != IPKV_OK) return rc;
     const char* table = nullptr;
@@ -941,7 +943,7 @@ ipkv_status ipkv_attend_runs(const ipkv_attn_shape* sh, int32_t n_rows,
         }
     }
     Plan plan;
-    build_plan(rows, heads_per_tile(sh->kind, sh->n_q_heads, sh->n_kv_heads), kv_splits, &plan);
+    build_plan(rows, heads_per_tile(sh->kind, sh->n_q_heads, sh->n_kv_heads), kv_splits, ctas_per_sm(sh->kind), &plan);
     const size_t table = align_up(plan.table_bytes(), 256);
     if (table + 256 + partial_bytes(plan.items.size(), sh->n_q_heads, sh->dim_v) > scratch_bytes) return IPKV_ENOMEM;
     cudaStream_t s = static_cast<cudaStream_t>(stream);

@@ -1,11 +1,322 @@
-// Compressed-latent (MLA) variant of the GPU-side decode attention. Placeholder until the kernel lands.
+// GPU-side decode attention over the GPU-resident share (Sec. 5.1), compressed-latent (MLA) variant:
+// every head of a sequence attends the same cached row [latent 512 | rope 64] per token with an absorbed
+// query of width 576, and the value is the row's first 512 columns (Sec. 6.1: the heads share one latent,
+// each latent is read from memory once).  The paper's kernel for this case is a CPU kernel; this one is
+// written for sm_100a.
+//
+// One CTA per (item, group of 16 query heads): a producer warp streams 64-token tiles (73 728 contiguous
+// bytes in the TILE block layout) into a 2-stage shared-memory ring with bulk asynchronous copies that
+// complete on mbarriers; the tile is read twice from shared memory — as K (ldmatrix) and as V
+// (ldmatrix.trans on the first eight 64-column panels) — and once from HBM.
+//
+// Eight consumer warps, three phases per tile:
+//   1. scores: warp (ds, th) multiplies the 16 query rows with d-slice ds (144 of the 576 columns) of
+//      token half th (32 tokens); the query fragments of its slice stay in registers for the whole CTA;
+//      partial scores go to shared memory.
+//   2. softmax: warp w owns query rows 2w, 2w+1: it sums the four d-slice partials, applies the scale,
+//      masks the ragged tail and updates the running max / sum of its rows (fp32, log2 domain); the
+//      weights are split p = p_hi + p_lo (two bf16) and written to shared memory with the rescale factor.
+//   3. output: warp w owns value columns [64w, 64w+64) (one panel): O = O*alpha + (P_hi + P_lo) V with
+//      fp32 accumulators in registers.
+// HBM traffic per KV token: 1152 bytes, read exactly once per group of 16 heads.
+#include <cuda_bf16.h>
+
 #include "kernels.h"
+#include "ptx.cuh"
 
 namespace ipkvi {
 
-cudaError_t launch_attend_mla(const AttnLaunch& a, cudaStream_t) {
+namespace {
+
+constexpr int kDqk = 576, kDv = 512;
+constexpr int kPanels = kDqk / 64;                 // 9
+constexpr int kConsumerWarps = 8;
+constexpr int kThreads = (kConsumerWarps + 1) * 32;
+constexpr int kStages = 2;
+constexpr int kStageBytes = kTileTokens * kDqk * 2;          // 73 728
+constexpr int kQPitch = kDqk * 2 + 16;                       // 1168
+constexpr int kSPitch = kTileTokens + 4;                     // floats
+constexpr int kPPitch = kTileTokens * 2 + 16;                // bytes (bf16 row of 64 tokens, padded)
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+constexpr int kOffQ = kStages * kStageBytes;                 // 147 456
+constexpr int kOffS = kOffQ + 16 * kQPitch;                  // partial scores [4][16][kSPitch] fp32
+constexpr int kOffPhi = kOffS + 4 * 16 * kSPitch * 4;
+constexpr int kOffPlo = kOffPhi + 16 * kPPitch;
+constexpr int kOffAlpha = kOffPlo + 16 * kPPitch;            // [16] fp32 rescale factors, then [16] m, [16] l
+constexpr int kOffBar = kOffAlpha + 3 * 16 * 4;
+constexpr int kSmemTotal = kOffBar + 2 * kStages * 8;
+
+struct MlaParams {
+    const __nv_bfloat16* q;
+    const char* bases[kMaxBases];
+    const Seg* segs;
+    const Item* items;
+    float* part_o;
+    float* part_lse;
+    uint32_t* status;
+    int Hq, n_hg;
+    int bt;
+    int64_t block_bytes;
+    float scale_log2;
+};
+
+__device__ __forceinline__ void consumer_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory"); }
+
+__global__ void __launch_bounds__(kThreads, 1) attn_mla_kernel(const MlaParams p) {
+    extern __shared__ unsigned char smem_dyn[];
+    unsigned char* smem = smem_dyn + ((1024u - (ptx::smem_addr(smem_dyn) & 1023u)) & 1023u);
+    const uint32_t s_base = ptx::smem_addr(smem);
+    const uint32_t s_q = s_base + kOffQ;
+    const uint32_t s_phi = s_base + kOffPhi, s_plo = s_base + kOffPlo;
+    const uint32_t s_full = s_base + kOffBar, s_empty = s_full + kStages * 8;
+    float* sp = reinterpret_cast<float*>(smem + kOffS);
+    float* s_alpha = reinterpret_cast<float*>(smem + kOffAlpha);
+    float* s_m = s_alpha + 16;
+    float* s_l = s_alpha + 32;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const Item item = p.items[blockIdx.x];
+    const Seg seg = p.segs[item.seg];
+    const int hg = blockIdx.y;
+    const int head0 = hg * 16;
+    const int n_heads = min(16, p.Hq - head0);
+
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            ptx::mbar_init(s_full + 8 * s, 1);
+            ptx::mbar_init(s_empty + 8 * s, kConsumerWarps);
+        }
+        ptx::mbar_fence_init();
+    }
+    for (int c = tid; c < 16 * (kDqk / 8); c += kThreads) {
+        const int r = c / (kDqk / 8), ch = c - r * (kDqk / 8);
+        uint4 val = make_uint4(0, 0, 0, 0);
+        if (r < n_heads) val = *reinterpret_cast<const uint4*>(p.q + (int64_t(item.row) * p.Hq + head0 + r) * kDqk + ch * 8);
+        *reinterpret_cast<uint4*>(smem + kOffQ + r * kQPitch + ch * 16) = val;
+    }
+    if (p.bt < kTileTokens) {
+        for (int c = tid; c < kStages * kStageBytes / 16; c += kThreads) reinterpret_cast<uint4*>(smem)[c] = make_uint4(0, 0, 0, 0);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+
+    const char* seg_base = p.bases[seg.base_id] + seg.off;
+    bool ok = true;
+
+    if (warp == kConsumerWarps) {
+        // ---------------- producer ----------------
+        if (lane == 0) {
+            for (int i = 0; i < item.ntiles; ++i) {
+                const int st = i % kStages;
+                if (i >= kStages && !ptx::mbar_wait(s_empty + 8 * st, ((i / kStages) - 1) & 1)) { ok = false; break; }
+                const int64_t t0 = int64_t(item.tile0 + i) * kTileTokens;
+                const uint32_t dst = s_base + st * kStageBytes;
+                const uint32_t bar = s_full + 8 * st;
+                if (p.bt >= kTileTokens) {
+                    const int64_t blk = t0 / p.bt;
+                    const int r0 = int(t0 - blk * p.bt);
+                    const char* src = seg_base + blk * p.block_bytes;
+                    ptx::mbar_expect_tx(bar, kStageBytes);
+                    if (p.bt == kTileTokens) {
+                        ptx::bulk_g2s(dst, src, kStageBytes, bar);
+                    } else {
+#pragma unroll
+                        for (int pn = 0; pn < kPanels; ++pn)
+                            ptx::bulk_g2s(dst + pn * 8192, src + int64_t(pn) * p.bt * 128 + int64_t(r0) * 128, 8192, bar);
+                    }
+                } else {
+                    const int nsub = kTileTokens / p.bt;
+                    const int64_t blk0 = t0 / p.bt;
+                    int live = 0;
+                    for (int j = 0; j < nsub; ++j) live += ((blk0 + j) * p.bt < seg.n_tokens);
+                    const uint32_t sub_bytes = uint32_t(p.bt) * 128;
+                    ptx::mbar_expect_tx(bar, uint32_t(live) * sub_bytes * kPanels);
+                    for (int j = 0; j < live; ++j) {
+                        const char* src = seg_base + (blk0 + j) * p.block_bytes;
+#pragma unroll
+                        for (int pn = 0; pn < kPanels; ++pn)
+                            ptx::bulk_g2s(dst + pn * 8192 + j * sub_bytes, src + int64_t(pn) * sub_bytes, sub_bytes, bar);
+                    }
+                }
+            }
+            const int first_pending = item.ntiles > kStages ? item.ntiles - kStages : 0;
+            for (int i = first_pending; i < item.ntiles; ++i)
+                if (!ptx::mbar_wait(s_full + 8 * (i % kStages), (i / kStages) & 1)) ok = false;
+            if (!ok) atomicOr(p.status, 1u);
+        }
+        return;      // the consumers synchronise among themselves on a named barrier
+    }
+
+    // ---------------- consumers ----------------
+    const int ds = warp & 3, th = warp >> 2;
+    const int mi = lane >> 3, r8 = lane & 7;
+    uint32_t qa[9][4];
+#pragma unroll
+    for (int ks = 0; ks < 9; ++ks) {
+        const int row = (mi & 1) * 8 + r8, chunk = ds * 18 + ks * 2 + (mi >> 1);
+        ptx::ldmatrix_x4(s_q + row * kQPitch + chunk * 16, qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3]);
+    }
+    float o[8][4];
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt) { o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f; }
+    // phase-2 ownership: this lane works on query row `srow`, tokens [stok, stok + 4) of every tile
+    const int srow = 2 * warp + (lane >> 4), stok = (lane & 15) * 4;
+    float m_run = -INFINITY, l_run = 0.f;
+
+    for (int i = 0; i < item.ntiles; ++i) {
+        const int st = i % kStages;
+        if (ok && !ptx::mbar_wait(s_full + 8 * st, (i / kStages) & 1)) ok = false;   // after a timeout: no more waits, but keep the barriers below matched
+        const int64_t t0 = int64_t(item.tile0 + i) * kTileTokens;
+        const int64_t left = int64_t(seg.n_tokens) - t0;
+        const int n_valid = left < kTileTokens ? int(left) : kTileTokens;
+        const uint32_t kb = s_base + st * kStageBytes;
+
+        // ---- phase 1: partial scores of d-slice ds for tokens [32 th, 32 th + 32) ----
+        {
+            float s[4][4];
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) { s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f; }
+#pragma unroll
+            for (int ks = 0; ks < 9; ++ks) {
+                const int chunk = ds * 18 + ks * 2 + (mi & 1);
+                const uint32_t col = (chunk >> 3) * 8192 + (((chunk & 7) ^ r8) << 4);
+#pragma unroll
+                for (int tg = 0; tg < 2; ++tg) {
+                    const int tok = th * 32 + tg * 16 + (mi >> 1) * 8 + r8;
+                    uint32_t b0, b1, b2, b3;
+                    ptx::ldmatrix_x4(kb + col + tok * 128, b0, b1, b2, b3);
+                    ptx::mma_bf16(s[2 * tg], qa[ks], b0, b1);
+                    ptx::mma_bf16(s[2 * tg + 1], qa[ks], b2, b3);
+                }
+            }
+            float* dst = sp + ds * 16 * kSPitch;
+            const int r0 = lane >> 2, c0 = th * 32 + 2 * (lane & 3);
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) {
+                *reinterpret_cast<float2*>(dst + r0 * kSPitch + c0 + nt * 8) = make_float2(s[nt][0], s[nt][1]);
+                *reinterpret_cast<float2*>(dst + (r0 + 8) * kSPitch + c0 + nt * 8) = make_float2(s[nt][2], s[nt][3]);
+            }
+        }
+        consumer_barrier();
+
+        // ---- phase 2: softmax bookkeeping for the rows this warp owns ----
+        {
+            float4 a = *reinterpret_cast<const float4*>(sp + srow * kSPitch + stok);
+#pragma unroll
+            for (int d = 1; d < 4; ++d) {
+                const float4 b = *reinterpret_cast<const float4*>(sp + (d * 16 + srow) * kSPitch + stok);
+                a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+            }
+            float sv[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) sv[j] = (stok + j < n_valid) ? sv[j] * p.scale_log2 : -INFINITY;
+            float mx = fmaxf(fmaxf(sv[0], sv[1]), fmaxf(sv[2], sv[3]));
+#pragma unroll
+            for (int d = 1; d < 16; d <<= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, d));
+            const float mn = fmaxf(m_run, mx);
+            const float ms = (mn == -INFINITY) ? 0.f : mn;
+            const float alpha = ptx::ex2(m_run - ms);
+            m_run = mn;
+            float pr[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) pr[j] = ptx::ex2(sv[j] - ms);
+            l_run = l_run * alpha + (pr[0] + pr[1] + pr[2] + pr[3]);
+            const uint32_t h0 = ptx::pack_bf16(pr[0], pr[1]), h1 = ptx::pack_bf16(pr[2], pr[3]);
+            const uint32_t l0 = ptx::pack_bf16(pr[0] - ptx::bf16_lo(h0), pr[1] - ptx::bf16_hi(h0));
+            const uint32_t l1 = ptx::pack_bf16(pr[2] - ptx::bf16_lo(h1), pr[3] - ptx::bf16_hi(h1));
+            *reinterpret_cast<uint2*>(smem + kOffPhi + srow * kPPitch + stok * 2) = make_uint2(h0, h1);
+            *reinterpret_cast<uint2*>(smem + kOffPlo + srow * kPPitch + stok * 2) = make_uint2(l0, l1);
+            if ((lane & 15) == 0) s_alpha[srow] = alpha;
+        }
+        consumer_barrier();
+
+        // ---- phase 3: O[:, 64 warp .. 64 warp + 64) = O * alpha + (P_hi + P_lo) V ----
+        {
+            const int r0 = lane >> 2;
+            const float a0 = s_alpha[r0], a1 = s_alpha[r0 + 8];
+            if (__any_sync(0xffffffffu, (a0 != 1.f) | (a1 != 1.f))) {
+#pragma unroll
+                for (int nt = 0; nt < 8; ++nt) { o[nt][0] *= a0; o[nt][1] *= a0; o[nt][2] *= a1; o[nt][3] *= a1; }
+            }
+            const uint32_t vb = kb + warp * 8192;
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+                uint32_t ph[4], pl[4];
+                const uint32_t poff = ((mi & 1) * 8 + r8) * kPPitch + (kk * 2 + (mi >> 1)) * 16;
+                ptx::ldmatrix_x4(s_phi + poff, ph[0], ph[1], ph[2], ph[3]);
+                ptx::ldmatrix_x4(s_plo + poff, pl[0], pl[1], pl[2], pl[3]);
+                const int tok = kk * 16 + (mi & 1) * 8 + r8;
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj) {
+                    const int chunk = 2 * jj + (mi >> 1);
+                    uint32_t b0, b1, b2, b3;
+                    ptx::ldmatrix_x4_trans(vb + tok * 128 + ((chunk ^ r8) << 4), b0, b1, b2, b3);
+                    ptx::mma_bf16(o[2 * jj], ph, b0, b1);
+                    ptx::mma_bf16(o[2 * jj + 1], ph, b2, b3);
+                    ptx::mma_bf16(o[2 * jj], pl, b0, b1);
+                    ptx::mma_bf16(o[2 * jj + 1], pl, b2, b3);
+                }
+            }
+        }
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(s_empty + 8 * st);
+    }
+    if (!ok && lane == 0) atomicOr(p.status, 1u);
+
+    // final normalisation: the row owners publish m and l, every warp scales its columns
+#pragma unroll
+    for (int d = 1; d < 16; d <<= 1) l_run += __shfl_xor_sync(0xffffffffu, l_run, d);
+    if ((lane & 15) == 0) { s_m[srow] = m_run; s_l[srow] = l_run; }
+    consumer_barrier();
+    {
+        const int r0 = lane >> 2, c0 = warp * 64 + 2 * (lane & 3);
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            const int row = r0 + half * 8;
+            if (row < n_heads) {
+                const float L = s_l[row];
+                const float inv = (L > 0.f) ? 1.f / L : 0.f;
+                float* dst = p.part_o + (int64_t(blockIdx.x) * p.Hq + head0 + row) * kDv + c0;
+#pragma unroll
+                for (int nt = 0; nt < 8; ++nt)
+                    *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(o[nt][2 * half] * inv, o[nt][2 * half + 1] * inv);
+            }
+        }
+        if (warp == 0 && lane < n_heads) {
+            const float M = s_m[lane], L = s_l[lane];
+            p.part_lse[int64_t(blockIdx.x) * p.Hq + head0 + lane] = (M == -INFINITY) ? -INFINITY : (M + log2f(L)) * kLn2;
+        }
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_attend_mla(const AttnLaunch& a, cudaStream_t s) {
     if (a.n_items <= 0) return cudaSuccess;
-    return cudaErrorNotSupported;
+    if (a.dim_qk != kDqk || a.dim_v != kDv || a.n_kv_heads != 1) return cudaErrorInvalidValue;
+    MlaParams p;
+    p.q = static_cast<const __nv_bfloat16*>(a.q);
+    for (int i = 0; i < kMaxBases; ++i) p.bases[i] = a.bases[i];
+    p.segs = a.segs; p.items = a.items;
+    p.part_o = a.part_o; p.part_lse = a.part_lse; p.status = a.status;
+    p.Hq = a.n_q_heads; p.n_hg = (a.n_q_heads + 15) / 16;
+    p.bt = a.bt;
+    p.block_bytes = int64_t(a.bt) * kDqk * 2;
+    p.scale_log2 = a.scale * kLog2e;
+    const int smem = kSmemTotal + 1024;
+    static bool configured[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64 || !configured[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(attn_mla_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64) configured[dev] = true;
+    }
+    dim3 grid(a.n_items, p.n_hg);
+    attn_mla_kernel<<<grid, kThreads, smem, s>>>(p);
+    return cudaGetLastError();
 }
 
 }  // namespace ipkvi

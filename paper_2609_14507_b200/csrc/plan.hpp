@@ -13,7 +13,6 @@
 namespace ipkvi {
 
 constexpr int kSmCount = 148;
-constexpr int kCtasPerSm = 2;
 constexpr int kTargetTilesPerItem = 16;
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -39,28 +38,53 @@ struct Plan {
     }
 };
 
-inline int tiles_per_item(int64_t total_tiles, int64_t max_row_tiles, int heads_per_tile, int kv_splits) {
+// Number of pieces a run of `nt` tiles is cut into when items hold at most `per` tiles, and the largest piece.
+inline int64_t pieces_of(int64_t nt, int64_t per) { return (nt + per - 1) / per; }
+
+// Tiles per item. With kv_splits > 0 the longest row is cut into that many pieces. Otherwise the size is
+// searched so that the grid (items x heads_per_tile CTAs, ctas_per_sm resident per SM) runs in as few
+// equally loaded waves as possible: cost = waves x (largest piece + a fixed per-CTA overhead in tile units).
+inline int tiles_per_item(const std::vector<int64_t>& seg_tiles, int64_t max_row_tiles, int heads_per_tile,
+                          int kv_splits, int ctas_per_sm) {
     if (kv_splits > 0) return int(std::max<int64_t>(1, (max_row_tiles + kv_splits - 1) / kv_splits));
-    // Fill the machine in whole waves: the grid is (items x heads_per_tile) CTAs, kCtasPerSm resident per SM.
-    const int64_t slots = int64_t(kSmCount) * kCtasPerSm;
-    const int64_t work = total_tiles * heads_per_tile;
-    const int64_t waves = std::max<int64_t>(1, (work + slots * kTargetTilesPerItem - 1) / (slots * kTargetTilesPerItem));
-    const int64_t per = (work + slots * waves - 1) / (slots * waves);
-    return int(std::max<int64_t>(1, per));
+    const int64_t slots = int64_t(kSmCount) * ctas_per_sm;
+    int64_t longest = 1;
+    for (int64_t nt : seg_tiles) longest = std::max(longest, nt);
+    int best = 1;
+    double best_cost = 1e300;
+    const int64_t hi = std::min<int64_t>(longest, 4 * kTargetTilesPerItem);
+    for (int64_t per = 1; per <= hi; ++per) {
+        int64_t items = 0, biggest = 0;
+        for (int64_t nt : seg_tiles) {
+            const int64_t pc = pieces_of(nt, per);
+            items += pc;
+            biggest = std::max(biggest, (nt + pc - 1) / pc);
+        }
+        const int64_t waves = (items * heads_per_tile + slots - 1) / slots;
+        const double cost = double(waves) * (double(biggest) + 2.0);     // ~2 tiles of fixed cost per CTA
+        if (cost < best_cost - 1e-9 || (cost < best_cost + 1e-9 && per > best)) { best_cost = cost; best = int(per); }
+    }
+    return best;
 }
 
 // rows[r] = segments of row r. Produces the device tables' host image.
-inline void build_plan(const std::vector<std::vector<PlanSeg>>& rows, int heads_per_tile, int kv_splits, Plan* plan) {
+inline void build_plan(const std::vector<std::vector<PlanSeg>>& rows, int heads_per_tile, int kv_splits, int ctas_per_sm, Plan* plan) {
     plan->segs.clear(); plan->items.clear(); plan->row_item_start.clear();
-    int64_t total_tiles = 0, max_row_tiles = 0, total_tokens = 0;
+    int64_t max_row_tiles = 0, total_tokens = 0;
+    std::vector<int64_t> seg_tiles;
     for (const auto& row : rows) {
         int64_t rt = 0;
-        for (const auto& s : row) { rt += (s.n_tokens + kTileTokens - 1) / kTileTokens; total_tokens += s.n_tokens; }
-        total_tiles += rt;
+        for (const auto& s : row) {
+            if (s.n_tokens <= 0) continue;
+            const int64_t nt = (s.n_tokens + kTileTokens - 1) / kTileTokens;
+            seg_tiles.push_back(nt);
+            rt += nt;
+            total_tokens += s.n_tokens;
+        }
         max_row_tiles = std::max(max_row_tiles, rt);
     }
     plan->total_tokens = total_tokens;
-    const int per = tiles_per_item(total_tiles, max_row_tiles, heads_per_tile, kv_splits);
+    const int per = tiles_per_item(seg_tiles, max_row_tiles, heads_per_tile, kv_splits, ctas_per_sm);
     for (size_t r = 0; r < rows.size(); ++r) {
         plan->row_item_start.push_back(int32_t(plan->items.size()));
         for (const auto& s : rows[r]) {

@@ -51,7 +51,7 @@ int shim_plan(int n_rows, const int32_t* row_start, const int64_t* seg_tokens, i
     for (int r = 0; r < n_rows; ++r)
         for (int k = row_start[r]; k < row_start[r + 1]; ++k) rows[r].push_back(PlanSeg{0, int64_t(k) * 4096, seg_tokens[k]});
     Plan plan;
-    build_plan(rows, heads_per_tile, kv_splits, &plan);
+    build_plan(rows, heads_per_tile, kv_splits, 2, &plan);
     const int n = int(plan.items.size());
     if (n > cap_items) return -n;
     for (int i = 0; i < n; ++i) {

@@ -240,3 +240,49 @@ def test_explicit_partial_flush_and_errors():
         assert e.value.status == 1
         with pytest.raises(binding.IpkvError):
             cache.locate(0, 1, 99)
+
+
+@pytest.mark.parametrize("resident", [2048, 0, 192])
+def test_mla_cache_decode_steps(resident):
+    """Compressed-latent cache through prefill, decode appends with evictions, attention (resident, fully
+    streamed, and a small ring) and merge."""
+    sh = synth.Shape("tiny-mla", "mla", 1, 16, 1, 576, 512, 192 ** -0.5)
+    rng = np.random.default_rng(70)
+    scale = float(np.float32(sh.scale))
+    seqs = [1, 0]
+    lens = {1: 321, 0: 64}
+    with make_cache(sh, 1, 2, block_tokens=64, window_tokens=64, chunk_tokens=128, n_slots=2, max_u_tokens_per_seq=700,
+                    max_p_tokens_per_seq=700, resident_tokens_per_seq=resident, share_num=2, share_den=5) as cache:
+        refs = {}
+        for s in seqs:
+            r = RefSeq(sh, 64, 64, 2, 5)
+            k, _ = synth.host_kv(sh, lens[s], seed=7000 + s)
+            cache.append_bulk(0, s, synth.bits_to_torch(k, DEV), None, lens[s], 1, 4)
+            r.bulk(k, None, 1, 4)
+            refs[s] = r
+        for step in range(200):
+            k = synth.normal_bf16(rng, (2, 1, 576))
+            cache.append(0, seqs, synth.bits_to_torch(k, DEV), None)
+            for i, s in enumerate(seqs):
+                refs[s].append(k[i:i + 1], None)
+            if step % 37 == 0 or step == 199:
+                q = synth.normal_bf16(rng, (2, 16, 576))
+                o = torch.zeros((2, 16, 512), device=DEV); lse = torch.zeros((2, 16), device=DEV)
+                cache.attend_gpu(0, seqs, synth.bits_to_torch(q, DEV), o, lse)
+                torch.cuda.synchronize()
+                parts = [refs[s].attend(q[i], "gpu", scale) for i, s in enumerate(seqs)]
+                check_partial(o.cpu().numpy(), lse.cpu().numpy(), np.stack([p[0] for p in parts]), np.stack([p[1] for p in parts]),
+                              f"mla step {step}")
+                cpu = [refs[s].attend(q[i], "cpu", scale) for i, s in enumerate(seqs)]
+                oc = torch.from_numpy(np.stack([p[0] for p in cpu]).astype(np.float32)).to(DEV)
+                lc = torch.from_numpy(np.stack([p[1] for p in cpu]).astype(np.float32)).to(DEV)
+                out = torch.zeros((32, 512), device=DEV); out_lse = torch.zeros(32, device=DEV)
+                cache.merge(32, 512, [o.view(32, 512), oc.view(32, 512)], [lse.view(-1), lc.view(-1)], out, out_lse)
+                torch.cuda.synchronize()
+                full = [refs[s].attend(q[i], "all", scale) for i, s in enumerate(seqs)]
+                check_partial(out.cpu().numpy().reshape(2, 16, 512), out_lse.cpu().numpy().reshape(2, 16),
+                              np.stack([p[0] for p in full]), np.stack([p[1] for p in full]), f"mla merged step {step}")
+        for s in seqs:
+            check_routing(cache, 0, s, refs[s], sample=range(0, len(refs[s].route), 5))
+            check_contents(cache, 0, s, refs[s], range(0, len(refs[s].route), 11))
+        assert cache.get_stats()["device_status"] == 0

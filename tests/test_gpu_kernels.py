@@ -119,3 +119,66 @@ def test_merge_matches_oracle(n_parts, dv, bf16_out):
     gl = lse.cpu().numpy().astype(np.float64)
     assert np.array_equal(np.isneginf(gl), np.isneginf(l_ref))
     np.testing.assert_allclose(gl[np.isfinite(l_ref)], l_ref[np.isfinite(l_ref)], atol=1e-5, rtol=1e-6)
+
+
+MLA_CASES = [
+    # (Hq, bt, run lengths per row, kv_splits)
+    (16, 64, [[4096 + 1]], 0),
+    (16, 64, [[700, 33], [64], [1]], 0),
+    (16, 64, [[2049], [], [517, 255]], 3),
+    (32, 64, [[500]], 0),                    # two groups of 16 heads
+    (5, 64, [[300, 10]], 0),                 # fewer than 16 heads
+    (16, 16, [[1000, 17]], 0),
+    (16, 32, [[70]], 0),
+    (16, 128, [[1000, 257]], 2),
+]
+
+
+@pytest.mark.parametrize("hq,bt,rows,kv_splits", MLA_CASES)
+def test_attend_runs_mla_matches_oracle(hq, bt, rows, kv_splits):
+    """Compressed-latent kind: cached row = [latent 512 | rope 64], V = the row's first 512 columns."""
+    scale = 192 ** -0.5
+    shape = shape_of(binding.MLA, hq, 1, 576, 512, bt, scale)
+    rng = np.random.default_rng(45)
+    n_rows = len(rows)
+    q = synth.normal_bf16(rng, (n_rows, hq, 576))
+    bufs, runs, rows_kv = [], [], []
+    for row in rows:
+        ks, rr = [], []
+        for n in row:
+            k = synth.normal_bf16(rng, (n, 1, 576))
+            buf = pack_run(shape, k, None)
+            bufs.append(buf); rr.append((buf, n)); ks.append(k)
+        runs.append(rr)
+        rows_kv.append((np.concatenate(ks) if ks else np.zeros((0, 1, 576), np.uint16), None))
+    total = sum(sum(r) for r in rows)
+    n_runs = sum(len(r) for r in rows)
+    scratch = torch.zeros(binding.ipkv_attend_scratch_bytes(shape, n_rows, n_runs, total, kv_splits), dtype=torch.uint8, device="cuda:0")
+    o = torch.full((n_rows, hq, 512), float("nan"), device="cuda:0")
+    lse = torch.full((n_rows, hq), float("nan"), device="cuda:0")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda:0")
+    binding.ipkv_attend_runs(shape, runs, synth.bits_to_torch(q, "cuda:0"), scratch, o, lse, kv_splits, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    o_ref, lse_ref = oracle_rows(q, rows_kv, float(np.float32(scale)), dv_alias=512)
+    check_partial(o.cpu().numpy(), lse.cpu().numpy(), o_ref, lse_ref, f"mla {hq} heads bt{bt}")
+
+
+def test_attend_runs_mla_peaked_softmax():
+    hq, bt, n = 16, 64, 333
+    scale = 192 ** -0.5
+    shape = shape_of(binding.MLA, hq, 1, 576, 512, bt, scale)
+    rng = np.random.default_rng(46)
+    q = synth.normal_bf16(rng, (1, hq, 576))
+    k = synth.f32_to_bf16_bits(rng.standard_normal((n, 1, 576)).astype(np.float32) * 0.05)
+    qf = synth.bf16_bits_to_f32(q[0])
+    k[100, 0] = synth.f32_to_bf16_bits(3.0 * np.sign(qf.sum(axis=0)))
+    k[7, 0] = synth.f32_to_bf16_bits(rng.standard_normal(576).astype(np.float32))
+    buf = pack_run(shape, k, None)
+    scratch = torch.zeros(binding.ipkv_attend_scratch_bytes(shape, 1, 1, n, 0), dtype=torch.uint8, device="cuda:0")
+    o = torch.zeros((1, hq, 512), device="cuda:0"); lse = torch.zeros((1, hq), device="cuda:0")
+    binding.ipkv_attend_runs(shape, [[(buf, n)]], synth.bits_to_torch(q, "cuda:0"), scratch, o, lse)
+    torch.cuda.synchronize()
+    o_ref, lse_ref = oracle_rows(q, [(k, None)], float(np.float32(scale)), dv_alias=512)
+    assert np.abs(o_ref).max() > 0.5                       # O of order one: the absolute tolerance binds
+    check_partial(o.cpu().numpy(), lse.cpu().numpy(), o_ref, lse_ref, "mla peaked")

@@ -91,8 +91,9 @@ def test_plan_fills_the_machine_in_whole_waves():
     # Qwen3-shaped step: 16 rows x 32769 tokens, 4 KV heads -> CTAs = items * 4 close to a multiple of 296
     p = host_shim.plan([[32768 - 256, 257]] * 16, 4)
     ctas = len(p["row"]) * 4
-    assert 296 * 4 <= ctas <= 296 * 8
-    assert p["ntiles"].max() <= 32
+    waves = -(-ctas // 296)
+    assert 3 <= waves <= 10 and ctas / (waves * 296) >= 0.9      # the last wave is nearly full
+    assert p["ntiles"].max() <= 64
 
 
 def test_layout_arithmetic_matches_header_formula():
