@@ -53,6 +53,61 @@ WORKLOADS = {
 DEFAULT_WORKLOAD = "mixtral-8x7b-bs16-32k-cpu25"
 BLOCK, WINDOW = 64, 256
 
+# BASELINE config 5: Qwen3 shape, batch 64, ragged context lengths uniform in [8192, 24576] (about 1M tokens in all),
+# CPU share swept 0 .. 90 %. 16 of the 48 layers are kept (every layer's launch is identical; 48 layers at share 0
+# with per-sequence rings sized for the longest sequence would not fit 180 GB).
+for _pct in range(0, 100, 10):
+    WORKLOADS[f"qwen3-ragged-bs64-1m-16layers-cpu{_pct}"] = dict(
+        shape=synth.Shape("qwen3-16l", "gqa", 16, 32, 4, 128, 128, 128 ** -0.5), batch=64, ctx=24576, share=(_pct, 100),
+        cfg_id=5, lens=synth.ragged_lengths(5, 64, 8192, 24576))
+WORKLOADS["qwen3-ragged-bs64-1m-2layers-cpu30"] = dict(
+    shape=synth.Shape("qwen3-2l", "gqa", 2, 32, 4, 128, 128, 128 ** -0.5), batch=64, ctx=24576, share=(3, 10), cfg_id=5,
+    lens=synth.ragged_lengths(5, 64, 8192, 24576))
+
+
+def seq_lens(wl):
+    """Context length of every sequence of the batch."""
+    return [int(x) for x in wl["lens"]] if "lens" in wl else [wl["ctx"]] * wl["batch"]
+
+
+def cpu_tokens(n, num0, den0):
+    """Prefill tokens the CPU side takes: whole blocks, floored (the library's and the oracle's rule)."""
+    return BLOCK * ((n // BLOCK) * num0 // den0)
+
+
+def kv_seed(wl, layer, seq, rank=0):
+    return 1000 * wl["cfg_id"] + layer * wl["batch"] + seq + 100000 * rank
+
+
+def make_cache(wl, device_index, decode_steps):
+    """The cache of a workload as the benchmark times it: GPU-side share HBM-resident, host copies of U and P off."""
+    from paper_2609_14507_b200 import binding
+    sh = wl["shape"]
+    num0, den0 = wl["share"]
+    longest = max(seq_lens(wl))
+    grow = WINDOW * (decode_steps // WINDOW + 2)
+    p_cap = longest - cpu_tokens(longest, num0, den0) + grow if num0 < den0 else grow
+    p_cap = max(p_cap, max(n - cpu_tokens(n, num0, den0) for n in seq_lens(wl)) + grow)
+    kind = binding.MLA if sh.kind == "mla" else binding.GQA
+    cfg = binding.make_config(kind, sh.n_layers, wl["batch"], sh.n_q_heads, sh.n_kv_heads, sh.dim_qk, sh.dim_v,
+                              block_tokens=BLOCK, window_tokens=WINDOW, chunk_tokens=512, n_slots=2,
+                              max_u_tokens_per_seq=longest + grow, max_p_tokens_per_seq=p_cap, resident_tokens_per_seq=p_cap,
+                              softmax_scale=sh.scale, share_num=num0, share_den=den0, device=device_index,
+                              flags=binding.FLAG_NO_HOST_U | binding.FLAG_NO_HOST_P)
+    return binding.Cache(cfg)
+
+
+def populate(cache, wl, dev, rank=0):
+    """Prefill every (layer, sequence) with seeded N(0,1) K/V, routed in one shot at the workload's share."""
+    import torch
+    sh = wl["shape"]
+    num0, den0 = wl["share"]
+    for layer in range(sh.n_layers):
+        for s, n in enumerate(seq_lens(wl)):
+            k, v = synth.device_kv(sh, n, kv_seed(wl, layer, s, rank), dev)
+            cache.append_bulk(layer, s, k, v, n, num0, den0)
+        torch.cuda.synchronize()
+
 
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -117,37 +172,39 @@ class ClockSampler:
 
 def oracle_sample(wl, seconds_target=15.0, threads=None):
     """Time the float64 oracle, as it stands, on a bounded sample of the workload: the GPU-side share of whole
-    sequences of layer 0 (all KV heads, all query heads), as many sequences as fit the time target."""
+    (layer, sequence) pairs (all KV heads, all query heads), as many pairs as fit the time target."""
     import torch
     from oracle import c_oracle
     sh = wl["shape"]
     num0, den0 = wl["share"]
-    n_cpu = BLOCK * ((wl["ctx"] // BLOCK) * num0 // den0)
+    lens = seq_lens(wl)
     if threads:
         c_oracle.set_threads(threads)
     dev = "cuda:0" if torch.cuda.is_available() else None
-    done_tokens, t_total, n_seq = 0, 0.0, 0
+    done_tokens, t_total, n_pairs = 0, 0.0, 0
     while True:
-        seed = 1000 * wl["cfg_id"] + n_seq
+        layer, s = divmod(n_pairs, wl["batch"])
+        n = lens[s]
+        seed = kv_seed(wl, layer, s)
         if dev:
-            kd, vd = synth.device_kv(sh, wl["ctx"], seed, dev)
+            kd, vd = synth.device_kv(sh, n, seed, dev)
             k, v = synth.torch_bits(kd), (synth.torch_bits(vd) if vd is not None else None)
             q = synth.torch_bits(synth.device_q(sh, 1, seed + 500000, dev))[0]
         else:
-            k, v = synth.host_kv(sh, wl["ctx"], seed)
+            k, v = synth.host_kv(sh, n, seed)
             q = synth.host_q(sh, 1, seed + 500000)[0]
-        idx = np.arange(n_cpu, wl["ctx"])
+        idx = np.arange(cpu_tokens(n, num0, den0), n)
         t0 = time.perf_counter()
         c_oracle.attend(q, k, sh.dim_v if v is None else v, idx, float(np.float32(sh.scale)))
         dt = time.perf_counter() - t0
         done_tokens += idx.size
         t_total += dt
-        n_seq += 1
-        if t_total >= seconds_target or n_seq >= sh.n_layers * wl["batch"]:
+        n_pairs += 1
+        if t_total >= seconds_target or n_pairs >= sh.n_layers * wl["batch"]:
             break
     return dict(value=done_tokens / t_total, unit=UNIT, cores=c_oracle.num_threads(), kind="oracle",
-                sample=f"{n_seq} of {sh.n_layers * wl['batch']} (layer, sequence) pairs, GPU-side share ({idx.size} tokens each), "
-                       f"all heads; {t_total:.1f} s of float64 C++ (OpenMP over query heads)")
+                sample=f"{n_pairs} of {sh.n_layers * wl['batch']} (layer, sequence) pairs, GPU-side share ({done_tokens} KV-tokens "
+                       f"in all), all heads; {t_total:.1f} s of float64 C++ (OpenMP over query heads)")
 
 
 def run_reference(args, wl, name):
@@ -165,7 +222,7 @@ def run_reference(args, wl, name):
     value = float(np.mean(per_step))
     info["value"] = value
     sh = wl["shape"]
-    n_tok = sh.n_layers * wl["batch"] * (wl["ctx"] - BLOCK * ((wl["ctx"] // BLOCK) * wl["share"][0] // wl["share"][1]) + 1)
+    n_tok = sh.n_layers * sum(n - cpu_tokens(n, *wl["share"]) + 1 for n in seq_lens(wl))
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * n_tok / value, "higher_is_better": True, "scaling": "weak",
@@ -209,24 +266,13 @@ def main():
     sh, B, ctx = wl["shape"], wl["batch"], wl["ctx"]
     num0, den0 = wl["share"]
     NL, Hq, Hkv, dqk, dv = sh.n_layers, sh.n_q_heads, sh.n_kv_heads, sh.dim_qk, sh.dim_v
-    n_cpu = BLOCK * ((ctx // BLOCK) * num0 // den0)
-    n_gpu0 = ctx - n_cpu
+    lens = seq_lens(wl)
+    n_cpu = sum(cpu_tokens(n, num0, den0) for n in lens) // B        # mean CPU-side tokens per sequence
+    n_gpu0 = sum(lens) // B - n_cpu
     total_steps = 2 * (args.warmup + args.steps) + 8
-    p_cap = n_gpu0 + WINDOW * (total_steps // WINDOW + 2)
-    kind = binding.MLA if sh.kind == "mla" else binding.GQA
-    cfg = binding.make_config(kind, NL, B, Hq, Hkv, dqk, dv, block_tokens=BLOCK, window_tokens=WINDOW, chunk_tokens=512,
-                              n_slots=2, max_u_tokens_per_seq=n_cpu + WINDOW * (total_steps // WINDOW + 2),
-                              max_p_tokens_per_seq=p_cap, resident_tokens_per_seq=p_cap, softmax_scale=sh.scale,
-                              share_num=num0, share_den=den0, device=local_rank,
-                              flags=binding.FLAG_NO_HOST_U | binding.FLAG_NO_HOST_P)
-    cache = binding.Cache(cfg)
+    cache = make_cache(wl, local_rank, total_steps)
     seq_ids = list(range(B))
-    # ---- populate: prefill routed in one shot, the GPU-side share lands in the resident ring -------------
-    for layer in range(NL):
-        for s in range(B):
-            k, v = synth.device_kv(sh, ctx, 1000 * wl["cfg_id"] + (layer * B + s) + 100 * rank, dev)
-            cache.append_bulk(layer, s, k, v, ctx, num0, den0)
-        torch.cuda.synchronize()
+    populate(cache, wl, dev, rank)
     g = torch.Generator(device=dev); g.manual_seed(77 + rank)
     bf = torch.bfloat16
     q = torch.randn((NL, B, Hq, dqk), generator=g, device=dev).to(bf)
@@ -358,8 +404,9 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": args.workload, "layers": NL, "batch": B, "context": ctx, "cpu_share": f"{num0}/{den0}",
-                       "gpu_share_tokens_per_seq": n_gpu0 + 1, "bytes_per_kv_token": bpt, "block_tokens": BLOCK, "window_tokens": WINDOW,
+            "config": {"workload": args.workload, "layers": NL, "batch": B,
+                       "context": ctx if "lens" not in wl else f"ragged {min(lens)}..{max(lens)} (sum {sum(lens)})",
+                       "cpu_share": f"{num0}/{den0}", "gpu_share_tokens_per_seq_mean": n_gpu0 + 1, "bytes_per_kv_token": bpt, "block_tokens": BLOCK, "window_tokens": WINDOW,
                        "gpu_share": "HBM-resident", "host_copies_of_U_and_P": "off (benchmark)", "cpu_partial": "synthetic values",
                        "l2": "inputs larger than L2 (each layer reads its own %.2f GB)" % (bytes_attended / max(1, n_launch) / 1e9),
                        "multi_gpu": "replicas only", "kv_splits": args.kv_splits},

@@ -42,7 +42,7 @@ def build(force=False, verbose=False):
     if failed:
         raise RuntimeError("nvcc failed")
     tmp = LIB + ".tmp.%d" % os.getpid()
-    subprocess.run([NVCC, "-shared", "-o", tmp] + objs + ["-lcudart"], check=True)
+    subprocess.run([NVCC, "-shared", "-arch=sm_100a", "-o", tmp] + objs + ["-lcudart"], check=True)
     os.replace(tmp, LIB)
     return LIB
 

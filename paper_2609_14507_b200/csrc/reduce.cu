@@ -1,9 +1,9 @@
 // Exact log-sum-exp joins (Sec. 4.2 "merged via log-sum-exp rescaling", Sec. 5.1 "merge exactly"):
 //   LSE = m + ln sum_i exp(LSE_i - m), m = max_i LSE_i;   O = sum_i exp(LSE_i - LSE) * O_i.
 //   split_reduce_kernel  second pass of split-K attention: joins the item partials of every
-//                        (row, query head), optionally folding in an earlier partial of the same row
-//   merge_kernel         joins up to 8 row-aligned partials (GPU share, CPU share, ...)
-// One warp per output row; lanes stride over the value columns with 16-byte accesses.
+//                        (row, query head), optionally folding in an earlier partial of the same row;
+//                        one CTA per output row, threads split over (items, columns)
+//   merge_kernel         joins up to 8 row-aligned partials (GPU share, CPU share, ...); one warp per row
 #include <cuda_bf16.h>
 
 #include "kernels.h"
@@ -13,49 +13,81 @@ namespace ipkvi {
 namespace {
 
 constexpr int kWarpsPerBlock = 4;
+constexpr int kReduceThreads = 256;
 
-__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+// One CTA per (row, query head). Threads are arranged as (item slice, 4-column group): every thread sums the
+// weighted partials of its slice of the row's items for its four columns; the slices are then added through
+// shared memory. CG = dv / 4 column groups, SL = 256 / CG slices.
+__global__ void __launch_bounds__(kReduceThreads)
 split_reduce_kernel(const float* __restrict__ part_o, const float* __restrict__ part_lse,
                     const int32_t* __restrict__ row_item_start, const float* acc_o, const float* acc_lse,
-                    float* out_o, float* out_lse, int n_rows, int Hq, int dv) {
-    const int wid = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
-    if (wid >= n_rows * Hq) return;
+                    float* out_o, float* out_lse, int Hq, int dv) {
+    extern __shared__ float4 red[];                 // [SL][CG]
+    __shared__ float s_warp[kReduceThreads / 32];
+    __shared__ float s_m;
+    __shared__ float s_zs[kReduceThreads / 16];    // weight sum of every item slice (SL <= 16)
+    const int wid = blockIdx.x;                      // row * Hq + h
     const int row = wid / Hq, h = wid - row * Hq;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int i0 = row_item_start[row], i1 = row_item_start[row + 1];
-    float m = acc_lse ? acc_lse[wid] : -INFINITY;
-    for (int i = i0 + lane; i < i1; i += 32) m = fmaxf(m, part_lse[int64_t(i) * Hq + h]);
+    const float la = acc_lse ? acc_lse[wid] : -INFINITY;
+
+    float m = la;
+    for (int i = i0 + tid; i < i1; i += kReduceThreads) m = fmaxf(m, part_lse[int64_t(i) * Hq + h]);
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, d));
+    if (lane == 0) s_warp[warp] = m;
+    __syncthreads();
+    if (tid == 0) {
+        float mm = s_warp[0];
+        for (int w = 1; w < kReduceThreads / 32; ++w) mm = fmaxf(mm, s_warp[w]);
+        s_m = mm;
+    }
+    __syncthreads();
+    m = s_m;
+    const int CG = dv >> 2, SL = kReduceThreads / CG;
+    const int cg = tid % CG, sl = tid / CG;
     float* oo = out_o + int64_t(wid) * dv;
-    if (m == -INFINITY) {                       // nothing attended: (0, -inf)
-        for (int c = lane * 4; c < dv; c += 128) *reinterpret_cast<float4*>(oo + c) = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (lane == 0) out_lse[wid] = -INFINITY;
+    if (m == -INFINITY) {                           // nothing attended: (0, -inf)
+        if (sl == 0) *reinterpret_cast<float4*>(oo + cg * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (tid == 0) out_lse[wid] = -INFINITY;
         return;
     }
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float z = 0.f;
-    for (int i = i0 + lane; i < i1; i += 32) z += __expf(part_lse[int64_t(i) * Hq + h] - m);
-#pragma unroll
-    for (int d = 16; d > 0; d >>= 1) z += __shfl_xor_sync(0xffffffffu, z, d);
-    const float wa = acc_lse ? __expf(acc_lse[wid] - m) : 0.f;
-    z += wa;
-    const float inv = 1.f / z;
-    for (int c = lane * 4; c < dv; c += 128) {
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (acc_o && wa != 0.f) {
-            const float4 v = *reinterpret_cast<const float4*>(acc_o + int64_t(wid) * dv + c);
-            acc.x = wa * v.x; acc.y = wa * v.y; acc.z = wa * v.z; acc.w = wa * v.w;
-        }
-        for (int i = i0; i < i1; ++i) {
+    {
+        const float* po = part_o + int64_t(h) * dv + cg * 4;
+        const int64_t stride = int64_t(Hq) * dv;
+#pragma unroll 4
+        for (int i = i0 + sl; i < i1; i += SL) {
             const float w = __expf(part_lse[int64_t(i) * Hq + h] - m);
-            const float4 v = *reinterpret_cast<const float4*>(part_o + (int64_t(i) * Hq + h) * dv + c);
+            const float4 v = *reinterpret_cast<const float4*>(po + int64_t(i) * stride);
             acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
+            z += w;
         }
-        acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
-        *reinterpret_cast<float4*>(oo + c) = acc;
+        red[sl * CG + cg] = acc;
     }
-    __syncwarp();   // every lane has read acc_lse[wid] (it may alias out_lse) before it is overwritten
-    if (lane == 0) out_lse[wid] = m + logf(z);
+    // every thread of a slice holds the same weight sum z; column group 0 publishes it
+    if (cg == 0) s_zs[sl] = z;
+    __syncthreads();
+    if (sl == 0) {
+        float4 t = red[cg];
+        for (int k = 1; k < SL; ++k) {
+            const float4 u = red[k * CG + cg];
+            t.x += u.x; t.y += u.y; t.z += u.z; t.w += u.w;
+        }
+        const float wa = (la == -INFINITY) ? 0.f : __expf(la - m);
+        if (wa != 0.f) {
+            const float4 v = *reinterpret_cast<const float4*>(acc_o + int64_t(wid) * dv + cg * 4);
+            t.x += wa * v.x; t.y += wa * v.y; t.z += wa * v.z; t.w += wa * v.w;
+        }
+        float zt = wa;
+        for (int k = 0; k < SL; ++k) zt += s_zs[k];      // fixed order: results are reproducible bit for bit
+        const float inv = 1.f / zt;
+        t.x *= inv; t.y *= inv; t.z *= inv; t.w *= inv;
+        *reinterpret_cast<float4*>(oo + cg * 4) = t;
+        if (cg == 0) out_lse[wid] = m + logf(zt);
+    }
 }
 
 __global__ void __launch_bounds__(kWarpsPerBlock * 32) merge_kernel(const MergeLaunch a) {
@@ -105,9 +137,10 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) merge_kernel(const MergeL
 cudaError_t launch_split_reduce(const AttnLaunch& a, cudaStream_t s) {
     const int total = a.n_rows * a.n_q_heads;
     if (total <= 0) return cudaSuccess;
-    const int grid = (total + kWarpsPerBlock - 1) / kWarpsPerBlock;
-    split_reduce_kernel<<<grid, kWarpsPerBlock * 32, 0, s>>>(a.part_o, a.part_lse, a.row_item_start, a.acc_o, a.acc_lse,
-                                                            a.out_o, a.out_lse, a.n_rows, a.n_q_heads, a.dim_v);
+    if (a.dim_v % 4 != 0 || a.dim_v / 4 > kReduceThreads || kReduceThreads % (a.dim_v / 4) != 0) return cudaErrorInvalidValue;
+    const size_t smem = size_t(kReduceThreads) * sizeof(float4);
+    split_reduce_kernel<<<total, kReduceThreads, smem, s>>>(a.part_o, a.part_lse, a.row_item_start, a.acc_o, a.acc_lse,
+                                                           a.out_o, a.out_lse, a.n_q_heads, a.dim_v);
     return cudaGetLastError();
 }
 

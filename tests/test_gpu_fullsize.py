@@ -1,0 +1,89 @@
+"""Parity at the benchmark's sizes and launch configuration, on sampled outputs the oracle computes one by one.
+
+The caches are built exactly as bench.py builds them (same shapes, seeds, shares, flags); one decode step is run
+(append, attend, merge) and, for a sample of (layer, sequence) pairs, the oracle recomputes the GPU-side partial of
+every head from the same bits (regenerated from the seed and copied to the host)."""
+import numpy as np
+import pytest
+
+import bench
+from oracle import c_oracle
+from paper_2609_14507_b200 import synth
+from tests.gpu_util import check_partial
+
+pytestmark = pytest.mark.gpu
+torch = pytest.importorskip("torch")
+DEV = "cuda:0"
+
+
+def _run_step_and_check(name, samples, kv_splits=0):
+    wl = bench.WORKLOADS[name]
+    sh, B = wl["shape"], wl["batch"]
+    num0, den0 = wl["share"]
+    lens = bench.seq_lens(wl)
+    need = sum(n - bench.cpu_tokens(n, num0, den0) for n in lens) * sh.n_layers * sh.bytes_per_token
+    free, _ = torch.cuda.mem_get_info()
+    if free < 1.3 * need:
+        pytest.skip(f"needs {need / 1e9:.0f} GB of device memory")
+    cache = bench.make_cache(wl, 0, 8)
+    try:
+        bench.populate(cache, wl, DEV)
+        g = torch.Generator(device=DEV); g.manual_seed(123)
+        ids = list(range(B))
+        scale = float(np.float32(sh.scale))
+        for layer in sorted({l for l, _ in samples}):
+            q = torch.randn((B, sh.n_q_heads, sh.dim_qk), generator=g, device=DEV).to(torch.bfloat16)
+            kn = torch.randn((B, sh.n_kv_heads, sh.dim_qk), generator=g, device=DEV).to(torch.bfloat16)
+            vn = None if sh.kind == "mla" else torch.randn((B, sh.n_kv_heads, sh.dim_v), generator=g, device=DEV).to(torch.bfloat16)
+            cache.append(layer, ids, kn, vn)
+            o = torch.zeros((B, sh.n_q_heads, sh.dim_v), device=DEV); lse = torch.zeros((B, sh.n_q_heads), device=DEV)
+            cache.attend_gpu(layer, ids, q, o, lse, kv_splits=kv_splits)
+            torch.cuda.synchronize()
+            o_h, lse_h, q_h = o.cpu().numpy(), lse.cpu().numpy(), synth.torch_bits(q)
+            kn_h, vn_h = synth.torch_bits(kn), (None if vn is None else synth.torch_bits(vn))
+            for (l, s) in samples:
+                if l != layer:
+                    continue
+                n = lens[s]
+                c = cache.counts(layer, s)
+                n_cpu = bench.cpu_tokens(n, num0, den0)
+                assert (c["n_u"], c["n_p"], c["n_w"]) == (n_cpu, n - n_cpu, 1)
+                kd, vd = synth.device_kv(sh, n, bench.kv_seed(wl, layer, s), DEV)
+                k = np.concatenate([synth.torch_bits(kd), kn_h[s:s + 1]])
+                v = sh.dim_v if vd is None else np.concatenate([synth.torch_bits(vd), vn_h[s:s + 1]])
+                o_ref, l_ref = c_oracle.attend(q_h[s], k, v, np.arange(n_cpu, n + 1), scale)
+                check_partial(o_h[s], lse_h[s], o_ref, l_ref, f"{name} layer {layer} seq {s}")
+                # contents of the newest token and of a few routed ones, bit for bit
+                for t in (n, n - 1, n_cpu, (n_cpu + n) // 2):
+                    kk, vv = cache.read_token(layer, s, t)
+                    np.testing.assert_array_equal(kk, k[t])
+                    if vv is not None:
+                        np.testing.assert_array_equal(vv, v[t])
+        assert cache.get_stats()["device_status"] == 0
+    finally:
+        cache.close()
+        torch.cuda.empty_cache()
+
+
+def test_mixtral_32k_bench_configuration():
+    _run_step_and_check("mixtral-8x7b-bs16-32k-cpu25", [(0, 0), (0, 15), (17, 6), (31, 9)])
+
+
+def test_qwen3_32k_share_sweep_sampled():
+    for name in ("qwen3-2layers-bs16-32k-cpu0",):
+        _run_step_and_check(name, [(0, 3), (1, 12)])
+    for num in (1, 3, 5, 7):                              # CPU share 10 / 30 / 50 / 70 %
+        wl = dict(bench.WORKLOADS["qwen3-2layers-bs16-32k-cpu0"], share=(num, 10))
+        bench.WORKLOADS["_tmp"] = wl
+        try:
+            _run_step_and_check("_tmp", [(1, num)])
+        finally:
+            del bench.WORKLOADS["_tmp"]
+
+
+def test_deepseek_mla_128k_sampled():
+    _run_step_and_check("deepseek-v2-lite-mla-2layers-bs8-128k-cpu40", [(0, 0), (1, 7)])
+
+
+def test_ragged_1m_token_batch_sampled():
+    _run_step_and_check("qwen3-ragged-bs64-1m-2layers-cpu30", [(0, 0), (0, 63), (1, 31), (1, 17)])
