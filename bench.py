@@ -65,6 +65,15 @@ WORKLOADS["qwen3-ragged-bs64-1m-2layers-cpu30"] = dict(
     lens=synth.ragged_lengths(5, 64, 8192, 24576))
 
 
+# Load reading of config 3 ("host-share chunks streamed H2D from pinned memory"): the oldest `stream_pct` % of every
+# sequence's P share is NOT device-resident; it lives in pinned host memory and is streamed through the PP slots on a
+# side stream each step while the resident rest is attended. 2 layers: the pinned host copy of P is 1 GB per layer.
+for _pct in (10, 30, 50, 70, 100):
+    WORKLOADS[f"qwen3-2layers-bs16-32k-stream{_pct}"] = dict(
+        shape=synth.Shape("qwen3-2l", "gqa", 2, 32, 4, 128, 128, 128 ** -0.5), batch=16, ctx=32768, share=(0, 1), cfg_id=3,
+        stream_pct=_pct, chunk_tokens=4096)
+
+
 def seq_lens(wl):
     """Context length of every sequence of the batch."""
     return [int(x) for x in wl["lens"]] if "lens" in wl else [wl["ctx"]] * wl["batch"]
@@ -89,11 +98,15 @@ def make_cache(wl, device_index, decode_steps):
     p_cap = longest - cpu_tokens(longest, num0, den0) + grow if num0 < den0 else grow
     p_cap = max(p_cap, max(n - cpu_tokens(n, num0, den0) for n in seq_lens(wl)) + grow)
     kind = binding.MLA if sh.kind == "mla" else binding.GQA
+    resident, flags = p_cap, binding.FLAG_NO_HOST_U | binding.FLAG_NO_HOST_P
+    if "stream_pct" in wl:
+        # keep the newest (100 - stream_pct) % of the prefill's P share resident; P itself lives in pinned host memory
+        resident = BLOCK * (((longest - cpu_tokens(longest, num0, den0)) * (100 - wl["stream_pct"]) // 100) // BLOCK)
+        flags = binding.FLAG_NO_HOST_U
     cfg = binding.make_config(kind, sh.n_layers, wl["batch"], sh.n_q_heads, sh.n_kv_heads, sh.dim_qk, sh.dim_v,
-                              block_tokens=BLOCK, window_tokens=WINDOW, chunk_tokens=512, n_slots=2,
-                              max_u_tokens_per_seq=longest + grow, max_p_tokens_per_seq=p_cap, resident_tokens_per_seq=p_cap,
-                              softmax_scale=sh.scale, share_num=num0, share_den=den0, device=device_index,
-                              flags=binding.FLAG_NO_HOST_U | binding.FLAG_NO_HOST_P)
+                              block_tokens=BLOCK, window_tokens=WINDOW, chunk_tokens=wl.get("chunk_tokens", 512), n_slots=2,
+                              max_u_tokens_per_seq=longest + grow, max_p_tokens_per_seq=p_cap, resident_tokens_per_seq=resident,
+                              softmax_scale=sh.scale, share_num=num0, share_den=den0, device=device_index, flags=flags)
     return binding.Cache(cfg)
 
 
@@ -331,6 +344,7 @@ def main():
     cache.profile_enable(False)
     st1 = cache.get_stats()
     bytes_attended = st1["kv_bytes_attended"] - st0["kv_bytes_attended"]
+    h2d_stream = st1["h2d_bytes"] - st0["h2d_bytes"]
     tokens = bytes_attended // bpt
     launches = sum(st1[k] - st0[k] for k in ("attend_kernels", "reduce_kernels", "merge_kernels", "append_kernels", "pack_kernels"))
     value = world * tokens / (ms * 1e-3)
@@ -413,6 +427,11 @@ def main():
             "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu,
             "step_gbs": world * bytes_attended / (ms * 1e-3) / 1e9,
         }
+        if "stream_pct" in wl:
+            line["streaming"] = {"h2d_bytes_per_step": h2d_stream / args.steps, "h2d_gbs": h2d_stream / (ms * 1e-3) / 1e9,
+                                 "streamed_pct_of_p_share": wl["stream_pct"], "chunk_tokens": wl.get("chunk_tokens", 512)}
+            line["config"]["gpu_share"] = "%d %% streamed H2D from pinned host memory each step, rest HBM-resident" % wl["stream_pct"]
+            line["config"]["host_copies_of_U_and_P"] = "P on (pinned), U off"
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

@@ -48,14 +48,10 @@ struct SeqState {
     std::vector<PRun> p_runs;
 };
 
-size_t partial_bytes(size_t n_items, int Hq, int dv) {
-    return align_up(n_items * size_t(Hq) * dv * sizeof(float), 256) + align_up(n_items * size_t(Hq) * sizeof(float), 256);
-}
-
-int64_t max_items_bound(int n_rows, int n_runs, int64_t total_tokens, int kv_splits) {
-    const int64_t tiles = (total_tokens + kTileTokens - 1) / kTileTokens + n_runs;
-    if (kv_splits > 0) return int64_t(n_runs) * (kv_splits + 1) + n_rows;
-    return tiles + n_runs + n_rows;   // the planner never makes items smaller than one tile
+// Bytes of the partial buffers for n_spans spans.
+size_t partial_bytes(size_t n_spans, const PartGeom& pg, int dv) {
+    const size_t rows = n_spans * size_t(pg.parts_per_span) * pg.rows_per_group;
+    return align_up(rows * dv * sizeof(float), 256) + align_up(rows * sizeof(float), 256);
 }
 
 bool shape_ok(int kind, int Hq, int Hkv, int dqk, int dv, int bt, std::string* why) {
@@ -331,24 +327,22 @@ void fill_launch(AttnLaunch* a, int kind, int Hq, int Hkv, int dqk, int dv, int 
                  const char* table_dev, char* partials, const void* q, int n_rows) {
     a->kind = kind; a->n_q_heads = Hq; a->n_kv_heads = Hkv; a->dim_qk = dqk; a->dim_v = dv; a->bt = bt; a->scale = scale;
     a->q = q;
+    const PartGeom pg = part_geom(kind, Hq, Hkv);
     size_t o = 0;
     a->segs = reinterpret_cast<const Seg*>(table_dev + o);
     o += align_up(plan.segs.size() * sizeof(Seg), 16);
-    a->items = reinterpret_cast<const Item*>(table_dev + o);
-    o += align_up(plan.items.size() * sizeof(Item), 16);
-    a->row_item_start = reinterpret_cast<const int32_t*>(table_dev + o);
-    a->n_items = int(plan.items.size());
+    a->spans = reinterpret_cast<const Span*>(table_dev + o);
+    o += align_up(plan.spans.size() * sizeof(Span), 16);
+    a->cta_span_start = reinterpret_cast<const int32_t*>(table_dev + o);
+    o += align_up(plan.cta_span_start.size() * sizeof(int32_t), 16);
+    a->rg_span_start = reinterpret_cast<const int32_t*>(table_dev + o);
+    a->n_spans = int(plan.spans.size());
+    a->n_ctas = plan.n_ctas();
     a->n_rows = n_rows;
+    a->n_gh = pg.n_gh;
+    const size_t rows = plan.spans.size() * size_t(pg.parts_per_span) * pg.rows_per_group;
     a->part_o = reinterpret_cast<float*>(partials);
-    a->part_lse = reinterpret_cast<float*>(partials + align_up(plan.items.size() * size_t(Hq) * dv * sizeof(float), 256));
-}
-
-int ctas_per_sm(int kind) { return kind == IPKV_MLA ? 1 : 2; }
-
-int heads_per_tile(int kind, int Hq, int Hkv) {
-    if (kind == IPKV_MLA) return (Hq + 15) / 16;
-    const int G = Hq / Hkv;
-    return Hkv * ((G + 15) / 16);
+    a->part_lse = reinterpret_cast<float*>(partials + align_up(rows * dv * sizeof(float), 256));
 }
 
 // One group of segments for all rows: attention + split reduce, folding into (out_o, out_lse) when `fold`.
@@ -356,8 +350,9 @@ ipkv_status run_group(ipkv* h, const std::vector<std::vector<PlanSeg>>& rows, co
                       const void* q, int kv_splits, bool fold, float* out_o, float* out_lse, cudaStream_t s) {
     const ipkv_config& c = h->cfg;
     Plan plan;
-    build_plan(rows, heads_per_tile(c.kind, c.n_q_heads, c.n_kv_heads), kv_splits, ctas_per_sm(c.kind), &plan);
-    ipkv_status rc = ensure_scratch(h, partial_bytes(plan.items.size(), c.n_q_heads, c.dim_v));
+    const PartGeom pg = part_geom(c.kind, c.n_q_heads, c.n_kv_heads);
+    build_plan(rows, pg.n_gh, kv_splits, pg.ctas_per_sm, &plan);
+    ipkv_status rc = ensure_scratch(h, partial_bytes(plan.spans.size(), pg, c.dim_v));
     if (rc != IPKV_OK) return rc;
     const char* table = nullptr;
     rc = upload_table(h, plan, s, &table);
@@ -370,7 +365,7 @@ ipkv_status run_group(ipkv* h, const std::vector<std::vector<PlanSeg>>& rows, co
     a.acc_lse = fold ? out_lse : nullptr;
     a.out_o = out_o; a.out_lse = out_lse;
     a.status = h->status_dev;
-    if (a.n_items > 0) {
+    if (a.n_spans > 0) {
         const bool timed = h->prof_on && h->prof_used + 2 <= h->prof_ev.size();
         if (timed) CU(h, cudaEventRecord(h->prof_ev[h->prof_used], s));
         CU(h, launch_attend(a, s));
@@ -916,10 +911,13 @@ ipkv_status ipkv_attend_scratch_bytes(const ipkv_attn_shape* sh, int32_t n_rows,
                                       int64_t total_tokens, int32_t kv_splits, size_t* out_bytes) {
     if (!sh || !out_bytes || n_rows < 0 || n_runs < 0 || total_tokens < 0 || kv_splits < 0) return IPKV_EINVAL;
     if (!shape_ok(sh->kind, sh->n_q_heads, sh->n_kv_heads, sh->dim_qk, sh->dim_v, sh->block_tokens, nullptr)) return IPKV_EINVAL;
-    const int64_t items = max_items_bound(n_rows, n_runs, total_tokens, kv_splits);
-    const size_t table = align_up(size_t(n_runs) * sizeof(Seg), 16) + align_up(size_t(items) * sizeof(Item), 16) +
-                         align_up(size_t(n_rows + 1) * sizeof(int32_t), 16);
-    *out_bytes = align_up(table, 256) + 256 + partial_bytes(size_t(items), sh->n_q_heads, sh->dim_v);
+    (void)total_tokens;
+    const PartGeom pg = part_geom(sh->kind, sh->n_q_heads, sh->n_kv_heads);
+    const int64_t spans = max_spans_bound(n_rows, n_runs, pg.n_gh, kv_splits, pg.ctas_per_sm);
+    const size_t table = align_up(size_t(n_runs) * sizeof(Seg), 16) + align_up(size_t(spans) * sizeof(Span), 16) +
+                         align_up(size_t(kSmCount * pg.ctas_per_sm + 1) * sizeof(int32_t), 16) +
+                         align_up((size_t(n_rows) * pg.n_gh + 1) * sizeof(int32_t), 16);
+    *out_bytes = align_up(table, 256) + 256 + partial_bytes(size_t(spans), pg, sh->dim_v);
     return IPKV_OK;
 }
 
@@ -943,9 +941,10 @@ ipkv_status ipkv_attend_runs(const ipkv_attn_shape* sh, int32_t n_rows,
         }
     }
     Plan plan;
-    build_plan(rows, heads_per_tile(sh->kind, sh->n_q_heads, sh->n_kv_heads), kv_splits, ctas_per_sm(sh->kind), &plan);
+    const PartGeom pg = part_geom(sh->kind, sh->n_q_heads, sh->n_kv_heads);
+    build_plan(rows, pg.n_gh, kv_splits, pg.ctas_per_sm, &plan);
     const size_t table = align_up(plan.table_bytes(), 256);
-    if (table + 256 + partial_bytes(plan.items.size(), sh->n_q_heads, sh->dim_v) > scratch_bytes) return IPKV_ENOMEM;
+    if (table + 256 + partial_bytes(plan.spans.size(), pg, sh->dim_v) > scratch_bytes) return IPKV_ENOMEM;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     std::vector<char> img(table, 0);
     plan.serialize(img.data());
@@ -958,7 +957,7 @@ ipkv_status ipkv_attend_runs(const ipkv_attn_shape* sh, int32_t n_rows,
     a.bases[0] = nullptr;
     a.out_o = o_part_dev; a.out_lse = lse_part_dev;
     a.status = status_dev ? status_dev : reinterpret_cast<uint32_t*>(static_cast<char*>(scratch_dev) + table);
-    if (a.n_items > 0 && launch_attend(a, s) != cudaSuccess) return IPKV_ECUDA;
+    if (a.n_spans > 0 && launch_attend(a, s) != cudaSuccess) return IPKV_ECUDA;
     if (launch_split_reduce(a, s) != cudaSuccess) return IPKV_ECUDA;
     return IPKV_OK;
 }

@@ -4,7 +4,8 @@
 // each latent is read from memory once).  The paper's kernel for this case is a CPU kernel; this one is
 // written for sm_100a.
 //
-// One CTA per (item, group of 16 query heads): a producer warp streams 64-token tiles (73 728 contiguous
+// Persistent split-K (one CTA per SM, each with an equally long contiguous chunk of the launch's tiles, cut
+// into spans where the (row, head group, run) changes): a producer warp streams 64-token tiles (73 728 contiguous
 // bytes in the TILE block layout) into a 2-stage shared-memory ring with bulk asynchronous copies that
 // complete on mbarriers; the tile is read twice from shared memory — as K (ldmatrix) and as V
 // (ldmatrix.trans on the first eight 64-column panels) — and once from HBM.
@@ -52,11 +53,12 @@ struct MlaParams {
     const __nv_bfloat16* q;
     const char* bases[kMaxBases];
     const Seg* segs;
-    const Item* items;
+    const Span* spans;
+    const int32_t* cta_span_start;
     float* part_o;
     float* part_lse;
     uint32_t* status;
-    int Hq, n_hg;
+    int Hq;
     int bt;
     int64_t block_bytes;
     float scale_log2;
@@ -77,11 +79,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_mla_kernel(const MlaParams p
     float* s_l = s_alpha + 32;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const Item item = p.items[blockIdx.x];
-    const Seg seg = p.segs[item.seg];
-    const int hg = blockIdx.y;
-    const int head0 = hg * 16;
-    const int n_heads = min(16, p.Hq - head0);
+    const int span_begin = p.cta_span_start[blockIdx.x], span_end = p.cta_span_start[blockIdx.x + 1];
 
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -90,59 +88,58 @@ __global__ void __launch_bounds__(kThreads, 1) attn_mla_kernel(const MlaParams p
         }
         ptx::mbar_fence_init();
     }
-    for (int c = tid; c < 16 * (kDqk / 8); c += kThreads) {
-        const int r = c / (kDqk / 8), ch = c - r * (kDqk / 8);
-        uint4 val = make_uint4(0, 0, 0, 0);
-        if (r < n_heads) val = *reinterpret_cast<const uint4*>(p.q + (int64_t(item.row) * p.Hq + head0 + r) * kDqk + ch * 8);
-        *reinterpret_cast<uint4*>(smem + kOffQ + r * kQPitch + ch * 16) = val;
-    }
     if (p.bt < kTileTokens) {
         for (int c = tid; c < kStages * kStageBytes / 16; c += kThreads) reinterpret_cast<uint4*>(smem)[c] = make_uint4(0, 0, 0, 0);
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     __syncthreads();
 
-    const char* seg_base = p.bases[seg.base_id] + seg.off;
     bool ok = true;
+    int it = 0;                      // tiles streamed so far by this CTA: stage = it % kStages
 
     if (warp == kConsumerWarps) {
-        // ---------------- producer ----------------
+        // ---------------- producer: streams the whole chunk, never pausing at span boundaries ----------------
         if (lane == 0) {
-            for (int i = 0; i < item.ntiles; ++i) {
-                const int st = i % kStages;
-                if (i >= kStages && !ptx::mbar_wait(s_empty + 8 * st, ((i / kStages) - 1) & 1)) { ok = false; break; }
-                const int64_t t0 = int64_t(item.tile0 + i) * kTileTokens;
-                const uint32_t dst = s_base + st * kStageBytes;
-                const uint32_t bar = s_full + 8 * st;
-                if (p.bt >= kTileTokens) {
-                    const int64_t blk = t0 / p.bt;
-                    const int r0 = int(t0 - blk * p.bt);
-                    const char* src = seg_base + blk * p.block_bytes;
-                    ptx::mbar_expect_tx(bar, kStageBytes);
-                    if (p.bt == kTileTokens) {
-                        ptx::bulk_g2s(dst, src, kStageBytes, bar);
+            for (int sn = span_begin; sn < span_end && ok; ++sn) {
+                const Span span = p.spans[sn];
+                const Seg seg = p.segs[span.seg];
+                const char* seg_base = p.bases[seg.base_id] + seg.off;
+                for (int i = 0; i < span.ntiles; ++i, ++it) {
+                    const int st = it % kStages;
+                    if (it >= kStages && !ptx::mbar_wait(s_empty + 8 * st, ((it / kStages) - 1) & 1)) { ok = false; break; }
+                    const int64_t t0 = int64_t(span.tile0 + i) * kTileTokens;
+                    const uint32_t dst = s_base + st * kStageBytes;
+                    const uint32_t bar = s_full + 8 * st;
+                    if (p.bt >= kTileTokens) {
+                        const int64_t blk = t0 / p.bt;
+                        const int r0 = int(t0 - blk * p.bt);
+                        const char* src = seg_base + blk * p.block_bytes;
+                        ptx::mbar_expect_tx(bar, kStageBytes);
+                        if (p.bt == kTileTokens) {
+                            ptx::bulk_g2s(dst, src, kStageBytes, bar);
+                        } else {
+#pragma unroll
+                            for (int pn = 0; pn < kPanels; ++pn)
+                                ptx::bulk_g2s(dst + pn * 8192, src + int64_t(pn) * p.bt * 128 + int64_t(r0) * 128, 8192, bar);
+                        }
                     } else {
+                        const int nsub = kTileTokens / p.bt;
+                        const int64_t blk0 = t0 / p.bt;
+                        int live = 0;
+                        for (int j = 0; j < nsub; ++j) live += ((blk0 + j) * p.bt < seg.n_tokens);
+                        const uint32_t sub_bytes = uint32_t(p.bt) * 128;
+                        ptx::mbar_expect_tx(bar, uint32_t(live) * sub_bytes * kPanels);
+                        for (int j = 0; j < live; ++j) {
+                            const char* src = seg_base + (blk0 + j) * p.block_bytes;
 #pragma unroll
-                        for (int pn = 0; pn < kPanels; ++pn)
-                            ptx::bulk_g2s(dst + pn * 8192, src + int64_t(pn) * p.bt * 128 + int64_t(r0) * 128, 8192, bar);
-                    }
-                } else {
-                    const int nsub = kTileTokens / p.bt;
-                    const int64_t blk0 = t0 / p.bt;
-                    int live = 0;
-                    for (int j = 0; j < nsub; ++j) live += ((blk0 + j) * p.bt < seg.n_tokens);
-                    const uint32_t sub_bytes = uint32_t(p.bt) * 128;
-                    ptx::mbar_expect_tx(bar, uint32_t(live) * sub_bytes * kPanels);
-                    for (int j = 0; j < live; ++j) {
-                        const char* src = seg_base + (blk0 + j) * p.block_bytes;
-#pragma unroll
-                        for (int pn = 0; pn < kPanels; ++pn)
-                            ptx::bulk_g2s(dst + pn * 8192 + j * sub_bytes, src + int64_t(pn) * sub_bytes, sub_bytes, bar);
+                            for (int pn = 0; pn < kPanels; ++pn)
+                                ptx::bulk_g2s(dst + pn * 8192 + j * sub_bytes, src + int64_t(pn) * sub_bytes, sub_bytes, bar);
+                        }
                     }
                 }
             }
-            const int first_pending = item.ntiles > kStages ? item.ntiles - kStages : 0;
-            for (int i = first_pending; i < item.ntiles; ++i)
+            const int first_pending = it > kStages ? it - kStages : 0;
+            for (int i = first_pending; i < it; ++i)
                 if (!ptx::mbar_wait(s_full + 8 * (i % kStages), (i / kStages) & 1)) ok = false;
             if (!ok) atomicOr(p.status, 1u);
         }
@@ -152,156 +149,173 @@ __global__ void __launch_bounds__(kThreads, 1) attn_mla_kernel(const MlaParams p
     // ---------------- consumers ----------------
     const int ds = warp & 3, th = warp >> 2;
     const int mi = lane >> 3, r8 = lane & 7;
-    uint32_t qa[9][4];
-#pragma unroll
-    for (int ks = 0; ks < 9; ++ks) {
-        const int row = (mi & 1) * 8 + r8, chunk = ds * 18 + ks * 2 + (mi >> 1);
-        ptx::ldmatrix_x4(s_q + row * kQPitch + chunk * 16, qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3]);
-    }
-    float o[8][4];
-#pragma unroll
-    for (int nt = 0; nt < 8; ++nt) { o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f; }
     // phase-2 ownership: this lane works on query row `srow`, tokens [stok, stok + 4) of every tile
     const int srow = 2 * warp + (lane >> 4), stok = (lane & 15) * 4;
-    float m_run = -INFINITY, l_run = 0.f;
 
-    for (int i = 0; i < item.ntiles; ++i) {
-        const int st = i % kStages;
-        if (ok && !ptx::mbar_wait(s_full + 8 * st, (i / kStages) & 1)) ok = false;   // after a timeout: no more waits, but keep the barriers below matched
-        const int64_t t0 = int64_t(item.tile0 + i) * kTileTokens;
-        const int64_t left = int64_t(seg.n_tokens) - t0;
-        const int n_valid = left < kTileTokens ? int(left) : kTileTokens;
-        const uint32_t kb = s_base + st * kStageBytes;
+    for (int sn = span_begin; sn < span_end; ++sn) {
+        const Span span = p.spans[sn];
+        const Seg seg = p.segs[span.seg];
+        const int head0 = span.gh * 16;
+        const int n_heads = min(16, p.Hq - head0);
 
-        // ---- phase 1: partial scores of d-slice ds for tokens [32 th, 32 th + 32) ----
-        {
-            float s[4][4];
-#pragma unroll
-            for (int nt = 0; nt < 4; ++nt) { s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f; }
-#pragma unroll
-            for (int ks = 0; ks < 9; ++ks) {
-                const int chunk = ds * 18 + ks * 2 + (mi & 1);
-                const uint32_t col = (chunk >> 3) * 8192 + (((chunk & 7) ^ r8) << 4);
-#pragma unroll
-                for (int tg = 0; tg < 2; ++tg) {
-                    const int tok = th * 32 + tg * 16 + (mi >> 1) * 8 + r8;
-                    uint32_t b0, b1, b2, b3;
-                    ptx::ldmatrix_x4(kb + col + tok * 128, b0, b1, b2, b3);
-                    ptx::mma_bf16(s[2 * tg], qa[ks], b0, b1);
-                    ptx::mma_bf16(s[2 * tg + 1], qa[ks], b2, b3);
-                }
-            }
-            float* dst = sp + ds * 16 * kSPitch;
-            const int r0 = lane >> 2, c0 = th * 32 + 2 * (lane & 3);
-#pragma unroll
-            for (int nt = 0; nt < 4; ++nt) {
-                *reinterpret_cast<float2*>(dst + r0 * kSPitch + c0 + nt * 8) = make_float2(s[nt][0], s[nt][1]);
-                *reinterpret_cast<float2*>(dst + (r0 + 8) * kSPitch + c0 + nt * 8) = make_float2(s[nt][2], s[nt][3]);
-            }
+        // query tile of the span's head group -> shared memory -> this warp's d-slice fragments
+        for (int c = tid; c < 16 * (kDqk / 8); c += kConsumerWarps * 32) {
+            const int r = c / (kDqk / 8), ch = c - r * (kDqk / 8);
+            uint4 val = make_uint4(0, 0, 0, 0);
+            if (r < n_heads) val = __ldg(reinterpret_cast<const uint4*>(p.q + (int64_t(span.row) * p.Hq + head0 + r) * kDqk + ch * 8));
+            *reinterpret_cast<uint4*>(smem + kOffQ + r * kQPitch + ch * 16) = val;
         }
         consumer_barrier();
-
-        // ---- phase 2: softmax bookkeeping for the rows this warp owns ----
-        {
-            float4 a = *reinterpret_cast<const float4*>(sp + srow * kSPitch + stok);
+        uint32_t qa[9][4];
 #pragma unroll
-            for (int d = 1; d < 4; ++d) {
-                const float4 b = *reinterpret_cast<const float4*>(sp + (d * 16 + srow) * kSPitch + stok);
-                a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
-            }
-            float sv[4] = {a.x, a.y, a.z, a.w};
-#pragma unroll
-            for (int j = 0; j < 4; ++j) sv[j] = (stok + j < n_valid) ? sv[j] * p.scale_log2 : -INFINITY;
-            float mx = fmaxf(fmaxf(sv[0], sv[1]), fmaxf(sv[2], sv[3]));
-#pragma unroll
-            for (int d = 1; d < 16; d <<= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, d));
-            const float mn = fmaxf(m_run, mx);
-            const float ms = (mn == -INFINITY) ? 0.f : mn;
-            const float alpha = ptx::ex2(m_run - ms);
-            m_run = mn;
-            float pr[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) pr[j] = ptx::ex2(sv[j] - ms);
-            l_run = l_run * alpha + (pr[0] + pr[1] + pr[2] + pr[3]);
-            const uint32_t h0 = ptx::pack_bf16(pr[0], pr[1]), h1 = ptx::pack_bf16(pr[2], pr[3]);
-            const uint32_t l0 = ptx::pack_bf16(pr[0] - ptx::bf16_lo(h0), pr[1] - ptx::bf16_hi(h0));
-            const uint32_t l1 = ptx::pack_bf16(pr[2] - ptx::bf16_lo(h1), pr[3] - ptx::bf16_hi(h1));
-            *reinterpret_cast<uint2*>(smem + kOffPhi + srow * kPPitch + stok * 2) = make_uint2(h0, h1);
-            *reinterpret_cast<uint2*>(smem + kOffPlo + srow * kPPitch + stok * 2) = make_uint2(l0, l1);
-            if ((lane & 15) == 0) s_alpha[srow] = alpha;
+        for (int ks = 0; ks < 9; ++ks) {
+            const int row = (mi & 1) * 8 + r8, chunk = ds * 18 + ks * 2 + (mi >> 1);
+            ptx::ldmatrix_x4(s_q + row * kQPitch + chunk * 16, qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3]);
         }
-        consumer_barrier();
+        float o[8][4];
+#pragma unroll
+        for (int nt = 0; nt < 8; ++nt) { o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f; }
+        float m_run = -INFINITY, l_run = 0.f;
 
-        // ---- phase 3: O[:, 64 warp .. 64 warp + 64) = O * alpha + (P_hi + P_lo) V ----
-        {
-            const int r0 = lane >> 2;
-            const float a0 = s_alpha[r0], a1 = s_alpha[r0 + 8];
-            if (__any_sync(0xffffffffu, (a0 != 1.f) | (a1 != 1.f))) {
+        for (int i = 0; i < span.ntiles; ++i, ++it) {
+            const int st = it % kStages;
+            if (ok && !ptx::mbar_wait(s_full + 8 * st, (it / kStages) & 1)) ok = false;   // after a timeout: no more waits, but keep the barriers below matched
+            const int64_t t0 = int64_t(span.tile0 + i) * kTileTokens;
+            const int64_t left = int64_t(seg.n_tokens) - t0;
+            const int n_valid = left < kTileTokens ? int(left) : kTileTokens;
+            const uint32_t kb = s_base + st * kStageBytes;
+
+            // ---- phase 1: partial scores of d-slice ds for tokens [32 th, 32 th + 32) ----
+            {
+                float s[4][4];
 #pragma unroll
-                for (int nt = 0; nt < 8; ++nt) { o[nt][0] *= a0; o[nt][1] *= a0; o[nt][2] *= a1; o[nt][3] *= a1; }
-            }
-            const uint32_t vb = kb + warp * 8192;
+                for (int nt = 0; nt < 4; ++nt) { s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f; }
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {
-                uint32_t ph[4], pl[4];
-                const uint32_t poff = ((mi & 1) * 8 + r8) * kPPitch + (kk * 2 + (mi >> 1)) * 16;
-                ptx::ldmatrix_x4(s_phi + poff, ph[0], ph[1], ph[2], ph[3]);
-                ptx::ldmatrix_x4(s_plo + poff, pl[0], pl[1], pl[2], pl[3]);
-                const int tok = kk * 16 + (mi & 1) * 8 + r8;
+                for (int ks = 0; ks < 9; ++ks) {
+                    const int chunk = ds * 18 + ks * 2 + (mi & 1);
+                    const uint32_t col = (chunk >> 3) * 8192 + (((chunk & 7) ^ r8) << 4);
 #pragma unroll
-                for (int jj = 0; jj < 4; ++jj) {
-                    const int chunk = 2 * jj + (mi >> 1);
-                    uint32_t b0, b1, b2, b3;
-                    ptx::ldmatrix_x4_trans(vb + tok * 128 + ((chunk ^ r8) << 4), b0, b1, b2, b3);
-                    ptx::mma_bf16(o[2 * jj], ph, b0, b1);
-                    ptx::mma_bf16(o[2 * jj + 1], ph, b2, b3);
-                    ptx::mma_bf16(o[2 * jj], pl, b0, b1);
-                    ptx::mma_bf16(o[2 * jj + 1], pl, b2, b3);
+                    for (int tg = 0; tg < 2; ++tg) {
+                        const int tok = th * 32 + tg * 16 + (mi >> 1) * 8 + r8;
+                        uint32_t b0, b1, b2, b3;
+                        ptx::ldmatrix_x4(kb + col + tok * 128, b0, b1, b2, b3);
+                        ptx::mma_bf16(s[2 * tg], qa[ks], b0, b1);
+                        ptx::mma_bf16(s[2 * tg + 1], qa[ks], b2, b3);
+                    }
+                }
+                float* dst = sp + ds * 16 * kSPitch;
+                const int r0 = lane >> 2, c0 = th * 32 + 2 * (lane & 3);
+#pragma unroll
+                for (int nt = 0; nt < 4; ++nt) {
+                    *reinterpret_cast<float2*>(dst + r0 * kSPitch + c0 + nt * 8) = make_float2(s[nt][0], s[nt][1]);
+                    *reinterpret_cast<float2*>(dst + (r0 + 8) * kSPitch + c0 + nt * 8) = make_float2(s[nt][2], s[nt][3]);
                 }
             }
+            consumer_barrier();
+
+            // ---- phase 2: softmax bookkeeping for the rows this warp owns ----
+            {
+                float4 a = *reinterpret_cast<const float4*>(sp + srow * kSPitch + stok);
+#pragma unroll
+                for (int d = 1; d < 4; ++d) {
+                    const float4 b = *reinterpret_cast<const float4*>(sp + (d * 16 + srow) * kSPitch + stok);
+                    a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+                }
+                float sv[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) sv[j] = (stok + j < n_valid) ? sv[j] * p.scale_log2 : -INFINITY;
+                float mx = fmaxf(fmaxf(sv[0], sv[1]), fmaxf(sv[2], sv[3]));
+#pragma unroll
+                for (int d = 1; d < 16; d <<= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, d));
+                const float mn = fmaxf(m_run, mx);
+                const float ms = (mn == -INFINITY) ? 0.f : mn;
+                const float alpha = ptx::ex2(m_run - ms);
+                m_run = mn;
+                float pr[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) pr[j] = ptx::ex2(sv[j] - ms);
+                l_run = l_run * alpha + (pr[0] + pr[1] + pr[2] + pr[3]);
+                const uint32_t h0 = ptx::pack_bf16(pr[0], pr[1]), h1 = ptx::pack_bf16(pr[2], pr[3]);
+                const uint32_t l0 = ptx::pack_bf16(pr[0] - ptx::bf16_lo(h0), pr[1] - ptx::bf16_hi(h0));
+                const uint32_t l1 = ptx::pack_bf16(pr[2] - ptx::bf16_lo(h1), pr[3] - ptx::bf16_hi(h1));
+                *reinterpret_cast<uint2*>(smem + kOffPhi + srow * kPPitch + stok * 2) = make_uint2(h0, h1);
+                *reinterpret_cast<uint2*>(smem + kOffPlo + srow * kPPitch + stok * 2) = make_uint2(l0, l1);
+                if ((lane & 15) == 0) s_alpha[srow] = alpha;
+            }
+            consumer_barrier();
+
+            // ---- phase 3: O[:, 64 warp .. 64 warp + 64) = O * alpha + (P_hi + P_lo) V ----
+            {
+                const int r0 = lane >> 2;
+                const float a0 = s_alpha[r0], a1 = s_alpha[r0 + 8];
+                if (__any_sync(0xffffffffu, (a0 != 1.f) | (a1 != 1.f))) {
+#pragma unroll
+                    for (int nt = 0; nt < 8; ++nt) { o[nt][0] *= a0; o[nt][1] *= a0; o[nt][2] *= a1; o[nt][3] *= a1; }
+                }
+                const uint32_t vb = kb + warp * 8192;
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {
+                    uint32_t ph[4], pl[4];
+                    const uint32_t poff = ((mi & 1) * 8 + r8) * kPPitch + (kk * 2 + (mi >> 1)) * 16;
+                    ptx::ldmatrix_x4(s_phi + poff, ph[0], ph[1], ph[2], ph[3]);
+                    ptx::ldmatrix_x4(s_plo + poff, pl[0], pl[1], pl[2], pl[3]);
+                    const int tok = kk * 16 + (mi & 1) * 8 + r8;
+#pragma unroll
+                    for (int jj = 0; jj < 4; ++jj) {
+                        const int chunk = 2 * jj + (mi >> 1);
+                        uint32_t b0, b1, b2, b3;
+                        ptx::ldmatrix_x4_trans(vb + tok * 128 + ((chunk ^ r8) << 4), b0, b1, b2, b3);
+                        ptx::mma_bf16(o[2 * jj], ph, b0, b1);
+                        ptx::mma_bf16(o[2 * jj + 1], ph, b2, b3);
+                        ptx::mma_bf16(o[2 * jj], pl, b0, b1);
+                        ptx::mma_bf16(o[2 * jj + 1], pl, b2, b3);
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(s_empty + 8 * st);
         }
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(s_empty + 8 * st);
+
+        // ---- end of span: the row owners publish m and l, every warp scales and writes its 64 columns ----
+#pragma unroll
+        for (int d = 1; d < 16; d <<= 1) l_run += __shfl_xor_sync(0xffffffffu, l_run, d);
+        if ((lane & 15) == 0) { s_m[srow] = m_run; s_l[srow] = l_run; }
+        consumer_barrier();
+        {
+            const int r0 = lane >> 2, c0 = warp * 64 + 2 * (lane & 3);
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                const int row = r0 + half * 8;
+                if (row < n_heads) {
+                    const float L = s_l[row];
+                    const float inv = (L > 0.f) ? 1.f / L : 0.f;
+                    float* dst = p.part_o + (int64_t(sn) * 16 + row) * kDv + c0;
+#pragma unroll
+                    for (int nt = 0; nt < 8; ++nt)
+                        *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(o[nt][2 * half] * inv, o[nt][2 * half + 1] * inv);
+                }
+            }
+            if (warp == 0 && lane < n_heads) {
+                const float M = s_m[lane], L = s_l[lane];
+                p.part_lse[int64_t(sn) * 16 + lane] = (M == -INFINITY) ? -INFINITY : (M + log2f(L)) * kLn2;
+            }
+        }
+        consumer_barrier();      // s_m / s_l / the query tile are reused by the next span
     }
     if (!ok && lane == 0) atomicOr(p.status, 1u);
-
-    // final normalisation: the row owners publish m and l, every warp scales its columns
-#pragma unroll
-    for (int d = 1; d < 16; d <<= 1) l_run += __shfl_xor_sync(0xffffffffu, l_run, d);
-    if ((lane & 15) == 0) { s_m[srow] = m_run; s_l[srow] = l_run; }
-    consumer_barrier();
-    {
-        const int r0 = lane >> 2, c0 = warp * 64 + 2 * (lane & 3);
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
-            const int row = r0 + half * 8;
-            if (row < n_heads) {
-                const float L = s_l[row];
-                const float inv = (L > 0.f) ? 1.f / L : 0.f;
-                float* dst = p.part_o + (int64_t(blockIdx.x) * p.Hq + head0 + row) * kDv + c0;
-#pragma unroll
-                for (int nt = 0; nt < 8; ++nt)
-                    *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(o[nt][2 * half] * inv, o[nt][2 * half + 1] * inv);
-            }
-        }
-        if (warp == 0 && lane < n_heads) {
-            const float M = s_m[lane], L = s_l[lane];
-            p.part_lse[int64_t(blockIdx.x) * p.Hq + head0 + lane] = (M == -INFINITY) ? -INFINITY : (M + log2f(L)) * kLn2;
-        }
-    }
 }
 
 }  // namespace
 
 cudaError_t launch_attend_mla(const AttnLaunch& a, cudaStream_t s) {
-    if (a.n_items <= 0) return cudaSuccess;
+    if (a.n_ctas <= 0 || a.n_spans <= 0) return cudaSuccess;
     if (a.dim_qk != kDqk || a.dim_v != kDv || a.n_kv_heads != 1) return cudaErrorInvalidValue;
     MlaParams p;
     p.q = static_cast<const __nv_bfloat16*>(a.q);
     for (int i = 0; i < kMaxBases; ++i) p.bases[i] = a.bases[i];
-    p.segs = a.segs; p.items = a.items;
+    p.segs = a.segs; p.spans = a.spans; p.cta_span_start = a.cta_span_start;
     p.part_o = a.part_o; p.part_lse = a.part_lse; p.status = a.status;
-    p.Hq = a.n_q_heads; p.n_hg = (a.n_q_heads + 15) / 16;
+    p.Hq = a.n_q_heads;
     p.bt = a.bt;
     p.block_bytes = int64_t(a.bt) * kDqk * 2;
     p.scale_log2 = a.scale * kLog2e;
@@ -314,8 +328,7 @@ cudaError_t launch_attend_mla(const AttnLaunch& a, cudaStream_t s) {
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
-    dim3 grid(a.n_items, p.n_hg);
-    attn_mla_kernel<<<grid, kThreads, smem, s>>>(p);
+    attn_mla_kernel<<<a.n_ctas, kThreads, smem, s>>>(p);
     return cudaGetLastError();
 }
 

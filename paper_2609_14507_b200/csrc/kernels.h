@@ -13,10 +13,11 @@ struct Seg {
     int32_t n_tokens;
     int32_t base_id;
 };
-// One unit of split-K work: tiles [tile0, tile0 + ntiles) of segment `seg` for query row `row`.
-// The partial it produces has the item's own index.
-struct Item {
-    int32_t row, seg, tile0, ntiles;
+// One span of split-K work: tiles [tile0, tile0 + ntiles) of segment `seg` for query row `row` and head
+// group `gh`.  A CTA processes a contiguous range of spans back to back; the partial(s) a span produces are
+// stored at the span's own index.
+struct Span {
+    int32_t row, gh, seg, tile0, ntiles;
 };
 
 constexpr int kMaxBases = 4;
@@ -27,12 +28,13 @@ struct AttnLaunch {
     float scale;                    // softmax scale applied to fp32 scores
     const void* q;                  // [n_rows][Hq][dqk] bf16
     const char* bases[kMaxBases];
-    const Seg* segs;                // device
-    const Item* items;              // device
-    const int32_t* row_item_start;  // device, [n_rows + 1]
-    int n_items, n_rows;
-    float* part_o;                  // [n_items][Hq][dv]
-    float* part_lse;                // [n_items][Hq]
+    const Seg* segs;                // device tables (see plan.hpp)
+    const Span* spans;
+    const int32_t* cta_span_start;  // [n_ctas + 1]
+    const int32_t* rg_span_start;   // [n_rows * n_gh + 1]
+    int n_spans, n_ctas, n_rows, n_gh;
+    float* part_o;                  // [n_spans * parts_per_span][rows_per_group][dv]
+    float* part_lse;                // [n_spans * parts_per_span][rows_per_group]
     const float* acc_o;             // optional earlier partial to fold in, [n_rows][Hq][dv]
     const float* acc_lse;
     float* out_o;                   // [n_rows][Hq][dv]
@@ -40,9 +42,27 @@ struct AttnLaunch {
     uint32_t* status;               // device word, OR-ed with an error bit if a bounded wait gives up
 };
 
-// Split-K attention: one partial (O, LSE) per (item, query head).
+// Geometry of the partial buffers: query heads per head group (rows of one partial), head groups per row,
+// partials per span (one per consumer warp for GQA, one for MLA), resident CTAs per SM.
+struct PartGeom {
+    int rows_per_group, n_gh, parts_per_span, ctas_per_sm;
+};
+inline PartGeom part_geom(int kind, int Hq, int Hkv) {
+    PartGeom g;
+    if (kind == 1) { g.rows_per_group = 16; g.n_gh = (Hq + 15) / 16; g.parts_per_span = 1; g.ctas_per_sm = 1; }
+    else {
+        const int G = Hq / Hkv;
+        g.rows_per_group = G < 16 ? G : 16;
+        g.n_gh = Hkv * ((G + 15) / 16);
+        g.parts_per_span = 4;
+        g.ctas_per_sm = 2;
+    }
+    return g;
+}
+
+// Split-K attention: partial (O, LSE) per span (and consumer warp), rows = the query heads of the span's group.
 cudaError_t launch_attend(const AttnLaunch& a, cudaStream_t s);
-// Second pass: per (row, head) LSE-reduce the row's item partials (and acc_*, if given) into out_*.
+// Second pass: per (row, head) LSE-reduce the partials of its head group's spans (and acc_*, if given) into out_*.
 cudaError_t launch_split_reduce(const AttnLaunch& a, cudaStream_t s);
 
 constexpr int kMaxMergeParts = 8;

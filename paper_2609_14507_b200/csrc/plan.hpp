@@ -1,7 +1,13 @@
 // Split-K planning for the GPU-side attention (host-only): turns the per-row list of block runs into
-// the segment / work-item tables the kernels read.  The sequence of one row is cut into items of
-// roughly equal numbers of 64-token tiles so that the grid fills the 148 SMs in whole waves; the
-// partials of a row's items are joined by the LSE reduce (the same exact merge as Sec. 5.1, n-way).
+// the tables the persistent attention kernels read.
+//
+// Work is counted in units of (64-token tile x head group): a head group is one KV head (x one group of
+// up to 16 of its query heads) for GQA, one group of up to 16 heads for MLA.  The units are laid out in
+// (row, head group, run, tile) order and cut into one contiguous, equally long chunk per CTA — one CTA
+// per resident slot of the 148 SMs, so the whole launch is a single balanced wave and every CTA streams
+// its chunk without a pause.  Where a chunk crosses from one (row, head group, run) to the next a new
+// span starts; every span produces its own partial (O, LSE) — one per consumer warp for GQA — and the
+// partials of a (row, head group) are joined by the LSE reduce (the same exact merge as Sec. 5.1, n-way).
 #pragma once
 #include <algorithm>
 #include <cstdint>
@@ -13,7 +19,6 @@
 namespace ipkvi {
 
 constexpr int kSmCount = 148;
-constexpr int kTargetTilesPerItem = 16;
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -21,88 +26,106 @@ struct PlanSeg { int base_id; int64_t off; int64_t n_tokens; };
 
 struct Plan {
     std::vector<Seg> segs;
-    std::vector<Item> items;
-    std::vector<int32_t> row_item_start;
+    std::vector<Span> spans;
+    std::vector<int32_t> cta_span_start;   // [n_ctas + 1]
+    std::vector<int32_t> rg_span_start;    // [n_rows * n_gh + 1]: spans of every (row, head group), contiguous
+    int n_gh = 1;
     int64_t total_tokens = 0;
+    int n_ctas() const { return int(cta_span_start.size()) - 1; }
     size_t table_bytes() const {
-        return align_up(segs.size() * sizeof(Seg), 16) + align_up(items.size() * sizeof(Item), 16) +
-               align_up(row_item_start.size() * sizeof(int32_t), 16);
+        return align_up(segs.size() * sizeof(Seg), 16) + align_up(spans.size() * sizeof(Span), 16) +
+               align_up(cta_span_start.size() * sizeof(int32_t), 16) + align_up(rg_span_start.size() * sizeof(int32_t), 16);
     }
     void serialize(char* dst) const {
         size_t o = 0;
         if (!segs.empty()) std::memcpy(dst + o, segs.data(), segs.size() * sizeof(Seg));
         o += align_up(segs.size() * sizeof(Seg), 16);
-        if (!items.empty()) std::memcpy(dst + o, items.data(), items.size() * sizeof(Item));
-        o += align_up(items.size() * sizeof(Item), 16);
-        std::memcpy(dst + o, row_item_start.data(), row_item_start.size() * sizeof(int32_t));
+        if (!spans.empty()) std::memcpy(dst + o, spans.data(), spans.size() * sizeof(Span));
+        o += align_up(spans.size() * sizeof(Span), 16);
+        std::memcpy(dst + o, cta_span_start.data(), cta_span_start.size() * sizeof(int32_t));
+        o += align_up(cta_span_start.size() * sizeof(int32_t), 16);
+        std::memcpy(dst + o, rg_span_start.data(), rg_span_start.size() * sizeof(int32_t));
     }
 };
 
-// Number of pieces a run of `nt` tiles is cut into when items hold at most `per` tiles, and the largest piece.
-inline int64_t pieces_of(int64_t nt, int64_t per) { return (nt + per - 1) / per; }
-
-// Tiles per item. With kv_splits > 0 the longest row is cut into that many pieces. Otherwise the size is
-// searched so that the grid (items x heads_per_tile CTAs, ctas_per_sm resident per SM) runs in as few
-// equally loaded waves as possible: cost = waves x (largest piece + a fixed per-CTA overhead in tile units).
-inline int tiles_per_item(const std::vector<int64_t>& seg_tiles, int64_t max_row_tiles, int heads_per_tile,
-                          int kv_splits, int ctas_per_sm) {
-    if (kv_splits > 0) return int(std::max<int64_t>(1, (max_row_tiles + kv_splits - 1) / kv_splits));
-    const int64_t slots = int64_t(kSmCount) * ctas_per_sm;
-    int64_t longest = 1;
-    for (int64_t nt : seg_tiles) longest = std::max(longest, nt);
-    int best = 1;
-    double best_cost = 1e300;
-    const int64_t hi = std::min<int64_t>(longest, 4 * kTargetTilesPerItem);
-    for (int64_t per = 1; per <= hi; ++per) {
-        int64_t items = 0, biggest = 0;
-        for (int64_t nt : seg_tiles) {
-            const int64_t pc = pieces_of(nt, per);
-            items += pc;
-            biggest = std::max(biggest, (nt + pc - 1) / pc);
-        }
-        const int64_t waves = (items * heads_per_tile + slots - 1) / slots;
-        const double cost = double(waves) * (double(biggest) + 2.0);     // ~2 tiles of fixed cost per CTA
-        if (cost < best_cost - 1e-9 || (cost < best_cost + 1e-9 && per > best)) { best_cost = cost; best = int(per); }
-    }
-    return best;
+// Upper bound on the number of spans build_plan can produce.
+inline int64_t max_spans_bound(int n_rows, int n_runs, int n_gh, int kv_splits, int ctas_per_sm) {
+    const int64_t pieces = int64_t(n_runs) * n_gh;               // one span per (row, head group, run) at least
+    if (kv_splits > 0) return pieces * (int64_t(kv_splits) + 1) + n_rows;
+    return pieces + int64_t(kSmCount) * ctas_per_sm + n_rows;    // plus one cut per CTA boundary
 }
 
-// rows[r] = segments of row r. Produces the device tables' host image.
-inline void build_plan(const std::vector<std::vector<PlanSeg>>& rows, int heads_per_tile, int kv_splits, int ctas_per_sm, Plan* plan) {
-    plan->segs.clear(); plan->items.clear(); plan->row_item_start.clear();
-    int64_t max_row_tiles = 0, total_tokens = 0;
-    std::vector<int64_t> seg_tiles;
-    for (const auto& row : rows) {
+// rows[r] = runs of row r.  n_gh = head groups per row.  kv_splits = 0: one balanced chunk per CTA slot;
+// kv_splits > 0: every (row, head group) is cut into about that many spans of equal length, one span per CTA
+// while they last (more spans than slots: several spans per CTA, still balanced).
+inline void build_plan(const std::vector<std::vector<PlanSeg>>& rows, int n_gh, int kv_splits, int ctas_per_sm, Plan* plan) {
+    plan->segs.clear(); plan->spans.clear(); plan->cta_span_start.clear(); plan->rg_span_start.clear();
+    plan->n_gh = n_gh;
+    const int64_t slots = int64_t(kSmCount) * ctas_per_sm;
+    // segments, and the tiles of every row
+    std::vector<std::vector<int32_t>> row_segs(rows.size());
+    int64_t total_tokens = 0, row_tiles_sum = 0, max_row_tiles = 0;
+    for (size_t r = 0; r < rows.size(); ++r) {
         int64_t rt = 0;
-        for (const auto& s : row) {
+        for (const auto& s : rows[r]) {
             if (s.n_tokens <= 0) continue;
-            const int64_t nt = (s.n_tokens + kTileTokens - 1) / kTileTokens;
-            seg_tiles.push_back(nt);
-            rt += nt;
+            row_segs[r].push_back(int32_t(plan->segs.size()));
+            plan->segs.push_back(Seg{s.off, int32_t(s.n_tokens), s.base_id});
+            rt += (s.n_tokens + kTileTokens - 1) / kTileTokens;
             total_tokens += s.n_tokens;
         }
+        row_tiles_sum += rt;
         max_row_tiles = std::max(max_row_tiles, rt);
     }
     plan->total_tokens = total_tokens;
-    const int per = tiles_per_item(seg_tiles, max_row_tiles, heads_per_tile, kv_splits, ctas_per_sm);
-    for (size_t r = 0; r < rows.size(); ++r) {
-        plan->row_item_start.push_back(int32_t(plan->items.size()));
-        for (const auto& s : rows[r]) {
-            if (s.n_tokens <= 0) continue;
-            const int32_t seg_id = int32_t(plan->segs.size());
-            plan->segs.push_back(Seg{s.off, int32_t(s.n_tokens), s.base_id});
-            const int64_t nt = (s.n_tokens + kTileTokens - 1) / kTileTokens;
-            // equal-sized pieces, so that no piece is a short straggler
-            const int64_t pieces = (nt + per - 1) / per;
-            int64_t t0 = 0;
-            for (int64_t k = 0; k < pieces; ++k) {
-                const int64_t cnt = nt / pieces + (k < nt % pieces ? 1 : 0);
-                plan->items.push_back(Item{int32_t(r), seg_id, int32_t(t0), int32_t(cnt)});
-                t0 += cnt;
+    const int64_t units = row_tiles_sum * n_gh;
+    // span length limit: kv_splits cuts rows explicitly; otherwise spans are only cut at CTA chunk boundaries
+    const int64_t piece = kv_splits > 0 ? std::max<int64_t>(1, (max_row_tiles + kv_splits - 1) / kv_splits) : INT64_MAX;
+
+    // pass 1: spans in (row, head group, run, tile) order, cut every `piece` tiles (kv_splits) ...
+    struct Raw { int32_t row, gh, seg, tile0, ntiles; };
+    std::vector<Raw> raw;
+    for (size_t r = 0; r < rows.size(); ++r)
+        for (int gh = 0; gh < n_gh; ++gh)
+            for (int32_t sid : row_segs[r]) {
+                const int64_t nt = (int64_t(plan->segs[sid].n_tokens) + kTileTokens - 1) / kTileTokens;
+                const int64_t pieces = (piece == INT64_MAX) ? 1 : (nt + piece - 1) / piece;
+                int64_t t0 = 0;
+                for (int64_t k = 0; k < pieces; ++k) {
+                    const int64_t cnt = nt / pieces + (k < nt % pieces ? 1 : 0);
+                    raw.push_back(Raw{int32_t(r), gh, sid, int32_t(t0), int32_t(cnt)});
+                    t0 += cnt;
+                }
             }
+    // ... pass 2: assign units to CTAs in equal contiguous chunks, cutting spans at chunk boundaries
+    int64_t n_ctas = std::min<int64_t>(slots, kv_splits > 0 ? int64_t(raw.size()) : units);
+    if (n_ctas < 1) n_ctas = units > 0 ? 1 : 0;
+    plan->cta_span_start.push_back(0);
+    int64_t done = 0;            // units assigned so far
+    int64_t cta = 0;
+    auto chunk_end = [&](int64_t c) { return (units * (c + 1)) / n_ctas; };   // balanced: differs by at most one unit
+    for (const Raw& rw : raw) {
+        int64_t t0 = rw.tile0, left = rw.ntiles;
+        while (left > 0) {
+            while (cta < n_ctas - 1 && done >= chunk_end(cta)) { plan->cta_span_start.push_back(int32_t(plan->spans.size())); ++cta; }
+            const int64_t room = (cta == n_ctas - 1) ? left : std::min<int64_t>(left, chunk_end(cta) - done);
+            plan->spans.push_back(Span{rw.row, rw.gh, rw.seg, int32_t(t0), int32_t(room)});
+            t0 += room; left -= room; done += room;
         }
     }
-    plan->row_item_start.push_back(int32_t(plan->items.size()));
+    while (int64_t(plan->cta_span_start.size()) < n_ctas + 1) plan->cta_span_start.push_back(int32_t(plan->spans.size()));
+    if (n_ctas == 0) plan->cta_span_start.assign(1, 0);
+    // spans of every (row, head group): contiguous because of the emission order
+    plan->rg_span_start.assign(rows.size() * size_t(n_gh) + 1, 0);
+    {
+        size_t k = 0;
+        for (size_t r = 0; r < rows.size(); ++r)
+            for (int gh = 0; gh < n_gh; ++gh) {
+                plan->rg_span_start[r * n_gh + gh] = int32_t(k);
+                while (k < plan->spans.size() && plan->spans[k].row == int32_t(r) && plan->spans[k].gh == gh) ++k;
+            }
+        plan->rg_span_start[rows.size() * size_t(n_gh)] = int32_t(k);
+    }
 }
 
 }  // namespace ipkvi

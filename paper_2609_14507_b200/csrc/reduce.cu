@@ -15,25 +15,40 @@ namespace {
 constexpr int kWarpsPerBlock = 4;
 constexpr int kReduceThreads = 256;
 
-// One CTA per (row, query head). Threads are arranged as (item slice, 4-column group): every thread sums the
-// weighted partials of its slice of the row's items for its four columns; the slices are then added through
-// shared memory. CG = dv / 4 column groups, SL = 256 / CG slices.
-__global__ void __launch_bounds__(kReduceThreads)
-split_reduce_kernel(const float* __restrict__ part_o, const float* __restrict__ part_lse,
-                    const int32_t* __restrict__ row_item_start, const float* acc_o, const float* acc_lse,
-                    float* out_o, float* out_lse, int Hq, int dv) {
+// One CTA per (row, query head). The partials to join are those of the spans of the head's group
+// (parts_per_span consecutive entries per span), row `rin` of each. Threads are arranged as
+// (entry slice, 4-column group): every thread sums the weighted partials of its slice for its four columns;
+// the slices are then added through shared memory. CG = dv / 4 column groups, SL = 256 / CG slices.
+struct ReduceParams {
+    const float* part_o;
+    const float* part_lse;
+    const int32_t* rg_span_start;
+    const float* acc_o;
+    const float* acc_lse;
+    float* out_o;
+    float* out_lse;
+    int Hq, dv, G, n_hg, n_gh, RG, NW;
+};
+
+__global__ void __launch_bounds__(kReduceThreads) split_reduce_kernel(const ReduceParams p) {
     extern __shared__ float4 red[];                 // [SL][CG]
     __shared__ float s_warp[kReduceThreads / 32];
     __shared__ float s_m;
-    __shared__ float s_zs[kReduceThreads / 16];    // weight sum of every item slice (SL <= 16)
+    __shared__ float s_zs[kReduceThreads / 16];    // weight sum of every entry slice (SL <= 16)
     const int wid = blockIdx.x;                      // row * Hq + h
-    const int row = wid / Hq, h = wid - row * Hq;
+    const int row = wid / p.Hq, h = wid - row * p.Hq;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int i0 = row_item_start[row], i1 = row_item_start[row + 1];
-    const float la = acc_lse ? acc_lse[wid] : -INFINITY;
+    const int g = h / p.G, hin = h - g * p.G;
+    const int gh = g * p.n_hg + hin / 16, rin = hin % 16;
+    const int sp0 = p.rg_span_start[row * p.n_gh + gh], sp1 = p.rg_span_start[row * p.n_gh + gh + 1];
+    const int64_t e0 = int64_t(sp0) * p.NW;
+    const int n = (sp1 - sp0) * p.NW;
+    const int dv = p.dv;
+    const float la = p.acc_lse ? p.acc_lse[wid] : -INFINITY;
+    const float* lse_base = p.part_lse + e0 * p.RG + rin;          // entry e at lse_base[e * RG]
 
     float m = la;
-    for (int i = i0 + tid; i < i1; i += kReduceThreads) m = fmaxf(m, part_lse[int64_t(i) * Hq + h]);
+    for (int e = tid; e < n; e += kReduceThreads) m = fmaxf(m, lse_base[int64_t(e) * p.RG]);
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, d));
     if (lane == 0) s_warp[warp] = m;
@@ -47,21 +62,23 @@ split_reduce_kernel(const float* __restrict__ part_o, const float* __restrict__ 
     m = s_m;
     const int CG = dv >> 2, SL = kReduceThreads / CG;
     const int cg = tid % CG, sl = tid / CG;
-    float* oo = out_o + int64_t(wid) * dv;
+    float* oo = p.out_o + int64_t(wid) * dv;
     if (m == -INFINITY) {                           // nothing attended: (0, -inf)
         if (sl == 0) *reinterpret_cast<float4*>(oo + cg * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (tid == 0) out_lse[wid] = -INFINITY;
+        if (tid == 0) p.out_lse[wid] = -INFINITY;
         return;
     }
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float z = 0.f;
     {
-        const float* po = part_o + int64_t(h) * dv + cg * 4;
-        const int64_t stride = int64_t(Hq) * dv;
+        const float* po = p.part_o + (e0 * p.RG + rin) * dv + cg * 4;
+        const int64_t stride = int64_t(p.RG) * dv;
 #pragma unroll 4
-        for (int i = i0 + sl; i < i1; i += SL) {
-            const float w = __expf(part_lse[int64_t(i) * Hq + h] - m);
-            const float4 v = *reinterpret_cast<const float4*>(po + int64_t(i) * stride);
+        for (int e = sl; e < n; e += SL) {
+            const float li = lse_base[int64_t(e) * p.RG];
+            if (li == -INFINITY) continue;          // a warp that saw no valid token
+            const float w = __expf(li - m);
+            const float4 v = *reinterpret_cast<const float4*>(po + int64_t(e) * stride);
             acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
             z += w;
         }
@@ -78,7 +95,7 @@ split_reduce_kernel(const float* __restrict__ part_o, const float* __restrict__ 
         }
         const float wa = (la == -INFINITY) ? 0.f : __expf(la - m);
         if (wa != 0.f) {
-            const float4 v = *reinterpret_cast<const float4*>(acc_o + int64_t(wid) * dv + cg * 4);
+            const float4 v = *reinterpret_cast<const float4*>(p.acc_o + int64_t(wid) * dv + cg * 4);
             t.x += wa * v.x; t.y += wa * v.y; t.z += wa * v.z; t.w += wa * v.w;
         }
         float zt = wa;
@@ -86,7 +103,7 @@ split_reduce_kernel(const float* __restrict__ part_o, const float* __restrict__ 
         const float inv = 1.f / zt;
         t.x *= inv; t.y *= inv; t.z *= inv; t.w *= inv;
         *reinterpret_cast<float4*>(oo + cg * 4) = t;
-        if (cg == 0) out_lse[wid] = m + logf(zt);
+        if (cg == 0) p.out_lse[wid] = m + logf(zt);
     }
 }
 
@@ -138,9 +155,16 @@ cudaError_t launch_split_reduce(const AttnLaunch& a, cudaStream_t s) {
     const int total = a.n_rows * a.n_q_heads;
     if (total <= 0) return cudaSuccess;
     if (a.dim_v % 4 != 0 || a.dim_v / 4 > kReduceThreads || kReduceThreads % (a.dim_v / 4) != 0) return cudaErrorInvalidValue;
+    const PartGeom pg = part_geom(a.kind, a.n_q_heads, a.n_kv_heads);
+    ReduceParams p;
+    p.part_o = a.part_o; p.part_lse = a.part_lse; p.rg_span_start = a.rg_span_start;
+    p.acc_o = a.acc_o; p.acc_lse = a.acc_lse; p.out_o = a.out_o; p.out_lse = a.out_lse;
+    p.Hq = a.n_q_heads; p.dv = a.dim_v;
+    p.G = a.kind == 1 ? a.n_q_heads : a.n_q_heads / a.n_kv_heads;
+    p.n_hg = (p.G + 15) / 16;
+    p.n_gh = pg.n_gh; p.RG = pg.rows_per_group; p.NW = pg.parts_per_span;
     const size_t smem = size_t(kReduceThreads) * sizeof(float4);
-    split_reduce_kernel<<<total, kReduceThreads, smem, s>>>(a.part_o, a.part_lse, a.row_item_start, a.acc_o, a.acc_lse,
-                                                           a.out_o, a.out_lse, a.n_q_heads, a.dim_v);
+    split_reduce_kernel<<<total, kReduceThreads, smem, s>>>(p);
     return cudaGetLastError();
 }
 

@@ -43,22 +43,28 @@ void shim_router_dump(void* r, int8_t* region, int64_t* blk, int32_t* off) {
     }
 }
 
-// plan: rows given as flat (row_start[n_rows+1], n_tokens[n_segs]); returns counts, fills arrays up to cap
-int shim_plan(int n_rows, const int32_t* row_start, const int64_t* seg_tokens, int heads_per_tile, int kv_splits,
-              int cap_items, int32_t* item_row, int32_t* item_seg, int32_t* item_tile0, int32_t* item_ntiles,
-              int32_t* row_item_start, int32_t* seg_tokens_out, int* n_segs_out) {
+// plan: rows given as flat (row_start[n_rows+1], n_tokens[n_segs]); fills the span table and the two index arrays
+int shim_plan(int n_rows, const int32_t* row_start, const int64_t* seg_tokens, int n_gh, int kv_splits, int ctas_per_sm,
+              int cap_spans, int32_t* span_fields /* [cap][5] */, int32_t* cta_span_start /* [<= 148*ctas_per_sm + 1] */,
+              int* n_ctas_out, int32_t* rg_span_start /* [n_rows*n_gh + 1] */, int32_t* seg_tokens_out, int* n_segs_out) {
     std::vector<std::vector<PlanSeg>> rows(n_rows);
     for (int r = 0; r < n_rows; ++r)
         for (int k = row_start[r]; k < row_start[r + 1]; ++k) rows[r].push_back(PlanSeg{0, int64_t(k) * 4096, seg_tokens[k]});
     Plan plan;
-    build_plan(rows, heads_per_tile, kv_splits, 2, &plan);
-    const int n = int(plan.items.size());
-    if (n > cap_items) return -n;
+    build_plan(rows, n_gh, kv_splits, ctas_per_sm, &plan);
+    const int n = int(plan.spans.size());
+    if (n > cap_spans) return -n;
+    int n_runs = 0;
+    for (int r = 0; r < n_rows; ++r) n_runs += row_start[r + 1] - row_start[r];
+    if (n > max_spans_bound(n_rows, n_runs, n_gh, kv_splits, ctas_per_sm)) return -1000000;   // the bound must hold
     for (int i = 0; i < n; ++i) {
-        item_row[i] = plan.items[i].row; item_seg[i] = plan.items[i].seg;
-        item_tile0[i] = plan.items[i].tile0; item_ntiles[i] = plan.items[i].ntiles;
+        const Span& sp = plan.spans[i];
+        int32_t* f = span_fields + 5 * i;
+        f[0] = sp.row; f[1] = sp.gh; f[2] = sp.seg; f[3] = sp.tile0; f[4] = sp.ntiles;
     }
-    for (int r = 0; r <= n_rows; ++r) row_item_start[r] = plan.row_item_start[r];
+    *n_ctas_out = plan.n_ctas();
+    for (size_t c = 0; c < plan.cta_span_start.size(); ++c) cta_span_start[c] = plan.cta_span_start[c];
+    for (size_t c = 0; c < plan.rg_span_start.size(); ++c) rg_span_start[c] = plan.rg_span_start[c];
     *n_segs_out = int(plan.segs.size());
     for (size_t k = 0; k < plan.segs.size(); ++k) seg_tokens_out[k] = plan.segs[k].n_tokens;
     return n;

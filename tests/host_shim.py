@@ -33,7 +33,7 @@ def lib():
         L.shim_router_len.restype = C.c_int64
         L.shim_router_counts.argtypes = [C.c_void_p, C.c_void_p]
         L.shim_router_dump.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
-        L.shim_plan.argtypes = [C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int] + [C.c_void_p] * 7
+        L.shim_plan.argtypes = [C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int] + [C.c_void_p] * 6
         L.shim_plan.restype = C.c_int
         L.shim_tile_chunk_offset.argtypes = [C.c_int32] * 3
         L.shim_tile_chunk_offset.restype = C.c_int64
@@ -84,8 +84,8 @@ class Router:
         return region, blk, off
 
 
-def plan(rows, heads_per_tile, kv_splits=0):
-    """rows: list of lists of segment token counts -> dict of the planner's tables."""
+def plan(rows, n_gh, kv_splits=0, ctas_per_sm=2):
+    """rows: list of lists of run token counts -> dict of the planner's tables."""
     row_start = np.zeros(len(rows) + 1, dtype=np.int32)
     segs = []
     for r, row in enumerate(rows):
@@ -93,13 +93,14 @@ def plan(rows, heads_per_tile, kv_splits=0):
         row_start[r + 1] = len(segs)
     seg_tokens = np.asarray(segs + [0], dtype=np.int64)
     cap = 1 << 16
-    a = [np.zeros(cap, dtype=np.int32) for _ in range(4)]
-    ris = np.zeros(len(rows) + 1, dtype=np.int32)
+    fields = np.zeros((cap, 5), dtype=np.int32)
+    cta = np.zeros(148 * ctas_per_sm + 2, dtype=np.int32)
+    rg = np.zeros(len(rows) * n_gh + 1, dtype=np.int32)
     seg_out = np.zeros(len(segs) + 1, dtype=np.int32)
-    n_segs = C.c_int()
-    n = lib().shim_plan(len(rows), row_start.ctypes.data, seg_tokens.ctypes.data, heads_per_tile, kv_splits, cap,
-                        a[0].ctypes.data, a[1].ctypes.data, a[2].ctypes.data, a[3].ctypes.data, ris.ctypes.data,
-                        seg_out.ctypes.data, C.byref(n_segs))
-    assert n >= 0
-    return dict(row=a[0][:n], seg=a[1][:n], tile0=a[2][:n], ntiles=a[3][:n], row_item_start=ris,
-                seg_tokens=seg_out[:n_segs.value])
+    n_segs, n_ctas = C.c_int(), C.c_int()
+    n = lib().shim_plan(len(rows), row_start.ctypes.data, seg_tokens.ctypes.data, n_gh, kv_splits, ctas_per_sm, cap,
+                        fields.ctypes.data, cta.ctypes.data, C.byref(n_ctas), rg.ctypes.data, seg_out.ctypes.data, C.byref(n_segs))
+    assert n >= 0, n
+    f = fields[:n]
+    return dict(row=f[:, 0], gh=f[:, 1], seg=f[:, 2], tile0=f[:, 3], ntiles=f[:, 4], cta_span_start=cta[:n_ctas.value + 1],
+                rg_span_start=rg, seg_tokens=seg_out[:n_segs.value])

@@ -57,43 +57,55 @@ def test_router_matches_oracle_on_paper_shaped_runs():
 
 def test_plan_covers_every_tile_exactly_once():
     rng = np.random.default_rng(32)
-    for trial in range(40):
+    for trial in range(60):
         n_rows = int(rng.integers(1, 20))
         rows = [[int(x) for x in rng.integers(0, 5000, size=rng.integers(0, 4))] for _ in range(n_rows)]
-        heads = int(rng.choice([1, 4, 8]))
+        n_gh = int(rng.choice([1, 4, 8]))
         splits = int(rng.choice([0, 0, 1, 3, 16]))
-        p = host_shim.plan(rows, heads, splits)
+        cps = int(rng.choice([1, 2]))
+        p = host_shim.plan(rows, n_gh, splits, cps)
         live = [[n for n in row if n > 0] for row in rows]
         assert list(p["seg_tokens"]) == [n for row in live for n in row]
-        assert p["row_item_start"][0] == 0 and p["row_item_start"][-1] == len(p["row"])
-        seg_id = 0
+        n_spans = len(p["row"])
+        css, rgs = p["cta_span_start"], p["rg_span_start"]
+        assert css[0] == 0 and css[-1] == n_spans and np.all(np.diff(css) >= 0) and len(css) - 1 <= 148 * cps
+        assert rgs[0] == 0 and rgs[-1] == n_spans and np.all(np.diff(rgs) >= 0)
+        assert np.all(p["ntiles"] >= 1)
+        seg_id0 = 0
         for r, row in enumerate(live):
-            i0, i1 = p["row_item_start"][r], p["row_item_start"][r + 1]
-            assert np.all(p["row"][i0:i1] == r)
-            covered = {}
-            for i in range(i0, i1):
-                assert p["ntiles"][i] >= 1
-                covered.setdefault(int(p["seg"][i]), []).append((int(p["tile0"][i]), int(p["ntiles"][i])))
-            for n in row:
-                pieces = sorted(covered.pop(seg_id))
-                t = 0
-                for t0, cnt in pieces:
-                    assert t0 == t
-                    t += cnt
-                assert t == -(-n // 64)
-                sizes = [c for _, c in pieces]
-                assert max(sizes) - min(sizes) <= 1          # balanced pieces
-                seg_id += 1
-            assert not covered
+            for gh in range(n_gh):
+                k0, k1 = rgs[r * n_gh + gh], rgs[r * n_gh + gh + 1]
+                assert np.all(p["row"][k0:k1] == r) and np.all(p["gh"][k0:k1] == gh)
+                covered = {}
+                for k in range(k0, k1):
+                    covered.setdefault(int(p["seg"][k]), []).append((int(p["tile0"][k]), int(p["ntiles"][k])))
+                for j, n in enumerate(row):
+                    t = 0
+                    for t0, cnt in sorted(covered.pop(seg_id0 + j)):
+                        assert t0 == t
+                        t += cnt
+                    assert t == -(-n // 64)
+                assert not covered
+            seg_id0 += len(row)
+        # every CTA gets the same number of tiles (within one) when the planner balances freely
+        loads = np.array([p["ntiles"][css[c]:css[c + 1]].sum() for c in range(len(css) - 1)])
+        if loads.size:
+            assert loads.sum() == p["ntiles"].sum()
+            assert loads.max() - loads.min() <= 1, (loads.min(), loads.max(), splits)
 
 
-def test_plan_fills_the_machine_in_whole_waves():
-    # Qwen3-shaped step: 16 rows x 32769 tokens, 4 KV heads -> CTAs = items * 4 close to a multiple of 296
+def test_plan_fills_the_machine_in_one_balanced_wave():
+    # Qwen3-shaped step: 16 rows x (32512 resident + 257 window tokens), 4 KV heads: 296 CTAs, equal loads
     p = host_shim.plan([[32768 - 256, 257]] * 16, 4)
-    ctas = len(p["row"]) * 4
-    waves = -(-ctas // 296)
-    assert 3 <= waves <= 10 and ctas / (waves * 296) >= 0.9      # the last wave is nearly full
-    assert p["ntiles"].max() <= 64
+    css = p["cta_span_start"]
+    assert len(css) - 1 == 296
+    loads = np.array([p["ntiles"][css[c]:css[c + 1]].sum() for c in range(296)])
+    assert loads.max() - loads.min() <= 1 and loads.sum() == 16 * 4 * (508 + 5)
+    # few spans: one cut per CTA boundary plus one per (row, head, run)
+    assert len(p["row"]) <= 296 + 16 * 4 * 2
+    # a tiny launch uses as many CTAs as it has tiles
+    p = host_shim.plan([[100], [1]], 4)
+    assert len(p["cta_span_start"]) - 1 == 4 * (2 + 1)
 
 
 def test_layout_arithmetic_matches_header_formula():
