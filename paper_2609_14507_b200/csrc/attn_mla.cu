@@ -260,15 +260,21 @@ __global__ void __launch_bounds__(kThreads, 1) attn_mla_kernel(const MlaParams p
                     ptx::ldmatrix_x4(s_phi + poff, ph[0], ph[1], ph[2], ph[3]);
                     ptx::ldmatrix_x4(s_plo + poff, pl[0], pl[1], pl[2], pl[3]);
                     const int tok = kk * 16 + (mi & 1) * 8 + r8;
+                    // all value fragments first, then the p_hi products, then the p_lo products: two MMAs on the
+                    // same accumulator are eight instructions apart
+                    uint32_t vf[4][4];
+#pragma unroll
+                    for (int jj = 0; jj < 4; ++jj)
+                        ptx::ldmatrix_x4_trans(vb + tok * 128 + (((2 * jj + (mi >> 1)) ^ r8) << 4), vf[jj][0], vf[jj][1], vf[jj][2], vf[jj][3]);
 #pragma unroll
                     for (int jj = 0; jj < 4; ++jj) {
-                        const int chunk = 2 * jj + (mi >> 1);
-                        uint32_t b0, b1, b2, b3;
-                        ptx::ldmatrix_x4_trans(vb + tok * 128 + ((chunk ^ r8) << 4), b0, b1, b2, b3);
-                        ptx::mma_bf16(o[2 * jj], ph, b0, b1);
-                        ptx::mma_bf16(o[2 * jj + 1], ph, b2, b3);
-                        ptx::mma_bf16(o[2 * jj], pl, b0, b1);
-                        ptx::mma_bf16(o[2 * jj + 1], pl, b2, b3);
+                        ptx::mma_bf16(o[2 * jj], ph, vf[jj][0], vf[jj][1]);
+                        ptx::mma_bf16(o[2 * jj + 1], ph, vf[jj][2], vf[jj][3]);
+                    }
+#pragma unroll
+                    for (int jj = 0; jj < 4; ++jj) {
+                        ptx::mma_bf16(o[2 * jj], pl, vf[jj][0], vf[jj][1]);
+                        ptx::mma_bf16(o[2 * jj + 1], pl, vf[jj][2], vf[jj][3]);
                     }
                 }
             }
