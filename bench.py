@@ -252,6 +252,8 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--kv-splits", type=int, default=0)
+    ap.add_argument("--separate-merge", action="store_true",
+                    help="join the CPU-side partial with a separate ipkv_merge launch instead of inside the split reduce")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -284,7 +286,7 @@ def main():
     n_gpu0 = sum(lens) // B - n_cpu
     total_steps = 2 * (args.warmup + args.steps) + 8
     cache = make_cache(wl, local_rank, total_steps)
-    seq_ids = list(range(B))
+    seq_ids = binding.seq_id_array(list(range(B)))
     populate(cache, wl, dev, rank)
     g = torch.Generator(device=dev); g.manual_seed(77 + rank)
     bf = torch.bfloat16
@@ -298,16 +300,22 @@ def main():
         o_cpu.zero_(); lse_cpu.fill_(float("-inf"))
     o_part = torch.zeros((B, Hq, dv), device=dev)
     lse_part = torch.zeros((B, Hq), device=dev)
-    out = torch.zeros((NL, B * Hq, dv), device=dev, dtype=bf)
+    fused = not args.separate_merge
+    out = torch.zeros((NL, B * Hq, dv), device=dev, dtype=torch.float32 if fused else bf)
     out_lse = torch.zeros((B * Hq,), device=dev)
+    cur = torch.cuda.current_stream()
     bpt = sh.bytes_per_token
 
     def step():
         for layer in range(NL):
-            cache.append(layer, seq_ids, k_new[layer], None if v_new is None else v_new[layer])
-            cache.attend_gpu(layer, seq_ids, q[layer], o_part, lse_part, kv_splits=args.kv_splits)
-            cache.merge(B * Hq, dv, [o_part.view(B * Hq, dv), o_cpu[layer]], [lse_part.view(-1), lse_cpu[layer]],
-                        out[layer], out_lse, out_is_bf16=True)
+            cache.append(layer, seq_ids, k_new[layer], None if v_new is None else v_new[layer], stream=cur)
+            if fused:      # the CPU-side partial is joined inside the split reduce: out = merged (O, LSE)
+                cache.attend_gpu(layer, seq_ids, q[layer], out[layer], out_lse, kv_splits=args.kv_splits, stream=cur,
+                                 fold_o=o_cpu[layer], fold_lse=lse_cpu[layer])
+            else:
+                cache.attend_gpu(layer, seq_ids, q[layer], o_part, lse_part, kv_splits=args.kv_splits, stream=cur)
+                cache.merge(B * Hq, dv, [o_part.view(B * Hq, dv), o_cpu[layer]], [lse_part.view(-1), lse_cpu[layer]],
+                            out[layer], out_lse, out_is_bf16=True, stream=cur)
 
     def barrier():
         torch.cuda.synchronize()
@@ -371,7 +379,8 @@ def main():
         hq = q.cpu().pin_memory(); hk = k_new.cpu().pin_memory()
         hv = None if v_new is None else v_new.cpu().pin_memory()
         hoc = o_cpu.cpu().pin_memory(); hlc = lse_cpu.cpu().pin_memory()
-        hout = torch.zeros((NL, B * Hq, dv), dtype=bf).pin_memory()
+        hout = torch.zeros((NL, B * Hq, dv), dtype=out.dtype).pin_memory()
+        doc = torch.empty_like(o_cpu[0]); dlc = torch.empty_like(lse_cpu[0])
         dq = torch.empty_like(q[0]); dk = torch.empty_like(k_new[0]); dvn = None if v_new is None else torch.empty_like(v_new[0])
 
         def step_e2e():
@@ -380,11 +389,17 @@ def main():
                 dk.copy_(hk[layer], non_blocking=True)
                 if dvn is not None:
                     dvn.copy_(hv[layer], non_blocking=True)
-                cache.append(layer, seq_ids, dk, dvn)
-                cache.attend_gpu(layer, seq_ids, dq, o_part, lse_part, kv_splits=args.kv_splits)
-                # the CPU-side partial is handed over in pinned host memory; ipkv_merge copies it in
-                cache.merge(B * Hq, dv, [o_part.view(B * Hq, dv), hoc[layer]], [lse_part.view(-1), hlc[layer]],
-                            out[layer], out_lse, out_is_bf16=True)
+                cache.append(layer, seq_ids, dk, dvn, stream=cur)
+                if fused:
+                    doc.copy_(hoc[layer], non_blocking=True)
+                    dlc.copy_(hlc[layer], non_blocking=True)
+                    cache.attend_gpu(layer, seq_ids, dq, out[layer], out_lse, kv_splits=args.kv_splits, stream=cur,
+                                     fold_o=doc, fold_lse=dlc)
+                else:
+                    cache.attend_gpu(layer, seq_ids, dq, o_part, lse_part, kv_splits=args.kv_splits, stream=cur)
+                    # the CPU-side partial is handed over in pinned host memory; ipkv_merge copies it in
+                    cache.merge(B * Hq, dv, [o_part.view(B * Hq, dv), hoc[layer]], [lse_part.view(-1), hlc[layer]],
+                                out[layer], out_lse, out_is_bf16=True, stream=cur)
                 hout[layer].copy_(out[layer], non_blocking=True)
             torch.cuda.synchronize()
 
@@ -403,7 +418,7 @@ def main():
         tok2 = (s1["kv_bytes_attended"] - s0["kv_bytes_attended"]) // bpt
         h2d = NL * (hq[0].numel() * 2 + hk[0].numel() * 2 + (0 if hv is None else hv[0].numel() * 2) + hoc[0].numel() * 4 + hlc[0].numel() * 4)
         e2e = {"value": world * tok2 / (ms2 * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
-               "d2h_bytes_per_step": NL * hout[0].numel() * 2, "ms_per_step": ms2 / args.steps}
+               "d2h_bytes_per_step": NL * hout[0].numel() * hout.element_size(), "ms_per_step": ms2 / args.steps}
     status = cache.get_stats()["device_status"]
     if status != 0:
         raise RuntimeError("a kernel reported a timed-out wait; the numbers are invalid")
@@ -423,7 +438,8 @@ def main():
                        "cpu_share": f"{num0}/{den0}", "gpu_share_tokens_per_seq_mean": n_gpu0 + 1, "bytes_per_kv_token": bpt, "block_tokens": BLOCK, "window_tokens": WINDOW,
                        "gpu_share": "HBM-resident", "host_copies_of_U_and_P": "off (benchmark)", "cpu_partial": "synthetic values",
                        "l2": "inputs larger than L2 (each layer reads its own %.2f GB)" % (bytes_attended / max(1, n_launch) / 1e9),
-                       "multi_gpu": "replicas only", "kv_splits": args.kv_splits},
+                       "multi_gpu": "replicas only", "kv_splits": args.kv_splits,
+                       "merge": "inside the split reduce" if fused else "separate ipkv_merge launch"},
             "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu,
             "step_gbs": world * bytes_attended / (ms * 1e-3) / 1e9,
         }

@@ -145,6 +145,12 @@ typedef struct {
   int32_t kv_splits;   /* 0 = automatic; otherwise the number of sequence chunks per (sequence, KV head) */
   int32_t reserved;
   void* side_stream;   /* stream for host-to-device chunk copies; NULL = the handle's own             */
+  /* Optional extra partial over a disjoint token set (typically the CPU-side partial, already on the
+     device): [n_seq][n_q_heads][dim_v] and [n_seq][n_q_heads] fp32.  When both are given it is folded in by
+     the same exact LSE join inside the split reduce, so the outputs are the MERGED (O, LSE) and no separate
+     ipkv_merge launch is needed for this step (Sec. 4.2: one join per step, performed on the GPU).        */
+  const float* fold_o_dev;
+  const float* fold_lse_dev;
 } ipkv_attend_opts;
 
 /* Attention over the GPU-side share (Sec. 5.1): the D-window plus every P token, device-resident ones

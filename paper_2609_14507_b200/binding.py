@@ -43,7 +43,8 @@ class Config(C.Structure):
 
 
 class AttendOpts(C.Structure):
-    _fields_ = [("kv_splits", C.c_int32), ("reserved", C.c_int32), ("side_stream", C.c_void_p)]
+    _fields_ = [("kv_splits", C.c_int32), ("reserved", C.c_int32), ("side_stream", C.c_void_p),
+                ("fold_o_dev", C.c_void_p), ("fold_lse_dev", C.c_void_p)]
 
 
 class Extent(C.Structure):
@@ -144,8 +145,15 @@ def _stream(stream):
 
 
 def _ids(seq_ids):
+    if isinstance(seq_ids, tuple) and len(seq_ids) == 2 and isinstance(seq_ids[1], int) and not isinstance(seq_ids[0], int):
+        return seq_ids                       # already marshalled by seq_id_array()
     arr = (C.c_int32 * len(seq_ids))(*[int(s) for s in seq_ids])
     return arr, len(seq_ids)
+
+
+def seq_id_array(seq_ids):
+    """Marshal a list of sequence ids once; the result can be passed wherever seq_ids is expected."""
+    return (C.c_int32 * len(seq_ids))(*[int(s) for s in seq_ids]), len(seq_ids)
 
 
 def make_config(kind, n_layers, max_seqs, n_q_heads, n_kv_heads, dim_qk, dim_v, *, block_tokens=64,
@@ -220,9 +228,10 @@ class Cache:
     def flush(self, layer=-1, seq=-1, stream=None):
         self._check(lib().ipkv_flush(self._h, layer, seq, _stream(stream)), "ipkv_flush")
 
-    def attend_gpu(self, layer, seq_ids, q, o_part, lse_part, kv_splits=0, side_stream=None, stream=None):
+    def attend_gpu(self, layer, seq_ids, q, o_part, lse_part, kv_splits=0, side_stream=None, stream=None,
+                   fold_o=None, fold_lse=None):
         ids, n = _ids(seq_ids)
-        opts = AttendOpts(kv_splits, 0, _stream(side_stream) if side_stream is not None else None)
+        opts = AttendOpts(kv_splits, 0, _stream(side_stream) if side_stream is not None else None, _ptr(fold_o), _ptr(fold_lse))
         self._check(lib().ipkv_attend_gpu(self._h, layer, ids, n, _ptr(q), C.byref(opts), _ptr(o_part), _ptr(lse_part),
                                           _stream(stream)), "ipkv_attend_gpu")
 

@@ -347,7 +347,8 @@ void fill_launch(AttnLaunch* a, int kind, int Hq, int Hkv, int dqk, int dv, int 
 
 // One group of segments for all rows: attention + split reduce, folding into (out_o, out_lse) when `fold`.
 ipkv_status run_group(ipkv* h, const std::vector<std::vector<PlanSeg>>& rows, const char* const bases[kMaxBases],
-                      const void* q, int kv_splits, bool fold, float* out_o, float* out_lse, cudaStream_t s) {
+                      const void* q, int kv_splits, const float* fold_o, const float* fold_lse, float* out_o, float* out_lse,
+                      cudaStream_t s) {
     const ipkv_config& c = h->cfg;
     Plan plan;
     const PartGeom pg = part_geom(c.kind, c.n_q_heads, c.n_kv_heads);
@@ -361,8 +362,8 @@ ipkv_status run_group(ipkv* h, const std::vector<std::vector<PlanSeg>>& rows, co
     fill_launch(&a, c.kind, c.n_q_heads, c.n_kv_heads, c.dim_qk, c.dim_v, c.block_tokens, h->scale, plan, table, h->scratch, q,
                 int(rows.size()));
     for (int i = 0; i < kMaxBases; ++i) a.bases[i] = bases[i];
-    a.acc_o = fold ? out_o : nullptr;
-    a.acc_lse = fold ? out_lse : nullptr;
+    a.acc_o = fold_o;
+    a.acc_lse = fold_lse;
     a.out_o = out_o; a.out_lse = out_lse;
     a.status = h->status_dev;
     if (a.n_spans > 0) {
@@ -668,7 +669,10 @@ ipkv_status ipkv_attend_gpu(ipkv_t* h, int32_t layer, const int32_t* seq_ids, in
         if (st.router.window_fill() > 0) rows[i].push_back(PlanSeg{1, h->w_off(seq), st.router.window_fill()});
     }
     const char* bases[kMaxBases] = {h->ring ? h->ring_layer(layer) : nullptr, h->w_layer(layer), h->pp_dev, nullptr};
-    ipkv_status rc = run_group(h, rows, bases, q_dev, kv_splits, false, o_part_dev, lse_part_dev, s);
+    const float* fold_o = opts ? opts->fold_o_dev : nullptr;
+    const float* fold_lse = opts ? opts->fold_lse_dev : nullptr;
+    if ((fold_o == nullptr) != (fold_lse == nullptr)) return fail(h, IPKV_EINVAL, "fold_o_dev and fold_lse_dev must be given together");
+    ipkv_status rc = run_group(h, rows, bases, q_dev, kv_splits, fold_o, fold_lse, o_part_dev, lse_part_dev, s);
     if (rc != IPKV_OK) return rc;
     if (max_stream_chunks == 0) return IPKV_OK;
 
@@ -699,7 +703,7 @@ ipkv_status ipkv_attend_gpu(ipkv_t* h, int32_t layer, const int32_t* seq_ids, in
         }
         CU(h, cudaEventRecord(h->slot_ready[slot], side));
         CU(h, cudaStreamWaitEvent(s, h->slot_ready[slot], 0));
-        rc = run_group(h, rows, bases, q_dev, kv_splits, true, o_part_dev, lse_part_dev, s);
+        rc = run_group(h, rows, bases, q_dev, kv_splits, o_part_dev, lse_part_dev, o_part_dev, lse_part_dev, s);
         if (rc != IPKV_OK) return rc;
         CU(h, cudaEventRecord(h->slot_free[slot], s));
         h->slot_free_set[slot] = 1;

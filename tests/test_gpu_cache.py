@@ -113,8 +113,13 @@ def test_config1_append_attend_merge():
         torch.cuda.synchronize()
         o_all, l_all = ref.attend(q[0], "all", scale)
         check_partial(out.cpu().numpy(), out_lse.cpu().numpy(), o_all, l_all, "merged")
+        # the same join folded into the split reduce: attend_gpu returns the merged result directly
+        o2 = torch.zeros((1, 32, 128), device=DEV); lse2 = torch.zeros((1, 32), device=DEV)
+        cache.attend_gpu(0, [0], qd, o2, lse2, fold_o=o_cpu_t.to(DEV), fold_lse=l_cpu_t.to(DEV))
+        torch.cuda.synchronize()
+        check_partial(o2.cpu().numpy()[0], lse2.cpu().numpy()[0], o_all, l_all, "merged inside the reduce")
         st = cache.get_stats()
-        assert st["device_status"] == 0 and st["attend_kernels"] == 1 and st["merge_kernels"] == 1
+        assert st["device_status"] == 0 and st["attend_kernels"] == 2 and st["merge_kernels"] == 1
 
 
 def test_merge_at_many_split_points_equals_unsplit():
