@@ -50,6 +50,16 @@ WORKLOADS = {
     # BASELINE config 1 (single layer, batch 1, 4K): latency-bound, for quick checks
     "small-gqa-bs1-4k-cpu50": dict(shape=synth.SMALL_GQA, batch=1, ctx=4096, share=(1, 2), cfg_id=1),
 }
+# dram__bytes_read.sum + dram__bytes_write.sum of one attention-kernel launch, from the ncu captures summarised under
+# profiles/ (captured on the 2-layer case, whose per-layer launch is the full-size workload's launch).
+DRAM_TRAFFIC_PER_LAUNCH = {
+    "mixtral-8x7b-bs16-32k-cpu25": 1615.1e6 + 6.7e6,        # profiles/attn_gqa_kernel_mixtral-2layers-bs16-32k-cpu25.md
+    "mixtral-2layers-bs16-32k-cpu25": 1615.1e6 + 6.7e6,
+    "qwen3-30b-a3b-bs16-32k-cpu0": 1076.2e6 + 6.6e6,        # profiles/attn_gqa_kernel_qwen3-2layers-bs16-32k-cpu0.md
+    "qwen3-2layers-bs16-32k-cpu0": 1076.2e6 + 6.6e6,
+    "deepseek-v2-lite-mla-bs8-128k-cpu40": 725.8e6 + 9.3e6,  # profiles/attn_mla_kernel_deepseek-v2-lite-2layers-bs8-128k-cpu40.md
+    "deepseek-v2-lite-mla-2layers-bs8-128k-cpu40": 725.8e6 + 9.3e6,
+}
 DEFAULT_WORKLOAD = "mixtral-8x7b-bs16-32k-cpu25"
 BLOCK, WINDOW = 64, 256
 
@@ -363,15 +373,7 @@ def main():
                 else "fallback 6650 GB/s", "unit": "GB/s", "frac": ach / peak, "frac_of_8000_nominal": ach / 8000.0,
                 "avg_launch_us": 1e3 * kern_ms / max(1, n_timed), "bytes_per_launch": bytes_attended / max(1, n_launch),
                 "traffic": None, "whole_step_gbs": world * bytes_attended / (ms * 1e-3) / 1e9}
-    traffic_path = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(traffic_path):
-        try:
-            with open(traffic_path) as f:
-                tj = json.load(f).get(args.workload)
-            if tj:
-                roofline["traffic"] = tj["dram_bytes_per_launch"]
-        except (OSError, ValueError, KeyError):
-            pass
+    roofline["traffic"] = DRAM_TRAFFIC_PER_LAUNCH.get(args.workload)
 
     # ---- end to end: host buffers in, host buffer out, through the same calls ---------------------------------
     e2e = None
