@@ -378,31 +378,32 @@ def main():
     # ---- end to end: host buffers in, host buffer out, through the same calls ---------------------------------
     e2e = None
     if not args.no_e2e:
+        # One step's inputs for all layers sit in pinned host memory (queries, new K/V tokens, the CPU engine's partials);
+        # each step copies them to the device (one copy per tensor), runs the path, and reads all layers' outputs back.
         hq = q.cpu().pin_memory(); hk = k_new.cpu().pin_memory()
         hv = None if v_new is None else v_new.cpu().pin_memory()
         hoc = o_cpu.cpu().pin_memory(); hlc = lse_cpu.cpu().pin_memory()
         hout = torch.zeros((NL, B * Hq, dv), dtype=out.dtype).pin_memory()
-        doc = torch.empty_like(o_cpu[0]); dlc = torch.empty_like(lse_cpu[0])
-        dq = torch.empty_like(q[0]); dk = torch.empty_like(k_new[0]); dvn = None if v_new is None else torch.empty_like(v_new[0])
+        dq = torch.empty_like(q); dk = torch.empty_like(k_new); dvn = None if v_new is None else torch.empty_like(v_new)
+        doc = torch.empty_like(o_cpu); dlc = torch.empty_like(lse_cpu)
 
         def step_e2e():
+            dq.copy_(hq, non_blocking=True)
+            dk.copy_(hk, non_blocking=True)
+            if dvn is not None:
+                dvn.copy_(hv, non_blocking=True)
+            doc.copy_(hoc, non_blocking=True)
+            dlc.copy_(hlc, non_blocking=True)
             for layer in range(NL):
-                dq.copy_(hq[layer], non_blocking=True)
-                dk.copy_(hk[layer], non_blocking=True)
-                if dvn is not None:
-                    dvn.copy_(hv[layer], non_blocking=True)
-                cache.append(layer, seq_ids, dk, dvn, stream=cur)
+                cache.append(layer, seq_ids, dk[layer], None if dvn is None else dvn[layer], stream=cur)
                 if fused:
-                    doc.copy_(hoc[layer], non_blocking=True)
-                    dlc.copy_(hlc[layer], non_blocking=True)
-                    cache.attend_gpu(layer, seq_ids, dq, out[layer], out_lse, kv_splits=args.kv_splits, stream=cur,
-                                     fold_o=doc, fold_lse=dlc)
+                    cache.attend_gpu(layer, seq_ids, dq[layer], out[layer], out_lse, kv_splits=args.kv_splits, stream=cur,
+                                     fold_o=doc[layer], fold_lse=dlc[layer])
                 else:
-                    cache.attend_gpu(layer, seq_ids, dq, o_part, lse_part, kv_splits=args.kv_splits, stream=cur)
-                    # the CPU-side partial is handed over in pinned host memory; ipkv_merge copies it in
-                    cache.merge(B * Hq, dv, [o_part.view(B * Hq, dv), hoc[layer]], [lse_part.view(-1), hlc[layer]],
+                    cache.attend_gpu(layer, seq_ids, dq[layer], o_part, lse_part, kv_splits=args.kv_splits, stream=cur)
+                    cache.merge(B * Hq, dv, [o_part.view(B * Hq, dv), doc[layer]], [lse_part.view(-1), dlc[layer]],
                                 out[layer], out_lse, out_is_bf16=True, stream=cur)
-                hout[layer].copy_(out[layer], non_blocking=True)
+            hout.copy_(out, non_blocking=True)
             torch.cuda.synchronize()
 
         for _ in range(args.warmup):

@@ -209,6 +209,26 @@ typedef struct {
 } ipkv_stats;
 ipkv_status ipkv_get_stats(ipkv_t* h, ipkv_stats* out);
 
+/* ---- roofline share policy (host only; Sec. 5.2-5.3) ------------------------------------------------
+ * Eq. 1: T_CPU(r) = r*A*L + C_cpu, T_GPU(r) = (1-r)*B*L + C_gpu, T = max(T_CPU, T_GPU) + T_merge.
+ * Eq. 2: r(L) = clamp01(B/(A+B) + (C_gpu - C_cpu)/((A+B)*L)); marginal share p = B/(A+B).
+ * A, B in seconds per KV token, overheads in seconds.  The policy keeps a sliding window of the CPU engine's
+ * per-step latencies (the paper uses 256 steps), back-computes A from them and returns the numerator of p over
+ * `share_den` for ipkv_set_share; B is calibrated once.  None of these calls touches a GPU. */
+typedef struct ipkv_policy ipkv_policy_t;
+typedef struct { double A, B, C_cpu, C_gpu; } ipkv_roofline;
+double ipkv_roofline_share(const ipkv_roofline* m, double L);                                   /* Eq. 2 */
+double ipkv_roofline_step_time(const ipkv_roofline* m, double r, double L, double t_merge,
+                               double* t_cpu_out, double* t_gpu_out);                           /* Eq. 1 */
+ipkv_status ipkv_policy_create(const ipkv_roofline* m, int32_t window_steps, int32_t share_den, ipkv_policy_t** out);
+ipkv_status ipkv_policy_destroy(ipkv_policy_t* p);
+/* one decode step of the CPU engine: its latency and the CPU-side KV tokens it attended */
+ipkv_status ipkv_policy_observe(ipkv_policy_t* p, double cpu_seconds, double cpu_tokens);
+/* re-estimate A, return the numerator of p = B/(A+B) over share_den and the current model */
+ipkv_status ipkv_policy_update(ipkv_policy_t* p, int32_t* share_num_out, ipkv_roofline* model_out);
+/* prefill share R(L0) = r(L0) as a numerator over share_den */
+ipkv_status ipkv_policy_prefill_share(const ipkv_policy_t* p, double L0, int32_t* share_num_out);
+
 /* Kernel timing for benchmarks.  While enabled, every attention-kernel launch of ipkv_attend_gpu is
  * bracketed by a pair of CUDA events on the launching stream.  ipkv_profile_read synchronises the device,
  * returns the summed kernel time (milliseconds) and the number of launches since the last read, and resets

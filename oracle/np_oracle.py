@@ -165,3 +165,28 @@ def footprint(bpt, n_layers, batch, seq, D, pingpong_tokens_per_seq, cpu_tokens_
     u = bpt * n_layers * batch * cpu_tokens_per_seq
     return dict(pingpong=bpt * batch * pingpong_tokens_per_seq, dwindow=bpt * n_layers * batch * D,
                 unpinned=u, pinned=full - u, full=full)
+
+
+# ---- roofline share model (Sec. 5.2-5.3) ----------------------------------------------------------------
+
+def engine_times(A, B, C_cpu, C_gpu, r, L):
+    """Eq. 1: (T_CPU, T_GPU) = (r A L + C_CPU, (1 - r) B L + C_GPU)."""
+    return r * A * L + C_cpu, (1.0 - r) * B * L + C_gpu
+
+
+def roofline_share(A, B, C_cpu, C_gpu, L):
+    """Eq. 2: r(L) = min(1, max(0, B/(A+B) + Delta/((A+B) L))), Delta = C_GPU - C_CPU."""
+    delta = C_gpu - C_cpu
+    return min(1.0, max(0.0, B / (A + B) + delta / ((A + B) * L)))
+
+
+def cumulative_share(p, R0, L0, L):
+    """Sec. 5.3: R(L) = p + (R(L0) - p) L0 / L."""
+    return p + (R0 - p) * L0 / L
+
+
+def estimate_A(latencies, cpu_tokens, C_cpu):
+    """Back-compute the CPU per-token cost from step latencies: T_CPU = A n + C_CPU summed over the window."""
+    latencies = np.asarray(latencies, dtype=np.float64)
+    cpu_tokens = np.asarray(cpu_tokens, dtype=np.float64)
+    return (latencies.sum() - latencies.size * C_cpu) / cpu_tokens.sum()

@@ -23,7 +23,8 @@ EXPORTS = [
     "ipkv_query_sizes", "ipkv_create", "ipkv_destroy", "ipkv_set_share", "ipkv_reset", "ipkv_append_bulk",
     "ipkv_append", "ipkv_flush", "ipkv_attend_gpu", "ipkv_merge", "ipkv_views", "ipkv_locate", "ipkv_counts",
     "ipkv_read_token", "ipkv_get_stats", "ipkv_profile_enable", "ipkv_profile_read", "ipkv_attend_scratch_bytes", "ipkv_attend_runs", "ipkv_pack_blocks",
-    "ipkv_attend_runs_noalloc", "ipkv_noalloc_scratch_limit",
+    "ipkv_attend_runs_noalloc", "ipkv_noalloc_scratch_limit", "ipkv_roofline_share", "ipkv_roofline_step_time",
+    "ipkv_policy_create", "ipkv_policy_destroy", "ipkv_policy_observe", "ipkv_policy_update", "ipkv_policy_prefill_share",
     "ipkv_block_bytes", "ipkv_status_str", "ipkv_last_error", "ipkv_version",
 ]
 
@@ -65,6 +66,10 @@ class AttnShape(C.Structure):
 
 class Run(C.Structure):
     _fields_ = [("blocks_dev", C.c_void_p), ("n_tokens", C.c_int64)]
+
+
+class Roofline(C.Structure):
+    _fields_ = [("A", C.c_double), ("B", C.c_double), ("C_cpu", C.c_double), ("C_gpu", C.c_double)]
 
 
 class IpkvError(RuntimeError):
@@ -115,6 +120,17 @@ def lib():
         f.restype = C.c_int
     L.ipkv_block_bytes.argtypes = [C.POINTER(AttnShape)]
     L.ipkv_block_bytes.restype = C.c_int64
+    L.ipkv_roofline_share.argtypes = [C.POINTER(Roofline), C.c_double]
+    L.ipkv_roofline_share.restype = C.c_double
+    L.ipkv_roofline_step_time.argtypes = [C.POINTER(Roofline), C.c_double, C.c_double, C.c_double, C.POINTER(C.c_double), C.POINTER(C.c_double)]
+    L.ipkv_roofline_step_time.restype = C.c_double
+    L.ipkv_policy_create.argtypes = [C.POINTER(Roofline), i32, i32, C.POINTER(vp)]
+    L.ipkv_policy_destroy.argtypes = [vp]
+    L.ipkv_policy_observe.argtypes = [vp, C.c_double, C.c_double]
+    L.ipkv_policy_update.argtypes = [vp, C.POINTER(i32), C.POINTER(Roofline)]
+    L.ipkv_policy_prefill_share.argtypes = [vp, C.c_double, C.POINTER(i32)]
+    for name in ("ipkv_policy_create", "ipkv_policy_destroy", "ipkv_policy_observe", "ipkv_policy_update", "ipkv_policy_prefill_share"):
+        getattr(L, name).restype = C.c_int
     L.ipkv_noalloc_scratch_limit.argtypes = []
     L.ipkv_noalloc_scratch_limit.restype = C.c_size_t
     L.ipkv_status_str.argtypes = [C.c_int]
@@ -288,6 +304,54 @@ def ipkv_merge(n_rows, dim_v, o_parts, lse_parts, o_out, lse_out=None, out_is_bf
     rc = lib().ipkv_merge(h, n_rows, dim_v, n, op, lp, _ptr(o_out), 1 if out_is_bf16 else 0, _ptr(lse_out), _stream(stream))
     if rc != OK:
         raise IpkvError(rc, "ipkv_merge", lib().ipkv_last_error(h).decode() if h else "")
+
+
+def ipkv_roofline_share(A, B, C_cpu, C_gpu, L):
+    """Eq. 2: the CPU share that balances the two engines at placed length L."""
+    return float(lib().ipkv_roofline_share(C.byref(Roofline(A, B, C_cpu, C_gpu)), L))
+
+
+def ipkv_roofline_step_time(A, B, C_cpu, C_gpu, r, L, t_merge=0.0):
+    """Eq. 1: (T, T_CPU, T_GPU) at share r."""
+    tc, tg = C.c_double(), C.c_double()
+    t = lib().ipkv_roofline_step_time(C.byref(Roofline(A, B, C_cpu, C_gpu)), r, L, t_merge, C.byref(tc), C.byref(tg))
+    return float(t), tc.value, tg.value
+
+
+class Policy:
+    """Owner of one ``ipkv_policy_t``: sliding-window feedback on the CPU cost A, marginal share p = B/(A+B)."""
+
+    def __init__(self, A, B, C_cpu, C_gpu, window_steps=256, share_den=64):
+        h = C.c_void_p()
+        rc = lib().ipkv_policy_create(C.byref(Roofline(A, B, C_cpu, C_gpu)), window_steps, share_den, C.byref(h))
+        if rc != OK:
+            raise IpkvError(rc, "ipkv_policy_create")
+        self._h = h
+
+    def __del__(self):
+        if getattr(self, "_h", None):
+            lib().ipkv_policy_destroy(self._h)
+            self._h = None
+
+    def observe(self, cpu_seconds, cpu_tokens):
+        rc = lib().ipkv_policy_observe(self._h, cpu_seconds, cpu_tokens)
+        if rc != OK:
+            raise IpkvError(rc, "ipkv_policy_observe")
+
+    def update(self):
+        """(share numerator, dict of the current model)."""
+        num, m = C.c_int32(), Roofline()
+        rc = lib().ipkv_policy_update(self._h, C.byref(num), C.byref(m))
+        if rc != OK:
+            raise IpkvError(rc, "ipkv_policy_update")
+        return num.value, dict(A=m.A, B=m.B, C_cpu=m.C_cpu, C_gpu=m.C_gpu)
+
+    def prefill_share(self, L0):
+        num = C.c_int32()
+        rc = lib().ipkv_policy_prefill_share(self._h, L0, C.byref(num))
+        if rc != OK:
+            raise IpkvError(rc, "ipkv_policy_prefill_share")
+        return num.value
 
 
 def make_shape(kind, n_q_heads, n_kv_heads, dim_qk, dim_v, block_tokens, softmax_scale=0.0):

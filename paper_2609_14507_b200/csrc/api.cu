@@ -22,6 +22,7 @@
 #include "../../include/ipkv.h"
 #include "kernels.h"
 #include "plan.hpp"
+#include "policy.hpp"
 #include "router.hpp"
 
 namespace ipkvi {
@@ -901,6 +902,64 @@ ipkv_status ipkv_profile_read(ipkv_t* h, double* attend_kernel_ms, int64_t* n_ti
     *n_timed = int64_t(h->prof_used / 2);
     *n_launches = h->prof_launches;
     h->prof_used = 0; h->prof_launches = 0;
+    return IPKV_OK;
+}
+
+// ---- roofline share policy (host only) ----------------------------------------------------------
+struct ipkv_policy {
+    SharePolicy impl;
+    ipkv_policy(const RooflineParams& m, int w, int d) : impl(m, w, d) {}
+};
+
+static bool roofline_ok(const ipkv_roofline* m) {
+    return m && m->A > 0.0 && m->B > 0.0 && std::isfinite(m->A) && std::isfinite(m->B) && std::isfinite(m->C_cpu) &&
+           std::isfinite(m->C_gpu) && m->C_cpu >= 0.0 && m->C_gpu >= 0.0;
+}
+
+double ipkv_roofline_share(const ipkv_roofline* m, double L) {
+    if (!roofline_ok(m)) return NAN;
+    return balanced_share(RooflineParams{m->A, m->B, m->C_cpu, m->C_gpu}, L);
+}
+
+double ipkv_roofline_step_time(const ipkv_roofline* m, double r, double L, double t_merge, double* t_cpu_out, double* t_gpu_out) {
+    if (!roofline_ok(m) || !(r >= 0.0 && r <= 1.0) || !(L >= 0.0)) return NAN;
+    const RooflineParams rp{m->A, m->B, m->C_cpu, m->C_gpu};
+    if (t_cpu_out) *t_cpu_out = engine_time_cpu(rp, r, L);
+    if (t_gpu_out) *t_gpu_out = engine_time_gpu(rp, r, L);
+    return step_time(rp, r, L, t_merge);
+}
+
+ipkv_status ipkv_policy_create(const ipkv_roofline* m, int32_t window_steps, int32_t share_den, ipkv_policy_t** out) {
+    if (!out) return IPKV_EINVAL;
+    *out = nullptr;
+    if (!roofline_ok(m) || window_steps <= 0 || share_den <= 0) return IPKV_EINVAL;
+    ipkv_policy* p = new (std::nothrow) ipkv_policy(RooflineParams{m->A, m->B, m->C_cpu, m->C_gpu}, window_steps, share_den);
+    if (!p) return IPKV_ENOMEM;
+    *out = p;
+    return IPKV_OK;
+}
+
+ipkv_status ipkv_policy_destroy(ipkv_policy_t* p) { delete p; return IPKV_OK; }
+
+ipkv_status ipkv_policy_observe(ipkv_policy_t* p, double cpu_seconds, double cpu_tokens) {
+    if (!p || !(cpu_seconds >= 0.0) || !(cpu_tokens >= 0.0) || !std::isfinite(cpu_seconds) || !std::isfinite(cpu_tokens)) return IPKV_EINVAL;
+    p->impl.observe(cpu_seconds, cpu_tokens);
+    return IPKV_OK;
+}
+
+ipkv_status ipkv_policy_update(ipkv_policy_t* p, int32_t* share_num_out, ipkv_roofline* model_out) {
+    if (!p || !share_num_out) return IPKV_EINVAL;
+    *share_num_out = p->impl.update();
+    if (model_out) {
+        const RooflineParams& m = p->impl.model();
+        model_out->A = m.A; model_out->B = m.B; model_out->C_cpu = m.C_cpu; model_out->C_gpu = m.C_gpu;
+    }
+    return IPKV_OK;
+}
+
+ipkv_status ipkv_policy_prefill_share(const ipkv_policy_t* p, double L0, int32_t* share_num_out) {
+    if (!p || !share_num_out || !(L0 >= 0.0)) return IPKV_EINVAL;
+    *share_num_out = p->impl.prefill_numerator(L0);
     return IPKV_OK;
 }
 
