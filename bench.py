@@ -447,7 +447,18 @@ def main():
             "step_gbs": world * bytes_attended / (ms * 1e-3) / 1e9,
         }
         if "stream_pct" in wl:
+            # the box's pinned host-to-device plateau, measured here with one 256 MB copy (best of 5)
+            hp = torch.empty(256 << 20, dtype=torch.uint8).pin_memory(); dp = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+            best = 1e9
+            for _ in range(5):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(); dp.copy_(hp, non_blocking=True); b.record(); torch.cuda.synchronize()
+                best = min(best, a.elapsed_time(b))
+            plateau = (256 << 20) / (best * 1e-3) / 1e9
+            t_h2d_ideal = h2d_stream / (plateau * 1e9) * 1e3          # ms over the timed region
             line["streaming"] = {"h2d_bytes_per_step": h2d_stream / args.steps, "h2d_gbs": h2d_stream / (ms * 1e-3) / 1e9,
+                                 "h2d_plateau_gbs": plateau, "attn_kernel_ms_per_step": kern_ms / args.steps,
+                                 "overlap_efficiency": max(t_h2d_ideal, kern_ms) / ms,
                                  "streamed_pct_of_p_share": wl["stream_pct"], "chunk_tokens": wl.get("chunk_tokens", 512)}
             line["config"]["gpu_share"] = "%d %% streamed H2D from pinned host memory each step, rest HBM-resident" % wl["stream_pct"]
             line["config"]["host_copies_of_U_and_P"] = "P on (pinned), U off"

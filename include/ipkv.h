@@ -162,6 +162,17 @@ ipkv_status ipkv_attend_gpu(ipkv_t* h, int32_t layer, const int32_t* seq_ids, in
                             const void* q_dev, const ipkv_attend_opts* opts,
                             float* o_part_dev, float* lse_part_dev, void* stream);
 
+/* CPU-side engine (Sec. 6.1): in-place attention over the CPU-side share, i.e. the tokens routed to region U,
+ * read where they lie (PLAIN blocks, no copy).  This is the paper's second engine, not a fallback for the GPU
+ * path: it attends a disjoint token range and its partial is joined by ipkv_merge / the fold option.
+ * q_host [n_seq][n_q_heads][dim_qk] bf16 in host memory; o_part_host [n_seq][n_q_heads][dim_v] and
+ * lse_part_host [n_seq][n_q_heads] fp32 in host memory (pinned memory lets the later copy to the GPU overlap).
+ * The call runs synchronously on the calling thread plus OpenMP workers (n_threads <= 0: all cores).
+ * U is filled by device-to-host copies queued by the append / flush calls: synchronise their stream first.
+ * Fails with IPKV_ESTATE if U contents are not kept (IPKV_FLAG_NO_HOST_U). */
+ipkv_status ipkv_attend_cpu(ipkv_t* h, int32_t layer, const int32_t* seq_ids, int32_t n_seq, const void* q_host,
+                            float* o_part_host, float* lse_part_host, int32_t n_threads);
+
 /* Exact n-way log-sum-exp join (Sec. 4.2, 5.1) of row-aligned partials over disjoint token sets:
  *   LSE = m + ln sum_i exp(LSE_i - m), m = max_i LSE_i;  O = sum_i exp(LSE_i - LSE) * O_i.
  * o_parts[i] [n_rows][dim_v] fp32, lse_parts[i] [n_rows] fp32; the pointer arrays are host memory;

@@ -21,7 +21,7 @@ STATUS_NAMES = {0: "OK", 1: "EINVAL", 2: "ENOMEM", 3: "ERANGE", 4: "ESTATE", 5: 
 
 EXPORTS = [
     "ipkv_query_sizes", "ipkv_create", "ipkv_destroy", "ipkv_set_share", "ipkv_reset", "ipkv_append_bulk",
-    "ipkv_append", "ipkv_flush", "ipkv_attend_gpu", "ipkv_merge", "ipkv_views", "ipkv_locate", "ipkv_counts",
+    "ipkv_append", "ipkv_flush", "ipkv_attend_gpu", "ipkv_attend_cpu", "ipkv_merge", "ipkv_views", "ipkv_locate", "ipkv_counts",
     "ipkv_read_token", "ipkv_get_stats", "ipkv_profile_enable", "ipkv_profile_read", "ipkv_attend_scratch_bytes", "ipkv_attend_runs", "ipkv_pack_blocks",
     "ipkv_attend_runs_noalloc", "ipkv_noalloc_scratch_limit", "ipkv_roofline_share", "ipkv_roofline_step_time",
     "ipkv_policy_create", "ipkv_policy_destroy", "ipkv_policy_observe", "ipkv_policy_update", "ipkv_policy_prefill_share",
@@ -101,6 +101,7 @@ def lib():
         "ipkv_append": [vp, i32, C.POINTER(i32), i32, vp, vp, vp],
         "ipkv_flush": [vp, i32, i32, vp],
         "ipkv_attend_gpu": [vp, i32, C.POINTER(i32), i32, vp, C.POINTER(AttendOpts), vp, vp, vp],
+        "ipkv_attend_cpu": [vp, i32, C.POINTER(i32), i32, vp, vp, vp, i32],
         "ipkv_merge": [vp, i32, i32, i32, C.POINTER(vp), C.POINTER(vp), vp, i32, vp, vp],
         "ipkv_views": [vp, i32, i32, C.POINTER(Extent), i32, C.POINTER(i32)],
         "ipkv_locate": [vp, i32, i32, i64, C.POINTER(i32), C.POINTER(i64), C.POINTER(i32)],
@@ -250,6 +251,12 @@ class Cache:
         opts = AttendOpts(kv_splits, 0, _stream(side_stream) if side_stream is not None else None, _ptr(fold_o), _ptr(fold_lse))
         self._check(lib().ipkv_attend_gpu(self._h, layer, ids, n, _ptr(q), C.byref(opts), _ptr(o_part), _ptr(lse_part),
                                           _stream(stream)), "ipkv_attend_gpu")
+
+    def attend_cpu(self, layer, seq_ids, q_host, o_part_host, lse_part_host, n_threads=0):
+        """CPU-side engine over the tokens routed to U; all tensors in host memory."""
+        ids, n = _ids(seq_ids)
+        self._check(lib().ipkv_attend_cpu(self._h, layer, ids, n, _ptr(q_host), _ptr(o_part_host), _ptr(lse_part_host), n_threads),
+                    "ipkv_attend_cpu")
 
     def merge(self, n_rows, dim_v, o_parts, lse_parts, o_out, lse_out=None, out_is_bf16=False, stream=None):
         ipkv_merge(n_rows, dim_v, o_parts, lse_parts, o_out, lse_out, out_is_bf16, stream, handle=self)

@@ -33,6 +33,11 @@ def build(force=False, verbose=False):
         cmd = [NVCC] + FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", src, "-o", obj]
         procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
         objs.append(obj)
+    for src in sorted(glob.glob(os.path.join(CSRC, "*.cpp"))):          # host-only parts (the CPU-side engine)
+        obj = os.path.join(OBJ_DIR, os.path.basename(src)[:-4] + ".o")
+        cmd = ["g++", "-std=c++17", "-O3", "-fopenmp", "-fPIC", "-c", src, "-o", obj]
+        procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
+        objs.append(obj)
     failed = False
     for src, p in procs:
         out, _ = p.communicate()
@@ -42,7 +47,7 @@ def build(force=False, verbose=False):
     if failed:
         raise RuntimeError("nvcc failed")
     tmp = LIB + ".tmp.%d" % os.getpid()
-    subprocess.run([NVCC, "-shared", "-arch=sm_100a", "-o", tmp] + objs + ["-lcudart"], check=True)
+    subprocess.run([NVCC, "-shared", "-arch=sm_100a", "-o", tmp] + objs + ["-lcudart", "-lgomp"], check=True)
     os.replace(tmp, LIB)
     return LIB
 

@@ -20,6 +20,7 @@
 #include <vector>
 
 #include "../../include/ipkv.h"
+#include "cpu_engine.h"
 #include "kernels.h"
 #include "plan.hpp"
 #include "policy.hpp"
@@ -709,6 +710,28 @@ ipkv_status ipkv_attend_gpu(ipkv_t* h, int32_t layer, const int32_t* seq_ids, in
         CU(h, cudaEventRecord(h->slot_free[slot], s));
         h->slot_free_set[slot] = 1;
     }
+    return IPKV_OK;
+}
+
+ipkv_status ipkv_attend_cpu(ipkv_t* h, int32_t layer, const int32_t* seq_ids, int32_t n_seq, const void* q_host,
+                            float* o_part_host, float* lse_part_host, int32_t n_threads) {
+    if (!h) return IPKV_EINVAL;
+    const ipkv_config& c = h->cfg;
+    if (layer < 0 || layer >= c.n_layers) return fail(h, IPKV_EINVAL, "layer out of range");
+    if (n_seq <= 0 || !seq_ids || !q_host || !o_part_host || !lse_part_host) return fail(h, IPKV_EINVAL, "bad arguments");
+    if (!h->u_host) return fail(h, IPKV_ESTATE, "U contents are not kept (IPKV_FLAG_NO_HOST_U): nothing for the CPU engine to read");
+    std::vector<CpuRun> runs;
+    std::vector<int32_t> start(1, 0);
+    for (int i = 0; i < n_seq; ++i) {
+        if (seq_ids[i] < 0 || seq_ids[i] >= c.max_seqs) return fail(h, IPKV_EINVAL, "sequence id out of range");
+        for (const Run& r : h->state(layer, seq_ids[i]).router.runs())
+            if (r.region == REGION_U) runs.push_back(CpuRun{h->u_ptr(layer, seq_ids[i], r.first_block), r.n_tokens});
+        start.push_back(int32_t(runs.size()));
+    }
+    CpuShape sh{c.n_q_heads, c.n_kv_heads, c.dim_qk, c.dim_v, h->geom.dim_v_stored, c.block_tokens, h->scale};
+    if (cpu_attend_batch(sh, n_seq, static_cast<const uint16_t*>(q_host), runs.data(), start.data(), o_part_host, lse_part_host,
+                         n_threads) != 0)
+        return fail(h, IPKV_EINVAL, "shape not supported by the CPU engine");
     return IPKV_OK;
 }
 

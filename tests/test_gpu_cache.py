@@ -291,3 +291,57 @@ def test_mla_cache_decode_steps(resident):
             check_routing(cache, 0, s, refs[s], sample=range(0, len(refs[s].route), 5))
             check_contents(cache, 0, s, refs[s], range(0, len(refs[s].route), 11))
         assert cache.get_stats()["device_status"] == 0
+
+
+@pytest.mark.parametrize("kind", ["gqa", "mla"])
+def test_two_engine_step_cpu_engine_plus_gpu_equals_unsplit(kind):
+    """The paper's full decode step: the CPU engine attends region U in place, the GPU attends W and P, and one LSE
+    join gives exact attention over the whole sequence. Prefill share plus decode evictions fill U on both paths
+    (one-shot PLAIN packing and TILE -> PLAIN conversion of evicted windows)."""
+    if kind == "gqa":
+        sh = synth.Shape("g", "gqa", 1, 32, 4, 128, 128, 128 ** -0.5)
+    else:
+        sh = synth.Shape("m", "mla", 1, 16, 1, 576, 512, 192 ** -0.5)
+    rng = np.random.default_rng(90)
+    scale = float(np.float32(sh.scale))
+    seqs, lens = [0, 1, 2], {0: 1500, 1: 0, 2: 333}
+    hq, dv = sh.n_q_heads, sh.dim_v
+    with make_cache(sh, 1, 3, block_tokens=64, window_tokens=128, chunk_tokens=256, max_u_tokens_per_seq=3000,
+                    max_p_tokens_per_seq=3000, resident_tokens_per_seq=3000, share_num=1, share_den=2) as cache:
+        refs = {}
+        for s in seqs:
+            r = RefSeq(sh, 64, 128, 1, 2)
+            k, v = synth.host_kv(sh, lens[s], seed=9000 + s)
+            cache.append_bulk(0, s, synth.bits_to_torch(k, DEV) if lens[s] else None,
+                              synth.bits_to_torch(v, DEV) if (v is not None and lens[s]) else None, lens[s], 3, 5)
+            r.bulk(k, v, 3, 5)
+            refs[s] = r
+        for step in range(700):
+            k = synth.normal_bf16(rng, (3, sh.n_kv_heads, sh.dim_qk))
+            v = None if sh.kind == "mla" else synth.normal_bf16(rng, (3, sh.n_kv_heads, sh.dim_v))
+            cache.append(0, seqs, synth.bits_to_torch(k, DEV), None if v is None else synth.bits_to_torch(v, DEV))
+            for i, s in enumerate(seqs):
+                refs[s].append(k[i:i + 1], None if v is None else v[i:i + 1])
+        torch.cuda.synchronize()                          # U is filled by device-to-host copies
+        q = synth.normal_bf16(rng, (3, hq, sh.dim_qk))
+        q_host = synth.bits_to_torch(q).pin_memory()
+        o_cpu = torch.zeros((3, hq, dv)).pin_memory(); l_cpu = torch.zeros((3, hq)).pin_memory()
+        cache.attend_cpu(0, seqs, q_host, o_cpu, l_cpu)
+        want = [refs[s].attend(q[i], "cpu", scale) for i, s in enumerate(seqs)]
+        assert all(r.route.counts()["n_flush_cpu"] >= 2 for r in refs.values())
+        check_partial(o_cpu.numpy(), l_cpu.numpy(), np.stack([w[0] for w in want]), np.stack([w[1] for w in want]), "cpu engine")
+        # GPU side with the CPU partial folded in by the split reduce = full attention
+        out = torch.zeros((3, hq, dv), device=DEV); out_lse = torch.zeros((3, hq), device=DEV)
+        cache.attend_gpu(0, seqs, q_host.to(DEV), out, out_lse, fold_o=o_cpu.to(DEV), fold_lse=l_cpu.to(DEV))
+        torch.cuda.synchronize()
+        full = [refs[s].attend(q[i], "all", scale) for i, s in enumerate(seqs)]
+        check_partial(out.cpu().numpy(), out_lse.cpu().numpy(), np.stack([w[0] for w in full]), np.stack([w[1] for w in full]),
+                      "two engines")
+        # and through ipkv_merge with the CPU partial handed over in pinned host memory
+        o_gpu = torch.zeros((3, hq, dv), device=DEV); l_gpu = torch.zeros((3, hq), device=DEV)
+        cache.attend_gpu(0, seqs, q_host.to(DEV), o_gpu, l_gpu)
+        out2 = torch.zeros((3 * hq, dv), device=DEV); out2_lse = torch.zeros(3 * hq, device=DEV)
+        cache.merge(3 * hq, dv, [o_gpu.view(-1, dv), o_cpu.view(-1, dv)], [l_gpu.view(-1), l_cpu.view(-1)], out2, out2_lse)
+        torch.cuda.synchronize()
+        check_partial(out2.cpu().numpy().reshape(3, hq, dv), out2_lse.cpu().numpy().reshape(3, hq),
+                      np.stack([w[0] for w in full]), np.stack([w[1] for w in full]), "two engines via ipkv_merge")
