@@ -37,7 +37,10 @@ WORKLOADS = {
     "mixtral-8x7b-bs16-32k-cpu25": dict(shape=synth.MIXTRAL, batch=16, ctx=32768, share=(1, 4), cfg_id=2),
     # BASELINE config 3 at CPU share 0: Qwen3-30B-A3B-shaped attention, 48 layers, batch 16, 32K context
     "qwen3-30b-a3b-bs16-32k-cpu0": dict(shape=synth.QWEN3, batch=16, ctx=32768, share=(0, 1), cfg_id=3),
+    "qwen3-30b-a3b-bs16-32k-cpu10": dict(shape=synth.QWEN3, batch=16, ctx=32768, share=(1, 10), cfg_id=3),
+    "qwen3-30b-a3b-bs16-32k-cpu30": dict(shape=synth.QWEN3, batch=16, ctx=32768, share=(3, 10), cfg_id=3),
     "qwen3-30b-a3b-bs16-32k-cpu50": dict(shape=synth.QWEN3, batch=16, ctx=32768, share=(1, 2), cfg_id=3),
+    "qwen3-30b-a3b-bs16-32k-cpu70": dict(shape=synth.QWEN3, batch=16, ctx=32768, share=(7, 10), cfg_id=3),
     # two layers of config 2: a few GB on the device, still far larger than L2 -- the size used for ncu captures
     "mixtral-2layers-bs16-32k-cpu25": dict(shape=synth.Shape("mixtral-2l", "gqa", 2, 32, 8, 128, 128, 128 ** -0.5), batch=16,
                                            ctx=32768, share=(1, 4), cfg_id=2),
