@@ -89,6 +89,7 @@ __global__ void __launch_bounds__(kThreads) attn_gqa_kernel(const GqaParams p) {
     if (warp == kConsumerWarps) {
         // ---------------- producer ----------------
         if (lane == 0) {
+            const uint64_t pol = ptx::l2_evict_first_policy();     // the KV stream is read once: first out of L2
             for (int sp = span_begin; sp < span_end && ok; ++sp) {
                 const Span span = p.spans[sp];
                 const Seg seg = p.segs[span.seg];
@@ -106,14 +107,14 @@ __global__ void __launch_bounds__(kThreads) attn_gqa_kernel(const GqaParams p) {
                         const char* src = seg_base + blk * p.block_bytes;
                         ptx::mbar_expect_tx(bar, SP::kStage);
                         if (p.bt == kTileTokens) {
-                            ptx::bulk_g2s(dst, src, SP::kStage, bar);          // K plane and V plane are adjacent
+                            ptx::bulk_g2s_hint(dst, src, SP::kStage, bar, pol);   // K plane and V plane are adjacent
                         } else {
                             const int64_t kplane = int64_t(p.bt) * D * 2;
 #pragma unroll
                             for (int pn = 0; pn < D / 64; ++pn) {
                                 const char* s0 = src + int64_t(pn) * p.bt * 128 + int64_t(r0) * 128;
-                                ptx::bulk_g2s(dst + pn * 8192, s0, 8192, bar);
-                                ptx::bulk_g2s(dst + SP::kPlane + pn * 8192, s0 + kplane, 8192, bar);
+                                ptx::bulk_g2s_hint(dst + pn * 8192, s0, 8192, bar, pol);
+                                ptx::bulk_g2s_hint(dst + SP::kPlane + pn * 8192, s0 + kplane, 8192, bar, pol);
                             }
                         }
                     } else {
@@ -128,8 +129,8 @@ __global__ void __launch_bounds__(kThreads) attn_gqa_kernel(const GqaParams p) {
                             const char* src = seg_base + (blk0 + j) * p.block_bytes;
 #pragma unroll
                             for (int pn = 0; pn < D / 64; ++pn) {
-                                ptx::bulk_g2s(dst + pn * 8192 + j * sub_bytes, src + int64_t(pn) * sub_bytes, sub_bytes, bar);
-                                ptx::bulk_g2s(dst + SP::kPlane + pn * 8192 + j * sub_bytes, src + kplane + int64_t(pn) * sub_bytes, sub_bytes, bar);
+                                ptx::bulk_g2s_hint(dst + pn * 8192 + j * sub_bytes, src + int64_t(pn) * sub_bytes, sub_bytes, bar, pol);
+                                ptx::bulk_g2s_hint(dst + SP::kPlane + pn * 8192 + j * sub_bytes, src + kplane + int64_t(pn) * sub_bytes, sub_bytes, bar, pol);
                             }
                         }
                     }

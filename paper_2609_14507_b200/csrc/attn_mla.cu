@@ -100,6 +100,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_mla_kernel(const MlaParams p
     if (warp == kConsumerWarps) {
         // ---------------- producer: streams the whole chunk, never pausing at span boundaries ----------------
         if (lane == 0) {
+            const uint64_t pol = ptx::l2_evict_first_policy();     // the KV stream is read once: first out of L2
             for (int sn = span_begin; sn < span_end && ok; ++sn) {
                 const Span span = p.spans[sn];
                 const Seg seg = p.segs[span.seg];
@@ -116,11 +117,11 @@ __global__ void __launch_bounds__(kThreads, 1) attn_mla_kernel(const MlaParams p
                         const char* src = seg_base + blk * p.block_bytes;
                         ptx::mbar_expect_tx(bar, kStageBytes);
                         if (p.bt == kTileTokens) {
-                            ptx::bulk_g2s(dst, src, kStageBytes, bar);
+                            ptx::bulk_g2s_hint(dst, src, kStageBytes, bar, pol);
                         } else {
 #pragma unroll
                             for (int pn = 0; pn < kPanels; ++pn)
-                                ptx::bulk_g2s(dst + pn * 8192, src + int64_t(pn) * p.bt * 128 + int64_t(r0) * 128, 8192, bar);
+                                ptx::bulk_g2s_hint(dst + pn * 8192, src + int64_t(pn) * p.bt * 128 + int64_t(r0) * 128, 8192, bar, pol);
                         }
                     } else {
                         const int nsub = kTileTokens / p.bt;
@@ -133,7 +134,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_mla_kernel(const MlaParams p
                             const char* src = seg_base + (blk0 + j) * p.block_bytes;
 #pragma unroll
                             for (int pn = 0; pn < kPanels; ++pn)
-                                ptx::bulk_g2s(dst + pn * 8192 + j * sub_bytes, src + int64_t(pn) * sub_bytes, sub_bytes, bar);
+                                ptx::bulk_g2s_hint(dst + pn * 8192 + j * sub_bytes, src + int64_t(pn) * sub_bytes, sub_bytes, bar, pol);
                         }
                     }
                 }
