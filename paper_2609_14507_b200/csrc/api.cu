@@ -114,6 +114,14 @@ struct ipkv {
     char* merge_stage = nullptr;
     size_t merge_stage_bytes = 0;
     uint32_t* status_dev = nullptr;
+    // write-back of evicted windows on the idle D2H direction: a device snapshot of every window (same shape as W),
+    // a copy stream, one "snapshot in use" event per layer, and a pinned bounce buffer for the unpinned region
+    char* wb_stage = nullptr;
+    char* wb_bounce = nullptr;
+    cudaStream_t copy = nullptr;
+    cudaEvent_t ev_wb = nullptr, ev_copy = nullptr;
+    std::vector<cudaEvent_t> wb_busy;
+    std::vector<char> wb_busy_set;
     cudaStream_t side = nullptr;
     std::vector<cudaEvent_t> slot_ready, slot_free;
     std::vector<char> slot_free_set;
@@ -202,21 +210,6 @@ void note_p_run(SeqState& s, const Run& r, int64_t bt) {
     s.p_runs.push_back(PRun{r.first_block, r.n_tokens});
 }
 
-// Copy blocks [j0, j1) of a P run from `src` (contiguous, block j0 first) into the resident ring.
-ipkv_status ring_store(ipkv* h, int layer, int seq, int64_t j0, int64_t j1, const char* src, cudaStream_t s) {
-    if (h->ring == 0) return IPKV_OK;
-    if (j1 - j0 > h->ring) { src += (j1 - j0 - h->ring) * h->bb; j0 = j1 - h->ring; }   // only the newest fit
-    char* base = h->ring_layer(layer) + h->ring_off(seq);
-    while (j0 < j1) {
-        const int64_t pos = j0 % h->ring;
-        const int64_t n = std::min(j1 - j0, h->ring - pos);
-        CU(h, cudaMemcpyAsync(base + pos * h->bb, src, size_t(n * h->bb), cudaMemcpyDeviceToDevice, s));
-        h->stats.d2d_bytes += uint64_t(n * h->bb);
-        src += n * h->bb; j0 += n;
-    }
-    return IPKV_OK;
-}
-
 ipkv_status ensure_staging(ipkv* h, size_t bytes) {
     if (h->staging_bytes >= bytes) return IPKV_OK;
     CU(h, cudaDeviceSynchronize());
@@ -227,42 +220,145 @@ ipkv_status ensure_staging(ipkv* h, size_t bytes) {
     return IPKV_OK;
 }
 
-ipkv_status do_flush(ipkv* h, int layer, int seq, cudaStream_t s) {
-    SeqState& st = h->state(layer, seq);
-    const int64_t fill = st.router.window_fill();
-    if (fill == 0) return IPKV_OK;
-    const int64_t nb = st.router.blocks_for(fill);
-    const int side = st.router.peek_eviction_side();
+struct BounceJob { std::vector<void*> dst; std::vector<const void*> src; std::vector<size_t> bytes; };
+void CUDART_CB bounce_to_unpinned(void* arg) {
+    BounceJob* j = static_cast<BounceJob*>(arg);
+    for (size_t i = 0; i < j->dst.size(); ++i) std::memcpy(j->dst[i], j->src[i], j->bytes[i]);
+    delete j;
+}
+
+// Evict the windows of the listed sequences of one layer (Sec. 4.2): each is one whole batch, routed to U or P.
+// The compute stream only takes a device-side snapshot of the batches (and refreshes the resident ring); the
+// device-to-host write-back runs on the copy stream, so it rides the otherwise idle D2H direction and decode steps
+// stay flat. Neighbouring sequences with the same destination are handled by one launch / one copy (a batch that
+// advances in lockstep evicts every sequence of a layer to the same side). Host contents are complete once the
+// copy stream has drained (sync_host()).
+ipkv_status flush_layer(ipkv* h, int layer, const int* seqs_in, int n, cudaStream_t s) {
     const bool no_u = h->cfg.flags & IPKV_FLAG_NO_HOST_U, no_p = h->cfg.flags & IPKV_FLAG_NO_HOST_P;
-    if (side == REGION_U) {
-        if (st.router.blocks_used(REGION_U) + nb > h->u_cap) return fail(h, IPKV_ERANGE, "eviction would exceed the capacity of U");
-    } else {
-        if (st.router.blocks_used(REGION_P) + nb > h->p_cap) return fail(h, IPKV_ERANGE, "eviction would exceed the capacity of P");
-        if (no_p && st.router.blocks_used(REGION_P) + nb > h->ring)
-            return fail(h, IPKV_ERANGE, "eviction would push P blocks out of the resident ring, and no host copy of P exists");
-    }
-    const Run r = st.router.evict();
-    const char* src = h->w_layer(layer) + h->w_off(seq);
-    h->stats.flushes += 1;
-    if (r.region == REGION_U) {
-        h->stats.flushes_to_u += 1;
-        if (!no_u) {
-            ipkv_status rc = ensure_staging(h, size_t(nb * h->bb));
-            if (rc != IPKV_OK) return rc;
-            CU(h, launch_tile_to_plain(h->geom, src, h->staging, nb, s));
-            h->stats.pack_kernels += 1;
-            CU(h, cudaMemcpyAsync(h->u_ptr(layer, seq, r.first_block), h->staging, size_t(nb * h->bb), cudaMemcpyDeviceToHost, s));
-            h->stats.d2h_bytes += uint64_t(nb * h->bb);
+    struct Job { int seq; Run r; int64_t nb; };
+    std::vector<int> seqs(seqs_in, seqs_in + n);
+    std::sort(seqs.begin(), seqs.end());
+    // pass 1: capacity checks for every sequence before anything changes
+    for (int seq : seqs) {
+        SeqState& st = h->state(layer, seq);
+        const int64_t fill = st.router.window_fill();
+        if (fill == 0) continue;
+        const int64_t nb = st.router.blocks_for(fill);
+        if (st.router.peek_eviction_side() == REGION_U) {
+            if (st.router.blocks_used(REGION_U) + nb > h->u_cap) return fail(h, IPKV_ERANGE, "eviction would exceed the capacity of U");
+        } else {
+            if (st.router.blocks_used(REGION_P) + nb > h->p_cap) return fail(h, IPKV_ERANGE, "eviction would exceed the capacity of P");
+            if (no_p && st.router.blocks_used(REGION_P) + nb > h->ring)
+                return fail(h, IPKV_ERANGE, "eviction would push P blocks out of the resident ring, and no host copy of P exists");
         }
-    } else {
-        if (!no_p) {
-            CU(h, cudaMemcpyAsync(h->p_ptr(layer, seq, r.first_block), src, size_t(nb * h->bb), cudaMemcpyDeviceToHost, s));
-            h->stats.d2h_bytes += uint64_t(nb * h->bb);
-        }
-        ipkv_status rc = ring_store(h, layer, seq, r.first_block, r.first_block + nb, src, s);
-        if (rc != IPKV_OK) return rc;
-        note_p_run(st, r, h->cfg.block_tokens);
     }
+    std::vector<Job> jobs;
+    bool need_wb = false;
+    for (int seq : seqs) {
+        SeqState& st = h->state(layer, seq);
+        if (st.router.window_fill() == 0) continue;
+        const int64_t nb = st.router.blocks_for(st.router.window_fill());
+        const Run r = st.router.evict();
+        jobs.push_back(Job{seq, r, nb});
+        h->stats.flushes += 1;
+        h->stats.flushes_to_u += (r.region == REGION_U);
+        need_wb |= (r.region == REGION_U) ? !no_u : !no_p;
+        if (r.region == REGION_P) note_p_run(st, r, h->cfg.block_tokens);
+    }
+    if (jobs.empty()) return IPKV_OK;
+    if (need_wb && h->wb_busy_set[layer]) CU(h, cudaStreamWaitEvent(s, h->wb_busy[layer], 0));   // previous write-back of this layer
+    const int64_t win_bytes = h->w_blocks * h->bb;
+    const int64_t layer_off = h->w_layer(layer) - h->w_dev;
+    // groups of neighbouring sequences with the same destination: [g0, g1) in `jobs`
+    std::vector<std::pair<size_t, size_t>> groups;
+    for (size_t i = 0; i < jobs.size();) {
+        size_t j = i + 1;
+        while (j < jobs.size() && jobs[j].seq == jobs[j - 1].seq + 1 && jobs[j].r.region == jobs[i].r.region) ++j;
+        groups.push_back({i, j});
+        i = j;
+    }
+    // ---- compute stream: snapshots of the evicted windows, refresh of the resident ring ----
+    CopySpans spans;
+    int n_spans = 0;
+    auto flush_spans = [&]() -> ipkv_status {
+        if (n_spans > 0) { CU(h, launch_copy_spans(spans, n_spans, s)); n_spans = 0; }
+        return IPKV_OK;
+    };
+    for (const auto& g : groups) {
+        const Job& first = jobs[g.first];
+        const int64_t n_seq_g = int64_t(g.second - g.first);
+        const char* src = h->w_layer(layer) + h->w_off(first.seq);
+        char* snap = h->wb_stage ? h->wb_stage + layer_off + h->w_off(first.seq) : nullptr;
+        if (first.r.region == REGION_U) {
+            if (!no_u) {
+                CU(h, launch_tile_to_plain(h->geom, src, snap, n_seq_g * h->w_blocks, s));
+                h->stats.pack_kernels += 1;
+            }
+        } else {
+            if (!no_p) {
+                CU(h, cudaMemcpyAsync(snap, src, size_t(n_seq_g * win_bytes), cudaMemcpyDeviceToDevice, s));
+                h->stats.d2d_bytes += uint64_t(n_seq_g * win_bytes);
+            }
+            if (h->ring > 0)
+                for (size_t k = g.first; k < g.second; ++k) {
+                    const Job& j = jobs[k];
+                    const char* wsrc = h->w_layer(layer) + h->w_off(j.seq);
+                    int64_t j0 = j.r.first_block, j1 = j.r.first_block + j.nb;
+                    if (j1 - j0 > h->ring) { wsrc += (j1 - j0 - h->ring) * h->bb; j0 = j1 - h->ring; }   // only the newest fit
+                    char* base = h->ring_layer(layer) + h->ring_off(j.seq);
+                    while (j0 < j1) {
+                        const int64_t pos = j0 % h->ring;
+                        const int64_t cnt = std::min(j1 - j0, h->ring - pos);
+                        spans.src[n_spans] = wsrc; spans.dst[n_spans] = base + pos * h->bb; spans.bytes[n_spans] = cnt * h->bb;
+                        h->stats.d2d_bytes += uint64_t(cnt * h->bb);
+                        if (++n_spans == kCopySpansPerLaunch) { ipkv_status rc = flush_spans(); if (rc != IPKV_OK) return rc; }
+                        wsrc += cnt * h->bb; j0 += cnt;
+                    }
+                }
+        }
+    }
+    { ipkv_status rc = flush_spans(); if (rc != IPKV_OK) return rc; }
+    if (!need_wb) return IPKV_OK;
+    // ---- copy stream: write-back ----
+    CU(h, cudaEventRecord(h->ev_wb, s));
+    CU(h, cudaStreamWaitEvent(h->copy, h->ev_wb, 0));
+    for (const auto& g : groups) {
+        const Job& first = jobs[g.first];
+        const int64_t n_seq_g = int64_t(g.second - g.first);
+        const char* snap = h->wb_stage + layer_off + h->w_off(first.seq);
+        if (first.r.region == REGION_U) {
+            if (no_u) continue;
+            // U is unpinned: the group lands in the pinned bounce buffer, then a host callback moves every batch
+            // to its place in U (stream-ordered, so the bounce buffer is free again before the next copy)
+            char* bounce = h->wb_bounce + h->w_off(first.seq);
+            CU(h, cudaMemcpyAsync(bounce, snap, size_t(n_seq_g * win_bytes), cudaMemcpyDeviceToHost, h->copy));
+            BounceJob* bj = new (std::nothrow) BounceJob();
+            if (!bj) return fail(h, IPKV_ENOMEM, "out of host memory");
+            for (size_t k = g.first; k < g.second; ++k) {
+                bj->dst.push_back(h->u_ptr(layer, jobs[k].seq, jobs[k].r.first_block));
+                bj->src.push_back(h->wb_bounce + h->w_off(jobs[k].seq));
+                bj->bytes.push_back(size_t(jobs[k].nb * h->bb));
+                h->stats.d2h_bytes += uint64_t(jobs[k].nb * h->bb);
+            }
+            CU(h, cudaLaunchHostFunc(h->copy, bounce_to_unpinned, bj));
+        } else {
+            if (no_p) continue;
+            for (size_t k = g.first; k < g.second; ++k) {
+                const size_t bytes = size_t(jobs[k].nb * h->bb);
+                CU(h, cudaMemcpyAsync(h->p_ptr(layer, jobs[k].seq, jobs[k].r.first_block), h->wb_stage + layer_off + h->w_off(jobs[k].seq),
+                                      bytes, cudaMemcpyDeviceToHost, h->copy));
+                h->stats.d2h_bytes += bytes;
+            }
+        }
+    }
+    CU(h, cudaEventRecord(h->wb_busy[layer], h->copy));
+    h->wb_busy_set[layer] = 1;
+    return IPKV_OK;
+}
+
+// Host-visible contents of U and P are complete after this.
+ipkv_status sync_host(ipkv* h) {
+    if (h->copy) CU(h, cudaStreamSynchronize(h->copy));
     return IPKV_OK;
 }
 
@@ -429,6 +525,12 @@ ipkv_status ipkv_destroy(ipkv_t* h) {
     if (h->table_dev) cudaFree(h->table_dev);
     if (h->merge_stage) cudaFree(h->merge_stage);
     if (h->status_dev) cudaFree(h->status_dev);
+    if (h->wb_stage) cudaFree(h->wb_stage);
+    if (h->wb_bounce) cudaFreeHost(h->wb_bounce);
+    for (auto e : h->wb_busy) if (e) cudaEventDestroy(e);
+    if (h->ev_wb) cudaEventDestroy(h->ev_wb);
+    if (h->ev_copy) cudaEventDestroy(h->ev_copy);
+    if (h->copy) cudaStreamDestroy(h->copy);
     for (int i = 0; i < ipkv::kTableParts; ++i) if (h->table_ev[i]) cudaEventDestroy(h->table_ev[i]);
     for (auto e : h->prof_ev) cudaEventDestroy(e);
     for (auto e : h->slot_ready) cudaEventDestroy(e);
@@ -489,6 +591,16 @@ ipkv_status ipkv_create(const ipkv_config* cfg, ipkv_t** out) {
     for (int i = 0; i < ipkv::kTableParts; ++i)
         if (cudaEventCreateWithFlags(&h->table_ev[i], cudaEventDisableTiming) != cudaSuccess) return bail(IPKV_ECUDA);
     if (cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking) != cudaSuccess) return bail(IPKV_ECUDA);
+    if (cudaStreamCreateWithFlags(&h->copy, cudaStreamNonBlocking) != cudaSuccess) return bail(IPKV_ECUDA);
+    if (cudaEventCreateWithFlags(&h->ev_wb, cudaEventDisableTiming) != cudaSuccess) return bail(IPKV_ECUDA);
+    if (cudaEventCreateWithFlags(&h->ev_copy, cudaEventDisableTiming) != cudaSuccess) return bail(IPKV_ECUDA);
+    h->wb_busy.resize(cfg->n_layers); h->wb_busy_set.assign(cfg->n_layers, 0);
+    for (int i = 0; i < cfg->n_layers; ++i)
+        if (cudaEventCreateWithFlags(&h->wb_busy[i], cudaEventDisableTiming) != cudaSuccess) return bail(IPKV_ECUDA);
+    if (h->sizes[0] > 0 || h->sizes[1] > 0) {      // some host copy is kept: snapshots of the windows for the write-back
+        if (cudaMalloc(&h->wb_stage, h->sizes[2]) != cudaSuccess) return bail(IPKV_ENOMEM);
+        if (h->sizes[0] > 0 && cudaMallocHost(&h->wb_bounce, size_t(int64_t(cfg->max_seqs) * h->w_blocks * h->bb)) != cudaSuccess) return bail(IPKV_ENOMEM);
+    }
     h->slot_ready.resize(cfg->n_slots); h->slot_free.resize(cfg->n_slots); h->slot_free_set.assign(cfg->n_slots, 0);
     for (int i = 0; i < cfg->n_slots; ++i) {
         if (cudaEventCreateWithFlags(&h->slot_ready[i], cudaEventDisableTiming) != cudaSuccess) return bail(IPKV_ECUDA);
@@ -584,12 +696,14 @@ ipkv_status ipkv_flush(ipkv_t* h, int32_t layer, int32_t seq, void* stream) {
     if (layer < -1 || layer >= h->cfg.n_layers) return fail(h, IPKV_EINVAL, "layer out of range");
     if (seq < -1 || seq >= h->cfg.max_seqs) return fail(h, IPKV_EINVAL, "sequence id out of range");
     CU(h, cudaSetDevice(h->cfg.device));
-    for (int l = 0; l < h->cfg.n_layers; ++l)
+    for (int l = 0; l < h->cfg.n_layers; ++l) {
+        if (layer >= 0 && l != layer) continue;
+        std::vector<int> seqs;
         for (int s = 0; s < h->cfg.max_seqs; ++s)
-            if ((layer < 0 || l == layer) && (seq < 0 || s == seq)) {
-                ipkv_status rc = do_flush(h, l, s, static_cast<cudaStream_t>(stream));
-                if (rc != IPKV_OK) return rc;
-            }
+            if (seq < 0 || s == seq) seqs.push_back(s);
+        ipkv_status rc = flush_layer(h, l, seqs.data(), int(seqs.size()), static_cast<cudaStream_t>(stream));
+        if (rc != IPKV_OK) return rc;
+    }
     return IPKV_OK;
 }
 
@@ -606,11 +720,15 @@ ipkv_status ipkv_append(ipkv_t* h, int32_t layer, const int32_t* seq_ids, int32_
     }
     CU(h, cudaSetDevice(c.device));
     // evict full windows first, so that the newest token is always GPU-side
-    for (int i = 0; i < n_seq; ++i)
-        if (h->state(layer, seq_ids[i]).router.window_full()) {
-            ipkv_status rc = do_flush(h, layer, seq_ids[i], s);
+    {
+        std::vector<int> full;
+        for (int i = 0; i < n_seq; ++i)
+            if (h->state(layer, seq_ids[i]).router.window_full()) full.push_back(seq_ids[i]);
+        if (!full.empty()) {
+            ipkv_status rc = flush_layer(h, layer, full.data(), int(full.size()), s);
             if (rc != IPKV_OK) return rc;
         }
+    }
     const int64_t k_row = int64_t(c.n_kv_heads) * c.dim_qk * 2, v_row = int64_t(c.n_kv_heads) * c.dim_v * 2;
     for (int base = 0; base < n_seq; base += kAppendRowsPerLaunch) {
         const int n = std::min(kAppendRowsPerLaunch, n_seq - base);
@@ -679,8 +797,10 @@ ipkv_status ipkv_attend_gpu(ipkv_t* h, int32_t layer, const int32_t* seq_ids, in
     if (max_stream_chunks == 0) return IPKV_OK;
 
     // groups 1..: host-only P chunks, streamed through the PP slots in overwrite-reuse order (Sec. 4.2)
-    CU(h, cudaEventRecord(h->ev_main, s));                 // P's host bytes were written by work on `s`
+    CU(h, cudaEventRecord(h->ev_main, s));                 // P's host bytes were written by work on `s` ...
     CU(h, cudaStreamWaitEvent(side, h->ev_main, 0));
+    CU(h, cudaEventRecord(h->ev_copy, h->copy));           // ... or by write-backs on the copy stream
+    CU(h, cudaStreamWaitEvent(side, h->ev_copy, 0));
     const int64_t chunk_bytes = h->chunk_blocks * h->bb;
     for (int64_t ch = 0; ch < max_stream_chunks; ++ch) {
         const int slot = int(ch % c.n_slots);
@@ -720,6 +840,8 @@ ipkv_status ipkv_attend_cpu(ipkv_t* h, int32_t layer, const int32_t* seq_ids, in
     if (layer < 0 || layer >= c.n_layers) return fail(h, IPKV_EINVAL, "layer out of range");
     if (n_seq <= 0 || !seq_ids || !q_host || !o_part_host || !lse_part_host) return fail(h, IPKV_EINVAL, "bad arguments");
     if (!h->u_host) return fail(h, IPKV_ESTATE, "U contents are not kept (IPKV_FLAG_NO_HOST_U): nothing for the CPU engine to read");
+    CU(h, cudaSetDevice(c.device));
+    { ipkv_status rc = sync_host(h); if (rc != IPKV_OK) return rc; }       // write-backs still in flight on the copy stream
     std::vector<CpuRun> runs;
     std::vector<int32_t> start(1, 0);
     for (int i = 0; i < n_seq; ++i) {

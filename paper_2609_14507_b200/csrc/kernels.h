@@ -82,6 +82,15 @@ cudaError_t launch_pack(const BlockGeom& g, int layout_tile, const void* k, cons
 // TILE-layout blocks -> PLAIN-layout blocks (eviction of a window batch to the CPU-compute region).
 cudaError_t launch_tile_to_plain(const BlockGeom& g, const void* src, void* dst, int64_t n_blocks, cudaStream_t s);
 
+// Several device-to-device copies in one launch (refreshing the resident ring after an eviction): 16-byte chunks.
+constexpr int kCopySpansPerLaunch = 64;
+struct CopySpans {
+    const char* src[kCopySpansPerLaunch];
+    char* dst[kCopySpansPerLaunch];
+    int64_t bytes[kCopySpansPerLaunch];      // multiples of 16
+};
+cudaError_t launch_copy_spans(const CopySpans& spans, int n, cudaStream_t s);
+
 constexpr int kAppendRowsPerLaunch = 64;
 struct AppendRows {
     int64_t dst_off[kAppendRowsPerLaunch];   // byte offset of the row's window (first block) from w_base

@@ -77,6 +77,14 @@ __global__ void append_kernel(BlockGeom g, const uint4* __restrict__ k, const ui
     }
 }
 
+__global__ void copy_spans_kernel(CopySpans sp) {
+    const int k = blockIdx.y;
+    const uint4* src = reinterpret_cast<const uint4*>(sp.src[k]);
+    uint4* dst = reinterpret_cast<uint4*>(sp.dst[k]);
+    const int64_t n = sp.bytes[k] / 16;
+    for (int64_t i = blockIdx.x * int64_t(blockDim.x) + threadIdx.x; i < n; i += int64_t(gridDim.x) * blockDim.x) dst[i] = src[i];
+}
+
 int grid_for(int64_t total, int threads) {
     int64_t b = (total + threads - 1) / threads;
     const int64_t cap = 148 * 16;
@@ -100,6 +108,15 @@ cudaError_t launch_tile_to_plain(const BlockGeom& g, const void* src, void* dst,
     if (n_blocks <= 0) return cudaSuccess;
     const int64_t total = n_blocks * (g.block_bytes() / 16);
     tile_to_plain_kernel<<<grid_for(total, 256), 256, 0, s>>>(g, static_cast<const char*>(src), static_cast<char*>(dst), n_blocks);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_copy_spans(const CopySpans& spans, int n, cudaStream_t s) {
+    if (n <= 0) return cudaSuccess;
+    int64_t longest = 0;
+    for (int i = 0; i < n; ++i) longest = spans.bytes[i] > longest ? spans.bytes[i] : longest;
+    dim3 grid(grid_for(longest / 16, 256) > 64 ? 64 : grid_for(longest / 16, 256), n);
+    copy_spans_kernel<<<grid, 256, 0, s>>>(spans);
     return cudaGetLastError();
 }
 
