@@ -87,6 +87,14 @@ for _pct in (10, 30, 50, 70, 100):
         stream_pct=_pct, chunk_tokens=4096)
 
 
+# Decode with the host copies of U and P switched ON (pinned P, unpinned U): every 256 steps each layer evicts its
+# D-window (8.4 MB per layer, device -> host). Used with --latency to look at per-step latency across evictions
+# (the paper reports P99/P50 = 1.03 over 1000 steps for this shape at batch 8, 8K context).
+for _pct, _share in ((0, (0, 1)), (50, (1, 2)), (100, (1, 1))):
+    WORKLOADS[f"qwen3-30b-a3b-bs8-8k-cpu{_pct}-hostcopies"] = dict(shape=synth.QWEN3, batch=8, ctx=8192, share=_share, cfg_id=3,
+                                                                   host_copies=True)
+
+
 def seq_lens(wl):
     """Context length of every sequence of the batch."""
     return [int(x) for x in wl["lens"]] if "lens" in wl else [wl["ctx"]] * wl["batch"]
@@ -112,6 +120,8 @@ def make_cache(wl, device_index, decode_steps):
     p_cap = max(p_cap, max(n - cpu_tokens(n, num0, den0) for n in seq_lens(wl)) + grow)
     kind = binding.MLA if sh.kind == "mla" else binding.GQA
     resident, flags = p_cap, binding.FLAG_NO_HOST_U | binding.FLAG_NO_HOST_P
+    if wl.get("host_copies"):
+        flags = 0
     if "stream_pct" in wl:
         # keep the newest (100 - stream_pct) % of the prefill's P share resident; P itself lives in pinned host memory
         resident = BLOCK * (((longest - cpu_tokens(longest, num0, den0)) * (100 - wl["stream_pct"]) // 100) // BLOCK)
@@ -267,6 +277,7 @@ def main():
     ap.add_argument("--kv-splits", type=int, default=0)
     ap.add_argument("--separate-merge", action="store_true",
                     help="join the CPU-side partial with a separate ipkv_merge launch instead of inside the split reduce")
+    ap.add_argument("--latency", action="store_true", help="also time every step separately and report P50 / P99 / max")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -354,13 +365,26 @@ def main():
     cache.profile_read()
     sampler.mark()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)] if args.latency else None
     e0.record()
-    for _ in range(args.steps):
+    for i in range(args.steps):
+        if marks:
+            marks[i].record()
         step()
+    if marks:
+        marks[-1].record()
     e1.record()
     barrier()
     clocks = sampler.stop() if rank == 0 else None
     ms = max_over_ranks(e0.elapsed_time(e1))
+    step_lat = None
+    if marks:
+        raw = [marks[i].elapsed_time(marks[i + 1]) for i in range(args.steps)]
+        lat = sorted(raw)
+        slowest = sorted(range(args.steps), key=lambda i: -raw[i])[:4]
+        p99 = lat[min(len(lat) - 1, int(0.99 * len(lat)))]
+        step_lat = {"p50_ms": lat[len(lat) // 2], "p99_ms": p99, "max_ms": lat[-1], "p99_over_p50": p99 / lat[len(lat) // 2],
+                    "slowest_steps": [(i, round(raw[i], 3)) for i in slowest]}
     kern_ms, n_timed, n_launch = cache.profile_read()
     cache.profile_enable(False)
     st1 = cache.get_stats()
@@ -449,6 +473,10 @@ def main():
             "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu,
             "step_gbs": world * bytes_attended / (ms * 1e-3) / 1e9,
         }
+        if step_lat:
+            line["step_latency"] = step_lat
+        if wl.get("host_copies"):
+            line["config"]["host_copies_of_U_and_P"] = "on (P pinned, U unpinned); write-back on a copy stream"
         if "stream_pct" in wl:
             # the box's pinned host-to-device plateau, measured here with one 256 MB copy (best of 5)
             hp = torch.empty(256 << 20, dtype=torch.uint8).pin_memory(); dp = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
