@@ -162,6 +162,17 @@ ipkv_status ipkv_attend_gpu(ipkv_t* h, int32_t layer, const int32_t* seq_ids, in
                             const void* q_dev, const ipkv_attend_opts* opts,
                             float* o_part_dev, float* lse_part_dev, void* stream);
 
+/* Block-sparse variant (Sec. 4.4): every row attends its D-window (if include_window != 0) plus the listed WHOLE P
+ * blocks only — the set a block-level top-k selection would return.  p_blocks: host array of block ordinals inside
+ * region P (as ipkv_views / ipkv_locate report them), the blocks of row r at p_blocks[row_block_start[r] ..
+ * row_block_start[r+1]), strictly increasing within a row.  Device-resident blocks are read in place; host-only blocks
+ * are gathered, one memcpy per block, into a contiguous pinned staging buffer the size of a PP slot and reach the
+ * device with one DMA per slot, the gather of the next slot overlapping the DMA of the current one.
+ * Other arguments and outputs as ipkv_attend_gpu. */
+ipkv_status ipkv_attend_gpu_sparse(ipkv_t* h, int32_t layer, const int32_t* seq_ids, int32_t n_seq, const void* q_dev,
+                                   const int64_t* p_blocks, const int32_t* row_block_start, int32_t include_window,
+                                   const ipkv_attend_opts* opts, float* o_part_dev, float* lse_part_dev, void* stream);
+
 /* CPU-side engine (Sec. 6.1): in-place attention over the CPU-side share, i.e. the tokens routed to region U,
  * read where they lie (PLAIN blocks, no copy).  This is the paper's second engine, not a fallback for the GPU
  * path: it attends a disjoint token range and its partial is joined by ipkv_merge / the fold option.

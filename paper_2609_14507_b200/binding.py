@@ -21,7 +21,7 @@ STATUS_NAMES = {0: "OK", 1: "EINVAL", 2: "ENOMEM", 3: "ERANGE", 4: "ESTATE", 5: 
 
 EXPORTS = [
     "ipkv_query_sizes", "ipkv_create", "ipkv_destroy", "ipkv_set_share", "ipkv_reset", "ipkv_append_bulk",
-    "ipkv_append", "ipkv_flush", "ipkv_attend_gpu", "ipkv_attend_cpu", "ipkv_merge", "ipkv_views", "ipkv_locate", "ipkv_counts",
+    "ipkv_append", "ipkv_flush", "ipkv_attend_gpu", "ipkv_attend_gpu_sparse", "ipkv_attend_cpu", "ipkv_merge", "ipkv_views", "ipkv_locate", "ipkv_counts",
     "ipkv_read_token", "ipkv_get_stats", "ipkv_profile_enable", "ipkv_profile_read", "ipkv_attend_scratch_bytes", "ipkv_attend_runs", "ipkv_pack_blocks",
     "ipkv_attend_runs_noalloc", "ipkv_noalloc_scratch_limit", "ipkv_roofline_share", "ipkv_roofline_step_time",
     "ipkv_policy_create", "ipkv_policy_destroy", "ipkv_policy_observe", "ipkv_policy_update", "ipkv_policy_prefill_share",
@@ -101,6 +101,8 @@ def lib():
         "ipkv_append": [vp, i32, C.POINTER(i32), i32, vp, vp, vp],
         "ipkv_flush": [vp, i32, i32, vp],
         "ipkv_attend_gpu": [vp, i32, C.POINTER(i32), i32, vp, C.POINTER(AttendOpts), vp, vp, vp],
+        "ipkv_attend_gpu_sparse": [vp, i32, C.POINTER(i32), i32, vp, C.POINTER(i64), C.POINTER(i32), i32, C.POINTER(AttendOpts),
+                                   vp, vp, vp],
         "ipkv_attend_cpu": [vp, i32, C.POINTER(i32), i32, vp, vp, vp, i32],
         "ipkv_merge": [vp, i32, i32, i32, C.POINTER(vp), C.POINTER(vp), vp, i32, vp, vp],
         "ipkv_views": [vp, i32, i32, C.POINTER(Extent), i32, C.POINTER(i32)],
@@ -251,6 +253,20 @@ class Cache:
         opts = AttendOpts(kv_splits, 0, _stream(side_stream) if side_stream is not None else None, _ptr(fold_o), _ptr(fold_lse))
         self._check(lib().ipkv_attend_gpu(self._h, layer, ids, n, _ptr(q), C.byref(opts), _ptr(o_part), _ptr(lse_part),
                                           _stream(stream)), "ipkv_attend_gpu")
+
+    def attend_gpu_sparse(self, layer, seq_ids, q, blocks_per_row, o_part, lse_part, include_window=True, kv_splits=0,
+                          stream=None, fold_o=None, fold_lse=None):
+        """Attention over the D-window plus the listed whole P blocks of every row (block ordinals in region P)."""
+        ids, n = _ids(seq_ids)
+        flat, start = [], [0]
+        for row in blocks_per_row:
+            flat += [int(b) for b in row]
+            start.append(len(flat))
+        blocks = (C.c_int64 * max(1, len(flat)))(*flat)
+        starts = (C.c_int32 * len(start))(*start)
+        opts = AttendOpts(kv_splits, 0, None, _ptr(fold_o), _ptr(fold_lse))
+        self._check(lib().ipkv_attend_gpu_sparse(self._h, layer, ids, n, _ptr(q), blocks, starts, 1 if include_window else 0,
+                                                 C.byref(opts), _ptr(o_part), _ptr(lse_part), _stream(stream)), "ipkv_attend_gpu_sparse")
 
     def attend_cpu(self, layer, seq_ids, q_host, o_part_host, lse_part_host, n_threads=0):
         """CPU-side engine over the tokens routed to U; all tensors in host memory."""

@@ -123,6 +123,10 @@ struct ipkv {
     std::vector<cudaEvent_t> wb_busy;
     std::vector<char> wb_busy_set;
     cudaStream_t side = nullptr;
+    // block-sparse path: two pinned gather buffers of one PP slot each, and the event of the DMA that last read each
+    char* gather[2] = {nullptr, nullptr};
+    cudaEvent_t gather_done[2] = {nullptr, nullptr};
+    bool gather_busy[2] = {false, false};
     std::vector<cudaEvent_t> slot_ready, slot_free;
     std::vector<char> slot_free_set;
     cudaEvent_t ev_main = nullptr;
@@ -525,6 +529,10 @@ ipkv_status ipkv_destroy(ipkv_t* h) {
     if (h->table_dev) cudaFree(h->table_dev);
     if (h->merge_stage) cudaFree(h->merge_stage);
     if (h->status_dev) cudaFree(h->status_dev);
+    for (int i = 0; i < 2; ++i) {
+        if (h->gather[i]) cudaFreeHost(h->gather[i]);
+        if (h->gather_done[i]) cudaEventDestroy(h->gather_done[i]);
+    }
     if (h->wb_stage) cudaFree(h->wb_stage);
     if (h->wb_bounce) cudaFreeHost(h->wb_bounce);
     for (auto e : h->wb_busy) if (e) cudaEventDestroy(e);
@@ -823,6 +831,110 @@ ipkv_status ipkv_attend_gpu(ipkv_t* h, int32_t layer, const int32_t* seq_ids, in
                 rows[i].push_back(PlanSeg{2, slot * h->slot_bytes() + int64_t(i) * chunk_bytes + (a - lo) * h->bb, tok});
             }
         }
+        CU(h, cudaEventRecord(h->slot_ready[slot], side));
+        CU(h, cudaStreamWaitEvent(s, h->slot_ready[slot], 0));
+        rc = run_group(h, rows, bases, q_dev, kv_splits, o_part_dev, lse_part_dev, o_part_dev, lse_part_dev, s);
+        if (rc != IPKV_OK) return rc;
+        CU(h, cudaEventRecord(h->slot_free[slot], s));
+        h->slot_free_set[slot] = 1;
+    }
+    return IPKV_OK;
+}
+
+ipkv_status ipkv_attend_gpu_sparse(ipkv_t* h, int32_t layer, const int32_t* seq_ids, int32_t n_seq, const void* q_dev,
+                                   const int64_t* p_blocks, const int32_t* row_block_start, int32_t include_window,
+                                   const ipkv_attend_opts* opts, float* o_part_dev, float* lse_part_dev, void* stream) {
+    if (!h) return IPKV_EINVAL;
+    const ipkv_config& c = h->cfg;
+    if (layer < 0 || layer >= c.n_layers) return fail(h, IPKV_EINVAL, "layer out of range");
+    if (n_seq <= 0 || !seq_ids || !q_dev || !o_part_dev || !lse_part_dev || !row_block_start) return fail(h, IPKV_EINVAL, "bad arguments");
+    if (n_seq > c.max_seqs) return fail(h, IPKV_EINVAL, "more rows than max_seqs");
+    if (row_block_start[0] != 0 || (row_block_start[n_seq] > 0 && !p_blocks)) return fail(h, IPKV_EINVAL, "bad block lists");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int kv_splits = opts ? opts->kv_splits : 0;
+    if (kv_splits < 0) return fail(h, IPKV_EINVAL, "kv_splits must be >= 0");
+    cudaStream_t side = (opts && opts->side_stream) ? static_cast<cudaStream_t>(opts->side_stream) : h->side;
+    const float* fold_o = opts ? opts->fold_o_dev : nullptr;
+    const float* fold_lse = opts ? opts->fold_lse_dev : nullptr;
+    if ((fold_o == nullptr) != (fold_lse == nullptr)) return fail(h, IPKV_EINVAL, "fold_o_dev and fold_lse_dev must be given together");
+    CU(h, cudaSetDevice(c.device));
+    h->stats.attend_calls += 1;
+    const int64_t bt = c.block_tokens;
+
+    // tokens held by P block j of a sequence (blocks are full except the last one of a placed run)
+    auto block_tokens = [&](const SeqState& st, int64_t j) -> int64_t {
+        for (const PRun& r : st.p_runs) {
+            const int64_t nb = (r.n_tokens + bt - 1) / bt;
+            if (j >= r.first_block && j < r.first_block + nb) return std::min<int64_t>(bt, r.n_tokens - (j - r.first_block) * bt);
+        }
+        return 0;
+    };
+    struct HostPick { int row; int64_t block; int64_t tokens; };
+    std::vector<HostPick> host_picks;                       // selected blocks that are not device-resident, row-major
+    std::vector<std::vector<PlanSeg>> rows(n_seq);
+    for (int i = 0; i < n_seq; ++i) {
+        const int seq = seq_ids[i];
+        if (seq < 0 || seq >= c.max_seqs) return fail(h, IPKV_EINVAL, "sequence id out of range");
+        SeqState& st = h->state(layer, seq);
+        const int64_t used = st.router.blocks_used(REGION_P);
+        const int64_t nr = std::max<int64_t>(0, used - h->ring);
+        if (row_block_start[i + 1] < row_block_start[i]) return fail(h, IPKV_EINVAL, "bad block lists");
+        int64_t prev = -1;
+        for (int k = row_block_start[i]; k < row_block_start[i + 1]; ++k) {
+            const int64_t j = p_blocks[k];
+            if (j <= prev || j >= used) return fail(h, IPKV_EINVAL, "block ordinals must be strictly increasing and inside region P");
+            prev = j;
+            const int64_t tok = block_tokens(st, j);
+            if (tok <= 0) return fail(h, IPKV_EINTERNAL, "selected block holds no tokens");
+            if (j < nr) { host_picks.push_back(HostPick{i, j, tok}); continue; }
+            // resident: extend the previous segment when this block directly follows it in the ring and that one is full
+            const int64_t off = h->ring_off(seq) + (j % h->ring) * h->bb;
+            if (!rows[i].empty() && rows[i].back().base_id == 0 && rows[i].back().n_tokens % bt == 0 &&
+                rows[i].back().off + (rows[i].back().n_tokens / bt) * h->bb == off)
+                rows[i].back().n_tokens += tok;
+            else
+                rows[i].push_back(PlanSeg{0, off, tok});
+        }
+        if (include_window && st.router.window_fill() > 0) rows[i].push_back(PlanSeg{1, h->w_off(seq), st.router.window_fill()});
+    }
+    const char* bases[kMaxBases] = {h->ring ? h->ring_layer(layer) : nullptr, h->w_layer(layer), h->pp_dev, nullptr};
+    ipkv_status rc = run_group(h, rows, bases, q_dev, kv_splits, fold_o, fold_lse, o_part_dev, lse_part_dev, s);
+    if (rc != IPKV_OK) return rc;
+    if (host_picks.empty()) return IPKV_OK;
+    if (c.flags & IPKV_FLAG_NO_HOST_P) return fail(h, IPKV_EINTERNAL, "host-only P blocks without a host copy");
+
+    // host-only picks: gather -> one DMA per slot -> attend, pipelined over two pinned gather buffers (Sec. 4.4)
+    const int64_t slot_blocks = int64_t(c.max_seqs) * h->chunk_blocks;        // blocks one PP slot holds
+    for (int b = 0; b < 2; ++b) {
+        if (!h->gather[b]) CU(h, cudaMallocHost(&h->gather[b], size_t(slot_blocks * h->bb)));
+        if (!h->gather_done[b]) CU(h, cudaEventCreateWithFlags(&h->gather_done[b], cudaEventDisableTiming));
+    }
+    CU(h, cudaEventRecord(h->ev_main, s));
+    CU(h, cudaStreamWaitEvent(side, h->ev_main, 0));
+    CU(h, cudaStreamSynchronize(h->copy));                 // the host reads P here: write-backs must have landed
+    CU(h, cudaStreamSynchronize(s));                       // ... including prefill copies queued on the compute stream
+    size_t next = 0;
+    for (int64_t round = 0; next < host_picks.size(); ++round) {
+        const int gb = int(round & 1), slot = int(round % c.n_slots);
+        if (h->gather_busy[gb]) CU(h, cudaEventSynchronize(h->gather_done[gb]));
+        for (int i = 0; i < n_seq; ++i) rows[i].clear();
+        int64_t filled = 0;
+        while (next < host_picks.size() && filled < slot_blocks) {
+            const HostPick& pk = host_picks[next];
+            std::memcpy(h->gather[gb] + filled * h->bb, h->p_ptr(layer, seq_ids[pk.row], pk.block), size_t(h->bb));   // one memcpy per block
+            const int64_t off = slot * h->slot_bytes() + filled * h->bb;
+            auto& rr = rows[pk.row];
+            if (!rr.empty() && rr.back().n_tokens % bt == 0 && rr.back().off + (rr.back().n_tokens / bt) * h->bb == off)
+                rr.back().n_tokens += pk.tokens;
+            else
+                rr.push_back(PlanSeg{2, off, pk.tokens});
+            ++filled; ++next;
+        }
+        if (h->slot_free_set[slot]) CU(h, cudaStreamWaitEvent(side, h->slot_free[slot], 0));
+        CU(h, cudaMemcpyAsync(h->pp_dev + slot * h->slot_bytes(), h->gather[gb], size_t(filled * h->bb), cudaMemcpyHostToDevice, side));
+        h->stats.h2d_bytes += uint64_t(filled * h->bb);
+        CU(h, cudaEventRecord(h->gather_done[gb], side));
+        h->gather_busy[gb] = true;
         CU(h, cudaEventRecord(h->slot_ready[slot], side));
         CU(h, cudaStreamWaitEvent(s, h->slot_ready[slot], 0));
         rc = run_group(h, rows, bases, q_dev, kv_splits, o_part_dev, lse_part_dev, o_part_dev, lse_part_dev, s);

@@ -345,3 +345,55 @@ def test_two_engine_step_cpu_engine_plus_gpu_equals_unsplit(kind):
         torch.cuda.synchronize()
         check_partial(out2.cpu().numpy().reshape(3, hq, dv), out2_lse.cpu().numpy().reshape(3, hq),
                       np.stack([w[0] for w in full]), np.stack([w[1] for w in full]), "two engines via ipkv_merge")
+
+
+@pytest.mark.parametrize("resident", [4096, 0, 320])
+def test_block_sparse_selection(resident):
+    """Whole-block selection (Sec. 4.4): attention over the D-window plus an arbitrary set of P blocks equals the oracle
+    over exactly those tokens, whether the blocks are device-resident, host-only (gathered and sent with one DMA per
+    slot) or a mix; an empty selection leaves the window only."""
+    sh = synth.Shape("tiny", "gqa", 1, 8, 2, 128, 128, 128 ** -0.5)
+    rng = np.random.default_rng(95)
+    scale = float(np.float32(sh.scale))
+    bt, D = 64, 64
+    seqs, lens = [0, 1], {0: 1000, 1: 700}
+    with make_cache(sh, 1, 2, block_tokens=bt, window_tokens=D, chunk_tokens=128, n_slots=2, max_u_tokens_per_seq=2000,
+                    max_p_tokens_per_seq=2000, resident_tokens_per_seq=resident, share_num=1, share_den=4) as cache:
+        refs = {}
+        for s in seqs:
+            r = RefSeq(sh, bt, D, 1, 4)
+            k, v = synth.host_kv(sh, lens[s], seed=9500 + s)
+            cache.append_bulk(0, s, synth.bits_to_torch(k, DEV), synth.bits_to_torch(v, DEV), lens[s], 1, 5)
+            r.bulk(k, v, 1, 5)
+            refs[s] = r
+        for step in range(300):
+            k = synth.normal_bf16(rng, (2, 2, 128)); v = synth.normal_bf16(rng, (2, 2, 128))
+            cache.append(0, seqs, synth.bits_to_torch(k, DEV), synth.bits_to_torch(v, DEV))
+            for i, s in enumerate(seqs):
+                refs[s].append(k[i:i + 1], v[i:i + 1])
+        torch.cuda.synchronize()
+        q = synth.normal_bf16(rng, (2, 8, 128))
+        for trial in range(4):
+            picks, idxs = [], []
+            for i, s in enumerate(seqs):
+                region, blk, off = refs[s].route.dump()
+                n_blocks = int(blk[region == 1].max()) + 1
+                sel = sorted(rng.choice(n_blocks, size=[n_blocks, 5, 1, 0][trial], replace=False).tolist())
+                picks.append(sel)
+                idx = np.nonzero(((region == 1) & np.isin(blk, sel)) | (region == 2))[0]
+                idxs.append(idx)
+            o = torch.zeros((2, 8, 128), device=DEV); lse = torch.zeros((2, 8), device=DEV)
+            cache.attend_gpu_sparse(0, seqs, synth.bits_to_torch(q, DEV), picks, o, lse)
+            torch.cuda.synchronize()
+            want = [c_oracle.attend(q[i], refs[s].k, refs[s].v, idxs[i], scale) for i, s in enumerate(seqs)]
+            check_partial(o.cpu().numpy(), lse.cpu().numpy(), np.stack([w[0] for w in want]), np.stack([w[1] for w in want]),
+                          f"sparse trial {trial} resident {resident}")
+        # all blocks selected = the dense path
+        o2 = torch.zeros((2, 8, 128), device=DEV); lse2 = torch.zeros((2, 8), device=DEV)
+        cache.attend_gpu(0, seqs, synth.bits_to_torch(q, DEV), o2, lse2)
+        torch.cuda.synchronize()
+        dense = [refs[s].attend(q[i], "gpu", scale) for i, s in enumerate(seqs)]
+        check_partial(o2.cpu().numpy(), lse2.cpu().numpy(), np.stack([w[0] for w in dense]), np.stack([w[1] for w in dense]), "dense")
+        with pytest.raises(binding.IpkvError):
+            cache.attend_gpu_sparse(0, seqs, synth.bits_to_torch(q, DEV), [[3, 2], []], o, lse)      # not increasing
+        assert cache.get_stats()["device_status"] == 0
