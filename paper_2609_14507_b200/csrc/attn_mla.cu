@@ -22,6 +22,8 @@
 // HBM traffic per KV token: 1152 bytes, read exactly once per group of 16 heads.
 #include <cuda_bf16.h>
 
+#include <cstdlib>
+
 #include "kernels.h"
 #include "ptx.cuh"
 
@@ -314,8 +316,13 @@ __global__ void __launch_bounds__(kThreads, 1) attn_mla_kernel(const MlaParams p
 
 }  // namespace
 
+cudaError_t launch_attend_mla_tc(const AttnLaunch& a, cudaStream_t s);
+
 cudaError_t launch_attend_mla(const AttnLaunch& a, cudaStream_t s) {
     if (a.n_ctas <= 0 || a.n_spans <= 0) return cudaSuccess;
+    // opt-in tcgen05 / TMEM variant (attn_mla_tc.cu): correct, but slower than this kernel for 16-head groups
+    static const bool use_tc = std::getenv("IPKV_MLA_TC") != nullptr;
+    if (use_tc) return launch_attend_mla_tc(a, s);
     if (a.dim_qk != kDqk || a.dim_v != kDv || a.n_kv_heads != 1) return cudaErrorInvalidValue;
     MlaParams p;
     p.q = static_cast<const __nv_bfloat16*>(a.q);

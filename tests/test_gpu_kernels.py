@@ -182,3 +182,16 @@ def test_attend_runs_mla_peaked_softmax():
     o_ref, lse_ref = oracle_rows(q, [(k, None)], float(np.float32(scale)), dv_alias=512)
     assert np.abs(o_ref).max() > 0.5                       # O of order one: the absolute tolerance binds
     check_partial(o.cpu().numpy(), lse.cpu().numpy(), o_ref, lse_ref, "mla peaked")
+
+
+def test_mla_tcgen05_variant_matches_oracle():
+    """The opt-in tcgen05 / TMEM kernel (IPKV_MLA_TC=1) passes the same MLA parity cases; run in a child process
+    because the switch is read once per process."""
+    import os
+    import subprocess
+    import sys
+    env = dict(os.environ, IPKV_MLA_TC="1")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run([sys.executable, "-m", "pytest", "-q", "-m", "gpu", "-x", os.path.join(root, "tests", "test_gpu_kernels.py"),
+                        "-k", "attend_runs_mla"], env=env, cwd=root, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
