@@ -145,6 +145,18 @@ def populate(cache, wl, dev, rank=0):
         torch.cuda.synchronize()
 
 
+def reduce_over_ranks(x, op, device):
+    """All-reduce of one float over the ranks of the default process group ("max" or "sum"); identity for one rank.
+    Replicas do not exchange data: this only combines the timings (max) and the work counts (sum) of the ranks."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(x)
+    t = torch.tensor([float(x)], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX if op == "max" else dist.ReduceOp.SUM)
+    return float(t.item())
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -348,11 +360,7 @@ def main():
         torch.cuda.synchronize()
 
     def max_over_ranks(x):
-        if world == 1:
-            return x
-        t = torch.tensor([x], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return reduce_over_ranks(x, "max", dev)
 
     sampler = ClockSampler(local_rank)
     if rank == 0:
@@ -392,14 +400,16 @@ def main():
     h2d_stream = st1["h2d_bytes"] - st0["h2d_bytes"]
     tokens = bytes_attended // bpt
     launches = sum(st1[k] - st0[k] for k in ("attend_kernels", "reduce_kernels", "merge_kernels", "append_kernels", "pack_kernels"))
-    value = world * tokens / (ms * 1e-3)
+    tokens_all = reduce_over_ranks(tokens, "sum", dev)              # every replica's work, slowest replica's time
+    bytes_all = reduce_over_ranks(bytes_attended, "sum", dev)
+    value = tokens_all / (ms * 1e-3)
     peak, peak_kind = measured_peaks()
     ach = (bytes_attended * (n_timed / max(1, n_launch))) / (kern_ms * 1e-3) / 1e9 if kern_ms > 0 else 0.0
     roofline = {"bound": "hbm", "kernel": "attn_gqa_kernel" if sh.kind == "gqa" else "attn_mla_kernel", "achieved": ach,
                 "peak": peak, "peak_kind": peak_kind + " copy bandwidth (MEASURED_PEAKS.json hbm_gbs)" if peak_kind == "measured"
                 else "fallback 6650 GB/s", "unit": "GB/s", "frac": ach / peak, "frac_of_8000_nominal": ach / 8000.0,
                 "avg_launch_us": 1e3 * kern_ms / max(1, n_timed), "bytes_per_launch": bytes_attended / max(1, n_launch),
-                "traffic": None, "whole_step_gbs": world * bytes_attended / (ms * 1e-3) / 1e9}
+                "traffic": None, "whole_step_gbs": bytes_all / (ms * 1e-3) / 1e9}
     roofline["traffic"] = DRAM_TRAFFIC_PER_LAUNCH.get(args.workload)
 
     # ---- end to end: host buffers in, host buffer out, through the same calls ---------------------------------
@@ -447,7 +457,7 @@ def main():
         s1 = cache.get_stats()
         tok2 = (s1["kv_bytes_attended"] - s0["kv_bytes_attended"]) // bpt
         h2d = NL * (hq[0].numel() * 2 + hk[0].numel() * 2 + (0 if hv is None else hv[0].numel() * 2) + hoc[0].numel() * 4 + hlc[0].numel() * 4)
-        e2e = {"value": world * tok2 / (ms2 * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+        e2e = {"value": reduce_over_ranks(tok2, "sum", dev) / (ms2 * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": NL * hout[0].numel() * hout.element_size(), "ms_per_step": ms2 / args.steps}
     status = cache.get_stats()["device_status"]
     if status != 0:
@@ -471,7 +481,7 @@ def main():
                        "multi_gpu": "replicas only", "kv_splits": args.kv_splits,
                        "merge": "inside the split reduce" if fused else "separate ipkv_merge launch"},
             "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu,
-            "step_gbs": world * bytes_attended / (ms * 1e-3) / 1e9,
+            "step_gbs": bytes_all / (ms * 1e-3) / 1e9,
         }
         if step_lat:
             line["step_latency"] = step_lat

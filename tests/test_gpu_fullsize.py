@@ -87,3 +87,30 @@ def test_deepseek_mla_128k_sampled():
 
 def test_ragged_1m_token_batch_sampled():
     _run_step_and_check("qwen3-ragged-bs64-1m-2layers-cpu30", [(0, 0), (0, 63), (1, 31), (1, 17)])
+
+
+def _with_workload(name, wl, samples):
+    bench.WORKLOADS[name] = wl
+    try:
+        _run_step_and_check(name, samples)
+    finally:
+        del bench.WORKLOADS[name]
+
+
+def test_half_million_token_single_sequence_mla():
+    """One very long sequence: 524 288 tokens of compressed-latent cache, every tile of it on one row (the planner cuts
+    it into 148 equal chunks); all 16 heads against the oracle."""
+    sh = synth.Shape("mla-1l", "mla", 1, 16, 1, 576, 512, 192 ** -0.5)
+    _with_workload("_long", dict(shape=sh, batch=1, ctx=1 << 19, share=(0, 1), cfg_id=7), [(0, 0)])
+
+
+def test_many_short_rows_gqa():
+    """256 sequences of 2 048 tokens: more rows than CTA slots in one launch, spans that cross rows inside a CTA."""
+    sh = synth.Shape("q-1l", "gqa", 1, 32, 4, 128, 128, 128 ** -0.5)
+    _with_workload("_rows", dict(shape=sh, batch=256, ctx=2048, share=(1, 4), cfg_id=8), [(0, 0), (0, 101), (0, 255)])
+
+
+def test_head_dim_64_and_wide_groups_in_a_cache():
+    """head_dim 64 with 24 query heads per KV head (two head groups per KV head) through the handle-based path."""
+    sh = synth.Shape("d64", "gqa", 2, 48, 2, 64, 64, 64 ** -0.5)
+    _with_workload("_d64", dict(shape=sh, batch=3, ctx=5000, share=(2, 5), cfg_id=9), [(0, 1), (1, 2)])
