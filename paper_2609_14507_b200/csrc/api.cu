@@ -151,6 +151,25 @@ struct ipkv {
 
 namespace {
 
+// Makes the handle's device current for the duration of a call and restores the caller's device afterwards.
+class DeviceGuard {
+public:
+    explicit DeviceGuard(int device) {
+        if (device < 0) return;                               // no device of its own: stay on the caller's
+        if (cudaGetDevice(&prev_) != cudaSuccess) prev_ = -1;
+        err_ = (prev_ == device) ? cudaSuccess : cudaSetDevice(device);
+        changed_ = (prev_ != device) && err_ == cudaSuccess;
+    }
+    ~DeviceGuard() { if (changed_ && prev_ >= 0) cudaSetDevice(prev_); }
+    cudaError_t error() const { return err_; }
+    DeviceGuard(const DeviceGuard&) = delete;
+    DeviceGuard& operator=(const DeviceGuard&) = delete;
+private:
+    int prev_ = -1;
+    cudaError_t err_ = cudaSuccess;
+    bool changed_ = false;
+};
+
 ipkv_status fail(ipkv* h, ipkv_status s, const std::string& msg) {
     if (h) h->err = msg;
     return s;
@@ -516,7 +535,7 @@ ipkv_status ipkv_query_sizes(const ipkv_config* cfg, size_t out_bytes[5]) {
 
 ipkv_status ipkv_destroy(ipkv_t* h) {
     if (!h) return IPKV_OK;
-    cudaSetDevice(h->cfg.device);
+    DeviceGuard dev_guard(h->cfg.device);
     cudaDeviceSynchronize();
     if (h->own[0] && h->u_host) std::free(h->u_host);
     if (h->own[1] && h->p_host) cudaFreeHost(h->p_host);
@@ -557,7 +576,8 @@ ipkv_status ipkv_create(const ipkv_config* cfg, ipkv_t** out) {
     if (rc != IPKV_OK) return rc;
     int n_dev = 0;
     if (cudaGetDeviceCount(&n_dev) != cudaSuccess || cfg->device < 0 || cfg->device >= n_dev) return IPKV_ECUDA;
-    if (cudaSetDevice(cfg->device) != cudaSuccess) return IPKV_ECUDA;
+    DeviceGuard dev_guard(cfg->device);
+    if (dev_guard.error() != cudaSuccess) return IPKV_ECUDA;
     ipkv* h = new (std::nothrow) ipkv();
     if (!h) return IPKV_ENOMEM;
     h->cfg = *cfg;
@@ -655,7 +675,8 @@ ipkv_status ipkv_append_bulk(ipkv_t* h, int32_t layer, int32_t seq, const void* 
     if (st.router.blocks_for(n_cpu) > h->u_cap) return fail(h, IPKV_ERANGE, "prefill exceeds the capacity of U");
     if (st.router.blocks_for(n_gpu) > h->p_cap) return fail(h, IPKV_ERANGE, "prefill exceeds the capacity of P");
     if (no_p && st.router.blocks_for(n_gpu) > h->ring) return fail(h, IPKV_ERANGE, "prefill exceeds the resident ring and no host copy of P exists");
-    CU(h, cudaSetDevice(c.device));
+    DeviceGuard dev_guard(c.device);
+    CU(h, dev_guard.error());
     Run placed[2];
     const int n_runs = st.router.bulk(n_tokens, num0, den0, placed);
     const int64_t k_row = int64_t(c.n_kv_heads) * c.dim_qk * 2, v_row = int64_t(c.n_kv_heads) * c.dim_v * 2;
@@ -703,7 +724,8 @@ ipkv_status ipkv_flush(ipkv_t* h, int32_t layer, int32_t seq, void* stream) {
     if (!h) return IPKV_EINVAL;
     if (layer < -1 || layer >= h->cfg.n_layers) return fail(h, IPKV_EINVAL, "layer out of range");
     if (seq < -1 || seq >= h->cfg.max_seqs) return fail(h, IPKV_EINVAL, "sequence id out of range");
-    CU(h, cudaSetDevice(h->cfg.device));
+    DeviceGuard dev_guard(h->cfg.device);
+    CU(h, dev_guard.error());
     for (int l = 0; l < h->cfg.n_layers; ++l) {
         if (layer >= 0 && l != layer) continue;
         std::vector<int> seqs;
@@ -726,7 +748,8 @@ ipkv_status ipkv_append(ipkv_t* h, int32_t layer, const int32_t* seq_ids, int32_
         if (seq_ids[i] < 0 || seq_ids[i] >= c.max_seqs) return fail(h, IPKV_EINVAL, "sequence id out of range");
         for (int j = 0; j < i; ++j) if (seq_ids[j] == seq_ids[i]) return fail(h, IPKV_EINVAL, "duplicate sequence id");
     }
-    CU(h, cudaSetDevice(c.device));
+    DeviceGuard dev_guard(c.device);
+    CU(h, dev_guard.error());
     // evict full windows first, so that the newest token is always GPU-side
     {
         std::vector<int> full;
@@ -768,7 +791,8 @@ ipkv_status ipkv_attend_gpu(ipkv_t* h, int32_t layer, const int32_t* seq_ids, in
     const int kv_splits = opts ? opts->kv_splits : 0;
     if (kv_splits < 0) return fail(h, IPKV_EINVAL, "kv_splits must be >= 0");
     cudaStream_t side = (opts && opts->side_stream) ? static_cast<cudaStream_t>(opts->side_stream) : h->side;
-    CU(h, cudaSetDevice(c.device));
+    DeviceGuard dev_guard(c.device);
+    CU(h, dev_guard.error());
     h->stats.attend_calls += 1;
     const int64_t bt = c.block_tokens;
 
@@ -857,7 +881,8 @@ ipkv_status ipkv_attend_gpu_sparse(ipkv_t* h, int32_t layer, const int32_t* seq_
     const float* fold_o = opts ? opts->fold_o_dev : nullptr;
     const float* fold_lse = opts ? opts->fold_lse_dev : nullptr;
     if ((fold_o == nullptr) != (fold_lse == nullptr)) return fail(h, IPKV_EINVAL, "fold_o_dev and fold_lse_dev must be given together");
-    CU(h, cudaSetDevice(c.device));
+    DeviceGuard dev_guard(c.device);
+    CU(h, dev_guard.error());
     h->stats.attend_calls += 1;
     const int64_t bt = c.block_tokens;
 
@@ -952,7 +977,8 @@ ipkv_status ipkv_attend_cpu(ipkv_t* h, int32_t layer, const int32_t* seq_ids, in
     if (layer < 0 || layer >= c.n_layers) return fail(h, IPKV_EINVAL, "layer out of range");
     if (n_seq <= 0 || !seq_ids || !q_host || !o_part_host || !lse_part_host) return fail(h, IPKV_EINVAL, "bad arguments");
     if (!h->u_host) return fail(h, IPKV_ESTATE, "U contents are not kept (IPKV_FLAG_NO_HOST_U): nothing for the CPU engine to read");
-    CU(h, cudaSetDevice(c.device));
+    DeviceGuard dev_guard(c.device);
+    CU(h, dev_guard.error());
     { ipkv_status rc = sync_host(h); if (rc != IPKV_OK) return rc; }       // write-backs still in flight on the copy stream
     std::vector<CpuRun> runs;
     std::vector<int32_t> start(1, 0);
@@ -975,7 +1001,8 @@ ipkv_status ipkv_merge(ipkv_t* h, int32_t n_rows, int32_t dim_v, int32_t n_parts
     if (n_rows < 0 || dim_v <= 0 || dim_v % 4 != 0 || n_parts < 1 || n_parts > kMaxMergeParts || !o_parts || !lse_parts || !o_out_dev)
         return fail(h, IPKV_EINVAL, "bad merge arguments");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (h) CU(h, cudaSetDevice(h->cfg.device));
+    DeviceGuard dev_guard(h ? h->cfg.device : -1);      // no handle: stay on the caller's device
+    if (h) CU(h, dev_guard.error());
     MergeLaunch m{};
     m.n_parts = n_parts; m.n_rows = n_rows; m.dim_v = dim_v;
     m.out_o = o_out_dev; m.out_is_bf16 = o_out_is_bf16; m.out_lse = lse_out_dev;
@@ -1088,7 +1115,8 @@ ipkv_status ipkv_read_token(ipkv_t* h, int32_t layer, int32_t seq, int64_t token
     int64_t blk;
     SeqState& st = h->state(layer, seq);
     if (!st.router.locate(token, &region, &blk, &off)) return fail(h, IPKV_ERANGE, "token index out of range");
-    CU(h, cudaSetDevice(h->cfg.device));
+    DeviceGuard dev_guard(h->cfg.device);
+    CU(h, dev_guard.error());
     CU(h, cudaDeviceSynchronize());
     std::vector<char> buf(size_t(h->bb));
     bool tile = true;
@@ -1126,7 +1154,8 @@ ipkv_status ipkv_read_token(ipkv_t* h, int32_t layer, int32_t seq, int64_t token
 
 ipkv_status ipkv_get_stats(ipkv_t* h, ipkv_stats* out) {
     if (!h || !out) return IPKV_EINVAL;
-    CU(h, cudaSetDevice(h->cfg.device));
+    DeviceGuard dev_guard(h->cfg.device);
+    CU(h, dev_guard.error());
     CU(h, cudaDeviceSynchronize());
     CU(h, cudaMemcpy(&h->stats.device_status, h->status_dev, sizeof(uint32_t), cudaMemcpyDeviceToHost));
     *out = h->stats;
@@ -1135,7 +1164,8 @@ ipkv_status ipkv_get_stats(ipkv_t* h, ipkv_stats* out) {
 
 ipkv_status ipkv_profile_enable(ipkv_t* h, int32_t on) {
     if (!h) return IPKV_EINVAL;
-    CU(h, cudaSetDevice(h->cfg.device));
+    DeviceGuard dev_guard(h->cfg.device);
+    CU(h, dev_guard.error());
     if (on && h->prof_ev.empty()) {
         h->prof_ev.resize(2 * 8192);
         for (auto& e : h->prof_ev) e = nullptr;
@@ -1147,7 +1177,8 @@ ipkv_status ipkv_profile_enable(ipkv_t* h, int32_t on) {
 
 ipkv_status ipkv_profile_read(ipkv_t* h, double* attend_kernel_ms, int64_t* n_timed, int64_t* n_launches) {
     if (!h || !attend_kernel_ms || !n_timed || !n_launches) return IPKV_EINVAL;
-    CU(h, cudaSetDevice(h->cfg.device));
+    DeviceGuard dev_guard(h->cfg.device);
+    CU(h, dev_guard.error());
     CU(h, cudaDeviceSynchronize());
     double total = 0.0;
     for (size_t i = 0; i + 1 < h->prof_used; i += 2) {
