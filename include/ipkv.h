@@ -78,6 +78,13 @@ typedef enum { IPKV_LAYOUT_PLAIN = 0, IPKV_LAYOUT_TILE = 1 } ipkv_layout;
                                   CPU engine keeps its own copy, and for benchmarks                       */
 #define IPKV_FLAG_NO_HOST_P 2u /* no host copy of P: every P block must stay device-resident, otherwise
                                   an append fails with IPKV_ERANGE                                        */
+#define IPKV_FLAG_GROW_P 4u    /* P grows batch by batch instead of being pinned in full by create (Sec. 4.3,
+                                  Sec. 7.7): create pins p_initial_tokens_per_seq per (layer, sequence) — the
+                                  prefill share — and a helper thread pins room for every later eviction batch
+                                  (window_tokens per (layer, sequence), all layers and sequences in one
+                                  cudaHostAlloc) one eviction window before the batch lands.  max_p_tokens_per_seq
+                                  stays the hard capacity.  Needs chunk_tokens % window_tokens == 0 and
+                                  p_initial_tokens_per_seq % chunk_tokens == 0; p_host_pinned must be NULL.      */
 
 /* The paper's PartitionSpec (Sec. 4.3): the four regions, block granularity, eviction batch size, and
  * the share that the roofline policy of Sec. 5.3 would supply, here as an exact rational. */
@@ -94,6 +101,7 @@ typedef struct {
   int64_t max_u_tokens_per_seq;   /* capacity of U per (layer, sequence)                               */
   int64_t max_p_tokens_per_seq;   /* capacity of P per (layer, sequence)                               */
   int64_t resident_tokens_per_seq;/* device ring for the newest P blocks; 0 = stream everything        */
+  int64_t p_initial_tokens_per_seq;/* IPKV_FLAG_GROW_P: part of P pinned by create; ignored otherwise   */
   float softmax_scale;            /* 0 => 1/sqrt(dim_qk)                                               */
   int32_t share_num, share_den;   /* marginal CPU share p = num/den of decode eviction batches         */
   int32_t device;                 /* CUDA device ordinal                                               */
@@ -108,7 +116,8 @@ typedef struct {
   void* pp_dev;        size_t pp_bytes;
 } ipkv_config;
 
-/* out_bytes[0..4] = U, P, W, resident ring, PP slots.  (Table 2 of the paper is these sizes.) */
+/* out_bytes[0..4] = U, P, W, resident ring, PP slots.  (Table 2 of the paper is these sizes.)
+ * With IPKV_FLAG_GROW_P out_bytes[1] is what create pins; P then grows up to its capacity. */
 ipkv_status ipkv_query_sizes(const ipkv_config* cfg, size_t out_bytes[5]);
 
 /* The paper's `init` (Sec. 4.3): sizes the regions and pre-allocates them. */
@@ -227,6 +236,10 @@ typedef struct {
   uint64_t kv_bytes_attended;   /* tokens * bytes per token, summed over attend calls            */
   uint64_t h2d_bytes, d2h_bytes, d2d_bytes;
   uint64_t flushes, flushes_to_u;
+  /* IPKV_FLAG_GROW_P: segments pinned so far, their bytes, the page-locking time spent (by create for the
+     first, by the helper thread for the rest), and how often / how long a call had to wait for a segment
+     that was not pinned yet (0 when the one-window lookahead covers the pinning, as Sec. 7.7 expects).  */
+  uint64_t p_segments, p_pinned_bytes, p_pin_us, p_grow_waits, p_grow_wait_us;
   uint32_t device_status;       /* nonzero after a kernel's bounded wait gave up (synchronises)  */
 } ipkv_stats;
 ipkv_status ipkv_get_stats(ipkv_t* h, ipkv_stats* out);

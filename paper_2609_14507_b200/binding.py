@@ -15,7 +15,7 @@ LIB_PATH = os.path.join(HERE, "libipkv.so")
 GQA, MLA = 0, 1
 REGION_U, REGION_P, REGION_W = 0, 1, 2
 LAYOUT_PLAIN, LAYOUT_TILE = 0, 1
-FLAG_NO_HOST_U, FLAG_NO_HOST_P = 1, 2
+FLAG_NO_HOST_U, FLAG_NO_HOST_P, FLAG_GROW_P = 1, 2, 4
 OK = 0
 STATUS_NAMES = {0: "OK", 1: "EINVAL", 2: "ENOMEM", 3: "ERANGE", 4: "ESTATE", 5: "ECUDA", 6: "ETIMEOUT", 7: "EINTERNAL"}
 
@@ -35,6 +35,7 @@ class Config(C.Structure):
         ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32), ("dim_qk", C.c_int32), ("dim_v", C.c_int32),
         ("block_tokens", C.c_int32), ("window_tokens", C.c_int32), ("chunk_tokens", C.c_int32), ("n_slots", C.c_int32),
         ("max_u_tokens_per_seq", C.c_int64), ("max_p_tokens_per_seq", C.c_int64), ("resident_tokens_per_seq", C.c_int64),
+        ("p_initial_tokens_per_seq", C.c_int64),
         ("softmax_scale", C.c_float), ("share_num", C.c_int32), ("share_den", C.c_int32), ("device", C.c_int32),
         ("flags", C.c_uint32),
         ("u_host", C.c_void_p), ("u_bytes", C.c_size_t), ("p_host_pinned", C.c_void_p), ("p_bytes", C.c_size_t),
@@ -56,7 +57,8 @@ class Extent(C.Structure):
 class Stats(C.Structure):
     _fields_ = [(n, C.c_uint64) for n in (
         "attend_calls", "attend_kernels", "reduce_kernels", "merge_kernels", "append_kernels", "pack_kernels",
-        "kv_bytes_attended", "h2d_bytes", "d2h_bytes", "d2d_bytes", "flushes", "flushes_to_u")] + [("device_status", C.c_uint32)]
+        "kv_bytes_attended", "h2d_bytes", "d2h_bytes", "d2d_bytes", "flushes", "flushes_to_u",
+        "p_segments", "p_pinned_bytes", "p_pin_us", "p_grow_waits", "p_grow_wait_us")] + [("device_status", C.c_uint32)]
 
 
 class AttnShape(C.Structure):
@@ -177,7 +179,8 @@ def seq_id_array(seq_ids):
 
 def make_config(kind, n_layers, max_seqs, n_q_heads, n_kv_heads, dim_qk, dim_v, *, block_tokens=64,
                 window_tokens=256, chunk_tokens=512, n_slots=2, max_u_tokens_per_seq=0, max_p_tokens_per_seq=0,
-                resident_tokens_per_seq=0, softmax_scale=0.0, share_num=0, share_den=1, device=0, flags=0):
+                resident_tokens_per_seq=0, softmax_scale=0.0, share_num=0, share_den=1, device=0, flags=0,
+                p_initial_tokens_per_seq=0):
     c = Config()
     c.struct_size = C.sizeof(Config)
     c.kind, c.n_layers, c.max_seqs = kind, n_layers, max_seqs
@@ -185,6 +188,7 @@ def make_config(kind, n_layers, max_seqs, n_q_heads, n_kv_heads, dim_qk, dim_v, 
     c.block_tokens, c.window_tokens, c.chunk_tokens, c.n_slots = block_tokens, window_tokens, chunk_tokens, n_slots
     c.max_u_tokens_per_seq, c.max_p_tokens_per_seq = max_u_tokens_per_seq, max_p_tokens_per_seq
     c.resident_tokens_per_seq = resident_tokens_per_seq
+    c.p_initial_tokens_per_seq = p_initial_tokens_per_seq
     c.softmax_scale = softmax_scale
     c.share_num, c.share_den, c.device, c.flags = share_num, share_den, device, flags
     return c

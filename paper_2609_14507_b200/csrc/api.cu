@@ -11,12 +11,16 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <chrono>
 #include <cmath>
+#include <condition_variable>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <string>
+#include <thread>
 #include <vector>
 
 #include "../../include/ipkv.h"
@@ -92,6 +96,19 @@ struct ipkv {
     size_t sizes[5] = {0, 0, 0, 0, 0};
     char *u_host = nullptr, *p_host = nullptr, *w_dev = nullptr, *res_dev = nullptr, *pp_dev = nullptr;
     bool own[5] = {false, false, false, false, false};
+    // Pin-ahead growth of P (Sec. 4.3, Sec. 7.7): P is a list of pinned segments, each holding the same range
+    // of block ordinals of every (layer, sequence) as [layer][seq][nb].  Segment 0 (the prefill share) is pinned
+    // by create; every later segment holds one eviction batch and is pinned by a helper thread one window
+    // before its first batch lands, so the page-locking never sits on the decode path.
+    struct PSegment { char* base = nullptr; int64_t b0 = 0, nb = 0; };
+    bool grow_p = false;
+    std::vector<PSegment> pseg;          // every segment P can ever have; `base` is set once, by the pinning thread
+    std::mutex pmu;
+    std::condition_variable pcv;
+    int p_requested = 0, p_ready = 0;    // segments [0, p_ready) are usable, [p_ready, p_requested) are being pinned
+    bool p_failed = false, p_quit = false;
+    std::thread p_thread;
+    uint64_t p_pinned_bytes = 0, p_pin_us = 0;   // written by the pinning thread under pmu
     std::vector<SeqState> st;
     // staging for layout conversion on the way to host memory
     char* staging = nullptr;
@@ -141,7 +158,10 @@ struct ipkv {
     SeqState& state(int layer, int seq) { return st[size_t(layer) * cfg.max_seqs + seq]; }
     int64_t seq_index(int layer, int seq) const { return int64_t(layer) * cfg.max_seqs + seq; }
     char* u_ptr(int layer, int seq, int64_t blk) { return u_host + (seq_index(layer, seq) * u_cap + blk) * bb; }
-    char* p_ptr(int layer, int seq, int64_t blk) { return p_host + (seq_index(layer, seq) * p_cap + blk) * bb; }
+    bool has_p() const { return p_host != nullptr || grow_p; }
+    int p_segment_of(int64_t blk) const {
+        return blk < pseg[0].nb ? 0 : 1 + int((blk - pseg[0].nb) / w_blocks);
+    }
     int64_t w_off(int seq) const { return int64_t(seq) * w_blocks * bb; }                       // inside a layer
     char* w_layer(int layer) { return w_dev + int64_t(layer) * cfg.max_seqs * w_blocks * bb; }
     int64_t ring_off(int seq) const { return int64_t(seq) * ring * bb; }                        // inside a layer
@@ -183,6 +203,97 @@ ipkv_status fail_cuda(ipkv* h, cudaError_t e, const char* what) {
         if (e__ != cudaSuccess) return fail_cuda((h), e__, #call);   \
     } while (0)
 
+// ---- pin-ahead growth of P ------------------------------------------------------------------------
+size_t p_segment_bytes(const ipkv* h, int k) {
+    return size_t(int64_t(h->cfg.n_layers) * h->cfg.max_seqs * h->pseg[size_t(k)].nb * h->bb);
+}
+
+// The pinning thread: page-locks the requested segments in order (cudaHostAlloc, as the paper does).
+void pin_worker(ipkv* h) {
+    cudaSetDevice(h->cfg.device);
+    std::unique_lock<std::mutex> lk(h->pmu);
+    for (;;) {
+        h->pcv.wait(lk, [&] { return h->p_quit || (!h->p_failed && h->p_ready < h->p_requested); });
+        if (h->p_quit) return;
+        const int k = h->p_ready;
+        const size_t bytes = p_segment_bytes(h, k);
+        lk.unlock();
+        const auto t0 = std::chrono::steady_clock::now();
+        void* p = nullptr;
+        const cudaError_t e = cudaHostAlloc(&p, bytes, cudaHostAllocDefault);
+        const auto t1 = std::chrono::steady_clock::now();
+        lk.lock();
+        if (e != cudaSuccess) {
+            cudaGetLastError();                    // the error state is this thread's own
+            h->p_failed = true;
+        } else {
+            h->pseg[size_t(k)].base = static_cast<char*>(p);
+            h->p_ready = k + 1;
+            h->p_pinned_bytes += bytes;
+            h->p_pin_us += uint64_t(std::chrono::duration_cast<std::chrono::microseconds>(t1 - t0).count());
+        }
+        h->pcv.notify_all();
+    }
+}
+
+// Ask for segments [0, upto] to be pinned (no wait).
+void p_request(ipkv* h, int upto) {
+    upto = std::min(upto, int(h->pseg.size()) - 1);
+    std::lock_guard<std::mutex> lk(h->pmu);
+    if (upto + 1 > h->p_requested) { h->p_requested = upto + 1; h->pcv.notify_all(); }
+}
+
+// Make sure segment k is usable; normally it was pinned a window ago and this returns at once.
+ipkv_status p_ensure(ipkv* h, int k) {
+    if (k < 0 || k >= int(h->pseg.size())) return fail(h, IPKV_ERANGE, "P block beyond the capacity of P");
+    std::unique_lock<std::mutex> lk(h->pmu);
+    if (k < h->p_ready) return IPKV_OK;
+    if (k + 1 > h->p_requested) { h->p_requested = k + 1; h->pcv.notify_all(); }
+    const auto t0 = std::chrono::steady_clock::now();
+    h->pcv.wait(lk, [&] { return h->p_failed || k < h->p_ready; });
+    h->stats.p_grow_waits += 1;
+    h->stats.p_grow_wait_us += uint64_t(std::chrono::duration_cast<std::chrono::microseconds>(std::chrono::steady_clock::now() - t0).count());
+    if (k >= h->p_ready) return fail(h, IPKV_ENOMEM, "could not pin the next segment of P");
+    return IPKV_OK;
+}
+
+// Host address of P block `blk` of (layer, seq) and how many blocks from there are contiguous in host memory.
+ipkv_status p_locate(ipkv* h, int layer, int seq, int64_t blk, char** ptr, int64_t* contiguous) {
+    if (!h->grow_p) {
+        *ptr = h->p_host + (h->seq_index(layer, seq) * h->p_cap + blk) * h->bb;
+        *contiguous = h->p_cap - blk;
+        return IPKV_OK;
+    }
+    const int k = h->p_segment_of(blk);
+    ipkv_status rc = p_ensure(h, k);
+    if (rc != IPKV_OK) return rc;
+    const ipkv::PSegment& sg = h->pseg[size_t(k)];
+    *ptr = sg.base + (h->seq_index(layer, seq) * sg.nb + (blk - sg.b0)) * h->bb;
+    *contiguous = sg.b0 + sg.nb - blk;
+    return IPKV_OK;
+}
+
+// Calls fn(host_ptr, first_block, n_blocks) for every host-contiguous piece of P blocks [lo, hi) of (layer, seq).
+template <class F>
+ipkv_status for_p_pieces(ipkv* h, int layer, int seq, int64_t lo, int64_t hi, F&& fn) {
+    while (lo < hi) {
+        char* ptr = nullptr;
+        int64_t contiguous = 0;
+        ipkv_status rc = p_locate(h, layer, seq, lo, &ptr, &contiguous);
+        if (rc != IPKV_OK) return rc;
+        const int64_t n = std::min(hi - lo, contiguous);
+        rc = fn(ptr, lo, n);
+        if (rc != IPKV_OK) return rc;
+        lo += n;
+    }
+    return IPKV_OK;
+}
+
+// A batch was placed in P blocks up to `last_blk`: pin the segment after the one it landed in (one window ahead).
+void p_note_placed(ipkv* h, int64_t last_blk) {
+    if (h->grow_p) p_request(h, h->p_segment_of(last_blk) + 1);
+}
+
 ipkv_status validate(const ipkv_config* c, std::string* why) {
     auto bad = [&](const char* m) { *why = m; return IPKV_EINVAL; };
     if (!c) return bad("config is NULL");
@@ -195,6 +306,13 @@ ipkv_status validate(const ipkv_config* c, std::string* why) {
     if (c->max_u_tokens_per_seq < 0 || c->max_p_tokens_per_seq < 0 || c->resident_tokens_per_seq < 0) return bad("negative capacity");
     if (c->share_den <= 0 || c->share_num < 0 || c->share_num > c->share_den) return bad("share must satisfy 0 <= num <= den, den > 0");
     if (!(c->softmax_scale >= 0.f) || std::isinf(c->softmax_scale)) return bad("softmax_scale must be finite and non-negative");
+    if (c->flags & IPKV_FLAG_GROW_P) {
+        if (c->flags & IPKV_FLAG_NO_HOST_P) return bad("IPKV_FLAG_GROW_P needs the host copy of P");
+        if (c->p_host_pinned) return bad("IPKV_FLAG_GROW_P: the library pins P itself, p_host_pinned must be NULL");
+        if (c->p_initial_tokens_per_seq < 0 || c->p_initial_tokens_per_seq > c->max_p_tokens_per_seq) return bad("p_initial_tokens_per_seq out of range");
+        if (c->p_initial_tokens_per_seq % c->chunk_tokens != 0) return bad("p_initial_tokens_per_seq must be a multiple of chunk_tokens");
+        if (c->chunk_tokens % c->window_tokens != 0) return bad("IPKV_FLAG_GROW_P: chunk_tokens must be a multiple of window_tokens");
+    }
     return IPKV_OK;
 }
 
@@ -209,6 +327,7 @@ void compute_sizes(const ipkv_config* c, int64_t* bb, int64_t* u_cap, int64_t* p
     const int64_t seqs = int64_t(c->n_layers) * c->max_seqs;
     sizes[0] = (c->flags & IPKV_FLAG_NO_HOST_U) ? 0 : size_t(seqs * *u_cap * *bb);
     sizes[1] = (c->flags & IPKV_FLAG_NO_HOST_P) ? 0 : size_t(seqs * *p_cap * *bb);
+    if (c->flags & IPKV_FLAG_GROW_P) sizes[1] = size_t(seqs * (c->p_initial_tokens_per_seq / bt) * *bb);   // what create pins
     sizes[2] = size_t(seqs * (c->window_tokens / bt) * *bb);
     sizes[3] = size_t(seqs * *ring * *bb);
     sizes[4] = size_t(int64_t(c->n_slots) * c->max_seqs * (c->chunk_tokens / bt) * *bb);
@@ -367,10 +486,16 @@ ipkv_status flush_layer(ipkv* h, int layer, const int* seqs_in, int n, cudaStrea
         } else {
             if (no_p) continue;
             for (size_t k = g.first; k < g.second; ++k) {
-                const size_t bytes = size_t(jobs[k].nb * h->bb);
-                CU(h, cudaMemcpyAsync(h->p_ptr(layer, jobs[k].seq, jobs[k].r.first_block), h->wb_stage + layer_off + h->w_off(jobs[k].seq),
-                                      bytes, cudaMemcpyDeviceToHost, h->copy));
-                h->stats.d2h_bytes += bytes;
+                const Job& j = jobs[k];
+                const char* snap_k = h->wb_stage + layer_off + h->w_off(j.seq);
+                ipkv_status rc = for_p_pieces(h, layer, j.seq, j.r.first_block, j.r.first_block + j.nb,
+                                              [&](char* dst, int64_t b, int64_t nblk) -> ipkv_status {
+                    CU(h, cudaMemcpyAsync(dst, snap_k + (b - j.r.first_block) * h->bb, size_t(nblk * h->bb), cudaMemcpyDeviceToHost, h->copy));
+                    h->stats.d2h_bytes += uint64_t(nblk * h->bb);
+                    return IPKV_OK;
+                });
+                if (rc != IPKV_OK) return rc;
+                p_note_placed(h, j.r.first_block + j.nb - 1);
             }
         }
     }
@@ -537,6 +662,12 @@ ipkv_status ipkv_destroy(ipkv_t* h) {
     if (!h) return IPKV_OK;
     DeviceGuard dev_guard(h->cfg.device);
     cudaDeviceSynchronize();
+    if (h->p_thread.joinable()) {
+        { std::lock_guard<std::mutex> lk(h->pmu); h->p_quit = true; }
+        h->pcv.notify_all();
+        h->p_thread.join();
+    }
+    for (auto& sg : h->pseg) if (sg.base) cudaFreeHost(sg.base);
     if (h->own[0] && h->u_host) std::free(h->u_host);
     if (h->own[1] && h->p_host) cudaFreeHost(h->p_host);
     if (h->own[2] && h->w_dev) cudaFree(h->w_dev);
@@ -593,8 +724,26 @@ ipkv_status ipkv_create(const ipkv_config* cfg, ipkv_t** out) {
                                                   {cfg->w_dev, cfg->w_bytes}, {cfg->resident_dev, cfg->resident_bytes},
                                                   {cfg->pp_dev, cfg->pp_bytes}};
     char** dst[5] = {&h->u_host, &h->p_host, &h->w_dev, &h->res_dev, &h->pp_dev};
+    h->grow_p = (cfg->flags & IPKV_FLAG_GROW_P) != 0;
+    if (h->grow_p) {
+        const int64_t nb0 = cfg->p_initial_tokens_per_seq / cfg->block_tokens;
+        h->pseg.push_back(ipkv::PSegment{nullptr, 0, nb0});
+        for (int64_t b = nb0; b < h->p_cap; b += h->w_blocks)
+            h->pseg.push_back(ipkv::PSegment{nullptr, b, h->w_blocks});   // the last one may reach past p_cap: capacity checks use p_cap
+        if (nb0 > 0) {                            // the prefill share: pinned here, "during model loading and warm-up"
+            void* p0 = nullptr;
+            const auto t0 = std::chrono::steady_clock::now();
+            if (cudaHostAlloc(&p0, h->sizes[1], cudaHostAllocDefault) != cudaSuccess) { cudaGetLastError(); return bail(IPKV_ENOMEM); }
+            h->pseg[0].base = static_cast<char*>(p0);
+            h->p_pinned_bytes = h->sizes[1];
+            h->p_pin_us = uint64_t(std::chrono::duration_cast<std::chrono::microseconds>(std::chrono::steady_clock::now() - t0).count());
+        }
+        h->p_ready = h->p_requested = 1;
+        h->p_thread = std::thread(pin_worker, h);
+        p_request(h, 1);                          // the first decode batch's segment, one window ahead
+    }
     for (int i = 0; i < 5; ++i) {
-        if (h->sizes[i] == 0) continue;
+        if (h->sizes[i] == 0 || (i == 1 && h->grow_p)) continue;
         if (prov[i].p) {
             if (prov[i].n < h->sizes[i]) return bail(IPKV_ENOMEM);
             *dst[i] = static_cast<char*>(prov[i].p);
@@ -625,7 +774,7 @@ ipkv_status ipkv_create(const ipkv_config* cfg, ipkv_t** out) {
     h->wb_busy.resize(cfg->n_layers); h->wb_busy_set.assign(cfg->n_layers, 0);
     for (int i = 0; i < cfg->n_layers; ++i)
         if (cudaEventCreateWithFlags(&h->wb_busy[i], cudaEventDisableTiming) != cudaSuccess) return bail(IPKV_ECUDA);
-    if (h->sizes[0] > 0 || h->sizes[1] > 0) {      // some host copy is kept: snapshots of the windows for the write-back
+    if (h->sizes[0] > 0 || h->sizes[1] > 0 || h->grow_p) {      // some host copy is kept: snapshots of the windows for the write-back
         if (cudaMalloc(&h->wb_stage, h->sizes[2]) != cudaSuccess) return bail(IPKV_ENOMEM);
         if (h->sizes[0] > 0 && cudaMallocHost(&h->wb_bounce, size_t(int64_t(cfg->max_seqs) * h->w_blocks * h->bb)) != cudaSuccess) return bail(IPKV_ENOMEM);
     }
@@ -709,10 +858,18 @@ ipkv_status ipkv_append_bulk(ipkv_t* h, int32_t layer, int32_t seq, const void* 
             const char* vs = v_dev ? static_cast<const char*>(v_dev) + (r.first_token + tok0) * v_row : nullptr;
             CU(h, launch_pack(h->geom, to_u ? 0 : 1, ks, vs, tok1 - tok0, dst, 0, s));
             h->stats.pack_kernels += 1;
-            char* host = to_u ? h->u_ptr(layer, seq, r.first_block + j) : (no_p ? nullptr : h->p_ptr(layer, seq, r.first_block + j));
-            if (host) {
-                CU(h, cudaMemcpyAsync(host, dst, size_t((j_end - j) * h->bb), cudaMemcpyDeviceToHost, s));
+            if (to_u) {
+                CU(h, cudaMemcpyAsync(h->u_ptr(layer, seq, r.first_block + j), dst, size_t((j_end - j) * h->bb), cudaMemcpyDeviceToHost, s));
                 h->stats.d2h_bytes += uint64_t((j_end - j) * h->bb);
+            } else if (!no_p) {
+                const int64_t b_lo = r.first_block + j;
+                rc = for_p_pieces(h, layer, seq, b_lo, r.first_block + j_end, [&](char* host, int64_t b, int64_t nblk) -> ipkv_status {
+                    CU(h, cudaMemcpyAsync(host, dst + (b - b_lo) * h->bb, size_t(nblk * h->bb), cudaMemcpyDeviceToHost, s));
+                    h->stats.d2h_bytes += uint64_t(nblk * h->bb);
+                    return IPKV_OK;
+                });
+                if (rc != IPKV_OK) return rc;
+                p_note_placed(h, r.first_block + j_end - 1);
             }
             j = j_end;
         }
@@ -834,25 +991,67 @@ ipkv_status ipkv_attend_gpu(ipkv_t* h, int32_t layer, const int32_t* seq_ids, in
     CU(h, cudaEventRecord(h->ev_copy, h->copy));           // ... or by write-backs on the copy stream
     CU(h, cudaStreamWaitEvent(side, h->ev_copy, 0));
     const int64_t chunk_bytes = h->chunk_blocks * h->bb;
+    // A chunk that lies in grown segments holds chunk_blocks / w_blocks whole eviction batches. Each batch is one
+    // contiguous [seq][w_blocks] range of host memory per layer, so it travels as ONE copy for all sequences (the
+    // paper's load unit: a whole batch, Sec. 4.2) and the slot is laid out [batch][seq][w_blocks]; the per-sequence
+    // form is kept for calls that list under half of the sequences, and for segment 0.
+    const int64_t seg0_blocks = h->grow_p ? h->pseg[0].nb : INT64_MAX;
+    const bool whole_batches = h->grow_p && int64_t(n_seq) * 2 >= c.max_seqs;
+    const int64_t batch_bytes = int64_t(c.max_seqs) * h->w_blocks * h->bb;      // one batch of every sequence, one layer
     for (int64_t ch = 0; ch < max_stream_chunks; ++ch) {
         const int slot = int(ch % c.n_slots);
         if (h->slot_free_set[slot]) CU(h, cudaStreamWaitEvent(side, h->slot_free[slot], 0));
+        const int64_t lo = ch * h->chunk_blocks;
+        const bool batched = whole_batches && lo >= seg0_blocks;
+        if (batched) {
+            int64_t hi_all = lo;                                       // blocks some listed sequence still needs from the host
+            for (int i = 0; i < n_seq; ++i) {
+                const int64_t nr = std::max<int64_t>(0, h->state(layer, seq_ids[i]).router.blocks_used(REGION_P) - h->ring);
+                hi_all = std::max(hi_all, std::min(nr, lo + h->chunk_blocks));
+            }
+            for (int64_t b = lo; b < hi_all; b += h->w_blocks) {
+                char* src = nullptr;
+                int64_t contiguous = 0;
+                rc = p_locate(h, layer, 0, b, &src, &contiguous);       // sequence 0's blocks open the batch
+                if (rc != IPKV_OK) return rc;
+                CU(h, cudaMemcpyAsync(h->pp_dev + slot * h->slot_bytes() + ((b - lo) / h->w_blocks) * batch_bytes, src, size_t(batch_bytes),
+                                      cudaMemcpyHostToDevice, side));
+                h->stats.h2d_bytes += uint64_t(batch_bytes);
+            }
+        }
         for (int i = 0; i < n_seq; ++i) {
             rows[i].clear();
             const int seq = seq_ids[i];
             SeqState& st = h->state(layer, seq);
             const int64_t nr = std::max<int64_t>(0, st.router.blocks_used(REGION_P) - h->ring);
-            const int64_t lo = ch * h->chunk_blocks, hi = std::min(nr, lo + h->chunk_blocks);
+            const int64_t hi = std::min(nr, lo + h->chunk_blocks);
             if (lo >= hi) continue;
-            char* dst = h->pp_dev + slot * h->slot_bytes() + int64_t(i) * chunk_bytes;
-            CU(h, cudaMemcpyAsync(dst, h->p_ptr(layer, seq, lo), size_t((hi - lo) * h->bb), cudaMemcpyHostToDevice, side));
-            h->stats.h2d_bytes += uint64_t((hi - lo) * h->bb);
+            const int64_t row_base = slot * h->slot_bytes() + int64_t(i) * chunk_bytes;
+            // slot offset of block j (lo <= j < hi) of this row
+            auto slot_off = [&](int64_t j) -> int64_t {
+                if (!batched) return row_base + (j - lo) * h->bb;
+                const int64_t batch = (j - lo) / h->w_blocks, within = (j - lo) % h->w_blocks;
+                return slot * h->slot_bytes() + batch * batch_bytes + (int64_t(seq) * h->w_blocks + within) * h->bb;
+            };
+            if (!batched) {
+                rc = for_p_pieces(h, layer, seq, lo, hi, [&](char* src, int64_t b, int64_t nblk) -> ipkv_status {
+                    CU(h, cudaMemcpyAsync(h->pp_dev + slot_off(b), src, size_t(nblk * h->bb), cudaMemcpyHostToDevice, side));
+                    h->stats.h2d_bytes += uint64_t(nblk * h->bb);
+                    return IPKV_OK;
+                });
+                if (rc != IPKV_OK) return rc;
+            }
             for (const PRun& r : st.p_runs) {
                 const int64_t nb = (r.n_tokens + bt - 1) / bt;
-                const int64_t a = std::max(lo, r.first_block), b = std::min(hi, r.first_block + nb);
-                if (a >= b) continue;
-                const int64_t tok = std::min(r.n_tokens - (a - r.first_block) * bt, (b - a) * bt);
-                rows[i].push_back(PlanSeg{2, slot * h->slot_bytes() + int64_t(i) * chunk_bytes + (a - lo) * h->bb, tok});
+                int64_t a = std::max(lo, r.first_block);
+                const int64_t b = std::min(hi, r.first_block + nb);
+                while (a < b) {
+                    // blocks [a, e) are contiguous in the slot: the whole range, or up to the end of the batch
+                    const int64_t e = batched ? std::min(b, lo + ((a - lo) / h->w_blocks + 1) * h->w_blocks) : b;
+                    const int64_t tok = std::min(r.n_tokens - (a - r.first_block) * bt, (e - a) * bt);
+                    rows[i].push_back(PlanSeg{2, slot_off(a), tok});
+                    a = e;
+                }
             }
         }
         CU(h, cudaEventRecord(h->slot_ready[slot], side));
@@ -946,7 +1145,11 @@ ipkv_status ipkv_attend_gpu_sparse(ipkv_t* h, int32_t layer, const int32_t* seq_
         int64_t filled = 0;
         while (next < host_picks.size() && filled < slot_blocks) {
             const HostPick& pk = host_picks[next];
-            std::memcpy(h->gather[gb] + filled * h->bb, h->p_ptr(layer, seq_ids[pk.row], pk.block), size_t(h->bb));   // one memcpy per block
+            char* blk_host = nullptr;
+            int64_t contiguous = 0;
+            ipkv_status lrc = p_locate(h, layer, seq_ids[pk.row], pk.block, &blk_host, &contiguous);
+            if (lrc != IPKV_OK) return lrc;
+            std::memcpy(h->gather[gb] + filled * h->bb, blk_host, size_t(h->bb));   // one memcpy per block
             const int64_t off = slot * h->slot_bytes() + filled * h->bb;
             auto& rr = rows[pk.row];
             if (!rr.empty() && rr.back().n_tokens % bt == 0 && rr.back().off + (rr.back().n_tokens / bt) * h->bb == off)
@@ -1044,26 +1247,52 @@ ipkv_status ipkv_views(ipkv_t* h, int32_t layer, int32_t seq, ipkv_extent* out, 
     if (!n_out || (cap > 0 && !out)) return fail(h, IPKV_EINVAL, "bad arguments");
     SeqState& st = h->state(layer, seq);
     const auto& runs = st.router.runs();
-    const int total = int(runs.size()) + (st.router.window_fill() > 0 ? 1 : 0);
+    const int64_t bt = h->cfg.block_tokens;
+    // with a grown P a run that crosses a segment boundary is reported as one extent per contiguous piece
+    auto p_pieces = [&](const Run& r) -> int {
+        if (!h->grow_p || r.region != REGION_P || r.n_tokens == 0) return 1;
+        const int64_t last = r.first_block + (r.n_tokens + bt - 1) / bt - 1;
+        return h->p_segment_of(last) - h->p_segment_of(r.first_block) + 1;
+    };
+    int total = st.router.window_fill() > 0 ? 1 : 0;
+    for (const Run& r : runs) total += p_pieces(r);
     *n_out = total;
     if (cap < total) return cap == 0 ? IPKV_OK : fail(h, IPKV_ERANGE, "extent array too small");
-    const int64_t bt = h->cfg.block_tokens;
     const int64_t used_p = st.router.blocks_used(REGION_P);
     const int64_t nr = std::max<int64_t>(0, used_p - h->ring);
     int k = 0;
-    for (const Run& r : runs) {
-        ipkv_extent& e = out[k++];
-        e.region = r.region; e.first_token = r.first_token; e.n_tokens = r.n_tokens; e.region_block = r.first_block;
-        e.block_bytes = h->bb; e.host_ptr = nullptr; e.dev_ptr = nullptr;
-        const int64_t nb = (r.n_tokens + bt - 1) / bt;
-        if (r.region == REGION_U) {
-            e.layout = IPKV_LAYOUT_PLAIN;
-            if (h->u_host) e.host_ptr = h->u_ptr(layer, seq, r.first_block);
-        } else {
-            e.layout = IPKV_LAYOUT_TILE;
-            if (h->p_host) e.host_ptr = h->p_ptr(layer, seq, r.first_block);
-            if (h->ring > 0 && r.first_block >= nr && (r.first_block % h->ring) + nb <= h->ring)
-                e.dev_ptr = h->ring_layer(layer) + h->ring_off(seq) + (r.first_block % h->ring) * h->bb;
+    for (const Run& whole : runs) {
+        const int64_t whole_nb = (whole.n_tokens + bt - 1) / bt;
+        int64_t done_blocks = 0;
+        for (int piece = 0, n_pieces = p_pieces(whole); piece < n_pieces; ++piece) {
+            Run r = whole;
+            if (n_pieces > 1) {
+                r.first_block = whole.first_block + done_blocks;
+                const ipkv::PSegment& sg = h->pseg[size_t(h->p_segment_of(r.first_block))];
+                const int64_t nblk = std::min(whole_nb - done_blocks, sg.b0 + sg.nb - r.first_block);
+                r.first_token = whole.first_token + done_blocks * bt;
+                r.n_tokens = std::min(whole.n_tokens - done_blocks * bt, nblk * bt);
+                done_blocks += nblk;
+            }
+            ipkv_extent& e = out[k++];
+            e.region = r.region; e.first_token = r.first_token; e.n_tokens = r.n_tokens; e.region_block = r.first_block;
+            e.block_bytes = h->bb; e.host_ptr = nullptr; e.dev_ptr = nullptr;
+            const int64_t nb = (r.n_tokens + bt - 1) / bt;
+            if (r.region == REGION_U) {
+                e.layout = IPKV_LAYOUT_PLAIN;
+                if (h->u_host) e.host_ptr = h->u_ptr(layer, seq, r.first_block);
+            } else {
+                e.layout = IPKV_LAYOUT_TILE;
+                if (h->has_p() && r.n_tokens > 0) {
+                    char* host = nullptr;
+                    int64_t contiguous = 0;
+                    rc = p_locate(h, layer, seq, r.first_block, &host, &contiguous);
+                    if (rc != IPKV_OK) return rc;
+                    e.host_ptr = host;
+                }
+                if (h->ring > 0 && r.first_block >= nr && (r.first_block % h->ring) + nb <= h->ring)
+                    e.dev_ptr = h->ring_layer(layer) + h->ring_off(seq) + (r.first_block % h->ring) * h->bb;
+            }
         }
     }
     if (st.router.window_fill() > 0) {
@@ -1126,8 +1355,12 @@ ipkv_status ipkv_read_token(ipkv_t* h, int32_t layer, int32_t seq, int64_t token
         std::memcpy(buf.data(), h->u_ptr(layer, seq, blk), size_t(h->bb));
         tile = false;
     } else if (region == REGION_P) {
-        if (h->p_host) {
-            std::memcpy(buf.data(), h->p_ptr(layer, seq, blk), size_t(h->bb));
+        if (h->has_p()) {
+            char* blk_host = nullptr;
+            int64_t contiguous = 0;
+            rc = p_locate(h, layer, seq, blk, &blk_host, &contiguous);
+            if (rc != IPKV_OK) return rc;
+            std::memcpy(buf.data(), blk_host, size_t(h->bb));
         } else {
             CU(h, cudaMemcpy(buf.data(), h->ring_layer(layer) + h->ring_off(seq) + (blk % h->ring) * h->bb, size_t(h->bb), cudaMemcpyDeviceToHost));
         }
@@ -1158,6 +1391,12 @@ ipkv_status ipkv_get_stats(ipkv_t* h, ipkv_stats* out) {
     CU(h, dev_guard.error());
     CU(h, cudaDeviceSynchronize());
     CU(h, cudaMemcpy(&h->stats.device_status, h->status_dev, sizeof(uint32_t), cudaMemcpyDeviceToHost));
+    if (h->grow_p) {
+        std::lock_guard<std::mutex> lk(h->pmu);
+        h->stats.p_segments = uint64_t(h->p_ready) - (h->pseg[0].nb == 0 ? 1 : 0);
+        h->stats.p_pinned_bytes = h->p_pinned_bytes;
+        h->stats.p_pin_us = h->p_pin_us;
+    }
     *out = h->stats;
     return h->stats.device_status ? fail(h, IPKV_ETIMEOUT, "a kernel's bounded wait gave up; results of that call are invalid") : IPKV_OK;
 }

@@ -397,3 +397,77 @@ def test_block_sparse_selection(resident):
         with pytest.raises(binding.IpkvError):
             cache.attend_gpu_sparse(0, seqs, synth.bits_to_torch(q, DEV), [[3, 2], []], o, lse)      # not increasing
         assert cache.get_stats()["device_status"] == 0
+
+
+@pytest.mark.parametrize("resident,seqs", [(0, [0, 2, 3]), (0, [3]), (96, [0, 1, 2, 3]), (4096, [0, 2, 3])])
+def test_pinned_region_grows_batch_by_batch(resident, seqs):
+    """P pinned a batch at a time (Sec. 4.3 / Sec. 7.7) instead of in full by create: same routing, same contents,
+    same attention.  The prefill of one sequence outgrows what create pinned (the call then waits for the helper
+    thread); decode batches land in segments pinned one window ahead.  Listing most sequences takes the
+    whole-batch H2D copies, listing one the per-sequence copies; a small resident ring mixes both with the ring."""
+    sh = synth.Shape("tiny", "gqa", 2, 8, 2, 128, 128, 128 ** -0.5)
+    n_layers, steps, bt, D = 2, 200, 16, 32
+    lens = {0: 100, 1: 40, 2: 0, 3: 257}
+    rng = np.random.default_rng(77)
+    scale = float(np.float32(sh.scale))
+    with make_cache(sh, n_layers, 4, block_tokens=bt, window_tokens=D, chunk_tokens=64, n_slots=2, max_u_tokens_per_seq=600,
+                    max_p_tokens_per_seq=640, p_initial_tokens_per_seq=64, resident_tokens_per_seq=resident,
+                    share_num=1, share_den=4, flags=binding.FLAG_GROW_P) as cache:
+        seg0 = binding.ipkv_query_sizes(cache.cfg)["p"]          # what create pins; the first batch's segment may follow at once
+        assert seg0 > 0 and cache.get_stats()["p_pinned_bytes"] in (seg0, seg0 + seg0 // 2)
+        refs = {}
+        for layer in range(n_layers):
+            for s in seqs:
+                r = RefSeq(sh, bt, D, 1, 4)
+                k, v = synth.host_kv(sh, lens[s], seed=7000 + 10 * layer + s)
+                cache.append_bulk(layer, s, synth.bits_to_torch(k, DEV) if lens[s] else None,
+                                  synth.bits_to_torch(v, DEV) if lens[s] else None, lens[s], 2, 5)
+                r.bulk(k, v, 2, 5)
+                refs[(layer, s)] = r
+        for step in range(steps):
+            for layer in range(n_layers):
+                k = synth.normal_bf16(rng, (len(seqs), 2, 128)); v = synth.normal_bf16(rng, (len(seqs), 2, 128))
+                cache.append(layer, seqs, synth.bits_to_torch(k, DEV), synth.bits_to_torch(v, DEV))
+                for i, s in enumerate(seqs):
+                    refs[(layer, s)].append(k[i:i + 1], v[i:i + 1])
+                if step % 17 == 0 or step == steps - 1:
+                    q = synth.normal_bf16(rng, (len(seqs), 8, 128))
+                    o = torch.zeros((len(seqs), 8, 128), device=DEV); lse = torch.zeros((len(seqs), 8), device=DEV)
+                    cache.attend_gpu(layer, seqs, synth.bits_to_torch(q, DEV), o, lse)
+                    parts = [refs[(layer, s)].attend(q[i], "gpu", scale) for i, s in enumerate(seqs)]
+                    torch.cuda.synchronize()
+                    check_partial(o.cpu().numpy(), lse.cpu().numpy(), np.stack([p[0] for p in parts]), np.stack([p[1] for p in parts]),
+                                  f"step {step} layer {layer}")
+        torch.cuda.synchronize()
+        for (layer, s), r in refs.items():
+            check_routing(cache, layer, s, r)
+            check_contents(cache, layer, s, r, range(0, len(r.route), 5))
+            # the extents tile the sequence in order, and every P extent's host pointer holds that extent's first token
+            ext = cache.views(layer, s)
+            assert [e.first_token for e in ext] == [int(x) for x in np.cumsum([0] + [e.n_tokens for e in ext[:-1]])]
+            assert sum(e.n_tokens for e in ext) == len(r.route)
+            for e in ext:
+                if e.region == 1:                     # P: TILE blocks, contiguous within the extent
+                    t0, n = e.first_token, e.n_tokens
+                    nb = -(-n // bt)
+                    want = layouts.blocks_image(r.k[t0:t0 + n], r.v[t0:t0 + n], bt, True)
+                    written = layouts.blocks_image(np.ones_like(r.k[t0:t0 + n]), np.ones_like(r.v[t0:t0 + n]), bt, True) != 0
+                    np.testing.assert_array_equal(host_bytes(e.host_ptr, nb * e.block_bytes)[written], want[written])   # rows past a partial block's end are unspecified
+        st = cache.get_stats()
+        p_blocks = max(r.route.counts()["p_blocks"] for r in refs.values())
+        assert st["device_status"] == 0
+        assert st["p_segments"] >= 1 + -(-(p_blocks - 64 // bt) // (D // bt))       # segment 0 + one per started batch range
+        assert st["p_pinned_bytes"] > binding.ipkv_query_sizes(cache.cfg)["p"]
+        if 3 in seqs:
+            assert st["p_grow_waits"] >= 1                                       # the long prefill outgrew segment 0
+
+
+def test_grow_p_rejects_bad_configs():
+    sh = synth.Shape("tiny", "gqa", 2, 8, 2, 128, 128, 128 ** -0.5)
+    base = dict(block_tokens=16, window_tokens=32, chunk_tokens=64, max_u_tokens_per_seq=64, max_p_tokens_per_seq=640)
+    for bad in (dict(p_initial_tokens_per_seq=32), dict(p_initial_tokens_per_seq=704), dict(window_tokens=48, chunk_tokens=64),
+                dict(flags=binding.FLAG_GROW_P | binding.FLAG_NO_HOST_P)):
+        kw = dict(base, flags=binding.FLAG_GROW_P)
+        kw.update(bad)
+        with pytest.raises(binding.IpkvError):
+            make_cache(sh, 1, 2, **kw)
