@@ -93,6 +93,15 @@ for _pct in (10, 30, 50, 70, 100):
 for _pct, _share in ((0, (0, 1)), (50, (1, 2)), (100, (1, 1))):
     WORKLOADS[f"qwen3-30b-a3b-bs8-8k-cpu{_pct}-hostcopies"] = dict(shape=synth.QWEN3, batch=8, ctx=8192, share=_share, cfg_id=3,
                                                                    host_copies=True)
+# The same decode with other eviction windows D (the paper: any D in 256-1024 leaves the steady state unchanged,
+# Sec. 4.2) and with P grown batch by batch, each batch's memory pinned one window ahead by a helper thread
+# (Sec. 4.3, Sec. 7.7), instead of pinned in full at start-up.  Used with --latency.
+for _d in (256, 512, 1024):
+    for _pct, _share in ((0, (0, 1)), (50, (1, 2))):
+        WORKLOADS[f"qwen3-30b-a3b-bs8-8k-cpu{_pct}-hostcopies-d{_d}"] = dict(
+            shape=synth.QWEN3, batch=8, ctx=8192, share=_share, cfg_id=3, host_copies=True, window=_d, chunk_tokens=1024)
+        WORKLOADS[f"qwen3-30b-a3b-bs8-8k-cpu{_pct}-growp-d{_d}"] = dict(
+            shape=synth.QWEN3, batch=8, ctx=8192, share=_share, cfg_id=3, host_copies=True, window=_d, chunk_tokens=1024, grow_p=True)
 
 
 def seq_lens(wl):
@@ -115,7 +124,8 @@ def make_cache(wl, device_index, decode_steps):
     sh = wl["shape"]
     num0, den0 = wl["share"]
     longest = max(seq_lens(wl))
-    grow = WINDOW * (decode_steps // WINDOW + 2)
+    window = wl.get("window", WINDOW)
+    grow = window * (decode_steps // window + 2)
     p_cap = longest - cpu_tokens(longest, num0, den0) + grow if num0 < den0 else grow
     p_cap = max(p_cap, max(n - cpu_tokens(n, num0, den0) for n in seq_lens(wl)) + grow)
     kind = binding.MLA if sh.kind == "mla" else binding.GQA
@@ -126,8 +136,16 @@ def make_cache(wl, device_index, decode_steps):
         # keep the newest (100 - stream_pct) % of the prefill's P share resident; P itself lives in pinned host memory
         resident = BLOCK * (((longest - cpu_tokens(longest, num0, den0)) * (100 - wl["stream_pct"]) // 100) // BLOCK)
         flags = binding.FLAG_NO_HOST_U
+    p_initial = 0
+    if wl.get("grow_p"):
+        # create pins the prefill's share (rounded up to whole chunks); decode batches get their memory as they come
+        chunk = wl.get("chunk_tokens", 512)
+        p_initial = -(-(longest - cpu_tokens(longest, num0, den0)) // chunk) * chunk
+        p_cap = max(p_cap, p_initial)
+        flags |= binding.FLAG_GROW_P
     cfg = binding.make_config(kind, sh.n_layers, wl["batch"], sh.n_q_heads, sh.n_kv_heads, sh.dim_qk, sh.dim_v,
-                              block_tokens=BLOCK, window_tokens=WINDOW, chunk_tokens=wl.get("chunk_tokens", 512), n_slots=2,
+                              block_tokens=BLOCK, window_tokens=window, chunk_tokens=wl.get("chunk_tokens", 512), n_slots=2,
+                              p_initial_tokens_per_seq=p_initial,
                               max_u_tokens_per_seq=longest + grow, max_p_tokens_per_seq=p_cap, resident_tokens_per_seq=resident,
                               softmax_scale=sh.scale, share_num=num0, share_den=den0, device=device_index, flags=flags)
     return binding.Cache(cfg)
@@ -522,7 +540,7 @@ def main():
             "dtype": "bf16", "data": "synthetic",
             "config": {"workload": args.workload, "layers": NL, "batch": B,
                        "context": ctx if "lens" not in wl else f"ragged {min(lens)}..{max(lens)} (sum {sum(lens)})",
-                       "cpu_share": f"{num0}/{den0}", "gpu_share_tokens_per_seq_mean": n_gpu0 + 1, "bytes_per_kv_token": bpt, "block_tokens": BLOCK, "window_tokens": WINDOW,
+                       "cpu_share": f"{num0}/{den0}", "gpu_share_tokens_per_seq_mean": n_gpu0 + 1, "bytes_per_kv_token": bpt, "block_tokens": BLOCK, "window_tokens": wl.get("window", WINDOW),
                        "gpu_share": "HBM-resident", "host_copies_of_U_and_P": "off (benchmark)", "cpu_partial": "synthetic values",
                        "l2": l2_note,
                        "multi_gpu": "replicas only", "kv_splits": args.kv_splits,
@@ -534,6 +552,12 @@ def main():
             line["step_latency"] = step_lat
         if wl.get("host_copies"):
             line["config"]["host_copies_of_U_and_P"] = "on (P pinned, U unpinned); write-back on a copy stream"
+        if wl.get("grow_p"):
+            line["config"]["host_copies_of_U_and_P"] += "; P grown batch by batch, pinned one window ahead by a helper thread"
+            line["p_growth"] = {k: st1[k] for k in ("p_segments", "p_pinned_bytes", "p_pin_us", "p_grow_waits", "p_grow_wait_us",
+                                                       "p_register_us", "p_register_calls", "p_register_max_us")}
+            line["p_growth"]["segments_pinned_in_timed_region"] = st1["p_segments"] - st0["p_segments"]
+            line["p_growth"]["pin_ms_per_mb"] = (st1["p_pin_us"] / 1e3) / max(1.0, st1["p_pinned_bytes"] / 1e6)
         if "stream_pct" in wl:
             # the box's pinned host-to-device plateau, measured here with a 256 MB copy (best of 10 after 2 warm-ups)
             hp = torch.empty(256 << 20, dtype=torch.uint8).pin_memory(); dp = torch.empty(256 << 20, dtype=torch.uint8, device=dev)

@@ -82,7 +82,9 @@ typedef enum { IPKV_LAYOUT_PLAIN = 0, IPKV_LAYOUT_TILE = 1 } ipkv_layout;
                                   Sec. 7.7): create pins p_initial_tokens_per_seq per (layer, sequence) — the
                                   prefill share — and a helper thread pins room for every later eviction batch
                                   (window_tokens per (layer, sequence), all layers and sequences in one
-                                  cudaHostAlloc) one eviction window before the batch lands.  max_p_tokens_per_seq
+                                  allocation, faulted in and then page-locked a layer's range at a time so that
+                                  no single driver call is long) one eviction window before the batch lands.
+                                  max_p_tokens_per_seq
                                   stays the hard capacity.  Needs chunk_tokens % window_tokens == 0 and
                                   p_initial_tokens_per_seq % chunk_tokens == 0; p_host_pinned must be NULL.      */
 
@@ -240,6 +242,7 @@ typedef struct {
      first, by the helper thread for the rest), and how often / how long a call had to wait for a segment
      that was not pinned yet (0 when the one-window lookahead covers the pinning, as Sec. 7.7 expects).  */
   uint64_t p_segments, p_pinned_bytes, p_pin_us, p_grow_waits, p_grow_wait_us;
+  uint64_t p_register_us, p_register_calls, p_register_max_us;  /* the page-locking calls alone: total, count, longest */
   uint32_t device_status;       /* nonzero after a kernel's bounded wait gave up (synchronises)  */
 } ipkv_stats;
 ipkv_status ipkv_get_stats(ipkv_t* h, ipkv_stats* out);

@@ -9,6 +9,7 @@
 //                    soon as its copy has landed and folded into the running partial
 //   ipkv_merge       LSE join with the CPU-side partial
 #include <cuda_runtime.h>
+#include <sys/mman.h>
 
 #include <algorithm>
 #include <chrono>
@@ -107,8 +108,10 @@ struct ipkv {
     std::condition_variable pcv;
     int p_requested = 0, p_ready = 0;    // segments [0, p_ready) are usable, [p_ready, p_requested) are being pinned
     bool p_failed = false, p_quit = false;
+    int p_waiters = 0;                   // calls blocked in p_ensure: the pinning thread then stops pacing itself
+    uint64_t p_tick = 0;                 // decode steps seen (appends to layer 0): the pinning thread's pace
     std::thread p_thread;
-    uint64_t p_pinned_bytes = 0, p_pin_us = 0;   // written by the pinning thread under pmu
+    uint64_t p_pinned_bytes = 0, p_pin_us = 0, p_register_us = 0, p_register_calls = 0, p_register_max_us = 0;   // under pmu
     std::vector<SeqState> st;
     // staging for layout conversion on the way to host memory
     char* staging = nullptr;
@@ -208,7 +211,67 @@ size_t p_segment_bytes(const ipkv* h, int k) {
     return size_t(int64_t(h->cfg.n_layers) * h->cfg.max_seqs * h->pseg[size_t(k)].nb * h->bb);
 }
 
-// The pinning thread: page-locks the requested segments in order (cudaHostAlloc, as the paper does).
+// Allocates and page-locks segment k.  One cudaHostAlloc of the whole segment (the paper's call) holds the driver's
+// lock for its full duration — measured here: 70-410 ms during which the decode thread's launches stall — so the
+// memory is allocated and faulted in with plain host calls first, and then registered with the driver one layer's
+// range at a time (a few MB, under a millisecond each; every copy the library issues lies inside one such range),
+// paced by the decode steps themselves when the decode thread is running beside it: at most one range per step, the
+// whole segment within half an eviction window.
+bool pin_segment(ipkv* h, int k, bool beside_decode, char** base_out) {
+    const size_t bytes = p_segment_bytes(h, k);
+    const size_t layer_bytes = bytes / size_t(h->cfg.n_layers);
+    void* p = nullptr;
+    if (posix_memalign(&p, size_t(2) << 20, bytes) != 0) return false;
+    // 2 MB pages where the kernel grants them: measured on the B200 host, faulting in drops from 0.36 to 0.12 ms/MB
+    // and page-locking a 4 MB range from 1.4 ms to 0.3 ms (a refusal changes nothing but the speed)
+    madvise(p, bytes, MADV_HUGEPAGE);
+    std::memset(p, 0, bytes);                                       // fault every page in before the driver sees it
+    const bool by_layer = layer_bytes % 4096 == 0;
+    const size_t piece = by_layer ? layer_bytes : bytes;
+    const uint64_t n_pieces = bytes / piece;
+    const uint64_t steps_per_piece = std::max<uint64_t>(1, uint64_t(h->cfg.window_tokens) / 2 / n_pieces);
+    size_t done = 0;
+    uint64_t reg_us = 0, reg_max = 0;
+    for (; done < bytes; done += piece) {
+        const auto r0 = std::chrono::steady_clock::now();
+        if (cudaHostRegister(static_cast<char*>(p) + done, piece, cudaHostRegisterDefault) != cudaSuccess) break;
+        const uint64_t us = uint64_t(std::chrono::duration_cast<std::chrono::microseconds>(std::chrono::steady_clock::now() - r0).count());
+        reg_us += us; reg_max = std::max(reg_max, us);
+        if (beside_decode && done + piece < bytes) {
+            // next range after `steps_per_piece` more decode steps; at once if a call is waiting for this segment,
+            // and after 2 ms anyway (nobody is decoding)
+            std::unique_lock<std::mutex> lk(h->pmu);
+            const uint64_t target = h->p_tick + steps_per_piece;
+            h->pcv.wait_for(lk, std::chrono::milliseconds(2), [&] { return h->p_quit || h->p_waiters > 0 || h->p_tick >= target; });
+            if (h->p_quit) { done += piece; break; }
+        }
+    }
+    {
+        std::lock_guard<std::mutex> lk(h->pmu);
+        h->p_register_us += reg_us; h->p_register_calls += done / piece; h->p_register_max_us = std::max(h->p_register_max_us, reg_max);
+    }
+    if (done < bytes) {
+        cudaGetLastError();
+        for (size_t u = 0; u < done; u += piece) cudaHostUnregister(static_cast<char*>(p) + u);
+        std::free(p);
+        return false;
+    }
+    *base_out = static_cast<char*>(p);
+    return true;
+}
+
+void unpin_segment(ipkv* h, int k) {
+    char* p = h->pseg[size_t(k)].base;
+    if (!p) return;
+    const size_t bytes = p_segment_bytes(h, k);
+    const size_t layer_bytes = bytes / size_t(h->cfg.n_layers);
+    const size_t piece = (layer_bytes % 4096 == 0) ? layer_bytes : bytes;
+    for (size_t u = 0; u < bytes; u += piece) cudaHostUnregister(p + u);
+    std::free(p);
+    h->pseg[size_t(k)].base = nullptr;
+}
+
+// The pinning thread: page-locks the requested segments in order.
 void pin_worker(ipkv* h) {
     cudaSetDevice(h->cfg.device);
     std::unique_lock<std::mutex> lk(h->pmu);
@@ -219,15 +282,14 @@ void pin_worker(ipkv* h) {
         const size_t bytes = p_segment_bytes(h, k);
         lk.unlock();
         const auto t0 = std::chrono::steady_clock::now();
-        void* p = nullptr;
-        const cudaError_t e = cudaHostAlloc(&p, bytes, cudaHostAllocDefault);
+        char* p = nullptr;
+        const bool ok = pin_segment(h, k, true, &p);
         const auto t1 = std::chrono::steady_clock::now();
         lk.lock();
-        if (e != cudaSuccess) {
-            cudaGetLastError();                    // the error state is this thread's own
+        if (!ok) {
             h->p_failed = true;
         } else {
-            h->pseg[size_t(k)].base = static_cast<char*>(p);
+            h->pseg[size_t(k)].base = p;
             h->p_ready = k + 1;
             h->p_pinned_bytes += bytes;
             h->p_pin_us += uint64_t(std::chrono::duration_cast<std::chrono::microseconds>(t1 - t0).count());
@@ -250,7 +312,10 @@ ipkv_status p_ensure(ipkv* h, int k) {
     if (k < h->p_ready) return IPKV_OK;
     if (k + 1 > h->p_requested) { h->p_requested = k + 1; h->pcv.notify_all(); }
     const auto t0 = std::chrono::steady_clock::now();
+    h->p_waiters += 1;
+    h->pcv.notify_all();
     h->pcv.wait(lk, [&] { return h->p_failed || k < h->p_ready; });
+    h->p_waiters -= 1;
     h->stats.p_grow_waits += 1;
     h->stats.p_grow_wait_us += uint64_t(std::chrono::duration_cast<std::chrono::microseconds>(std::chrono::steady_clock::now() - t0).count());
     if (k >= h->p_ready) return fail(h, IPKV_ENOMEM, "could not pin the next segment of P");
@@ -667,7 +732,7 @@ ipkv_status ipkv_destroy(ipkv_t* h) {
         h->pcv.notify_all();
         h->p_thread.join();
     }
-    for (auto& sg : h->pseg) if (sg.base) cudaFreeHost(sg.base);
+    for (size_t k = 0; k < h->pseg.size(); ++k) unpin_segment(h, int(k));
     if (h->own[0] && h->u_host) std::free(h->u_host);
     if (h->own[1] && h->p_host) cudaFreeHost(h->p_host);
     if (h->own[2] && h->w_dev) cudaFree(h->w_dev);
@@ -731,10 +796,10 @@ ipkv_status ipkv_create(const ipkv_config* cfg, ipkv_t** out) {
         for (int64_t b = nb0; b < h->p_cap; b += h->w_blocks)
             h->pseg.push_back(ipkv::PSegment{nullptr, b, h->w_blocks});   // the last one may reach past p_cap: capacity checks use p_cap
         if (nb0 > 0) {                            // the prefill share: pinned here, "during model loading and warm-up"
-            void* p0 = nullptr;
+            char* p0 = nullptr;
             const auto t0 = std::chrono::steady_clock::now();
-            if (cudaHostAlloc(&p0, h->sizes[1], cudaHostAllocDefault) != cudaSuccess) { cudaGetLastError(); return bail(IPKV_ENOMEM); }
-            h->pseg[0].base = static_cast<char*>(p0);
+            if (!pin_segment(h, 0, false, &p0)) return bail(IPKV_ENOMEM);
+            h->pseg[0].base = p0;
             h->p_pinned_bytes = h->sizes[1];
             h->p_pin_us = uint64_t(std::chrono::duration_cast<std::chrono::microseconds>(std::chrono::steady_clock::now() - t0).count());
         }
@@ -907,6 +972,11 @@ ipkv_status ipkv_append(ipkv_t* h, int32_t layer, const int32_t* seq_ids, int32_
     }
     DeviceGuard dev_guard(c.device);
     CU(h, dev_guard.error());
+    if (h->grow_p && layer == 0) {                  // one decode step further: the pinning thread paces itself by these
+        std::lock_guard<std::mutex> lk(h->pmu);
+        h->p_tick += 1;
+        h->pcv.notify_all();
+    }
     // evict full windows first, so that the newest token is always GPU-side
     {
         std::vector<int> full;
@@ -1396,6 +1466,9 @@ ipkv_status ipkv_get_stats(ipkv_t* h, ipkv_stats* out) {
         h->stats.p_segments = uint64_t(h->p_ready) - (h->pseg[0].nb == 0 ? 1 : 0);
         h->stats.p_pinned_bytes = h->p_pinned_bytes;
         h->stats.p_pin_us = h->p_pin_us;
+        h->stats.p_register_us = h->p_register_us;
+        h->stats.p_register_calls = h->p_register_calls;
+        h->stats.p_register_max_us = h->p_register_max_us;
     }
     *out = h->stats;
     return h->stats.device_status ? fail(h, IPKV_ETIMEOUT, "a kernel's bounded wait gave up; results of that call are invalid") : IPKV_OK;
