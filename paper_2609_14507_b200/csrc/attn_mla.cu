@@ -38,7 +38,7 @@ constexpr int kThreads = (kConsumerWarps + 1) * 32;
 constexpr int kStages = 2;
 constexpr int kStageBytes = kTileTokens * kDqk * 2;          // 73 728
 constexpr int kQPitch = kDqk * 2 + 16;                       // 1168
-constexpr int kSPitch = kTileTokens + 4;                     // floats
+constexpr int kSPitch = kTileTokens + 8;                     // floats; rows 8 banks apart: the phase-1 float2 stores of 8 rows x 8 words spread over all 32 banks
 constexpr int kPPitch = kTileTokens * 2 + 16;                // bytes (bf16 row of 64 tokens, padded)
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
