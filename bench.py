@@ -344,6 +344,8 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--kv-splits", type=int, default=0)
+    ap.add_argument("--static-schedule", action="store_true",
+                    help="fixed tile assignment in the grouped-query kernel (bit-reproducible) instead of dynamic balancing")
     ap.add_argument("--separate-merge", action="store_true",
                     help="join the CPU-side partial with a separate ipkv_merge launch instead of inside the split reduce")
     ap.add_argument("--latency", action="store_true", help="also time every step separately and report P50 / P99 / max")
@@ -403,10 +405,10 @@ def main():
         for layer in range(NL):
             cache.append(layer, seq_ids, k_new[layer], None if v_new is None else v_new[layer], stream=cur)
             if fused:      # the CPU-side partial is joined inside the split reduce: out = merged (O, LSE)
-                cache.attend_gpu(layer, seq_ids, q[layer], out[layer], out_lse, kv_splits=args.kv_splits, stream=cur,
+                cache.attend_gpu(layer, seq_ids, q[layer], out[layer], out_lse, kv_splits=args.kv_splits, static_schedule=args.static_schedule, stream=cur,
                                  fold_o=o_cpu[layer], fold_lse=lse_cpu[layer])
             else:
-                cache.attend_gpu(layer, seq_ids, q[layer], o_part, lse_part, kv_splits=args.kv_splits, stream=cur)
+                cache.attend_gpu(layer, seq_ids, q[layer], o_part, lse_part, kv_splits=args.kv_splits, static_schedule=args.static_schedule, stream=cur)
                 cache.merge(B * Hq, dv, [o_part.view(B * Hq, dv), o_cpu[layer]], [lse_part.view(-1), lse_cpu[layer]],
                             out[layer], out_lse, out_is_bf16=True, stream=cur)
 
@@ -491,10 +493,10 @@ def main():
             for layer in range(NL):
                 cache.append(layer, seq_ids, dk[layer], None if dvn is None else dvn[layer], stream=cur)
                 if fused:
-                    cache.attend_gpu(layer, seq_ids, dq[layer], out[layer], out_lse, kv_splits=args.kv_splits, stream=cur,
+                    cache.attend_gpu(layer, seq_ids, dq[layer], out[layer], out_lse, kv_splits=args.kv_splits, static_schedule=args.static_schedule, stream=cur,
                                      fold_o=doc[layer], fold_lse=dlc[layer])
                 else:
-                    cache.attend_gpu(layer, seq_ids, dq[layer], o_part, lse_part, kv_splits=args.kv_splits, stream=cur)
+                    cache.attend_gpu(layer, seq_ids, dq[layer], o_part, lse_part, kv_splits=args.kv_splits, static_schedule=args.static_schedule, stream=cur)
                     cache.merge(B * Hq, dv, [o_part.view(B * Hq, dv), doc[layer]], [lse_part.view(-1), dlc[layer]],
                                 out[layer], out_lse, out_is_bf16=True, stream=cur)
             hout.copy_(out, non_blocking=True)
@@ -543,7 +545,7 @@ def main():
                        "cpu_share": f"{num0}/{den0}", "gpu_share_tokens_per_seq_mean": n_gpu0 + 1, "bytes_per_kv_token": bpt, "block_tokens": BLOCK, "window_tokens": wl.get("window", WINDOW),
                        "gpu_share": "HBM-resident", "host_copies_of_U_and_P": "off (benchmark)", "cpu_partial": "synthetic values",
                        "l2": l2_note,
-                       "multi_gpu": "replicas only", "kv_splits": args.kv_splits,
+                       "multi_gpu": "replicas only", "kv_splits": args.kv_splits, "schedule": "static" if args.static_schedule else "dynamic balancing (GQA kernel)",
                        "merge": "inside the split reduce" if fused else "separate ipkv_merge launch"},
             "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu,
             "step_gbs": bytes_all / (ms * 1e-3) / 1e9,

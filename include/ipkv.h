@@ -152,9 +152,16 @@ ipkv_status ipkv_append(ipkv_t* h, int32_t layer, const int32_t* seq_ids, int32_
  * (Sec. 5.3).  layer = -1 / seq = -1 mean all.  A placed batch never moves again.  No-op on an empty window. */
 ipkv_status ipkv_flush(ipkv_t* h, int32_t layer, int32_t seq, void* stream);
 
+/* By default the grouped-query kernel balances its load while it runs: a CTA that finishes its share of the
+ * tiles early (some SMs get more memory bandwidth than others) takes over tiles of the CTAs that are behind.
+ * Which tiles end up in which partial then differs from launch to launch, so the fp32 results can differ in the
+ * last bits between two identical calls.  This flag keeps the fixed assignment: bit-reproducible, a few
+ * percent slower.  (The stateless entry points below always use the fixed assignment.) */
+#define IPKV_ATTEND_STATIC_SCHEDULE 1
+
 typedef struct {
   int32_t kv_splits;   /* 0 = automatic; otherwise the number of sequence chunks per (sequence, KV head) */
-  int32_t reserved;
+  int32_t flags;       /* IPKV_ATTEND_* bits                                                          */
   void* side_stream;   /* stream for host-to-device chunk copies; NULL = the handle's own             */
   /* Optional extra partial over a disjoint token set (typically the CPU-side partial, already on the
      device): [n_seq][n_q_heads][dim_v] and [n_seq][n_q_heads] fp32.  When both are given it is folded in by

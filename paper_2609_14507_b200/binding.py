@@ -16,6 +16,7 @@ GQA, MLA = 0, 1
 REGION_U, REGION_P, REGION_W = 0, 1, 2
 LAYOUT_PLAIN, LAYOUT_TILE = 0, 1
 FLAG_NO_HOST_U, FLAG_NO_HOST_P, FLAG_GROW_P = 1, 2, 4
+ATTEND_STATIC_SCHEDULE = 1
 OK = 0
 STATUS_NAMES = {0: "OK", 1: "EINVAL", 2: "ENOMEM", 3: "ERANGE", 4: "ESTATE", 5: "ECUDA", 6: "ETIMEOUT", 7: "EINTERNAL"}
 
@@ -45,7 +46,7 @@ class Config(C.Structure):
 
 
 class AttendOpts(C.Structure):
-    _fields_ = [("kv_splits", C.c_int32), ("reserved", C.c_int32), ("side_stream", C.c_void_p),
+    _fields_ = [("kv_splits", C.c_int32), ("flags", C.c_int32), ("side_stream", C.c_void_p),
                 ("fold_o_dev", C.c_void_p), ("fold_lse_dev", C.c_void_p)]
 
 
@@ -253,14 +254,14 @@ class Cache:
         self._check(lib().ipkv_flush(self._h, layer, seq, _stream(stream)), "ipkv_flush")
 
     def attend_gpu(self, layer, seq_ids, q, o_part, lse_part, kv_splits=0, side_stream=None, stream=None,
-                   fold_o=None, fold_lse=None):
+                   fold_o=None, fold_lse=None, static_schedule=False):
         ids, n = _ids(seq_ids)
-        opts = AttendOpts(kv_splits, 0, _stream(side_stream) if side_stream is not None else None, _ptr(fold_o), _ptr(fold_lse))
+        opts = AttendOpts(kv_splits, ATTEND_STATIC_SCHEDULE if static_schedule else 0, _stream(side_stream) if side_stream is not None else None, _ptr(fold_o), _ptr(fold_lse))
         self._check(lib().ipkv_attend_gpu(self._h, layer, ids, n, _ptr(q), C.byref(opts), _ptr(o_part), _ptr(lse_part),
                                           _stream(stream)), "ipkv_attend_gpu")
 
     def attend_gpu_sparse(self, layer, seq_ids, q, blocks_per_row, o_part, lse_part, include_window=True, kv_splits=0,
-                          stream=None, fold_o=None, fold_lse=None):
+                          stream=None, fold_o=None, fold_lse=None, static_schedule=False):
         """Attention over the D-window plus the listed whole P blocks of every row (block ordinals in region P)."""
         ids, n = _ids(seq_ids)
         flat, start = [], [0]
@@ -269,7 +270,7 @@ class Cache:
             start.append(len(flat))
         blocks = (C.c_int64 * max(1, len(flat)))(*flat)
         starts = (C.c_int32 * len(start))(*start)
-        opts = AttendOpts(kv_splits, 0, None, _ptr(fold_o), _ptr(fold_lse))
+        opts = AttendOpts(kv_splits, ATTEND_STATIC_SCHEDULE if static_schedule else 0, None, _ptr(fold_o), _ptr(fold_lse))
         self._check(lib().ipkv_attend_gpu_sparse(self._h, layer, ids, n, _ptr(q), blocks, starts, 1 if include_window else 0,
                                                  C.byref(opts), _ptr(o_part), _ptr(lse_part), _stream(stream)), "ipkv_attend_gpu_sparse")
 

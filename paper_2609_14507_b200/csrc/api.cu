@@ -134,6 +134,12 @@ struct ipkv {
     char* merge_stage = nullptr;
     size_t merge_stage_bytes = 0;
     uint32_t* status_dev = nullptr;
+    // scheduling words of the dynamically balanced attention kernel: two sets used by alternate launches; the
+    // split reduce of one launch zeroes the set of the next
+    int32_t* steal_dev = nullptr;
+    static constexpr int kStealWords = 1 << 16;     // per set
+    int steal_dirty[2] = {0, 0};                     // words a launch has written in each set
+    unsigned steal_epoch = 0;
     // write-back of evicted windows on the idle D2H direction: a device snapshot of every window (same shape as W),
     // a copy stream, one "snapshot in use" event per layer, and a pinned bounce buffer for the unpinned region
     char* wb_stage = nullptr;
@@ -635,7 +641,7 @@ ipkv_status ensure_scratch(ipkv* h, size_t bytes) {
 }
 
 void fill_launch(AttnLaunch* a, int kind, int Hq, int Hkv, int dqk, int dv, int bt, float scale, const Plan& plan,
-                 const char* table_dev, char* partials, const void* q, int n_rows) {
+                 const char* table_dev, char* partials, const void* q, int n_rows, size_t extra_partials = 0) {
     a->kind = kind; a->n_q_heads = Hq; a->n_kv_heads = Hkv; a->dim_qk = dqk; a->dim_v = dv; a->bt = bt; a->scale = scale;
     a->q = q;
     const PartGeom pg = part_geom(kind, Hq, Hkv);
@@ -647,11 +653,13 @@ void fill_launch(AttnLaunch* a, int kind, int Hq, int Hkv, int dqk, int dv, int 
     a->cta_span_start = reinterpret_cast<const int32_t*>(table_dev + o);
     o += align_up(plan.cta_span_start.size() * sizeof(int32_t), 16);
     a->rg_span_start = reinterpret_cast<const int32_t*>(table_dev + o);
+    o += align_up(plan.rg_span_start.size() * sizeof(int32_t), 16);
+    a->cta_tiles = reinterpret_cast<const int32_t*>(table_dev + o);
     a->n_spans = int(plan.spans.size());
     a->n_ctas = plan.n_ctas();
     a->n_rows = n_rows;
     a->n_gh = pg.n_gh;
-    const size_t rows = plan.spans.size() * size_t(pg.parts_per_span) * pg.rows_per_group;
+    const size_t rows = (plan.spans.size() + extra_partials) * size_t(pg.parts_per_span) * pg.rows_per_group;
     a->part_o = reinterpret_cast<float*>(partials);
     a->part_lse = reinterpret_cast<float*>(partials + align_up(rows * dv * sizeof(float), 256));
 }
@@ -659,19 +667,35 @@ void fill_launch(AttnLaunch* a, int kind, int Hq, int Hkv, int dqk, int dv, int 
 // One group of segments for all rows: attention + split reduce, folding into (out_o, out_lse) when `fold`.
 ipkv_status run_group(ipkv* h, const std::vector<std::vector<PlanSeg>>& rows, const char* const bases[kMaxBases],
                       const void* q, int kv_splits, const float* fold_o, const float* fold_lse, float* out_o, float* out_lse,
-                      cudaStream_t s) {
+                      cudaStream_t s, bool static_schedule = false) {
     const ipkv_config& c = h->cfg;
     Plan plan;
     const PartGeom pg = part_geom(c.kind, c.n_q_heads, c.n_kv_heads);
     build_plan(rows, pg.n_gh, kv_splits, pg.ctas_per_sm, &plan);
-    ipkv_status rc = ensure_scratch(h, partial_bytes(plan.spans.size(), pg, c.dim_v));
+    // dynamic balancing: every CTA may fill up to kStealSlots extra partials (GQA kernel; more than one CTA)
+    const size_t n_tags = size_t(plan.n_ctas()) * kStealSlots;
+    const bool balance = !static_schedule && c.kind == IPKV_GQA && plan.n_ctas() > 1 &&
+                         n_tags + plan.spans.size() + 2 * size_t(plan.n_ctas()) <= size_t(ipkv::kStealWords);
+    const size_t extra = balance ? n_tags : 0;
+    ipkv_status rc = ensure_scratch(h, partial_bytes(plan.spans.size() + extra, pg, c.dim_v));
     if (rc != IPKV_OK) return rc;
     const char* table = nullptr;
     rc = upload_table(h, plan, s, &table);
     if (rc != IPKV_OK) return rc;
     AttnLaunch a{};
     fill_launch(&a, c.kind, c.n_q_heads, c.n_kv_heads, c.dim_qk, c.dim_v, c.block_tokens, h->scale, plan, table, h->scratch, q,
-                int(rows.size()));
+                int(rows.size()), extra);
+    if (balance) {
+        const int set = int(h->steal_epoch & 1u), other = set ^ 1;
+        int32_t* words = h->steal_dev + size_t(set) * ipkv::kStealWords;
+        a.steal_tags = words;
+        a.steal_next = words + n_tags;
+        h->steal_dirty[set] = int(n_tags + plan.spans.size() + 2 * size_t(plan.n_ctas()));
+        a.steal_clear = h->steal_dev + size_t(other) * ipkv::kStealWords;     // used by the balanced launch after this one
+        a.steal_clear_words = h->steal_dirty[other];
+        h->steal_dirty[other] = 0;
+        h->steal_epoch += 1;
+    }
     for (int i = 0; i < kMaxBases; ++i) a.bases[i] = bases[i];
     a.acc_o = fold_o;
     a.acc_lse = fold_lse;
@@ -744,6 +768,7 @@ ipkv_status ipkv_destroy(ipkv_t* h) {
     if (h->table_dev) cudaFree(h->table_dev);
     if (h->merge_stage) cudaFree(h->merge_stage);
     if (h->status_dev) cudaFree(h->status_dev);
+    if (h->steal_dev) cudaFree(h->steal_dev);
     for (int i = 0; i < 2; ++i) {
         if (h->gather[i]) cudaFreeHost(h->gather[i]);
         if (h->gather_done[i]) cudaEventDestroy(h->gather_done[i]);
@@ -827,6 +852,8 @@ ipkv_status ipkv_create(const ipkv_config* cfg, ipkv_t** out) {
 
     if (cudaMalloc(&h->status_dev, 256) != cudaSuccess) return bail(IPKV_ENOMEM);
     if (cudaMemset(h->status_dev, 0, 256) != cudaSuccess) return bail(IPKV_ECUDA);
+    if (cudaMalloc(&h->steal_dev, 2 * size_t(ipkv::kStealWords) * sizeof(int32_t)) != cudaSuccess) return bail(IPKV_ENOMEM);
+    if (cudaMemset(h->steal_dev, 0, 2 * size_t(ipkv::kStealWords) * sizeof(int32_t)) != cudaSuccess) return bail(IPKV_ECUDA);
     h->table_cap = 1 << 20;
     if (cudaMallocHost(&h->table_pinned, h->table_cap) != cudaSuccess) return bail(IPKV_ENOMEM);
     if (cudaMalloc(&h->table_dev, h->table_cap) != cudaSuccess) return bail(IPKV_ENOMEM);
@@ -1017,6 +1044,7 @@ ipkv_status ipkv_attend_gpu(ipkv_t* h, int32_t layer, const int32_t* seq_ids, in
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int kv_splits = opts ? opts->kv_splits : 0;
     if (kv_splits < 0) return fail(h, IPKV_EINVAL, "kv_splits must be >= 0");
+    const bool static_schedule = opts && (opts->flags & IPKV_ATTEND_STATIC_SCHEDULE);
     cudaStream_t side = (opts && opts->side_stream) ? static_cast<cudaStream_t>(opts->side_stream) : h->side;
     DeviceGuard dev_guard(c.device);
     CU(h, dev_guard.error());
@@ -1051,7 +1079,7 @@ ipkv_status ipkv_attend_gpu(ipkv_t* h, int32_t layer, const int32_t* seq_ids, in
     const float* fold_o = opts ? opts->fold_o_dev : nullptr;
     const float* fold_lse = opts ? opts->fold_lse_dev : nullptr;
     if ((fold_o == nullptr) != (fold_lse == nullptr)) return fail(h, IPKV_EINVAL, "fold_o_dev and fold_lse_dev must be given together");
-    ipkv_status rc = run_group(h, rows, bases, q_dev, kv_splits, fold_o, fold_lse, o_part_dev, lse_part_dev, s);
+    ipkv_status rc = run_group(h, rows, bases, q_dev, kv_splits, fold_o, fold_lse, o_part_dev, lse_part_dev, s, static_schedule);
     if (rc != IPKV_OK) return rc;
     if (max_stream_chunks == 0) return IPKV_OK;
 
@@ -1126,7 +1154,7 @@ ipkv_status ipkv_attend_gpu(ipkv_t* h, int32_t layer, const int32_t* seq_ids, in
         }
         CU(h, cudaEventRecord(h->slot_ready[slot], side));
         CU(h, cudaStreamWaitEvent(s, h->slot_ready[slot], 0));
-        rc = run_group(h, rows, bases, q_dev, kv_splits, o_part_dev, lse_part_dev, o_part_dev, lse_part_dev, s);
+        rc = run_group(h, rows, bases, q_dev, kv_splits, o_part_dev, lse_part_dev, o_part_dev, lse_part_dev, s, static_schedule);
         if (rc != IPKV_OK) return rc;
         CU(h, cudaEventRecord(h->slot_free[slot], s));
         h->slot_free_set[slot] = 1;
@@ -1146,6 +1174,7 @@ ipkv_status ipkv_attend_gpu_sparse(ipkv_t* h, int32_t layer, const int32_t* seq_
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int kv_splits = opts ? opts->kv_splits : 0;
     if (kv_splits < 0) return fail(h, IPKV_EINVAL, "kv_splits must be >= 0");
+    const bool static_schedule = opts && (opts->flags & IPKV_ATTEND_STATIC_SCHEDULE);
     cudaStream_t side = (opts && opts->side_stream) ? static_cast<cudaStream_t>(opts->side_stream) : h->side;
     const float* fold_o = opts ? opts->fold_o_dev : nullptr;
     const float* fold_lse = opts ? opts->fold_lse_dev : nullptr;
@@ -1192,7 +1221,7 @@ ipkv_status ipkv_attend_gpu_sparse(ipkv_t* h, int32_t layer, const int32_t* seq_
         if (include_window && st.router.window_fill() > 0) rows[i].push_back(PlanSeg{1, h->w_off(seq), st.router.window_fill()});
     }
     const char* bases[kMaxBases] = {h->ring ? h->ring_layer(layer) : nullptr, h->w_layer(layer), h->pp_dev, nullptr};
-    ipkv_status rc = run_group(h, rows, bases, q_dev, kv_splits, fold_o, fold_lse, o_part_dev, lse_part_dev, s);
+    ipkv_status rc = run_group(h, rows, bases, q_dev, kv_splits, fold_o, fold_lse, o_part_dev, lse_part_dev, s, static_schedule);
     if (rc != IPKV_OK) return rc;
     if (host_picks.empty()) return IPKV_OK;
     if (c.flags & IPKV_FLAG_NO_HOST_P) return fail(h, IPKV_EINTERNAL, "host-only P blocks without a host copy");
@@ -1235,7 +1264,7 @@ ipkv_status ipkv_attend_gpu_sparse(ipkv_t* h, int32_t layer, const int32_t* seq_
         h->gather_busy[gb] = true;
         CU(h, cudaEventRecord(h->slot_ready[slot], side));
         CU(h, cudaStreamWaitEvent(s, h->slot_ready[slot], 0));
-        rc = run_group(h, rows, bases, q_dev, kv_splits, o_part_dev, lse_part_dev, o_part_dev, lse_part_dev, s);
+        rc = run_group(h, rows, bases, q_dev, kv_splits, o_part_dev, lse_part_dev, o_part_dev, lse_part_dev, s, static_schedule);
         if (rc != IPKV_OK) return rc;
         CU(h, cudaEventRecord(h->slot_free[slot], s));
         h->slot_free_set[slot] = 1;
@@ -1579,7 +1608,8 @@ ipkv_status ipkv_attend_scratch_bytes(const ipkv_attn_shape* sh, int32_t n_rows,
     const int64_t spans = max_spans_bound(n_rows, n_runs, pg.n_gh, kv_splits, pg.ctas_per_sm);
     const size_t table = align_up(size_t(n_runs) * sizeof(Seg), 16) + align_up(size_t(spans) * sizeof(Span), 16) +
                          align_up(size_t(kSmCount * pg.ctas_per_sm + 1) * sizeof(int32_t), 16) +
-                         align_up((size_t(n_rows) * pg.n_gh + 1) * sizeof(int32_t), 16);
+                         align_up((size_t(n_rows) * pg.n_gh + 1) * sizeof(int32_t), 16) +
+                         align_up(size_t(kSmCount * pg.ctas_per_sm) * sizeof(int32_t), 16);
     *out_bytes = align_up(table, 256) + 256 + partial_bytes(size_t(spans), pg, sh->dim_v);
     return IPKV_OK;
 }

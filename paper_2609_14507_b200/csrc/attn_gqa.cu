@@ -40,6 +40,11 @@ struct GqaParams {
     float* part_o;
     float* part_lse;
     uint32_t* status;
+    int32_t* next;       // dynamic schedule: tiles claimed so far of every span [n_spans], of every CTA's chunk [n_ctas], and the
+                         // number of CTAs that came to help with every chunk [n_ctas] (all zero at launch); null = static schedule
+    const int32_t* cta_tiles;   // tiles in every CTA's chunk
+    int32_t* tags;       // [n_ctas * kStealSlots]: span + 1 of every extra partial a CTA filled (zero at launch); null = no stealing
+    int n_spans, n_ctas;
     int Hq, G, n_hg, RG;
     int bt;
     int64_t head_bytes, block_bytes;
@@ -52,8 +57,19 @@ struct SmemPlan {
     static constexpr int kStage = 2 * kPlane;
     static constexpr int kStagesBytes = STAGES * kStage;
     static constexpr int kBarOff = kStagesBytes;
-    static constexpr int kTotal = kBarOff + 2 * STAGES * 8;
+    static constexpr int kMetaOff = kBarOff + 2 * STAGES * 8;     // one StageMeta (16 bytes) per stage
+    static constexpr int kTotal = kMetaOff + STAGES * 16;
 };
+
+// What the producer tells the consumers about the tile in a stage.
+struct StageMeta {
+    int32_t slot;        // index of the partial this tile is accumulated into; kEndSlot = no more tiles
+    int32_t n_valid;     // live tokens of the tile (64 except at the end of a run)
+    int32_t q_row;       // row * Hq + first query head of the tile's head group
+    int32_t n_heads;     // query heads in the group (at most 16)
+};
+constexpr int32_t kEndSlot = -1;
+constexpr int kMinSteal = 3;        // a span is worth stealing from while at least this many tiles are unclaimed
 
 template <int D, int STAGES, bool DUP>
 __global__ void __launch_bounds__(kThreads) attn_gqa_kernel(const GqaParams p) {
@@ -64,9 +80,11 @@ __global__ void __launch_bounds__(kThreads) attn_gqa_kernel(const GqaParams p) {
     const uint32_t s_base = ptx::smem_addr(smem);
     const uint32_t s_full = s_base + SP::kBarOff;
     const uint32_t s_empty = s_full + STAGES * 8;
+    volatile StageMeta* s_meta = reinterpret_cast<volatile StageMeta*>(smem + SP::kMetaOff);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int span_begin = p.cta_span_start[blockIdx.x], span_end = p.cta_span_start[blockIdx.x + 1];
+    const bool dynamic = p.next != nullptr;
 
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -87,60 +105,163 @@ __global__ void __launch_bounds__(kThreads) attn_gqa_kernel(const GqaParams p) {
     int it = 0;                      // tiles streamed so far by this CTA: stage = it % STAGES
 
     if (warp == kConsumerWarps) {
-        // ---------------- producer ----------------
-        if (lane == 0) {
+        // ---------------- producer: lane 0 claims tiles and issues copies; the whole warp looks for work to take over ----------------
+        {
             const uint64_t pol = ptx::l2_evict_first_policy();     // the KV stream is read once: first out of L2
-            for (int sp = span_begin; sp < span_end && ok; ++sp) {
-                const Span span = p.spans[sp];
-                const Seg seg = p.segs[span.seg];
-                const int g = span.gh / p.n_hg;
-                const char* seg_base = p.bases[seg.base_id] + seg.off + int64_t(g) * p.head_bytes;
-                for (int i = 0; i < span.ntiles; ++i, ++it) {
-                    const int st = it % STAGES;
-                    if (it >= STAGES && !ptx::mbar_wait(s_empty + 8 * st, ((it / STAGES) - 1) & 1)) { ok = false; break; }
-                    const int64_t t0 = int64_t(span.tile0 + i) * kTileTokens;
-                    const uint32_t dst = s_base + st * SP::kStage;
-                    const uint32_t bar = s_full + 8 * st;
-                    if (p.bt >= kTileTokens) {
-                        const int64_t blk = t0 / p.bt;
-                        const int r0 = int(t0 - blk * p.bt);
-                        const char* src = seg_base + blk * p.block_bytes;
-                        ptx::mbar_expect_tx(bar, SP::kStage);
-                        if (p.bt == kTileTokens) {
-                            ptx::bulk_g2s_hint(dst, src, SP::kStage, bar, pol);   // K plane and V plane are adjacent
-                        } else {
-                            const int64_t kplane = int64_t(p.bt) * D * 2;
-#pragma unroll
-                            for (int pn = 0; pn < D / 64; ++pn) {
-                                const char* s0 = src + int64_t(pn) * p.bt * 128 + int64_t(r0) * 128;
-                                ptx::bulk_g2s_hint(dst + pn * 8192, s0, 8192, bar, pol);
-                                ptx::bulk_g2s_hint(dst + SP::kPlane + pn * 8192, s0 + kplane, 8192, bar, pol);
-                            }
-                        }
+            // stream tile `tile` of a span into the next stage, to be accumulated into partial `slot`
+            auto issue = [&](const Span& span, const Seg& seg, const char* seg_base, int tile, int slot) -> bool {
+                const int st = it % STAGES;
+                if (it >= STAGES && !ptx::mbar_wait(s_empty + 8 * st, ((it / STAGES) - 1) & 1)) return false;
+                const int64_t t0 = int64_t(tile) * kTileTokens;
+                const int64_t left = int64_t(seg.n_tokens) - t0;
+                const int g = span.gh / p.n_hg, hg = span.gh - g * p.n_hg;
+                s_meta[st].slot = slot;
+                s_meta[st].n_valid = left < kTileTokens ? int(left) : kTileTokens;
+                s_meta[st].q_row = span.row * p.Hq + g * p.G + hg * 16;
+                s_meta[st].n_heads = min(16, p.G - hg * 16);
+                const uint32_t dst = s_base + st * SP::kStage;
+                const uint32_t bar = s_full + 8 * st;
+                if (p.bt >= kTileTokens) {
+                    const int64_t blk = t0 / p.bt;
+                    const int r0 = int(t0 - blk * p.bt);
+                    const char* src = seg_base + blk * p.block_bytes;
+                    ptx::mbar_expect_tx(bar, SP::kStage);
+                    if (p.bt == kTileTokens) {
+                        ptx::bulk_g2s_hint(dst, src, SP::kStage, bar, pol);   // K plane and V plane are adjacent
                     } else {
-                        const int nsub = kTileTokens / p.bt;
-                        const int64_t blk0 = t0 / p.bt;
-                        int live = 0;
-                        for (int j = 0; j < nsub; ++j) live += ((blk0 + j) * p.bt < seg.n_tokens);
-                        const uint32_t sub_bytes = uint32_t(p.bt) * 128;
-                        ptx::mbar_expect_tx(bar, uint32_t(live) * sub_bytes * 2 * (D / 64));
                         const int64_t kplane = int64_t(p.bt) * D * 2;
-                        for (int j = 0; j < live; ++j) {
-                            const char* src = seg_base + (blk0 + j) * p.block_bytes;
 #pragma unroll
-                            for (int pn = 0; pn < D / 64; ++pn) {
-                                ptx::bulk_g2s_hint(dst + pn * 8192 + j * sub_bytes, src + int64_t(pn) * sub_bytes, sub_bytes, bar, pol);
-                                ptx::bulk_g2s_hint(dst + SP::kPlane + pn * 8192 + j * sub_bytes, src + kplane + int64_t(pn) * sub_bytes, sub_bytes, bar, pol);
-                            }
+                        for (int pn = 0; pn < D / 64; ++pn) {
+                            const char* s0 = src + int64_t(pn) * p.bt * 128 + int64_t(r0) * 128;
+                            ptx::bulk_g2s_hint(dst + pn * 8192, s0, 8192, bar, pol);
+                            ptx::bulk_g2s_hint(dst + SP::kPlane + pn * 8192, s0 + kplane, 8192, bar, pol);
+                        }
+                    }
+                } else {
+                    const int nsub = kTileTokens / p.bt;
+                    const int64_t blk0 = t0 / p.bt;
+                    int live = 0;
+                    for (int j = 0; j < nsub; ++j) live += ((blk0 + j) * p.bt < seg.n_tokens);
+                    const uint32_t sub_bytes = uint32_t(p.bt) * 128;
+                    ptx::mbar_expect_tx(bar, uint32_t(live) * sub_bytes * 2 * (D / 64));
+                    const int64_t kplane = int64_t(p.bt) * D * 2;
+                    for (int j = 0; j < live; ++j) {
+                        const char* src = seg_base + (blk0 + j) * p.block_bytes;
+#pragma unroll
+                        for (int pn = 0; pn < D / 64; ++pn) {
+                            ptx::bulk_g2s_hint(dst + pn * 8192 + j * sub_bytes, src + int64_t(pn) * sub_bytes, sub_bytes, bar, pol);
+                            ptx::bulk_g2s_hint(dst + SP::kPlane + pn * 8192 + j * sub_bytes, src + kplane + int64_t(pn) * sub_bytes, sub_bytes, bar, pol);
                         }
                     }
                 }
+                ++it;
+                return true;
+            };
+            // All unclaimed tiles of one span. Tiles are claimed in batches that shrink as the span runs out (an eighth
+            // of what is left, 8 at most), so that little is locked in when other CTAs come to help, and the claim of
+            // the next batch is under way while the copies of the current one are issued. Returns the number of
+            // tiles streamed (-1 after a timeout).
+            auto drain = [&](int sp, int chunk, int slot, int32_t* tag) -> int {
+                const Span span = p.spans[sp];
+                const Seg seg = p.segs[span.seg];
+                const char* seg_base = p.bases[seg.base_id] + seg.off + int64_t(span.gh / p.n_hg) * p.head_bytes;
+                int n = 0;
+                if (!dynamic) {
+                    for (int t = 0; t < span.ntiles; ++t, ++n)
+                        if (!issue(span, seg, seg_base, span.tile0 + t, slot)) return -1;
+                    return n;
+                }
+                // the owner takes an eighth of what is left per claim, a helper a quarter
+                const int shift = tag ? 2 : 3;
+                auto batch = [shift](int left) { const int b = left >> shift; return b > 8 ? 8 : (b < 1 ? 1 : b); };
+                int b = batch(span.ntiles - *reinterpret_cast<volatile int32_t*>(p.next + sp));
+                int t0 = atomicAdd(p.next + sp, b);
+                while (t0 < span.ntiles) {
+                    const int first = t0, last = min(t0 + b, span.ntiles);
+                    const int left = span.ntiles - last;           // as far as this CTA knows
+                    b = batch(left);
+                    t0 = left > 0 ? atomicAdd(p.next + sp, b) : span.ntiles;
+                    if (n == 0 && tag) *tag = sp + 1;              // this CTA's extra partial `slot` belongs to span sp
+                    atomicAdd(p.next + p.n_spans + chunk, last - first);     // what is left of the chunk, for CTAs looking for work
+                    for (int t = first; t < last; ++t, ++n)
+                        if (!issue(span, seg, seg_base, span.tile0 + t, slot)) return -1;
+                }
+                return n;
+            };
+            // own chunk first: the partial of a span lives at the span's index
+            if (lane == 0)
+                for (int sp = span_begin; sp < span_end && ok; ++sp) ok = drain(sp, int(blockIdx.x), sp, nullptr) >= 0;
+            // then help the CTAs that are behind (some SMs get less of the memory bandwidth than others): pick the chunk with
+            // the most unclaimed tiles per CTA already working on it, take tiles from the span its owner will reach last,
+            // and accumulate them into one of this CTA's extra partials
+            if (dynamic && p.tags) {
+                int32_t* claimed = p.next + p.n_spans;
+                int32_t* helpers = claimed + p.n_ctas;
+                int used = 0;
+                for (int attempt = 0; used < kStealSlots && attempt < 3 * kStealSlots; ++attempt) {
+                    if (!__shfl_sync(0xffffffffu, int(ok), 0)) break;
+                    // the warp scans the chunks, kScan independent pairs of loads per lane and round
+                    constexpr int kScan = 10;
+                    int best = -1, best_score = 0;
+                    for (int base = 0; base < p.n_ctas; base += 32 * kScan) {
+                        int left[kScan], hl[kScan];
+#pragma unroll
+                        for (int k = 0; k < kScan; ++k) {
+                            const int c = base + k * 32 + lane;
+                            left[k] = c < p.n_ctas ? __ldg(p.cta_tiles + c) - __ldcg(claimed + c) : 0;
+                            hl[k] = c < p.n_ctas ? __ldcg(helpers + c) : 0;
+                        }
+#pragma unroll
+                        for (int k = 0; k < kScan; ++k) {
+                            const int score = left[k] >= kMinSteal ? (left[k] << 6) / (1 + hl[k]) : 0;
+                            if (score > best_score) { best_score = score; best = base + k * 32 + lane; }
+                        }
+                    }
+                    // every lane now holds the best chunk of its share. Helpers that arrive together must not all pick
+                    // the same one: take the candidate of a lane chosen by CTA and attempt, among the lanes whose
+                    // candidate scores at least three quarters of the best
+                    int top = best_score;
+#pragma unroll
+                    for (int d = 16; d > 0; d >>= 1) top = max(top, __shfl_xor_sync(0xffffffffu, top, d));
+                    if (top <= 0) break;
+                    const unsigned good = __ballot_sync(0xffffffffu, best_score > 0 && best_score >= top - (top >> 2));
+                    const int rot = (int(blockIdx.x) * 7 + attempt * 13) & 31;
+                    const unsigned turned = (good >> rot) | (rot ? good << (32 - rot) : 0u);
+                    const int pick = (__ffs(turned) - 1 + rot) & 31;
+                    const int victim = __shfl_sync(0xffffffffu, best, pick);
+                    int n = 0;
+                    if (lane == 0) {
+                        atomicAdd(helpers + victim, 1);
+                        // the last span of the victim's chunk that still has unclaimed tiles
+                        int sp = p.cta_span_start[victim + 1] - 1;
+                        const int sp_first = p.cta_span_start[victim];
+                        while (sp >= sp_first && __ldcg(p.next + sp) >= p.spans[sp].ntiles) --sp;
+                        if (sp >= sp_first) {
+                            n = drain(sp, victim, p.n_spans + int(blockIdx.x) * kStealSlots + used, p.tags + int(blockIdx.x) * kStealSlots + used);
+                            if (n < 0) ok = false;
+                        }
+                    }
+                    n = __shfl_sync(0xffffffffu, n, 0);
+                    if (n > 0) ++used;
+                }
             }
-            // do not leave the CTA while copies of ours may still be in flight
-            const int first_pending = it > STAGES ? it - STAGES : 0;
-            for (int i = first_pending; i < it; ++i)
-                if (!ptx::mbar_wait(s_full + 8 * (i % STAGES), (i / STAGES) & 1)) ok = false;
-            if (!ok) atomicOr(p.status, 1u);
+            if (lane == 0) {
+                // tell the consumers that nothing follows
+                if (ok) {
+                    const int st = it % STAGES;
+                    if (it >= STAGES && !ptx::mbar_wait(s_empty + 8 * st, ((it / STAGES) - 1) & 1)) ok = false;
+                    if (ok) {
+                        s_meta[st].slot = kEndSlot;
+                        ptx::mbar_expect_tx(s_full + 8 * st, 0);
+                        ++it;
+                    }
+                }
+                // do not leave the CTA while copies of ours may still be in flight
+                const int first_pending = it > STAGES ? it - STAGES : 0;
+                for (int i = first_pending; i < it; ++i)
+                    if (!ptx::mbar_wait(s_full + 8 * (i % STAGES), (i / STAGES) & 1)) ok = false;
+                if (!ok) atomicOr(p.status, 1u);
+            }
         }
         return;
     }
@@ -158,17 +279,61 @@ __global__ void __launch_bounds__(kThreads) attn_gqa_kernel(const GqaParams p) {
     const int tokV = warp * 16 + (mi & 1) * 8 + r8;      // V: matrices 0,2 tokens 0-7; 1,3 tokens 8-15
     const int tcol = warp * 16 + c0;                     // token of accumulator element 0 (n-tile 0)
 
-    for (int sp = span_begin; sp < span_end; ++sp) {
-        const Span span = p.spans[sp];
-        const Seg seg = p.segs[span.seg];
-        const int g = span.gh / p.n_hg, hg = span.gh - g * p.n_hg;
-        const int head0 = g * p.G + hg * 16;                  // first query head of this span's group
-        const int n_heads = min(16, p.G - hg * 16);
+    if (dynamic) {
+        // a span of this CTA's chunk may be taken over completely by other CTAs: its partial then stays empty
+        for (int sp = span_begin; sp < span_end; ++sp) {
+            const int64_t prow = (int64_t(sp) * kConsumerWarps + warp) * p.RG;
+            if ((lane & 3) == 0) {
+                if (r0 < p.RG) p.part_lse[prow + r0] = -INFINITY;
+                if (!DUP && r0 + 8 < p.RG) p.part_lse[prow + r0 + 8] = -INFINITY;
+            }
+        }
+    }
 
-        // query fragments straight from global memory (a few KB per span, L2-resident)
-        uint32_t qa[D / 16][4];
-        {
-            const __nv_bfloat16* qrow0 = p.q + (int64_t(span.row) * p.Hq + head0 + r0) * D + c0;
+    uint32_t qa[D / 16][4];
+    float o[D / 8][4];
+    float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+    int cur_slot = kEndSlot, n_heads = 0;
+
+    // this warp's normalised partial of the tiles accumulated so far (rows = the group's query heads)
+    auto flush = [&]() {
+        l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
+        l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+        if (!DUP) {
+            l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
+            l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+        }
+        const int64_t prow = (int64_t(cur_slot) * kConsumerWarps + warp) * p.RG;
+        if (r0 < n_heads) {
+            const float inv = l0 > 0.f ? 1.f / l0 : 0.f;
+            float* dst = p.part_o + (prow + r0) * D + c0;
+#pragma unroll
+            for (int nt = 0; nt < D / 8; ++nt) {
+                const float x = DUP ? o[nt][0] + o[nt][2] : o[nt][0], y = DUP ? o[nt][1] + o[nt][3] : o[nt][1];
+                *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(x * inv, y * inv);
+            }
+            if ((lane & 3) == 0) p.part_lse[prow + r0] = (m0 == -INFINITY) ? -INFINITY : (m0 + log2f(l0)) * kLn2;
+        }
+        if (!DUP && r0 + 8 < n_heads) {
+            const float inv = l1 > 0.f ? 1.f / l1 : 0.f;
+            float* dst = p.part_o + (prow + r0 + 8) * D + c0;
+#pragma unroll
+            for (int nt = 0; nt < D / 8; ++nt) *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(o[nt][2] * inv, o[nt][3] * inv);
+            if ((lane & 3) == 0) p.part_lse[prow + r0 + 8] = (m1 == -INFINITY) ? -INFINITY : (m1 + log2f(l1)) * kLn2;
+        }
+    };
+
+    for (;; ++it) {
+        const int st = it % STAGES;
+        if (!ptx::mbar_wait(s_full + 8 * st, (it / STAGES) & 1)) { ok = false; break; }   // after a timeout: give up
+        const int slot = s_meta[st].slot;
+        if (slot != cur_slot) {
+            if (cur_slot != kEndSlot) flush();
+            if (slot == kEndSlot) break;
+            cur_slot = slot;
+            n_heads = s_meta[st].n_heads;
+            // query fragments straight from global memory (a few KB per span, L2-resident)
+            const __nv_bfloat16* qrow0 = p.q + (int64_t(s_meta[st].q_row) + r0) * D + c0;
             const bool v0 = r0 < n_heads, v1 = !DUP && (r0 + 8 < n_heads);
 #pragma unroll
             for (int ks = 0; ks < D / 16; ++ks) {
@@ -181,18 +346,12 @@ __global__ void __launch_bounds__(kThreads) attn_gqa_kernel(const GqaParams p) {
                     qa[ks][3] = v1 ? __ldg(reinterpret_cast<const uint32_t*>(qrow0 + 8 * D + ks * 16 + 8)) : 0u;
                 }
             }
-        }
-        float o[D / 8][4];
 #pragma unroll
-        for (int nt = 0; nt < D / 8; ++nt) { o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f; }
-        float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
-
-        for (int i = 0; i < span.ntiles; ++i, ++it) {
-            const int st = it % STAGES;
-            if (ok && !ptx::mbar_wait(s_full + 8 * st, (it / STAGES) & 1)) ok = false;   // after a timeout: stop waiting
-            const int64_t t0 = int64_t(span.tile0 + i) * kTileTokens;
-            const int64_t left = int64_t(seg.n_tokens) - t0;
-            const int n_valid = left < kTileTokens ? int(left) : kTileTokens;
+            for (int nt = 0; nt < D / 8; ++nt) { o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f; }
+            m0 = m1 = -INFINITY; l0 = l1 = 0.f;
+        }
+        const int n_valid = s_meta[st].n_valid;
+        {
             if (warp * 16 < n_valid) {
                 const uint32_t kb = s_base + st * SP::kStage;
                 const uint32_t vb = kb + SP::kPlane;
@@ -278,32 +437,6 @@ __global__ void __launch_bounds__(kThreads) attn_gqa_kernel(const GqaParams p) {
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(s_empty + 8 * st);
         }
-
-        // ---- end of span: this warp's normalised partial (rows = the group's query heads) ----
-        l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
-        l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
-        if (!DUP) {
-            l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
-            l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
-        }
-        const int64_t prow = (int64_t(sp) * kConsumerWarps + warp) * p.RG;
-        if (r0 < n_heads) {
-            const float inv = l0 > 0.f ? 1.f / l0 : 0.f;
-            float* dst = p.part_o + (prow + r0) * D + c0;
-#pragma unroll
-            for (int nt = 0; nt < D / 8; ++nt) {
-                const float x = DUP ? o[nt][0] + o[nt][2] : o[nt][0], y = DUP ? o[nt][1] + o[nt][3] : o[nt][1];
-                *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(x * inv, y * inv);
-            }
-            if ((lane & 3) == 0) p.part_lse[prow + r0] = (m0 == -INFINITY) ? -INFINITY : (m0 + log2f(l0)) * kLn2;
-        }
-        if (!DUP && r0 + 8 < n_heads) {
-            const float inv = l1 > 0.f ? 1.f / l1 : 0.f;
-            float* dst = p.part_o + (prow + r0 + 8) * D + c0;
-#pragma unroll
-            for (int nt = 0; nt < D / 8; ++nt) *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(o[nt][2] * inv, o[nt][3] * inv);
-            if ((lane & 3) == 0) p.part_lse[prow + r0 + 8] = (m1 == -INFINITY) ? -INFINITY : (m1 + log2f(l1)) * kLn2;
-        }
     }
     if (!ok && lane == 0) atomicOr(p.status, 1u);
 }
@@ -316,6 +449,7 @@ cudaError_t launch_gqa(const AttnLaunch& a, cudaStream_t s) {
     for (int i = 0; i < kMaxBases; ++i) p.bases[i] = a.bases[i];
     p.segs = a.segs; p.spans = a.spans; p.cta_span_start = a.cta_span_start;
     p.part_o = a.part_o; p.part_lse = a.part_lse; p.status = a.status;
+    p.next = a.steal_next; p.tags = a.steal_tags; p.n_spans = a.n_spans; p.n_ctas = a.n_ctas; p.cta_tiles = a.cta_tiles;
     p.Hq = a.n_q_heads; p.G = a.n_q_heads / a.n_kv_heads;
     p.n_hg = (p.G + 15) / 16;
     p.RG = part_geom(0, a.n_q_heads, a.n_kv_heads).rows_per_group;

@@ -32,6 +32,7 @@ struct AttnLaunch {
     const Span* spans;
     const int32_t* cta_span_start;  // [n_ctas + 1]
     const int32_t* rg_span_start;   // [n_rows * n_gh + 1]
+    const int32_t* cta_tiles;       // [n_ctas] tiles per chunk
     int n_spans, n_ctas, n_rows, n_gh;
     float* part_o;                  // [n_spans * parts_per_span][rows_per_group][dv]
     float* part_lse;                // [n_spans * parts_per_span][rows_per_group]
@@ -40,7 +41,16 @@ struct AttnLaunch {
     float* out_o;                   // [n_rows][Hq][dv]
     float* out_lse;                 // [n_rows][Hq]
     uint32_t* status;               // device word, OR-ed with an error bit if a bounded wait gives up
+    // Dynamic load balancing of the GQA kernel (all null = static schedule with bit-reproducible results): a CTA
+    // that has finished its chunk takes tiles from the spans that are furthest behind and accumulates them into
+    // extra partials of its own, stored after the spans' partials (kStealSlots per CTA).
+    int32_t* steal_next;            // [n_spans + 2 * n_ctas]: tiles claimed so far of every span, tiles claimed of every CTA's
+                                    // chunk, CTAs that came to help with every chunk; zero when the kernel starts
+    int32_t* steal_tags;            // [n_ctas * kStealSlots] span + 1 of every extra partial filled; zero when the kernel starts
+    int32_t* steal_clear;           // words the split reduce sets to zero for the launch after this one
+    int steal_clear_words;
 };
+constexpr int kStealSlots = 4;
 
 // Geometry of the partial buffers: query heads per head group (rows of one partial), head groups per row,
 // partials per span (one per consumer warp for GQA, one for MLA), resident CTAs per SM.

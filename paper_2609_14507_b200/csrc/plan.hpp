@@ -29,12 +29,14 @@ struct Plan {
     std::vector<Span> spans;
     std::vector<int32_t> cta_span_start;   // [n_ctas + 1]
     std::vector<int32_t> rg_span_start;    // [n_rows * n_gh + 1]: spans of every (row, head group), contiguous
+    std::vector<int32_t> cta_tiles;        // [n_ctas]: tiles in every CTA's chunk (for the dynamic balancing of the GQA kernel)
     int n_gh = 1;
     int64_t total_tokens = 0;
     int n_ctas() const { return int(cta_span_start.size()) - 1; }
     size_t table_bytes() const {
         return align_up(segs.size() * sizeof(Seg), 16) + align_up(spans.size() * sizeof(Span), 16) +
-               align_up(cta_span_start.size() * sizeof(int32_t), 16) + align_up(rg_span_start.size() * sizeof(int32_t), 16);
+               align_up(cta_span_start.size() * sizeof(int32_t), 16) + align_up(rg_span_start.size() * sizeof(int32_t), 16) +
+               align_up(cta_tiles.size() * sizeof(int32_t), 16);
     }
     void serialize(char* dst) const {
         size_t o = 0;
@@ -45,6 +47,8 @@ struct Plan {
         std::memcpy(dst + o, cta_span_start.data(), cta_span_start.size() * sizeof(int32_t));
         o += align_up(cta_span_start.size() * sizeof(int32_t), 16);
         std::memcpy(dst + o, rg_span_start.data(), rg_span_start.size() * sizeof(int32_t));
+        o += align_up(rg_span_start.size() * sizeof(int32_t), 16);
+        if (!cta_tiles.empty()) std::memcpy(dst + o, cta_tiles.data(), cta_tiles.size() * sizeof(int32_t));
     }
 };
 
@@ -59,7 +63,7 @@ inline int64_t max_spans_bound(int n_rows, int n_runs, int n_gh, int kv_splits, 
 // kv_splits > 0: every (row, head group) is cut into about that many spans of equal length, one span per CTA
 // while they last (more spans than slots: several spans per CTA, still balanced).
 inline void build_plan(const std::vector<std::vector<PlanSeg>>& rows, int n_gh, int kv_splits, int ctas_per_sm, Plan* plan) {
-    plan->segs.clear(); plan->spans.clear(); plan->cta_span_start.clear(); plan->rg_span_start.clear();
+    plan->segs.clear(); plan->spans.clear(); plan->cta_span_start.clear(); plan->rg_span_start.clear(); plan->cta_tiles.clear();
     plan->n_gh = n_gh;
     const int64_t slots = int64_t(kSmCount) * ctas_per_sm;
     // segments, and the tiles of every row
@@ -115,6 +119,10 @@ inline void build_plan(const std::vector<std::vector<PlanSeg>>& rows, int n_gh, 
     }
     while (int64_t(plan->cta_span_start.size()) < n_ctas + 1) plan->cta_span_start.push_back(int32_t(plan->spans.size()));
     if (n_ctas == 0) plan->cta_span_start.assign(1, 0);
+    plan->cta_tiles.assign(size_t(plan->n_ctas()), 0);
+    for (int c = 0; c < plan->n_ctas(); ++c)
+        for (int32_t k = plan->cta_span_start[size_t(c)]; k < plan->cta_span_start[size_t(c) + 1]; ++k)
+            plan->cta_tiles[size_t(c)] += plan->spans[size_t(k)].ntiles;
     // spans of every (row, head group): contiguous because of the emission order
     plan->rg_span_start.assign(rows.size() * size_t(n_gh) + 1, 0);
     {

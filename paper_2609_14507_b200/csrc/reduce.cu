@@ -28,13 +28,20 @@ struct ReduceParams {
     float* out_o;
     float* out_lse;
     int Hq, dv, G, n_hg, n_gh, RG, NW;
+    const int32_t* tags;       // extra partials written by CTAs that helped other spans: tags[i] = span + 1 (0 = unused)
+    int n_tags, n_spans;       // extra partial i is stored as if it were span n_spans + i
+    int32_t* clear;            // scheduling words to zero for the next launch
+    int clear_words;
 };
+constexpr int kMaxExtra = 2048;
 
 __global__ void __launch_bounds__(kReduceThreads) split_reduce_kernel(const ReduceParams p) {
     extern __shared__ float4 red[];                 // [SL][CG]
     __shared__ float s_warp[kReduceThreads / 32];
     __shared__ float s_m;
     __shared__ float s_zs[kReduceThreads / 16];    // weight sum of every entry slice (SL <= 16)
+    __shared__ int s_extra[kMaxExtra];             // extra partials that belong to this (row, head group)
+    __shared__ int s_n_extra;
     const int wid = blockIdx.x;                      // row * Hq + h
     const int row = wid / p.Hq, h = wid - row * p.Hq;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -42,13 +49,36 @@ __global__ void __launch_bounds__(kReduceThreads) split_reduce_kernel(const Redu
     const int gh = g * p.n_hg + hin / 16, rin = hin % 16;
     const int sp0 = p.rg_span_start[row * p.n_gh + gh], sp1 = p.rg_span_start[row * p.n_gh + gh + 1];
     const int64_t e0 = int64_t(sp0) * p.NW;
-    const int n = (sp1 - sp0) * p.NW;
+    const int n_own = (sp1 - sp0) * p.NW;
     const int dv = p.dv;
     const float la = p.acc_lse ? p.acc_lse[wid] : -INFINITY;
-    const float* lse_base = p.part_lse + e0 * p.RG + rin;          // entry e at lse_base[e * RG]
+    for (int i = blockIdx.x * kReduceThreads + tid; i < p.clear_words; i += gridDim.x * kReduceThreads) p.clear[i] = 0;
+    if (tid == 0) s_n_extra = 0;
+    __syncthreads();
+    if (p.tags) {
+        // all loads first (independent), then the matches
+        int tag[kMaxExtra / kReduceThreads];
+#pragma unroll
+        for (int j = 0; j < kMaxExtra / kReduceThreads; ++j) {
+            const int i = j * kReduceThreads + tid;
+            tag[j] = i < p.n_tags ? __ldg(p.tags + i) - 1 : -1;
+        }
+#pragma unroll
+        for (int j = 0; j < kMaxExtra / kReduceThreads; ++j)
+            if (tag[j] >= sp0 && tag[j] < sp1) s_extra[atomicAdd(&s_n_extra, 1)] = j * kReduceThreads + tid;
+        __syncthreads();
+    }
+    const int n = n_own + s_n_extra * p.NW;
+    // entry e of this (row, head group): the spans' own partials first, then the extra ones
+    auto entry = [&](int e) -> int64_t {
+        if (e < n_own) return e0 + e;
+        const int k = (e - n_own) / p.NW;
+        return int64_t(p.n_spans + s_extra[k]) * p.NW + (e - n_own - k * p.NW);
+    };
+    const float* lse_base = p.part_lse + rin;                      // entry e at lse_base[entry(e) * RG]
 
     float m = la;
-    for (int e = tid; e < n; e += kReduceThreads) m = fmaxf(m, lse_base[int64_t(e) * p.RG]);
+    for (int e = tid; e < n; e += kReduceThreads) m = fmaxf(m, lse_base[entry(e) * p.RG]);
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, d));
     if (lane == 0) s_warp[warp] = m;
@@ -71,14 +101,15 @@ __global__ void __launch_bounds__(kReduceThreads) split_reduce_kernel(const Redu
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float z = 0.f;
     {
-        const float* po = p.part_o + (e0 * p.RG + rin) * dv + cg * 4;
+        const float* po = p.part_o + int64_t(rin) * dv + cg * 4;
         const int64_t stride = int64_t(p.RG) * dv;
 #pragma unroll 4
         for (int e = sl; e < n; e += SL) {
-            const float li = lse_base[int64_t(e) * p.RG];
+            const int64_t ee = entry(e);
+            const float li = lse_base[ee * p.RG];
             if (li == -INFINITY) continue;          // a warp that saw no valid token
             const float w = __expf(li - m);
-            const float4 v = *reinterpret_cast<const float4*>(po + int64_t(e) * stride);
+            const float4 v = *reinterpret_cast<const float4*>(po + ee * stride);
             acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
             z += w;
         }
@@ -163,6 +194,9 @@ cudaError_t launch_split_reduce(const AttnLaunch& a, cudaStream_t s) {
     p.G = a.kind == 1 ? a.n_q_heads : a.n_q_heads / a.n_kv_heads;
     p.n_hg = (p.G + 15) / 16;
     p.n_gh = pg.n_gh; p.RG = pg.rows_per_group; p.NW = pg.parts_per_span;
+    p.tags = a.steal_tags; p.n_tags = a.steal_tags ? a.n_ctas * kStealSlots : 0; p.n_spans = a.n_spans;
+    p.clear = a.steal_clear; p.clear_words = a.steal_clear ? a.steal_clear_words : 0;
+    if (p.n_tags > kMaxExtra) return cudaErrorInvalidValue;
     const size_t smem = size_t(kReduceThreads) * sizeof(float4);
     split_reduce_kernel<<<total, kReduceThreads, smem, s>>>(p);
     return cudaGetLastError();
