@@ -16,6 +16,17 @@
 // span: at the end of a span every warp writes its own normalised partial (O, natural-log LSE) and the
 // LSE reduce joins the partials of all spans and warps of a (row, head).
 //
+// Dynamic balancing (default for the handle-based calls).  With equal chunks the CTAs do not finish together:
+// some SMs are consistently served less of the memory bandwidth than others (end times spread over +-10 %),
+// and a kernel is as slow as its last CTA.  So tiles are not handed out by position but claimed: every span has
+// a counter that its owner advances in batches (an eighth of what is left per claim, the next claim issued
+// before the current batch is copied), and a CTA whose own chunk is exhausted picks the chunk with the most
+// unclaimed tiles per CTA already working on it, claims tiles from the span that chunk's owner would reach
+// last, and accumulates them into an extra partial of its own (kStealSlots per CTA, tagged with the span so
+// that the reduce finds them).  A partial is an exact softmax state over whatever set of tokens went into it, so
+// any assignment of tiles to partials gives the same attention; only the fp32 summation order changes.  No CTA
+// ever waits for another one.  The static schedule (null counters) visits the same tiles in plan order.
+//
 // HBM traffic per KV token: bytes_per_token, read exactly once.
 #include <cuda_bf16.h>
 
@@ -69,7 +80,7 @@ struct StageMeta {
     int32_t n_heads;     // query heads in the group (at most 16)
 };
 constexpr int32_t kEndSlot = -1;
-constexpr int kMinSteal = 3;        // a span is worth stealing from while at least this many tiles are unclaimed
+constexpr int kMinSteal = 3;        // a chunk is worth helping while at least this many of its tiles are unclaimed
 
 template <int D, int STAGES, bool DUP>
 __global__ void __launch_bounds__(kThreads) attn_gqa_kernel(const GqaParams p) {

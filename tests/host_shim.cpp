@@ -46,7 +46,8 @@ void shim_router_dump(void* r, int8_t* region, int64_t* blk, int32_t* off) {
 // plan: rows given as flat (row_start[n_rows+1], n_tokens[n_segs]); fills the span table and the two index arrays
 int shim_plan(int n_rows, const int32_t* row_start, const int64_t* seg_tokens, int n_gh, int kv_splits, int ctas_per_sm,
               int cap_spans, int32_t* span_fields /* [cap][5] */, int32_t* cta_span_start /* [<= 148*ctas_per_sm + 1] */,
-              int* n_ctas_out, int32_t* rg_span_start /* [n_rows*n_gh + 1] */, int32_t* seg_tokens_out, int* n_segs_out) {
+              int* n_ctas_out, int32_t* rg_span_start /* [n_rows*n_gh + 1] */, int32_t* seg_tokens_out, int* n_segs_out,
+              int32_t* cta_tiles /* [<= 148*ctas_per_sm] */, int64_t* table_bytes_out) {
     std::vector<std::vector<PlanSeg>> rows(n_rows);
     for (int r = 0; r < n_rows; ++r)
         for (int k = row_start[r]; k < row_start[r + 1]; ++k) rows[r].push_back(PlanSeg{0, int64_t(k) * 4096, seg_tokens[k]});
@@ -65,6 +66,14 @@ int shim_plan(int n_rows, const int32_t* row_start, const int64_t* seg_tokens, i
     *n_ctas_out = plan.n_ctas();
     for (size_t c = 0; c < plan.cta_span_start.size(); ++c) cta_span_start[c] = plan.cta_span_start[c];
     for (size_t c = 0; c < plan.rg_span_start.size(); ++c) rg_span_start[c] = plan.rg_span_start[c];
+    for (size_t c = 0; c < plan.cta_tiles.size(); ++c) cta_tiles[c] = plan.cta_tiles[c];
+    {   // the serialised image has exactly table_bytes() bytes: write it into a guarded buffer
+        const size_t tb = plan.table_bytes();
+        std::vector<char> img(tb + 64, char(0x5a));
+        plan.serialize(img.data());
+        for (size_t i = tb; i < tb + 64; ++i) if (img[i] != char(0x5a)) return -2000000;
+        *table_bytes_out = int64_t(tb);
+    }
     *n_segs_out = int(plan.segs.size());
     for (size_t k = 0; k < plan.segs.size(); ++k) seg_tokens_out[k] = plan.segs[k].n_tokens;
     return n;

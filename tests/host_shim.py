@@ -33,7 +33,7 @@ def lib():
         L.shim_router_len.restype = C.c_int64
         L.shim_router_counts.argtypes = [C.c_void_p, C.c_void_p]
         L.shim_router_dump.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
-        L.shim_plan.argtypes = [C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int] + [C.c_void_p] * 6
+        L.shim_plan.argtypes = [C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int] + [C.c_void_p] * 8
         L.shim_plan.restype = C.c_int
         L.shim_tile_chunk_offset.argtypes = [C.c_int32] * 3
         L.shim_tile_chunk_offset.restype = C.c_int64
@@ -97,10 +97,13 @@ def plan(rows, n_gh, kv_splits=0, ctas_per_sm=2):
     cta = np.zeros(148 * ctas_per_sm + 2, dtype=np.int32)
     rg = np.zeros(len(rows) * n_gh + 1, dtype=np.int32)
     seg_out = np.zeros(len(segs) + 1, dtype=np.int32)
-    n_segs, n_ctas = C.c_int(), C.c_int()
+    n_segs, n_ctas, table_bytes = C.c_int(), C.c_int(), C.c_int64()
+    cta_tiles = np.zeros(148 * ctas_per_sm + 2, dtype=np.int32)
     n = lib().shim_plan(len(rows), row_start.ctypes.data, seg_tokens.ctypes.data, n_gh, kv_splits, ctas_per_sm, cap,
-                        fields.ctypes.data, cta.ctypes.data, C.byref(n_ctas), rg.ctypes.data, seg_out.ctypes.data, C.byref(n_segs))
+                        fields.ctypes.data, cta.ctypes.data, C.byref(n_ctas), rg.ctypes.data, seg_out.ctypes.data, C.byref(n_segs),
+                        cta_tiles.ctypes.data, C.byref(table_bytes))
     assert n >= 0, n
     f = fields[:n]
     return dict(row=f[:, 0], gh=f[:, 1], seg=f[:, 2], tile0=f[:, 3], ntiles=f[:, 4], cta_span_start=cta[:n_ctas.value + 1],
-                rg_span_start=rg, seg_tokens=seg_out[:n_segs.value])
+                rg_span_start=rg, seg_tokens=seg_out[:n_segs.value], cta_tiles=cta_tiles[:n_ctas.value],
+                table_bytes=table_bytes.value)

@@ -471,3 +471,43 @@ def test_grow_p_rejects_bad_configs():
         kw.update(bad)
         with pytest.raises(binding.IpkvError):
             make_cache(sh, 1, 2, **kw)
+
+
+def test_static_schedule_is_bit_reproducible_and_dynamic_agrees():
+    """The grouped-query kernel balances its load while it runs (CTAs that finish early take over tiles of the ones
+    behind), so which tiles meet in which partial can change from launch to launch.  With
+    IPKV_ATTEND_STATIC_SCHEDULE the assignment is fixed: two calls give identical bits.  Both schedules compute the
+    same attention: they agree with each other far inside the parity tolerance, and with the oracle."""
+    sh = synth.Shape("mid", "gqa", 1, 32, 4, 128, 128, 128 ** -0.5)
+    n_seq, ctx = 12, 6000            # 12 x 4 x 94 tiles: every CTA of the persistent grid has work, some have several spans
+    scale = float(np.float32(sh.scale))
+    with make_cache(sh, 1, n_seq, block_tokens=64, window_tokens=256, chunk_tokens=512, max_u_tokens_per_seq=64,
+                    max_p_tokens_per_seq=ctx + 512, resident_tokens_per_seq=ctx + 512,
+                    flags=binding.FLAG_NO_HOST_U | binding.FLAG_NO_HOST_P) as cache:
+        ks, vs = [], []
+        for s in range(n_seq):
+            k, v = synth.host_kv(sh, ctx - 37 * s, seed=9100 + s)
+            cache.append_bulk(0, s, synth.bits_to_torch(k, DEV), synth.bits_to_torch(v, DEV), ctx - 37 * s, 0, 1)
+            ks.append(k); vs.append(v)
+        q = synth.host_q(sh, n_seq, seed=9200)
+        qd = synth.bits_to_torch(q, DEV)
+        seqs = list(range(n_seq))
+
+        def run(static):
+            o = torch.zeros((n_seq, 32, 128), device=DEV); lse = torch.zeros((n_seq, 32), device=DEV)
+            cache.attend_gpu(0, seqs, qd, o, lse, static_schedule=static)
+            torch.cuda.synchronize()
+            return o.cpu().numpy(), lse.cpu().numpy()
+
+        o_s1, l_s1 = run(True)
+        o_s2, l_s2 = run(True)
+        np.testing.assert_array_equal(o_s1, o_s2)
+        np.testing.assert_array_equal(l_s1, l_s2)
+        for _ in range(3):                                   # alternate launches use alternate sets of scheduling words
+            o_d, l_d = run(False)
+            assert np.abs(o_d - o_s1).max() < 2e-5 and np.abs(l_d - l_s1).max() < 2e-5
+        for s in (0, 5, 11):
+            o_ref, l_ref = c_oracle.attend(q[s], ks[s], vs[s], np.arange(ks[s].shape[0]), scale)
+            check_partial(o_d[s], l_d[s], o_ref, l_ref, f"dynamic schedule, sequence {s}")
+            check_partial(o_s1[s], l_s1[s], o_ref, l_ref, f"static schedule, sequence {s}")
+        assert cache.get_stats()["device_status"] == 0

@@ -71,6 +71,9 @@ def test_plan_covers_every_tile_exactly_once():
         assert css[0] == 0 and css[-1] == n_spans and np.all(np.diff(css) >= 0) and len(css) - 1 <= 148 * cps
         assert rgs[0] == 0 and rgs[-1] == n_spans and np.all(np.diff(rgs) >= 0)
         assert np.all(p["ntiles"] >= 1)
+        # tiles per chunk, the table the dynamically balanced kernel looks for work in
+        assert list(p["cta_tiles"]) == [int(p["ntiles"][css[c]:css[c + 1]].sum()) for c in range(len(css) - 1)]
+        assert p["table_bytes"] > 0
         seg_id0 = 0
         for r, row in enumerate(live):
             for gh in range(n_gh):
