@@ -673,10 +673,10 @@ ipkv_status run_group(ipkv* h, const std::vector<std::vector<PlanSeg>>& rows, co
     const PartGeom pg = part_geom(c.kind, c.n_q_heads, c.n_kv_heads);
     build_plan(rows, pg.n_gh, kv_splits, pg.ctas_per_sm, &plan);
     // dynamic balancing: every CTA may fill up to kStealSlots extra partials (GQA kernel; more than one CTA)
-    const size_t n_tags = size_t(plan.n_ctas()) * kStealSlots;
-    const bool balance = !static_schedule && c.kind == IPKV_GQA && plan.n_ctas() > 1 &&
-                         n_tags + plan.spans.size() + 2 * size_t(plan.n_ctas()) <= size_t(ipkv::kStealWords);
-    const size_t extra = balance ? n_tags : 0;
+    const size_t n_lists = rows.size() * size_t(pg.n_gh) * (1 + kStealListCap);
+    const size_t steal_words = n_lists + plan.spans.size() + 2 * size_t(plan.n_ctas());
+    const bool balance = !static_schedule && c.kind == IPKV_GQA && plan.n_ctas() > 1 && steal_words <= size_t(ipkv::kStealWords);
+    const size_t extra = balance ? size_t(plan.n_ctas()) * kStealSlots : 0;
     ipkv_status rc = ensure_scratch(h, partial_bytes(plan.spans.size() + extra, pg, c.dim_v));
     if (rc != IPKV_OK) return rc;
     const char* table = nullptr;
@@ -688,9 +688,9 @@ ipkv_status run_group(ipkv* h, const std::vector<std::vector<PlanSeg>>& rows, co
     if (balance) {
         const int set = int(h->steal_epoch & 1u), other = set ^ 1;
         int32_t* words = h->steal_dev + size_t(set) * ipkv::kStealWords;
-        a.steal_tags = words;
-        a.steal_next = words + n_tags;
-        h->steal_dirty[set] = int(n_tags + plan.spans.size() + 2 * size_t(plan.n_ctas()));
+        a.steal_lists = words;
+        a.steal_next = words + n_lists;
+        h->steal_dirty[set] = int(steal_words);
         a.steal_clear = h->steal_dev + size_t(other) * ipkv::kStealWords;     // used by the balanced launch after this one
         a.steal_clear_words = h->steal_dirty[other];
         h->steal_dirty[other] = 0;

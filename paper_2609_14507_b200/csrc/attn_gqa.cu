@@ -22,8 +22,8 @@
 // a counter that its owner advances in batches (an eighth of what is left per claim, the next claim issued
 // before the current batch is copied), and a CTA whose own chunk is exhausted picks the chunk with the most
 // unclaimed tiles per CTA already working on it, claims tiles from the span that chunk's owner would reach
-// last, and accumulates them into an extra partial of its own (kStealSlots per CTA, tagged with the span so
-// that the reduce finds them).  A partial is an exact softmax state over whatever set of tokens went into it, so
+// last, and accumulates them into an extra partial of its own (kStealSlots per CTA, entered in the list of the
+// span's (row, head group), where the reduce finds it).  A partial is an exact softmax state over whatever set of tokens went into it, so
 // any assignment of tiles to partials gives the same attention; only the fp32 summation order changes.  No CTA
 // ever waits for another one.  The static schedule (null counters) visits the same tiles in plan order.
 //
@@ -54,8 +54,9 @@ struct GqaParams {
     int32_t* next;       // dynamic schedule: tiles claimed so far of every span [n_spans], of every CTA's chunk [n_ctas], and the
                          // number of CTAs that came to help with every chunk [n_ctas] (all zero at launch); null = static schedule
     const int32_t* cta_tiles;   // tiles in every CTA's chunk
-    int32_t* tags;       // [n_ctas * kStealSlots]: span + 1 of every extra partial a CTA filled (zero at launch); null = no stealing
-    int n_spans, n_ctas;
+    int32_t* lists;      // per (row, head group): the number of extra partials CTAs filled for it [n_rows * n_gh], then their indices
+                         // [n_rows * n_gh][kStealListCap] (all zero at launch); null = no CTA helps another
+    int n_spans, n_ctas, n_rows, n_gh;
     int Hq, G, n_hg, RG;
     int bt;
     int64_t head_bytes, block_bytes;
@@ -172,7 +173,7 @@ __global__ void __launch_bounds__(kThreads) attn_gqa_kernel(const GqaParams p) {
             // of what is left, 8 at most), so that little is locked in when other CTAs come to help, and the claim of
             // the next batch is under way while the copies of the current one are issued. Returns the number of
             // tiles streamed (-1 after a timeout).
-            auto drain = [&](int sp, int chunk, int slot, int32_t* tag) -> int {
+            auto drain = [&](int sp, int chunk, int slot, bool helping) -> int {
                 const Span span = p.spans[sp];
                 const Seg seg = p.segs[span.seg];
                 const char* seg_base = p.bases[seg.base_id] + seg.off + int64_t(span.gh / p.n_hg) * p.head_bytes;
@@ -183,7 +184,7 @@ __global__ void __launch_bounds__(kThreads) attn_gqa_kernel(const GqaParams p) {
                     return n;
                 }
                 // the owner takes an eighth of what is left per claim, a helper a quarter
-                const int shift = tag ? 2 : 3;
+                const int shift = helping ? 2 : 3;
                 auto batch = [shift](int left) { const int b = left >> shift; return b > 8 ? 8 : (b < 1 ? 1 : b); };
                 int b = batch(span.ntiles - *reinterpret_cast<volatile int32_t*>(p.next + sp));
                 int t0 = atomicAdd(p.next + sp, b);
@@ -192,7 +193,6 @@ __global__ void __launch_bounds__(kThreads) attn_gqa_kernel(const GqaParams p) {
                     const int left = span.ntiles - last;           // as far as this CTA knows
                     b = batch(left);
                     t0 = left > 0 ? atomicAdd(p.next + sp, b) : span.ntiles;
-                    if (n == 0 && tag) *tag = sp + 1;              // this CTA's extra partial `slot` belongs to span sp
                     atomicAdd(p.next + p.n_spans + chunk, last - first);     // what is left of the chunk, for CTAs looking for work
                     for (int t = first; t < last; ++t, ++n)
                         if (!issue(span, seg, seg_base, span.tile0 + t, slot)) return -1;
@@ -201,11 +201,11 @@ __global__ void __launch_bounds__(kThreads) attn_gqa_kernel(const GqaParams p) {
             };
             // own chunk first: the partial of a span lives at the span's index
             if (lane == 0)
-                for (int sp = span_begin; sp < span_end && ok; ++sp) ok = drain(sp, int(blockIdx.x), sp, nullptr) >= 0;
+                for (int sp = span_begin; sp < span_end && ok; ++sp) ok = drain(sp, int(blockIdx.x), sp, false) >= 0;
             // then help the CTAs that are behind (some SMs get less of the memory bandwidth than others): pick the chunk with
             // the most unclaimed tiles per CTA already working on it, take tiles from the span its owner will reach last,
             // and accumulate them into one of this CTA's extra partials
-            if (dynamic && p.tags) {
+            if (dynamic && p.lists) {
                 int32_t* claimed = p.next + p.n_spans;
                 int32_t* helpers = claimed + p.n_ctas;
                 int used = 0;
@@ -240,20 +240,35 @@ __global__ void __launch_bounds__(kThreads) attn_gqa_kernel(const GqaParams p) {
                     const unsigned turned = (good >> rot) | (rot ? good << (32 - rot) : 0u);
                     const int pick = (__ffs(turned) - 1 + rot) & 31;
                     const int victim = __shfl_sync(0xffffffffu, best, pick);
-                    int n = 0;
+                    // lane 0: the last span of the victim's chunk that still has unclaimed tiles; one of this CTA's extra
+                    // partials is entered in the list of the span's (row, head group) unless that list is full
+                    const int mine = int(blockIdx.x) * kStealSlots + used;
+                    int sp = -1;
                     if (lane == 0) {
                         atomicAdd(helpers + victim, 1);
-                        // the last span of the victim's chunk that still has unclaimed tiles
-                        int sp = p.cta_span_start[victim + 1] - 1;
+                        sp = p.cta_span_start[victim + 1] - 1;
                         const int sp_first = p.cta_span_start[victim];
                         while (sp >= sp_first && __ldcg(p.next + sp) >= p.spans[sp].ntiles) --sp;
-                        if (sp >= sp_first) {
-                            n = drain(sp, victim, p.n_spans + int(blockIdx.x) * kStealSlots + used, p.tags + int(blockIdx.x) * kStealSlots + used);
-                            if (n < 0) ok = false;
+                        if (sp < sp_first) sp = -1;
+                        if (sp >= 0) {
+                            const int rg = p.spans[sp].row * p.n_gh + p.spans[sp].gh;
+                            const int k = atomicAdd(p.lists + rg, 1);
+                            if (k < kStealListCap) p.lists[p.n_rows * p.n_gh + rg * kStealListCap + k] = mine;
+                            else sp = -1;
                         }
                     }
-                    n = __shfl_sync(0xffffffffu, n, 0);
-                    if (n > 0) ++used;
+                    sp = __shfl_sync(0xffffffffu, sp, 0);
+                    if (sp < 0) continue;
+                    // the partial is listed from now on: empty until tiles arrive (the span may run out first)
+                    for (int i = lane; i < kConsumerWarps * p.RG; i += 32)
+                        p.part_lse[(int64_t(p.n_spans) + mine) * kConsumerWarps * p.RG + i] = -INFINITY;
+                    __syncwarp();
+                    ++used;
+                    int n = 0;
+                    if (lane == 0) {
+                        n = drain(sp, victim, p.n_spans + mine, true);
+                        if (n < 0) ok = false;
+                    }
                 }
             }
             if (lane == 0) {
@@ -460,7 +475,8 @@ cudaError_t launch_gqa(const AttnLaunch& a, cudaStream_t s) {
     for (int i = 0; i < kMaxBases; ++i) p.bases[i] = a.bases[i];
     p.segs = a.segs; p.spans = a.spans; p.cta_span_start = a.cta_span_start;
     p.part_o = a.part_o; p.part_lse = a.part_lse; p.status = a.status;
-    p.next = a.steal_next; p.tags = a.steal_tags; p.n_spans = a.n_spans; p.n_ctas = a.n_ctas; p.cta_tiles = a.cta_tiles;
+    p.next = a.steal_next; p.lists = a.steal_lists; p.n_spans = a.n_spans; p.n_ctas = a.n_ctas; p.cta_tiles = a.cta_tiles;
+    p.n_rows = a.n_rows; p.n_gh = a.n_gh;
     p.Hq = a.n_q_heads; p.G = a.n_q_heads / a.n_kv_heads;
     p.n_hg = (p.G + 15) / 16;
     p.RG = part_geom(0, a.n_q_heads, a.n_kv_heads).rows_per_group;

@@ -43,14 +43,16 @@ struct AttnLaunch {
     uint32_t* status;               // device word, OR-ed with an error bit if a bounded wait gives up
     // Dynamic load balancing of the GQA kernel (all null = static schedule with bit-reproducible results): a CTA
     // that has finished its chunk takes tiles from the spans that are furthest behind and accumulates them into
-    // extra partials of its own, stored after the spans' partials (kStealSlots per CTA).
+    // extra partials of its own, stored after the spans' partials (kStealSlots per CTA) and listed per (row, head group).
     int32_t* steal_next;            // [n_spans + 2 * n_ctas]: tiles claimed so far of every span, tiles claimed of every CTA's
                                     // chunk, CTAs that came to help with every chunk; zero when the kernel starts
-    int32_t* steal_tags;            // [n_ctas * kStealSlots] span + 1 of every extra partial filled; zero when the kernel starts
+    int32_t* steal_lists;           // [n_rows * n_gh] number of extra partials of every (row, head group), then
+                                    // [n_rows * n_gh][kStealListCap] their indices; zero when the kernel starts
     int32_t* steal_clear;           // words the split reduce sets to zero for the launch after this one
     int steal_clear_words;
 };
-constexpr int kStealSlots = 4;
+constexpr int kStealSlots = 4;      // extra partials a CTA can fill
+constexpr int kStealListCap = 16;   // extra partials a (row, head group) can take
 
 // Geometry of the partial buffers: query heads per head group (rows of one partial), head groups per row,
 // partials per span (one per consumer warp for GQA, one for MLA), resident CTAs per SM.

@@ -14,6 +14,8 @@ namespace {
 
 constexpr int kWarpsPerBlock = 4;
 constexpr int kReduceThreads = 256;
+constexpr int kPrefetch = 4;       // partial outputs per thread requested up front
+constexpr int kLseCache = 512;     // LSE values kept in shared memory between the two passes
 
 // One CTA per (row, query head). The partials to join are those of the spans of the head's group
 // (parts_per_span consecutive entries per span), row `rin` of each. Threads are arranged as
@@ -28,19 +30,19 @@ struct ReduceParams {
     float* out_o;
     float* out_lse;
     int Hq, dv, G, n_hg, n_gh, RG, NW;
-    const int32_t* tags;       // extra partials written by CTAs that helped other spans: tags[i] = span + 1 (0 = unused)
-    int n_tags, n_spans;       // extra partial i is stored as if it were span n_spans + i
-    int32_t* clear;            // scheduling words to zero for the next launch
+    const int32_t* extra_count;   // per (row, head group): extra partials written by CTAs that helped with its spans (null: none)
+    const int32_t* extra_list;    // [n_rows * n_gh][kStealListCap] their indices; extra partial i is stored as if it were span n_spans + i
+    int n_spans;
+    int32_t* clear;               // scheduling words to zero for the next launch
     int clear_words;
 };
-constexpr int kMaxExtra = 2048;
 
 __global__ void __launch_bounds__(kReduceThreads) split_reduce_kernel(const ReduceParams p) {
     extern __shared__ float4 red[];                 // [SL][CG]
     __shared__ float s_warp[kReduceThreads / 32];
-    __shared__ float s_m;
+    __shared__ float s_w[kLseCache];               // LSE of the first entries
     __shared__ float s_zs[kReduceThreads / 16];    // weight sum of every entry slice (SL <= 16)
-    __shared__ int s_extra[kMaxExtra];             // extra partials that belong to this (row, head group)
+    __shared__ int s_extra[kStealListCap];         // extra partials that belong to this (row, head group)
     __shared__ int s_n_extra;
     const int wid = blockIdx.x;                      // row * Hq + h
     const int row = wid / p.Hq, h = wid - row * p.Hq;
@@ -53,21 +55,14 @@ __global__ void __launch_bounds__(kReduceThreads) split_reduce_kernel(const Redu
     const int dv = p.dv;
     const float la = p.acc_lse ? p.acc_lse[wid] : -INFINITY;
     for (int i = blockIdx.x * kReduceThreads + tid; i < p.clear_words; i += gridDim.x * kReduceThreads) p.clear[i] = 0;
-    if (tid == 0) s_n_extra = 0;
-    __syncthreads();
-    if (p.tags) {
-        // all loads first (independent), then the matches
-        int tag[kMaxExtra / kReduceThreads];
-#pragma unroll
-        for (int j = 0; j < kMaxExtra / kReduceThreads; ++j) {
-            const int i = j * kReduceThreads + tid;
-            tag[j] = i < p.n_tags ? __ldg(p.tags + i) - 1 : -1;
-        }
-#pragma unroll
-        for (int j = 0; j < kMaxExtra / kReduceThreads; ++j)
-            if (tag[j] >= sp0 && tag[j] < sp1) s_extra[atomicAdd(&s_n_extra, 1)] = j * kReduceThreads + tid;
-        __syncthreads();
+    if (p.extra_count) {
+        const int rg = row * p.n_gh + gh;
+        if (tid < kStealListCap) s_extra[tid] = p.extra_list[rg * kStealListCap + tid];
+        if (tid == kStealListCap) s_n_extra = min(p.extra_count[rg], kStealListCap);
+    } else if (tid == 0) {
+        s_n_extra = 0;
     }
+    __syncthreads();
     const int n = n_own + s_n_extra * p.NW;
     // entry e of this (row, head group): the spans' own partials first, then the extra ones
     auto entry = [&](int e) -> int64_t {
@@ -76,45 +71,69 @@ __global__ void __launch_bounds__(kReduceThreads) split_reduce_kernel(const Redu
         return int64_t(p.n_spans + s_extra[k]) * p.NW + (e - n_own - k * p.NW);
     };
     const float* lse_base = p.part_lse + rin;                      // entry e at lse_base[entry(e) * RG]
+    const int CG = dv >> 2, SL = kReduceThreads / CG;
+    const int cg = tid % CG, sl = tid / CG;
+    const float* po = p.part_o + int64_t(rin) * dv + cg * 4;
+    const int64_t stride = int64_t(p.RG) * dv;
+
+    // The partial outputs of this thread's first entries are requested before anything is known about their
+    // weights, so that their latency overlaps the two passes over the LSE values (an entry that turns out to be
+    // empty may hold anything: it is loaded but never used).
+    float4 pre[kPrefetch];
+#pragma unroll
+    for (int j = 0; j < kPrefetch; ++j) {
+        const int e = sl + j * SL;
+        pre[j] = e < n ? *reinterpret_cast<const float4*>(po + entry(e) * stride) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    float4 fold = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (p.acc_o && sl == 0) fold = *reinterpret_cast<const float4*>(p.acc_o + int64_t(wid) * dv + cg * 4);
 
     float m = la;
-    for (int e = tid; e < n; e += kReduceThreads) m = fmaxf(m, lse_base[entry(e) * p.RG]);
+    for (int e = tid; e < n; e += kReduceThreads) {
+        const float li = lse_base[entry(e) * p.RG];
+        if (e < kLseCache) s_w[e] = li;
+        m = fmaxf(m, li);
+    }
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, d));
     if (lane == 0) s_warp[warp] = m;
     __syncthreads();
-    if (tid == 0) {
+    {
         float mm = s_warp[0];
+#pragma unroll
         for (int w = 1; w < kReduceThreads / 32; ++w) mm = fmaxf(mm, s_warp[w]);
-        s_m = mm;
+        m = mm;
     }
-    __syncthreads();
-    m = s_m;
-    const int CG = dv >> 2, SL = kReduceThreads / CG;
-    const int cg = tid % CG, sl = tid / CG;
     float* oo = p.out_o + int64_t(wid) * dv;
     if (m == -INFINITY) {                           // nothing attended: (0, -inf)
         if (sl == 0) *reinterpret_cast<float4*>(oo + cg * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
         if (tid == 0) p.out_lse[wid] = -INFINITY;
         return;
     }
+    // weight of entry e (0 for an empty one); the first kLseCache LSE values are in shared memory
+    auto weight = [&](int e) -> float {
+        const float li = e < kLseCache ? s_w[e] : lse_base[entry(e) * p.RG];
+        return li == -INFINITY ? 0.f : __expf(li - m);
+    };
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float z = 0.f;
-    {
-        const float* po = p.part_o + int64_t(rin) * dv + cg * 4;
-        const int64_t stride = int64_t(p.RG) * dv;
-#pragma unroll 4
-        for (int e = sl; e < n; e += SL) {
-            const int64_t ee = entry(e);
-            const float li = lse_base[ee * p.RG];
-            if (li == -INFINITY) continue;          // a warp that saw no valid token
-            const float w = __expf(li - m);
-            const float4 v = *reinterpret_cast<const float4*>(po + ee * stride);
-            acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
+#pragma unroll
+    for (int j = 0; j < kPrefetch; ++j) {
+        const int e = sl + j * SL;
+        const float w = e < n ? weight(e) : 0.f;
+        if (w != 0.f) {
+            acc.x += w * pre[j].x; acc.y += w * pre[j].y; acc.z += w * pre[j].z; acc.w += w * pre[j].w;
             z += w;
         }
-        red[sl * CG + cg] = acc;
     }
+    for (int e = sl + kPrefetch * SL; e < n; e += SL) {
+        const float w = weight(e);
+        if (w == 0.f) continue;                     // a warp that saw no valid token
+        const float4 v = *reinterpret_cast<const float4*>(po + entry(e) * stride);
+        acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
+        z += w;
+    }
+    red[sl * CG + cg] = acc;
     // every thread of a slice holds the same weight sum z; column group 0 publishes it
     if (cg == 0) s_zs[sl] = z;
     __syncthreads();
@@ -125,10 +144,7 @@ __global__ void __launch_bounds__(kReduceThreads) split_reduce_kernel(const Redu
             t.x += u.x; t.y += u.y; t.z += u.z; t.w += u.w;
         }
         const float wa = (la == -INFINITY) ? 0.f : __expf(la - m);
-        if (wa != 0.f) {
-            const float4 v = *reinterpret_cast<const float4*>(p.acc_o + int64_t(wid) * dv + cg * 4);
-            t.x += wa * v.x; t.y += wa * v.y; t.z += wa * v.z; t.w += wa * v.w;
-        }
+        if (wa != 0.f) { t.x += wa * fold.x; t.y += wa * fold.y; t.z += wa * fold.z; t.w += wa * fold.w; }
         float zt = wa;
         for (int k = 0; k < SL; ++k) zt += s_zs[k];      // fixed order: results are reproducible bit for bit
         const float inv = 1.f / zt;
@@ -194,9 +210,8 @@ cudaError_t launch_split_reduce(const AttnLaunch& a, cudaStream_t s) {
     p.G = a.kind == 1 ? a.n_q_heads : a.n_q_heads / a.n_kv_heads;
     p.n_hg = (p.G + 15) / 16;
     p.n_gh = pg.n_gh; p.RG = pg.rows_per_group; p.NW = pg.parts_per_span;
-    p.tags = a.steal_tags; p.n_tags = a.steal_tags ? a.n_ctas * kStealSlots : 0; p.n_spans = a.n_spans;
+    p.extra_count = a.steal_lists; p.extra_list = a.steal_lists ? a.steal_lists + a.n_rows * a.n_gh : nullptr; p.n_spans = a.n_spans;
     p.clear = a.steal_clear; p.clear_words = a.steal_clear ? a.steal_clear_words : 0;
-    if (p.n_tags > kMaxExtra) return cudaErrorInvalidValue;
     const size_t smem = size_t(kReduceThreads) * sizeof(float4);
     split_reduce_kernel<<<total, kReduceThreads, smem, s>>>(p);
     return cudaGetLastError();
