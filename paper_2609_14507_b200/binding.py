@@ -16,7 +16,7 @@ GQA, MLA = 0, 1
 REGION_U, REGION_P, REGION_W = 0, 1, 2
 LAYOUT_PLAIN, LAYOUT_TILE = 0, 1
 FLAG_NO_HOST_U, FLAG_NO_HOST_P, FLAG_GROW_P = 1, 2, 4
-ATTEND_STATIC_SCHEDULE = 1
+ATTEND_STATIC_SCHEDULE, ATTEND_BALANCE = 1, 2
 OK = 0
 STATUS_NAMES = {0: "OK", 1: "EINVAL", 2: "ENOMEM", 3: "ERANGE", 4: "ESTATE", 5: "ECUDA", 6: "ETIMEOUT", 7: "EINTERNAL"}
 
@@ -254,9 +254,9 @@ class Cache:
         self._check(lib().ipkv_flush(self._h, layer, seq, _stream(stream)), "ipkv_flush")
 
     def attend_gpu(self, layer, seq_ids, q, o_part, lse_part, kv_splits=0, side_stream=None, stream=None,
-                   fold_o=None, fold_lse=None, static_schedule=False):
+                   fold_o=None, fold_lse=None, static_schedule=False, force_balance=False):
         ids, n = _ids(seq_ids)
-        opts = AttendOpts(kv_splits, ATTEND_STATIC_SCHEDULE if static_schedule else 0, _stream(side_stream) if side_stream is not None else None, _ptr(fold_o), _ptr(fold_lse))
+        opts = AttendOpts(kv_splits, (ATTEND_STATIC_SCHEDULE if static_schedule else 0) | (ATTEND_BALANCE if force_balance else 0), _stream(side_stream) if side_stream is not None else None, _ptr(fold_o), _ptr(fold_lse))
         self._check(lib().ipkv_attend_gpu(self._h, layer, ids, n, _ptr(q), C.byref(opts), _ptr(o_part), _ptr(lse_part),
                                           _stream(stream)), "ipkv_attend_gpu")
 

@@ -55,6 +55,8 @@ struct SeqState {
     std::vector<PRun> p_runs;
 };
 
+constexpr int kMinTilesPerCtaToBalance = 48;
+
 // Bytes of the partial buffers for n_spans spans.
 size_t partial_bytes(size_t n_spans, const PartGeom& pg, int dv) {
     const size_t rows = n_spans * size_t(pg.parts_per_span) * pg.rows_per_group;
@@ -667,7 +669,7 @@ void fill_launch(AttnLaunch* a, int kind, int Hq, int Hkv, int dqk, int dv, int 
 // One group of segments for all rows: attention + split reduce, folding into (out_o, out_lse) when `fold`.
 ipkv_status run_group(ipkv* h, const std::vector<std::vector<PlanSeg>>& rows, const char* const bases[kMaxBases],
                       const void* q, int kv_splits, const float* fold_o, const float* fold_lse, float* out_o, float* out_lse,
-                      cudaStream_t s, bool static_schedule = false) {
+                      cudaStream_t s, int schedule_flags = 0) {
     const ipkv_config& c = h->cfg;
     Plan plan;
     const PartGeom pg = part_geom(c.kind, c.n_q_heads, c.n_kv_heads);
@@ -675,7 +677,13 @@ ipkv_status run_group(ipkv* h, const std::vector<std::vector<PlanSeg>>& rows, co
     // dynamic balancing: every CTA may fill up to kStealSlots extra partials (GQA kernel; more than one CTA)
     const size_t n_lists = rows.size() * size_t(pg.n_gh) * (1 + kStealListCap);
     const size_t steal_words = n_lists + plan.spans.size() + 2 * size_t(plan.n_ctas());
-    const bool balance = !static_schedule && c.kind == IPKV_GQA && plan.n_ctas() > 1 && steal_words <= size_t(ipkv::kStealWords);
+    // balancing pays once the chunks are long enough (measured: from about 50 tiles per CTA the shorter attention
+    // kernel outweighs the longer split reduce, which has the extra partials to look at)
+    int64_t plan_tiles = 0;
+    for (int32_t t : plan.cta_tiles) plan_tiles += t;
+    const bool balance = !(schedule_flags & IPKV_ATTEND_STATIC_SCHEDULE) && c.kind == IPKV_GQA && plan.n_ctas() > 1 &&
+                         steal_words <= size_t(ipkv::kStealWords) &&
+                         ((schedule_flags & IPKV_ATTEND_BALANCE) || plan_tiles >= int64_t(kMinTilesPerCtaToBalance) * plan.n_ctas());
     const size_t extra = balance ? size_t(plan.n_ctas()) * kStealSlots : 0;
     ipkv_status rc = ensure_scratch(h, partial_bytes(plan.spans.size() + extra, pg, c.dim_v));
     if (rc != IPKV_OK) return rc;
@@ -1044,7 +1052,7 @@ ipkv_status ipkv_attend_gpu(ipkv_t* h, int32_t layer, const int32_t* seq_ids, in
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int kv_splits = opts ? opts->kv_splits : 0;
     if (kv_splits < 0) return fail(h, IPKV_EINVAL, "kv_splits must be >= 0");
-    const bool static_schedule = opts && (opts->flags & IPKV_ATTEND_STATIC_SCHEDULE);
+    const int static_schedule = opts ? opts->flags & (IPKV_ATTEND_STATIC_SCHEDULE | IPKV_ATTEND_BALANCE) : 0;
     cudaStream_t side = (opts && opts->side_stream) ? static_cast<cudaStream_t>(opts->side_stream) : h->side;
     DeviceGuard dev_guard(c.device);
     CU(h, dev_guard.error());
@@ -1174,7 +1182,7 @@ ipkv_status ipkv_attend_gpu_sparse(ipkv_t* h, int32_t layer, const int32_t* seq_
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int kv_splits = opts ? opts->kv_splits : 0;
     if (kv_splits < 0) return fail(h, IPKV_EINVAL, "kv_splits must be >= 0");
-    const bool static_schedule = opts && (opts->flags & IPKV_ATTEND_STATIC_SCHEDULE);
+    const int static_schedule = opts ? opts->flags & (IPKV_ATTEND_STATIC_SCHEDULE | IPKV_ATTEND_BALANCE) : 0;
     cudaStream_t side = (opts && opts->side_stream) ? static_cast<cudaStream_t>(opts->side_stream) : h->side;
     const float* fold_o = opts ? opts->fold_o_dev : nullptr;
     const float* fold_lse = opts ? opts->fold_lse_dev : nullptr;

@@ -495,7 +495,7 @@ def test_static_schedule_is_bit_reproducible_and_dynamic_agrees():
 
         def run(static):
             o = torch.zeros((n_seq, 32, 128), device=DEV); lse = torch.zeros((n_seq, 32), device=DEV)
-            cache.attend_gpu(0, seqs, qd, o, lse, static_schedule=static)
+            cache.attend_gpu(0, seqs, qd, o, lse, static_schedule=static, force_balance=not static)
             torch.cuda.synchronize()
             return o.cpu().numpy(), lse.cpu().numpy()
 
@@ -510,4 +510,42 @@ def test_static_schedule_is_bit_reproducible_and_dynamic_agrees():
             o_ref, l_ref = c_oracle.attend(q[s], ks[s], vs[s], np.arange(ks[s].shape[0]), scale)
             check_partial(o_d[s], l_d[s], o_ref, l_ref, f"dynamic schedule, sequence {s}")
             check_partial(o_s1[s], l_s1[s], o_ref, l_ref, f"static schedule, sequence {s}")
+        assert cache.get_stats()["device_status"] == 0
+
+
+@pytest.mark.parametrize("G,dim", [(8, 128), (4, 128), (16, 64), (2, 64)])
+def test_balanced_schedule_on_ragged_multi_run_rows(G, dim):
+    """The dynamically balanced kernel on rows made of several runs (ring wrap + window), ragged lengths, tails that
+    are not multiples of a tile, group sizes with and without the duplicated-row trick, both head dims: every output
+    against the oracle, and a second launch (the other set of scheduling words) gives the same answer."""
+    hkv = 2
+    sh = synth.Shape("mix", "gqa", 1, hkv * G, hkv, dim, dim, dim ** -0.5)
+    lens = [3000, 777, 64, 1, 4097, 2500, 0, 1999]
+    scale = float(np.float32(sh.scale))
+    with make_cache(sh, 1, len(lens), block_tokens=16, window_tokens=64, chunk_tokens=256, max_u_tokens_per_seq=64,
+                    max_p_tokens_per_seq=4608, resident_tokens_per_seq=4608, share_num=0, share_den=1,
+                    flags=binding.FLAG_NO_HOST_U | binding.FLAG_NO_HOST_P) as cache:
+        rng = np.random.default_rng(4242)
+        ks, vs = [], []
+        for s, n in enumerate(lens):
+            k, v = synth.host_kv(sh, n, seed=9300 + s)
+            cache.append_bulk(0, s, synth.bits_to_torch(k, DEV) if n else None, synth.bits_to_torch(v, DEV) if n else None, n, 0, 1)
+            ks.append(k); vs.append(v)
+        seqs = list(range(len(lens)))
+        for step in range(70):                               # decode steps: a flush after 64, so rows get a window run too
+            k = synth.normal_bf16(rng, (len(lens), hkv, dim)); v = synth.normal_bf16(rng, (len(lens), hkv, dim))
+            cache.append(0, seqs, synth.bits_to_torch(k, DEV), synth.bits_to_torch(v, DEV))
+            for s in seqs:
+                ks[s] = np.concatenate([ks[s], k[s:s + 1]]); vs[s] = np.concatenate([vs[s], v[s:s + 1]])
+        q = synth.host_q(sh, len(lens), seed=9400)
+        outs = []
+        for _ in range(2):
+            o = torch.zeros((len(lens), hkv * G, dim), device=DEV); lse = torch.zeros((len(lens), hkv * G), device=DEV)
+            cache.attend_gpu(0, seqs, synth.bits_to_torch(q, DEV), o, lse, force_balance=True)
+            torch.cuda.synchronize()
+            outs.append((o.cpu().numpy(), lse.cpu().numpy()))
+        for s in seqs:
+            o_ref, l_ref = c_oracle.attend(q[s], ks[s], vs[s], np.arange(ks[s].shape[0]), scale)
+            check_partial(outs[1][0][s], outs[1][1][s], o_ref, l_ref, f"sequence {s}")
+        assert np.abs(outs[0][0] - outs[1][0]).max() < 2e-5
         assert cache.get_stats()["device_status"] == 0
