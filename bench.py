@@ -344,6 +344,8 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--kv-splits", type=int, default=0)
+    ap.add_argument("--profile-reduce", action="store_true",
+                    help="diagnostic: the kernel timed by CUDA events is the split reduce, not the attention kernel (the roofline object is then meaningless)")
     ap.add_argument("--static-schedule", action="store_true",
                     help="fixed tile assignment in the grouped-query kernel (bit-reproducible) instead of dynamic balancing")
     ap.add_argument("--separate-merge", action="store_true",
@@ -428,7 +430,7 @@ def main():
         step()
     barrier()
     st0 = cache.get_stats()
-    cache.profile_enable(True)
+    cache.profile_enable(True, reduce=args.profile_reduce)
     cache.profile_read()
     sampler.mark()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)

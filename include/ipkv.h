@@ -281,7 +281,7 @@ ipkv_status ipkv_policy_prefill_share(const ipkv_policy_t* p, double L0, int32_t
  * bracketed by a pair of CUDA events on the launching stream.  ipkv_profile_read synchronises the device,
  * returns the summed kernel time (milliseconds) and the number of launches since the last read, and resets
  * both.  At most 8192 launches are kept between two reads; later ones are counted but not timed. */
-ipkv_status ipkv_profile_enable(ipkv_t* h, int32_t on);
+ipkv_status ipkv_profile_enable(ipkv_t* h, int32_t on);   /* 0 off, 1 attention kernels, 2 split-reduce kernels instead */
 ipkv_status ipkv_profile_read(ipkv_t* h, double* attend_kernel_ms, int64_t* n_timed, int64_t* n_launches);
 
 /* ---- stateless kernel entry points (no handle) ------------------------------------------------- */

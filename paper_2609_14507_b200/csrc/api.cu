@@ -162,6 +162,7 @@ struct ipkv {
     std::string err;
     // optional kernel timing
     bool prof_on = false;
+    bool prof_reduce = false;              // time the split reduce instead of the attention kernel
     std::vector<cudaEvent_t> prof_ev;      // pairs
     size_t prof_used = 0;                  // events used
     int64_t prof_launches = 0;
@@ -710,14 +711,19 @@ ipkv_status run_group(ipkv* h, const std::vector<std::vector<PlanSeg>>& rows, co
     a.out_o = out_o; a.out_lse = out_lse;
     a.status = h->status_dev;
     if (a.n_spans > 0) {
-        const bool timed = h->prof_on && h->prof_used + 2 <= h->prof_ev.size();
+        const bool timed = h->prof_on && !h->prof_reduce && h->prof_used + 2 <= h->prof_ev.size();
         if (timed) CU(h, cudaEventRecord(h->prof_ev[h->prof_used], s));
         CU(h, launch_attend(a, s));
         if (timed) { CU(h, cudaEventRecord(h->prof_ev[h->prof_used + 1], s)); h->prof_used += 2; }
         if (h->prof_on) h->prof_launches += 1;
         h->stats.attend_kernels += 1;
     }
-    CU(h, launch_split_reduce(a, s));
+    {
+        const bool timed = h->prof_on && h->prof_reduce && h->prof_used + 2 <= h->prof_ev.size();
+        if (timed) CU(h, cudaEventRecord(h->prof_ev[h->prof_used], s));
+        CU(h, launch_split_reduce(a, s));
+        if (timed) { CU(h, cudaEventRecord(h->prof_ev[h->prof_used + 1], s)); h->prof_used += 2; }
+    }
     h->stats.reduce_kernels += 1;
     h->stats.kv_bytes_attended += uint64_t(plan.total_tokens) * uint64_t(h->bb / c.block_tokens);
     return IPKV_OK;
@@ -1521,6 +1527,7 @@ ipkv_status ipkv_profile_enable(ipkv_t* h, int32_t on) {
         for (auto& e : h->prof_ev) CU(h, cudaEventCreate(&e));
     }
     h->prof_on = on != 0;
+    h->prof_reduce = on == 2;
     return IPKV_OK;
 }
 

@@ -37,7 +37,7 @@ struct ReduceParams {
     int clear_words;
 };
 
-__global__ void __launch_bounds__(kReduceThreads) split_reduce_kernel(const ReduceParams p) {
+__global__ void __launch_bounds__(kReduceThreads, 4) split_reduce_kernel(const ReduceParams p) {
     extern __shared__ float4 red[];                 // [SL][CG]
     __shared__ float s_warp[kReduceThreads / 32];
     __shared__ float s_w[kLseCache];               // LSE of the first entries
@@ -49,21 +49,24 @@ __global__ void __launch_bounds__(kReduceThreads) split_reduce_kernel(const Redu
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = h / p.G, hin = h - g * p.G;
     const int gh = g * p.n_hg + hin / 16, rin = hin % 16;
-    const int sp0 = p.rg_span_start[row * p.n_gh + gh], sp1 = p.rg_span_start[row * p.n_gh + gh + 1];
-    const int64_t e0 = int64_t(sp0) * p.NW;
-    const int n_own = (sp1 - sp0) * p.NW;
-    const int dv = p.dv;
+    // the list of extra partials is requested together with the span range: one round of latency for both
+    const int rg = row * p.n_gh + gh;
+    const int sp0 = p.rg_span_start[rg], sp1 = p.rg_span_start[rg + 1];
+    int list_entry = 0, list_count = 0;
+    if (p.extra_count) {
+        if (tid < kStealListCap) list_entry = p.extra_list[rg * kStealListCap + tid];
+        if (tid == kStealListCap) list_count = min(p.extra_count[rg], kStealListCap);
+    }
     const float la = p.acc_lse ? p.acc_lse[wid] : -INFINITY;
     for (int i = blockIdx.x * kReduceThreads + tid; i < p.clear_words; i += gridDim.x * kReduceThreads) p.clear[i] = 0;
-    if (p.extra_count) {
-        const int rg = row * p.n_gh + gh;
-        if (tid < kStealListCap) s_extra[tid] = p.extra_list[rg * kStealListCap + tid];
-        if (tid == kStealListCap) s_n_extra = min(p.extra_count[rg], kStealListCap);
-    } else if (tid == 0) {
-        s_n_extra = 0;
-    }
+    if (tid < kStealListCap) s_extra[tid] = list_entry;
+    if (tid == kStealListCap) s_n_extra = list_count;
     __syncthreads();
-    const int n = n_own + s_n_extra * p.NW;
+    const int64_t e0 = int64_t(sp0) * p.NW;
+    const int n_own = (sp1 - sp0) * p.NW;
+    const int n_x = s_n_extra * p.NW;               // entries of the extra partials
+    const int n = n_own + n_x;
+    const int dv = p.dv;
     // entry e of this (row, head group): the spans' own partials first, then the extra ones
     auto entry = [&](int e) -> int64_t {
         if (e < n_own) return e0 + e;
@@ -76,14 +79,19 @@ __global__ void __launch_bounds__(kReduceThreads) split_reduce_kernel(const Redu
     const float* po = p.part_o + int64_t(rin) * dv + cg * 4;
     const int64_t stride = int64_t(p.RG) * dv;
 
-    // The partial outputs of this thread's first entries are requested before anything is known about their
-    // weights, so that their latency overlaps the two passes over the LSE values (an entry that turns out to be
-    // empty may hold anything: it is loaded but never used).
-    float4 pre[kPrefetch];
+    // The partial outputs of this thread's first entries (own and extra) are requested before anything is known about
+    // their weights, so that their latency overlaps the two passes over the LSE values (an entry that turns out to
+    // be empty may hold anything: it is loaded but never used).
+    float4 pre[kPrefetch], prx[kPrefetch];
 #pragma unroll
     for (int j = 0; j < kPrefetch; ++j) {
         const int e = sl + j * SL;
-        pre[j] = e < n ? *reinterpret_cast<const float4*>(po + entry(e) * stride) : make_float4(0.f, 0.f, 0.f, 0.f);
+        pre[j] = e < n_own ? *reinterpret_cast<const float4*>(po + (e0 + e) * stride) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int j = 0; j < kPrefetch; ++j) {
+        const int x = sl + j * SL;
+        prx[j] = x < n_x ? *reinterpret_cast<const float4*>(po + entry(n_own + x) * stride) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
     float4 fold = make_float4(0.f, 0.f, 0.f, 0.f);
     if (p.acc_o && sl == 0) fold = *reinterpret_cast<const float4*>(p.acc_o + int64_t(wid) * dv + cg * 4);
@@ -117,21 +125,27 @@ __global__ void __launch_bounds__(kReduceThreads) split_reduce_kernel(const Redu
     };
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float z = 0.f;
+    auto add = [&](float w, const float4& v) {
+        if (w != 0.f) { acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w; z += w; }
+    };
+    // own entries, then extra ones; in each group the prefetched ones first, the rest loaded only if they count
 #pragma unroll
     for (int j = 0; j < kPrefetch; ++j) {
         const int e = sl + j * SL;
-        const float w = e < n ? weight(e) : 0.f;
-        if (w != 0.f) {
-            acc.x += w * pre[j].x; acc.y += w * pre[j].y; acc.z += w * pre[j].z; acc.w += w * pre[j].w;
-            z += w;
-        }
+        add(e < n_own ? weight(e) : 0.f, pre[j]);
     }
-    for (int e = sl + kPrefetch * SL; e < n; e += SL) {
+    for (int e = sl + kPrefetch * SL; e < n_own; e += SL) {
         const float w = weight(e);
-        if (w == 0.f) continue;                     // a warp that saw no valid token
-        const float4 v = *reinterpret_cast<const float4*>(po + entry(e) * stride);
-        acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
-        z += w;
+        if (w != 0.f) add(w, *reinterpret_cast<const float4*>(po + (e0 + e) * stride));
+    }
+#pragma unroll
+    for (int j = 0; j < kPrefetch; ++j) {
+        const int x = sl + j * SL;
+        add(x < n_x ? weight(n_own + x) : 0.f, prx[j]);
+    }
+    for (int x = sl + kPrefetch * SL; x < n_x; x += SL) {
+        const float w = weight(n_own + x);
+        if (w != 0.f) add(w, *reinterpret_cast<const float4*>(po + entry(n_own + x) * stride));
     }
     red[sl * CG + cg] = acc;
     // every thread of a slice holds the same weight sum z; column group 0 publishes it
