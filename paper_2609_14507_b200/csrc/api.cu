@@ -675,7 +675,7 @@ ipkv_status run_group(ipkv* h, const std::vector<std::vector<PlanSeg>>& rows, co
     Plan plan;
     const PartGeom pg = part_geom(c.kind, c.n_q_heads, c.n_kv_heads);
     build_plan(rows, pg.n_gh, kv_splits, pg.ctas_per_sm, &plan);
-    // dynamic balancing: every CTA may fill up to kStealSlots extra partials (GQA kernel; more than one CTA)
+    // dynamic balancing (grouped-query kernel): every CTA may fill up to kStealSlots extra partials
     const size_t n_lists = rows.size() * size_t(pg.n_gh) * (1 + kStealListCap);
     const size_t steal_words = n_lists + plan.spans.size() + 2 * size_t(plan.n_ctas());
     // balancing pays once the chunks are long enough (measured: from about 50 tiles per CTA the shorter attention
