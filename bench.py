@@ -547,7 +547,7 @@ def main():
                        "cpu_share": f"{num0}/{den0}", "gpu_share_tokens_per_seq_mean": n_gpu0 + 1, "bytes_per_kv_token": bpt, "block_tokens": BLOCK, "window_tokens": wl.get("window", WINDOW),
                        "gpu_share": "HBM-resident", "host_copies_of_U_and_P": "off (benchmark)", "cpu_partial": "synthetic values",
                        "l2": l2_note,
-                       "multi_gpu": "replicas only", "kv_splits": args.kv_splits, "schedule": "static" if args.static_schedule else "dynamic balancing (GQA kernel)",
+                       "multi_gpu": "replicas only", "kv_splits": args.kv_splits, "schedule": "static" if args.static_schedule else "dynamic balancing (GQA kernel, launches of at least 48 tiles per CTA)",
                        "merge": "inside the split reduce" if fused else "separate ipkv_merge launch"},
             "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu,
             "step_gbs": bytes_all / (ms * 1e-3) / 1e9,

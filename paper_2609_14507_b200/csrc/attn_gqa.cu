@@ -244,6 +244,35 @@ __global__ void __launch_bounds__(kThreads) attn_gqa_kernel(const GqaParams p) {
         }
     };
 
+    // start a partial: query fragments of its head group straight from global memory (a few KB, L2-resident), empty state
+    auto begin_partial = [&](int q_row, int nh) {
+        n_heads = nh;
+        const __nv_bfloat16* qrow0 = p.q + (int64_t(q_row) + r0) * D + c0;
+        const bool v0 = r0 < n_heads, v1 = !DUP && (r0 + 8 < n_heads);
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks) {
+            const uint32_t x0 = v0 ? __ldg(reinterpret_cast<const uint32_t*>(qrow0 + ks * 16)) : 0u;
+            const uint32_t x2 = v0 ? __ldg(reinterpret_cast<const uint32_t*>(qrow0 + ks * 16 + 8)) : 0u;
+            qa[ks][0] = x0; qa[ks][2] = x2;
+            if (DUP) { qa[ks][1] = x0; qa[ks][3] = x2; }
+            else {
+                qa[ks][1] = v1 ? __ldg(reinterpret_cast<const uint32_t*>(qrow0 + 8 * D + ks * 16)) : 0u;
+                qa[ks][3] = v1 ? __ldg(reinterpret_cast<const uint32_t*>(qrow0 + 8 * D + ks * 16 + 8)) : 0u;
+            }
+        }
+#pragma unroll
+        for (int nt = 0; nt < D / 8; ++nt) { o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f; }
+        m0 = m1 = -INFINITY; l0 = l1 = 0.f;
+    };
+    // The first tiles are almost always those of the CTA's own first span: its query fragments are fetched while the
+    // first copies are in flight. (If another partial comes first, this one is written out empty, which is what it is.)
+    if (span_begin < span_end) {
+        const Span first = p.spans[span_begin];
+        const int g = first.gh / p.n_hg, hg = first.gh - g * p.n_hg;
+        cur_slot = span_begin;
+        begin_partial(first.row * p.Hq + g * p.G + hg * 16, min(16, p.G - hg * 16));
+    }
+
     for (;; ++it) {
         const int st = it % STAGES;
         if (!ptx::mbar_wait(s_full + 8 * st, (it / STAGES) & 1)) { ok = false; break; }   // after a timeout: give up
@@ -252,24 +281,7 @@ __global__ void __launch_bounds__(kThreads) attn_gqa_kernel(const GqaParams p) {
             if (cur_slot != kEndSlot) flush();
             if (slot == kEndSlot) break;
             cur_slot = slot;
-            n_heads = s_meta[st].n_heads;
-            // query fragments straight from global memory (a few KB per span, L2-resident)
-            const __nv_bfloat16* qrow0 = p.q + (int64_t(s_meta[st].q_row) + r0) * D + c0;
-            const bool v0 = r0 < n_heads, v1 = !DUP && (r0 + 8 < n_heads);
-#pragma unroll
-            for (int ks = 0; ks < D / 16; ++ks) {
-                const uint32_t x0 = v0 ? __ldg(reinterpret_cast<const uint32_t*>(qrow0 + ks * 16)) : 0u;
-                const uint32_t x2 = v0 ? __ldg(reinterpret_cast<const uint32_t*>(qrow0 + ks * 16 + 8)) : 0u;
-                qa[ks][0] = x0; qa[ks][2] = x2;
-                if (DUP) { qa[ks][1] = x0; qa[ks][3] = x2; }
-                else {
-                    qa[ks][1] = v1 ? __ldg(reinterpret_cast<const uint32_t*>(qrow0 + 8 * D + ks * 16)) : 0u;
-                    qa[ks][3] = v1 ? __ldg(reinterpret_cast<const uint32_t*>(qrow0 + 8 * D + ks * 16 + 8)) : 0u;
-                }
-            }
-#pragma unroll
-            for (int nt = 0; nt < D / 8; ++nt) { o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f; }
-            m0 = m1 = -INFINITY; l0 = l1 = 0.f;
+            begin_partial(s_meta[st].q_row, s_meta[st].n_heads);
         }
         const int n_valid = s_meta[st].n_valid;
         {

@@ -14,7 +14,7 @@ namespace {
 
 constexpr int kWarpsPerBlock = 4;
 constexpr int kReduceThreads = 256;
-constexpr int kPrefetch = 4;       // partial outputs per thread requested up front
+constexpr int kPrefetch = 2;       // partial outputs per thread requested up front (of the own and of the extra partials)
 constexpr int kLseCache = 512;     // LSE values kept in shared memory between the two passes
 
 // One CTA per (row, query head). The partials to join are those of the spans of the head's group
@@ -37,7 +37,10 @@ struct ReduceParams {
     int clear_words;
 };
 
-__global__ void __launch_bounds__(kReduceThreads, 4) split_reduce_kernel(const ReduceParams p) {
+// EXTRAS: the launch was dynamically balanced and may have extra partials (kept out of the plain instantiation, which
+// then needs few enough registers for five CTAs per SM: launches with thousands of (row, head) pairs run in fewer waves).
+template <bool EXTRAS>
+__global__ void __launch_bounds__(kReduceThreads, EXTRAS ? 4 : 5) split_reduce_kernel(const ReduceParams p) {
     extern __shared__ float4 red[];                 // [SL][CG]
     __shared__ float s_warp[kReduceThreads / 32];
     __shared__ float s_w[kLseCache];               // LSE of the first entries
@@ -53,7 +56,7 @@ __global__ void __launch_bounds__(kReduceThreads, 4) split_reduce_kernel(const R
     const int rg = row * p.n_gh + gh;
     const int sp0 = p.rg_span_start[rg], sp1 = p.rg_span_start[rg + 1];
     int list_entry = 0, list_count = 0;
-    if (p.extra_count) {
+    if (EXTRAS) {
         if (tid < kStealListCap) list_entry = p.extra_list[rg * kStealListCap + tid];
         if (tid == kStealListCap) list_count = min(p.extra_count[rg], kStealListCap);
     }
@@ -64,7 +67,7 @@ __global__ void __launch_bounds__(kReduceThreads, 4) split_reduce_kernel(const R
     __syncthreads();
     const int64_t e0 = int64_t(sp0) * p.NW;
     const int n_own = (sp1 - sp0) * p.NW;
-    const int n_x = s_n_extra * p.NW;               // entries of the extra partials
+    const int n_x = EXTRAS ? s_n_extra * p.NW : 0;  // entries of the extra partials
     const int n = n_own + n_x;
     const int dv = p.dv;
     // entry e of this (row, head group): the spans' own partials first, then the extra ones
@@ -82,14 +85,15 @@ __global__ void __launch_bounds__(kReduceThreads, 4) split_reduce_kernel(const R
     // The partial outputs of this thread's first entries (own and extra) are requested before anything is known about
     // their weights, so that their latency overlaps the two passes over the LSE values (an entry that turns out to
     // be empty may hold anything: it is loaded but never used).
-    float4 pre[kPrefetch], prx[kPrefetch];
+    constexpr int kPrefetchX = EXTRAS ? kPrefetch : 1;
+    float4 pre[kPrefetch], prx[kPrefetchX];
 #pragma unroll
     for (int j = 0; j < kPrefetch; ++j) {
         const int e = sl + j * SL;
         pre[j] = e < n_own ? *reinterpret_cast<const float4*>(po + (e0 + e) * stride) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
 #pragma unroll
-    for (int j = 0; j < kPrefetch; ++j) {
+    for (int j = 0; j < kPrefetchX; ++j) {
         const int x = sl + j * SL;
         prx[j] = x < n_x ? *reinterpret_cast<const float4*>(po + entry(n_own + x) * stride) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
@@ -139,11 +143,11 @@ __global__ void __launch_bounds__(kReduceThreads, 4) split_reduce_kernel(const R
         if (w != 0.f) add(w, *reinterpret_cast<const float4*>(po + (e0 + e) * stride));
     }
 #pragma unroll
-    for (int j = 0; j < kPrefetch; ++j) {
+    for (int j = 0; j < kPrefetchX; ++j) {
         const int x = sl + j * SL;
         add(x < n_x ? weight(n_own + x) : 0.f, prx[j]);
     }
-    for (int x = sl + kPrefetch * SL; x < n_x; x += SL) {
+    for (int x = sl + kPrefetchX * SL; x < n_x; x += SL) {
         const float w = weight(n_own + x);
         if (w != 0.f) add(w, *reinterpret_cast<const float4*>(po + entry(n_own + x) * stride));
     }
@@ -227,7 +231,8 @@ cudaError_t launch_split_reduce(const AttnLaunch& a, cudaStream_t s) {
     p.extra_count = a.steal_lists; p.extra_list = a.steal_lists ? a.steal_lists + a.n_rows * a.n_gh : nullptr; p.n_spans = a.n_spans;
     p.clear = a.steal_clear; p.clear_words = a.steal_clear ? a.steal_clear_words : 0;
     const size_t smem = size_t(kReduceThreads) * sizeof(float4);
-    split_reduce_kernel<<<total, kReduceThreads, smem, s>>>(p);
+    if (p.extra_count) split_reduce_kernel<true><<<total, kReduceThreads, smem, s>>>(p);
+    else split_reduce_kernel<false><<<total, kReduceThreads, smem, s>>>(p);
     return cudaGetLastError();
 }
 
