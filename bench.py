@@ -344,6 +344,7 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--kv-splits", type=int, default=0)
+    ap.add_argument("--no-read-ceiling", action="store_true", help="skip the read-only bandwidth probe reported in roofline.read_ceiling")
     ap.add_argument("--profile-reduce", action="store_true",
                     help="diagnostic: the kernel timed by CUDA events is the split reduce, not the attention kernel (the roofline object is then meaningless)")
     ap.add_argument("--static-schedule", action="store_true",
@@ -472,6 +473,15 @@ def main():
                 "avg_launch_us": 1e3 * kern_ms / max(1, n_timed), "bytes_per_launch": bytes_attended / max(1, n_launch),
                 "traffic": None, "whole_step_gbs": bytes_all / (ms * 1e-3) / 1e9}
     roofline["traffic"] = DRAM_TRAFFIC_PER_LAUNCH.get(args.workload)
+    if rank == 0 and world == 1 and not args.no_read_ceiling:
+        # context for the fraction above: what a pure read of one launch's bytes through the same copy ring reaches
+        try:
+            torch.cuda.synchronize()
+            best, mean = binding.ipkv_probe_read_bandwidth(local_rank, max(256 << 20, int(bytes_attended / max(1, n_launch))), 10)
+            roofline["read_ceiling"] = {"best": best, "mean": mean, "unit": "GB/s", "frac_of_best": ach / best if best > 0 else None,
+                                        "what": "read-only stream through the kernels' copy ring, no arithmetic, same bytes as one launch"}
+        except binding.IpkvError as e:                    # e.g. no memory left for the probe's buffers
+            roofline["read_ceiling"] = {"error": str(e)}
 
     # ---- end to end: host buffers in, host buffer out, through the same calls ---------------------------------
     e2e = None

@@ -284,6 +284,13 @@ ipkv_status ipkv_policy_prefill_share(const ipkv_policy_t* p, double L0, int32_t
 ipkv_status ipkv_profile_enable(ipkv_t* h, int32_t on);   /* 0 off, 1 attention kernels, 2 split-reduce kernels instead */
 ipkv_status ipkv_profile_read(ipkv_t* h, double* attend_kernel_ms, int64_t* n_timed, int64_t* n_launches);
 
+/* Measurement aid (no counterpart in the paper): the rate, in GB/s, at which the SMs of `device` read `bytes` bytes
+ * (>= 64 MB; use more than the L2 holds) of freshly allocated device memory through the same bulk-copy / mbarrier ring
+ * the attention kernels use, with no arithmetic.  Decode attention only reads the KV bytes, a copy reads and writes
+ * them: this is the read-only ceiling shown beside the copy bandwidth.  Allocates 2 x bytes for the duration of the
+ * call, runs 3 warm-up and `reps` timed launches (CUDA events), returns the best and the mean. */
+ipkv_status ipkv_probe_read_bandwidth(int32_t device, size_t bytes, int32_t reps, double* best_gbs, double* mean_gbs);
+
 /* ---- stateless kernel entry points (no handle) ------------------------------------------------- */
 
 typedef struct {

@@ -26,7 +26,7 @@ EXPORTS = [
     "ipkv_read_token", "ipkv_get_stats", "ipkv_profile_enable", "ipkv_profile_read", "ipkv_attend_scratch_bytes", "ipkv_attend_runs", "ipkv_pack_blocks",
     "ipkv_attend_runs_noalloc", "ipkv_noalloc_scratch_limit", "ipkv_roofline_share", "ipkv_roofline_step_time",
     "ipkv_policy_create", "ipkv_policy_destroy", "ipkv_policy_observe", "ipkv_policy_update", "ipkv_policy_prefill_share",
-    "ipkv_block_bytes", "ipkv_status_str", "ipkv_last_error", "ipkv_version",
+    "ipkv_block_bytes", "ipkv_status_str", "ipkv_last_error", "ipkv_version", "ipkv_probe_read_bandwidth",
 ]
 
 
@@ -194,6 +194,16 @@ def make_config(kind, n_layers, max_seqs, n_q_heads, n_kv_heads, dim_qk, dim_v, 
     c.softmax_scale = softmax_scale
     c.share_num, c.share_den, c.device, c.flags = share_num, share_den, device, flags
     return c
+
+
+def ipkv_probe_read_bandwidth(device=0, nbytes=1 << 30, reps=10):
+    """(best, mean) GB/s of a read-only stream through the attention kernels' copy ring, no arithmetic."""
+    best, mean = C.c_double(), C.c_double()
+    lib().ipkv_probe_read_bandwidth.argtypes = [C.c_int32, C.c_size_t, C.c_int32, C.POINTER(C.c_double), C.POINTER(C.c_double)]
+    rc = lib().ipkv_probe_read_bandwidth(device, nbytes, reps, C.byref(best), C.byref(mean))
+    if rc != OK:
+        raise IpkvError(rc, "ipkv_probe_read_bandwidth")
+    return best.value, mean.value
 
 
 def ipkv_query_sizes(cfg):

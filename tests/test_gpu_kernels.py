@@ -195,3 +195,11 @@ def test_mla_tcgen05_variant_matches_oracle():
     r = subprocess.run([sys.executable, "-m", "pytest", "-q", "-m", "gpu", "-x", os.path.join(root, "tests", "test_gpu_kernels.py"),
                         "-k", "attend_runs_mla"], env=env, cwd=root, capture_output=True, text=True, timeout=600)
     assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
+
+
+def test_read_bandwidth_probe_runs():
+    """The measurement aid behind `roofline.read_ceiling`: a read-only stream through the kernels' copy ring."""
+    best, mean = binding.ipkv_probe_read_bandwidth(0, 256 << 20, 3)
+    assert 500.0 < mean <= best < 20000.0
+    with pytest.raises(binding.IpkvError):
+        binding.ipkv_probe_read_bandwidth(0, 1 << 20, 3)          # below the 64 MB minimum
