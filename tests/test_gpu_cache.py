@@ -549,3 +549,36 @@ def test_balanced_schedule_on_ragged_multi_run_rows(G, dim):
             check_partial(outs[1][0][s], outs[1][1][s], o_ref, l_ref, f"sequence {s}")
         assert np.abs(outs[0][0] - outs[1][0]).max() < 2e-5
         assert cache.get_stats()["device_status"] == 0
+
+
+def test_balanced_launches_of_changing_shape_stay_consistent():
+    """Back-to-back balanced launches whose plans differ (other row subsets, other split counts, growing windows): the
+    two sets of scheduling words are reused with different layouts every time, and each launch relies on the previous
+    one's reduce having zeroed its set.  Every result must match the fixed schedule of the same call."""
+    sh = synth.Shape("mid", "gqa", 1, 16, 4, 128, 128, 128 ** -0.5)
+    lens = [5000, 3100, 4096, 1500, 2800, 900, 4700, 3900]
+    with make_cache(sh, 1, len(lens), block_tokens=64, window_tokens=128, chunk_tokens=512, max_u_tokens_per_seq=64,
+                    max_p_tokens_per_seq=6144, resident_tokens_per_seq=6144,
+                    flags=binding.FLAG_NO_HOST_U | binding.FLAG_NO_HOST_P) as cache:
+        rng = np.random.default_rng(808)
+        for s, n in enumerate(lens):
+            k, v = synth.host_kv(sh, n, seed=9500 + s)
+            cache.append_bulk(0, s, synth.bits_to_torch(k, DEV), synth.bits_to_torch(v, DEV), n, 0, 1)
+        all_seqs = list(range(len(lens)))
+        subsets = [all_seqs, [0, 2, 4, 6], all_seqs, [7], [1, 3, 5, 7, 0], all_seqs, [2, 6]]
+        for round_ in range(21):
+            k = synth.normal_bf16(rng, (len(lens), 4, 128)); v = synth.normal_bf16(rng, (len(lens), 4, 128))
+            cache.append(0, all_seqs, synth.bits_to_torch(k, DEV), synth.bits_to_torch(v, DEV))
+            seqs = subsets[round_ % len(subsets)]
+            splits = (0, 0, 3, 0, 7)[round_ % 5]
+            q = synth.normal_bf16(rng, (len(seqs), 16, 128))
+            qd = synth.bits_to_torch(q, DEV)
+            res = []
+            for static in (False, True):
+                o = torch.zeros((len(seqs), 16, 128), device=DEV); lse = torch.zeros((len(seqs), 16), device=DEV)
+                cache.attend_gpu(0, seqs, qd, o, lse, kv_splits=splits, static_schedule=static, force_balance=not static)
+                torch.cuda.synchronize()
+                res.append((o.cpu().numpy(), lse.cpu().numpy()))
+            assert np.abs(res[0][0] - res[1][0]).max() < 2e-5, round_
+            assert np.abs(res[0][1] - res[1][1]).max() < 2e-5, round_
+        assert cache.get_stats()["device_status"] == 0
