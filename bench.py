@@ -435,7 +435,7 @@ def main():
     cache.profile_read()
     sampler.mark()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)] if args.latency else None
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]       # one event per step: medians and tails
     e0.record()
     for i in range(args.steps):
         if marks:
@@ -447,10 +447,11 @@ def main():
     barrier()
     clocks = sampler.stop() if rank == 0 else None
     ms = max_over_ranks(e0.elapsed_time(e1))
+    raw = [marks[i].elapsed_time(marks[i + 1]) for i in range(args.steps)]
+    lat = sorted(raw)
+    step_ms = {"median": lat[len(lat) // 2], "best": lat[0]}
     step_lat = None
-    if marks:
-        raw = [marks[i].elapsed_time(marks[i + 1]) for i in range(args.steps)]
-        lat = sorted(raw)
+    if args.latency:
         slowest = sorted(range(args.steps), key=lambda i: -raw[i])[:4]
         p99 = lat[min(len(lat) - 1, int(0.99 * len(lat)))]
         step_lat = {"p50_ms": lat[len(lat) // 2], "p99_ms": p99, "max_ms": lat[-1], "p99_over_p50": p99 / lat[len(lat) // 2],
@@ -560,7 +561,7 @@ def main():
                        "multi_gpu": "replicas only", "kv_splits": args.kv_splits, "schedule": "static" if args.static_schedule else "dynamic balancing (GQA kernel, launches of at least 48 tiles per CTA)",
                        "merge": "inside the split reduce" if fused else "separate ipkv_merge launch"},
             "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu,
-            "step_gbs": bytes_all / (ms * 1e-3) / 1e9,
+            "step_gbs": bytes_all / (ms * 1e-3) / 1e9, "step_ms": step_ms,
         }
         if step_lat:
             line["step_latency"] = step_lat
