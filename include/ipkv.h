@@ -253,7 +253,8 @@ typedef struct {
      that was not pinned yet (0 when the one-window lookahead covers the pinning, as Sec. 7.7 expects).  */
   uint64_t p_segments, p_pinned_bytes, p_pin_us, p_grow_waits, p_grow_wait_us;
   uint64_t p_register_us, p_register_calls, p_register_max_us;  /* the page-locking calls alone: total, count, longest */
-  uint32_t device_status;       /* nonzero after a kernel's bounded wait gave up (synchronises)  */
+  uint32_t device_status;       /* nonzero after a kernel's bounded wait gave up (synchronises): bit 0 a producer
+                                   got no free stage, bit 1 a consumer got no tile, bit 2 a copy did not land  */
 } ipkv_stats;
 ipkv_status ipkv_get_stats(ipkv_t* h, ipkv_stats* out);
 

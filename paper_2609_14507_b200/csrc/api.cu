@@ -1514,7 +1514,14 @@ ipkv_status ipkv_get_stats(ipkv_t* h, ipkv_stats* out) {
         h->stats.p_register_max_us = h->p_register_max_us;
     }
     *out = h->stats;
-    return h->stats.device_status ? fail(h, IPKV_ETIMEOUT, "a kernel's bounded wait gave up; results of that call are invalid") : IPKV_OK;
+    if (h->stats.device_status) {
+        std::string where;
+        if (h->stats.device_status & kStatusNoFreeStage) where += " [a producer got no free stage]";
+        if (h->stats.device_status & kStatusNoTile) where += " [a consumer got no tile]";
+        if (h->stats.device_status & kStatusCopyNotLanded) where += " [a copy did not land]";
+        return fail(h, IPKV_ETIMEOUT, "a kernel's bounded wait gave up; results of that call are invalid" + where);
+    }
+    return IPKV_OK;
 }
 
 ipkv_status ipkv_profile_enable(ipkv_t* h, int32_t on) {

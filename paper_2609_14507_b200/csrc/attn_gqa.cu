@@ -167,10 +167,11 @@ __global__ void __launch_bounds__(kThreads) attn_gqa_kernel(const GqaParams p) {
             sched.lse_per_partial = kConsumerWarps * p.RG;
             ok = produce_tiles(sched, lane, issue);
             if (lane == 0) {
+                if (!ok) atomicOr(p.status, kStatusNoFreeStage);
                 // tell the consumers that nothing follows
                 if (ok) {
                     const int st = it % STAGES;
-                    if (it >= STAGES && !ptx::mbar_wait(s_empty + 8 * st, ((it / STAGES) - 1) & 1)) ok = false;
+                    if (it >= STAGES && !ptx::mbar_wait(s_empty + 8 * st, ((it / STAGES) - 1) & 1)) { ok = false; atomicOr(p.status, kStatusNoFreeStage); }
                     if (ok) {
                         s_meta[st].slot = kEndSlot;
                         ptx::mbar_expect_tx(s_full + 8 * st, 0);
@@ -180,8 +181,7 @@ __global__ void __launch_bounds__(kThreads) attn_gqa_kernel(const GqaParams p) {
                 // do not leave the CTA while copies of ours may still be in flight
                 const int first_pending = it > STAGES ? it - STAGES : 0;
                 for (int i = first_pending; i < it; ++i)
-                    if (!ptx::mbar_wait(s_full + 8 * (i % STAGES), (i / STAGES) & 1)) ok = false;
-                if (!ok) atomicOr(p.status, 1u);
+                    if (!ptx::mbar_wait(s_full + 8 * (i % STAGES), (i / STAGES) & 1)) atomicOr(p.status, kStatusCopyNotLanded);
             }
         }
         return;
@@ -371,7 +371,7 @@ __global__ void __launch_bounds__(kThreads) attn_gqa_kernel(const GqaParams p) {
             if (lane == 0) ptx::mbar_arrive(s_empty + 8 * st);
         }
     }
-    if (!ok && lane == 0) atomicOr(p.status, 1u);
+    if (!ok && lane == 0) atomicOr(p.status, kStatusNoTile);
 }
 
 template <int D, int STAGES, bool DUP>

@@ -144,7 +144,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_mla_kernel(const MlaParams p
             const int first_pending = it > kStages ? it - kStages : 0;
             for (int i = first_pending; i < it; ++i)
                 if (!ptx::mbar_wait(s_full + 8 * (i % kStages), (i / kStages) & 1)) ok = false;
-            if (!ok) atomicOr(p.status, 1u);
+            if (!ok) atomicOr(p.status, kStatusNoFreeStage | kStatusCopyNotLanded);
         }
         return;      // the consumers synchronise among themselves on a named barrier
     }
@@ -311,7 +311,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_mla_kernel(const MlaParams p
         }
         consumer_barrier();      // s_m / s_l / the query tile are reused by the next span
     }
-    if (!ok && lane == 0) atomicOr(p.status, 1u);
+    if (!ok && lane == 0) atomicOr(p.status, kStatusNoTile);
 }
 
 }  // namespace

@@ -22,6 +22,11 @@ struct Span {
 
 constexpr int kMaxBases = 4;
 
+// Bits of the device status word: which bounded wait of a kernel gave up.
+constexpr uint32_t kStatusNoFreeStage = 1u;     // the producer waited for the consumers to release a stage
+constexpr uint32_t kStatusNoTile = 2u;          // a consumer waited for a tile (or the end marker) to arrive
+constexpr uint32_t kStatusCopyNotLanded = 4u;   // the producer waited for its last copies before leaving
+
 struct AttnLaunch {
     int kind;                       // 0 = GQA, 1 = compressed latent (MLA)
     int n_q_heads, n_kv_heads, dim_qk, dim_v, bt;
