@@ -349,6 +349,8 @@ def main():
                     help="diagnostic: the kernel timed by CUDA events is the split reduce, not the attention kernel (the roofline object is then meaningless)")
     ap.add_argument("--static-schedule", action="store_true",
                     help="fixed tile assignment in the grouped-query kernel (bit-reproducible) instead of dynamic balancing")
+    ap.add_argument("--separate-append", action="store_true",
+                    help="ipkv_append as a call and a launch of its own instead of riding in ipkv_attend_gpu")
     ap.add_argument("--separate-merge", action="store_true",
                     help="join the CPU-side partial with a separate ipkv_merge launch instead of inside the split reduce")
     ap.add_argument("--latency", action="store_true", help="also time every step separately and report P50 / P99 / max")
@@ -406,12 +408,15 @@ def main():
 
     def step():
         for layer in range(NL):
-            cache.append(layer, seq_ids, k_new[layer], None if v_new is None else v_new[layer], stream=cur)
+            # the append rides in the attention call (the kernel writes the new rows where it can) unless --separate-append
+            app = {} if args.separate_append else dict(append_k=k_new[layer], append_v=None if v_new is None else v_new[layer])
+            if args.separate_append:
+                cache.append(layer, seq_ids, k_new[layer], None if v_new is None else v_new[layer], stream=cur)
             if fused:      # the CPU-side partial is joined inside the split reduce: out = merged (O, LSE)
                 cache.attend_gpu(layer, seq_ids, q[layer], out[layer], out_lse, kv_splits=args.kv_splits, static_schedule=args.static_schedule, stream=cur,
-                                 fold_o=o_cpu[layer], fold_lse=lse_cpu[layer])
+                                 fold_o=o_cpu[layer], fold_lse=lse_cpu[layer], **app)
             else:
-                cache.attend_gpu(layer, seq_ids, q[layer], o_part, lse_part, kv_splits=args.kv_splits, static_schedule=args.static_schedule, stream=cur)
+                cache.attend_gpu(layer, seq_ids, q[layer], o_part, lse_part, kv_splits=args.kv_splits, static_schedule=args.static_schedule, stream=cur, **app)
                 cache.merge(B * Hq, dv, [o_part.view(B * Hq, dv), o_cpu[layer]], [lse_part.view(-1), lse_cpu[layer]],
                             out[layer], out_lse, out_is_bf16=True, stream=cur)
 
@@ -504,12 +509,14 @@ def main():
             doc.copy_(hoc, non_blocking=True)
             dlc.copy_(hlc, non_blocking=True)
             for layer in range(NL):
-                cache.append(layer, seq_ids, dk[layer], None if dvn is None else dvn[layer], stream=cur)
+                app = {} if args.separate_append else dict(append_k=dk[layer], append_v=None if dvn is None else dvn[layer])
+                if args.separate_append:
+                    cache.append(layer, seq_ids, dk[layer], None if dvn is None else dvn[layer], stream=cur)
                 if fused:
                     cache.attend_gpu(layer, seq_ids, dq[layer], out[layer], out_lse, kv_splits=args.kv_splits, static_schedule=args.static_schedule, stream=cur,
-                                     fold_o=doc[layer], fold_lse=dlc[layer])
+                                     fold_o=doc[layer], fold_lse=dlc[layer], **app)
                 else:
-                    cache.attend_gpu(layer, seq_ids, dq[layer], o_part, lse_part, kv_splits=args.kv_splits, static_schedule=args.static_schedule, stream=cur)
+                    cache.attend_gpu(layer, seq_ids, dq[layer], o_part, lse_part, kv_splits=args.kv_splits, static_schedule=args.static_schedule, stream=cur, **app)
                     cache.merge(B * Hq, dv, [o_part.view(B * Hq, dv), doc[layer]], [lse_part.view(-1), dlc[layer]],
                                 out[layer], out_lse, out_is_bf16=True, stream=cur)
             hout.copy_(out, non_blocking=True)
@@ -559,7 +566,8 @@ def main():
                        "gpu_share": "HBM-resident", "host_copies_of_U_and_P": "off (benchmark)", "cpu_partial": "synthetic values",
                        "l2": l2_note,
                        "multi_gpu": "replicas only", "kv_splits": args.kv_splits, "schedule": "static" if args.static_schedule else "dynamic balancing (GQA kernel, launches of at least 48 tiles per CTA)",
-                       "merge": "inside the split reduce" if fused else "separate ipkv_merge launch"},
+                       "merge": "inside the split reduce" if fused else "separate ipkv_merge launch",
+                       "append": "separate ipkv_append" if args.separate_append else "inside ipkv_attend_gpu (written by the attention kernel for GQA)"},
             "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu,
             "step_gbs": bytes_all / (ms * 1e-3) / 1e9, "step_ms": step_ms,
         }

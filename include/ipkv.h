@@ -172,6 +172,14 @@ typedef struct {
      ipkv_merge launch is needed for this step (Sec. 4.2: one join per step, performed on the GPU).        */
   const float* fold_o_dev;
   const float* fold_lse_dev;
+  /* Optional fused decode append (ipkv_attend_gpu only): one new token for each listed sequence,
+     k [n_seq][n_kv_heads][dim_qk], v [n_seq][n_kv_heads][dim_v] (NULL for IPKV_MLA), appended exactly as ipkv_append
+     would (full windows are evicted first) and attended by the same call.  Where the kernel can, it writes the new
+     rows into the D-window itself (grouped-query caches with block_tokens >= 64: the warp that owns the token's slice
+     of the tile patches the tile in shared memory and stores the rows to the window), which saves the append launch of
+     every layer; otherwise the library launches its append kernel first.  The result is the same either way.   */
+  const void* append_k_dev;
+  const void* append_v_dev;
 } ipkv_attend_opts;
 
 /* Attention over the GPU-side share (Sec. 5.1): the D-window plus every P token, device-resident ones
@@ -248,6 +256,7 @@ typedef struct {
   uint64_t kv_bytes_attended;   /* tokens * bytes per token, summed over attend calls            */
   uint64_t h2d_bytes, d2h_bytes, d2d_bytes;
   uint64_t flushes, flushes_to_u;
+  uint64_t fused_appends;       /* ipkv_attend_gpu calls whose kernel wrote the appended rows itself     */
   /* IPKV_FLAG_GROW_P: segments pinned so far, their bytes, the page-locking time spent (by create for the
      first, by the helper thread for the rest), and how often / how long a call had to wait for a segment
      that was not pinned yet (0 when the one-window lookahead covers the pinning, as Sec. 7.7 expects).  */

@@ -47,7 +47,7 @@ class Config(C.Structure):
 
 class AttendOpts(C.Structure):
     _fields_ = [("kv_splits", C.c_int32), ("flags", C.c_int32), ("side_stream", C.c_void_p),
-                ("fold_o_dev", C.c_void_p), ("fold_lse_dev", C.c_void_p)]
+                ("fold_o_dev", C.c_void_p), ("fold_lse_dev", C.c_void_p), ("append_k_dev", C.c_void_p), ("append_v_dev", C.c_void_p)]
 
 
 class Extent(C.Structure):
@@ -58,7 +58,7 @@ class Extent(C.Structure):
 class Stats(C.Structure):
     _fields_ = [(n, C.c_uint64) for n in (
         "attend_calls", "attend_kernels", "reduce_kernels", "merge_kernels", "append_kernels", "pack_kernels",
-        "kv_bytes_attended", "h2d_bytes", "d2h_bytes", "d2d_bytes", "flushes", "flushes_to_u",
+        "kv_bytes_attended", "h2d_bytes", "d2h_bytes", "d2d_bytes", "flushes", "flushes_to_u", "fused_appends",
         "p_segments", "p_pinned_bytes", "p_pin_us", "p_grow_waits", "p_grow_wait_us",
         "p_register_us", "p_register_calls", "p_register_max_us")] + [("device_status", C.c_uint32)]
 
@@ -264,9 +264,12 @@ class Cache:
         self._check(lib().ipkv_flush(self._h, layer, seq, _stream(stream)), "ipkv_flush")
 
     def attend_gpu(self, layer, seq_ids, q, o_part, lse_part, kv_splits=0, side_stream=None, stream=None,
-                   fold_o=None, fold_lse=None, static_schedule=False, force_balance=False):
+                   fold_o=None, fold_lse=None, static_schedule=False, force_balance=False, append_k=None, append_v=None):
+        """append_k / append_v: one new token per listed sequence, appended first (fused into the kernel where possible)."""
         ids, n = _ids(seq_ids)
-        opts = AttendOpts(kv_splits, (ATTEND_STATIC_SCHEDULE if static_schedule else 0) | (ATTEND_BALANCE if force_balance else 0), _stream(side_stream) if side_stream is not None else None, _ptr(fold_o), _ptr(fold_lse))
+        opts = AttendOpts(kv_splits, (ATTEND_STATIC_SCHEDULE if static_schedule else 0) | (ATTEND_BALANCE if force_balance else 0),
+                          _stream(side_stream) if side_stream is not None else None, _ptr(fold_o), _ptr(fold_lse),
+                          _ptr(append_k), _ptr(append_v))
         self._check(lib().ipkv_attend_gpu(self._h, layer, ids, n, _ptr(q), C.byref(opts), _ptr(o_part), _ptr(lse_part),
                                           _stream(stream)), "ipkv_attend_gpu")
 

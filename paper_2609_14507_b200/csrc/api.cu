@@ -670,7 +670,7 @@ void fill_launch(AttnLaunch* a, int kind, int Hq, int Hkv, int dqk, int dv, int 
 // One group of segments for all rows: attention + split reduce, folding into (out_o, out_lse) when `fold`.
 ipkv_status run_group(ipkv* h, const std::vector<std::vector<PlanSeg>>& rows, const char* const bases[kMaxBases],
                       const void* q, int kv_splits, const float* fold_o, const float* fold_lse, float* out_o, float* out_lse,
-                      cudaStream_t s, int schedule_flags = 0) {
+                      cudaStream_t s, int schedule_flags = 0, const void* append_k = nullptr, const void* append_v = nullptr) {
     const ipkv_config& c = h->cfg;
     Plan plan;
     const PartGeom pg = part_geom(c.kind, c.n_q_heads, c.n_kv_heads);
@@ -710,6 +710,7 @@ ipkv_status run_group(ipkv* h, const std::vector<std::vector<PlanSeg>>& rows, co
     a.acc_lse = fold_lse;
     a.out_o = out_o; a.out_lse = out_lse;
     a.status = h->status_dev;
+    a.append_k = append_k; a.append_v = append_v;
     if (a.n_spans > 0) {
         const bool timed = h->prof_on && !h->prof_reduce && h->prof_used + 2 <= h->prof_ev.size();
         if (timed) CU(h, cudaEventRecord(h->prof_ev[h->prof_used], s));
@@ -1000,19 +1001,19 @@ ipkv_status ipkv_flush(ipkv_t* h, int32_t layer, int32_t seq, void* stream) {
     return IPKV_OK;
 }
 
-ipkv_status ipkv_append(ipkv_t* h, int32_t layer, const int32_t* seq_ids, int32_t n_seq,
-                        const void* k_dev, const void* v_dev, void* stream) {
-    if (!h) return IPKV_EINVAL;
+namespace {
+
+// The routing half of a decode append (Sec. 4.2) and, unless `defer_copy`, the copy of the new rows into the windows.
+// With `defer_copy` the caller's attention launch writes the rows itself (fused append).
+ipkv_status append_tokens(ipkv* h, int32_t layer, const int32_t* seq_ids, int32_t n_seq, const void* k_dev, const void* v_dev,
+                          cudaStream_t s, bool defer_copy) {
     const ipkv_config& c = h->cfg;
     if (layer < 0 || layer >= c.n_layers) return fail(h, IPKV_EINVAL, "layer out of range");
     if (n_seq < 0 || (n_seq > 0 && (!seq_ids || !k_dev || (c.kind == IPKV_GQA && !v_dev)))) return fail(h, IPKV_EINVAL, "bad arguments");
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
     for (int i = 0; i < n_seq; ++i) {
         if (seq_ids[i] < 0 || seq_ids[i] >= c.max_seqs) return fail(h, IPKV_EINVAL, "sequence id out of range");
         for (int j = 0; j < i; ++j) if (seq_ids[j] == seq_ids[i]) return fail(h, IPKV_EINVAL, "duplicate sequence id");
     }
-    DeviceGuard dev_guard(c.device);
-    CU(h, dev_guard.error());
     if (h->grow_p && layer == 0) {                  // one decode step further: the pinning thread paces itself by these
         std::lock_guard<std::mutex> lk(h->pmu);
         h->p_tick += 1;
@@ -1037,12 +1038,23 @@ ipkv_status ipkv_append(ipkv_t* h, int32_t layer, const int32_t* seq_ids, int32_
             rows.dst_off[i] = h->w_off(seq_ids[base + i]);
             rows.slot[i] = int32_t(st.router.stage());
         }
+        if (defer_copy) continue;
         const char* ks = static_cast<const char*>(k_dev) + base * k_row;
         const char* vs = v_dev ? static_cast<const char*>(v_dev) + base * v_row : nullptr;
         CU(h, launch_append(h->geom, ks, vs, c.dim_v, h->w_layer(layer), rows, n, s));
         h->stats.append_kernels += 1;
     }
     return IPKV_OK;
+}
+
+}  // namespace
+
+ipkv_status ipkv_append(ipkv_t* h, int32_t layer, const int32_t* seq_ids, int32_t n_seq,
+                        const void* k_dev, const void* v_dev, void* stream) {
+    if (!h) return IPKV_EINVAL;
+    DeviceGuard dev_guard(h->cfg.device);
+    CU(h, dev_guard.error());
+    return append_tokens(h, layer, seq_ids, n_seq, k_dev, v_dev, static_cast<cudaStream_t>(stream), false);
 }
 
 ipkv_status ipkv_attend_gpu(ipkv_t* h, int32_t layer, const int32_t* seq_ids, int32_t n_seq,
@@ -1064,6 +1076,18 @@ ipkv_status ipkv_attend_gpu(ipkv_t* h, int32_t layer, const int32_t* seq_ids, in
     CU(h, dev_guard.error());
     h->stats.attend_calls += 1;
     const int64_t bt = c.block_tokens;
+
+    // append first, if asked to: routing now; the rows themselves are written by the attention kernel where it can
+    // (grouped-query kernel, blocks of at least one tile), by the append kernel otherwise
+    const void* app_k = opts ? opts->append_k_dev : nullptr;
+    const void* app_v = opts ? opts->append_v_dev : nullptr;
+    bool fused_append = false;
+    if (app_k) {
+        fused_append = c.kind == IPKV_GQA && bt >= kTileTokens;
+        ipkv_status arc = append_tokens(h, layer, seq_ids, n_seq, app_k, app_v, s, fused_append);
+        if (arc != IPKV_OK) return arc;
+        if (fused_append) h->stats.fused_appends += 1;
+    }
 
     // group 0: everything already on the device (resident ring + D-window)
     std::vector<std::vector<PlanSeg>> rows(n_seq);
@@ -1087,13 +1111,14 @@ ipkv_status ipkv_attend_gpu(ipkv_t* h, int32_t layer, const int32_t* seq_ids, in
                 j += n;
             }
         }
-        if (st.router.window_fill() > 0) rows[i].push_back(PlanSeg{1, h->w_off(seq), st.router.window_fill()});
+        if (st.router.window_fill() > 0) rows[i].push_back(PlanSeg{1, h->w_off(seq), st.router.window_fill(), fused_append});
     }
     const char* bases[kMaxBases] = {h->ring ? h->ring_layer(layer) : nullptr, h->w_layer(layer), h->pp_dev, nullptr};
     const float* fold_o = opts ? opts->fold_o_dev : nullptr;
     const float* fold_lse = opts ? opts->fold_lse_dev : nullptr;
     if ((fold_o == nullptr) != (fold_lse == nullptr)) return fail(h, IPKV_EINVAL, "fold_o_dev and fold_lse_dev must be given together");
-    ipkv_status rc = run_group(h, rows, bases, q_dev, kv_splits, fold_o, fold_lse, o_part_dev, lse_part_dev, s, static_schedule);
+    ipkv_status rc = run_group(h, rows, bases, q_dev, kv_splits, fold_o, fold_lse, o_part_dev, lse_part_dev, s, static_schedule,
+                               fused_append ? app_k : nullptr, fused_append ? app_v : nullptr);
     if (rc != IPKV_OK) return rc;
     if (max_stream_chunks == 0) return IPKV_OK;
 

@@ -44,6 +44,8 @@ struct GqaParams {
     float* part_o;
     float* part_lse;
     uint32_t* status;
+    const __nv_bfloat16* append_k;   // fused append: new K / V rows [n_rows][n_kv_heads][D], or null
+    const __nv_bfloat16* append_v;
     int32_t* next;       // dynamic schedule: tiles claimed so far of every span [n_spans], of every CTA's chunk [n_ctas], and the
                          // number of CTAs that came to help with every chunk [n_ctas] (all zero at launch); null = static schedule
     const int32_t* cta_tiles;   // tiles in every CTA's chunk
@@ -62,8 +64,8 @@ struct SmemPlan {
     static constexpr int kStage = 2 * kPlane;
     static constexpr int kStagesBytes = STAGES * kStage;
     static constexpr int kBarOff = kStagesBytes;
-    static constexpr int kMetaOff = kBarOff + 2 * STAGES * 8;     // one StageMeta (16 bytes) per stage
-    static constexpr int kTotal = kMetaOff + STAGES * 16;
+    static constexpr int kMetaOff = kBarOff + 2 * STAGES * 8;     // one StageMeta (32 bytes) per stage
+    static constexpr int kTotal = kMetaOff + STAGES * 32;
 };
 
 template <int D, int STAGES, bool DUP>
@@ -110,7 +112,7 @@ __global__ void __launch_bounds__(kThreads) attn_gqa_kernel(const GqaParams p) {
             auto issue = [&](int sp, const Span& span, int tile, int slot) -> bool {
                 if (sp != cached_sp) {                             // first tile of a span: where its run lives
                     seg = p.segs[span.seg];
-                    seg_base = p.bases[seg.base_id] + seg.off + int64_t(span.gh / p.n_hg) * p.head_bytes;
+                    seg_base = p.bases[seg.base_id & kSegBaseMask] + seg.off + int64_t(span.gh / p.n_hg) * p.head_bytes;
                     cached_sp = sp;
                 }
                 const int st = it % STAGES;
@@ -122,6 +124,17 @@ __global__ void __launch_bounds__(kThreads) attn_gqa_kernel(const GqaParams p) {
                 s_meta[st].n_valid = left < kTileTokens ? int(left) : kTileTokens;
                 s_meta[st].q_row = span.row * p.Hq + g * p.G + hg * 16;
                 s_meta[st].n_heads = min(16, p.G - hg * 16);
+                int patch_tok = -1;
+                if ((seg.base_id & kSegAppended) && tile == (seg.n_tokens - 1) / kTileTokens) {
+                    // the run's last token comes with the launch (block_tokens >= 64 here: one block holds the tile)
+                    patch_tok = (seg.n_tokens - 1) % kTileTokens;
+                    const int64_t blk = t0 / p.bt;
+                    const uint64_t g_row = reinterpret_cast<uint64_t>(seg_base + blk * p.block_bytes + (t0 - blk * p.bt + patch_tok) * 128);
+                    s_meta[st].kv_row = span.row * (p.Hq / p.G) + g;
+                    s_meta[st].g_lo = uint32_t(g_row);
+                    s_meta[st].g_hi = uint32_t(g_row >> 32);
+                }
+                s_meta[st].patch_tok = patch_tok;
                 const uint32_t dst = s_base + st * SP::kStage;
                 const uint32_t bar = s_full + 8 * st;
                 if (p.bt >= kTileTokens) {
@@ -285,6 +298,23 @@ __global__ void __launch_bounds__(kThreads) attn_gqa_kernel(const GqaParams p) {
         }
         const int n_valid = s_meta[st].n_valid;
         {
+            const int ptok = s_meta[st].patch_tok;
+            if (ptok >= 0 && (ptok >> 4) == warp) {
+                // fused append: this warp owns the new token's slice of the tile; lanes 0-15 bring its K row, 16-31 its V row
+                const int chunk = lane & 15;
+                const bool is_v = lane >= 16;
+                if (chunk < D / 8) {
+                    const __nv_bfloat16* src = (is_v ? p.append_v : p.append_k) + int64_t(s_meta[st].kv_row) * D + chunk * 8;
+                    const uint4 val = __ldg(reinterpret_cast<const uint4*>(src));
+                    const uint32_t swz = uint32_t((chunk & 7) ^ (ptok & 7)) << 4;
+                    const uint32_t s_off = uint32_t(is_v ? SP::kPlane : 0) + (chunk >> 3) * 8192 + ptok * 128 + swz;
+                    *reinterpret_cast<uint4*>(smem + st * SP::kStage + s_off) = val;
+                    char* g_row = reinterpret_cast<char*>(uint64_t(s_meta[st].g_lo) | (uint64_t(s_meta[st].g_hi) << 32));
+                    *reinterpret_cast<uint4*>(g_row + int64_t(chunk >> 3) * p.bt * 128 + swz + (is_v ? int64_t(p.bt) * D * 2 : 0)) = val;
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // before the stage goes back to the copy engine
+                __syncwarp();
+            }
             if (warp * 16 < n_valid) {
                 const uint32_t kb = s_base + st * SP::kStage;
                 const uint32_t vb = kb + SP::kPlane;
@@ -382,6 +412,7 @@ cudaError_t launch_gqa(const AttnLaunch& a, cudaStream_t s) {
     for (int i = 0; i < kMaxBases; ++i) p.bases[i] = a.bases[i];
     p.segs = a.segs; p.spans = a.spans; p.cta_span_start = a.cta_span_start;
     p.part_o = a.part_o; p.part_lse = a.part_lse; p.status = a.status;
+    p.append_k = static_cast<const __nv_bfloat16*>(a.append_k); p.append_v = static_cast<const __nv_bfloat16*>(a.append_v);
     p.next = a.steal_next; p.lists = a.steal_lists; p.n_spans = a.n_spans; p.n_ctas = a.n_ctas; p.cta_tiles = a.cta_tiles;
     p.n_rows = a.n_rows; p.n_gh = a.n_gh;
     p.Hq = a.n_q_heads; p.G = a.n_q_heads / a.n_kv_heads;

@@ -106,7 +106,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_mla_kernel(const MlaParams p
             for (int sn = span_begin; sn < span_end && ok; ++sn) {
                 const Span span = p.spans[sn];
                 const Seg seg = p.segs[span.seg];
-                const char* seg_base = p.bases[seg.base_id] + seg.off;
+                const char* seg_base = p.bases[seg.base_id & kSegBaseMask] + seg.off;
                 for (int i = 0; i < span.ntiles; ++i, ++it) {
                     const int st = it % kStages;
                     if (it >= kStages && !ptx::mbar_wait(s_empty + 8 * st, ((it / kStages) - 1) & 1)) { ok = false; break; }

@@ -11,8 +11,13 @@ namespace ipkvi {
 struct Seg {
     int64_t off;
     int32_t n_tokens;
-    int32_t base_id;
+    int32_t base_id;     // index into bases (low byte); kSegAppended: the run's last token is written by this launch
 };
+// Fused append (grouped-query kernel): the last token of a flagged run is not in memory yet. The launch carries the
+// new K/V rows; the consumer warp that owns the token's 16-token slice writes them into the shared-memory tile once
+// its copy has landed (and into the run itself, for the launches to come), then computes as usual.
+constexpr int32_t kSegAppended = 0x100;
+constexpr int32_t kSegBaseMask = 0xff;
 // One span of split-K work: tiles [tile0, tile0 + ntiles) of segment `seg` for query row `row` and head
 // group `gh`.  A CTA processes a contiguous range of spans back to back; the partial(s) a span produces are
 // stored at the span's own index.
@@ -46,6 +51,8 @@ struct AttnLaunch {
     float* out_o;                   // [n_rows][Hq][dv]
     float* out_lse;                 // [n_rows][Hq]
     uint32_t* status;               // device word, OR-ed with an error bit if a bounded wait gives up
+    const void* append_k;           // fused append: [n_rows][n_kv_heads][dim_qk] bf16 new K rows (null: none)
+    const void* append_v;           // [n_rows][n_kv_heads][dim_v]
     // Dynamic load balancing of the GQA kernel (all null = static schedule with bit-reproducible results): a CTA
     // that has finished its chunk takes tiles from the spans that are furthest behind and accumulates them into
     // extra partials of its own, stored after the spans' partials (kStealSlots per CTA) and listed per (row, head group).

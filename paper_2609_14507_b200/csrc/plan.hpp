@@ -22,7 +22,7 @@ constexpr int kSmCount = 148;
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-struct PlanSeg { int base_id; int64_t off; int64_t n_tokens; };
+struct PlanSeg { int base_id; int64_t off; int64_t n_tokens; bool appended = false; };
 
 struct Plan {
     std::vector<Seg> segs;
@@ -74,7 +74,7 @@ inline void build_plan(const std::vector<std::vector<PlanSeg>>& rows, int n_gh, 
         for (const auto& s : rows[r]) {
             if (s.n_tokens <= 0) continue;
             row_segs[r].push_back(int32_t(plan->segs.size()));
-            plan->segs.push_back(Seg{s.off, int32_t(s.n_tokens), s.base_id});
+            plan->segs.push_back(Seg{s.off, int32_t(s.n_tokens), s.base_id | (s.appended ? kSegAppended : 0)});
             rt += (s.n_tokens + kTileTokens - 1) / kTileTokens;
             total_tokens += s.n_tokens;
         }

@@ -23,6 +23,9 @@ struct StageMeta {
     int32_t n_valid;     // live tokens of the tile (64 except at the end of a run)
     int32_t q_row;       // row * Hq + first query head of the tile's head group
     int32_t n_heads;     // query heads in the group (at most 16)
+    int32_t patch_tok;   // fused append: token of this tile whose K/V rows come with the launch, -1 = none
+    int32_t kv_row;      // ... their index (row * n_kv_heads + kv head) in the launch's new K/V rows
+    uint32_t g_lo, g_hi; // ... and the global address of the token's K row in panel 0 of its block
 };
 constexpr int32_t kEndSlot = -1;
 constexpr int kMinSteal = 3;        // a chunk is worth helping while at least this many of its tiles are unclaimed

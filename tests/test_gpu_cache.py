@@ -177,13 +177,18 @@ def test_decode_steps_with_evictions(resident, chunk, bt, D):
                     r.route.set_share(2)
             for layer in range(n_layers):
                 k = synth.normal_bf16(rng, (len(seqs), 2, 128)); v = synth.normal_bf16(rng, (len(seqs), 2, 128))
-                cache.append(layer, seqs, synth.bits_to_torch(k, DEV), synth.bits_to_torch(v, DEV))
+                attend_now = step % 13 == 0 or step == steps - 1
+                fused = attend_now and step % 2 == 0        # the append rides in the attention call (written by the kernel
+                kd, vd = synth.bits_to_torch(k, DEV), synth.bits_to_torch(v, DEV)      # itself when blocks hold a whole tile)
+                if not fused:
+                    cache.append(layer, seqs, kd, vd)
                 for i, s in enumerate(seqs):
                     refs[(layer, s)].append(k[i:i + 1], v[i:i + 1])
-                if step % 13 == 0 or step == steps - 1:
+                if attend_now:
                     q = synth.normal_bf16(rng, (len(seqs), 8, 128))
                     o = torch.zeros((len(seqs), 8, 128), device=DEV); lse = torch.zeros((len(seqs), 8), device=DEV)
-                    cache.attend_gpu(layer, seqs, synth.bits_to_torch(q, DEV), o, lse)
+                    cache.attend_gpu(layer, seqs, synth.bits_to_torch(q, DEV), o, lse, append_k=kd if fused else None,
+                                     append_v=vd if fused else None, force_balance=(step % 26 == 0))
                     parts = [refs[(layer, s)].attend(q[i], "gpu", scale) for i, s in enumerate(seqs)]
                     torch.cuda.synchronize()
                     check_partial(o.cpu().numpy(), lse.cpu().numpy(), np.stack([p[0] for p in parts]), np.stack([p[1] for p in parts]),
@@ -203,6 +208,7 @@ def test_decode_steps_with_evictions(resident, chunk, bt, D):
             check_contents(cache, layer, s, r, range(0, len(r.route), 7))
         st = cache.get_stats()
         assert st["device_status"] == 0 and st["flushes"] > 0 and 0 < st["flushes_to_u"] < st["flushes"]
+        assert (st["fused_appends"] > 0) == (bt >= 64)
 
 
 def test_explicit_partial_flush_and_errors():
@@ -582,3 +588,44 @@ def test_balanced_launches_of_changing_shape_stay_consistent():
             assert np.abs(res[0][0] - res[1][0]).max() < 2e-5, round_
             assert np.abs(res[0][1] - res[1][1]).max() < 2e-5, round_
         assert cache.get_stats()["device_status"] == 0
+
+
+@pytest.mark.parametrize("G,dim,bt", [(8, 128, 64), (4, 128, 128), (16, 64, 64), (32, 128, 64)])
+def test_fused_append_writes_the_window_and_attends_the_new_token(G, dim, bt):
+    """Decode steps whose append rides in the attention call: the kernel patches the new token into the tile it has
+    just loaded and stores it to the D-window.  After every step the output equals the oracle over all tokens including
+    the new one; afterwards every token reads back bit-exact (the kernel's stores are what later steps and the
+    evictions see).  Groups wider than 16 heads visit the tile once per head group."""
+    hkv = 2
+    sh = synth.Shape("fa", "gqa", 1, hkv * G, hkv, dim, dim, dim ** -0.5)
+    lens = [700, 63, 64, 0, 129]
+    scale = float(np.float32(sh.scale))
+    with make_cache(sh, 1, len(lens), block_tokens=bt, window_tokens=2 * bt, chunk_tokens=4 * bt, max_u_tokens_per_seq=1024,
+                    max_p_tokens_per_seq=2048, resident_tokens_per_seq=2048, share_num=1, share_den=2) as cache:
+        rng = np.random.default_rng(606)
+        refs = []
+        for s, n in enumerate(lens):
+            r = RefSeq(sh, bt, 2 * bt, 1, 2)
+            k, v = synth.host_kv(sh, n, seed=9600 + s)
+            cache.append_bulk(0, s, synth.bits_to_torch(k, DEV) if n else None, synth.bits_to_torch(v, DEV) if n else None, n, 1, 3)
+            r.bulk(k, v, 1, 3)
+            refs.append(r)
+        seqs = list(range(len(lens)))
+        for step in range(3 * bt + 5):                      # crosses tile boundaries and three evictions per sequence
+            k = synth.normal_bf16(rng, (len(lens), hkv, dim)); v = synth.normal_bf16(rng, (len(lens), hkv, dim))
+            q = synth.normal_bf16(rng, (len(lens), hkv * G, dim))
+            o = torch.zeros((len(lens), hkv * G, dim), device=DEV); lse = torch.zeros((len(lens), hkv * G), device=DEV)
+            cache.attend_gpu(0, seqs, synth.bits_to_torch(q, DEV), o, lse, append_k=synth.bits_to_torch(k, DEV),
+                             append_v=synth.bits_to_torch(v, DEV), force_balance=(step % 3 == 0), kv_splits=(0, 2)[step % 2])
+            for s in seqs:
+                refs[s].append(k[s:s + 1], v[s:s + 1])
+            if step % 9 == 0 or step > 3 * bt:
+                torch.cuda.synchronize()
+                parts = [refs[s].attend(q[s], "gpu", scale) for s in seqs]
+                check_partial(o.cpu().numpy(), lse.cpu().numpy(), np.stack([p[0] for p in parts]), np.stack([p[1] for p in parts]), f"step {step}")
+        torch.cuda.synchronize()
+        for s in seqs:
+            check_routing(cache, 0, s, refs[s], sample=range(0, len(refs[s].route), 11))
+            check_contents(cache, 0, s, refs[s], range(0, len(refs[s].route), 3))
+        st = cache.get_stats()
+        assert st["device_status"] == 0 and st["fused_appends"] == 3 * bt + 5 and st["append_kernels"] == 0
