@@ -273,13 +273,17 @@ def test_mla_cache_decode_steps(resident):
             refs[s] = r
         for step in range(200):
             k = synth.normal_bf16(rng, (2, 1, 576))
-            cache.append(0, seqs, synth.bits_to_torch(k, DEV), None)
+            attend_now = step % 37 == 0 or step % 10 == 3 or step == 199
+            fused = attend_now and step % 2 == 1                  # the new latent row rides in the attention call
+            kd = synth.bits_to_torch(k, DEV)
+            if not fused:
+                cache.append(0, seqs, kd, None)
             for i, s in enumerate(seqs):
                 refs[s].append(k[i:i + 1], None)
-            if step % 37 == 0 or step == 199:
+            if attend_now:
                 q = synth.normal_bf16(rng, (2, 16, 576))
                 o = torch.zeros((2, 16, 512), device=DEV); lse = torch.zeros((2, 16), device=DEV)
-                cache.attend_gpu(0, seqs, synth.bits_to_torch(q, DEV), o, lse)
+                cache.attend_gpu(0, seqs, synth.bits_to_torch(q, DEV), o, lse, append_k=kd if fused else None)
                 torch.cuda.synchronize()
                 parts = [refs[s].attend(q[i], "gpu", scale) for i, s in enumerate(seqs)]
                 check_partial(o.cpu().numpy(), lse.cpu().numpy(), np.stack([p[0] for p in parts]), np.stack([p[1] for p in parts]),
@@ -295,8 +299,9 @@ def test_mla_cache_decode_steps(resident):
                               np.stack([p[0] for p in full]), np.stack([p[1] for p in full]), f"mla merged step {step}")
         for s in seqs:
             check_routing(cache, 0, s, refs[s], sample=range(0, len(refs[s].route), 5))
-            check_contents(cache, 0, s, refs[s], range(0, len(refs[s].route), 11))
-        assert cache.get_stats()["device_status"] == 0
+            check_contents(cache, 0, s, refs[s], range(0, len(refs[s].route), 3))
+        st = cache.get_stats()
+        assert st["device_status"] == 0 and st["fused_appends"] >= 10
 
 
 @pytest.mark.parametrize("kind", ["gqa", "mla"])
