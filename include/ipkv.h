@@ -175,9 +175,9 @@ typedef struct {
   /* Optional fused decode append (ipkv_attend_gpu only): one new token for each listed sequence,
      k [n_seq][n_kv_heads][dim_qk], v [n_seq][n_kv_heads][dim_v] (NULL for IPKV_MLA), appended exactly as ipkv_append
      would (full windows are evicted first) and attended by the same call.  Where the kernel can, it writes the new
-     rows into the D-window itself (block_tokens >= 64: a warp patches the tile in shared memory once its copy
-     has landed and stores the rows to the window), which saves the append launch of every layer; otherwise the
-     library launches its append kernel first.  The result is the same either way.                               */
+     rows into the D-window itself (grouped-query caches with block_tokens >= 64: the warp that owns the token's slice
+     of the tile patches the tile in shared memory and stores the rows to the window), which saves the append launch of
+     every layer; otherwise the library launches its append kernel first.  The result is the same either way.   */
   const void* append_k_dev;
   const void* append_v_dev;
 } ipkv_attend_opts;

@@ -1078,13 +1078,12 @@ ipkv_status ipkv_attend_gpu(ipkv_t* h, int32_t layer, const int32_t* seq_ids, in
     const int64_t bt = c.block_tokens;
 
     // append first, if asked to: routing now; the rows themselves are written by the attention kernel where it can
-    // (blocks of at least one tile), by the append kernel otherwise
+    // (grouped-query kernel, blocks of at least one tile), by the append kernel otherwise
     const void* app_k = opts ? opts->append_k_dev : nullptr;
     const void* app_v = opts ? opts->append_v_dev : nullptr;
     bool fused_append = false;
     if (app_k) {
-        static const bool mla_tc = std::getenv("IPKV_MLA_TC") != nullptr;        // the opt-in tcgen05 variant has no fused append
-        fused_append = bt >= kTileTokens && !(c.kind == IPKV_MLA && mla_tc);
+        fused_append = c.kind == IPKV_GQA && bt >= kTileTokens;
         ipkv_status arc = append_tokens(h, layer, seq_ids, n_seq, app_k, app_v, s, fused_append);
         if (arc != IPKV_OK) return arc;
         if (fused_append) h->stats.fused_appends += 1;

@@ -60,7 +60,6 @@ struct MlaParams {
     float* part_o;
     float* part_lse;
     uint32_t* status;
-    const __nv_bfloat16* append_k;   // fused append: new latent rows [n_rows][576], or null
     int Hq;
     int bt;
     int64_t block_bytes;
@@ -145,7 +144,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_mla_kernel(const MlaParams p
             const int first_pending = it > kStages ? it - kStages : 0;
             for (int i = first_pending; i < it; ++i)
                 if (!ptx::mbar_wait(s_full + 8 * (i % kStages), (i / kStages) & 1)) ok = false;
-            if (!ok) atomicOr(p.status, kStatusNoFreeStage | kStatusCopyNotLanded);
+            if (!ok) atomicOr(p.status, 2u);
         }
         return;      // the consumers synchronise among themselves on a named barrier
     }
@@ -188,24 +187,6 @@ __global__ void __launch_bounds__(kThreads, 1) attn_mla_kernel(const MlaParams p
             const int64_t left = int64_t(seg.n_tokens) - t0;
             const int n_valid = left < kTileTokens ? int(left) : kTileTokens;
             const uint32_t kb = s_base + st * kStageBytes;
-
-            // fused append: the run's last token comes with the launch. Warp 0 writes its row (72 chunks of 16 bytes) into
-            // the tile that has just landed and into the run itself; everybody waits for it (every warp reads every row).
-            if ((seg.base_id & kSegAppended) && span.tile0 + i == (seg.n_tokens - 1) / kTileTokens) {
-                if (warp == 0) {
-                    const int ptok = (seg.n_tokens - 1) % kTileTokens;
-                    const int64_t blk = t0 / p.bt;
-                    char* g_row = const_cast<char*>(p.bases[seg.base_id & kSegBaseMask]) + seg.off + blk * p.block_bytes + (t0 - blk * p.bt + ptok) * 128;
-                    for (int chunk = lane; chunk < kDqk / 8; chunk += 32) {
-                        const uint4 val = __ldg(reinterpret_cast<const uint4*>(p.append_k + int64_t(span.row) * kDqk + chunk * 8));
-                        const uint32_t swz = uint32_t((chunk & 7) ^ (ptok & 7)) << 4;
-                        *reinterpret_cast<uint4*>(smem + st * kStageBytes + (chunk >> 3) * 8192 + ptok * 128 + swz) = val;
-                        *reinterpret_cast<uint4*>(g_row + int64_t(chunk >> 3) * p.bt * 128 + swz) = val;
-                    }
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // before the stage goes back to the copy engine
-                }
-                consumer_barrier();
-            }
 
             // ---- phase 1: partial scores of d-slice ds for tokens [32 th, 32 th + 32) ----
             {
@@ -330,7 +311,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_mla_kernel(const MlaParams p
         }
         consumer_barrier();      // s_m / s_l / the query tile are reused by the next span
     }
-    if (!ok && lane == 0) atomicOr(p.status, kStatusNoTile);
+    if (!ok && lane == 0) atomicOr(p.status, 2u);
 }
 
 }  // namespace
@@ -348,7 +329,6 @@ cudaError_t launch_attend_mla(const AttnLaunch& a, cudaStream_t s) {
     for (int i = 0; i < kMaxBases; ++i) p.bases[i] = a.bases[i];
     p.segs = a.segs; p.spans = a.spans; p.cta_span_start = a.cta_span_start;
     p.part_o = a.part_o; p.part_lse = a.part_lse; p.status = a.status;
-    p.append_k = static_cast<const __nv_bfloat16*>(a.append_k);
     p.Hq = a.n_q_heads;
     p.bt = a.bt;
     p.block_bytes = int64_t(a.bt) * kDqk * 2;

@@ -301,7 +301,7 @@ def test_mla_cache_decode_steps(resident):
             check_routing(cache, 0, s, refs[s], sample=range(0, len(refs[s].route), 5))
             check_contents(cache, 0, s, refs[s], range(0, len(refs[s].route), 3))
         st = cache.get_stats()
-        assert st["device_status"] == 0 and st["fused_appends"] >= 10
+        assert st["device_status"] == 0 and st["fused_appends"] == 0        # this kind appends with the append kernel inside the call
 
 
 @pytest.mark.parametrize("kind", ["gqa", "mla"])
