@@ -69,7 +69,7 @@ struct SmemPlan {
 };
 
 template <int D, int STAGES, bool DUP>
-__global__ void __launch_bounds__(kThreads) attn_gqa_kernel(const GqaParams p) {
+__global__ void __launch_bounds__(kThreads, 2) attn_gqa_kernel(const GqaParams p) {
     using SP = SmemPlan<D, STAGES>;
     extern __shared__ unsigned char smem_dyn[];
     // align the ring to 1024 bytes so that the 128-byte chunk swizzle maps onto distinct banks
