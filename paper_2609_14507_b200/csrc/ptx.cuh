@@ -1,5 +1,5 @@
 // Thin wrappers over the sm_100a PTX used by the attention kernels: mbarrier, bulk asynchronous
-// copies (the TMA engine, non-tensor form, never multicast), ldmatrix and the bf16 tensor-core MMA.
+// copies (the TMA engine, non-tensor form, one destination CTA), ldmatrix and the bf16 tensor-core MMA.
 #pragma once
 #include <cstdint>
 
