@@ -1,7 +1,7 @@
 """Parity at the benchmark's sizes and launch configuration, on sampled outputs the oracle computes one by one.
 
-The caches are built exactly as bench.py builds them (same shapes, seeds, shares, flags); one decode step is run
-(append, attend, merge) and, for a sample of (layer, sequence) pairs, the oracle recomputes the GPU-side partial of
+The caches are built exactly as bench.py builds them (same shapes, seeds, shares, flags); one decode step is run the
+way bench.py runs it (append riding in the attention call, balanced schedule, fold in the split reduce) and, for a sample of (layer, sequence) pairs, the oracle recomputes the GPU-side partial of
 every head from the same bits (regenerated from the seed and copied to the host)."""
 import numpy as np
 import pytest
@@ -35,9 +35,13 @@ def _run_step_and_check(name, samples, kv_splits=0):
             q = torch.randn((B, sh.n_q_heads, sh.dim_qk), generator=g, device=DEV).to(torch.bfloat16)
             kn = torch.randn((B, sh.n_kv_heads, sh.dim_qk), generator=g, device=DEV).to(torch.bfloat16)
             vn = None if sh.kind == "mla" else torch.randn((B, sh.n_kv_heads, sh.dim_v), generator=g, device=DEV).to(torch.bfloat16)
-            cache.append(layer, ids, kn, vn)
+            # as bench.py issues a layer: the append rides in the attention call (written by the kernel itself for the
+            # grouped-query shapes), launches this long are dynamically balanced, and a partial is folded in by the
+            # split reduce (an empty one here, so that the output stays the GPU-side partial the oracle recomputes)
             o = torch.zeros((B, sh.n_q_heads, sh.dim_v), device=DEV); lse = torch.zeros((B, sh.n_q_heads), device=DEV)
-            cache.attend_gpu(layer, ids, q, o, lse, kv_splits=kv_splits)
+            fold_o = torch.zeros((B, sh.n_q_heads, sh.dim_v), device=DEV)
+            fold_lse = torch.full((B, sh.n_q_heads), float("-inf"), device=DEV)
+            cache.attend_gpu(layer, ids, q, o, lse, kv_splits=kv_splits, append_k=kn, append_v=vn, fold_o=fold_o, fold_lse=fold_lse)
             torch.cuda.synchronize()
             o_h, lse_h, q_h = o.cpu().numpy(), lse.cpu().numpy(), synth.torch_bits(q)
             kn_h, vn_h = synth.torch_bits(kn), (None if vn is None else synth.torch_bits(vn))
