@@ -345,6 +345,11 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--kv-splits", type=int, default=0)
     ap.add_argument("--no-read-ceiling", action="store_true", help="skip the read-only bandwidth probe reported in roofline.read_ceiling")
+    ap.add_argument("--time-every", type=int, default=4,
+                    help="CUDA events around every N-th attention launch of the timed region (every launch does the same work; an event "
+                         "between two kernels costs the step several microseconds, so bracketing all of them would slow what is measured)")
+    ap.add_argument("--no-kernel-timing", action="store_true",
+                    help="diagnostic: no CUDA events around the attention launches (the roofline object is then empty); shows what the events cost the step")
     ap.add_argument("--profile-reduce", action="store_true",
                     help="diagnostic: the kernel timed by CUDA events is the split reduce, not the attention kernel (the roofline object is then meaningless)")
     ap.add_argument("--static-schedule", action="store_true",
@@ -436,7 +441,7 @@ def main():
         step()
     barrier()
     st0 = cache.get_stats()
-    cache.profile_enable(True, reduce=args.profile_reduce)
+    cache.profile_enable(not args.no_kernel_timing, reduce=args.profile_reduce, every=args.time_every)
     cache.profile_read()
     sampler.mark()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -565,7 +570,7 @@ def main():
                        "cpu_share": f"{num0}/{den0}", "gpu_share_tokens_per_seq_mean": n_gpu0 + 1, "bytes_per_kv_token": bpt, "block_tokens": BLOCK, "window_tokens": wl.get("window", WINDOW),
                        "gpu_share": "HBM-resident", "host_copies_of_U_and_P": "off (benchmark)", "cpu_partial": "synthetic values",
                        "l2": l2_note,
-                       "multi_gpu": "replicas only", "kv_splits": args.kv_splits, "schedule": "static" if args.static_schedule else "dynamic balancing (GQA kernel, launches of at least 48 tiles per CTA)",
+                       "multi_gpu": "replicas only", "kv_splits": args.kv_splits, "kernel_timing": "CUDA events around every %d%s attention launch" % (args.time_every, "th" if args.time_every != 1 else "st"), "schedule": "static" if args.static_schedule else "dynamic balancing (GQA kernel, launches of at least 48 tiles per CTA)",
                        "merge": "inside the split reduce" if fused else "separate ipkv_merge launch",
                        "append": "separate ipkv_append" if args.separate_append else "inside ipkv_attend_gpu (written by the attention kernel for GQA)"},
             "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu,

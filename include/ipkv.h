@@ -291,7 +291,10 @@ ipkv_status ipkv_policy_prefill_share(const ipkv_policy_t* p, double L0, int32_t
  * bracketed by a pair of CUDA events on the launching stream.  ipkv_profile_read synchronises the device,
  * returns the summed kernel time (milliseconds) and the number of launches since the last read, and resets
  * both.  At most 8192 launches are kept between two reads; later ones are counted but not timed. */
-ipkv_status ipkv_profile_enable(ipkv_t* h, int32_t on);   /* 0 off, 1 attention kernels, 2 split-reduce kernels instead */
+/* on: 0 off, 1 attention kernels, 2 split-reduce kernels instead; plus 256 * n to bracket only every n-th launch (an
+ * event between two kernels keeps the second from starting while the first drains, which costs the step several
+ * microseconds per bracketed launch). */
+ipkv_status ipkv_profile_enable(ipkv_t* h, int32_t on);
 ipkv_status ipkv_profile_read(ipkv_t* h, double* attend_kernel_ms, int64_t* n_timed, int64_t* n_launches);
 
 /* Measurement aid (no counterpart in the paper): the rate, in GB/s, at which the SMs of `device` read `bytes` bytes

@@ -323,9 +323,9 @@ class Cache:
                     "ipkv_read_token")
         return k, v
 
-    def profile_enable(self, on=True, reduce=False):
-        """Time every attention-kernel launch (or, with reduce=True, every split-reduce launch) with CUDA events."""
-        self._check(lib().ipkv_profile_enable(self._h, (2 if reduce else 1) if on else 0), "ipkv_profile_enable")
+    def profile_enable(self, on=True, reduce=False, every=1):
+        """Time every `every`-th attention-kernel launch (or, with reduce=True, split-reduce launch) with CUDA events."""
+        self._check(lib().ipkv_profile_enable(self._h, ((2 if reduce else 1) + 256 * max(1, int(every))) if on else 0), "ipkv_profile_enable")
 
     def profile_read(self):
         """(summed attention-kernel milliseconds, launches timed, launches seen) since the last read."""

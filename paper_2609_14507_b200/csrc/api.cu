@@ -163,6 +163,8 @@ struct ipkv {
     // optional kernel timing
     bool prof_on = false;
     bool prof_reduce = false;              // time the split reduce instead of the attention kernel
+    int prof_stride = 1;                   // time every prof_stride-th launch
+    int64_t prof_seen = 0;
     std::vector<cudaEvent_t> prof_ev;      // pairs
     size_t prof_used = 0;                  // events used
     int64_t prof_launches = 0;
@@ -712,7 +714,8 @@ ipkv_status run_group(ipkv* h, const std::vector<std::vector<PlanSeg>>& rows, co
     a.status = h->status_dev;
     a.append_k = append_k; a.append_v = append_v;
     if (a.n_spans > 0) {
-        const bool timed = h->prof_on && !h->prof_reduce && h->prof_used + 2 <= h->prof_ev.size();
+        const bool sampled = h->prof_on && (h->prof_seen++ % h->prof_stride) == 0;
+        const bool timed = sampled && !h->prof_reduce && h->prof_used + 2 <= h->prof_ev.size();
         if (timed) CU(h, cudaEventRecord(h->prof_ev[h->prof_used], s));
         CU(h, launch_attend(a, s));
         if (timed) { CU(h, cudaEventRecord(h->prof_ev[h->prof_used + 1], s)); h->prof_used += 2; }
@@ -720,7 +723,7 @@ ipkv_status run_group(ipkv* h, const std::vector<std::vector<PlanSeg>>& rows, co
         h->stats.attend_kernels += 1;
     }
     {
-        const bool timed = h->prof_on && h->prof_reduce && h->prof_used + 2 <= h->prof_ev.size();
+        const bool timed = h->prof_on && h->prof_reduce && ((h->prof_seen - 1) % h->prof_stride) == 0 && h->prof_used + 2 <= h->prof_ev.size();
         if (timed) CU(h, cudaEventRecord(h->prof_ev[h->prof_used], s));
         CU(h, launch_split_reduce(a, s));
         if (timed) { CU(h, cudaEventRecord(h->prof_ev[h->prof_used + 1], s)); h->prof_used += 2; }
@@ -1559,7 +1562,9 @@ ipkv_status ipkv_profile_enable(ipkv_t* h, int32_t on) {
         for (auto& e : h->prof_ev) CU(h, cudaEventCreate(&e));
     }
     h->prof_on = on != 0;
-    h->prof_reduce = on == 2;
+    h->prof_reduce = (on & 3) == 2;
+    h->prof_stride = (on >> 8) > 0 ? (on >> 8) : 1;
+    h->prof_seen = 0;
     return IPKV_OK;
 }
 
