@@ -498,7 +498,7 @@ def main():
     e2e = None
     if not args.no_e2e:
         # One step's inputs for all layers sit in pinned host memory (queries, new K/V tokens, the CPU engine's partials);
-        # each step copies them to the device (one copy per tensor), runs the path, and reads all layers' outputs back.
+        # each step copies them to the device, runs the path, and reads all layers' outputs back.
         hq = q.cpu().pin_memory(); hk = k_new.cpu().pin_memory()
         hv = None if v_new is None else v_new.cpu().pin_memory()
         hoc = o_cpu.cpu().pin_memory(); hlc = lse_cpu.cpu().pin_memory()
@@ -506,26 +506,47 @@ def main():
         dq = torch.empty_like(q); dk = torch.empty_like(k_new); dvn = None if v_new is None else torch.empty_like(v_new)
         doc = torch.empty_like(o_cpu); dlc = torch.empty_like(lse_cpu)
 
+        # The copies run on a stream of their own, in four groups of layers: the layers of a group start as soon as the
+        # group's inputs have landed, so only the first group's copies (and the last group's read-back) are not hidden
+        # behind the other groups' kernels, the way a server overlaps its transfers with the previous layers' work.
+        cs = torch.cuda.Stream()
+        n_groups = min(4, NL)
+        bounds = [NL * g // n_groups for g in range(n_groups + 1)]
+        landed = [torch.cuda.Event() for _ in range(n_groups)]
+        computed = [torch.cuda.Event() for _ in range(n_groups)]
+        step_done = torch.cuda.Event()
+
         def step_e2e():
-            dq.copy_(hq, non_blocking=True)
-            dk.copy_(hk, non_blocking=True)
-            if dvn is not None:
-                dvn.copy_(hv, non_blocking=True)
-            doc.copy_(hoc, non_blocking=True)
-            dlc.copy_(hlc, non_blocking=True)
-            for layer in range(NL):
-                app = {} if args.separate_append else dict(append_k=dk[layer], append_v=None if dvn is None else dvn[layer])
-                if args.separate_append:
-                    cache.append(layer, seq_ids, dk[layer], None if dvn is None else dvn[layer], stream=cur)
-                if fused:
-                    cache.attend_gpu(layer, seq_ids, dq[layer], out[layer], out_lse, kv_splits=args.kv_splits, static_schedule=args.static_schedule, stream=cur,
-                                     fold_o=doc[layer], fold_lse=dlc[layer], **app)
-                else:
-                    cache.attend_gpu(layer, seq_ids, dq[layer], o_part, lse_part, kv_splits=args.kv_splits, static_schedule=args.static_schedule, stream=cur, **app)
-                    cache.merge(B * Hq, dv, [o_part.view(B * Hq, dv), doc[layer]], [lse_part.view(-1), dlc[layer]],
-                                out[layer], out_lse, out_is_bf16=True, stream=cur)
-            hout.copy_(out, non_blocking=True)
-            torch.cuda.synchronize()
+            cs.wait_event(step_done)                     # the previous step's kernels no longer read the input buffers
+            with torch.cuda.stream(cs):
+                for g in range(n_groups):
+                    lo, hi = bounds[g], bounds[g + 1]
+                    dq[lo:hi].copy_(hq[lo:hi], non_blocking=True)
+                    dk[lo:hi].copy_(hk[lo:hi], non_blocking=True)
+                    if dvn is not None:
+                        dvn[lo:hi].copy_(hv[lo:hi], non_blocking=True)
+                    doc[lo:hi].copy_(hoc[lo:hi], non_blocking=True)
+                    dlc[lo:hi].copy_(hlc[lo:hi], non_blocking=True)
+                    landed[g].record(cs)
+            for g in range(n_groups):
+                cur.wait_event(landed[g])
+                for layer in range(bounds[g], bounds[g + 1]):
+                    app = {} if args.separate_append else dict(append_k=dk[layer], append_v=None if dvn is None else dvn[layer])
+                    if args.separate_append:
+                        cache.append(layer, seq_ids, dk[layer], None if dvn is None else dvn[layer], stream=cur)
+                    if fused:
+                        cache.attend_gpu(layer, seq_ids, dq[layer], out[layer], out_lse, kv_splits=args.kv_splits, static_schedule=args.static_schedule, stream=cur,
+                                         fold_o=doc[layer], fold_lse=dlc[layer], **app)
+                    else:
+                        cache.attend_gpu(layer, seq_ids, dq[layer], o_part, lse_part, kv_splits=args.kv_splits, static_schedule=args.static_schedule, stream=cur, **app)
+                        cache.merge(B * Hq, dv, [o_part.view(B * Hq, dv), doc[layer]], [lse_part.view(-1), dlc[layer]],
+                                    out[layer], out_lse, out_is_bf16=True, stream=cur)
+                computed[g].record(cur)
+                with torch.cuda.stream(cs):
+                    cs.wait_event(computed[g])
+                    hout[bounds[g]:bounds[g + 1]].copy_(out[bounds[g]:bounds[g + 1]], non_blocking=True)
+            step_done.record(cur)
+            torch.cuda.synchronize()                     # the step's result is on the host
 
         for _ in range(args.warmup):
             step_e2e()
