@@ -158,6 +158,8 @@ struct ipkv {
     std::vector<cudaEvent_t> slot_ready, slot_free;
     std::vector<char> slot_free_set;
     cudaEvent_t ev_main = nullptr;
+    cudaEvent_t ev_p_host = nullptr;       // after the last copy into P's host memory that a compute stream carried (prefill)
+    bool ev_p_host_set = false;
     ipkv_stats stats;
     std::string err;
     // optional kernel timing
@@ -802,6 +804,7 @@ ipkv_status ipkv_destroy(ipkv_t* h) {
     for (auto e : h->slot_ready) cudaEventDestroy(e);
     for (auto e : h->slot_free) cudaEventDestroy(e);
     if (h->ev_main) cudaEventDestroy(h->ev_main);
+    if (h->ev_p_host) cudaEventDestroy(h->ev_p_host);
     if (h->side) cudaStreamDestroy(h->side);
     delete h;
     return IPKV_OK;
@@ -894,6 +897,7 @@ ipkv_status ipkv_create(const ipkv_config* cfg, ipkv_t** out) {
         if (cudaEventCreateWithFlags(&h->slot_free[i], cudaEventDisableTiming) != cudaSuccess) return bail(IPKV_ECUDA);
     }
     if (cudaEventCreateWithFlags(&h->ev_main, cudaEventDisableTiming) != cudaSuccess) return bail(IPKV_ECUDA);
+    if (cudaEventCreateWithFlags(&h->ev_p_host, cudaEventDisableTiming) != cudaSuccess) return bail(IPKV_ECUDA);
     if (cudaDeviceSynchronize() != cudaSuccess) return bail(IPKV_ECUDA);
     *out = h;
     return IPKV_OK;
@@ -938,6 +942,7 @@ ipkv_status ipkv_append_bulk(ipkv_t* h, int32_t layer, int32_t seq, const void* 
     CU(h, dev_guard.error());
     Run placed[2];
     const int n_runs = st.router.bulk(n_tokens, num0, den0, placed);
+    bool wrote_p_host = false;
     const int64_t k_row = int64_t(c.n_kv_heads) * c.dim_qk * 2, v_row = int64_t(c.n_kv_heads) * c.dim_v * 2;
     const size_t stage_cap = size_t(std::max<int64_t>(h->bb, (int64_t(32) << 20) / h->bb * h->bb));
     for (int i = 0; i < n_runs; ++i) {
@@ -980,9 +985,14 @@ ipkv_status ipkv_append_bulk(ipkv_t* h, int32_t layer, int32_t seq, const void* 
                 });
                 if (rc != IPKV_OK) return rc;
                 p_note_placed(h, r.first_block + j_end - 1);
+                wrote_p_host = true;
             }
             j = j_end;
         }
+    }
+    if (wrote_p_host) {                        // the streamed attention path reads these bytes on another stream
+        CU(h, cudaEventRecord(h->ev_p_host, s));
+        h->ev_p_host_set = true;
     }
     return IPKV_OK;
 }
@@ -1126,9 +1136,11 @@ ipkv_status ipkv_attend_gpu(ipkv_t* h, int32_t layer, const int32_t* seq_ids, in
     if (max_stream_chunks == 0) return IPKV_OK;
 
     // groups 1..: host-only P chunks, streamed through the PP slots in overwrite-reuse order (Sec. 4.2)
-    CU(h, cudaEventRecord(h->ev_main, s));                 // P's host bytes were written by work on `s` ...
-    CU(h, cudaStreamWaitEvent(side, h->ev_main, 0));
-    CU(h, cudaEventRecord(h->ev_copy, h->copy));           // ... or by write-backs on the copy stream
+    // P's host bytes were written by a prefill copy on a compute stream or by write-backs on the copy stream. The side
+    // stream waits for exactly those, not for everything queued on `s`: the copies of this layer's chunks then run
+    // while the previous layer's kernels are still going.
+    if (h->ev_p_host_set) CU(h, cudaStreamWaitEvent(side, h->ev_p_host, 0));
+    CU(h, cudaEventRecord(h->ev_copy, h->copy));
     CU(h, cudaStreamWaitEvent(side, h->ev_copy, 0));
     const int64_t chunk_bytes = h->chunk_blocks * h->bb;
     // A chunk that lies in grown segments holds chunk_blocks / w_blocks whole eviction batches. Each batch is one
