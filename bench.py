@@ -333,9 +333,47 @@ def h2d_microbench():
                       "22.2 at 1 MB, 8.7 at 192 KB; pageable 10; strided 4.6"}))
 
 
+def cpu_engine_microbench():
+    """The CPU-side engine (in-place attention over the unpinned region, Sec. 6.1) on the host cores of this machine: the
+    quantity the roofline policy calls A (seconds per CPU-side KV token, Eq. 1).  Qwen3 and DeepSeek-V2-Lite shapes,
+    one layer; the CPU share sits in U (PLAIN blocks, unpinned), written there by the library's own prefill routing."""
+    import torch
+    from paper_2609_14507_b200 import binding
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    out = {}
+    for name, sh, batch, n_u in (("qwen3 (GQA 32/4, d 128)", synth.QWEN3, 16, 16384), ("deepseek-v2-lite (latent 576/512, 16 heads)", synth.DSV2_LITE, 8, 16384)):
+        kind = binding.MLA if sh.kind == "mla" else binding.GQA
+        cfg = binding.make_config(kind, 1, batch, sh.n_q_heads, sh.n_kv_heads, sh.dim_qk, sh.dim_v, block_tokens=BLOCK, window_tokens=WINDOW,
+                                  chunk_tokens=512, max_u_tokens_per_seq=n_u, max_p_tokens_per_seq=2 * WINDOW, resident_tokens_per_seq=2 * WINDOW,
+                                  softmax_scale=sh.scale, flags=binding.FLAG_NO_HOST_P)
+        with binding.Cache(cfg) as cache:
+            for s_ in range(batch):
+                k, v = synth.device_kv(sh, n_u + WINDOW, 4242 + s_, dev)
+                cache.append_bulk(0, s_, k, v, n_u + WINDOW, n_u, n_u + WINDOW)      # the first n_u tokens go to U
+            torch.cuda.synchronize()
+            cache.get_stats()                                                          # drains the write-back stream
+            q = torch.randn((batch, sh.n_q_heads, sh.dim_qk)).to(torch.bfloat16)
+            o = torch.zeros((batch, sh.n_q_heads, sh.dim_v)); lse = torch.zeros((batch, sh.n_q_heads))
+            ids = list(range(batch))
+            times = []
+            for _ in range(6):
+                t0 = time.perf_counter()
+                cache.attend_cpu(0, ids, q, o, lse)
+                times.append(time.perf_counter() - t0)
+            t = statistics.median(times[1:])
+            tokens = batch * n_u
+            out[name] = {"cpu_tokens": tokens, "seconds": t, "kv_tokens_per_s": tokens / t, "gb_per_s": tokens * sh.bytes_per_token / t / 1e9,
+                         "A_seconds_per_token_per_sequence_batch": t / n_u, "threads": os.cpu_count()}
+    print(json.dumps({"cpu_engine_microbench": out}))
+
+
 def main():
     if "--h2d-microbench" in sys.argv:
         h2d_microbench()
+        return
+    if "--cpu-engine-microbench" in sys.argv:
+        cpu_engine_microbench()
         return
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
