@@ -22,6 +22,26 @@ def _deps_mtime():
     return max(os.path.getmtime(f) for f in files)
 
 
+# The CPU engine's tile kernel is compiled once per x86-64 instruction-set level; cpu_engine.cpp picks one at run time.
+CPU_KERNEL_LEVELS = (("v4", ["-march=x86-64-v4"]), ("v3", ["-march=x86-64-v3"]), ("base", []))
+
+
+def cpu_engine_commands(obj_dir):
+    """(command, object) pairs that compile the host-only sources (also used by the tests' CPU-engine shim)."""
+    out = []
+    base = ["g++", "-std=c++17", "-O3", "-fopenmp", "-fPIC", "-Wno-psabi"]
+    for src in sorted(glob.glob(os.path.join(CSRC, "*.cpp"))):
+        name = os.path.basename(src)[:-4]
+        if name == "cpu_engine_kernel":
+            for level, flags in CPU_KERNEL_LEVELS:
+                obj = os.path.join(obj_dir, f"{name}_{level}.o")
+                out.append((base + flags + [f"-DIPKV_CPU_KERNEL=attend_chunk_{level}", "-c", src, "-o", obj], obj))
+        else:
+            obj = os.path.join(obj_dir, name + ".o")
+            out.append((base + ["-c", src, "-o", obj], obj))
+    return out
+
+
 def build(force=False, verbose=False):
     if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _deps_mtime():
         return LIB
@@ -33,10 +53,8 @@ def build(force=False, verbose=False):
         cmd = [NVCC] + FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", src, "-o", obj]
         procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
         objs.append(obj)
-    for src in sorted(glob.glob(os.path.join(CSRC, "*.cpp"))):          # host-only parts (the CPU-side engine)
-        obj = os.path.join(OBJ_DIR, os.path.basename(src)[:-4] + ".o")
-        cmd = ["g++", "-std=c++17", "-O3", "-fopenmp", "-fPIC", "-c", src, "-o", obj]
-        procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
+    for cmd, obj in cpu_engine_commands(OBJ_DIR):                       # host-only parts (the CPU-side engine)
+        procs.append((cmd[-3], subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
         objs.append(obj)
     failed = False
     for src, p in procs:

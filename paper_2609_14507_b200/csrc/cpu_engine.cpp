@@ -26,100 +26,37 @@
 
 namespace ipkvi {
 
+// cpu_engine_kernel.cpp, compiled per instruction-set level
+void attend_chunk_v4(const CpuShape&, const float*, int, int, const CpuRun*, int, int64_t, int64_t, float*, float*, float*);
+void attend_chunk_v3(const CpuShape&, const float*, int, int, const CpuRun*, int, int64_t, int64_t, float*, float*, float*);
+void attend_chunk_base(const CpuShape&, const float*, int, int, const CpuRun*, int, int64_t, int64_t, float*, float*, float*);
+
 namespace {
 
-constexpr int kTile = 16;          // tokens widened and scored at a time
-constexpr int kMaxDim = 576;
-constexpr int kMaxGroup = 128;     // query heads sharing one KV head (MLA: all heads)
+using ChunkFn = void (*)(const CpuShape&, const float*, int, int, const CpuRun*, int, int64_t, int64_t, float*, float*, float*);
 
-#if defined(__x86_64__) && defined(__GNUC__) && !defined(__clang__)
-#define IPKV_CLONES __attribute__((target_clones("avx512f", "avx2,fma", "default")))
-#else
-#define IPKV_CLONES
+ChunkFn pick_kernel() {
+#if defined(__x86_64__) && defined(__GNUC__)
+    __builtin_cpu_init();
+    if (__builtin_cpu_supports("avx512f") && __builtin_cpu_supports("avx512bw") && __builtin_cpu_supports("avx512dq") &&
+        __builtin_cpu_supports("avx512vl"))
+        return attend_chunk_v4;
+    if (__builtin_cpu_supports("avx2") && __builtin_cpu_supports("fma")) return attend_chunk_v3;
 #endif
-
-inline void widen(const uint16_t* src, float* dst, int n) {
-    for (int i = 0; i < n; ++i) {
-        const uint32_t w = uint32_t(src[i]) << 16;
-        std::memcpy(dst + i, &w, 4);
-    }
+    return attend_chunk_base;
 }
 
 struct Partial {            // online-softmax state of one (row, KV head, chunk): per head m, l; O is unnormalised
     std::vector<float> m, l, o;
 };
 
-// One item: tokens [t_begin, t_end) of the concatenated CPU-side runs of a row, for KV head g.
-IPKV_CLONES
-void attend_chunk(const CpuShape& sh, const float* qf /*[G][dqk], pre-scaled*/, int G, int g,
-                  const CpuRun* runs, int n_runs, int64_t t_begin, int64_t t_end, float* m, float* l, float* o) {
-    const int dqk = sh.dim_qk, dv = sh.dim_v;
-    const bool alias_v = sh.dim_v_stored == 0;
-    const int64_t head_bytes = int64_t(sh.bt) * (dqk + sh.dim_v_stored) * 2;
-    const int64_t block_bytes = head_bytes * sh.n_kv_heads;
-    alignas(64) float kf[kTile * kMaxDim];
-    alignas(64) float vf_store[kTile * kMaxDim];
-    float s[kMaxGroup][kTile];
-    for (int h = 0; h < G; ++h) { m[h] = -std::numeric_limits<float>::infinity(); l[h] = 0.f; }
-    std::fill(o, o + size_t(G) * dv, 0.f);
-
-    int64_t run_first = 0;                       // token index of the current run's first token
-    for (int r = 0; r < n_runs; ++r) {
-        const int64_t run_last = run_first + runs[r].n_tokens;
-        const int64_t lo = std::max(t_begin, run_first), hi = std::min(t_end, run_last);
-        for (int64_t t0 = lo; t0 < hi; t0 += kTile) {
-            const int nt = int(std::min<int64_t>(kTile, hi - t0));
-            // widen the tile's K rows (and V rows) once; every head of the group reuses them
-            for (int j = 0; j < nt; ++j) {
-                const int64_t rel = t0 + j - run_first;
-                const int64_t blk = rel / sh.bt, off = rel - blk * sh.bt;
-                const char* head = runs[r].blocks + blk * block_bytes + int64_t(g) * head_bytes;
-                widen(reinterpret_cast<const uint16_t*>(head + off * dqk * 2), kf + j * dqk, dqk);
-                if (!alias_v)
-                    widen(reinterpret_cast<const uint16_t*>(head + int64_t(sh.bt) * dqk * 2 + off * dv * 2), vf_store + j * dv, dv);
-            }
-            const float* vf = alias_v ? kf : vf_store;
-            const int vpitch = alias_v ? dqk : dv;
-            for (int h = 0; h < G; ++h) {
-                const float* qh = qf + size_t(h) * dqk;
-                float mx = -std::numeric_limits<float>::infinity();
-                for (int j = 0; j < nt; ++j) {
-                    const float* kr = kf + j * dqk;
-                    float acc = 0.f;
-#pragma omp simd reduction(+ : acc)
-                    for (int i = 0; i < dqk; ++i) acc += qh[i] * kr[i];
-                    s[h][j] = acc;
-                    mx = std::max(mx, acc);
-                }
-                const float mn = std::max(m[h], mx);
-                const float alpha = std::exp(m[h] - mn);          // exp(-inf) = 0 on the first tile
-                float* oh = o + size_t(h) * dv;
-                if (alpha != 1.f) {
-#pragma omp simd
-                    for (int c = 0; c < dv; ++c) oh[c] *= alpha;
-                }
-                float lsum = 0.f;
-                for (int j = 0; j < nt; ++j) {
-                    const float pj = std::exp(s[h][j] - mn);
-                    lsum += pj;
-                    const float* vr = vf + j * vpitch;
-#pragma omp simd
-                    for (int c = 0; c < dv; ++c) oh[c] += pj * vr[c];
-                }
-                l[h] = l[h] * alpha + lsum;
-                m[h] = mn;
-            }
-        }
-        run_first = run_last;
-    }
-}
-
 }  // namespace
 
 int cpu_attend_batch(const CpuShape& sh, int n_rows, const uint16_t* q, const CpuRun* runs, const int32_t* row_run_start,
                      float* o_out, float* lse_out, int n_threads) {
     const int G = sh.n_q_heads / sh.n_kv_heads;
-    if (G > kMaxGroup || sh.dim_qk > kMaxDim || sh.dim_v > kMaxDim) return -1;
+    if (G > kCpuMaxGroup || sh.dim_qk > kCpuMaxDim || sh.dim_v > kCpuMaxDim || sh.dim_qk % 16 != 0 || sh.dim_v % 16 != 0) return -1;
+    static const ChunkFn attend = pick_kernel();
     struct Item { int row, g; int64_t t0, t1; };
     std::vector<Item> items;
     std::vector<int> first_item(size_t(n_rows) * sh.n_kv_heads + 1, 0);
@@ -152,7 +89,7 @@ int cpu_attend_batch(const CpuShape& sh, int n_rows, const uint16_t* q, const Cp
         const Item& it = items[size_t(i)];
         Partial& p = parts[size_t(i)];
         p.m.resize(G); p.l.resize(G); p.o.resize(size_t(G) * sh.dim_v);
-        attend_chunk(sh, qf.data() + (size_t(it.row) * sh.n_q_heads + size_t(it.g) * G) * sh.dim_qk, G, it.g,
+        attend(sh, qf.data() + (size_t(it.row) * sh.n_q_heads + size_t(it.g) * G) * sh.dim_qk, G, it.g,
                      runs + row_run_start[it.row], row_run_start[it.row + 1] - row_run_start[it.row], it.t0, it.t1,
                      p.m.data(), p.l.data(), p.o.data());
     }

@@ -4,6 +4,9 @@
 
 namespace ipkvi {
 
+constexpr int kCpuMaxDim = 576;      // widest head dimension the tile kernel holds
+constexpr int kCpuMaxGroup = 128;    // most query heads sharing one KV head (compressed latent: all heads)
+
 struct CpuShape {
     int n_q_heads, n_kv_heads, dim_qk, dim_v;
     int dim_v_stored;     // 0 for the compressed-latent kind: V aliases the first dim_v columns of K

@@ -16,26 +16,36 @@ LIB = os.path.join(HERE, "libcpu_engine_shim.so")
 
 
 def _lib():
-    srcs = [os.path.join(HERE, "cpu_engine_shim.cpp"), os.path.join(CSRC, "cpu_engine.cpp")]
-    deps = srcs + [os.path.join(CSRC, "cpu_engine.h")]
+    from paper_2609_14507_b200 import build as lib_build
+    obj_dir = os.path.join(HERE, "..", "paper_2609_14507_b200", "build")
+    os.makedirs(obj_dir, exist_ok=True)
+    cmds = lib_build.cpu_engine_commands(obj_dir)
+    deps = [os.path.join(HERE, "cpu_engine_shim.cpp"), os.path.join(CSRC, "cpu_engine.h"), os.path.join(CSRC, "cpu_engine.cpp"),
+            os.path.join(CSRC, "cpu_engine_kernel.cpp")]
     if not os.path.exists(LIB) or os.path.getmtime(LIB) < max(os.path.getmtime(d) for d in deps):
+        for cmd, _ in cmds:
+            subprocess.run(cmd, check=True)
         tmp = LIB + ".tmp.%d" % os.getpid()
-        subprocess.run(["g++", "-O3", "-std=c++17", "-fopenmp", "-fPIC", "-shared", "-o", tmp] + srcs, check=True)
+        subprocess.run(["g++", "-O2", "-std=c++17", "-fopenmp", "-fPIC", "-shared", "-o", tmp, os.path.join(HERE, "cpu_engine_shim.cpp")] +
+                       [obj for _, obj in cmds], check=True)
         os.replace(tmp, LIB)
     return C.CDLL(LIB)
 
 
-def run_engine(sh, k, v, q, runs, bt, threads=0):
+def run_engine(sh, k, v, q, runs, bt, threads=0, reps=1, seconds=None):
     L = _lib()
     n = k.shape[0]
     o = np.zeros((sh.n_q_heads, sh.dim_v), np.float32)
     lse = np.zeros(sh.n_q_heads, np.float32)
     rt = np.asarray(runs, np.int64)
+    best = C.c_double()
     rc = L.shim_cpu_attend(sh.n_q_heads, sh.n_kv_heads, sh.dim_qk, sh.dim_v, bt, C.c_float(np.float32(sh.scale)), C.c_int64(n),
                            k.ctypes.data_as(C.c_void_p), None if v is None else v.ctypes.data_as(C.c_void_p), len(runs),
                            rt.ctypes.data_as(C.c_void_p), q.ctypes.data_as(C.c_void_p), o.ctypes.data_as(C.c_void_p),
-                           lse.ctypes.data_as(C.c_void_p), threads)
+                           lse.ctypes.data_as(C.c_void_p), threads, reps, C.byref(best))
     assert rc == 0, rc
+    if seconds is not None:
+        seconds.append(best.value)
     return o, lse
 
 
