@@ -1,8 +1,8 @@
 // CPU-side in-place attention over the unpinned compute region (Sec. 6.1): the engine that produces the
 // CPU partial (O, LSE) which ipkv_merge joins with the GPU partial.
 //
-// Follows the paper's CPU kernel in spirit, written for whatever vector width the host has (the compiler
-// clones the hot loop for AVX-512, AVX2 and baseline x86-64 and picks one at load time):
+// Follows the paper's CPU kernel in spirit, written for whatever vector width the host has (the tile kernel,
+// cpu_engine_kernel.cpp, is compiled for AVX-512, AVX2 + FMA and baseline x86-64; one is picked at first use):
 //   * zero-copy: K/V are read where write-time routing put them — PLAIN blocks of region U, per KV head
 //     K[bt][dqk] then V[bt][dv], addressed with strides, never gathered into a contiguous copy;
 //   * scores are never materialised beyond a 16-token tile; online softmax keeps a running max and sum per

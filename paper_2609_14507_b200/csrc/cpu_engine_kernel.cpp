@@ -25,7 +25,7 @@ constexpr int kMaxGroup = kCpuMaxGroup;
 
 
 // 16 fp32 lanes as one value: GCC lowers it to one AVX-512 register, two AVX2 registers or four SSE registers,
-// whichever the clone of the caller is compiled for.
+// whichever level this file is being compiled for.
 typedef float v16f __attribute__((vector_size(64)));
 typedef int32_t v16i __attribute__((vector_size(64)));
 
