@@ -23,6 +23,7 @@
 #include <cuda_bf16.h>
 
 #include "kernels.h"
+#include "launch.cuh"
 #include "ptx.cuh"
 #include "schedule.cuh"
 
@@ -97,6 +98,10 @@ __global__ void __launch_bounds__(kThreads, 2) attn_gqa_kernel(const GqaParams p
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     __syncthreads();
+    // Everything above may run while the previous kernel of the stream drains; the queries, the scheduling words and the
+    // partials' scratch belong to it until it has completed.
+    ptx::grid_dependency_wait();
+    ptx::grid_launch_dependents();
 
     bool ok = true;
     int it = 0;                      // tiles streamed so far by this CTA: stage = it % STAGES
@@ -431,8 +436,7 @@ cudaError_t launch_gqa(const AttnLaunch& a, cudaStream_t s) {
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
-    attn_gqa_kernel<D, STAGES, DUP><<<a.n_ctas, kThreads, smem, s>>>(p);
-    return cudaGetLastError();
+    return launch_overlapped(attn_gqa_kernel<D, STAGES, DUP>, a.n_ctas, kThreads, size_t(smem), s, p);
 }
 
 }  // namespace

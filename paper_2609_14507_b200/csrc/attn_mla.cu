@@ -25,6 +25,7 @@
 #include <cstdlib>
 
 #include "kernels.h"
+#include "launch.cuh"
 #include "ptx.cuh"
 
 namespace ipkvi {
@@ -95,6 +96,10 @@ __global__ void __launch_bounds__(kThreads, 1) attn_mla_kernel(const MlaParams p
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     __syncthreads();
+    // Everything above may run while the previous kernel of the stream drains (it may be the append that writes this
+    // launch's newest token, or the reduce that still reads the partials' scratch).
+    ptx::grid_dependency_wait();
+    ptx::grid_launch_dependents();
 
     bool ok = true;
     int it = 0;                      // tiles streamed so far by this CTA: stage = it % kStages
@@ -342,8 +347,7 @@ cudaError_t launch_attend_mla(const AttnLaunch& a, cudaStream_t s) {
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
-    attn_mla_kernel<<<a.n_ctas, kThreads, smem, s>>>(p);
-    return cudaGetLastError();
+    return launch_overlapped(attn_mla_kernel, a.n_ctas, kThreads, size_t(smem), s, p);
 }
 
 }  // namespace ipkvi

@@ -5,6 +5,8 @@
 //   tile_to_plain_kernel an evicted window batch, TILE -> PLAIN, on its way to the CPU-compute region
 // All three move 16-byte chunks; one thread per chunk, consecutive threads on consecutive source chunks.
 #include "kernels.h"
+#include "launch.cuh"
+#include "ptx.cuh"
 
 namespace ipkvi {
 
@@ -58,6 +60,8 @@ __global__ void tile_to_plain_kernel(BlockGeom g, const char* __restrict__ src, 
 
 __global__ void append_kernel(BlockGeom g, const uint4* __restrict__ k, const uint4* __restrict__ v,
                               char* __restrict__ w_base, AppendRows rows) {
+    ptx::grid_dependency_wait();       // launched so that it may come in under the previous kernel's tail (launch.cuh)
+    ptx::grid_launch_dependents();
     const int row = blockIdx.x;
     const int kc = g.dim_qk / 8, vc = g.dim_v_stored / 8;
     const int per_token = (kc + vc) * g.n_kv_heads;
@@ -123,8 +127,7 @@ cudaError_t launch_copy_spans(const CopySpans& spans, int n, cudaStream_t s) {
 cudaError_t launch_append(const BlockGeom& g, const void* k, const void* v, int /*dim_v_src*/, char* w_base,
                           const AppendRows& rows, int n_rows, cudaStream_t s) {
     if (n_rows <= 0) return cudaSuccess;
-    append_kernel<<<n_rows, 128, 0, s>>>(g, static_cast<const uint4*>(k), static_cast<const uint4*>(v), w_base, rows);
-    return cudaGetLastError();
+    return launch_overlapped(append_kernel, n_rows, 128, size_t(0), s, g, static_cast<const uint4*>(k), static_cast<const uint4*>(v), w_base, rows);
 }
 
 }  // namespace ipkvi

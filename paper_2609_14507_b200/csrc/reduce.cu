@@ -7,6 +7,8 @@
 #include <cuda_bf16.h>
 
 #include "kernels.h"
+#include "launch.cuh"
+#include "ptx.cuh"
 
 namespace ipkvi {
 
@@ -55,6 +57,8 @@ __global__ void __launch_bounds__(kReduceThreads, EXTRAS ? 4 : 5) split_reduce_k
     // the list of extra partials is requested together with the span range: one round of latency for both
     const int rg = row * p.n_gh + gh;
     const int sp0 = p.rg_span_start[rg], sp1 = p.rg_span_start[rg + 1];
+    ptx::grid_dependency_wait();        // the attention kernel's partials and lists are complete from here on
+    ptx::grid_launch_dependents();
     int list_entry = 0, list_count = 0;
     if (EXTRAS) {
         if (tid < kStealListCap) list_entry = p.extra_list[rg * kStealListCap + tid];
@@ -231,9 +235,8 @@ cudaError_t launch_split_reduce(const AttnLaunch& a, cudaStream_t s) {
     p.extra_count = a.steal_lists; p.extra_list = a.steal_lists ? a.steal_lists + a.n_rows * a.n_gh : nullptr; p.n_spans = a.n_spans;
     p.clear = a.steal_clear; p.clear_words = a.steal_clear ? a.steal_clear_words : 0;
     const size_t smem = size_t(kReduceThreads) * sizeof(float4);
-    if (p.extra_count) split_reduce_kernel<true><<<total, kReduceThreads, smem, s>>>(p);
-    else split_reduce_kernel<false><<<total, kReduceThreads, smem, s>>>(p);
-    return cudaGetLastError();
+    if (p.extra_count) return launch_overlapped(split_reduce_kernel<true>, total, kReduceThreads, smem, s, p);
+    return launch_overlapped(split_reduce_kernel<false>, total, kReduceThreads, smem, s, p);
 }
 
 cudaError_t launch_merge(const MergeLaunch& m, cudaStream_t s) {
