@@ -63,7 +63,9 @@ def _run_step_and_check(name, samples, kv_splits=0):
                     np.testing.assert_array_equal(kk, k[t])
                     if vv is not None:
                         np.testing.assert_array_equal(vv, v[t])
-        assert cache.get_stats()["device_status"] == 0
+        stats = cache.get_stats()
+        assert stats["device_status"] == 0
+        return stats
     finally:
         cache.close()
         torch.cuda.empty_cache()
@@ -83,6 +85,14 @@ def test_qwen3_32k_share_sweep_sampled():
             _run_step_and_check("_tmp", [(1, num)])
         finally:
             del bench.WORKLOADS["_tmp"]
+
+
+def test_qwen3_32k_streamed_load_reading_sampled():
+    """The load reading of the same configuration: half of every sequence's P share is not device-resident and comes
+    through the slot ring from pinned host memory while the resident rest is attended."""
+    stats = _run_step_and_check("qwen3-2layers-bs16-32k-stream50", [(0, 5), (1, 10)])
+    # half of 16 x 32 768 tokens x 2 048 bytes went through the slots for each of the two layers
+    assert stats["h2d_bytes"] >= 2 * 16 * 16000 * 2048
 
 
 def test_deepseek_mla_128k_sampled():
