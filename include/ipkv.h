@@ -161,6 +161,11 @@ ipkv_status ipkv_flush(ipkv_t* h, int32_t layer, int32_t seq, void* stream);
 /* The balancing is switched on by the library when the launch is long enough for it to pay (about 50 tiles of 64
  * tokens per CTA); this flag switches it on for any size (tests use it to exercise the path on small inputs). */
 #define IPKV_ATTEND_BALANCE 2
+/* Stream ordering.  The attention, split-reduce and append kernels are launched so that each may become resident while the previous
+ * kernel of its stream drains (programmatic dependent launch); it waits for that kernel to complete before it reads
+ * or writes anything a previous kernel could have touched, so the results are those of plain stream order, behind
+ * the library's own kernels and behind the caller's.  The environment variable IPKV_NO_LAUNCH_OVERLAP (any value,
+ * read once per process) restores plain launches. */
 
 typedef struct {
   int32_t kv_splits;   /* 0 = automatic; otherwise the number of sequence chunks per (sequence, KV head) */
