@@ -56,12 +56,12 @@ WORKLOADS = {
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention-kernel launch, from the ncu captures summarised under
 # profiles/ (captured on the 2-layer case, whose per-layer launch is the full-size workload's launch).
 DRAM_TRAFFIC_PER_LAUNCH = {
-    "mixtral-8x7b-bs16-32k-cpu25": 1615.2e6 + 5.6e6,        # profiles/attn_gqa_kernel_mixtral-2layers-bs16-32k-cpu25.md
-    "mixtral-2layers-bs16-32k-cpu25": 1615.2e6 + 5.6e6,
-    "qwen3-30b-a3b-bs16-32k-cpu0": 1076.1e6 + 5.5e6,        # profiles/attn_gqa_kernel_qwen3-2layers-bs16-32k-cpu0.md
-    "qwen3-2layers-bs16-32k-cpu0": 1076.1e6 + 5.5e6,
-    "deepseek-v2-lite-mla-bs8-128k-cpu40": 725.7e6 + 6.8e6,  # profiles/attn_mla_kernel_deepseek-v2-lite-2layers-bs8-128k-cpu40.md
-    "deepseek-v2-lite-mla-2layers-bs8-128k-cpu40": 725.7e6 + 6.8e6,
+    "mixtral-8x7b-bs16-32k-cpu25": 1615.2e6 + 5.3e6,        # profiles/attn_gqa_kernel_mixtral-2layers-bs16-32k-cpu25.md
+    "mixtral-2layers-bs16-32k-cpu25": 1615.2e6 + 5.3e6,
+    "qwen3-30b-a3b-bs16-32k-cpu0": 1076.1e6 + 4.6e6,        # profiles/attn_gqa_kernel_qwen3-2layers-bs16-32k-cpu0.md
+    "qwen3-2layers-bs16-32k-cpu0": 1076.1e6 + 4.6e6,
+    "deepseek-v2-lite-mla-bs8-128k-cpu40": 725.7e6 + 5.6e6,  # profiles/attn_mla_kernel_deepseek-v2-lite-2layers-bs8-128k-cpu40.md
+    "deepseek-v2-lite-mla-2layers-bs8-128k-cpu40": 725.7e6 + 5.6e6,
 }
 DEFAULT_WORKLOAD = "mixtral-8x7b-bs16-32k-cpu25"
 BLOCK, WINDOW = 64, 256
