@@ -383,7 +383,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--kv-splits", type=int, default=0)
     ap.add_argument("--no-read-ceiling", action="store_true", help="skip the read-only bandwidth probe reported in roofline.read_ceiling")
-    ap.add_argument("--time-every", type=int, default=4,
+    ap.add_argument("--time-every", type=int, default=13,
                     help="CUDA events around every N-th attention launch of the timed region (every launch does the same work; an event "
                          "between two kernels costs the step several microseconds, so bracketing all of them would slow what is measured)")
     ap.add_argument("--no-kernel-timing", action="store_true",
@@ -479,6 +479,8 @@ def main():
         step()
     barrier()
     st0 = cache.get_stats()
+    # short runs bracket more of their launches, so that at least about two dozen are timed
+    args.time_every = max(1, min(args.time_every, args.steps * sh.n_layers // 24))
     cache.profile_enable(not args.no_kernel_timing, reduce=args.profile_reduce, every=args.time_every)
     cache.profile_read()
     sampler.mark()
