@@ -546,41 +546,50 @@ def main():
         dq = torch.empty_like(q); dk = torch.empty_like(k_new); dvn = None if v_new is None else torch.empty_like(v_new)
         doc = torch.empty_like(o_cpu); dlc = torch.empty_like(lse_cpu)
 
-        # The copies run on a stream of their own, in four groups of layers: the layers of a group start as soon as the
-        # group's inputs have landed, so only the first group's copies (and the last group's read-back) are not hidden
+        # The copies run on a stream of their own, in groups of layers: the layers of a group start as soon as the
+        # group's inputs have landed, so only the first group's copies and the last group's read-back are not hidden
         # behind the other groups' kernels, the way a server overlaps its transfers with the previous layers' work.
+        # Those two groups are therefore small (one layer in front, two at the end).
         cs = torch.cuda.Stream()
-        n_groups = min(4, NL)
-        bounds = [NL * g // n_groups for g in range(n_groups + 1)]
+        bounds = sorted({0, min(1, NL), min(4, NL), max(NL // 2, min(4, NL)), max(NL - 2, NL // 2), NL})
+        n_groups = len(bounds) - 1
         landed = [torch.cuda.Event() for _ in range(n_groups)]
         computed = [torch.cuda.Event() for _ in range(n_groups)]
         step_done = torch.cuda.Event()
 
+        def copy_in(g):
+            lo, hi = bounds[g], bounds[g + 1]
+            with torch.cuda.stream(cs):
+                dq[lo:hi].copy_(hq[lo:hi], non_blocking=True)
+                dk[lo:hi].copy_(hk[lo:hi], non_blocking=True)
+                if dvn is not None:
+                    dvn[lo:hi].copy_(hv[lo:hi], non_blocking=True)
+                doc[lo:hi].copy_(hoc[lo:hi], non_blocking=True)
+                dlc[lo:hi].copy_(hlc[lo:hi], non_blocking=True)
+                landed[g].record(cs)
+
+        def run_layer(layer):
+            app = {} if args.separate_append else dict(append_k=dk[layer], append_v=None if dvn is None else dvn[layer])
+            if args.separate_append:
+                cache.append(layer, seq_ids, dk[layer], None if dvn is None else dvn[layer], stream=cur)
+            if fused:
+                cache.attend_gpu(layer, seq_ids, dq[layer], out[layer], out_lse, kv_splits=args.kv_splits, static_schedule=args.static_schedule, stream=cur,
+                                 fold_o=doc[layer], fold_lse=dlc[layer], **app)
+            else:
+                cache.attend_gpu(layer, seq_ids, dq[layer], o_part, lse_part, kv_splits=args.kv_splits, static_schedule=args.static_schedule, stream=cur, **app)
+                cache.merge(B * Hq, dv, [o_part.view(B * Hq, dv), doc[layer]], [lse_part.view(-1), dlc[layer]],
+                            out[layer], out_lse, out_is_bf16=True, stream=cur)
+
         def step_e2e():
             cs.wait_event(step_done)                     # the previous step's kernels no longer read the input buffers
-            with torch.cuda.stream(cs):
-                for g in range(n_groups):
-                    lo, hi = bounds[g], bounds[g + 1]
-                    dq[lo:hi].copy_(hq[lo:hi], non_blocking=True)
-                    dk[lo:hi].copy_(hk[lo:hi], non_blocking=True)
-                    if dvn is not None:
-                        dvn[lo:hi].copy_(hv[lo:hi], non_blocking=True)
-                    doc[lo:hi].copy_(hoc[lo:hi], non_blocking=True)
-                    dlc[lo:hi].copy_(hlc[lo:hi], non_blocking=True)
-                    landed[g].record(cs)
+            copy_in(0)
             for g in range(n_groups):
                 cur.wait_event(landed[g])
-                for layer in range(bounds[g], bounds[g + 1]):
-                    app = {} if args.separate_append else dict(append_k=dk[layer], append_v=None if dvn is None else dvn[layer])
-                    if args.separate_append:
-                        cache.append(layer, seq_ids, dk[layer], None if dvn is None else dvn[layer], stream=cur)
-                    if fused:
-                        cache.attend_gpu(layer, seq_ids, dq[layer], out[layer], out_lse, kv_splits=args.kv_splits, static_schedule=args.static_schedule, stream=cur,
-                                         fold_o=doc[layer], fold_lse=dlc[layer], **app)
-                    else:
-                        cache.attend_gpu(layer, seq_ids, dq[layer], o_part, lse_part, kv_splits=args.kv_splits, static_schedule=args.static_schedule, stream=cur, **app)
-                        cache.merge(B * Hq, dv, [o_part.view(B * Hq, dv), doc[layer]], [lse_part.view(-1), dlc[layer]],
-                                    out[layer], out_lse, out_is_bf16=True, stream=cur)
+                run_layer(bounds[g])
+                if g + 1 < n_groups:
+                    copy_in(g + 1)                       # issued once this group has a kernel queued: the device never waits for the host here
+                for layer in range(bounds[g] + 1, bounds[g + 1]):
+                    run_layer(layer)
                 computed[g].record(cur)
                 with torch.cuda.stream(cs):
                     cs.wait_event(computed[g])
