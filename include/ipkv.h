@@ -262,6 +262,8 @@ typedef struct {
   uint64_t h2d_bytes, d2h_bytes, d2d_bytes;
   uint64_t flushes, flushes_to_u;
   uint64_t fused_appends;       /* ipkv_attend_gpu calls whose kernel wrote the appended rows itself     */
+  uint64_t early_launches;      /* attention launches allowed to fill their copy ring before the previous kernel
+                                   of the stream had completed (no K/V byte they read could still be in flight) */
   /* IPKV_FLAG_GROW_P: segments pinned so far, their bytes, the page-locking time spent (by create for the
      first, by the helper thread for the rest), and how often / how long a call had to wait for a segment
      that was not pinned yet (0 when the one-window lookahead covers the pinning, as Sec. 7.7 expects).  */

@@ -58,7 +58,7 @@ class Extent(C.Structure):
 class Stats(C.Structure):
     _fields_ = [(n, C.c_uint64) for n in (
         "attend_calls", "attend_kernels", "reduce_kernels", "merge_kernels", "append_kernels", "pack_kernels",
-        "kv_bytes_attended", "h2d_bytes", "d2h_bytes", "d2d_bytes", "flushes", "flushes_to_u", "fused_appends",
+        "kv_bytes_attended", "h2d_bytes", "d2h_bytes", "d2d_bytes", "flushes", "flushes_to_u", "fused_appends", "early_launches",
         "p_segments", "p_pinned_bytes", "p_pin_us", "p_grow_waits", "p_grow_wait_us",
         "p_register_us", "p_register_calls", "p_register_max_us")] + [("device_status", C.c_uint32)]
 

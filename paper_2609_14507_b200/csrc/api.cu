@@ -160,6 +160,14 @@ struct ipkv {
     cudaEvent_t ev_main = nullptr;
     cudaEvent_t ev_p_host = nullptr;       // after the last copy into P's host memory that a compute stream carried (prefill)
     bool ev_p_host_set = false;
+    // Which attention launches may start their first copies before the previous kernel of the stream has completed
+    // (AttnLaunch::early_tiles).  launch_seq counts the attention launches enqueued so far; kv_written_at[layer] is the
+    // value it must have reached before a launch on that layer may do so: one whole attention + reduce pair has then
+    // been enqueued, on the same stream, after the last operation that wrote the layer's device-side K/V.
+    uint64_t launch_seq = 0;
+    std::vector<uint64_t> kv_written_at;
+    cudaStream_t launch_stream = nullptr;
+    bool launch_stream_valid = false;
     ipkv_stats stats;
     std::string err;
     // optional kernel timing
@@ -453,7 +461,16 @@ void CUDART_CB bounce_to_unpinned(void* arg) {
 // stay flat. Neighbouring sequences with the same destination are handled by one launch / one copy (a batch that
 // advances in lockstep evicts every sequence of a layer to the same side). Host contents are complete once the
 // copy stream has drained (sync_host()).
+// Something is about to write device-side K/V of `layer` (all layers if negative): a standalone operation, or with
+// `inside_launch` the next attention launch itself (fused append).
+void note_kv_write(ipkv* h, int layer, bool inside_launch = false) {
+    const uint64_t at = h->launch_seq + 1 + (inside_launch ? 1 : 0);
+    for (int l = 0; l < int(h->kv_written_at.size()); ++l)
+        if (layer < 0 || l == layer) h->kv_written_at[l] = std::max(h->kv_written_at[l], at);
+}
+
 ipkv_status flush_layer(ipkv* h, int layer, const int* seqs_in, int n, cudaStream_t s) {
+    note_kv_write(h, layer);
     const bool no_u = h->cfg.flags & IPKV_FLAG_NO_HOST_U, no_p = h->cfg.flags & IPKV_FLAG_NO_HOST_P;
     struct Job { int seq; Run r; int64_t nb; };
     std::vector<int> seqs(seqs_in, seqs_in + n);
@@ -674,7 +691,8 @@ void fill_launch(AttnLaunch* a, int kind, int Hq, int Hkv, int dqk, int dv, int 
 // One group of segments for all rows: attention + split reduce, folding into (out_o, out_lse) when `fold`.
 ipkv_status run_group(ipkv* h, const std::vector<std::vector<PlanSeg>>& rows, const char* const bases[kMaxBases],
                       const void* q, int kv_splits, const float* fold_o, const float* fold_lse, float* out_o, float* out_lse,
-                      cudaStream_t s, int schedule_flags = 0, const void* append_k = nullptr, const void* append_v = nullptr) {
+                      cudaStream_t s, int schedule_flags = 0, const void* append_k = nullptr, const void* append_v = nullptr,
+                      int layer = -1, bool device_resident_only = false) {
     const ipkv_config& c = h->cfg;
     Plan plan;
     const PartGeom pg = part_geom(c.kind, c.n_q_heads, c.n_kv_heads);
@@ -716,6 +734,15 @@ ipkv_status run_group(ipkv* h, const std::vector<std::vector<PlanSeg>>& rows, co
     a.status = h->status_dev;
     a.append_k = append_k; a.append_v = append_v;
     if (a.n_spans > 0) {
+        // may this launch fill its copy ring before the previous kernel has completed? (see ipkv::kv_written_at)
+        if (!h->launch_stream_valid || h->launch_stream != s) {
+            note_kv_write(h, -1);                   // another stream: nothing is known about what ran before
+            h->launch_stream = s; h->launch_stream_valid = true;
+        }
+        a.early_tiles = (!balance && c.kind == IPKV_GQA && device_resident_only && layer >= 0 && h->launch_seq >= h->kv_written_at[layer]) ? 1 : 0;
+        if (append_k && layer >= 0) note_kv_write(h, layer, true);     // the kernel itself writes the new rows into the window
+        h->stats.early_launches += uint64_t(a.early_tiles);
+        h->launch_seq += 1;
         const bool sampled = h->prof_on && (h->prof_seen++ % h->prof_stride) == 0;
         const bool timed = sampled && !h->prof_reduce && h->prof_used + 2 <= h->prof_ev.size();
         if (timed) CU(h, cudaEventRecord(h->prof_ev[h->prof_used], s));
@@ -869,6 +896,7 @@ ipkv_status ipkv_create(const ipkv_config* cfg, ipkv_t** out) {
         if (i >= 2 && cudaMemset(*dst[i], 0, h->sizes[i]) != cudaSuccess) return bail(IPKV_ECUDA);
     }
     h->st.resize(size_t(cfg->n_layers) * cfg->max_seqs);
+    h->kv_written_at.assign(size_t(cfg->n_layers), 0);
     for (auto& s : h->st) s.router.init(cfg->block_tokens, cfg->window_tokens, cfg->share_num, cfg->share_den);
 
     if (cudaMalloc(&h->status_dev, 256) != cudaSuccess) return bail(IPKV_ENOMEM);
@@ -931,6 +959,7 @@ ipkv_status ipkv_append_bulk(ipkv_t* h, int32_t layer, int32_t seq, const void* 
     if (n_tokens > 0 && (!k_dev || (c.kind == IPKV_GQA && !v_dev))) return fail(h, IPKV_EINVAL, "K/V pointer is NULL");
     SeqState& st = h->state(layer, seq);
     if (st.router.length() != 0) return fail(h, IPKV_ESTATE, "bulk append is only legal on an empty sequence");
+    note_kv_write(h, layer);
     const int64_t bt = c.block_tokens;
     const int64_t n_cpu = st.router.prefill_cpu_tokens(n_tokens, num0, den0);
     const int64_t n_gpu = n_tokens - n_cpu;
@@ -1052,6 +1081,7 @@ ipkv_status append_tokens(ipkv* h, int32_t layer, const int32_t* seq_ids, int32_
             rows.slot[i] = int32_t(st.router.stage());
         }
         if (defer_copy) continue;
+        note_kv_write(h, layer);
         const char* ks = static_cast<const char*>(k_dev) + base * k_row;
         const char* vs = v_dev ? static_cast<const char*>(v_dev) + base * v_row : nullptr;
         CU(h, launch_append(h->geom, ks, vs, c.dim_v, h->w_layer(layer), rows, n, s));
@@ -1131,7 +1161,7 @@ ipkv_status ipkv_attend_gpu(ipkv_t* h, int32_t layer, const int32_t* seq_ids, in
     const float* fold_lse = opts ? opts->fold_lse_dev : nullptr;
     if ((fold_o == nullptr) != (fold_lse == nullptr)) return fail(h, IPKV_EINVAL, "fold_o_dev and fold_lse_dev must be given together");
     ipkv_status rc = run_group(h, rows, bases, q_dev, kv_splits, fold_o, fold_lse, o_part_dev, lse_part_dev, s, static_schedule,
-                               fused_append ? app_k : nullptr, fused_append ? app_v : nullptr);
+                               fused_append ? app_k : nullptr, fused_append ? app_v : nullptr, layer, true);
     if (rc != IPKV_OK) return rc;
     if (max_stream_chunks == 0) return IPKV_OK;
 

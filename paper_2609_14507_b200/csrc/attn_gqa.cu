@@ -53,6 +53,7 @@ struct GqaParams {
     int32_t* lists;      // per (row, head group): the number of extra partials CTAs filled for it [n_rows * n_gh], then their indices
                          // [n_rows * n_gh][kStealListCap] (all zero at launch); null = no CTA helps another
     int n_spans, n_ctas, n_rows, n_gh;
+    int early;          // the producer may issue its first copies before the previous kernel of the stream has completed
     int Hq, G, n_hg, RG;
     int bt;
     int64_t head_bytes, block_bytes;
@@ -100,8 +101,14 @@ __global__ void __launch_bounds__(kThreads, 2) attn_gqa_kernel(const GqaParams p
     __syncthreads();
     // Everything above may run while the previous kernel of the stream drains; the queries, the scheduling words and the
     // partials' scratch belong to it until it has completed.
-    ptx::grid_dependency_wait();
-    ptx::grid_launch_dependents();
+    // With the fixed schedule and a host that vouches for the K/V bytes (GqaParams::early), the producer does not wait
+    // here: it fills the ring first and waits before its first refill, so the copies' latency overlaps the previous
+    // kernel's drain as well. (The balanced schedule claims its tiles from words that kernel may still clear.)
+    const bool early = p.early && !dynamic;
+    if (!(early && warp == kConsumerWarps)) {
+        ptx::grid_dependency_wait();
+        ptx::grid_launch_dependents();      // only ever after a wait has returned: the next kernel's start then implies the previous one's end
+    }
 
     bool ok = true;
     int it = 0;                      // tiles streamed so far by this CTA: stage = it % STAGES
@@ -114,7 +121,9 @@ __global__ void __launch_bounds__(kThreads, 2) attn_gqa_kernel(const GqaParams p
             int cached_sp = -1;
             Seg seg{};
             const char* seg_base = nullptr;
+            bool waited = !early;
             auto issue = [&](int sp, const Span& span, int tile, int slot) -> bool {
+                if (!waited && it >= STAGES) { ptx::grid_dependency_wait(); waited = true; }
                 if (sp != cached_sp) {                             // first tile of a span: where its run lives
                     seg = p.segs[span.seg];
                     seg_base = p.bases[seg.base_id & kSegBaseMask] + seg.off + int64_t(span.gh / p.n_hg) * p.head_bytes;
@@ -420,6 +429,7 @@ cudaError_t launch_gqa(const AttnLaunch& a, cudaStream_t s) {
     p.append_k = static_cast<const __nv_bfloat16*>(a.append_k); p.append_v = static_cast<const __nv_bfloat16*>(a.append_v);
     p.next = a.steal_next; p.lists = a.steal_lists; p.n_spans = a.n_spans; p.n_ctas = a.n_ctas; p.cta_tiles = a.cta_tiles;
     p.n_rows = a.n_rows; p.n_gh = a.n_gh;
+    p.early = a.early_tiles;
     p.Hq = a.n_q_heads; p.G = a.n_q_heads / a.n_kv_heads;
     p.n_hg = (p.G + 15) / 16;
     p.RG = part_geom(0, a.n_q_heads, a.n_kv_heads).rows_per_group;

@@ -53,6 +53,8 @@ struct AttnLaunch {
     uint32_t* status;               // device word, OR-ed with an error bit if a bounded wait gives up
     const void* append_k;           // fused append: [n_rows][n_kv_heads][dim_qk] bf16 new K rows (null: none)
     const void* append_v;           // [n_rows][n_kv_heads][dim_v]
+    int early_tiles;                // 1: no K/V byte this launch reads was written by the kernel before it in the stream, so the
+                                    // first copies may be issued before that kernel has completed (see launch.cuh)
     // Dynamic load balancing of the GQA kernel (all null = static schedule with bit-reproducible results): a CTA
     // that has finished its chunk takes tiles from the spans that are furthest behind and accumulates them into
     // extra partials of its own, stored after the spans' partials (kStealSlots per CTA) and listed per (row, head group).

@@ -634,3 +634,80 @@ def test_fused_append_writes_the_window_and_attends_the_new_token(G, dim, bt):
             check_contents(cache, 0, s, refs[s], range(0, len(refs[s].route), 3))
         st = cache.get_stats()
         assert st["device_status"] == 0 and st["fused_appends"] == 3 * bt + 5 and st["append_kernels"] == 0
+
+
+def test_early_copy_start_reads_no_stale_bytes():
+    """Fixed-schedule launches fill their copy ring before the previous kernel of the stream has completed when the
+    library knows that nothing they read can still be in flight.  Two identical caches take the same decode steps
+    (fused appends, evictions, an occasional separate append, three layers): one on a single stream, where that
+    applies, one hopping between two event-ordered streams, where it never does.  The fixed schedule is
+    bit-reproducible, so every output must be identical bit for bit; some steps are also checked against the oracle."""
+    hkv, G, dim, bt, NL = 2, 4, 128, 64, 3
+    sh = synth.Shape("early", "gqa", NL, hkv * G, hkv, dim, dim, dim ** -0.5)
+    lens = [900, 64, 333, 1]
+    scale = float(np.float32(sh.scale))
+    kw = dict(block_tokens=bt, window_tokens=2 * bt, chunk_tokens=4 * bt, max_u_tokens_per_seq=1024, max_p_tokens_per_seq=2048,
+              resident_tokens_per_seq=2048, share_num=1, share_den=3)
+    with make_cache(sh, NL, len(lens), **kw) as ca, make_cache(sh, NL, len(lens), **kw) as cb:
+        refs = []
+        for s, n in enumerate(lens):
+            r = [RefSeq(sh, bt, 2 * bt, 1, 3) for _ in range(NL)]
+            for layer in range(NL):
+                k, v = synth.host_kv(sh, n, seed=7700 + 10 * s + layer)
+                for c in (ca, cb):
+                    c.append_bulk(layer, s, synth.bits_to_torch(k, DEV), synth.bits_to_torch(v, DEV), n, 1, 3)
+                r[layer].bulk(k, v, 1, 3)
+            refs.append(r)
+        torch.cuda.synchronize()
+        rng = np.random.default_rng(4242)
+        seqs = list(range(len(lens)))
+        n_steps = 2 * bt + 9                                # two evictions per sequence
+        plan = []                                           # (layer, separate append?, host k, v, q, device k, v, q)
+        for step in range(n_steps):
+            for layer in range(NL):
+                k = synth.normal_bf16(rng, (len(lens), hkv, dim)); v = synth.normal_bf16(rng, (len(lens), hkv, dim))
+                q = synth.normal_bf16(rng, (len(lens), hkv * G, dim))
+                plan.append((layer, step % 7 == 3 and layer == 1, k, v, q,
+                             synth.bits_to_torch(k, DEV), synth.bits_to_torch(v, DEV), synth.bits_to_torch(q, DEV)))
+        s0 = torch.cuda.Stream(); s1 = torch.cuda.Stream()
+        torch.cuda.synchronize()
+
+        def run(c, hopping):
+            """All launches back to back, no host synchronisation in between."""
+            outs, hop, ev = [], 0, torch.cuda.Event()
+            ev.record(s0)
+            for layer, separate, _, _, _, kd, vd, qd in plan:
+                st = s0
+                if hopping:                                 # change stream on every launch, ordered by an event
+                    st = (s0, s1)[hop]; hop ^= 1
+                    st.wait_event(ev)
+                with torch.cuda.stream(st):
+                    o = torch.zeros((len(lens), hkv * G, dim), device=DEV); lse = torch.zeros((len(lens), hkv * G), device=DEV)
+                    if separate:                            # now and then the append is a call of its own
+                        c.append(layer, seqs, kd, vd, stream=st)
+                        c.attend_gpu(layer, seqs, qd, o, lse, static_schedule=True, stream=st)
+                    else:
+                        c.attend_gpu(layer, seqs, qd, o, lse, static_schedule=True, append_k=kd, append_v=vd, stream=st)
+                    o.record_stream(st); lse.record_stream(st)
+                if hopping:
+                    ev.record(st)
+                outs.append((o, lse))
+            torch.cuda.synchronize()
+            return outs
+
+        outs_a = run(ca, False)
+        outs_b = run(cb, True)
+        n_launch = len(plan)
+        for i, (layer, _, k, v, q, _, _, _) in enumerate(plan):
+            for s in seqs:
+                refs[s][layer].append(k[s:s + 1], v[s:s + 1])
+            assert torch.equal(outs_a[i][0], outs_b[i][0]) and torch.equal(outs_a[i][1], outs_b[i][1]), f"launch {i} layer {layer}"
+            if i % 61 == 0 or i >= n_launch - NL:
+                parts = [refs[s][layer].attend(q[s], "gpu", scale) for s in seqs]
+                check_partial(outs_a[i][0].cpu().numpy(), outs_a[i][1].cpu().numpy(), np.stack([p[0] for p in parts]),
+                              np.stack([p[1] for p in parts]), f"launch {i} layer {layer}")
+        sa, sb = ca.get_stats(), cb.get_stats()
+        assert sa["device_status"] == 0 and sb["device_status"] == 0
+        assert sb["early_launches"] == 0
+        # on one stream most launches qualify: all but the first ones, those right after an eviction or a separate append
+        assert sa["early_launches"] > n_launch // 2
