@@ -164,8 +164,10 @@ ipkv_status ipkv_flush(ipkv_t* h, int32_t layer, int32_t seq, void* stream);
 /* Stream ordering.  The attention, split-reduce and append kernels are launched so that each may become resident while the previous
  * kernel of its stream drains (programmatic dependent launch); it waits for that kernel to complete before it reads
  * or writes anything a previous kernel could have touched, so the results are those of plain stream order, behind
- * the library's own kernels and behind the caller's.  The environment variable IPKV_NO_LAUNCH_OVERLAP (any value,
- * read once per process) restores plain launches. */
+ * the library's own kernels and behind the caller's.  An attention launch whose K/V bytes the library knows to be
+ * settled (nothing it enqueued since the launch before the previous one wrote them) also starts its first copies
+ * before that wait.  The environment variables IPKV_NO_LAUNCH_OVERLAP and IPKV_NO_EARLY_COPIES (any value, read once
+ * per process) restore plain launches / switch the early copies off. */
 
 typedef struct {
   int32_t kv_splits;   /* 0 = automatic; otherwise the number of sequence chunks per (sequence, KV head) */

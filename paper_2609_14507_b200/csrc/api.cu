@@ -739,7 +739,8 @@ ipkv_status run_group(ipkv* h, const std::vector<std::vector<PlanSeg>>& rows, co
             note_kv_write(h, -1);                   // another stream: nothing is known about what ran before
             h->launch_stream = s; h->launch_stream_valid = true;
         }
-        a.early_tiles = (!balance && c.kind == IPKV_GQA && device_resident_only && layer >= 0 && h->launch_seq >= h->kv_written_at[layer]) ? 1 : 0;
+        static const bool early_allowed = std::getenv("IPKV_NO_EARLY_COPIES") == nullptr;
+        a.early_tiles = (early_allowed && c.kind == IPKV_GQA && device_resident_only && layer >= 0 && h->launch_seq >= h->kv_written_at[layer]) ? 1 : 0;
         if (append_k && layer >= 0) note_kv_write(h, layer, true);     // the kernel itself writes the new rows into the window
         h->stats.early_launches += uint64_t(a.early_tiles);
         h->launch_seq += 1;

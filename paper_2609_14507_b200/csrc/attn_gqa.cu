@@ -101,10 +101,11 @@ __global__ void __launch_bounds__(kThreads, 2) attn_gqa_kernel(const GqaParams p
     __syncthreads();
     // Everything above may run while the previous kernel of the stream drains; the queries, the scheduling words and the
     // partials' scratch belong to it until it has completed.
-    // With the fixed schedule and a host that vouches for the K/V bytes (GqaParams::early), the producer does not wait
-    // here: it fills the ring first and waits before its first refill, so the copies' latency overlaps the previous
-    // kernel's drain as well. (The balanced schedule claims its tiles from words that kernel may still clear.)
-    const bool early = p.early && !dynamic;
+    // With a host that vouches for the K/V bytes (GqaParams::early) the producer does not wait here: it fills the ring
+    // first, so the copies' latency overlaps the previous kernel's drain as well, and waits before its first refill
+    // (fixed schedule) or before its first claim (balanced schedule: the scheduling words may still be being cleared by
+    // that kernel, so the first tiles of every chunk are its owner's without a claim).
+    const bool early = p.early != 0;
     if (!(early && warp == kConsumerWarps)) {
         ptx::grid_dependency_wait();
         ptx::grid_launch_dependents();      // only ever after a wait has returned: the next kernel's start then implies the previous one's end
@@ -192,7 +193,8 @@ __global__ void __launch_bounds__(kThreads, 2) attn_gqa_kernel(const GqaParams p
             sched.next = p.next; sched.lists = p.lists; sched.part_lse = p.part_lse;
             sched.n_spans = p.n_spans; sched.n_ctas = p.n_ctas; sched.n_rows = p.n_rows; sched.n_gh = p.n_gh;
             sched.lse_per_partial = kConsumerWarps * p.RG;
-            ok = produce_tiles(sched, lane, issue);
+            sched.head_tiles = (early && dynamic) ? STAGES : 0;
+            ok = produce_tiles(sched, lane, issue, [&]() { if (!waited) { ptx::grid_dependency_wait(); waited = true; } });
             if (lane == 0) {
                 if (!ok) atomicOr(p.status, kStatusNoFreeStage);
                 // tell the consumers that nothing follows

@@ -41,12 +41,17 @@ struct SchedParams {
     float* part_lse;
     int n_spans, n_ctas, n_rows, n_gh;
     int lse_per_partial;        // LSE values of one span's partial(s): parts_per_span * rows_per_group
+    int head_tiles;             // dynamic schedule: this many tiles at the start of every CTA's chunk (of its first span) are the
+                                // owner's without a claim, so that it can stream them before it may touch the scheduling words;
+                                // the span's counter then counts the tiles after them.  0 = every tile is claimed
 };
 
 // Runs in the producer warp (all 32 lanes).  issue(span_index, span, tile, slot) -> bool streams one tile (called by
-// lane 0 only; false after a timed-out wait).  Returns false after a timeout.
-template <class Issue>
-__device__ __forceinline__ bool produce_tiles(const SchedParams& p, int lane, Issue&& issue) {
+// lane 0 only; false after a timed-out wait).  settle() is called by every lane before its first access to the
+// scheduling words (it waits for the previous kernel of the stream unless the lane has done so already).  Returns
+// false after a timeout.
+template <class Issue, class Settle>
+__device__ __forceinline__ bool produce_tiles(const SchedParams& p, int lane, Issue&& issue, Settle&& settle) {
     const bool dynamic = p.next != nullptr;
     const int span_begin = p.cta_span_start[blockIdx.x], span_end = p.cta_span_start[blockIdx.x + 1];
     bool ok = true;
@@ -62,25 +67,36 @@ __device__ __forceinline__ bool produce_tiles(const SchedParams& p, int lane, Is
                 if (!issue(sp, span, span.tile0 + t, slot)) return -1;
             return n;
         }
-        // the owner takes an eighth of what is left per claim, a helper a quarter
+        // the chunk's first tiles are its owner's without a claim (head_tiles): streamed before anything else
+        const int head = sp == p.cta_span_start[chunk] ? min(p.head_tiles, span.ntiles) : 0;
+        if (head > 0 && !helping) {
+            for (int t = 0; t < head; ++t, ++n)
+                if (!issue(sp, span, span.tile0 + t, slot)) return -1;
+            settle();
+            atomicAdd(p.next + p.n_spans + chunk, head);     // they count as claimed for CTAs looking for work
+        }
+        settle();
+        // the owner takes an eighth of what is left per claim, a helper a quarter; the counter counts the tiles after the head
+        const int avail = span.ntiles - head;
         const int shift = helping ? 2 : 3;
         auto batch = [shift](int left) { const int b = left >> shift; return b > 8 ? 8 : (b < 1 ? 1 : b); };
-        int b = batch(span.ntiles - *reinterpret_cast<volatile int32_t*>(p.next + sp));
+        int b = batch(avail - *reinterpret_cast<volatile int32_t*>(p.next + sp));
         int t0 = atomicAdd(p.next + sp, b);
-        while (t0 < span.ntiles) {
-            const int first = t0, last = min(t0 + b, span.ntiles);
-            const int left = span.ntiles - last;           // as far as this CTA knows
+        while (t0 < avail) {
+            const int first = t0, last = min(t0 + b, avail);
+            const int left = avail - last;                 // as far as this CTA knows
             b = batch(left);
-            t0 = left > 0 ? atomicAdd(p.next + sp, b) : span.ntiles;
+            t0 = left > 0 ? atomicAdd(p.next + sp, b) : avail;
             atomicAdd(p.next + p.n_spans + chunk, last - first);     // what is left of the chunk, for CTAs looking for work
             for (int t = first; t < last; ++t, ++n)
-                if (!issue(sp, span, span.tile0 + t, slot)) return -1;
+                if (!issue(sp, span, span.tile0 + head + t, slot)) return -1;
         }
         return n;
     };
     // own chunk first: the partial of a span lives at the span's index
     if (lane == 0)
         for (int sp = span_begin; sp < span_end && ok; ++sp) ok = drain(sp, int(blockIdx.x), sp, false) >= 0;
+    settle();
     // then help the CTAs that are behind (some SMs get less of the memory bandwidth than others): pick the chunk with
     // the most unclaimed tiles per CTA already working on it, take tiles from the span its owner will reach last,
     // and accumulate them into one of this CTA's extra partials
@@ -127,7 +143,7 @@ __device__ __forceinline__ bool produce_tiles(const SchedParams& p, int lane, Is
                 atomicAdd(helpers + victim, 1);
                 sp = p.cta_span_start[victim + 1] - 1;
                 const int sp_first = p.cta_span_start[victim];
-                while (sp >= sp_first && __ldcg(p.next + sp) >= p.spans[sp].ntiles) --sp;
+                while (sp >= sp_first && __ldcg(p.next + sp) >= p.spans[sp].ntiles - (sp == sp_first ? min(p.head_tiles, p.spans[sp].ntiles) : 0)) --sp;
                 if (sp < sp_first) sp = -1;
                 if (sp >= 0) {
                     const int rg = p.spans[sp].row * p.n_gh + p.spans[sp].gh;
