@@ -10,6 +10,11 @@
 // of its own (kStealSlots per CTA, entered in the list of the span's (row, head group), where the reduce finds it).  A
 // partial is an exact softmax state over whatever set of tokens went into it, so any assignment of tiles to partials
 // gives the same attention; only the fp32 summation order changes.  No CTA ever waits for another one.
+//
+// Head tiles.  When the launch may start its copies before the previous kernel of the stream has completed (see
+// launch.cuh), the scheduling words cannot be touched yet: that kernel may still be clearing them.  The first
+// head_tiles tiles of every chunk then belong to the chunk's owner without a claim, the counter of the chunk's first
+// span counts the tiles after them, and a producer streams its head tiles, waits, and claims only afterwards.
 #pragma once
 #include <cstdint>
 
