@@ -642,7 +642,9 @@ def main():
                        "l2": l2_note,
                        "multi_gpu": "replicas only", "kv_splits": args.kv_splits, "kernel_timing": "CUDA events around every %d%s attention launch" % (args.time_every, "th" if args.time_every != 1 else "st"), "schedule": "static" if args.static_schedule else "dynamic balancing (GQA kernel, launches of at least 48 tiles per CTA)",
                        "merge": "inside the split reduce" if fused else "separate ipkv_merge launch",
-                       "append": "separate ipkv_append" if args.separate_append else "inside ipkv_attend_gpu (written by the attention kernel for GQA)"},
+                       "append": "separate ipkv_append" if args.separate_append else "inside ipkv_attend_gpu (written by the attention kernel for GQA)",
+                       "launch_overlap": "programmatic dependent launch; %d of %d attention launches started their copies before the previous kernel had completed"
+                                         % (st1["early_launches"] - st0["early_launches"], st1["attend_kernels"] - st0["attend_kernels"])},
             "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu,
             "step_gbs": bytes_all / (ms * 1e-3) / 1e9, "step_ms": step_ms,
         }

@@ -163,9 +163,12 @@ struct ipkv {
     // Which attention launches may start their first copies before the previous kernel of the stream has completed
     // (AttnLaunch::early_tiles).  launch_seq counts the attention launches enqueued so far; kv_written_at[layer] is the
     // value it must have reached before a launch on that layer may do so: one whole attention + reduce pair has then
-    // been enqueued, on the same stream, after the last operation that wrote the layer's device-side K/V.
+    // been enqueued, on the same stream, after the last operation that wrote the layer's device-side K/V.  The D-window
+    // is written by every append and the ring only by evictions, so the two are tracked apart: a launch right behind an
+    // append kernel may still start early on its ring tiles.
     uint64_t launch_seq = 0;
-    std::vector<uint64_t> kv_written_at;
+    std::vector<uint64_t> kv_written_at;     // resident ring of the layer
+    std::vector<uint64_t> w_written_at;      // D-window of the layer
     cudaStream_t launch_stream = nullptr;
     bool launch_stream_valid = false;
     ipkv_stats stats;
@@ -463,10 +466,13 @@ void CUDART_CB bounce_to_unpinned(void* arg) {
 // copy stream has drained (sync_host()).
 // Something is about to write device-side K/V of `layer` (all layers if negative): a standalone operation, or with
 // `inside_launch` the next attention launch itself (fused append).
-void note_kv_write(ipkv* h, int layer, bool inside_launch = false) {
+void note_kv_write(ipkv* h, int layer, bool inside_launch = false, bool window_only = false) {
     const uint64_t at = h->launch_seq + 1 + (inside_launch ? 1 : 0);
-    for (int l = 0; l < int(h->kv_written_at.size()); ++l)
-        if (layer < 0 || l == layer) h->kv_written_at[l] = std::max(h->kv_written_at[l], at);
+    for (int l = 0; l < int(h->kv_written_at.size()); ++l) {
+        if (layer >= 0 && l != layer) continue;
+        h->w_written_at[l] = std::max(h->w_written_at[l], at);
+        if (!window_only) h->kv_written_at[l] = std::max(h->kv_written_at[l], at);
+    }
 }
 
 ipkv_status flush_layer(ipkv* h, int layer, const int* seqs_in, int n, cudaStream_t s) {
@@ -740,9 +746,11 @@ ipkv_status run_group(ipkv* h, const std::vector<std::vector<PlanSeg>>& rows, co
             h->launch_stream = s; h->launch_stream_valid = true;
         }
         static const bool early_allowed = std::getenv("IPKV_NO_EARLY_COPIES") == nullptr;
-        a.early_tiles = (early_allowed && c.kind == IPKV_GQA && device_resident_only && layer >= 0 && h->launch_seq >= h->kv_written_at[layer]) ? 1 : 0;
-        if (append_k && layer >= 0) note_kv_write(h, layer, true);     // the kernel itself writes the new rows into the window
-        h->stats.early_launches += uint64_t(a.early_tiles);
+        a.early_tiles = 0;                                              // 1: ring tiles only, 2: window tiles too
+        if (early_allowed && device_resident_only && layer >= 0 && h->launch_seq >= h->kv_written_at[layer])
+            a.early_tiles = h->launch_seq >= h->w_written_at[layer] ? 2 : 1;
+        if (append_k && layer >= 0) note_kv_write(h, layer, true, true);     // the kernel itself writes the new rows into the window
+        h->stats.early_launches += a.early_tiles ? 1 : 0;
         h->launch_seq += 1;
         const bool sampled = h->prof_on && (h->prof_seen++ % h->prof_stride) == 0;
         const bool timed = sampled && !h->prof_reduce && h->prof_used + 2 <= h->prof_ev.size();
@@ -898,6 +906,7 @@ ipkv_status ipkv_create(const ipkv_config* cfg, ipkv_t** out) {
     }
     h->st.resize(size_t(cfg->n_layers) * cfg->max_seqs);
     h->kv_written_at.assign(size_t(cfg->n_layers), 0);
+    h->w_written_at.assign(size_t(cfg->n_layers), 0);
     for (auto& s : h->st) s.router.init(cfg->block_tokens, cfg->window_tokens, cfg->share_num, cfg->share_den);
 
     if (cudaMalloc(&h->status_dev, 256) != cudaSuccess) return bail(IPKV_ENOMEM);
@@ -1082,7 +1091,7 @@ ipkv_status append_tokens(ipkv* h, int32_t layer, const int32_t* seq_ids, int32_
             rows.slot[i] = int32_t(st.router.stage());
         }
         if (defer_copy) continue;
-        note_kv_write(h, layer);
+        note_kv_write(h, layer, false, true);
         const char* ks = static_cast<const char*>(k_dev) + base * k_row;
         const char* vs = v_dev ? static_cast<const char*>(v_dev) + base * v_row : nullptr;
         CU(h, launch_append(h->geom, ks, vs, c.dim_v, h->w_layer(layer), rows, n, s));

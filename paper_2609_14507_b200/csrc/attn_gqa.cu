@@ -53,7 +53,8 @@ struct GqaParams {
     int32_t* lists;      // per (row, head group): the number of extra partials CTAs filled for it [n_rows * n_gh], then their indices
                          // [n_rows * n_gh][kStealListCap] (all zero at launch); null = no CTA helps another
     int n_spans, n_ctas, n_rows, n_gh;
-    int early;          // the producer may issue its first copies before the previous kernel of the stream has completed
+    int early;          // nonzero: the producer may issue its first copies of ring tiles (2: of window tiles too) before the
+                        // previous kernel of the stream has completed
     int Hq, G, n_hg, RG;
     int bt;
     int64_t head_bytes, block_bytes;
@@ -130,6 +131,8 @@ __global__ void __launch_bounds__(kThreads, 2) attn_gqa_kernel(const GqaParams p
                     seg_base = p.bases[seg.base_id & kSegBaseMask] + seg.off + int64_t(span.gh / p.n_hg) * p.head_bytes;
                     cached_sp = sp;
                 }
+                // a tile of the D-window may have been written by the kernel in front of this one (an append kernel)
+                if (!waited && p.early < 2 && (seg.base_id & kSegBaseMask) == kSegBaseWindow) { ptx::grid_dependency_wait(); waited = true; }
                 const int st = it % STAGES;
                 if (it >= STAGES && !ptx::mbar_wait(s_empty + 8 * st, ((it / STAGES) - 1) & 1)) return false;
                 const int64_t t0 = int64_t(tile) * kTileTokens;

@@ -65,6 +65,7 @@ struct MlaParams {
     int bt;
     int64_t block_bytes;
     float scale_log2;
+    int early;           // nonzero: the first copies of ring tiles (2: of window tiles too) need not wait for the previous kernel
 };
 
 __device__ __forceinline__ void consumer_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory"); }
@@ -98,8 +99,13 @@ __global__ void __launch_bounds__(kThreads, 1) attn_mla_kernel(const MlaParams p
     __syncthreads();
     // Everything above may run while the previous kernel of the stream drains (it may be the append that writes this
     // launch's newest token, or the reduce that still reads the partials' scratch).
-    ptx::grid_dependency_wait();
-    ptx::grid_launch_dependents();
+    // With a host that vouches for the bytes (MlaParams::early) the producer fills the ring first and waits before its
+    // first refill or its first window tile; it never signals the dependents itself, so that signal always follows a wait.
+    const bool early = p.early != 0;
+    if (!(early && warp == kConsumerWarps)) {
+        ptx::grid_dependency_wait();
+        ptx::grid_launch_dependents();
+    }
 
     bool ok = true;
     int it = 0;                      // tiles streamed so far by this CTA: stage = it % kStages
@@ -108,11 +114,16 @@ __global__ void __launch_bounds__(kThreads, 1) attn_mla_kernel(const MlaParams p
         // ---------------- producer: streams the whole chunk, never pausing at span boundaries ----------------
         if (lane == 0) {
             const uint64_t pol = ptx::l2_evict_first_policy();     // the KV stream is read once: first out of L2
+            bool waited = !early;
             for (int sn = span_begin; sn < span_end && ok; ++sn) {
                 const Span span = p.spans[sn];
                 const Seg seg = p.segs[span.seg];
                 const char* seg_base = p.bases[seg.base_id & kSegBaseMask] + seg.off;
                 for (int i = 0; i < span.ntiles; ++i, ++it) {
+                    if (!waited && (it >= kStages || (p.early < 2 && (seg.base_id & kSegBaseMask) == kSegBaseWindow))) {
+                        ptx::grid_dependency_wait();
+                        waited = true;
+                    }
                     const int st = it % kStages;
                     if (it >= kStages && !ptx::mbar_wait(s_empty + 8 * st, ((it / kStages) - 1) & 1)) { ok = false; break; }
                     const int64_t t0 = int64_t(span.tile0 + i) * kTileTokens;
@@ -338,6 +349,7 @@ cudaError_t launch_attend_mla(const AttnLaunch& a, cudaStream_t s) {
     p.bt = a.bt;
     p.block_bytes = int64_t(a.bt) * kDqk * 2;
     p.scale_log2 = a.scale * kLog2e;
+    p.early = a.early_tiles;
     const int smem = kSmemTotal + 1024;
     static bool configured[64] = {};
     int dev = 0;

@@ -18,6 +18,7 @@ struct Seg {
 // its copy has landed (and into the run itself, for the launches to come), then computes as usual.
 constexpr int32_t kSegAppended = 0x100;
 constexpr int32_t kSegBaseMask = 0xff;
+constexpr int32_t kSegBaseWindow = 1;     // bases[1] is the layer's D-window (bases[0] the resident ring, bases[2] the slots)
 // One span of split-K work: tiles [tile0, tile0 + ntiles) of segment `seg` for query row `row` and head
 // group `gh`.  A CTA processes a contiguous range of spans back to back; the partial(s) a span produces are
 // stored at the span's own index.
@@ -53,8 +54,9 @@ struct AttnLaunch {
     uint32_t* status;               // device word, OR-ed with an error bit if a bounded wait gives up
     const void* append_k;           // fused append: [n_rows][n_kv_heads][dim_qk] bf16 new K rows (null: none)
     const void* append_v;           // [n_rows][n_kv_heads][dim_v]
-    int early_tiles;                // 1: no K/V byte this launch reads was written by the kernel before it in the stream, so the
-                                    // first copies may be issued before that kernel has completed (see launch.cuh)
+    int early_tiles;                // nonzero: no ring byte this launch reads (2: no window byte either) was written by the kernel
+                                    // before it in the stream, so the first copies of such tiles may be issued before that
+                                    // kernel has completed (see launch.cuh)
     // Dynamic load balancing of the GQA kernel (all null = static schedule with bit-reproducible results): a CTA
     // that has finished its chunk takes tiles from the spans that are furthest behind and accumulates them into
     // extra partials of its own, stored after the spans' partials (kStealSlots per CTA) and listed per (row, head group).

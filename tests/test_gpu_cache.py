@@ -636,7 +636,7 @@ def test_fused_append_writes_the_window_and_attends_the_new_token(G, dim, bt):
         assert st["device_status"] == 0 and st["fused_appends"] == 3 * bt + 5 and st["append_kernels"] == 0
 
 
-@pytest.mark.parametrize("mode", ["static", "balanced"])
+@pytest.mark.parametrize("mode", ["static", "balanced", "mla"])
 def test_early_copy_start_reads_no_stale_bytes(mode):
     """Attention launches fill their copy ring before the previous kernel of the stream has completed when the
     library knows that nothing they read can still be in flight.  Two identical caches take the same decode steps
@@ -646,9 +646,11 @@ def test_early_copy_start_reads_no_stale_bytes(mode):
     appended tokens are made to carry nearly all of the softmax weight (keys and queries along one direction), so
     that a single token read stale would move the output far beyond the tolerance, and every launch of both caches is
     checked against the oracle."""
-    static = mode == "static"
-    hkv, G, dim, bt, NL = 2, 4, 128, 64, 3
-    sh = synth.Shape("early", "gqa", NL, hkv * G, hkv, dim, dim, dim ** -0.5)
+    static = mode != "balanced"
+    mla = mode == "mla"                                     # its append is a kernel in front of the attention kernel: ring tiles only
+    hkv, G, dim, bt, NL = (1, 16, 576, 64, 3) if mla else (2, 4, 128, 64, 3)
+    dv = 512 if mla else dim
+    sh = synth.Shape("early", "mla" if mla else "gqa", NL, hkv * G, hkv, dim, dv, (192 if mla else dim) ** -0.5)
     lens = [900, 64, 333, 1]
     scale = float(np.float32(sh.scale))
     kw = dict(block_tokens=bt, window_tokens=2 * bt, chunk_tokens=4 * bt, max_u_tokens_per_seq=1024, max_p_tokens_per_seq=2048,
@@ -660,8 +662,8 @@ def test_early_copy_start_reads_no_stale_bytes(mode):
             for layer in range(NL):
                 k, v = synth.host_kv(sh, n, seed=7700 + 10 * s + layer)
                 for c in (ca, cb):
-                    c.append_bulk(layer, s, synth.bits_to_torch(k, DEV), synth.bits_to_torch(v, DEV), n, 1, 3)
-                r[layer].bulk(k, v, 1, 3)
+                    c.append_bulk(layer, s, synth.bits_to_torch(k, DEV), None if mla else synth.bits_to_torch(v, DEV), n, 1, 3)
+                r[layer].bulk(k, None if mla else v, 1, 3)
             refs.append(r)
         torch.cuda.synchronize()
         rng = np.random.default_rng(4242)
@@ -674,8 +676,10 @@ def test_early_copy_start_reads_no_stale_bytes(mode):
                 q = synth.normal_bf16(rng, (len(lens), hkv * G, dim))
                 if not static:                              # bf16 1.0 = 0x3F80: score 128 * scale = 11.3 for every appended token
                     k[:] = 0x3F80; q[:] = 0x3F80
+                if mla:
+                    v = None
                 plan.append((layer, step % 7 == 3 and layer == 1, k, v, q,
-                             synth.bits_to_torch(k, DEV), synth.bits_to_torch(v, DEV), synth.bits_to_torch(q, DEV)))
+                             synth.bits_to_torch(k, DEV), None if mla else synth.bits_to_torch(v, DEV), synth.bits_to_torch(q, DEV)))
         s0 = torch.cuda.Stream(); s1 = torch.cuda.Stream()
         torch.cuda.synchronize()
 
@@ -689,7 +693,7 @@ def test_early_copy_start_reads_no_stale_bytes(mode):
                     st = (s0, s1)[hop]; hop ^= 1
                     st.wait_event(ev)
                 with torch.cuda.stream(st):
-                    o = torch.zeros((len(lens), hkv * G, dim), device=DEV); lse = torch.zeros((len(lens), hkv * G), device=DEV)
+                    o = torch.zeros((len(lens), hkv * G, dv), device=DEV); lse = torch.zeros((len(lens), hkv * G), device=DEV)
                     if separate:                            # now and then the append is a call of its own
                         c.append(layer, seqs, kd, vd, stream=st)
                         c.attend_gpu(layer, seqs, qd, o, lse, static_schedule=static, force_balance=not static, stream=st)
@@ -707,7 +711,7 @@ def test_early_copy_start_reads_no_stale_bytes(mode):
         n_launch = len(plan)
         for i, (layer, _, k, v, q, _, _, _) in enumerate(plan):
             for s in seqs:
-                refs[s][layer].append(k[s:s + 1], v[s:s + 1])
+                refs[s][layer].append(k[s:s + 1], None if mla else v[s:s + 1])
             if static:
                 assert torch.equal(outs_a[i][0], outs_b[i][0]) and torch.equal(outs_a[i][1], outs_b[i][1]), f"launch {i} layer {layer}"
             if not static or i % 61 == 0 or i >= n_launch - NL:
