@@ -724,3 +724,103 @@ def test_early_copy_start_reads_no_stale_bytes(mode):
         assert sb["early_launches"] == 0
         # on one stream most launches qualify: all but the first ones, those right after an eviction or a separate append
         assert sa["early_launches"] > n_launch // 2
+
+
+def test_early_copy_start_under_a_random_program():
+    """A seeded random program of everything that writes device-side K/V (fused and separate appends, explicit flushes,
+    reset + bulk append) mixed with attention launches over two layers, run back to back on a single stream (where
+    launches start their copies early whenever the library's bookkeeping allows it) and on two event-ordered streams
+    (where it never does): every launch must give the same bits, and the last launches must match the oracle."""
+    hkv, G, dim, bt, NL, NS = 2, 4, 128, 64, 2, 3
+    sh = synth.Shape("earlyrand", "gqa", NL, hkv * G, hkv, dim, dim, dim ** -0.5)
+    scale = float(np.float32(sh.scale))
+    kw = dict(block_tokens=bt, window_tokens=2 * bt, chunk_tokens=4 * bt, max_u_tokens_per_seq=4096, max_p_tokens_per_seq=4096,
+              resident_tokens_per_seq=4096, share_num=1, share_den=4)
+    rng = np.random.default_rng(90210)
+    seqs = list(range(NS))
+    prog = []                                               # ("bulk", layer, seq, k, v) | ("reset", seq) | ("flush", layer, seq) | ("attend", layer, mode, k, v, q)
+    for s in seqs:
+        for layer in range(NL):
+            n = int(rng.integers(1, 700))
+            k, v = synth.host_kv(sh, n, seed=8800 + 10 * s + layer)
+            prog.append(("bulk", layer, s, k, v))
+    for i in range(260):
+        u = rng.random()
+        layer = int(rng.integers(0, NL)) if u > 0.5 else i % NL
+        if u < 0.04:
+            s = int(rng.integers(0, NS))
+            prog.append(("reset", s))
+            for l in range(NL):
+                n = int(rng.integers(1, 500))
+                k, v = synth.host_kv(sh, n, seed=9900 + i * 7 + l)
+                prog.append(("bulk", l, s, k, v))
+        elif u < 0.12:
+            prog.append(("flush", layer, int(rng.integers(-1, NS))))
+        else:
+            mode = "none" if u < 0.22 else ("separate" if u < 0.37 else "fused")
+            k = synth.normal_bf16(rng, (NS, hkv, dim)); v = synth.normal_bf16(rng, (NS, hkv, dim))
+            prog.append(("attend", layer, mode, k, v, synth.normal_bf16(rng, (NS, hkv * G, dim))))
+    dev = [tuple(synth.bits_to_torch(x, DEV) if isinstance(x, np.ndarray) else x for x in op) for op in prog]
+    s0 = torch.cuda.Stream(); s1 = torch.cuda.Stream()
+    torch.cuda.synchronize()
+
+    def run(c, hopping):
+        outs, hop, ev = [], 0, torch.cuda.Event()
+        ev.record(s0)
+        for op in dev:
+            st = s0
+            if hopping:                                     # every attention launch runs on the other stream than the one before it
+                if op[0] == "attend":
+                    hop ^= 1
+                st = (s0, s1)[hop]
+                st.wait_event(ev)
+            with torch.cuda.stream(st):
+                if op[0] == "bulk":
+                    c.append_bulk(op[1], op[2], op[3], op[4], op[3].shape[0], 1, 3, stream=st)
+                elif op[0] == "reset":
+                    c.reset(op[1])
+                elif op[0] == "flush":
+                    c.flush(op[1], op[2], stream=st)
+                else:
+                    _, layer, mode, kd, vd, qd = op
+                    o = torch.zeros((NS, hkv * G, dim), device=DEV); lse = torch.zeros((NS, hkv * G), device=DEV)
+                    if mode == "separate":
+                        c.append(layer, seqs, kd, vd, stream=st)
+                    app = dict(append_k=kd, append_v=vd) if mode == "fused" else {}
+                    c.attend_gpu(layer, seqs, qd, o, lse, static_schedule=True, stream=st, **app)
+                    o.record_stream(st); lse.record_stream(st)
+                    outs.append((o, lse))
+            if hopping:
+                ev.record(st)
+        torch.cuda.synchronize()
+        return outs
+
+    with make_cache(sh, NL, NS, **kw) as ca, make_cache(sh, NL, NS, **kw) as cb:
+        outs_a = run(ca, False)
+        outs_b = run(cb, True)
+        sa, sb = ca.get_stats(), cb.get_stats()
+    assert sa["device_status"] == 0 and sb["device_status"] == 0
+    assert sb["early_launches"] == 0 and sa["early_launches"] > len(outs_a) // 3
+    for i, (a, b) in enumerate(zip(outs_a, outs_b)):
+        assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1]), f"attention launch {i}"
+    # the oracle's view of the same program, checked on the last launch of every layer
+    refs = {(l, s): None for l in range(NL) for s in seqs}
+    last, j = {}, 0
+    for op in prog:
+        if op[0] == "bulk":
+            r = RefSeq(sh, bt, 2 * bt, 1, 4); r.bulk(op[3], op[4], 1, 3); refs[(op[1], op[2])] = r
+        elif op[0] == "flush":
+            for s in seqs:
+                if op[2] < 0 or s == op[2]:
+                    refs[(op[1], s)].route.flush()
+        elif op[0] == "attend":
+            _, layer, mode, k, v, q = op
+            if mode != "none":
+                for s in seqs:
+                    refs[(layer, s)].append(k[s:s + 1], v[s:s + 1])
+            last[layer] = (j, q, [(refs[(layer, s)].k.copy(), refs[(layer, s)].v.copy(), refs[(layer, s)].route.dump()[0].copy()) for s in seqs])
+            j += 1
+    for layer, (j, q, snap) in last.items():
+        parts = [c_oracle.attend(q[s], snap[s][0], snap[s][1], np.nonzero(snap[s][2] != 0)[0], scale) for s in seqs]
+        check_partial(outs_a[j][0].cpu().numpy(), outs_a[j][1].cpu().numpy(), np.stack([p[0] for p in parts]),
+                      np.stack([p[1] for p in parts]), f"last launch of layer {layer}")
