@@ -449,19 +449,25 @@ def main():
     cur = torch.cuda.current_stream()
     bpt = sh.bytes_per_token
 
+    # per-layer views once, not per call: slicing a tensor costs the host a few microseconds, which the small
+    # (host-bound) configuration would otherwise pay six times per layer
+    q_l = [q[l] for l in range(NL)]; k_l = [k_new[l] for l in range(NL)]
+    v_l = [None if v_new is None else v_new[l] for l in range(NL)]
+    out_l = [out[l] for l in range(NL)]; oc_l = [o_cpu[l] for l in range(NL)]; lc_l = [lse_cpu[l] for l in range(NL)]
+    apps = [{} if args.separate_append else dict(append_k=k_l[l], append_v=v_l[l]) for l in range(NL)]
+
     def step():
         for layer in range(NL):
             # the append rides in the attention call (the kernel writes the new rows where it can) unless --separate-append
-            app = {} if args.separate_append else dict(append_k=k_new[layer], append_v=None if v_new is None else v_new[layer])
             if args.separate_append:
-                cache.append(layer, seq_ids, k_new[layer], None if v_new is None else v_new[layer], stream=cur)
+                cache.append(layer, seq_ids, k_l[layer], v_l[layer], stream=cur)
             if fused:      # the CPU-side partial is joined inside the split reduce: out = merged (O, LSE)
-                cache.attend_gpu(layer, seq_ids, q[layer], out[layer], out_lse, kv_splits=args.kv_splits, static_schedule=args.static_schedule, stream=cur,
-                                 fold_o=o_cpu[layer], fold_lse=lse_cpu[layer], **app)
+                cache.attend_gpu(layer, seq_ids, q_l[layer], out_l[layer], out_lse, kv_splits=args.kv_splits, static_schedule=args.static_schedule, stream=cur,
+                                 fold_o=oc_l[layer], fold_lse=lc_l[layer], **apps[layer])
             else:
-                cache.attend_gpu(layer, seq_ids, q[layer], o_part, lse_part, kv_splits=args.kv_splits, static_schedule=args.static_schedule, stream=cur, **app)
-                cache.merge(B * Hq, dv, [o_part.view(B * Hq, dv), o_cpu[layer]], [lse_part.view(-1), lse_cpu[layer]],
-                            out[layer], out_lse, out_is_bf16=True, stream=cur)
+                cache.attend_gpu(layer, seq_ids, q_l[layer], o_part, lse_part, kv_splits=args.kv_splits, static_schedule=args.static_schedule, stream=cur, **apps[layer])
+                cache.merge(B * Hq, dv, [o_part.view(B * Hq, dv), oc_l[layer]], [lse_part.view(-1), lc_l[layer]],
+                            out_l[layer], out_lse, out_is_bf16=True, stream=cur)
 
     def barrier():
         torch.cuda.synchronize()
@@ -568,17 +574,21 @@ def main():
                 dlc[lo:hi].copy_(hlc[lo:hi], non_blocking=True)
                 landed[g].record(cs)
 
+        dq_l = [dq[l] for l in range(NL)]; dk_l = [dk[l] for l in range(NL)]
+        dv_l = [None if dvn is None else dvn[l] for l in range(NL)]
+        doc_l = [doc[l] for l in range(NL)]; dlc_l = [dlc[l] for l in range(NL)]
+        dapps = [{} if args.separate_append else dict(append_k=dk_l[l], append_v=dv_l[l]) for l in range(NL)]
+
         def run_layer(layer):
-            app = {} if args.separate_append else dict(append_k=dk[layer], append_v=None if dvn is None else dvn[layer])
             if args.separate_append:
-                cache.append(layer, seq_ids, dk[layer], None if dvn is None else dvn[layer], stream=cur)
+                cache.append(layer, seq_ids, dk_l[layer], dv_l[layer], stream=cur)
             if fused:
-                cache.attend_gpu(layer, seq_ids, dq[layer], out[layer], out_lse, kv_splits=args.kv_splits, static_schedule=args.static_schedule, stream=cur,
-                                 fold_o=doc[layer], fold_lse=dlc[layer], **app)
+                cache.attend_gpu(layer, seq_ids, dq_l[layer], out_l[layer], out_lse, kv_splits=args.kv_splits, static_schedule=args.static_schedule, stream=cur,
+                                 fold_o=doc_l[layer], fold_lse=dlc_l[layer], **dapps[layer])
             else:
-                cache.attend_gpu(layer, seq_ids, dq[layer], o_part, lse_part, kv_splits=args.kv_splits, static_schedule=args.static_schedule, stream=cur, **app)
-                cache.merge(B * Hq, dv, [o_part.view(B * Hq, dv), doc[layer]], [lse_part.view(-1), dlc[layer]],
-                            out[layer], out_lse, out_is_bf16=True, stream=cur)
+                cache.attend_gpu(layer, seq_ids, dq_l[layer], o_part, lse_part, kv_splits=args.kv_splits, static_schedule=args.static_schedule, stream=cur, **dapps[layer])
+                cache.merge(B * Hq, dv, [o_part.view(B * Hq, dv), doc_l[layer]], [lse_part.view(-1), dlc_l[layer]],
+                            out_l[layer], out_lse, out_is_bf16=True, stream=cur)
 
         def step_e2e():
             cs.wait_event(step_done)                     # the previous step's kernels no longer read the input buffers
