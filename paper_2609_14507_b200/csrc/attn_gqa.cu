@@ -19,6 +19,10 @@
 // Tiles are handed to the CTAs either in plan order or, by default for launches that are long enough, by the dynamic
 // balancing of schedule.cuh (CTAs that finish early take over tiles of the ones that are behind).
 //
+// The kernel is launched so that it may become resident while the previous kernel of the stream drains (launch.cuh):
+// everything up to the first use of the queries, the scheduling words or the partials' scratch runs before the wait
+// for that kernel, and when the host knows the K/V bytes to be settled the producer even fills the copy ring first.
+//
 // HBM traffic per KV token: bytes_per_token, read exactly once.
 #include <cuda_bf16.h>
 
