@@ -368,7 +368,61 @@ def cpu_engine_microbench():
     print(json.dumps({"cpu_engine_microbench": out}))
 
 
+def graph_microbench():
+    """A launch-bound case replayed from a CUDA graph: the stateless attention call on the small configuration's
+    shape (one sequence of 4096 tokens, 32 query / 4 KV heads, d 128: 4 MB of K/V, L2-resident) issued call by call
+    (host: planner, table upload, two launches) against the same call recorded once and replayed."""
+    import torch
+    from paper_2609_14507_b200 import binding
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    shape = binding.AttnShape(binding.GQA, 32, 4, 128, 128, BLOCK, 128 ** -0.5)
+    n = 4096
+    g = torch.Generator(device=dev); g.manual_seed(1)
+    k = torch.randn((n, 4, 128), generator=g, device=dev).to(torch.bfloat16)
+    v = torch.randn((n, 4, 128), generator=g, device=dev).to(torch.bfloat16)
+    q = torch.randn((1, 32, 128), generator=g, device=dev).to(torch.bfloat16)
+    blocks = torch.zeros((n // BLOCK) * binding.ipkv_block_bytes(shape), dtype=torch.uint8, device=dev)
+    binding.ipkv_pack_blocks(shape, binding.LAYOUT_TILE, k, v, n, blocks)
+    runs = [[(blocks, n)]]
+    o = torch.zeros((1, 32, 128), device=dev); lse = torch.zeros((1, 32), device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    def call():
+        binding.ipkv_attend_runs_noalloc(shape, runs, q, o, lse, 0, status)
+
+    def timed(fn, reps):
+        for _ in range(20):
+            fn()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(reps):
+            fn()
+        b.record(); torch.cuda.synchronize()
+        return a.elapsed_time(b) * 1e3 / reps
+
+    direct_us = timed(call, 2000)
+    o_direct = o.clone()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        call()
+    replay_us = timed(graph.replay, 2000)
+    many = torch.cuda.CUDAGraph()                            # 32 calls per graph, as 32 layers of a step would be
+    with torch.cuda.graph(many):
+        for _ in range(32):
+            call()
+    many_us = timed(many.replay, 200) / 32
+    assert torch.equal(o, o_direct) and int(status.item()) == 0
+    print(json.dumps({"graph_microbench": {"shape": "1 x 4096 tokens, GQA 32/4, d 128 (4.2 MB of K/V)", "direct_call_us": direct_us,
+                                           "graph_replay_us": replay_us, "graph_of_32_calls_us_per_call": many_us,
+                                           "kv_tokens_per_s_direct": n / (direct_us * 1e-6), "kv_tokens_per_s_graph_of_32": n / (many_us * 1e-6)}}))
+
+
 def main():
+    if "--graph-microbench" in sys.argv:
+        graph_microbench()
+        return
     if "--h2d-microbench" in sys.argv:
         h2d_microbench()
         return

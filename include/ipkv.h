@@ -353,7 +353,9 @@ ipkv_status ipkv_attend_runs(const ipkv_attn_shape* shape, int32_t n_rows,
  *     A larger kv_splits or batch needs more; use ipkv_attend_runs with your own scratch then.
  *   - The array is one per GPU and is held from library load to process exit by every GPU that runs it.
  *   - The first call on a device resolves the array's device address (cudaGetSymbolAddress, with that device
- *     current).  Make that first call outside any stream capture.
+ *     current).  Make that first call outside any stream capture.  After that the call (like ipkv_attend_runs) may be
+ *     recorded into a CUDA graph: under capture the launch tables travel as kernel parameters, which the graph keeps
+ *     by value, instead of as a copy from a temporary host image; the graph is valid for the runs it was recorded with.
  *   - All calls on a device share the array and each finds the previous call's bytes in it; nothing needs
  *     clearing between calls, but two calls whose work overlaps on the GPU (different streams without an
  *     ordering event, or another host thread) race on it.  Order them.

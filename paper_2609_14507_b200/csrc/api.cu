@@ -1745,13 +1745,22 @@ ipkv_status ipkv_attend_runs(const ipkv_attn_shape* sh, int32_t n_rows,
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     std::vector<char> img(table, 0);
     plan.serialize(img.data());
-    // pageable source: the runtime stages it before returning, so `img` may go out of scope
-    if (cudaMemcpyAsync(scratch_dev, img.data(), table, cudaMemcpyHostToDevice, s) != cudaSuccess) return IPKV_ECUDA;
+    // Outside a capture the tables go up as one copy from this pageable image (the runtime stages it before returning, so
+    // `img` may go out of scope).  A captured copy would be replayed from the image's address long after it is gone, so
+    // under capture the tables travel as kernel parameters instead, which a graph keeps by value.
+    cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(s, &capturing) != cudaSuccess) return IPKV_ECUDA;
+    if (capturing == cudaStreamCaptureStatusNone) {
+        if (cudaMemcpyAsync(scratch_dev, img.data(), table, cudaMemcpyHostToDevice, s) != cudaSuccess) return IPKV_ECUDA;
+    } else if (launch_upload_by_value(scratch_dev, img.data(), table, s) != cudaSuccess) {
+        return IPKV_ECUDA;
+    }
     AttnLaunch a{};
     const float scale = sh->softmax_scale > 0.f ? sh->softmax_scale : 1.0f / std::sqrt(float(sh->dim_qk));
     fill_launch(&a, sh->kind, sh->n_q_heads, sh->n_kv_heads, sh->dim_qk, sh->dim_v, sh->block_tokens, scale, plan,
                 static_cast<const char*>(scratch_dev), static_cast<char*>(scratch_dev) + table + 256, q_dev, n_rows);
     a.bases[0] = nullptr;
+    a.plain_launch = capturing == cudaStreamCaptureStatusNone ? 0 : 1;
     a.out_o = o_part_dev; a.out_lse = lse_part_dev;
     a.status = status_dev ? status_dev : reinterpret_cast<uint32_t*>(static_cast<char*>(scratch_dev) + table);
     if (a.n_spans > 0 && launch_attend(a, s) != cudaSuccess) return IPKV_ECUDA;

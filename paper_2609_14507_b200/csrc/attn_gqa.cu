@@ -455,7 +455,7 @@ cudaError_t launch_gqa(const AttnLaunch& a, cudaStream_t s) {
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
-    return launch_overlapped(attn_gqa_kernel<D, STAGES, DUP>, a.n_ctas, kThreads, size_t(smem), s, p);
+    return launch_ordered(!a.plain_launch, attn_gqa_kernel<D, STAGES, DUP>, a.n_ctas, kThreads, size_t(smem), s, p);
 }
 
 }  // namespace

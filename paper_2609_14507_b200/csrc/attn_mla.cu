@@ -359,7 +359,7 @@ cudaError_t launch_attend_mla(const AttnLaunch& a, cudaStream_t s) {
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
-    return launch_overlapped(attn_mla_kernel, a.n_ctas, kThreads, size_t(smem), s, p);
+    return launch_ordered(!a.plain_launch, attn_mla_kernel, a.n_ctas, kThreads, size_t(smem), s, p);
 }
 
 }  // namespace ipkvi

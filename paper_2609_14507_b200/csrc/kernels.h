@@ -54,6 +54,7 @@ struct AttnLaunch {
     uint32_t* status;               // device word, OR-ed with an error bit if a bounded wait gives up
     const void* append_k;           // fused append: [n_rows][n_kv_heads][dim_qk] bf16 new K rows (null: none)
     const void* append_v;           // [n_rows][n_kv_heads][dim_v]
+    int plain_launch;               // 1: the tables were written by the kernel right in front of this launch: no launch overlap
     int early_tiles;                // nonzero: no ring byte this launch reads (2: no window byte either) was written by the kernel
                                     // before it in the stream, so the first copies of such tiles may be issued before that
                                     // kernel has completed (see launch.cuh)
@@ -118,6 +119,10 @@ struct CopySpans {
     int64_t bytes[kCopySpansPerLaunch];      // multiples of 16
 };
 cudaError_t launch_copy_spans(const CopySpans& spans, int n, cudaStream_t s);
+// Writes `bytes` (a multiple of 16) of host data to device memory with kernels that carry the data as launch
+// parameters: unlike a copy from pageable memory, such a launch keeps nothing but a value, so it can be recorded
+// into a CUDA graph and replayed after the host buffer is gone.
+cudaError_t launch_upload_by_value(void* dst_dev, const void* src_host, size_t bytes, cudaStream_t s);
 
 constexpr int kAppendRowsPerLaunch = 64;
 struct AppendRows {

@@ -18,8 +18,10 @@ inline bool overlap_launches() {
     return on;
 }
 
+// `overlap` false launches plainly: for a kernel whose launch tables were written by the kernel right in front of it
+// (it reads them before its wait).
 template <typename... Params, typename... Args>
-inline cudaError_t launch_overlapped(void (*kernel)(Params...), int grid, int block, size_t smem, cudaStream_t s, Args&&... args) {
+inline cudaError_t launch_ordered(bool overlap, void (*kernel)(Params...), int grid, int block, size_t smem, cudaStream_t s, Args&&... args) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(unsigned(grid));
     cfg.blockDim = dim3(unsigned(block));
@@ -27,10 +29,15 @@ inline cudaError_t launch_overlapped(void (*kernel)(Params...), int grid, int bl
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = overlap_launches() ? 1 : 0;
+    attr[0].val.programmaticStreamSerializationAllowed = (overlap && overlap_launches()) ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<Args&&>(args)...);
+}
+
+template <typename... Params, typename... Args>
+inline cudaError_t launch_overlapped(void (*kernel)(Params...), int grid, int block, size_t smem, cudaStream_t s, Args&&... args) {
+    return launch_ordered(true, kernel, grid, block, smem, s, static_cast<Args&&>(args)...);
 }
 
 }  // namespace ipkvi

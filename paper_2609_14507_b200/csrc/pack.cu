@@ -4,6 +4,8 @@
 //   append_kernel        one new decode token per sequence -> its D-window slot (TILE layout)
 //   tile_to_plain_kernel an evicted window batch, TILE -> PLAIN, on its way to the CPU-compute region
 // All three move 16-byte chunks; one thread per chunk, consecutive threads on consecutive source chunks.
+#include <cstring>
+
 #include "kernels.h"
 #include "launch.cuh"
 #include "ptx.cuh"
@@ -89,6 +91,15 @@ __global__ void copy_spans_kernel(CopySpans sp) {
     for (int64_t i = blockIdx.x * int64_t(blockDim.x) + threadIdx.x; i < n; i += int64_t(gridDim.x) * blockDim.x) dst[i] = src[i];
 }
 
+constexpr int kUploadChunk = 16384;             // bytes of data per launch (kernel parameters may be up to 32 764 bytes on this architecture)
+struct UploadChunk { uint4 v[kUploadChunk / 16]; };
+
+__global__ void upload_by_value_kernel(UploadChunk c, uint4* dst, int n16) {
+    ptx::grid_dependency_wait();
+    ptx::grid_launch_dependents();
+    for (int i = threadIdx.x; i < n16; i += blockDim.x) dst[i] = c.v[i];
+}
+
 int grid_for(int64_t total, int threads) {
     int64_t b = (total + threads - 1) / threads;
     const int64_t cap = 148 * 16;
@@ -122,6 +133,19 @@ cudaError_t launch_copy_spans(const CopySpans& spans, int n, cudaStream_t s) {
     dim3 grid(grid_for(longest / 16, 256) > 64 ? 64 : grid_for(longest / 16, 256), n);
     copy_spans_kernel<<<grid, 256, 0, s>>>(spans);
     return cudaGetLastError();
+}
+
+cudaError_t launch_upload_by_value(void* dst_dev, const void* src_host, size_t bytes, cudaStream_t s) {
+    if (bytes % 16 != 0) return cudaErrorInvalidValue;
+    for (size_t off = 0; off < bytes; off += kUploadChunk) {
+        const size_t n = bytes - off < size_t(kUploadChunk) ? bytes - off : size_t(kUploadChunk);
+        UploadChunk c;
+        std::memcpy(c.v, static_cast<const char*>(src_host) + off, n);
+        upload_by_value_kernel<<<1, 128, 0, s>>>(c, reinterpret_cast<uint4*>(static_cast<char*>(dst_dev) + off), int(n / 16));
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
 }
 
 cudaError_t launch_append(const BlockGeom& g, const void* k, const void* v, int /*dim_v_src*/, char* w_base,

@@ -235,8 +235,8 @@ cudaError_t launch_split_reduce(const AttnLaunch& a, cudaStream_t s) {
     p.extra_count = a.steal_lists; p.extra_list = a.steal_lists ? a.steal_lists + a.n_rows * a.n_gh : nullptr; p.n_spans = a.n_spans;
     p.clear = a.steal_clear; p.clear_words = a.steal_clear ? a.steal_clear_words : 0;
     const size_t smem = size_t(kReduceThreads) * sizeof(float4);
-    if (p.extra_count) return launch_overlapped(split_reduce_kernel<true>, total, kReduceThreads, smem, s, p);
-    return launch_overlapped(split_reduce_kernel<false>, total, kReduceThreads, smem, s, p);
+    if (p.extra_count) return launch_ordered(!a.plain_launch, split_reduce_kernel<true>, total, kReduceThreads, smem, s, p);
+    return launch_ordered(!a.plain_launch, split_reduce_kernel<false>, total, kReduceThreads, smem, s, p);
 }
 
 cudaError_t launch_merge(const MergeLaunch& m, cudaStream_t s) {

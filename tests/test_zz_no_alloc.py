@@ -76,3 +76,45 @@ def test_noalloc_rejects_problems_beyond_its_array():
         binding.ipkv_attend_runs_noalloc(shape, rows, q, o, lse, kv_splits=64)
     assert e.value.status == 3
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("kind", ["gqa", "mla"])
+def test_stateless_call_can_be_recorded_into_a_cuda_graph(kind):
+    """Under stream capture the launch tables travel as kernel parameters (a captured copy from the call's temporary
+    host image would be replayed after the image is gone), so the recorded graph can be replayed: it gives the bits of
+    a direct call, and follows new queries written into the same buffer."""
+    if kind == "gqa":
+        shape, q, runs, _keep = _case(73, [[1500, 64], [700], [33]])
+    else:
+        shape = shape_of(binding.MLA, 16, 1, 576, 512, 64)
+        rng = np.random.default_rng(74)
+        q = synth.bits_to_torch(synth.normal_bf16(rng, (2, 16, 576)), "cuda:0")
+        _keep = [pack_run(shape, synth.normal_bf16(rng, (n, 1, 576)), None) for n in (900, 130)]
+        runs = [[(_keep[0], 900)], [(_keep[1], 130)]]
+    n_rows = len(runs)
+
+    def direct():
+        o = torch.full((n_rows, shape.n_q_heads, shape.dim_v), float("nan"), device="cuda:0")
+        lse = torch.full((n_rows, shape.n_q_heads), float("nan"), device="cuda:0")
+        binding.ipkv_attend_runs_noalloc(shape, runs, q, o, lse, 2)
+        torch.cuda.synchronize()
+        return o.clone(), lse.clone()
+
+    o_ref, l_ref = direct()                                  # also resolves the array's address outside the capture
+    o_g = torch.full((n_rows, shape.n_q_heads, shape.dim_v), float("nan"), device="cuda:0")
+    l_g = torch.full((n_rows, shape.n_q_heads), float("nan"), device="cuda:0")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda:0")
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        binding.ipkv_attend_runs_noalloc(shape, runs, q, o_g, l_g, 2, status)
+    torch.cuda.synchronize()
+    assert torch.isnan(o_g).all()                            # recording ran nothing
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(o_g, o_ref) and torch.equal(l_g, l_ref) and int(status.item()) == 0
+    q.copy_(synth.bits_to_torch(synth.normal_bf16(np.random.default_rng(75), tuple(q.shape)), "cuda:0"))
+    o_ref2, l_ref2 = direct()
+    assert not torch.equal(o_ref2, o_ref)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(o_g, o_ref2) and torch.equal(l_g, l_ref2)
