@@ -4,6 +4,8 @@
 //   append_kernel        one new decode token per sequence -> its D-window slot (TILE layout)
 //   tile_to_plain_kernel an evicted window batch, TILE -> PLAIN, on its way to the CPU-compute region
 // All three move 16-byte chunks; one thread per chunk, consecutive threads on consecutive source chunks.
+// (Also here: upload_by_value_kernel, which writes launch tables carried as kernel parameters, for calls recorded into a
+// CUDA graph.)
 #include <cstring>
 
 #include "kernels.h"
