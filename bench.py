@@ -272,7 +272,14 @@ def oracle_sample(wl, seconds_target=15.0, threads=None):
         n_pairs += 1
         if t_total >= seconds_target or n_pairs >= sh.n_layers * wl["batch"]:
             break
-    return dict(value=done_tokens / t_total, unit=UNIT, cores=c_oracle.num_threads(), kind="oracle",
+    # the same code on one thread, on the last pair of the sample
+    used = c_oracle.num_threads()
+    c_oracle.set_threads(1)
+    t0 = time.perf_counter()
+    c_oracle.attend(q, k, sh.dim_v if v is None else v, idx, float(np.float32(sh.scale)))
+    single = idx.size / (time.perf_counter() - t0)
+    c_oracle.set_threads(used)
+    return dict(value=done_tokens / t_total, unit=UNIT, cores=used, kind="oracle", host_cpus=os.cpu_count(), single_thread_value=single,
                 sample=f"{n_pairs} of {sh.n_layers * wl['batch']} (layer, sequence) pairs, GPU-side share ({done_tokens} KV-tokens "
                        f"in all), all heads; {t_total:.1f} s of float64 C++ (OpenMP over query heads)")
 
