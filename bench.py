@@ -715,7 +715,7 @@ def main():
                        "cpu_share": f"{num0}/{den0}", "gpu_share_tokens_per_seq_mean": n_gpu0 + 1, "bytes_per_kv_token": bpt, "block_tokens": BLOCK, "window_tokens": wl.get("window", WINDOW),
                        "gpu_share": "HBM-resident", "host_copies_of_U_and_P": "off (benchmark)", "cpu_partial": "synthetic values",
                        "l2": l2_note,
-                       "multi_gpu": "replicas only", "kv_splits": args.kv_splits, "kernel_timing": "CUDA events around every %d%s attention launch" % (args.time_every, "th" if args.time_every != 1 else "st"), "schedule": "static" if args.static_schedule else "dynamic balancing (GQA kernel, launches of at least 48 tiles per CTA)",
+                       "multi_gpu": "replicas only", "kv_splits": args.kv_splits, "kernel_timing": "CUDA events around every %d%s attention launch" % (args.time_every, "th" if args.time_every != 1 else "st"), "schedule": "static" if args.static_schedule else "dynamic balancing (GQA kernel, launches long enough for it to pay: from 64 tiles per CTA)",
                        "merge": "inside the split reduce" if fused else "separate ipkv_merge launch",
                        "append": "separate ipkv_append" if args.separate_append else "inside ipkv_attend_gpu (written by the attention kernel for GQA)",
                        "launch_overlap": "programmatic dependent launch; %d of %d attention launches started their copies before the previous kernel had completed"

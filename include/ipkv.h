@@ -158,8 +158,8 @@ ipkv_status ipkv_flush(ipkv_t* h, int32_t layer, int32_t seq, void* stream);
  * last bits between two identical calls.  This flag keeps the fixed assignment: bit-reproducible, a few
  * percent slower.  (The stateless entry points below always use the fixed assignment.) */
 #define IPKV_ATTEND_STATIC_SCHEDULE 1
-/* The balancing is switched on by the library when the launch is long enough for it to pay (about 50 tiles of 64
- * tokens per CTA); this flag switches it on for any size (tests use it to exercise the path on small inputs). */
+/* The balancing is switched on by the library when the launch is long enough for it to pay (from 64 tiles of 64
+ * tokens per CTA, more when the batch is large); this flag switches it on for any size (tests use it to exercise the path on small inputs). */
 #define IPKV_ATTEND_BALANCE 2
 /* Stream ordering.  The attention, split-reduce and append kernels are launched so that each may become resident while the previous
  * kernel of its stream drains (programmatic dependent launch); it waits for that kernel to complete before it reads
