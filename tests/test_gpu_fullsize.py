@@ -103,6 +103,17 @@ def test_ragged_1m_token_batch_sampled():
     _run_step_and_check("qwen3-ragged-bs64-1m-2layers-cpu30", [(0, 0), (0, 63), (1, 31), (1, 17)])
 
 
+def test_ragged_1m_token_batch_fixed_schedule_sampled():
+    """The same batch at a CPU share of 60 %: short enough for the library to keep the fixed schedule (with the early
+    copy start), where the 30 % case above is balanced."""
+    wl = dict(bench.WORKLOADS["qwen3-ragged-bs64-1m-2layers-cpu30"], share=(6, 10))
+    bench.WORKLOADS["_ragged60"] = wl
+    try:
+        _run_step_and_check("_ragged60", [(0, 7), (1, 40), (1, 63)])
+    finally:
+        del bench.WORKLOADS["_ragged60"]
+
+
 def _with_workload(name, wl, samples):
     bench.WORKLOADS[name] = wl
     try:
