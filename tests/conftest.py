@@ -12,6 +12,17 @@ def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run on the B200 box)")
 
 
+def pytest_sessionstart(session):
+    """Bring the in-tree library up to date with its sources before anything loads it (a no-op when it is; the binding
+    itself never builds and refuses to run without the library)."""
+    try:
+        from paper_2609_14507_b200 import build
+        if os.path.exists(build.NVCC):
+            build.build()
+    except Exception as e:                                  # the tests that need the library will say so themselves
+        sys.stderr.write(f"conftest: could not build libipkv.so: {e}\n")
+
+
 def read_golden(name="paper_tables.txt"):
     """key -> float from a ``tests/golden`` text fixture."""
     out = {}
