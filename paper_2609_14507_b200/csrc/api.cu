@@ -55,11 +55,6 @@ struct SeqState {
     std::vector<PRun> p_runs;
 };
 
-// Dynamic balancing pays when the attention launch is long enough for what it saves (about 2 % of the kernel) to outweigh
-// what it costs the split reduce (extra partials to read, one CTA fewer per SM): measured cross-over at 60-70 tiles per
-// CTA when the reduce fits one wave of CTAs (16 rows x 32 heads) and at about 135 when it takes 3.5 (64 rows x 32 heads).
-constexpr int kMinTilesPerCtaToBalance = 64;
-constexpr int kMinTilesPerCtaPerReduceWave = 28;
 
 // Bytes of the partial buffers for n_spans spans.
 size_t partial_bytes(size_t n_spans, const PartGeom& pg, int dv) {
@@ -710,11 +705,10 @@ ipkv_status run_group(ipkv* h, const std::vector<std::vector<PlanSeg>>& rows, co
     // dynamic balancing (grouped-query kernel): every CTA may fill up to kStealSlots extra partials
     const size_t n_lists = rows.size() * size_t(pg.n_gh) * (1 + kStealListCap);
     const size_t steal_words = n_lists + plan.spans.size() + 2 * size_t(plan.n_ctas());
-    // balancing pays once the chunks are long enough (see kMinTilesPerCtaToBalance)
+    // balancing pays once the chunks are long enough (plan.hpp)
     int64_t plan_tiles = 0;
     for (int32_t t : plan.cta_tiles) plan_tiles += t;
-    const double reduce_waves = std::max(1.0, double(rows.size()) * c.n_q_heads / (kSmCount * 4.0));
-    const int64_t min_tiles_per_cta = kMinTilesPerCtaToBalance + int64_t(kMinTilesPerCtaPerReduceWave * (reduce_waves - 1.0));
+    const int64_t min_tiles_per_cta = min_tiles_per_cta_to_balance(int64_t(rows.size()), c.n_q_heads);
     const bool balance = !(schedule_flags & IPKV_ATTEND_STATIC_SCHEDULE) && c.kind == IPKV_GQA && plan.n_ctas() > 1 &&
                          steal_words <= size_t(ipkv::kStealWords) &&
                          ((schedule_flags & IPKV_ATTEND_BALANCE) || plan_tiles >= min_tiles_per_cta * plan.n_ctas());

@@ -22,6 +22,17 @@ constexpr int kSmCount = 148;
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// When the grouped-query kernel balances its load while it runs (schedule.cuh).  Balancing makes the attention kernel
+// about 2 % faster and the split reduce slower (extra partials to read, one CTA fewer per SM), so it pays only when the
+// launch is long against its reduce: measured cross-over at 60-70 tiles per CTA when the reduce fits one wave of CTAs
+// (16 rows x 32 heads) and at about 135 when it takes 3.5 (64 rows x 32 heads).
+constexpr int kMinTilesPerCtaToBalance = 64;
+constexpr int kMinTilesPerCtaPerReduceWave = 28;
+inline int64_t min_tiles_per_cta_to_balance(int64_t n_rows, int n_q_heads) {
+    const double waves = double(n_rows) * n_q_heads / (kSmCount * 4.0);
+    return kMinTilesPerCtaToBalance + (waves > 1.0 ? int64_t(kMinTilesPerCtaPerReduceWave * (waves - 1.0)) : 0);
+}
+
 struct PlanSeg { int base_id; int64_t off; int64_t n_tokens; bool appended = false; };
 
 struct Plan {

@@ -43,6 +43,8 @@ void shim_router_dump(void* r, int8_t* region, int64_t* blk, int32_t* off) {
     }
 }
 
+int64_t shim_min_tiles_to_balance(int64_t n_rows, int n_q_heads) { return min_tiles_per_cta_to_balance(n_rows, n_q_heads); }
+
 // plan: rows given as flat (row_start[n_rows+1], n_tokens[n_segs]); fills the span table and the two index arrays
 int shim_plan(int n_rows, const int32_t* row_start, const int64_t* seg_tokens, int n_gh, int kv_splits, int ctas_per_sm,
               int cap_spans, int32_t* span_fields /* [cap][5] */, int32_t* cta_span_start /* [<= 148*ctas_per_sm + 1] */,

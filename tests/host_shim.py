@@ -35,6 +35,8 @@ def lib():
         L.shim_router_dump.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.shim_plan.argtypes = [C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int] + [C.c_void_p] * 8
         L.shim_plan.restype = C.c_int
+        L.shim_min_tiles_to_balance.argtypes = [C.c_int64, C.c_int]
+        L.shim_min_tiles_to_balance.restype = C.c_int64
         L.shim_tile_chunk_offset.argtypes = [C.c_int32] * 3
         L.shim_tile_chunk_offset.restype = C.c_int64
         L.shim_plain_chunk_offset.argtypes = [C.c_int32] * 3

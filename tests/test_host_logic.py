@@ -111,6 +111,17 @@ def test_plan_fills_the_machine_in_one_balanced_wave():
     assert len(p["cta_span_start"]) - 1 == 4 * (2 + 1)
 
 
+def test_balancing_threshold_follows_the_measured_crossovers():
+    """The rule that decides when the grouped-query kernel balances its load: 64 tiles per CTA while the split reduce
+    fits one wave of CTAs, more for larger batches (the two measured cross-overs: 60-70 tiles per CTA for 16 rows x
+    32 heads, about 135 for 64 rows x 32 heads); monotone in the batch."""
+    f = host_shim.lib().shim_min_tiles_to_balance
+    assert f(16, 32) == 64 and f(1, 8) == 64 and f(18, 32) == 64
+    assert 125 <= f(64, 32) <= 140
+    vals = [f(r, 32) for r in range(1, 400, 7)]
+    assert vals == sorted(vals)
+
+
 def test_layout_arithmetic_matches_header_formula():
     L = host_shim.lib()
     for bt in (16, 64, 256):
