@@ -124,43 +124,45 @@ __global__ void __launch_bounds__(kThreads, 1) attn_mla_kernel(const MlaParams p
                         ptx::grid_dependency_wait();
                         waited = true;
                     }
+                    // Everything that can be known before the stage is free is computed before the wait: the time between
+                    // the consumers' release and the start of the copy is time in which the stage holds nothing.
                     const int st = it % kStages;
-                    if (it >= kStages && !ptx::mbar_wait(s_empty + 8 * st, ((it / kStages) - 1) & 1)) { ok = false; break; }
                     const int64_t t0 = int64_t(span.tile0 + i) * kTileTokens;
                     const uint32_t dst = s_base + st * kStageBytes;
                     const uint32_t bar = s_full + 8 * st;
-                    if (p.bt >= kTileTokens) {
-                        const int64_t blk = t0 / p.bt;
-                        const int r0 = int(t0 - blk * p.bt);
-                        const char* src = seg_base + blk * p.block_bytes;
+                    const int64_t blk = t0 / p.bt;
+                    const char* src = seg_base + blk * p.block_bytes;
+                    const int64_t row_off = (t0 - blk * p.bt) * 128;
+                    int live = 0;
+                    if (p.bt < kTileTokens)
+                        for (int j = 0; j < kTileTokens / p.bt; ++j) live += ((blk + j) * p.bt < seg.n_tokens);
+                    if (it >= kStages && !ptx::mbar_wait(s_empty + 8 * st, ((it / kStages) - 1) & 1)) { ok = false; break; }
+                    if (p.bt == kTileTokens) {
                         ptx::mbar_expect_tx(bar, kStageBytes);
-                        if (p.bt == kTileTokens) {
-                            ptx::bulk_g2s_hint(dst, src, kStageBytes, bar, pol);
-                        } else {
+                        ptx::bulk_g2s_hint(dst, src, kStageBytes, bar, pol);
+                    } else if (p.bt > kTileTokens) {
+                        ptx::mbar_expect_tx(bar, kStageBytes);
 #pragma unroll
-                            for (int pn = 0; pn < kPanels; ++pn)
-                                ptx::bulk_g2s_hint(dst + pn * 8192, src + int64_t(pn) * p.bt * 128 + int64_t(r0) * 128, 8192, bar, pol);
-                        }
+                        for (int pn = 0; pn < kPanels; ++pn)
+                            ptx::bulk_g2s_hint(dst + pn * 8192, src + int64_t(pn) * p.bt * 128 + row_off, 8192, bar, pol);
                     } else {
-                        const int nsub = kTileTokens / p.bt;
-                        const int64_t blk0 = t0 / p.bt;
-                        int live = 0;
-                        for (int j = 0; j < nsub; ++j) live += ((blk0 + j) * p.bt < seg.n_tokens);
                         const uint32_t sub_bytes = uint32_t(p.bt) * 128;
                         ptx::mbar_expect_tx(bar, uint32_t(live) * sub_bytes * kPanels);
                         for (int j = 0; j < live; ++j) {
-                            const char* src = seg_base + (blk0 + j) * p.block_bytes;
+                            const char* sj = src + j * p.block_bytes;
 #pragma unroll
                             for (int pn = 0; pn < kPanels; ++pn)
-                                ptx::bulk_g2s_hint(dst + pn * 8192 + j * sub_bytes, src + int64_t(pn) * sub_bytes, sub_bytes, bar, pol);
+                                ptx::bulk_g2s_hint(dst + pn * 8192 + j * sub_bytes, sj + int64_t(pn) * sub_bytes, sub_bytes, bar, pol);
                         }
                     }
                 }
             }
             const int first_pending = it > kStages ? it - kStages : 0;
+            bool landed = true;
             for (int i = first_pending; i < it; ++i)
-                if (!ptx::mbar_wait(s_full + 8 * (i % kStages), (i / kStages) & 1)) ok = false;
-            if (!ok) atomicOr(p.status, 2u);
+                if (!ptx::mbar_wait(s_full + 8 * (i % kStages), (i / kStages) & 1)) landed = false;
+            if (!ok) atomicOr(p.status, kStatusNoFreeStage);
+            if (!landed) atomicOr(p.status, kStatusCopyNotLanded);
         }
         return;      // the consumers synchronise among themselves on a named barrier
     }
@@ -327,7 +329,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_mla_kernel(const MlaParams p
         }
         consumer_barrier();      // s_m / s_l / the query tile are reused by the next span
     }
-    if (!ok && lane == 0) atomicOr(p.status, 2u);
+    if (!ok && lane == 0) atomicOr(p.status, kStatusNoTile);
 }
 
 }  // namespace

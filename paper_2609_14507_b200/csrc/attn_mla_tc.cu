@@ -199,9 +199,11 @@ __global__ void __launch_bounds__(kThreads, 1) attn_mla_tc_kernel(const MlaTcPar
                 }
             }
             const int first_pending = it > kStages ? it - kStages : 0;
+            bool landed = true;
             for (int i = first_pending; i < it; ++i)
-                if (!ptx::mbar_wait(b_full + 8 * (i & 1), (i >> 1) & 1)) ok = false;
-            if (!ok) atomicOr(p.status, 1u);
+                if (!ptx::mbar_wait(b_full + 8 * (i & 1), (i >> 1) & 1)) landed = false;
+            if (!ok) atomicOr(p.status, kStatusNoFreeStage);
+            if (!landed) atomicOr(p.status, kStatusCopyNotLanded);
         }
     } else if (warp == 5) {
         // ---------------- MMA issuer (one thread) ----------------
@@ -252,7 +254,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_mla_tc_kernel(const MlaTcPar
                     umma_commit(b_odone);
                 }
             }
-            if (!ok) atomicOr(p.status, 1u);
+            if (!ok) atomicOr(p.status, kStatusNoTile);
         }
     } else {
         // ---------------- softmax / rescale / epilogue warps (TMEM lane quadrant = warp) ----------------
@@ -390,7 +392,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_mla_tc_kernel(const MlaTcPar
             }
             softmax_barrier();
         }
-        if (!ok && lane == 0) atomicOr(p.status, 1u);
+        if (!ok && lane == 0) atomicOr(p.status, kStatusNoTile);
     }
 
     tc_fence_before();

@@ -2,6 +2,7 @@
 #pragma once
 #include <cuda_runtime.h>
 #include <cstdint>
+#include <cstdlib>
 
 #include "layout.cuh"
 
@@ -76,6 +77,7 @@ constexpr int kStealListCap = 16;   // extra partials a (row, head group) can ta
 struct PartGeom {
     int rows_per_group, n_gh, parts_per_span, ctas_per_sm;
 };
+
 inline PartGeom part_geom(int kind, int Hq, int Hkv) {
     PartGeom g;
     if (kind == 1) { g.rows_per_group = 16; g.n_gh = (Hq + 15) / 16; g.parts_per_span = 1; g.ctas_per_sm = 1; }

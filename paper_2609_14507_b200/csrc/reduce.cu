@@ -19,10 +19,12 @@ constexpr int kReduceThreads = 256;
 constexpr int kPrefetch = 2;       // partial outputs per thread requested up front (of the own and of the extra partials)
 constexpr int kLseCache = 512;     // LSE values kept in shared memory between the two passes
 
-// One CTA per (row, query head). The partials to join are those of the spans of the head's group
-// (parts_per_span consecutive entries per span), row `rin` of each. Threads are arranged as
+// One CTA per (row, query head, slab of up to 128 value columns). The partials to join are those of the spans of
+// the head's group (parts_per_span consecutive entries per span), row `rin` of each. Threads are arranged as
 // (entry slice, 4-column group): every thread sums the weighted partials of its slice for its four columns;
-// the slices are then added through shared memory. CG = dv / 4 column groups, SL = 256 / CG slices.
+// the slices are then added through shared memory. CG = slab / 4 column groups, SL = 256 / CG slices: with at
+// most 128 columns per CTA there are at least 8 slices, so a thread has few entries to fetch one after the other
+// (a 512-column head handled by one CTA had two slices and ten dependent loads per thread).
 struct ReduceParams {
     const float* part_o;
     const float* part_lse;
@@ -32,6 +34,7 @@ struct ReduceParams {
     float* out_o;
     float* out_lse;
     int Hq, dv, G, n_hg, n_gh, RG, NW;
+    int CS, dvl;                  // column slabs per (row, head) and columns per slab
     const int32_t* extra_count;   // per (row, head group): extra partials written by CTAs that helped with its spans (null: none)
     const int32_t* extra_list;    // [n_rows * n_gh][kStealListCap] their indices; extra partial i is stored as if it were span n_spans + i
     int n_spans;
@@ -49,7 +52,8 @@ __global__ void __launch_bounds__(kReduceThreads, EXTRAS ? 4 : 5) split_reduce_k
     __shared__ float s_zs[kReduceThreads / 16];    // weight sum of every entry slice (SL <= 16)
     __shared__ int s_extra[kStealListCap];         // extra partials that belong to this (row, head group)
     __shared__ int s_n_extra;
-    const int wid = blockIdx.x;                      // row * Hq + h
+    const int wid = blockIdx.x / p.CS;               // row * Hq + h
+    const int col0 = (blockIdx.x - wid * p.CS) * p.dvl;
     const int row = wid / p.Hq, h = wid - row * p.Hq;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = h / p.G, hin = h - g * p.G;
@@ -81,9 +85,9 @@ __global__ void __launch_bounds__(kReduceThreads, EXTRAS ? 4 : 5) split_reduce_k
         return int64_t(p.n_spans + s_extra[k]) * p.NW + (e - n_own - k * p.NW);
     };
     const float* lse_base = p.part_lse + rin;                      // entry e at lse_base[entry(e) * RG]
-    const int CG = dv >> 2, SL = kReduceThreads / CG;
+    const int CG = p.dvl >> 2, SL = kReduceThreads / CG;
     const int cg = tid % CG, sl = tid / CG;
-    const float* po = p.part_o + int64_t(rin) * dv + cg * 4;
+    const float* po = p.part_o + int64_t(rin) * dv + col0 + cg * 4;
     const int64_t stride = int64_t(p.RG) * dv;
 
     // The partial outputs of this thread's first entries (own and extra) are requested before anything is known about
@@ -102,7 +106,7 @@ __global__ void __launch_bounds__(kReduceThreads, EXTRAS ? 4 : 5) split_reduce_k
         prx[j] = x < n_x ? *reinterpret_cast<const float4*>(po + entry(n_own + x) * stride) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
     float4 fold = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (p.acc_o && sl == 0) fold = *reinterpret_cast<const float4*>(p.acc_o + int64_t(wid) * dv + cg * 4);
+    if (p.acc_o && sl == 0) fold = *reinterpret_cast<const float4*>(p.acc_o + int64_t(wid) * dv + col0 + cg * 4);
 
     float m = la;
     for (int e = tid; e < n; e += kReduceThreads) {
@@ -120,10 +124,10 @@ __global__ void __launch_bounds__(kReduceThreads, EXTRAS ? 4 : 5) split_reduce_k
         for (int w = 1; w < kReduceThreads / 32; ++w) mm = fmaxf(mm, s_warp[w]);
         m = mm;
     }
-    float* oo = p.out_o + int64_t(wid) * dv;
+    float* oo = p.out_o + int64_t(wid) * dv + col0;
     if (m == -INFINITY) {                           // nothing attended: (0, -inf)
         if (sl == 0) *reinterpret_cast<float4*>(oo + cg * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (tid == 0) p.out_lse[wid] = -INFINITY;
+        if (tid == 0 && col0 == 0) p.out_lse[wid] = -INFINITY;
         return;
     }
     // weight of entry e (0 for an empty one); the first kLseCache LSE values are in shared memory
@@ -172,7 +176,7 @@ __global__ void __launch_bounds__(kReduceThreads, EXTRAS ? 4 : 5) split_reduce_k
         const float inv = 1.f / zt;
         t.x *= inv; t.y *= inv; t.z *= inv; t.w *= inv;
         *reinterpret_cast<float4*>(oo + cg * 4) = t;
-        if (cg == 0) p.out_lse[wid] = m + logf(zt);
+        if (cg == 0 && col0 == 0) p.out_lse[wid] = m + logf(zt);
     }
 }
 
@@ -223,7 +227,6 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) merge_kernel(const MergeL
 cudaError_t launch_split_reduce(const AttnLaunch& a, cudaStream_t s) {
     const int total = a.n_rows * a.n_q_heads;
     if (total <= 0) return cudaSuccess;
-    if (a.dim_v % 4 != 0 || a.dim_v / 4 > kReduceThreads || kReduceThreads % (a.dim_v / 4) != 0) return cudaErrorInvalidValue;
     const PartGeom pg = part_geom(a.kind, a.n_q_heads, a.n_kv_heads);
     ReduceParams p;
     p.part_o = a.part_o; p.part_lse = a.part_lse; p.rg_span_start = a.rg_span_start;
@@ -232,11 +235,14 @@ cudaError_t launch_split_reduce(const AttnLaunch& a, cudaStream_t s) {
     p.G = a.kind == 1 ? a.n_q_heads : a.n_q_heads / a.n_kv_heads;
     p.n_hg = (p.G + 15) / 16;
     p.n_gh = pg.n_gh; p.RG = pg.rows_per_group; p.NW = pg.parts_per_span;
+    p.dvl = a.dim_v > 128 && a.dim_v % 128 == 0 ? 128 : a.dim_v;
+    p.CS = a.dim_v / p.dvl;
+    if (p.dvl % 4 != 0 || p.dvl / 4 > kReduceThreads || kReduceThreads % (p.dvl / 4) != 0) return cudaErrorInvalidValue;
     p.extra_count = a.steal_lists; p.extra_list = a.steal_lists ? a.steal_lists + a.n_rows * a.n_gh : nullptr; p.n_spans = a.n_spans;
     p.clear = a.steal_clear; p.clear_words = a.steal_clear ? a.steal_clear_words : 0;
     const size_t smem = size_t(kReduceThreads) * sizeof(float4);
-    if (p.extra_count) return launch_ordered(!a.plain_launch, split_reduce_kernel<true>, total, kReduceThreads, smem, s, p);
-    return launch_ordered(!a.plain_launch, split_reduce_kernel<false>, total, kReduceThreads, smem, s, p);
+    if (p.extra_count) return launch_ordered(!a.plain_launch, split_reduce_kernel<true>, total * p.CS, kReduceThreads, smem, s, p);
+    return launch_ordered(!a.plain_launch, split_reduce_kernel<false>, total * p.CS, kReduceThreads, smem, s, p);
 }
 
 cudaError_t launch_merge(const MergeLaunch& m, cudaStream_t s) {
