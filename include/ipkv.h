@@ -335,7 +335,9 @@ ipkv_status ipkv_attend_scratch_bytes(const ipkv_attn_shape* shape, int32_t n_ro
  * runs[row_run_start[r] .. row_run_start[r+1]).  runs and row_run_start are host arrays.
  * scratch_dev: device memory of at least ipkv_attend_scratch_bytes (256-byte aligned), private to this
  * call until the work queued on `stream` has completed.  Outputs as in ipkv_attend_gpu.
- * status_dev: optional device uint32 that receives a nonzero value if a bounded wait gave up. */
+ * status_dev: optional device uint32 that is OR-ed with the bits below if a bounded wait inside a kernel gave up
+ * (bit 0: the copy engine's thread found no free stage; bit 1: a consumer's tile did not arrive; bit 2: a copy had
+ * not landed when its CTA left); the results of that call are then invalid.  With NULL a timeout goes unreported. */
 ipkv_status ipkv_attend_runs(const ipkv_attn_shape* shape, int32_t n_rows,
                              const ipkv_run* runs, const int32_t* row_run_start,
                              const void* q_dev, int32_t kv_splits,
@@ -351,11 +353,13 @@ ipkv_status ipkv_attend_runs(const ipkv_attn_shape* shape, int32_t n_rows,
  *   - Limit: the call needs ipkv_attend_scratch_bytes(shape, n_rows, n_runs, total tokens, kv_splits) bytes;
  *     if that exceeds ipkv_noalloc_scratch_limit() (16 MiB) it returns IPKV_ERANGE and does nothing.
  *     A larger kv_splits or batch needs more; use ipkv_attend_runs with your own scratch then.
- *   - The array is one per GPU and is held from library load to process exit by every GPU that runs it.
- *   - The first call on a device resolves the array's device address (cudaGetSymbolAddress, with that device
- *     current).  Make that first call outside any stream capture.  After that the call (like ipkv_attend_runs) may be
- *     recorded into a CUDA graph: under capture the launch tables travel as kernel parameters, which the graph keeps
- *     by value, instead of as a copy from a temporary host image; the graph is valid for the runs it was recorded with.
+ *   - The array is one per GPU.  The first call on a device resolves its device address (cudaGetSymbolAddress, with
+ *     that device current); with CUDA's lazy module loading that is also the moment the driver sets the 16 MiB aside
+ *     on that GPU, which keeps them until the process exits.  So make one warm-up call per device at start-up, before
+ *     the memory is handed to a pool (afterwards the first call could fail with IPKV_ECUDA) and outside any stream
+ *     capture.  The address is remembered per device ordinal: after a cudaDeviceReset the library must be reloaded.
+ *   - The launch tables (a few KB) go up with a cudaMemcpyAsync from a temporary pageable host image: the runtime
+ *     stages it before the call returns, so the call is asynchronous to the GPU but not free of host-side work.
  *   - All calls on a device share the array and each finds the previous call's bytes in it; nothing needs
  *     clearing between calls, but two calls whose work overlaps on the GPU (different streams without an
  *     ordering event, or another host thread) race on it.  Order them.

@@ -14,7 +14,7 @@
 
 namespace {
 
-constexpr size_t kStaticScratchBytes = size_t(16) << 20;   // 16 MiB, held by every GPU that loads the library
+constexpr size_t kStaticScratchBytes = size_t(16) << 20;   // 16 MiB, held by every GPU on which the entry point has run
 
 // File-scope device array. In host code this name is only a stand-in for the symbol, not a device address:
 // the address the kernels need comes from cudaGetSymbolAddress, once per device.
@@ -24,7 +24,9 @@ constexpr int kMaxDevices = 64;
 std::mutex g_mu;
 void* g_scratch_addr[kMaxDevices] = {};
 
-// Device address of the array on the CURRENT device (resolved on first use on that device).
+// Device address of the array on the CURRENT device, resolved on first use on that device.  With CUDA's lazy module
+// loading that first use is also what makes the driver materialise the array on the device, so it can fail on a device
+// whose memory is already taken; the address is remembered per device ordinal and is stale after a cudaDeviceReset.
 cudaError_t static_scratch_address(void** out) {
     int dev = -1;
     cudaError_t e = cudaGetDevice(&dev);
@@ -68,8 +70,9 @@ ipkv_status ipkv_attend_runs_noalloc(const ipkv_attn_shape* shape, int32_t n_row
     // Every call shares the array and finds the previous call's bytes in it. Nothing in it has to start at
     // zero: the tables and the partials are rewritten in full before they are read, and the status word kept
     // in the array (used only when status_dev is NULL) is never read back.
-    return ipkv_attend_runs(shape, n_rows, runs, row_run_start, q_dev, kv_splits, scratch, kStaticScratchBytes,
-                            o_part_dev, lse_part_dev, status_dev, stream);
+    rc = ipkv_attend_runs(shape, n_rows, runs, row_run_start, q_dev, kv_splits, scratch, kStaticScratchBytes,
+                          o_part_dev, lse_part_dev, status_dev, stream);
+    return rc == IPKV_ENOMEM ? IPKV_ERANGE : rc;            // "does not fit the array" is a range error of this call
 }
 
 }  // extern "C"

@@ -63,11 +63,16 @@ struct Plan {
     }
 };
 
-// Upper bound on the number of spans build_plan can produce.
+// Upper bound on the number of spans build_plan can produce.  Pass 1 emits one piece per (row, head group, run), or,
+// with kv_splits, at most kv_splits + 1 pieces of it (a row's runs share the row's kv_splits pieces, each run rounds up
+// once); pass 2 then cuts a piece wherever a CTA's chunk ends inside it: one cut per CTA boundary, and there are never
+// more CTAs than pieces (kv_splits > 0) or than CTA slots.
 inline int64_t max_spans_bound(int n_rows, int n_runs, int n_gh, int kv_splits, int ctas_per_sm) {
-    const int64_t pieces = int64_t(n_runs) * n_gh;               // one span per (row, head group, run) at least
-    if (kv_splits > 0) return pieces * (int64_t(kv_splits) + 1) + n_rows;
-    return pieces + int64_t(kSmCount) * ctas_per_sm + n_rows;    // plus one cut per CTA boundary
+    const int64_t slots = int64_t(kSmCount) * ctas_per_sm;
+    int64_t pieces = int64_t(n_runs) * n_gh;
+    if (kv_splits > 0) pieces *= int64_t(kv_splits) + 1;
+    const int64_t cuts = kv_splits > 0 ? std::min(slots, pieces) : slots;
+    return pieces + cuts + n_rows;
 }
 
 // rows[r] = runs of row r.  n_gh = head groups per row.  kv_splits = 0: one balanced chunk per CTA slot;

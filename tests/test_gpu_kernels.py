@@ -41,6 +41,7 @@ GQA_CASES = [
     (32, 4, 128, 32, [[1000, 33]], 2),
     (32, 4, 128, 128, [[1000, 257]], 0),          # large blocks: several tiles per block
     (32, 4, 128, 256, [[5000, 100], [256]], 0),
+    (32, 4, 128, 64, [[6400], [6208]], 4),        # ragged rows with explicit splits: CTA cuts fall inside the pieces
 ]
 
 
@@ -131,6 +132,7 @@ MLA_CASES = [
     (16, 16, [[1000, 17]], 0),
     (16, 32, [[70]], 0),
     (16, 128, [[1000, 257]], 2),
+    (16, 64, [[6400], [6208]], 8),           # ragged rows with explicit splits: CTA cuts fall inside the pieces
 ]
 
 

@@ -111,6 +111,26 @@ def test_plan_fills_the_machine_in_one_balanced_wave():
     assert len(p["cta_span_start"]) - 1 == 4 * (2 + 1)
 
 
+def test_span_bound_and_scratch_size_hold_for_ragged_rows_with_explicit_splits():
+    """With kv_splits the planner first cuts every row into pieces and then cuts pieces again where a CTA's chunk ends;
+    ragged rows make those second cuts fall inside pieces.  The span bound (checked inside the shim) and the scratch
+    size the library reports must cover the plan that is actually built."""
+    from paper_2609_14507_b200 import binding
+    shapes = [(binding.GQA, 32, 4, 128, 128, 4, 8, 4, 2), (binding.MLA, 16, 1, 576, 512, 1, 16, 1, 1)]
+    cases = [[32768 - 192 * i for i in range(16)], [6400, 6208], [70000, 69000, 50, 1], [4096] * 40 + [33]]
+    for kind, hq, hkv, dqk, dv, n_gh, rows_per_group, parts, cps in shapes:
+        shape = binding.make_shape(kind, hq, hkv, dqk, dv, 64, 0.0)
+        for lens in cases:
+            for splits in (2, 4, 8, 64):
+                rows = [[n] for n in lens]
+                p = host_shim.plan(rows, n_gh, splits, cps)           # raises if the bound is exceeded
+                n_spans = len(p["row"])
+                part_rows = n_spans * parts * rows_per_group
+                need = -(-p["table_bytes"] // 256) * 256 + 256 + -(-part_rows * dv * 4 // 256) * 256 + -(-part_rows * 4 // 256) * 256
+                got = binding.ipkv_attend_scratch_bytes(shape, len(rows), len(rows), sum(lens), splits)
+                assert need <= got, (kind, lens[:2], splits, n_spans, need, got)
+
+
 def test_balancing_threshold_follows_the_measured_crossovers():
     """The rule that decides when the grouped-query kernel balances its load: 64 tiles per CTA while the split reduce
     fits one wave of CTAs, more for larger batches (the two measured cross-overs: 60-70 tiles per CTA for 16 rows x
