@@ -274,7 +274,18 @@ typedef struct {
   uint32_t device_status;       /* nonzero after a kernel's bounded wait gave up (synchronises): bit 0 a producer
                                    got no free stage, bit 1 a consumer got no tile, bit 2 a copy did not land  */
 } ipkv_stats;
+/* Synchronises the device and fills *out.  If a bounded wait inside one of the handle's kernels gave up since the last
+ * call, *out is still filled (device_status says which wait), the call returns IPKV_ETIMEOUT (the results of the
+ * attention calls since the last ipkv_get_stats are then invalid) and the device word is cleared, so the calls that
+ * follow are judged on their own. */
 ipkv_status ipkv_get_stats(ipkv_t* h, ipkv_stats* out);
+
+/* Self-test of the failure path (no counterpart in the paper): enqueues a one-CTA kernel in which a consumer thread
+ * waits limit_us microseconds (1 .. 1 000 000) for a tile that is announced on its stage barrier and never copied.
+ * The wait runs out, the kernel records "a consumer got no tile" in the handle's status word and returns; nothing
+ * faults and nothing spins without a limit.  The next ipkv_get_stats then returns IPKV_ETIMEOUT, the one after it
+ * IPKV_OK.  The attention kernels' own waits use the same routine with a limit of two seconds. */
+ipkv_status ipkv_selftest_expire_wait(ipkv_t* h, uint32_t limit_us, void* stream);
 
 /* ---- roofline share policy (host only; Sec. 5.2-5.3) ------------------------------------------------
  * Eq. 1: T_CPU(r) = r*A*L + C_cpu, T_GPU(r) = (1-r)*B*L + C_gpu, T = max(T_CPU, T_GPU) + T_merge.

@@ -1594,12 +1594,19 @@ ipkv_status ipkv_get_stats(ipkv_t* h, ipkv_stats* out) {
     }
     *out = h->stats;
     if (h->stats.device_status) {
-        std::string where;
-        if (h->stats.device_status & kStatusNoFreeStage) where += " [a producer got no free stage]";
-        if (h->stats.device_status & kStatusNoTile) where += " [a consumer got no tile]";
-        if (h->stats.device_status & kStatusCopyNotLanded) where += " [a copy did not land]";
-        return fail(h, IPKV_ETIMEOUT, "a kernel's bounded wait gave up; results of that call are invalid" + where);
+        // reported once: the word is cleared so that the calls after this one are judged on their own
+        CU(h, cudaMemset(h->status_dev, 0, sizeof(uint32_t)));
+        return fail(h, IPKV_ETIMEOUT, "a kernel's bounded wait gave up; results of that call are invalid" +
+                                          describe_device_status(h->stats.device_status));
     }
+    return IPKV_OK;
+}
+
+ipkv_status ipkv_selftest_expire_wait(ipkv_t* h, uint32_t limit_us, void* stream) {
+    if (!h || limit_us == 0 || limit_us > 1000000u) return IPKV_EINVAL;
+    DeviceGuard dev_guard(h->cfg.device);
+    CU(h, dev_guard.error());
+    CU(h, launch_expire_wait(h->status_dev, uint64_t(limit_us) * 1000ull, static_cast<cudaStream_t>(stream)));
     return IPKV_OK;
 }
 

@@ -126,6 +126,10 @@ cudaError_t launch_copy_spans(const CopySpans& spans, int n, cudaStream_t s);
 // into a CUDA graph and replayed after the host buffer is gone.
 cudaError_t launch_upload_by_value(void* dst_dev, const void* src_host, size_t bytes, cudaStream_t s);
 
+// Self-test: a one-CTA kernel whose consumer waits `limit_ns` for a tile that is announced and never copied, gives up
+// and ORs kStatusNoTile into *status (probe.cu).
+cudaError_t launch_expire_wait(uint32_t* status, uint64_t limit_ns, cudaStream_t s);
+
 constexpr int kAppendRowsPerLaunch = 64;
 struct AppendRows {
     int64_t dst_off[kAppendRowsPerLaunch];   // byte offset of the row's window (first block) from w_base

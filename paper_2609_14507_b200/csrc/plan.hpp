@@ -12,6 +12,7 @@
 #include <algorithm>
 #include <cstdint>
 #include <cstring>
+#include <string>
 #include <vector>
 
 #include "kernels.h"
@@ -31,6 +32,16 @@ constexpr int kMinTilesPerCtaPerReduceWave = 28;
 inline int64_t min_tiles_per_cta_to_balance(int64_t n_rows, int n_q_heads) {
     const double waves = double(n_rows) * n_q_heads / (kSmCount * 4.0);
     return kMinTilesPerCtaToBalance + (waves > 1.0 ? int64_t(kMinTilesPerCtaPerReduceWave * (waves - 1.0)) : 0);
+}
+
+// What the bits of the device status word mean, for error messages (empty for 0).
+inline std::string describe_device_status(uint32_t status) {
+    std::string where;
+    if (status & kStatusNoFreeStage) where += " [a producer got no free stage]";
+    if (status & kStatusNoTile) where += " [a consumer got no tile]";
+    if (status & kStatusCopyNotLanded) where += " [a copy did not land]";
+    if (status & ~(kStatusNoFreeStage | kStatusNoTile | kStatusCopyNotLanded)) where += " [unknown bits]";
+    return where;
 }
 
 struct PlanSeg { int base_id; int64_t off; int64_t n_tokens; bool appended = false; };

@@ -7,6 +7,7 @@
 #include <cstdint>
 
 #include "../../include/ipkv.h"
+#include "kernels.h"
 #include "ptx.cuh"
 
 namespace ipkvi {
@@ -40,11 +41,34 @@ __global__ void __launch_bounds__(32) read_ring_kernel(const char* src, int64_t 
             ptx::bulk_g2s_hint(s_base + st * kProbeStageBytes, base + i * kProbeStageBytes, kProbeStageBytes, s_full + 8 * st, pol);
         }
     }
-    if (!ok) atomicOr(status, 1u);
+    if (!ok) atomicOr(status, kStatusNoTile);
     if (acc == 0x9e3779b9u) *sink = acc;               // keeps the loads alive
 }
 
+
+// Self-test of the bounded waits: one CTA; its producer thread announces a tile on a stage barrier (expect_tx) and
+// then issues no copy for it; a consumer thread waits for that tile with a short limit.  The wait runs out, the
+// consumer records kStatusNoTile and the kernel returns: nothing spins without a limit, nothing faults, no copy is in
+// flight when the CTA leaves.
+__global__ void __launch_bounds__(64) expire_wait_kernel(uint32_t* status, uint64_t limit_ns) {
+    __shared__ __align__(8) uint64_t bar_storage;
+    const uint32_t bar = ptx::smem_addr(&bar_storage);
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(bar, 1);
+        ptx::mbar_fence_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) ptx::mbar_expect_tx(bar, 16);          // a tile of 16 bytes that never comes
+    if (threadIdx.x == 32 && !ptx::mbar_wait(bar, 0, limit_ns)) atomicOr(status, kStatusNoTile);
+}
+
 }  // namespace
+
+cudaError_t launch_expire_wait(uint32_t* status, uint64_t limit_ns, cudaStream_t s) {
+    expire_wait_kernel<<<1, 64, 0, s>>>(status, limit_ns);
+    return cudaGetLastError();
+}
+
 }  // namespace ipkvi
 
 using namespace ipkvi;

@@ -38,13 +38,15 @@ __device__ __forceinline__ uint64_t globaltimer_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-// Bounded wait: gives up after about two seconds and reports failure instead of spinning forever.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+// Bounded wait: gives up after `limit_ns` (two seconds unless the caller says otherwise) and reports failure instead of
+// spinning forever.
+constexpr uint64_t kWaitLimitNs = 2000000000ull;
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint64_t limit_ns = kWaitLimitNs) {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = globaltimer_ns();
     uint32_t n = 0;
     while (!mbar_try_wait(bar, parity)) {
-        if ((++n & 63u) == 0 && globaltimer_ns() - t0 > 2000000000ull) return false;
+        if ((++n & 63u) == 0 && globaltimer_ns() - t0 > limit_ns) return false;
     }
     return true;
 }

@@ -81,6 +81,15 @@ int shim_plan(int n_rows, const int32_t* row_start, const int64_t* seg_tokens, i
     return n;
 }
 
+// the text the library puts behind IPKV_ETIMEOUT for a device status word
+int shim_describe_status(uint32_t status, char* out, int cap) {
+    const std::string s = describe_device_status(status);
+    if (int(s.size()) + 1 > cap) return -1;
+    std::memcpy(out, s.c_str(), s.size() + 1);
+    return int(s.size());
+}
+uint32_t shim_status_bit(int which) { return which == 0 ? kStatusNoFreeStage : which == 1 ? kStatusNoTile : kStatusCopyNotLanded; }
+
 int64_t shim_tile_chunk_offset(int32_t bt, int32_t t, int32_t chunk) { return tile_chunk_offset(bt, t, chunk); }
 int64_t shim_plain_chunk_offset(int32_t d, int32_t t, int32_t chunk) { return plain_chunk_offset(d, t, chunk); }
 int64_t shim_block_bytes(int32_t hkv, int32_t dqk, int32_t dv_stored, int32_t bt) {

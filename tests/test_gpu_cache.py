@@ -1,6 +1,7 @@
 """GPU parity of the handle-based path (create / append / flush / attend_gpu / merge / views) against the
 oracle: routing indices and region contents bit-exact, partial and merged outputs within tolerance."""
 import ctypes as C
+import time
 
 import numpy as np
 import pytest
@@ -824,3 +825,35 @@ def test_early_copy_start_under_a_random_program():
         parts = [c_oracle.attend(q[s], snap[s][0], snap[s][1], np.nonzero(snap[s][2] != 0)[0], scale) for s in seqs]
         check_partial(outs_a[j][0].cpu().numpy(), outs_a[j][1].cpu().numpy(), np.stack([p[0] for p in parts]),
                       np.stack([p[1] for p in parts]), f"last launch of layer {layer}")
+
+
+def test_a_wait_that_runs_out_is_reported_once_and_the_handle_stays_usable():
+    """Failure detection without a fault: a one-CTA self-test kernel waits 1 ms for a tile that is announced and never
+    copied, gives up, records the status bit and returns.  The next ipkv_get_stats reports IPKV_ETIMEOUT (and says
+    which wait), the word is cleared, and a normal attention call on the same handle then works and matches the oracle."""
+    sh = synth.SMALL_GQA
+    L = 300
+    k, v = synth.host_kv(sh, L, seed=71)
+    q = synth.host_q(sh, 1, seed=72)
+    cfg = binding.make_config(binding.GQA, 1, 1, sh.n_q_heads, sh.n_kv_heads, sh.dim_qk, sh.dim_v, block_tokens=64,
+                              window_tokens=256, chunk_tokens=512, max_u_tokens_per_seq=1024, max_p_tokens_per_seq=1024,
+                              resident_tokens_per_seq=1024, softmax_scale=sh.scale)
+    with binding.Cache(cfg) as cache:
+        cache.append_bulk(0, 0, synth.bits_to_torch(k, DEV), synth.bits_to_torch(v, DEV), L, 0, 1)
+        assert cache.get_stats()["device_status"] == 0
+        t0 = time.perf_counter()
+        cache.selftest_expire_wait(1000)
+        with pytest.raises(binding.IpkvError) as err:
+            cache.get_stats()
+        assert time.perf_counter() - t0 < 1.0                       # the wait gave up after a millisecond, not after two seconds
+        assert err.value.status == 6 and "no tile" in str(err.value)  # IPKV_ETIMEOUT
+        assert cache.get_stats()["device_status"] == 0              # reported once
+        o = torch.zeros((1, sh.n_q_heads, sh.dim_v), device=DEV); lse = torch.zeros((1, sh.n_q_heads), device=DEV)
+        cache.attend_gpu(0, [0], synth.bits_to_torch(q, DEV), o, lse)
+        torch.cuda.synchronize()
+        assert cache.get_stats()["device_status"] == 0
+        o_ref, l_ref = c_oracle.attend(q[0], k, v, np.arange(L), float(np.float32(sh.scale)))
+        check_partial(o.cpu().numpy()[0], lse.cpu().numpy()[0], o_ref, l_ref, "after a reported timeout")
+    with pytest.raises(binding.IpkvError):
+        with binding.Cache(cfg) as cache:
+            cache.selftest_expire_wait(0)                           # limit out of range

@@ -208,3 +208,24 @@ def test_bad_configs_are_rejected_and_no_gpu_fails_loudly():
         with pytest.raises(binding.IpkvError) as e:
             binding.Cache(cfg)
         assert e.value.status == 5          # IPKV_ECUDA: no silent CPU path
+
+
+def test_device_status_word_maps_to_the_documented_messages():
+    """Bits of the device status word (which bounded wait of a kernel gave up) -> the text behind IPKV_ETIMEOUT."""
+    import ctypes
+    L = host_shim.lib()
+    L.shim_status_bit.restype = ctypes.c_uint32
+    bits = [L.shim_status_bit(i) for i in range(3)]
+    assert bits == [1, 2, 4]                      # the values include/ipkv.h documents for ipkv_stats.device_status
+
+    def text(word):
+        buf = ctypes.create_string_buffer(256)
+        assert L.shim_describe_status(ctypes.c_uint32(word), buf, 256) >= 0
+        return buf.value.decode()
+
+    assert text(0) == ""
+    assert "free stage" in text(1) and "tile" not in text(1)
+    assert "no tile" in text(2) and "free stage" not in text(2)
+    assert "did not land" in text(4)
+    assert all(k in text(7) for k in ("free stage", "no tile", "did not land"))
+    assert "unknown" in text(8)

@@ -1,4 +1,4 @@
-"""The allocation-free attention entry point against the ordinary one.
+"""The allocation-free attention entry point against the ordinary one and against the oracle.
 
 ipkv_attend_runs_noalloc is for callers that cannot allocate device memory where they call attention (a server
 whose pool owns all memory, a latency-critical loop, a plug-in that may not allocate): its scratch is a fixed
@@ -9,7 +9,7 @@ import numpy as np
 import pytest
 
 from paper_2609_14507_b200 import binding, synth
-from tests.gpu_util import pack_run, shape_of
+from tests.gpu_util import check_partial, oracle_rows, pack_run, shape_of
 
 pytestmark = pytest.mark.gpu
 torch = pytest.importorskip("torch")
@@ -75,6 +75,95 @@ def test_noalloc_rejects_problems_beyond_its_array():
     with pytest.raises(binding.IpkvError) as e:
         binding.ipkv_attend_runs_noalloc(shape, rows, q, o, lse, kv_splits=64)
     assert e.value.status == 3
+    torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("kind", ["gqa", "mla"])
+def test_noalloc_matches_the_oracle(kind):
+    """The call judged on its own, not through the ordinary entry point: element-wise against the float64 oracle."""
+    rng = np.random.default_rng(81)
+    rows = [[1500, 70], [333], []]
+    if kind == "gqa":
+        hq, hkv, dqk, dv, scale = 32, 4, 128, 128, 128 ** -0.5
+        shape = shape_of(binding.GQA, hq, hkv, dqk, dv, 64)
+    else:
+        hq, hkv, dqk, dv, scale = 16, 1, 576, 512, 192 ** -0.5
+        shape = shape_of(binding.MLA, hq, hkv, dqk, dv, 64, scale)
+    q = synth.normal_bf16(rng, (len(rows), hq, dqk))
+    keep, runs, rows_kv = [], [], []
+    for row in rows:
+        ks, vs, rr = [], [], []
+        for n in row:
+            k = synth.normal_bf16(rng, (n, hkv, dqk))
+            v = None if kind == "mla" else synth.normal_bf16(rng, (n, hkv, dv))
+            buf = pack_run(shape, k, v)
+            keep.append(buf); rr.append((buf, n)); ks.append(k); vs.append(v)
+        runs.append(rr)
+        kk = np.concatenate(ks) if ks else np.zeros((0, hkv, dqk), np.uint16)
+        vv = None if kind == "mla" else (np.concatenate(vs) if vs else np.zeros((0, hkv, dv), np.uint16))
+        rows_kv.append((kk, vv))
+    o = torch.full((len(rows), hq, dv), float("nan"), device="cuda:0")
+    lse = torch.full((len(rows), hq), float("nan"), device="cuda:0")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda:0")
+    binding.ipkv_attend_runs_noalloc(shape, runs, synth.bits_to_torch(q, "cuda:0"), o, lse, 3, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    o_ref, l_ref = oracle_rows(q, rows_kv, float(np.float32(scale)), dv_alias=dv if kind == "mla" else None)
+    check_partial(o.cpu().numpy(), lse.cpu().numpy(), o_ref, l_ref, f"noalloc {kind}")
+
+
+def test_noalloc_leaves_device_memory_as_it_found_it():
+    """What the name promises: across a hundred calls neither the driver's free memory nor the caller's own allocator
+    moves.  The measurement starts after a first burst of the same hundred calls: the first call on a device makes the
+    driver set the array aside, and a fresh process's first queue of launches this deep makes the driver grow its own
+    launch buffers once; neither is an allocation by the call."""
+    shape, q, runs, _keep = _case(82, [[2000, 64], [500]])
+    o = torch.zeros((2, shape.n_q_heads, shape.dim_v), device="cuda:0")
+    lse = torch.zeros((2, shape.n_q_heads), device="cuda:0")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda:0")
+
+    def burst():
+        for _ in range(100):
+            binding.ipkv_attend_runs_noalloc(shape, runs, q, o, lse, 2, status)
+        torch.cuda.synchronize()
+        return torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+
+    import gc
+    gc.collect()                    # tensors of earlier tests must not be released in the middle of the measurement
+    burst()
+    before = burst()
+    after = burst()
+    assert after == before, (before, after)
+    assert int(status.item()) == 0
+
+
+def test_noalloc_accepts_the_largest_problem_that_fits_and_refuses_the_next():
+    """The limit is the array's 16 MiB: with one 64-token run per row and no explicit splits, the largest batch whose
+    scratch still fits is computed (all rows share one run), and one row more is refused with IPKV_ERANGE."""
+    shape = shape_of(binding.GQA, 32, 4, 128, 128, 64)
+    limit = binding.ipkv_noalloc_scratch_limit()
+    need = lambda n: binding.ipkv_attend_scratch_bytes(shape, n, n, 64 * n, 0)
+    n = 1
+    while need(n + 1) <= limit:
+        n += 1
+    assert need(n) <= limit < need(n + 1) and n > 64
+    rng = np.random.default_rng(83)
+    k = synth.normal_bf16(rng, (64, 4, 128)); v = synth.normal_bf16(rng, (64, 4, 128))
+    buf = pack_run(shape, k, v)
+    q = synth.normal_bf16(rng, (n + 1, 32, 128))
+    qd = synth.bits_to_torch(q, "cuda:0")
+    o = torch.full((n + 1, 32, 128), float("nan"), device="cuda:0"); lse = torch.full((n + 1, 32), float("nan"), device="cuda:0")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda:0")
+    binding.ipkv_attend_runs_noalloc(shape, [[(buf, 64)]] * n, qd[:n], o[:n], lse[:n], 0, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    sample = [0, n // 2, n - 1]
+    o_ref, l_ref = oracle_rows(q[sample], [(k, v)] * len(sample), float(np.float32(128 ** -0.5)))
+    check_partial(o.cpu().numpy()[sample], lse.cpu().numpy()[sample], o_ref, l_ref, "noalloc at the limit")
+    assert torch.isfinite(o[:n]).all()
+    with pytest.raises(binding.IpkvError) as e:
+        binding.ipkv_attend_runs_noalloc(shape, [[(buf, 64)]] * (n + 1), qd, o, lse, 0, status)
+    assert e.value.status == 3                                     # IPKV_ERANGE, nothing launched
     torch.cuda.synchronize()
 
 
