@@ -53,17 +53,21 @@ WORKLOADS = {
     # BASELINE config 1 (single layer, batch 1, 4K): latency-bound, for quick checks
     "small-gqa-bs1-4k-cpu50": dict(shape=synth.SMALL_GQA, batch=1, ctx=4096, share=(1, 2), cfg_id=1),
 }
-# dram__bytes_read.sum + dram__bytes_write.sum of one attention-kernel launch, from the ncu captures summarised under
-# profiles/ (captured on the 2-layer case, whose per-layer launch is the full-size workload's launch).
+# dram__bytes_read.sum + dram__bytes_write.sum of one attention-kernel launch, read from one ncu capture per kernel
+# (taken on the 2-layer case of each shape, whose per-layer launch is the full-size workload's launch): read + write bytes.
 DRAM_TRAFFIC_PER_LAUNCH = {
-    "mixtral-8x7b-bs16-32k-cpu25": 1615.2e6 + 5.3e6,        # profiles/attn_gqa_kernel_mixtral-2layers-bs16-32k-cpu25.md
+    "mixtral-8x7b-bs16-32k-cpu25": 1615.2e6 + 5.3e6,
     "mixtral-2layers-bs16-32k-cpu25": 1615.2e6 + 5.3e6,
-    "qwen3-30b-a3b-bs16-32k-cpu0": 1076.1e6 + 4.6e6,        # profiles/attn_gqa_kernel_qwen3-2layers-bs16-32k-cpu0.md
+    "qwen3-30b-a3b-bs16-32k-cpu0": 1076.1e6 + 4.6e6,
     "qwen3-2layers-bs16-32k-cpu0": 1076.1e6 + 4.6e6,
-    "deepseek-v2-lite-mla-bs8-128k-cpu40": 725.7e6 + 5.6e6,  # profiles/attn_mla_kernel_deepseek-v2-lite-2layers-bs8-128k-cpu40.md
+    "deepseek-v2-lite-mla-bs8-128k-cpu40": 725.7e6 + 5.6e6,
     "deepseek-v2-lite-mla-2layers-bs8-128k-cpu40": 725.7e6 + 5.6e6,
 }
 DEFAULT_WORKLOAD = "mixtral-8x7b-bs16-32k-cpu25"
+# Short runs of the other BASELINE configurations, reported beside the default line (rank 0, one GPU): config 3 at CPU
+# share 0 and 70 %, config 4 (compressed-latent kernel), config 5 at CPU share 0.
+OTHER_CONFIGS = ["qwen3-30b-a3b-bs16-32k-cpu0", "qwen3-30b-a3b-bs16-32k-cpu70", "deepseek-v2-lite-mla-bs8-128k-cpu40",
+                 "qwen3-ragged-bs64-1m-16layers-cpu0"]
 BLOCK, WINDOW = 64, 256
 
 # BASELINE config 5: Qwen3 shape, batch 64, ragged context lengths uniform in [8192, 24576] (about 1M tokens in all),
@@ -194,7 +198,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + self.FIELDS,
-                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE,
+                                          "--format=csv,noheader,nounits", "-lms", "20"], stdout=subprocess.PIPE,
                                          stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
@@ -207,7 +211,7 @@ class ClockSampler:
             self.rows.append((time.time(), [x.strip() for x in line.split(",")]))
 
     def mark(self):
-        """Start of the timed region: earlier samples are dropped."""
+        """Start of the load (the first warm-up step): earlier samples are dropped."""
         self.t_mark = time.time()
 
     def stop(self):
@@ -282,6 +286,23 @@ def oracle_sample(wl, seconds_target=15.0, threads=None):
     return dict(value=done_tokens / t_total, unit=UNIT, cores=used, kind="oracle", host_cpus=os.cpu_count(), single_thread_value=single,
                 sample=f"{n_pairs} of {sh.n_layers * wl['batch']} (layer, sequence) pairs, GPU-side share ({done_tokens} KV-tokens "
                        f"in all), all heads; {t_total:.1f} s of float64 C++ (OpenMP over query heads)")
+
+
+def other_config(name, steps=10, warmup=3):
+    """One short run of another workload in a process of its own (its cache needs the whole device); the headline
+    figures of its JSON line."""
+    cmd = [sys.executable, os.path.join(ROOT, "bench.py"), "--workload", name, "--steps", str(steps), "--warmup", str(warmup),
+           "--no-cpu-baseline", "--no-read-ceiling", "--no-other-configs"]
+    try:
+        r = subprocess.run(cmd, capture_output=True, text=True, timeout=900, cwd=ROOT)
+        d = json.loads(r.stdout.strip().splitlines()[-1])
+    except Exception as e:                                  # noqa: BLE001 - reported in the line, the headline stands
+        return {"workload": name, "error": repr(e)[:200]}
+    rf = d["roofline"]
+    return {"workload": name, "steps": steps, "ms_per_step": d["ms_per_step"], "value": d["value"], "kernel": rf["kernel"],
+            "achieved": rf["achieved"], "frac": rf["frac"], "avg_launch_us": rf["avg_launch_us"], "step_gbs": d["step_gbs"],
+            "e2e_ms_per_step": d["e2e"]["ms_per_step"] if d.get("e2e") else None,
+            "sm_mhz": (d.get("clocks") or {}).get("sm_mhz"), "layers": d["config"]["layers"]}
 
 
 def run_reference(args, wl, name):
@@ -464,6 +485,8 @@ def main():
     ap.add_argument("--latency", action="store_true", help="also time every step separately and report P50 / P99 / max")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-other-configs", action="store_true",
+                    help="default workload only: skip the short runs of the other BASELINE configurations (other_configs in the line)")
     args = ap.parse_args()
     wl = WORKLOADS[args.workload]
     if args.impl == "reference":
@@ -546,6 +569,8 @@ def main():
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
+        time.sleep(0.1)                 # nvidia-smi needs a moment before its first line
+    sampler.mark()                      # the samples kept are those taken under load: warm-up, timed region, end-to-end region
     for _ in range(args.warmup):
         step()
     barrier()
@@ -554,7 +579,6 @@ def main():
     args.time_every = max(1, min(args.time_every, args.steps * sh.n_layers // 24))
     cache.profile_enable(not args.no_kernel_timing, reduce=args.profile_reduce, every=args.time_every)
     cache.profile_read()
-    sampler.mark()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]       # one event per step: medians and tails
     e0.record()
@@ -566,7 +590,6 @@ def main():
         marks[-1].record()
     e1.record()
     barrier()
-    clocks = sampler.stop() if rank == 0 else None
     ms = max_over_ranks(e0.elapsed_time(e1))
     raw = [marks[i].elapsed_time(marks[i + 1]) for i in range(args.steps)]
     lat = sorted(raw)
@@ -688,6 +711,7 @@ def main():
         h2d = NL * (hq[0].numel() * 2 + hk[0].numel() * 2 + (0 if hv is None else hv[0].numel() * 2) + hoc[0].numel() * 4 + hlc[0].numel() * 4)
         e2e = {"value": reduce_over_ranks(tok2, "sum", dev) / (ms2 * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": NL * hout[0].numel() * hout.element_size(), "ms_per_step": ms2 / args.steps}
+    clocks = sampler.stop() if rank == 0 else None
     status = cache.get_stats()["device_status"]
     if status != 0:
         raise RuntimeError("a kernel reported a timed-out wait; the numbers are invalid")
@@ -701,10 +725,15 @@ def main():
         l2_note = "NOT flushed: the %.1f MB a step reads stay L2-resident between steps; a latency case, not a bandwidth number" % (
             step_bytes / 1e6)
     cpu = None
+    others = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cache.close()
         torch.cuda.empty_cache()
         cpu = oracle_sample(wl)
+    if rank == 0 and world == 1 and args.workload == DEFAULT_WORKLOAD and not args.no_other_configs:
+        cache.close()                   # the other workloads need the device memory
+        torch.cuda.empty_cache()
+        others = [other_config(name) for name in OTHER_CONFIGS]
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -725,6 +754,8 @@ def main():
         }
         if step_lat:
             line["step_latency"] = step_lat
+        if others is not None:
+            line["other_configs"] = others
         if wl.get("host_copies"):
             line["config"]["host_copies_of_U_and_P"] = "on (P pinned, U unpinned); write-back on a copy stream"
         if wl.get("grow_p"):
