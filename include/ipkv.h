@@ -216,6 +216,9 @@ ipkv_status ipkv_attend_gpu_sparse(ipkv_t* h, int32_t layer, const int32_t* seq_
  * lse_part_host [n_seq][n_q_heads] fp32 in host memory (pinned memory lets the later copy to the GPU overlap).
  * The call runs synchronously on the calling thread plus OpenMP workers (n_threads <= 0: all cores).
  * U is filled by device-to-host copies queued by the append / flush calls: synchronise their stream first.
+ * This call may run on a second host thread while ipkv_attend_gpu / ipkv_merge of the same handle run on the first
+ * (the paper's step: both engines at once, one join): it only reads the routing state.  No call that changes routing
+ * (append, flush, set_share, reset) may run at the same time.
  * Fails with IPKV_ESTATE if U contents are not kept (IPKV_FLAG_NO_HOST_U). */
 ipkv_status ipkv_attend_cpu(ipkv_t* h, int32_t layer, const int32_t* seq_ids, int32_t n_seq, const void* q_host,
                             float* o_part_host, float* lse_part_host, int32_t n_threads);

@@ -1,6 +1,7 @@
 """GPU parity of the handle-based path (create / append / flush / attend_gpu / merge / views) against the
 oracle: routing indices and region contents bit-exact, partial and merged outputs within tolerance."""
 import ctypes as C
+import threading
 import time
 
 import numpy as np
@@ -857,3 +858,79 @@ def test_a_wait_that_runs_out_is_reported_once_and_the_handle_stays_usable():
     with pytest.raises(binding.IpkvError):
         with binding.Cache(cfg) as cache:
             cache.selftest_expire_wait(0)                           # limit out of range
+
+
+def test_closed_loop_two_engines_run_concurrently_and_the_policy_steers_the_share():
+    """The method's feedback loop on a live cache (Sec. 4.2, 5.2, 5.3): every decode step a host thread runs the CPU
+    engine over region U while the GPU attends P and the D-window; the two partials are joined once; the CPU engine's
+    wall time goes into the policy's sliding window, and once per D-window the policy's new marginal share is handed to
+    ipkv_set_share.  The share sequence the policy produced (whatever this host's speed made it) is replayed into the
+    oracle's router: routing must agree bit for bit, merged outputs within tolerance, across several evictions."""
+    sh = synth.Shape("q-loop", "gqa", 1, 32, 4, 128, 128, 128 ** -0.5)
+    rng = np.random.default_rng(97)
+    scale = float(np.float32(sh.scale))
+    bt, D, den, B, L0, steps = 64, 64, 16, 3, 1536, 4 * 64 + 9
+    hq, dv = sh.n_q_heads, sh.dim_v
+    # B = seconds per KV token on the GPU side: a guess that a first estimate of A then has to be weighed against
+    policy = binding.Policy(A=2e-7, B=2e-7, C_cpu=0.0, C_gpu=0.0, window_steps=64, share_den=den)
+    num0 = policy.prefill_share(L0)
+    assert 0 <= num0 <= den
+    with make_cache(sh, 1, B, block_tokens=bt, window_tokens=D, chunk_tokens=256, max_u_tokens_per_seq=4096,
+                    max_p_tokens_per_seq=4096, resident_tokens_per_seq=4096, share_num=num0, share_den=den) as cache:
+        seqs = list(range(B))
+        refs = []
+        for s_ in seqs:
+            r = RefSeq(sh, bt, D, num0, den)
+            k, v = synth.host_kv(sh, L0, seed=9700 + s_)
+            cache.append_bulk(0, s_, synth.bits_to_torch(k, DEV), synth.bits_to_torch(v, DEV), L0, num0, den)
+            r.bulk(k, v, num0, den)
+            refs.append(r)
+        q_host = torch.zeros((B, hq, sh.dim_qk), dtype=torch.bfloat16).pin_memory()
+        o_cpu = torch.zeros((B, hq, dv)).pin_memory(); l_cpu = torch.zeros((B, hq)).pin_memory()
+        o_gpu = torch.zeros((B, hq, dv), device=DEV); l_gpu = torch.zeros((B, hq), device=DEV)
+        out = torch.zeros((B * hq, dv), device=DEV); out_lse = torch.zeros(B * hq, device=DEV)
+        shares, overlapped, t_cpu_box = [], 0, [0.0]
+
+        def cpu_side():
+            t0 = time.perf_counter()
+            cache.attend_cpu(0, seqs, q_host, o_cpu, l_cpu)
+            t_cpu_box[0] = time.perf_counter() - t0
+
+        for step in range(steps):
+            k = synth.normal_bf16(rng, (B, sh.n_kv_heads, sh.dim_qk)); v = synth.normal_bf16(rng, (B, sh.n_kv_heads, dv))
+            cache.append(0, seqs, synth.bits_to_torch(k, DEV), synth.bits_to_torch(v, DEV))
+            for i, r in enumerate(refs):
+                r.append(k[i:i + 1], v[i:i + 1])
+            q = synth.normal_bf16(rng, (B, hq, sh.dim_qk))
+            q_host.copy_(synth.bits_to_torch(q))
+            # the two engines, at the same time: the thread computes over U in place, this thread queues the GPU side
+            th = threading.Thread(target=cpu_side)
+            th.start()
+            cache.attend_gpu(0, seqs, q_host.to(DEV, non_blocking=True), o_gpu, l_gpu)
+            overlapped += th.is_alive()
+            th.join()
+            cache.merge(B * hq, dv, [o_gpu.view(-1, dv), o_cpu.view(-1, dv)], [l_gpu.view(-1), l_cpu.view(-1)], out, out_lse)
+            n_u = sum(r.route.counts()["n_u"] for r in refs)
+            policy.observe(t_cpu_box[0], float(n_u))
+            if (step + 1) % D == 0:                      # once per D-window: re-estimate A, steer the next eviction batches
+                num, model = policy.update()
+                assert 0 <= num <= den and model["A"] > 0
+                cache.set_share(num)
+                for r in refs:
+                    r.route.set_share(num)
+                shares.append(num)
+            if step in (0, D - 1, D, 2 * D + 5, steps - 1):
+                torch.cuda.synchronize()
+                full = [r.attend(q[i], "all", scale) for i, r in enumerate(refs)]
+                check_partial(out.cpu().numpy().reshape(B, hq, dv), out_lse.cpu().numpy().reshape(B, hq),
+                              np.stack([w[0] for w in full]), np.stack([w[1] for w in full]), f"closed loop step {step}")
+                cpu_ref = [r.attend(q[i], "cpu", scale) for i, r in enumerate(refs)]
+                check_partial(o_cpu.numpy(), l_cpu.numpy(), np.stack([w[0] for w in cpu_ref]), np.stack([w[1] for w in cpu_ref]),
+                              f"CPU engine step {step}")
+        torch.cuda.synchronize()
+        assert len(shares) == 4 and all(r.route.counts()["n_flush"] >= 4 for r in refs)
+        for s_, r in enumerate(refs):
+            check_routing(cache, 0, s_, r)
+            check_contents(cache, 0, s_, r, [0, L0 - 1, L0, L0 + D, L0 + steps - 1])
+        assert overlapped > 0                            # the CPU engine was still running when the GPU call had returned
+        assert cache.get_stats()["device_status"] == 0
