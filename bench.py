@@ -400,6 +400,118 @@ def cpu_engine_microbench():
     print(json.dumps({"cpu_engine_microbench": out}))
 
 
+def two_engine_bench(steps=None, resident=False):
+    """The paper's whole decode step with both engines live (Sec. 4.2, Eq. 1-2): per layer a host thread runs the CPU
+    engine over region U in place WHILE the GPU attends P and the D-window; one join per layer; the CPU engine's wall
+    time feeds the policy's sliding window and once per D-window the policy's marginal share goes to ipkv_set_share.
+    Qwen3 shape, batch 8, 8K context, 12 layers, host copies of U and P on.  By default the GPU side is the paper's:
+    nothing of P stays on the device, every chunk is streamed from pinned host memory through two slots each step
+    (`--two-engine-resident` keeps P in HBM instead: the B200 adaptation, where the GPU side is so much cheaper per
+    token than the CPU side that Eq. 2 sends the share to zero)."""
+    import queue
+    import torch
+    from paper_2609_14507_b200 import binding
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    sh = synth.Shape("qwen3-12l", "gqa", 12, 32, 4, 128, 128, 128 ** -0.5)
+    NL, Bn, L0, D, den = sh.n_layers, 8, 8192, 64, 64
+    steps = steps or 5 * D
+    cap = L0 + steps + 2 * D
+    num0 = den // 2                                          # prefill share 1/2; the decode batches follow the policy
+    policy = None                                            # created after the first steps have calibrated B
+    cfg = binding.make_config(binding.GQA, NL, Bn, sh.n_q_heads, sh.n_kv_heads, sh.dim_qk, sh.dim_v, block_tokens=BLOCK,
+                              window_tokens=D, chunk_tokens=1024, n_slots=2, max_u_tokens_per_seq=cap, max_p_tokens_per_seq=cap,
+                              resident_tokens_per_seq=cap if resident else 0, softmax_scale=sh.scale, share_num=num0, share_den=den,
+                              flags=0)
+    ids = list(range(Bn))
+    with binding.Cache(cfg) as cache:
+        for layer in range(NL):
+            for s_ in range(Bn):
+                k, v = synth.device_kv(sh, L0, 31000 + layer * Bn + s_, dev)
+                cache.append_bulk(layer, s_, k, v, L0, num0, den)
+            torch.cuda.synchronize()
+        g = torch.Generator(device=dev); g.manual_seed(5)
+        bf = torch.bfloat16
+        q = torch.randn((NL, Bn, sh.n_q_heads, sh.dim_qk), generator=g, device=dev).to(bf)
+        kn = torch.randn((NL, Bn, sh.n_kv_heads, sh.dim_qk), generator=g, device=dev).to(bf)
+        vn = torch.randn((NL, Bn, sh.n_kv_heads, sh.dim_v), generator=g, device=dev).to(bf)
+        q_host = q.cpu().pin_memory()
+        rows, dv = Bn * sh.n_q_heads, sh.dim_v
+        o_cpu = torch.zeros((NL, rows, dv)).pin_memory(); l_cpu = torch.zeros((NL, rows)).pin_memory()
+        o_gpu = torch.zeros((rows, dv), device=dev); l_gpu = torch.zeros((rows,), device=dev)
+        out = torch.zeros((NL, rows, dv), device=dev); out_lse = torch.zeros((rows,), device=dev)
+        jobs, done = queue.Queue(), queue.Queue()
+
+        def worker():                                       # the CPU engine's thread: one layer per job
+            while True:
+                layer = jobs.get()
+                if layer is None:
+                    return
+                t0 = time.perf_counter()
+                cache.attend_cpu(layer, ids, q_host[layer], o_cpu[layer].view(Bn, sh.n_q_heads, dv), l_cpu[layer].view(Bn, sh.n_q_heads))
+                done.put(time.perf_counter() - t0)
+
+        th = threading.Thread(target=worker, daemon=True)
+        th.start()
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(NL)]
+        rec, shares = [], [num0]
+        for step in range(steps):
+            for layer in range(NL):                         # routing first: nothing may change it while the CPU engine reads it
+                cache.append(layer, ids, kn[layer], vn[layer])
+            torch.cuda.synchronize()
+            t_cpu = 0.0
+            w0 = time.perf_counter()
+            for layer in range(NL):
+                jobs.put(layer)
+                ev[layer][0].record()
+                cache.attend_gpu(layer, ids, q[layer], o_gpu.view(Bn, sh.n_q_heads, dv), l_gpu.view(Bn, sh.n_q_heads))
+                ev[layer][1].record()
+                t_cpu += done.get()                         # the join: both partials of the layer exist
+                ev[layer][2].record()
+                cache.merge(rows, dv, [o_gpu, o_cpu[layer]], [l_gpu, l_cpu[layer]], out[layer], out_lse)
+                ev[layer][3].record()
+            torch.cuda.synchronize()
+            wall = time.perf_counter() - w0
+            t_gpu = sum(ev[l][0].elapsed_time(ev[l][1]) for l in range(NL)) * 1e-3
+            t_merge = sum(ev[l][2].elapsed_time(ev[l][3]) for l in range(NL)) * 1e-3
+            c = [cache.counts(0, s_) for s_ in ids]
+            n_u = sum(x["n_u"] for x in c); n_g = sum(x["n_p"] + x["n_w"] for x in c)
+            if policy is None and step == 2:
+                # B (seconds per GPU-side KV token of one layer) is calibrated once, from the step just timed; A starts equal
+                b_cal = t_gpu / NL / max(1.0, n_g)
+                policy = binding.Policy(A=b_cal, B=b_cal, C_cpu=0.0, C_gpu=0.0, window_steps=256, share_den=den)
+            if policy is not None:
+                policy.observe(t_cpu / NL, float(n_u))     # one layer's CPU latency and the CPU-side tokens it attended
+            rec.append((wall, t_cpu, t_gpu, t_merge, n_u, n_g))
+            if (step + 1) % D == 0:
+                num, model = policy.update()
+                cache.set_share(num)
+                shares.append(num)
+        jobs.put(None)
+        th.join()
+        st = cache.get_stats()
+    tail = rec[len(rec) // 2:]                               # the second half: the policy has settled
+    med = lambda i: statistics.median(r[i] for r in tail)
+    wall, t_cpu, t_gpu, t_merge, n_u, n_g = (med(i) for i in range(6))
+    # the GPU-side time seen by the events contains the wait for the CPU side's join only through the merge: t_gpu is the
+    # attention call's own device time (for the streamed mode: copies and kernels of every chunk)
+    A = t_cpu / NL / max(1.0, n_u); Bc = t_gpu / NL / max(1.0, n_g)
+    L = (n_u + n_g) / Bn
+    r_eq2 = binding.ipkv_roofline_share(A, Bc, 0.0, 0.0, L)
+    print(json.dumps({"two_engine": {
+        "workload": "qwen3 shape, %d layers, batch %d, context %d + %d decode steps, D %d, GPU side %s" % (
+            NL, Bn, L0, steps, D, "HBM-resident" if resident else "streamed from pinned host memory (paper mode)"),
+        "per_step_ms": {"wall": wall * 1e3, "sum_T_cpu": t_cpu * 1e3, "sum_T_gpu": t_gpu * 1e3, "sum_T_merge": t_merge * 1e3,
+                        "eq1_max_plus_merge": (max(t_cpu, t_gpu) + t_merge) * 1e3},
+        "wall_over_eq1": wall / (max(t_cpu, t_gpu) + t_merge),
+        "cpu_share_now": n_u / max(1.0, n_u + n_g), "share_numerators_over_%d" % den: shares,
+        "A_s_per_cpu_token": A, "B_s_per_gpu_token": Bc, "eq2_share_from_measured_A_B": r_eq2,
+        "host_threads": os.cpu_count(), "device_status": st["device_status"],
+        "note": "T_cpu: wall time of ipkv_attend_cpu on its thread; T_gpu, T_merge: CUDA events on the stream; medians over the "
+                "second half of the steps; the engines run concurrently per layer, the join is ipkv_merge with the CPU partial "
+                "in pinned host memory"}}))
+
+
 def graph_microbench():
     """A launch-bound case replayed from a CUDA graph: the stateless attention call on the small configuration's
     shape (one sequence of 4096 tokens, 32 query / 4 KV heads, d 128: 4 MB of K/V, L2-resident) issued call by call
@@ -460,6 +572,9 @@ def main():
         return
     if "--cpu-engine-microbench" in sys.argv:
         cpu_engine_microbench()
+        return
+    if "--two-engine" in sys.argv or "--two-engine-resident" in sys.argv:
+        two_engine_bench(resident="--two-engine-resident" in sys.argv)
         return
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
