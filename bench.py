@@ -67,16 +67,15 @@ DEFAULT_WORKLOAD = "mixtral-8x7b-bs16-32k-cpu25"
 # Short runs of the other BASELINE configurations, reported beside the default line (rank 0, one GPU): config 3 at CPU
 # share 0 and 70 %, config 4 (compressed-latent kernel), config 5 at CPU share 0.
 OTHER_CONFIGS = ["qwen3-30b-a3b-bs16-32k-cpu0", "qwen3-30b-a3b-bs16-32k-cpu70", "deepseek-v2-lite-mla-bs8-128k-cpu40",
-                 "qwen3-ragged-bs64-1m-16layers-cpu0"]
+                 "qwen3-ragged-bs64-1m-cpu0"]
 BLOCK, WINDOW = 64, 256
 
-# BASELINE config 5: Qwen3 shape, batch 64, ragged context lengths uniform in [8192, 24576] (about 1M tokens in all),
-# CPU share swept 0 .. 90 %. 16 of the 48 layers are kept (every layer's launch is identical; 48 layers at share 0
-# with per-sequence rings sized for the longest sequence would not fit 180 GB).
+# BASELINE config 5: Qwen3 shape, 48 layers, batch 64, ragged context lengths uniform in [8192, 24576] (about 1M tokens
+# in all), CPU share swept 0 .. 90 %.  Every sequence's part of the resident ring is sized for that sequence
+# (ipkv_config.resident_tokens_by_seq), so the batch holds its 103 GB at share 0 and not the longest sequence's ring 64 times.
 for _pct in range(0, 100, 10):
-    WORKLOADS[f"qwen3-ragged-bs64-1m-16layers-cpu{_pct}"] = dict(
-        shape=synth.Shape("qwen3-16l", "gqa", 16, 32, 4, 128, 128, 128 ** -0.5), batch=64, ctx=24576, share=(_pct, 100),
-        cfg_id=5, lens=synth.ragged_lengths(5, 64, 8192, 24576))
+    WORKLOADS[f"qwen3-ragged-bs64-1m-cpu{_pct}"] = dict(
+        shape=synth.QWEN3, batch=64, ctx=24576, share=(_pct, 100), cfg_id=5, lens=synth.ragged_lengths(5, 64, 8192, 24576))
 WORKLOADS["qwen3-ragged-bs64-1m-2layers-cpu30"] = dict(
     shape=synth.Shape("qwen3-2l", "gqa", 2, 32, 4, 128, 128, 128 ** -0.5), batch=64, ctx=24576, share=(3, 10), cfg_id=5,
     lens=synth.ragged_lengths(5, 64, 8192, 24576))
@@ -134,6 +133,10 @@ def make_cache(wl, device_index, decode_steps):
     p_cap = max(p_cap, max(n - cpu_tokens(n, num0, den0) for n in seq_lens(wl)) + grow)
     kind = binding.MLA if sh.kind == "mla" else binding.GQA
     resident, flags = p_cap, binding.FLAG_NO_HOST_U | binding.FLAG_NO_HOST_P
+    by_seq = None
+    if "lens" in wl and not wl.get("host_copies") and "stream_pct" not in wl:
+        # ragged batch: every sequence's ring holds its own GPU-side share plus the decode steps' growth
+        by_seq = [n - cpu_tokens(n, num0, den0) + grow if num0 < den0 else grow for n in seq_lens(wl)]
     if wl.get("host_copies"):
         flags = 0
     if "stream_pct" in wl:
@@ -151,6 +154,7 @@ def make_cache(wl, device_index, decode_steps):
                               block_tokens=BLOCK, window_tokens=window, chunk_tokens=wl.get("chunk_tokens", 512), n_slots=2,
                               p_initial_tokens_per_seq=p_initial,
                               max_u_tokens_per_seq=longest + grow, max_p_tokens_per_seq=p_cap, resident_tokens_per_seq=resident,
+                              resident_tokens_by_seq=by_seq,
                               softmax_scale=sh.scale, share_num=num0, share_den=den0, device=device_index, flags=flags)
     return binding.Cache(cfg)
 

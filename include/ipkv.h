@@ -116,6 +116,11 @@ typedef struct {
   void* w_dev;         size_t w_bytes;
   void* resident_dev;  size_t resident_bytes;
   void* pp_dev;        size_t pp_bytes;
+  /* Optional ring capacity per sequence: host array [max_seqs] of token counts, read by ipkv_query_sizes and
+     ipkv_create only (it need not outlive them); NULL => resident_tokens_per_seq for every sequence.  Every layer's
+     ring is one run of block slots divided among the sequences in this proportion, so a ragged batch reserves what
+     each sequence needs instead of the longest sequence's ring for all (Sec. 4.1: blocks are the unit of placement). */
+  const int64_t* resident_tokens_by_seq;
 } ipkv_config;
 
 /* out_bytes[0..4] = U, P, W, resident ring, PP slots.  (Table 2 of the paper is these sizes.)

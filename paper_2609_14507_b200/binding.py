@@ -43,6 +43,7 @@ class Config(C.Structure):
         ("u_host", C.c_void_p), ("u_bytes", C.c_size_t), ("p_host_pinned", C.c_void_p), ("p_bytes", C.c_size_t),
         ("w_dev", C.c_void_p), ("w_bytes", C.c_size_t), ("resident_dev", C.c_void_p), ("resident_bytes", C.c_size_t),
         ("pp_dev", C.c_void_p), ("pp_bytes", C.c_size_t),
+        ("resident_tokens_by_seq", C.POINTER(C.c_int64)),
     ]
 
 
@@ -184,7 +185,7 @@ def seq_id_array(seq_ids):
 def make_config(kind, n_layers, max_seqs, n_q_heads, n_kv_heads, dim_qk, dim_v, *, block_tokens=64,
                 window_tokens=256, chunk_tokens=512, n_slots=2, max_u_tokens_per_seq=0, max_p_tokens_per_seq=0,
                 resident_tokens_per_seq=0, softmax_scale=0.0, share_num=0, share_den=1, device=0, flags=0,
-                p_initial_tokens_per_seq=0):
+                p_initial_tokens_per_seq=0, resident_tokens_by_seq=None):
     c = Config()
     c.struct_size = C.sizeof(Config)
     c.kind, c.n_layers, c.max_seqs = kind, n_layers, max_seqs
@@ -195,6 +196,11 @@ def make_config(kind, n_layers, max_seqs, n_q_heads, n_kv_heads, dim_qk, dim_v, 
     c.p_initial_tokens_per_seq = p_initial_tokens_per_seq
     c.softmax_scale = softmax_scale
     c.share_num, c.share_den, c.device, c.flags = share_num, share_den, device, flags
+    if resident_tokens_by_seq is not None:                  # per-sequence ring capacities (read by query_sizes / create only)
+        if len(resident_tokens_by_seq) != max_seqs:
+            raise ValueError("resident_tokens_by_seq needs one entry per sequence")
+        c._ring_keepalive = (C.c_int64 * max_seqs)(*[int(x) for x in resident_tokens_by_seq])
+        c.resident_tokens_by_seq = C.cast(c._ring_keepalive, C.POINTER(C.c_int64))
     return c
 
 

@@ -28,6 +28,7 @@
 #include "cpu_engine.h"
 #include "kernels.h"
 #include "plan.hpp"
+#include "ring.hpp"
 #include "policy.hpp"
 #include "router.hpp"
 
@@ -93,7 +94,7 @@ struct ipkv {
     float scale = 0.f;
     int64_t bb = 0;                 // block bytes
     int64_t u_cap = 0, p_cap = 0;   // blocks per (layer, seq)
-    int64_t ring = 0;               // resident blocks per (layer, seq)
+    RingMap rmap;                   // resident ring: block slots of every sequence inside a layer's ring
     int64_t w_blocks = 0, chunk_blocks = 0;
     size_t sizes[5] = {0, 0, 0, 0, 0};
     char *u_host = nullptr, *p_host = nullptr, *w_dev = nullptr, *res_dev = nullptr, *pp_dev = nullptr;
@@ -190,8 +191,9 @@ struct ipkv {
     }
     int64_t w_off(int seq) const { return int64_t(seq) * w_blocks * bb; }                       // inside a layer
     char* w_layer(int layer) { return w_dev + int64_t(layer) * cfg.max_seqs * w_blocks * bb; }
-    int64_t ring_off(int seq) const { return int64_t(seq) * ring * bb; }                        // inside a layer
-    char* ring_layer(int layer) { return res_dev + int64_t(layer) * cfg.max_seqs * ring * bb; }
+    int64_t ring_of(int seq) const { return rmap.blocks(seq); }                                 // block slots of the sequence
+    int64_t ring_off(int seq) const { return rmap.first_slot(seq) * bb; }                       // inside a layer
+    char* ring_layer(int layer) { return res_dev + int64_t(layer) * rmap.total() * bb; }
     int64_t slot_bytes() const { return int64_t(cfg.max_seqs) * chunk_blocks * bb; }
 };
 
@@ -392,6 +394,9 @@ ipkv_status validate(const ipkv_config* c, std::string* why) {
     if (c->chunk_tokens <= 0 || c->chunk_tokens % c->block_tokens != 0) return bad("chunk_tokens must be a positive multiple of block_tokens");
     if (c->n_slots < 2) return bad("n_slots must be at least 2");
     if (c->max_u_tokens_per_seq < 0 || c->max_p_tokens_per_seq < 0 || c->resident_tokens_per_seq < 0) return bad("negative capacity");
+    if (c->resident_tokens_by_seq)
+        for (int s = 0; s < c->max_seqs; ++s)
+            if (c->resident_tokens_by_seq[s] < 0) return bad("negative capacity in resident_tokens_by_seq");
     if (c->share_den <= 0 || c->share_num < 0 || c->share_num > c->share_den) return bad("share must satisfy 0 <= num <= den, den > 0");
     if (!(c->softmax_scale >= 0.f) || std::isinf(c->softmax_scale)) return bad("softmax_scale must be finite and non-negative");
     if (c->flags & IPKV_FLAG_GROW_P) {
@@ -404,20 +409,20 @@ ipkv_status validate(const ipkv_config* c, std::string* why) {
     return IPKV_OK;
 }
 
-void compute_sizes(const ipkv_config* c, int64_t* bb, int64_t* u_cap, int64_t* p_cap, int64_t* ring, size_t sizes[5]) {
+void compute_sizes(const ipkv_config* c, int64_t* bb, int64_t* u_cap, int64_t* p_cap, RingMap* ring, size_t sizes[5]) {
     const BlockGeom g = make_geom(c->kind, c->n_kv_heads, c->dim_qk, c->dim_v, c->block_tokens);
     *bb = g.block_bytes();
     const int64_t bt = c->block_tokens;
     // +1 block: a run always starts on a block boundary, so an explicit partial eviction can waste one
     *u_cap = (c->max_u_tokens_per_seq + bt - 1) / bt + (c->max_u_tokens_per_seq > 0 ? 1 : 0);
     *p_cap = (c->max_p_tokens_per_seq + bt - 1) / bt + (c->max_p_tokens_per_seq > 0 ? 1 : 0);
-    *ring = (c->resident_tokens_per_seq + bt - 1) / bt;
+    ring->init(c->max_seqs, c->resident_tokens_per_seq, c->resident_tokens_by_seq, bt);
     const int64_t seqs = int64_t(c->n_layers) * c->max_seqs;
     sizes[0] = (c->flags & IPKV_FLAG_NO_HOST_U) ? 0 : size_t(seqs * *u_cap * *bb);
     sizes[1] = (c->flags & IPKV_FLAG_NO_HOST_P) ? 0 : size_t(seqs * *p_cap * *bb);
     if (c->flags & IPKV_FLAG_GROW_P) sizes[1] = size_t(seqs * (c->p_initial_tokens_per_seq / bt) * *bb);   // what create pins
     sizes[2] = size_t(seqs * (c->window_tokens / bt) * *bb);
-    sizes[3] = size_t(seqs * *ring * *bb);
+    sizes[3] = size_t(int64_t(c->n_layers) * ring->total() * *bb);
     sizes[4] = size_t(int64_t(c->n_slots) * c->max_seqs * (c->chunk_tokens / bt) * *bb);
 }
 
@@ -490,7 +495,7 @@ ipkv_status flush_layer(ipkv* h, int layer, const int* seqs_in, int n, cudaStrea
             if (st.router.blocks_used(REGION_U) + nb > h->u_cap) return fail(h, IPKV_ERANGE, "eviction would exceed the capacity of U");
         } else {
             if (st.router.blocks_used(REGION_P) + nb > h->p_cap) return fail(h, IPKV_ERANGE, "eviction would exceed the capacity of P");
-            if (no_p && st.router.blocks_used(REGION_P) + nb > h->ring)
+            if (no_p && st.router.blocks_used(REGION_P) + nb > h->ring_of(seq))
                 return fail(h, IPKV_ERANGE, "eviction would push P blocks out of the resident ring, and no host copy of P exists");
         }
     }
@@ -541,16 +546,18 @@ ipkv_status flush_layer(ipkv* h, int layer, const int* seqs_in, int n, cudaStrea
                 CU(h, cudaMemcpyAsync(snap, src, size_t(n_seq_g * win_bytes), cudaMemcpyDeviceToDevice, s));
                 h->stats.d2d_bytes += uint64_t(n_seq_g * win_bytes);
             }
-            if (h->ring > 0)
+            if (h->rmap.total() > 0)
                 for (size_t k = g.first; k < g.second; ++k) {
                     const Job& j = jobs[k];
+                    const int64_t ring = h->ring_of(j.seq);
+                    if (ring == 0) continue;
                     const char* wsrc = h->w_layer(layer) + h->w_off(j.seq);
                     int64_t j0 = j.r.first_block, j1 = j.r.first_block + j.nb;
-                    if (j1 - j0 > h->ring) { wsrc += (j1 - j0 - h->ring) * h->bb; j0 = j1 - h->ring; }   // only the newest fit
+                    if (j1 - j0 > ring) { wsrc += (j1 - j0 - ring) * h->bb; j0 = j1 - ring; }   // only the newest fit
                     char* base = h->ring_layer(layer) + h->ring_off(j.seq);
                     while (j0 < j1) {
-                        const int64_t pos = j0 % h->ring;
-                        const int64_t cnt = std::min(j1 - j0, h->ring - pos);
+                        const int64_t pos = j0 % ring;
+                        const int64_t cnt = std::min(j1 - j0, ring - pos);
                         spans.src[n_spans] = wsrc; spans.dst[n_spans] = base + pos * h->bb; spans.bytes[n_spans] = cnt * h->bb;
                         h->stats.d2d_bytes += uint64_t(cnt * h->bb);
                         if (++n_spans == kCopySpansPerLaunch) { ipkv_status rc = flush_spans(); if (rc != IPKV_OK) return rc; }
@@ -797,7 +804,8 @@ ipkv_status ipkv_query_sizes(const ipkv_config* cfg, size_t out_bytes[5]) {
     std::string why;
     ipkv_status rc = validate(cfg, &why);
     if (rc != IPKV_OK || !out_bytes) return IPKV_EINVAL;
-    int64_t bb, u_cap, p_cap, ring;
+    int64_t bb, u_cap, p_cap;
+    RingMap ring;
     compute_sizes(cfg, &bb, &u_cap, &p_cap, &ring, out_bytes);
     return IPKV_OK;
 }
@@ -861,7 +869,8 @@ ipkv_status ipkv_create(const ipkv_config* cfg, ipkv_t** out) {
     std::memset(&h->stats, 0, sizeof h->stats);
     h->geom = make_geom(cfg->kind, cfg->n_kv_heads, cfg->dim_qk, cfg->dim_v, cfg->block_tokens);
     h->scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / std::sqrt(float(cfg->dim_qk));
-    compute_sizes(cfg, &h->bb, &h->u_cap, &h->p_cap, &h->ring, h->sizes);
+    compute_sizes(cfg, &h->bb, &h->u_cap, &h->p_cap, &h->rmap, h->sizes);
+    h->cfg.resident_tokens_by_seq = nullptr;        // the capacities were copied: the caller's array need not outlive the call
     h->w_blocks = cfg->window_tokens / cfg->block_tokens;
     h->chunk_blocks = cfg->chunk_tokens / cfg->block_tokens;
 
@@ -975,7 +984,7 @@ ipkv_status ipkv_append_bulk(ipkv_t* h, int32_t layer, int32_t seq, const void* 
     const bool no_u = c.flags & IPKV_FLAG_NO_HOST_U, no_p = c.flags & IPKV_FLAG_NO_HOST_P;
     if (st.router.blocks_for(n_cpu) > h->u_cap) return fail(h, IPKV_ERANGE, "prefill exceeds the capacity of U");
     if (st.router.blocks_for(n_gpu) > h->p_cap) return fail(h, IPKV_ERANGE, "prefill exceeds the capacity of P");
-    if (no_p && st.router.blocks_for(n_gpu) > h->ring) return fail(h, IPKV_ERANGE, "prefill exceeds the resident ring and no host copy of P exists");
+    if (no_p && st.router.blocks_for(n_gpu) > h->ring_of(seq)) return fail(h, IPKV_ERANGE, "prefill exceeds the resident ring and no host copy of P exists");
     DeviceGuard dev_guard(c.device);
     CU(h, dev_guard.error());
     Run placed[2];
@@ -989,15 +998,16 @@ ipkv_status ipkv_append_bulk(ipkv_t* h, int32_t layer, int32_t seq, const void* 
         const bool to_u = r.region == REGION_U;
         if (!to_u) note_p_run(st, r, bt);
         if (to_u && no_u) continue;
-        const int64_t first_resident = to_u ? nb : std::max<int64_t>(0, nb - h->ring);   // relative block index
+        const int64_t ring = h->ring_of(seq);
+        const int64_t first_resident = to_u ? nb : std::max<int64_t>(0, nb - ring);   // relative block index
         int64_t j = 0;
         while (j < nb) {
             const bool resident = !to_u && j >= first_resident;
             int64_t j_end;
             char* dst;
             if (resident) {
-                const int64_t pos = (r.first_block + j) % h->ring;
-                j_end = std::min(nb, j + (h->ring - pos));
+                const int64_t pos = (r.first_block + j) % ring;
+                j_end = std::min(nb, j + (ring - pos));
                 dst = h->ring_layer(layer) + h->ring_off(seq) + pos * h->bb;
             } else {
                 if (!to_u && no_p) { j = first_resident; continue; }
@@ -1148,7 +1158,8 @@ ipkv_status ipkv_attend_gpu(ipkv_t* h, int32_t layer, const int32_t* seq_ids, in
         const int seq = seq_ids[i];
         SeqState& st = h->state(layer, seq);
         const int64_t used = st.router.blocks_used(REGION_P);
-        const int64_t nr = std::max<int64_t>(0, used - h->ring);      // blocks [0, nr) are host-only
+        const int64_t ring = h->ring_of(seq);
+        const int64_t nr = std::max<int64_t>(0, used - ring);      // blocks [0, nr) are host-only
         if (nr > 0 && (c.flags & IPKV_FLAG_NO_HOST_P)) return fail(h, IPKV_EINTERNAL, "host-only P blocks without a host copy");
         max_stream_chunks = std::max(max_stream_chunks, (nr + h->chunk_blocks - 1) / h->chunk_blocks);
         for (const PRun& r : st.p_runs) {
@@ -1156,8 +1167,8 @@ ipkv_status ipkv_attend_gpu(ipkv_t* h, int32_t layer, const int32_t* seq_ids, in
             int64_t j = std::max(r.first_block, nr);
             const int64_t end = r.first_block + nb;
             while (j < end) {
-                const int64_t pos = j % h->ring;
-                const int64_t n = std::min(end - j, h->ring - pos);
+                const int64_t pos = j % ring;
+                const int64_t n = std::min(end - j, ring - pos);
                 const int64_t tok = std::min(r.n_tokens - (j - r.first_block) * bt, n * bt);
                 rows[i].push_back(PlanSeg{0, h->ring_off(seq) + pos * h->bb, tok});
                 j += n;
@@ -1165,7 +1176,7 @@ ipkv_status ipkv_attend_gpu(ipkv_t* h, int32_t layer, const int32_t* seq_ids, in
         }
         if (st.router.window_fill() > 0) rows[i].push_back(PlanSeg{1, h->w_off(seq), st.router.window_fill(), fused_append});
     }
-    const char* bases[kMaxBases] = {h->ring ? h->ring_layer(layer) : nullptr, h->w_layer(layer), h->pp_dev, nullptr};
+    const char* bases[kMaxBases] = {h->rmap.total() ? h->ring_layer(layer) : nullptr, h->w_layer(layer), h->pp_dev, nullptr};
     const float* fold_o = opts ? opts->fold_o_dev : nullptr;
     const float* fold_lse = opts ? opts->fold_lse_dev : nullptr;
     if ((fold_o == nullptr) != (fold_lse == nullptr)) return fail(h, IPKV_EINVAL, "fold_o_dev and fold_lse_dev must be given together");
@@ -1197,7 +1208,7 @@ ipkv_status ipkv_attend_gpu(ipkv_t* h, int32_t layer, const int32_t* seq_ids, in
         if (batched) {
             int64_t hi_all = lo;                                       // blocks some listed sequence still needs from the host
             for (int i = 0; i < n_seq; ++i) {
-                const int64_t nr = std::max<int64_t>(0, h->state(layer, seq_ids[i]).router.blocks_used(REGION_P) - h->ring);
+                const int64_t nr = std::max<int64_t>(0, h->state(layer, seq_ids[i]).router.blocks_used(REGION_P) - h->ring_of(seq_ids[i]));
                 hi_all = std::max(hi_all, std::min(nr, lo + h->chunk_blocks));
             }
             for (int64_t b = lo; b < hi_all; b += h->w_blocks) {
@@ -1214,7 +1225,7 @@ ipkv_status ipkv_attend_gpu(ipkv_t* h, int32_t layer, const int32_t* seq_ids, in
             rows[i].clear();
             const int seq = seq_ids[i];
             SeqState& st = h->state(layer, seq);
-            const int64_t nr = std::max<int64_t>(0, st.router.blocks_used(REGION_P) - h->ring);
+            const int64_t nr = std::max<int64_t>(0, st.router.blocks_used(REGION_P) - h->ring_of(seq));
             const int64_t hi = std::min(nr, lo + h->chunk_blocks);
             if (lo >= hi) continue;
             const int64_t row_base = slot * h->slot_bytes() + int64_t(i) * chunk_bytes;
@@ -1293,7 +1304,8 @@ ipkv_status ipkv_attend_gpu_sparse(ipkv_t* h, int32_t layer, const int32_t* seq_
         if (seq < 0 || seq >= c.max_seqs) return fail(h, IPKV_EINVAL, "sequence id out of range");
         SeqState& st = h->state(layer, seq);
         const int64_t used = st.router.blocks_used(REGION_P);
-        const int64_t nr = std::max<int64_t>(0, used - h->ring);
+        const int64_t ring = h->ring_of(seq);
+        const int64_t nr = std::max<int64_t>(0, used - ring);
         if (row_block_start[i + 1] < row_block_start[i]) return fail(h, IPKV_EINVAL, "bad block lists");
         int64_t prev = -1;
         for (int k = row_block_start[i]; k < row_block_start[i + 1]; ++k) {
@@ -1304,7 +1316,7 @@ ipkv_status ipkv_attend_gpu_sparse(ipkv_t* h, int32_t layer, const int32_t* seq_
             if (tok <= 0) return fail(h, IPKV_EINTERNAL, "selected block holds no tokens");
             if (j < nr) { host_picks.push_back(HostPick{i, j, tok}); continue; }
             // resident: extend the previous segment when this block directly follows it in the ring and that one is full
-            const int64_t off = h->ring_off(seq) + (j % h->ring) * h->bb;
+            const int64_t off = h->ring_off(seq) + (j % ring) * h->bb;
             if (!rows[i].empty() && rows[i].back().base_id == 0 && rows[i].back().n_tokens % bt == 0 &&
                 rows[i].back().off + (rows[i].back().n_tokens / bt) * h->bb == off)
                 rows[i].back().n_tokens += tok;
@@ -1313,7 +1325,7 @@ ipkv_status ipkv_attend_gpu_sparse(ipkv_t* h, int32_t layer, const int32_t* seq_
         }
         if (include_window && st.router.window_fill() > 0) rows[i].push_back(PlanSeg{1, h->w_off(seq), st.router.window_fill()});
     }
-    const char* bases[kMaxBases] = {h->ring ? h->ring_layer(layer) : nullptr, h->w_layer(layer), h->pp_dev, nullptr};
+    const char* bases[kMaxBases] = {h->rmap.total() ? h->ring_layer(layer) : nullptr, h->w_layer(layer), h->pp_dev, nullptr};
     ipkv_status rc = run_group(h, rows, bases, q_dev, kv_splits, fold_o, fold_lse, o_part_dev, lse_part_dev, s, static_schedule);
     if (rc != IPKV_OK) return rc;
     if (host_picks.empty()) return IPKV_OK;
@@ -1451,7 +1463,8 @@ ipkv_status ipkv_views(ipkv_t* h, int32_t layer, int32_t seq, ipkv_extent* out, 
     *n_out = total;
     if (cap < total) return cap == 0 ? IPKV_OK : fail(h, IPKV_ERANGE, "extent array too small");
     const int64_t used_p = st.router.blocks_used(REGION_P);
-    const int64_t nr = std::max<int64_t>(0, used_p - h->ring);
+    const int64_t ring = h->ring_of(seq);
+    const int64_t nr = std::max<int64_t>(0, used_p - ring);
     int k = 0;
     for (const Run& whole : runs) {
         const int64_t whole_nb = (whole.n_tokens + bt - 1) / bt;
@@ -1482,8 +1495,8 @@ ipkv_status ipkv_views(ipkv_t* h, int32_t layer, int32_t seq, ipkv_extent* out, 
                     if (rc != IPKV_OK) return rc;
                     e.host_ptr = host;
                 }
-                if (h->ring > 0 && r.first_block >= nr && (r.first_block % h->ring) + nb <= h->ring)
-                    e.dev_ptr = h->ring_layer(layer) + h->ring_off(seq) + (r.first_block % h->ring) * h->bb;
+                if (ring > 0 && r.first_block >= nr && (r.first_block % ring) + nb <= ring)
+                    e.dev_ptr = h->ring_layer(layer) + h->ring_off(seq) + (r.first_block % ring) * h->bb;
             }
         }
     }
@@ -1514,7 +1527,7 @@ ipkv_status ipkv_counts(ipkv_t* h, int32_t layer, int32_t seq, int64_t counts[6]
     counts[0] = st.router.tokens_in(REGION_U);
     counts[1] = st.router.tokens_in(REGION_P);
     counts[2] = st.router.tokens_in(REGION_W);
-    const int64_t nr = std::max<int64_t>(0, st.router.blocks_used(REGION_P) - h->ring);
+    const int64_t nr = std::max<int64_t>(0, st.router.blocks_used(REGION_P) - h->ring_of(seq));
     int64_t res = 0;
     const int64_t bt = h->cfg.block_tokens;
     for (const PRun& r : st.p_runs) {
@@ -1554,7 +1567,7 @@ ipkv_status ipkv_read_token(ipkv_t* h, int32_t layer, int32_t seq, int64_t token
             if (rc != IPKV_OK) return rc;
             std::memcpy(buf.data(), blk_host, size_t(h->bb));
         } else {
-            CU(h, cudaMemcpy(buf.data(), h->ring_layer(layer) + h->ring_off(seq) + (blk % h->ring) * h->bb, size_t(h->bb), cudaMemcpyDeviceToHost));
+            CU(h, cudaMemcpy(buf.data(), h->ring_layer(layer) + h->ring_off(seq) + (blk % h->ring_of(seq)) * h->bb, size_t(h->bb), cudaMemcpyDeviceToHost));
         }
     } else {
         const int64_t wb = off / bt;

@@ -6,6 +6,7 @@
 #include <vector>
 
 #include "../paper_2609_14507_b200/csrc/plan.hpp"
+#include "../paper_2609_14507_b200/csrc/ring.hpp"
 #include "../paper_2609_14507_b200/csrc/router.hpp"
 
 using namespace ipkvi;
@@ -89,6 +90,25 @@ int shim_describe_status(uint32_t status, char* out, int cap) {
     return int(s.size());
 }
 uint32_t shim_status_bit(int which) { return which == 0 ? kStatusNoFreeStage : which == 1 ? kStatusNoTile : kStatusCopyNotLanded; }
+
+// resident ring: slot of P block j of every sequence, for the newest blocks when `used[s]` P blocks exist.
+// out_slots gets, sequence after sequence, the slots of blocks [first_resident, used); returns how many were written.
+int64_t shim_ring_slots(int n_seqs, int64_t uniform_tokens, const int64_t* tokens_by_seq, int64_t bt, const int64_t* used,
+                        int64_t* out_slots, int64_t cap_out, int64_t* total_out, int64_t* caps_out) {
+    RingMap m;
+    m.init(n_seqs, uniform_tokens, tokens_by_seq, bt);
+    *total_out = m.total();
+    int64_t n = 0;
+    for (int s = 0; s < n_seqs; ++s) {
+        caps_out[s] = m.blocks(s);
+        if (m.blocks(s) == 0) continue;
+        for (int64_t j = m.first_resident(s, used[s]); j < used[s]; ++j) {
+            if (n >= cap_out) return -1;
+            out_slots[n++] = m.slot(s, j);
+        }
+    }
+    return n;
+}
 
 int64_t shim_tile_chunk_offset(int32_t bt, int32_t t, int32_t chunk) { return tile_chunk_offset(bt, t, chunk); }
 int64_t shim_plain_chunk_offset(int32_t d, int32_t t, int32_t chunk) { return plain_chunk_offset(d, t, chunk); }

@@ -934,3 +934,48 @@ def test_closed_loop_two_engines_run_concurrently_and_the_policy_steers_the_shar
             check_contents(cache, 0, s_, r, [0, L0 - 1, L0, L0 + D, L0 + steps - 1])
         assert overlapped > 0                            # the CPU engine was still running when the GPU call had returned
         assert cache.get_stats()["device_status"] == 0
+
+
+def test_ring_capacity_per_sequence():
+    """resident_tokens_by_seq: three sequences whose parts of the resident ring hold nothing, four blocks and everything.
+    Prefill and decode evictions wrap each part at its own size; blocks that fall out of a short part are streamed from
+    the pinned host copy; the GPU-side partial, the routing and the token contents match the oracle for all three."""
+    sh = synth.Shape("tiny", "gqa", 2, 8, 2, 128, 128, 128 ** -0.5)
+    rng = np.random.default_rng(98)
+    scale = float(np.float32(sh.scale))
+    bt, D = 64, 64
+    seqs, lens, caps = [0, 1, 2], [900, 1000, 700], [0, 256, 4096]
+    with make_cache(sh, 2, 3, block_tokens=bt, window_tokens=D, chunk_tokens=128, n_slots=2, max_u_tokens_per_seq=2048,
+                    max_p_tokens_per_seq=2048, resident_tokens_per_seq=64, resident_tokens_by_seq=caps,
+                    share_num=1, share_den=4) as cache:
+        refs = {}
+        for layer in range(2):
+            for s_ in seqs:
+                r = RefSeq(sh, bt, D, 1, 4)
+                k, v = synth.host_kv(sh, lens[s_], seed=9800 + 10 * layer + s_)
+                cache.append_bulk(layer, s_, synth.bits_to_torch(k, DEV), synth.bits_to_torch(v, DEV), lens[s_], 1, 3)
+                r.bulk(k, v, 1, 3)
+                refs[(layer, s_)] = r
+        for step in range(3 * D + 7):
+            for layer in range(2):
+                k = synth.normal_bf16(rng, (3, 2, 128)); v = synth.normal_bf16(rng, (3, 2, 128))
+                cache.append(layer, seqs, synth.bits_to_torch(k, DEV), synth.bits_to_torch(v, DEV))
+                for i, s_ in enumerate(seqs):
+                    refs[(layer, s_)].append(k[i:i + 1], v[i:i + 1])
+            if step % 50 == 0 or step == 3 * D + 6:
+                for layer in range(2):
+                    q = synth.normal_bf16(rng, (3, sh.n_q_heads, 128))
+                    o = torch.zeros((3, sh.n_q_heads, 128), device=DEV); lse = torch.zeros((3, sh.n_q_heads), device=DEV)
+                    cache.attend_gpu(layer, seqs, synth.bits_to_torch(q, DEV), o, lse)
+                    torch.cuda.synchronize()
+                    want = [refs[(layer, s_)].attend(q[i], "gpu", scale) for i, s_ in enumerate(seqs)]
+                    check_partial(o.cpu().numpy(), lse.cpu().numpy(), np.stack([w[0] for w in want]), np.stack([w[1] for w in want]),
+                                  f"per-sequence ring, layer {layer}, step {step}")
+        torch.cuda.synchronize()
+        for (layer, s_), r in refs.items():
+            check_routing(cache, layer, s_, r, sample=range(0, len(r.k), 37))
+            check_contents(cache, layer, s_, r, [0, 300, lens[s_] - 1, lens[s_], len(r.k) - 1])
+        # the sequence without a ring keeps nothing on the device but its window; the one with a large part keeps all of P
+        c0, c2 = cache.counts(0, 0), cache.counts(0, 2)
+        assert c0["n_p_resident"] == 0 and c2["n_p_resident"] == c2["n_p"]
+        assert cache.get_stats()["device_status"] == 0

@@ -114,6 +114,19 @@ def test_ragged_1m_token_batch_fixed_schedule_sampled():
         del bench.WORKLOADS["_ragged60"]
 
 
+@pytest.mark.parametrize("num,den", [(0, 1), (9, 10)])
+def test_ragged_1m_token_batch_at_the_ends_of_the_share_sweep(num, den):
+    """CPU share 0 (the longest launches, dynamically balanced, every sequence's ring at its own size) and 90 % (the
+    shortest, fixed schedule): the two ends of the sweep, where the planner behaves most differently."""
+    wl = dict(bench.WORKLOADS["qwen3-ragged-bs64-1m-2layers-cpu30"], share=(num, den))
+    name = f"_ragged_{num}_{den}"
+    bench.WORKLOADS[name] = wl
+    try:
+        _run_step_and_check(name, [(0, 0), (0, 41), (1, 63), (1, 5)])
+    finally:
+        del bench.WORKLOADS[name]
+
+
 def _with_workload(name, wl, samples):
     bench.WORKLOADS[name] = wl
     try:

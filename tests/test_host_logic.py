@@ -229,3 +229,43 @@ def test_device_status_word_maps_to_the_documented_messages():
     assert "did not land" in text(4)
     assert all(k in text(7) for k in ("free stage", "no tile", "did not land"))
     assert "unknown" in text(8)
+
+
+def test_resident_ring_never_hands_a_slot_out_twice():
+    """Per-sequence ring capacities: the slots of all blocks that are resident at the same time (the newest cap[s] P
+    blocks of every sequence) are distinct and inside the layer's ring, whatever the capacities and fill levels; a
+    uniform capacity is the special case; the sizes the library reports follow the capacities."""
+    import ctypes
+    from paper_2609_14507_b200 import binding
+    L = host_shim.lib()
+    L.shim_ring_slots.restype = ctypes.c_int64
+    vp, i64 = ctypes.c_void_p, ctypes.c_int64
+    L.shim_ring_slots.argtypes = [ctypes.c_int, i64, vp, i64, vp, vp, i64, ctypes.POINTER(i64), vp]
+    rng = np.random.default_rng(51)
+    for trial in range(200):
+        n = int(rng.integers(1, 40))
+        bt = int(rng.choice([16, 32, 64, 128]))
+        by_seq = rng.integers(0, 3000, size=n).astype(np.int64) if trial % 3 else None
+        uniform = int(rng.integers(0, 3000))
+        used = rng.integers(0, 120, size=n).astype(np.int64)
+        out = np.zeros(200000, dtype=np.int64); caps = np.zeros(n, dtype=np.int64); total = ctypes.c_int64()
+        k = L.shim_ring_slots(n, uniform, by_seq.ctypes.data if by_seq is not None else None, bt,
+                              used.ctypes.data, out.ctypes.data, out.size, ctypes.byref(total), caps.ctypes.data)
+        assert k >= 0
+        want_caps = [-(-int(t) // bt) for t in (by_seq if by_seq is not None else [uniform] * n)]
+        assert list(caps) == want_caps and total.value == sum(want_caps)
+        slots = out[:k]
+        assert k == sum(min(int(u), c) for u, c in zip(used, want_caps))
+        assert len(set(slots.tolist())) == k                              # no slot twice
+        assert k == 0 or (slots.min() >= 0 and slots.max() < total.value)
+    # the sizes: every layer's ring is the sum of the sequences' capacities
+    lens = [100, 6400, 0, 777]
+    cfg = binding.make_config(binding.GQA, 3, 4, 32, 4, 128, 128, block_tokens=64, window_tokens=256, chunk_tokens=512,
+                              max_u_tokens_per_seq=64, max_p_tokens_per_seq=8192, resident_tokens_per_seq=8192,
+                              resident_tokens_by_seq=lens, flags=binding.FLAG_NO_HOST_U | binding.FLAG_NO_HOST_P)
+    sizes = binding.ipkv_query_sizes(cfg)
+    assert sizes["resident"] == 3 * sum(-(-x // 64) for x in lens) * 64 * 2048
+    cfg_u = binding.make_config(binding.GQA, 3, 4, 32, 4, 128, 128, block_tokens=64, window_tokens=256, chunk_tokens=512,
+                                max_u_tokens_per_seq=64, max_p_tokens_per_seq=8192, resident_tokens_per_seq=8192,
+                                flags=binding.FLAG_NO_HOST_U | binding.FLAG_NO_HOST_P)
+    assert binding.ipkv_query_sizes(cfg_u)["resident"] == 3 * 4 * 128 * 64 * 2048
