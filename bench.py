@@ -663,7 +663,17 @@ def main():
     out_l = [out[l] for l in range(NL)]; oc_l = [o_cpu[l] for l in range(NL)]; lc_l = [lse_cpu[l] for l in range(NL)]
     apps = [{} if args.separate_append else dict(append_k=k_l[l], append_v=v_l[l]) for l in range(NL)]
 
+    # the fused form of a layer (append riding in the call, CPU partial folded by the reduce) with its arguments marshalled once
+    calls = None
+    if fused and not args.separate_append:
+        calls = [cache.attend_gpu_call(l, seq_ids, q_l[l], out_l[l], out_lse, kv_splits=args.kv_splits, static_schedule=args.static_schedule,
+                                       stream=cur, fold_o=oc_l[l], fold_lse=lc_l[l], **apps[l]) for l in range(NL)]
+
     def step():
+        if calls is not None:
+            for call in calls:
+                call()
+            return
         for layer in range(NL):
             # the append rides in the attention call (the kernel writes the new rows where it can) unless --separate-append
             if args.separate_append:

@@ -281,6 +281,24 @@ class Cache:
         self._check(lib().ipkv_attend_gpu(self._h, layer, ids, n, _ptr(q), C.byref(opts), _ptr(o_part), _ptr(lse_part),
                                           _stream(stream)), "ipkv_attend_gpu")
 
+    def attend_gpu_call(self, layer, seq_ids, q, o_part, lse_part, kv_splits=0, side_stream=None, stream=None,
+                        fold_o=None, fold_lse=None, static_schedule=False, force_balance=False, append_k=None, append_v=None):
+        """The same call as attend_gpu with its arguments marshalled once: returns a function of no arguments that issues
+        ipkv_attend_gpu on the given buffers (for loops that call a layer with the same tensors every step)."""
+        ids, n = _ids(seq_ids)
+        opts = AttendOpts(kv_splits, (ATTEND_STATIC_SCHEDULE if static_schedule else 0) | (ATTEND_BALANCE if force_balance else 0),
+                          _stream(side_stream) if side_stream is not None else None, _ptr(fold_o), _ptr(fold_lse),
+                          _ptr(append_k), _ptr(append_v))
+        fn, check = lib().ipkv_attend_gpu, self._check
+        args = (self._h, layer, ids, n, _ptr(q), C.byref(opts), _ptr(o_part), _ptr(lse_part), _stream(stream))
+        keep = (opts, ids, q, o_part, lse_part, fold_o, fold_lse, append_k, append_v)      # the buffers stay alive with the call
+
+        def call(_keep=keep):
+            rc = fn(*args)
+            if rc != OK:
+                check(rc, "ipkv_attend_gpu")
+        return call
+
     def attend_gpu_sparse(self, layer, seq_ids, q, blocks_per_row, o_part, lse_part, include_window=True, kv_splits=0,
                           stream=None, fold_o=None, fold_lse=None, static_schedule=False):
         """Attention over the D-window plus the listed whole P blocks of every row (block ordinals in region P)."""

@@ -63,6 +63,7 @@ struct GqaParams {
     int bt;
     int64_t head_bytes, block_bytes;
     float scale_log2;
+    int win_tail;       // valid tokens in the last tile of runs flagged kSegTailParam
 };
 
 template <int D, int STAGES>
@@ -132,6 +133,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_gqa_kernel(const GqaParams p
                 if (!waited && it >= STAGES) { ptx::grid_dependency_wait(); waited = true; }
                 if (sp != cached_sp) {                             // first tile of a span: where its run lives
                     seg = p.segs[span.seg];
+                    if (seg.base_id & kSegTailParam) seg.n_tokens += p.win_tail - kTileTokens;
                     seg_base = p.bases[seg.base_id & kSegBaseMask] + seg.off + int64_t(span.gh / p.n_hg) * p.head_bytes;
                     cached_sp = sp;
                 }
@@ -439,6 +441,7 @@ cudaError_t launch_gqa(const AttnLaunch& a, cudaStream_t s) {
     p.next = a.steal_next; p.lists = a.steal_lists; p.n_spans = a.n_spans; p.n_ctas = a.n_ctas; p.cta_tiles = a.cta_tiles;
     p.n_rows = a.n_rows; p.n_gh = a.n_gh;
     p.early = a.early_tiles;
+    p.win_tail = a.win_tail;
     p.Hq = a.n_q_heads; p.G = a.n_q_heads / a.n_kv_heads;
     p.n_hg = (p.G + 15) / 16;
     p.RG = part_geom(0, a.n_q_heads, a.n_kv_heads).rows_per_group;

@@ -65,6 +65,7 @@ struct MlaParams {
     int bt;
     int64_t block_bytes;
     float scale_log2;
+    int win_tail;        // valid tokens in the last tile of runs flagged kSegTailParam
     int early;           // nonzero: the first copies of ring tiles (2: of window tiles too) need not wait for the previous kernel
 };
 
@@ -117,7 +118,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_mla_kernel(const MlaParams p
             bool waited = !early;
             for (int sn = span_begin; sn < span_end && ok; ++sn) {
                 const Span span = p.spans[sn];
-                const Seg seg = p.segs[span.seg];
+                Seg seg = p.segs[span.seg];
+                if (seg.base_id & kSegTailParam) seg.n_tokens += p.win_tail - kTileTokens;
                 const char* seg_base = p.bases[seg.base_id & kSegBaseMask] + seg.off;
                 for (int i = 0; i < span.ntiles; ++i, ++it) {
                     if (!waited && (it >= kStages || (p.early < 2 && (seg.base_id & kSegBaseMask) == kSegBaseWindow))) {
@@ -175,7 +177,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_mla_kernel(const MlaParams p
 
     for (int sn = span_begin; sn < span_end; ++sn) {
         const Span span = p.spans[sn];
-        const Seg seg = p.segs[span.seg];
+        Seg seg = p.segs[span.seg];
+        if (seg.base_id & kSegTailParam) seg.n_tokens += p.win_tail - kTileTokens;
         const int head0 = span.gh * 16;
         const int n_heads = min(16, p.Hq - head0);
 
@@ -352,6 +355,7 @@ cudaError_t launch_attend_mla(const AttnLaunch& a, cudaStream_t s) {
     p.block_bytes = int64_t(a.bt) * kDqk * 2;
     p.scale_log2 = a.scale * kLog2e;
     p.early = a.early_tiles;
+    p.win_tail = a.win_tail;
     const int smem = kSmemTotal + 1024;
     static bool configured[64] = {};
     int dev = 0;

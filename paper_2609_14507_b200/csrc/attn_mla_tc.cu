@@ -73,6 +73,7 @@ struct MlaTcParams {
     int bt;
     int64_t block_bytes;
     float scale_log2;
+    int win_tail;        // valid tokens in the last tile of runs flagged kSegTailParam
 };
 
 // Shared-memory matrix descriptor, 128-byte swizzle. lbo / sbo in bytes.
@@ -162,7 +163,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_mla_tc_kernel(const MlaTcPar
             const uint64_t pol = ptx::l2_evict_first_policy();
             for (int sn = span_begin; sn < span_end && ok; ++sn) {
                 const Span span = p.spans[sn];
-                const Seg seg = p.segs[span.seg];
+                Seg seg = p.segs[span.seg];
+                if (seg.base_id & kSegTailParam) seg.n_tokens += p.win_tail - kTileTokens;
                 const char* seg_base = p.bases[seg.base_id & kSegBaseMask] + seg.off;
                 for (int i = 0; i < span.ntiles; ++i, ++it) {
                     const int st = it & 1;
@@ -263,7 +265,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_mla_tc_kernel(const MlaTcPar
         int span_no = 0;
         for (int sn = span_begin; sn < span_end; ++sn, ++span_no) {
             const Span span = p.spans[sn];
-            const Seg seg = p.segs[span.seg];
+            Seg seg = p.segs[span.seg];
+            if (seg.base_id & kSegTailParam) seg.n_tokens += p.win_tail - kTileTokens;
             const int head0 = span.gh * 16;
             const int n_heads = min(16, p.Hq - head0);
             // query tile -> K-major swizzled operand [9 panels][16 rows][128 B]
@@ -417,6 +420,7 @@ cudaError_t launch_attend_mla_tc(const AttnLaunch& a, cudaStream_t s) {
     p.bt = a.bt;
     p.block_bytes = int64_t(a.bt) * kDqk * 2;
     p.scale_log2 = a.scale * kLog2e;
+    p.win_tail = a.win_tail;
     const int smem = kSmemTotal + 1024;
     static bool configured[64] = {};
     int dev = 0;

@@ -19,6 +19,11 @@ struct Seg {
 // its copy has landed (and into the run itself, for the launches to come), then computes as usual.
 constexpr int32_t kSegAppended = 0x100;
 constexpr int32_t kSegBaseMask = 0xff;
+// The run's token count in the table is rounded up to whole 64-token tiles; the real count is that minus 64 plus the
+// launch parameter win_tail (1..64).  Set on the D-window runs of a launch when all of them end at the same offset inside
+// their last tile, which is the case while a batch decodes in lockstep: the table then stays the same from step to step
+// (only win_tail moves) until a window grows into a new tile or is evicted, and need not be uploaded again.
+constexpr int32_t kSegTailParam = 0x200;
 constexpr int32_t kSegBaseWindow = 1;     // bases[1] is the layer's D-window (bases[0] the resident ring, bases[2] the slots)
 // One span of split-K work: tiles [tile0, tile0 + ntiles) of segment `seg` for query row `row` and head
 // group `gh`.  A CTA processes a contiguous range of spans back to back; the partial(s) a span produces are
@@ -55,6 +60,7 @@ struct AttnLaunch {
     uint32_t* status;               // device word, OR-ed with an error bit if a bounded wait gives up
     const void* append_k;           // fused append: [n_rows][n_kv_heads][dim_qk] bf16 new K rows (null: none)
     const void* append_v;           // [n_rows][n_kv_heads][dim_v]
+    int win_tail;                   // valid tokens in the last tile of the runs flagged kSegTailParam (1..64)
     int plain_launch;               // 1: the tables were written by the kernel right in front of this launch: no launch overlap
     int early_tiles;                // nonzero: no ring byte this launch reads (2: no window byte either) was written by the kernel
                                     // before it in the stream, so the first copies of such tiles may be issued before that

@@ -44,7 +44,7 @@ inline std::string describe_device_status(uint32_t status) {
     return where;
 }
 
-struct PlanSeg { int base_id; int64_t off; int64_t n_tokens; bool appended = false; };
+struct PlanSeg { int base_id; int64_t off; int64_t n_tokens; bool appended = false; bool tail_param = false; };
 
 struct Plan {
     std::vector<Seg> segs;
@@ -101,7 +101,8 @@ inline void build_plan(const std::vector<std::vector<PlanSeg>>& rows, int n_gh, 
         for (const auto& s : rows[r]) {
             if (s.n_tokens <= 0) continue;
             row_segs[r].push_back(int32_t(plan->segs.size()));
-            plan->segs.push_back(Seg{s.off, int32_t(s.n_tokens), s.base_id | (s.appended ? kSegAppended : 0)});
+            const int64_t n_table = s.tail_param ? (s.n_tokens + kTileTokens - 1) / kTileTokens * kTileTokens : s.n_tokens;
+            plan->segs.push_back(Seg{s.off, int32_t(n_table), s.base_id | (s.appended ? kSegAppended : 0) | (s.tail_param ? kSegTailParam : 0)});
             rt += (s.n_tokens + kTileTokens - 1) / kTileTokens;
             total_tokens += s.n_tokens;
         }

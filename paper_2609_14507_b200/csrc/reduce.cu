@@ -15,7 +15,6 @@ namespace ipkvi {
 namespace {
 
 constexpr int kWarpsPerBlock = 4;
-constexpr int kReduceThreads = 256;
 constexpr int kPrefetch = 2;       // partial outputs per thread requested up front (of the own and of the extra partials)
 constexpr int kLseCache = 512;     // LSE values kept in shared memory between the two passes
 
@@ -44,8 +43,12 @@ struct ReduceParams {
 
 // EXTRAS: the launch was dynamically balanced and may have extra partials (kept out of the plain instantiation, which
 // then needs few enough registers for five CTAs per SM: launches with thousands of (row, head) pairs run in fewer waves).
-template <bool EXTRAS>
-__global__ void __launch_bounds__(kReduceThreads, EXTRAS ? 4 : 5) split_reduce_kernel(const ReduceParams p) {
+// THREADS: 256, or 128 for launches with so many (row, head) pairs that 256-thread CTAs would need several waves (a
+// ragged batch of 64 sequences x 32 heads: 2048 CTAs, at five per SM 2.8 waves, measured 10.4 us; with 128 threads all
+// of them are resident at once).
+template <bool EXTRAS, int THREADS>
+__global__ void __launch_bounds__(THREADS, THREADS == 256 ? (EXTRAS ? 4 : 5) : 10) split_reduce_kernel(const ReduceParams p) {
+    constexpr int kReduceThreads = THREADS;
     extern __shared__ float4 red[];                 // [SL][CG]
     __shared__ float s_warp[kReduceThreads / 32];
     __shared__ float s_w[kLseCache];               // LSE of the first entries
@@ -237,12 +240,19 @@ cudaError_t launch_split_reduce(const AttnLaunch& a, cudaStream_t s) {
     p.n_gh = pg.n_gh; p.RG = pg.rows_per_group; p.NW = pg.parts_per_span;
     p.dvl = a.dim_v > 128 && a.dim_v % 128 == 0 ? 128 : a.dim_v;
     p.CS = a.dim_v / p.dvl;
-    if (p.dvl % 4 != 0 || p.dvl / 4 > kReduceThreads || kReduceThreads % (p.dvl / 4) != 0) return cudaErrorInvalidValue;
+    if (p.dvl % 4 != 0 || p.dvl / 4 > 128 || 128 % (p.dvl / 4) != 0) return cudaErrorInvalidValue;
     p.extra_count = a.steal_lists; p.extra_list = a.steal_lists ? a.steal_lists + a.n_rows * a.n_gh : nullptr; p.n_spans = a.n_spans;
     p.clear = a.steal_clear; p.clear_words = a.steal_clear ? a.steal_clear_words : 0;
-    const size_t smem = size_t(kReduceThreads) * sizeof(float4);
-    if (p.extra_count) return launch_ordered(!a.plain_launch, split_reduce_kernel<true>, total * p.CS, kReduceThreads, smem, s, p);
-    return launch_ordered(!a.plain_launch, split_reduce_kernel<false>, total * p.CS, kReduceThreads, smem, s, p);
+    // one wave of 256-thread CTAs holds 148 x 5 of them; beyond that, and when a slab leaves at least two entry slices, halve the CTAs
+    const bool narrow = int64_t(total) * p.CS > 148 * 5 && p.dvl <= 256;
+    const int threads = narrow ? 128 : 256;
+    const size_t smem = size_t(threads) * sizeof(float4);
+    if (p.extra_count) {
+        if (narrow) return launch_ordered(!a.plain_launch, split_reduce_kernel<true, 128>, total * p.CS, threads, smem, s, p);
+        return launch_ordered(!a.plain_launch, split_reduce_kernel<true, 256>, total * p.CS, threads, smem, s, p);
+    }
+    if (narrow) return launch_ordered(!a.plain_launch, split_reduce_kernel<false, 128>, total * p.CS, threads, smem, s, p);
+    return launch_ordered(!a.plain_launch, split_reduce_kernel<false, 256>, total * p.CS, threads, smem, s, p);
 }
 
 cudaError_t launch_merge(const MergeLaunch& m, cudaStream_t s) {
@@ -253,3 +263,4 @@ cudaError_t launch_merge(const MergeLaunch& m, cudaStream_t s) {
 }
 
 }  // namespace ipkvi
+
