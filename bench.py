@@ -309,6 +309,23 @@ def other_config(name, steps=10, warmup=3):
             "sm_mhz": (d.get("clocks") or {}).get("sm_mhz"), "layers": d["config"]["layers"]}
 
 
+def replica_envs(n, port, base_env=None):
+    """Environment of each of n replica processes on this node (one per GPU): what a launcher would have set."""
+    base = dict(os.environ if base_env is None else base_env)
+    return [dict(base, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+            for r in range(n)]
+
+
+def spawn_replicas(n, argv):
+    """`bench.py --gpus N` without a launcher: start the N replica processes here (rank 0 prints the JSON line) and wait."""
+    import socket
+    s = socket.socket(); s.bind(("127.0.0.1", 0)); port = s.getsockname()[1]; s.close()
+    procs = [subprocess.Popen([sys.executable, os.path.join(ROOT, "bench.py")] + argv, env=env, cwd=ROOT)
+             for env in replica_envs(n, port)]
+    codes = [p.wait() for p in procs]
+    return max(codes, key=abs) if any(codes) else 0
+
+
 def run_reference(args, wl, name):
     """--impl reference: the oracle on the host cores, on the same workload and metric; each step is a bounded sample."""
     rank = int(os.environ.get("RANK", "0"))
@@ -608,6 +625,9 @@ def main():
                     help="default workload only: skip the short runs of the other BASELINE configurations (other_configs in the line)")
     args = ap.parse_args()
     wl = WORKLOADS[args.workload]
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # no launcher: this process starts the replicas itself (one process per GPU, replicas only) and waits for them
+        sys.exit(spawn_replicas(args.gpus, sys.argv[1:]))
     if args.impl == "reference":
         run_reference(args, wl, args.workload)
         return

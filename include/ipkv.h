@@ -295,6 +295,12 @@ ipkv_status ipkv_get_stats(ipkv_t* h, ipkv_stats* out);
  * IPKV_OK.  The attention kernels' own waits use the same routine with a limit of two seconds. */
 ipkv_status ipkv_selftest_expire_wait(ipkv_t* h, uint32_t limit_us, void* stream);
 
+/* Self-test of the host-side failure path (no counterpart in the paper): the next attention launch of this handle is
+ * refused on the host before anything reaches the GPU and its call returns IPKV_ECUDA.  If that call carried a fused
+ * append, the routing state already counts the new tokens; the library then writes their rows with its append kernel,
+ * so the windows hold what the routing says and the next calls see every token. */
+ipkv_status ipkv_selftest_fail_next_launch(ipkv_t* h);
+
 /* ---- roofline share policy (host only; Sec. 5.2-5.3) ------------------------------------------------
  * Eq. 1: T_CPU(r) = r*A*L + C_cpu, T_GPU(r) = (1-r)*B*L + C_gpu, T = max(T_CPU, T_GPU) + T_merge.
  * Eq. 2: r(L) = clamp01(B/(A+B) + (C_gpu - C_cpu)/((A+B)*L)); marginal share p = B/(A+B).

@@ -27,7 +27,7 @@ EXPORTS = [
     "ipkv_attend_runs_noalloc", "ipkv_noalloc_scratch_limit", "ipkv_roofline_share", "ipkv_roofline_step_time",
     "ipkv_policy_create", "ipkv_policy_destroy", "ipkv_policy_observe", "ipkv_policy_update", "ipkv_policy_prefill_share",
     "ipkv_block_bytes", "ipkv_status_str", "ipkv_last_error", "ipkv_version", "ipkv_probe_read_bandwidth",
-    "ipkv_selftest_expire_wait",
+    "ipkv_selftest_expire_wait", "ipkv_selftest_fail_next_launch",
 ]
 
 
@@ -117,6 +117,7 @@ def lib():
         "ipkv_read_token": [vp, i32, i32, i64, vp, vp],
         "ipkv_get_stats": [vp, C.POINTER(Stats)],
         "ipkv_selftest_expire_wait": [vp, C.c_uint32, vp],
+        "ipkv_selftest_fail_next_launch": [vp],
         "ipkv_profile_enable": [vp, i32],
         "ipkv_profile_read": [vp, C.POINTER(C.c_double), C.POINTER(i64), C.POINTER(i64)],
         "ipkv_attend_scratch_bytes": [C.POINTER(AttnShape), i32, i32, i64, i32, C.POINTER(C.c_size_t)],
@@ -363,6 +364,9 @@ class Cache:
         s = Stats()
         self._check(lib().ipkv_get_stats(self._h, C.byref(s)), "ipkv_get_stats")
         return {n: getattr(s, n) for n, _ in Stats._fields_}
+
+    def selftest_fail_next_launch(self):
+        self._check(lib().ipkv_selftest_fail_next_launch(self._h), "ipkv_selftest_fail_next_launch")
 
     def selftest_expire_wait(self, limit_us, stream=None):
         self._check(lib().ipkv_selftest_expire_wait(self._h, limit_us, _stream(stream)), "ipkv_selftest_expire_wait")

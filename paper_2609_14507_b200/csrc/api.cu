@@ -138,6 +138,7 @@ struct ipkv {
     uint32_t* status_dev = nullptr;
     // scheduling words of the dynamically balanced attention kernel: two sets used by alternate launches; the
     // split reduce of one launch zeroes the set of the next
+    bool fail_next_launch = false;                   // self-test: the next attention launch is refused on the host
     int32_t* steal_dev = nullptr;
     static constexpr int kStealWords = 1 << 16;     // per set
     int steal_dirty[2] = {0, 0};                     // words a launch has written in each set
@@ -724,6 +725,10 @@ ipkv_status run_group(ipkv* h, std::vector<std::vector<PlanSeg>>& rows, const ch
                       cudaStream_t s, int schedule_flags = 0, const void* append_k = nullptr, const void* append_v = nullptr,
                       int layer = -1, bool device_resident_only = false) {
     const ipkv_config& c = h->cfg;
+    if (h->fail_next_launch) {
+        h->fail_next_launch = false;
+        return fail(h, IPKV_ECUDA, "attention launch refused (ipkv_selftest_fail_next_launch)");
+    }
     Plan plan;
     const PartGeom pg = part_geom(c.kind, c.n_q_heads, c.n_kv_heads);
     const int win_tail = window_tail(rows);
@@ -1129,6 +1134,28 @@ ipkv_status append_tokens(ipkv* h, int32_t layer, const int32_t* seq_ids, int32_
     return IPKV_OK;
 }
 
+// The rows of tokens that append_tokens has already staged (defer_copy) go into their window slots with the append
+// kernel after all: used when the attention launch that was to write them did not happen.
+ipkv_status write_staged_rows(ipkv* h, int32_t layer, const int32_t* seq_ids, int32_t n_seq, const void* k_dev, const void* v_dev,
+                              cudaStream_t s) {
+    const ipkv_config& c = h->cfg;
+    const int64_t k_row = int64_t(c.n_kv_heads) * c.dim_qk * 2, v_row = int64_t(c.n_kv_heads) * c.dim_v * 2;
+    for (int base = 0; base < n_seq; base += kAppendRowsPerLaunch) {
+        const int n = std::min(kAppendRowsPerLaunch, n_seq - base);
+        AppendRows rows;
+        for (int i = 0; i < n; ++i) {
+            rows.dst_off[i] = h->w_off(seq_ids[base + i]);
+            rows.slot[i] = int32_t(h->state(layer, seq_ids[base + i]).router.window_fill() - 1);
+        }
+        note_kv_write(h, layer, false, true);
+        const char* ks = static_cast<const char*>(k_dev) + base * k_row;
+        const char* vs = v_dev ? static_cast<const char*>(v_dev) + base * v_row : nullptr;
+        CU(h, launch_append(h->geom, ks, vs, c.dim_v, h->w_layer(layer), rows, n, s));
+        h->stats.append_kernels += 1;
+    }
+    return IPKV_OK;
+}
+
 }  // namespace
 
 ipkv_status ipkv_append(ipkv_t* h, int32_t layer, const int32_t* seq_ids, int32_t n_seq,
@@ -1158,6 +1185,10 @@ ipkv_status ipkv_attend_gpu(ipkv_t* h, int32_t layer, const int32_t* seq_ids, in
     CU(h, dev_guard.error());
     h->stats.attend_calls += 1;
     const int64_t bt = c.block_tokens;
+
+    const float* fold_o = opts ? opts->fold_o_dev : nullptr;
+    const float* fold_lse = opts ? opts->fold_lse_dev : nullptr;
+    if ((fold_o == nullptr) != (fold_lse == nullptr)) return fail(h, IPKV_EINVAL, "fold_o_dev and fold_lse_dev must be given together");
 
     // append first, if asked to: routing now; the rows themselves are written by the attention kernel where it can
     // (grouped-query kernel, blocks of at least one tile), by the append kernel otherwise
@@ -1197,12 +1228,18 @@ ipkv_status ipkv_attend_gpu(ipkv_t* h, int32_t layer, const int32_t* seq_ids, in
         if (st.router.window_fill() > 0) rows[i].push_back(PlanSeg{1, h->w_off(seq), st.router.window_fill(), fused_append});
     }
     const char* bases[kMaxBases] = {h->rmap.total() ? h->ring_layer(layer) : nullptr, h->w_layer(layer), h->pp_dev, nullptr};
-    const float* fold_o = opts ? opts->fold_o_dev : nullptr;
-    const float* fold_lse = opts ? opts->fold_lse_dev : nullptr;
-    if ((fold_o == nullptr) != (fold_lse == nullptr)) return fail(h, IPKV_EINVAL, "fold_o_dev and fold_lse_dev must be given together");
     ipkv_status rc = run_group(h, rows, bases, q_dev, kv_splits, fold_o, fold_lse, o_part_dev, lse_part_dev, s, static_schedule,
                                fused_append ? app_k : nullptr, fused_append ? app_v : nullptr, layer, true);
-    if (rc != IPKV_OK) return rc;
+    if (rc != IPKV_OK) {
+        // The routing state already counts the new tokens.  If the launch that was to write their rows did not happen, the
+        // append kernel writes them, so that the windows hold what the routing says they hold; the attention itself failed.
+        if (fused_append) {
+            const std::string why = h->err;
+            write_staged_rows(h, layer, seq_ids, n_seq, app_k, app_v, s);
+            h->err = why;
+        }
+        return rc;
+    }
     if (max_stream_chunks == 0) return IPKV_OK;
 
     // groups 1..: host-only P chunks, streamed through the PP slots in overwrite-reuse order (Sec. 4.2)
@@ -1640,6 +1677,12 @@ ipkv_status ipkv_selftest_expire_wait(ipkv_t* h, uint32_t limit_us, void* stream
     DeviceGuard dev_guard(h->cfg.device);
     CU(h, dev_guard.error());
     CU(h, launch_expire_wait(h->status_dev, uint64_t(limit_us) * 1000ull, static_cast<cudaStream_t>(stream)));
+    return IPKV_OK;
+}
+
+ipkv_status ipkv_selftest_fail_next_launch(ipkv_t* h) {
+    if (!h) return IPKV_EINVAL;
+    h->fail_next_launch = true;
     return IPKV_OK;
 }
 

@@ -66,3 +66,20 @@ def test_single_rank_reduction_is_identity():
     sys.path.insert(0, ROOT)
     import bench
     assert bench.reduce_over_ranks(3.5, "max", "cpu") == 3.5 and bench.reduce_over_ranks(7, "sum", "cpu") == 7.0
+
+
+def test_gpus_flag_without_a_launcher_starts_one_replica_per_gpu():
+    """`bench.py --gpus N` with no WORLD_SIZE in the environment spawns the N replicas itself: every rank gets its own
+    RANK / LOCAL_RANK, the common WORLD_SIZE and a loopback rendezvous; checked here on the environments and, end to
+    end, on the reference arm (rank 0 prints the line, rank 1 stays quiet), which needs no GPU."""
+    sys.path.insert(0, ROOT)
+    import bench
+    envs = bench.replica_envs(3, 29999, base_env={"PATH": "/bin"})
+    assert [e["RANK"] for e in envs] == ["0", "1", "2"] and [e["LOCAL_RANK"] for e in envs] == ["0", "1", "2"]
+    assert all(e["WORLD_SIZE"] == "3" and e["MASTER_ADDR"] == "127.0.0.1" and e["MASTER_PORT"] == "29999" and e["PATH"] == "/bin" for e in envs)
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "small-gqa-bs1-4k-cpu50",
+                        "--steps", "1", "--warmup", "0", "--gpus", "2"], env=env, cwd=ROOT, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [l for l in r.stdout.splitlines() if l.strip()]
+    assert len(lines) == 1 and json.loads(lines[0])["n_gpus"] == 2

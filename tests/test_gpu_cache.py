@@ -979,3 +979,39 @@ def test_ring_capacity_per_sequence():
         c0, c2 = cache.counts(0, 0), cache.counts(0, 2)
         assert c0["n_p_resident"] == 0 and c2["n_p_resident"] == c2["n_p"]
         assert cache.get_stats()["device_status"] == 0
+
+
+def test_failed_launch_behind_a_fused_append_leaves_the_window_consistent():
+    """A host-side failure injected between the routing of a fused append and the attention launch that was to write
+    its rows: the call fails, but the token is in its window slot (written by the append kernel instead), and the next
+    step attends every token, the one of the failed call included."""
+    sh = synth.SMALL_GQA
+    L = 500
+    rng = np.random.default_rng(99)
+    k, v = synth.host_kv(sh, L, seed=991)
+    with make_cache(sh, 1, 1, block_tokens=64, window_tokens=256, chunk_tokens=512, max_u_tokens_per_seq=1024,
+                    max_p_tokens_per_seq=1024, resident_tokens_per_seq=1024) as cache:
+        ref = RefSeq(sh, 64, 256, 0, 1)
+        cache.append_bulk(0, 0, synth.bits_to_torch(k, DEV), synth.bits_to_torch(v, DEV), L, 1, 4)
+        ref.bulk(k, v, 1, 4)
+        o = torch.zeros((1, sh.n_q_heads, sh.dim_v), device=DEV); lse = torch.zeros((1, sh.n_q_heads), device=DEV)
+        for step in range(3):
+            kn = synth.normal_bf16(rng, (1, sh.n_kv_heads, sh.dim_qk)); vn = synth.normal_bf16(rng, (1, sh.n_kv_heads, sh.dim_v))
+            q = synth.normal_bf16(rng, (1, sh.n_q_heads, sh.dim_qk))
+            if step == 1:
+                cache.selftest_fail_next_launch()
+                with pytest.raises(binding.IpkvError) as err:
+                    cache.attend_gpu(0, [0], synth.bits_to_torch(q, DEV), o, lse, append_k=synth.bits_to_torch(kn, DEV),
+                                     append_v=synth.bits_to_torch(vn, DEV))
+                assert err.value.status == 5                   # IPKV_ECUDA, from the host
+            else:
+                cache.attend_gpu(0, [0], synth.bits_to_torch(q, DEV), o, lse, append_k=synth.bits_to_torch(kn, DEV),
+                                 append_v=synth.bits_to_torch(vn, DEV))
+            ref.append(kn, vn)                                 # routed in every case
+            torch.cuda.synchronize()
+            check_routing(cache, 0, 0, ref)
+            check_contents(cache, 0, 0, ref, [L - 1, L + step])
+            if step != 1:
+                want = ref.attend(q[0], "gpu", float(np.float32(sh.scale)))
+                check_partial(o.cpu().numpy()[0], lse.cpu().numpy()[0], want[0], want[1], f"step {step}")
+        assert cache.get_stats()["device_status"] == 0
