@@ -280,7 +280,8 @@ typedef struct {
   uint64_t p_segments, p_pinned_bytes, p_pin_us, p_grow_waits, p_grow_wait_us;
   uint64_t p_register_us, p_register_calls, p_register_max_us;  /* the page-locking calls alone: total, count, longest */
   uint32_t device_status;       /* nonzero after a kernel's bounded wait gave up (synchronises): bit 0 a producer
-                                   got no free stage, bit 1 a consumer got no tile, bit 2 a copy did not land  */
+                                   got no free stage, bit 1 a consumer got no tile, bit 2 a copy did not land;
+                                   bit 3 (bounds-checked build) a computed address left its region             */
 } ipkv_stats;
 /* Synchronises the device and fills *out.  If a bounded wait inside one of the handle's kernels gave up since the last
  * call, *out is still filled (device_status says which wait), the call returns IPKV_ETIMEOUT (the results of the
@@ -300,6 +301,15 @@ ipkv_status ipkv_selftest_expire_wait(ipkv_t* h, uint32_t limit_us, void* stream
  * append, the routing state already counts the new tokens; the library then writes their rows with its append kernel,
  * so the windows hold what the routing says and the next calls see every token. */
 ipkv_status ipkv_selftest_fail_next_launch(ipkv_t* h);
+
+/* Bounds-checked build (libipkv_checked.so, compiled with -DIPKV_CHECKED; ipkv_version() says so): every source address
+ * the attention kernels compute for a copy, every partial row they store and every window slot the append paths write is
+ * compared with the extent of its region.  A violation is recorded (device_status bit 3), the access is not made (a read
+ * is redirected to the region's first bytes, a write is dropped), and the next ipkv_get_stats returns IPKV_EINTERNAL.
+ * This self-test call (no counterpart in the paper) declares region base_id of the handle (0 resident ring of a layer,
+ * 1 D-windows of a layer, 2 PP slots) to be only `bytes` long (0 restores the real extent): launches that reach
+ * beyond then trip the check while touching nothing but valid memory.  IPKV_ESTATE in the ordinary build. */
+ipkv_status ipkv_selftest_declare_bounds(ipkv_t* h, int32_t base_id, int64_t bytes);
 
 /* ---- roofline share policy (host only; Sec. 5.2-5.3) ------------------------------------------------
  * Eq. 1: T_CPU(r) = r*A*L + C_cpu, T_GPU(r) = (1-r)*B*L + C_gpu, T = max(T_CPU, T_GPU) + T_merge.

@@ -27,7 +27,7 @@ EXPORTS = [
     "ipkv_attend_runs_noalloc", "ipkv_noalloc_scratch_limit", "ipkv_roofline_share", "ipkv_roofline_step_time",
     "ipkv_policy_create", "ipkv_policy_destroy", "ipkv_policy_observe", "ipkv_policy_update", "ipkv_policy_prefill_share",
     "ipkv_block_bytes", "ipkv_status_str", "ipkv_last_error", "ipkv_version", "ipkv_probe_read_bandwidth",
-    "ipkv_selftest_expire_wait", "ipkv_selftest_fail_next_launch",
+    "ipkv_selftest_expire_wait", "ipkv_selftest_fail_next_launch", "ipkv_selftest_declare_bounds",
 ]
 
 
@@ -88,10 +88,13 @@ _lib = None
 
 
 def lib():
-    """Load ``libipkv.so`` (built by ``paper_2609_14507_b200.build``); raises if it is absent."""
-    global _lib
+    """Load ``libipkv.so`` (built by ``paper_2609_14507_b200.build``); raises if it is absent.  With IPKV_LIB_VARIANT=checked
+    in the environment the bounds-checked build ``libipkv_checked.so`` is loaded instead (same ABI)."""
+    global _lib, LIB_PATH
     if _lib is not None:
         return _lib
+    if os.environ.get("IPKV_LIB_VARIANT") == "checked":
+        LIB_PATH = os.path.join(os.path.dirname(LIB_PATH), "libipkv_checked.so")
     if not os.path.exists(LIB_PATH):
         raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2609_14507_b200.build` "
                            "(there is no fallback path)")
@@ -118,6 +121,7 @@ def lib():
         "ipkv_get_stats": [vp, C.POINTER(Stats)],
         "ipkv_selftest_expire_wait": [vp, C.c_uint32, vp],
         "ipkv_selftest_fail_next_launch": [vp],
+        "ipkv_selftest_declare_bounds": [vp, i32, i64],
         "ipkv_profile_enable": [vp, i32],
         "ipkv_profile_read": [vp, C.POINTER(C.c_double), C.POINTER(i64), C.POINTER(i64)],
         "ipkv_attend_scratch_bytes": [C.POINTER(AttnShape), i32, i32, i64, i32, C.POINTER(C.c_size_t)],
@@ -125,6 +129,8 @@ def lib():
         "ipkv_pack_blocks": [C.POINTER(AttnShape), i32, vp, vp, i64, vp, vp],
         "ipkv_attend_runs_noalloc": [C.POINTER(AttnShape), i32, C.POINTER(Run), C.POINTER(i32), vp, i32, vp, vp, vp, vp],
     }
+    L.ipkv_version.restype = C.c_char_p
+    L.ipkv_version_bytes = lambda: L.ipkv_version()
     for name, args in sig.items():
         f = getattr(L, name)
         f.argtypes = args
@@ -364,6 +370,9 @@ class Cache:
         s = Stats()
         self._check(lib().ipkv_get_stats(self._h, C.byref(s)), "ipkv_get_stats")
         return {n: getattr(s, n) for n, _ in Stats._fields_}
+
+    def selftest_declare_bounds(self, base_id, nbytes):
+        self._check(lib().ipkv_selftest_declare_bounds(self._h, base_id, nbytes), "ipkv_selftest_declare_bounds")
 
     def selftest_fail_next_launch(self):
         self._check(lib().ipkv_selftest_fail_next_launch(self._h), "ipkv_selftest_fail_next_launch")

@@ -11,6 +11,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libipkv.so")
+LIB_CHECKED = os.path.join(HERE, "libipkv_checked.so")       # the same sources with -DIPKV_CHECKED: bounds-checked kernels
 OBJ_DIR = os.path.join(HERE, "build")
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-std=c++17", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
@@ -42,7 +43,10 @@ def cpu_engine_commands(obj_dir):
     return out
 
 
-def build(force=False, verbose=False):
+def build(force=False, verbose=False, checked=False):
+    """Build libipkv.so, or with checked=True libipkv_checked.so (every kernel compiled with -DIPKV_CHECKED)."""
+    LIB = LIB_CHECKED if checked else globals()["LIB"]
+    OBJ_DIR = globals()["OBJ_DIR"] + ("_checked" if checked else "")
     if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _deps_mtime():
         return LIB
     os.makedirs(OBJ_DIR, exist_ok=True)
@@ -50,7 +54,8 @@ def build(force=False, verbose=False):
     procs = []
     for src in sorted(glob.glob(os.path.join(CSRC, "*.cu"))):
         obj = os.path.join(OBJ_DIR, os.path.basename(src)[:-3] + ".o")
-        cmd = [NVCC] + FLAGS + os.environ.get("IPKV_EXTRA_NVCC", "").split() + (["-Xptxas", "-v"] if verbose else []) + ["-c", src, "-o", obj]
+        cmd = ([NVCC] + FLAGS + (["-DIPKV_CHECKED"] if checked else []) + os.environ.get("IPKV_EXTRA_NVCC", "").split() +
+               (["-Xptxas", "-v"] if verbose else []) + ["-c", src, "-o", obj])
         procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
         objs.append(obj)
     for cmd, obj in cpu_engine_commands(OBJ_DIR):                       # host-only parts (the CPU-side engine)
@@ -72,3 +77,4 @@ def build(force=False, verbose=False):
 
 if __name__ == "__main__":
     print(build(force=True, verbose="-v" in sys.argv))
+    print(build(force=True, checked=True))

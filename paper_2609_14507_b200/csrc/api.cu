@@ -192,6 +192,16 @@ struct ipkv {
     }
     int64_t w_off(int seq) const { return int64_t(seq) * w_blocks * bb; }                       // inside a layer
     char* w_layer(int layer) { return w_dev + int64_t(layer) * cfg.max_seqs * w_blocks * bb; }
+    // extent of the memory behind base `id` of a launch (0 ring of one layer, 1 D-windows of one layer, 2 PP slots), for the
+    // bounds-checked build; a self-test may declare one of them smaller than it is (selftest_bounds)
+    int64_t selftest_bounds[kMaxBases] = {0, 0, 0, 0};
+    int64_t region_bytes(int id) const {
+        if (id >= 0 && id < kMaxBases && selftest_bounds[id] > 0) return selftest_bounds[id];
+        if (id == 0) return rmap.total() * bb;
+        if (id == kSegBaseWindow) return int64_t(cfg.max_seqs) * w_blocks * bb;
+        if (id == 2) return int64_t(sizes[4]);
+        return 0;
+    }
     int64_t ring_of(int seq) const { return rmap.blocks(seq); }                                 // block slots of the sequence
     int64_t ring_off(int seq) const { return rmap.first_slot(seq) * bb; }                       // inside a layer
     char* ring_layer(int layer) { return res_dev + int64_t(layer) * rmap.total() * bb; }
@@ -697,6 +707,7 @@ void fill_launch(AttnLaunch* a, int kind, int Hq, int Hkv, int dqk, int dv, int 
     a->n_rows = n_rows;
     a->n_gh = pg.n_gh;
     const size_t rows = (plan.spans.size() + extra_partials) * size_t(pg.parts_per_span) * pg.rows_per_group;
+    a->part_rows = int64_t(rows);
     a->part_o = reinterpret_cast<float*>(partials);
     a->part_lse = reinterpret_cast<float*>(partials + align_up(rows * dv * sizeof(float), 256));
 }
@@ -763,7 +774,7 @@ ipkv_status run_group(ipkv* h, std::vector<std::vector<PlanSeg>>& rows, const ch
         h->steal_dirty[other] = 0;
         h->steal_epoch += 1;
     }
-    for (int i = 0; i < kMaxBases; ++i) a.bases[i] = bases[i];
+    for (int i = 0; i < kMaxBases; ++i) { a.bases[i] = bases[i]; a.base_bytes[i] = bases[i] ? h->region_bytes(i) : 0; }
     a.acc_o = fold_o;
     a.acc_lse = fold_lse;
     a.out_o = out_o; a.out_lse = out_lse;
@@ -807,7 +818,7 @@ ipkv_status run_group(ipkv* h, std::vector<std::vector<PlanSeg>>& rows, const ch
 // ---- C ABI --------------------------------------------------------------------------------------
 extern "C" {
 
-const char* ipkv_version(void) { return "ipkv 0.1 (sm_100a)"; }
+const char* ipkv_version(void) { return kChecked ? "ipkv 0.2 (sm_100a, bounds-checked build)" : "ipkv 0.2 (sm_100a)"; }
 
 const char* ipkv_status_str(ipkv_status s) {
     switch (s) {
@@ -1128,7 +1139,7 @@ ipkv_status append_tokens(ipkv* h, int32_t layer, const int32_t* seq_ids, int32_
         note_kv_write(h, layer, false, true);
         const char* ks = static_cast<const char*>(k_dev) + base * k_row;
         const char* vs = v_dev ? static_cast<const char*>(v_dev) + base * v_row : nullptr;
-        CU(h, launch_append(h->geom, ks, vs, c.dim_v, h->w_layer(layer), rows, n, s));
+        CU(h, launch_append(h->geom, ks, vs, c.dim_v, h->w_layer(layer), rows, n, s, h->region_bytes(kSegBaseWindow), h->status_dev));
         h->stats.append_kernels += 1;
     }
     return IPKV_OK;
@@ -1150,7 +1161,7 @@ ipkv_status write_staged_rows(ipkv* h, int32_t layer, const int32_t* seq_ids, in
         note_kv_write(h, layer, false, true);
         const char* ks = static_cast<const char*>(k_dev) + base * k_row;
         const char* vs = v_dev ? static_cast<const char*>(v_dev) + base * v_row : nullptr;
-        CU(h, launch_append(h->geom, ks, vs, c.dim_v, h->w_layer(layer), rows, n, s));
+        CU(h, launch_append(h->geom, ks, vs, c.dim_v, h->w_layer(layer), rows, n, s, h->region_bytes(kSegBaseWindow), h->status_dev));
         h->stats.append_kernels += 1;
     }
     return IPKV_OK;
@@ -1666,6 +1677,9 @@ ipkv_status ipkv_get_stats(ipkv_t* h, ipkv_stats* out) {
     if (h->stats.device_status) {
         // reported once: the word is cleared so that the calls after this one are judged on their own
         CU(h, cudaMemset(h->status_dev, 0, sizeof(uint32_t)));
+        if (h->stats.device_status & kStatusBadIndex)
+            return fail(h, IPKV_EINTERNAL, "bounds-checked build: an index left its region; the access was not made" +
+                                               describe_device_status(h->stats.device_status));
         return fail(h, IPKV_ETIMEOUT, "a kernel's bounded wait gave up; results of that call are invalid" +
                                           describe_device_status(h->stats.device_status));
     }
@@ -1677,6 +1691,13 @@ ipkv_status ipkv_selftest_expire_wait(ipkv_t* h, uint32_t limit_us, void* stream
     DeviceGuard dev_guard(h->cfg.device);
     CU(h, dev_guard.error());
     CU(h, launch_expire_wait(h->status_dev, uint64_t(limit_us) * 1000ull, static_cast<cudaStream_t>(stream)));
+    return IPKV_OK;
+}
+
+ipkv_status ipkv_selftest_declare_bounds(ipkv_t* h, int32_t base_id, int64_t bytes) {
+    if (!h || base_id < 0 || base_id >= kMaxBases || bytes < 0) return IPKV_EINVAL;
+    if (!kChecked) return fail(h, IPKV_ESTATE, "not a bounds-checked build (libipkv_checked.so)");
+    h->selftest_bounds[base_id] = bytes;
     return IPKV_OK;
 }
 

@@ -64,6 +64,8 @@ struct GqaParams {
     int64_t head_bytes, block_bytes;
     float scale_log2;
     int win_tail;       // valid tokens in the last tile of runs flagged kSegTailParam
+    int64_t base_bytes[kMaxBases];   // bounds-checked build: extent behind every base (0: not checked)
+    int64_t part_rows;               // bounds-checked build: rows of partial storage
 };
 
 template <int D, int STAGES>
@@ -128,6 +130,9 @@ __global__ void __launch_bounds__(kThreads, 2) attn_gqa_kernel(const GqaParams p
             int cached_sp = -1;
             Seg seg{};
             const char* seg_base = nullptr;
+            const char* chk_lo = nullptr;       // bounds-checked build: the region the current run must lie in
+            int64_t chk_n = 0;
+            auto CHK = [&](const char* src, uint32_t bytes) { return ptx::checked_src<kChecked>(src, bytes, chk_lo, chk_n, p.status, kStatusBadIndex); };
             bool waited = !early;
             auto issue = [&](int sp, const Span& span, int tile, int slot) -> bool {
                 if (!waited && it >= STAGES) { ptx::grid_dependency_wait(); waited = true; }
@@ -135,6 +140,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_gqa_kernel(const GqaParams p
                     seg = p.segs[span.seg];
                     if (seg.base_id & kSegTailParam) seg.n_tokens += p.win_tail - kTileTokens;
                     seg_base = p.bases[seg.base_id & kSegBaseMask] + seg.off + int64_t(span.gh / p.n_hg) * p.head_bytes;
+                    chk_lo = p.bases[seg.base_id & kSegBaseMask]; chk_n = p.base_bytes[seg.base_id & kSegBaseMask];
                     cached_sp = sp;
                 }
                 // a tile of the D-window may have been written by the kernel in front of this one (an append kernel)
@@ -157,6 +163,11 @@ __global__ void __launch_bounds__(kThreads, 2) attn_gqa_kernel(const GqaParams p
                     s_meta[st].kv_row = span.row * (p.Hq / p.G) + g;
                     s_meta[st].g_lo = uint32_t(g_row);
                     s_meta[st].g_hi = uint32_t(g_row >> 32);
+                    if (kChecked && chk_n > 0) {           // the new rows' K and V chunks must land inside the window region
+                        const char* row_lo = reinterpret_cast<const char*>(g_row);
+                        const char* row_hi = row_lo + int64_t(D / 64 - 1) * p.bt * 128 + 128 + int64_t(p.bt) * D * 2;
+                        if (row_lo < chk_lo || row_hi > chk_lo + chk_n) { atomicOr(p.status, kStatusBadIndex); patch_tok = -1; }
+                    }
                 }
                 s_meta[st].patch_tok = patch_tok;
                 const uint32_t dst = s_base + st * SP::kStage;
@@ -167,14 +178,14 @@ __global__ void __launch_bounds__(kThreads, 2) attn_gqa_kernel(const GqaParams p
                     const char* src = seg_base + blk * p.block_bytes;
                     ptx::mbar_expect_tx(bar, SP::kStage);
                     if (p.bt == kTileTokens) {
-                        ptx::bulk_g2s_hint(dst, src, SP::kStage, bar, pol);   // K plane and V plane are adjacent
+                        ptx::bulk_g2s_hint(dst, CHK(src, SP::kStage), SP::kStage, bar, pol);   // K plane and V plane are adjacent
                     } else {
                         const int64_t kplane = int64_t(p.bt) * D * 2;
 #pragma unroll
                         for (int pn = 0; pn < D / 64; ++pn) {
                             const char* s0 = src + int64_t(pn) * p.bt * 128 + int64_t(r0) * 128;
-                            ptx::bulk_g2s_hint(dst + pn * 8192, s0, 8192, bar, pol);
-                            ptx::bulk_g2s_hint(dst + SP::kPlane + pn * 8192, s0 + kplane, 8192, bar, pol);
+                            ptx::bulk_g2s_hint(dst + pn * 8192, CHK(s0, 8192), 8192, bar, pol);
+                            ptx::bulk_g2s_hint(dst + SP::kPlane + pn * 8192, CHK(s0 + kplane, 8192), 8192, bar, pol);
                         }
                     }
                 } else {
@@ -189,8 +200,8 @@ __global__ void __launch_bounds__(kThreads, 2) attn_gqa_kernel(const GqaParams p
                         const char* src = seg_base + (blk0 + j) * p.block_bytes;
 #pragma unroll
                         for (int pn = 0; pn < D / 64; ++pn) {
-                            ptx::bulk_g2s_hint(dst + pn * 8192 + j * sub_bytes, src + int64_t(pn) * sub_bytes, sub_bytes, bar, pol);
-                            ptx::bulk_g2s_hint(dst + SP::kPlane + pn * 8192 + j * sub_bytes, src + kplane + int64_t(pn) * sub_bytes, sub_bytes, bar, pol);
+                            ptx::bulk_g2s_hint(dst + pn * 8192 + j * sub_bytes, CHK(src + int64_t(pn) * sub_bytes, sub_bytes), sub_bytes, bar, pol);
+                            ptx::bulk_g2s_hint(dst + SP::kPlane + pn * 8192 + j * sub_bytes, CHK(src + kplane + int64_t(pn) * sub_bytes, sub_bytes), sub_bytes, bar, pol);
                         }
                     }
                 }
@@ -263,6 +274,10 @@ __global__ void __launch_bounds__(kThreads, 2) attn_gqa_kernel(const GqaParams p
             l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
         }
         const int64_t prow = (int64_t(cur_slot) * kConsumerWarps + warp) * p.RG;
+        if (kChecked && (prow < 0 || prow + p.RG > p.part_rows)) {    // the partial's rows must lie inside the scratch
+            if (lane == 0) atomicOr(p.status, kStatusBadIndex);
+            return;
+        }
         if (r0 < n_heads) {
             const float inv = l0 > 0.f ? 1.f / l0 : 0.f;
             float* dst = p.part_o + (prow + r0) * D + c0;
@@ -442,6 +457,8 @@ cudaError_t launch_gqa(const AttnLaunch& a, cudaStream_t s) {
     p.n_rows = a.n_rows; p.n_gh = a.n_gh;
     p.early = a.early_tiles;
     p.win_tail = a.win_tail;
+    for (int i = 0; i < kMaxBases; ++i) p.base_bytes[i] = a.base_bytes[i];
+    p.part_rows = a.part_rows;
     p.Hq = a.n_q_heads; p.G = a.n_q_heads / a.n_kv_heads;
     p.n_hg = (p.G + 15) / 16;
     p.RG = part_geom(0, a.n_q_heads, a.n_kv_heads).rows_per_group;

@@ -66,6 +66,8 @@ struct MlaParams {
     int64_t block_bytes;
     float scale_log2;
     int win_tail;        // valid tokens in the last tile of runs flagged kSegTailParam
+    int64_t base_bytes[kMaxBases];   // bounds-checked build: extent behind every base (0: not checked)
+    int64_t part_rows;               // bounds-checked build: rows of partial storage
     int early;           // nonzero: the first copies of ring tiles (2: of window tiles too) need not wait for the previous kernel
 };
 
@@ -121,6 +123,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_mla_kernel(const MlaParams p
                 Seg seg = p.segs[span.seg];
                 if (seg.base_id & kSegTailParam) seg.n_tokens += p.win_tail - kTileTokens;
                 const char* seg_base = p.bases[seg.base_id & kSegBaseMask] + seg.off;
+                const char* chk_lo = p.bases[seg.base_id & kSegBaseMask];       // bounds-checked build: the region the run must lie in
+                const int64_t chk_n = p.base_bytes[seg.base_id & kSegBaseMask];
+                auto CHK = [&](const char* a, uint32_t bytes) { return ptx::checked_src<kChecked>(a, bytes, chk_lo, chk_n, p.status, kStatusBadIndex); };
                 for (int i = 0; i < span.ntiles; ++i, ++it) {
                     if (!waited && (it >= kStages || (p.early < 2 && (seg.base_id & kSegBaseMask) == kSegBaseWindow))) {
                         ptx::grid_dependency_wait();
@@ -141,12 +146,12 @@ __global__ void __launch_bounds__(kThreads, 1) attn_mla_kernel(const MlaParams p
                     if (it >= kStages && !ptx::mbar_wait(s_empty + 8 * st, ((it / kStages) - 1) & 1)) { ok = false; break; }
                     if (p.bt == kTileTokens) {
                         ptx::mbar_expect_tx(bar, kStageBytes);
-                        ptx::bulk_g2s_hint(dst, src, kStageBytes, bar, pol);
+                        ptx::bulk_g2s_hint(dst, CHK(src, kStageBytes), kStageBytes, bar, pol);
                     } else if (p.bt > kTileTokens) {
                         ptx::mbar_expect_tx(bar, kStageBytes);
 #pragma unroll
                         for (int pn = 0; pn < kPanels; ++pn)
-                            ptx::bulk_g2s_hint(dst + pn * 8192, src + int64_t(pn) * p.bt * 128 + row_off, 8192, bar, pol);
+                            ptx::bulk_g2s_hint(dst + pn * 8192, CHK(src + int64_t(pn) * p.bt * 128 + row_off, 8192), 8192, bar, pol);
                     } else {
                         const uint32_t sub_bytes = uint32_t(p.bt) * 128;
                         ptx::mbar_expect_tx(bar, uint32_t(live) * sub_bytes * kPanels);
@@ -154,7 +159,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_mla_kernel(const MlaParams p
                             const char* sj = src + j * p.block_bytes;
 #pragma unroll
                             for (int pn = 0; pn < kPanels; ++pn)
-                                ptx::bulk_g2s_hint(dst + pn * 8192 + j * sub_bytes, sj + int64_t(pn) * sub_bytes, sub_bytes, bar, pol);
+                                ptx::bulk_g2s_hint(dst + pn * 8192 + j * sub_bytes, CHK(sj + int64_t(pn) * sub_bytes, sub_bytes), sub_bytes, bar, pol);
                         }
                     }
                 }
@@ -311,7 +316,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_mla_kernel(const MlaParams p
         for (int d = 1; d < 16; d <<= 1) l_run += __shfl_xor_sync(0xffffffffu, l_run, d);
         if ((lane & 15) == 0) { s_m[srow] = m_run; s_l[srow] = l_run; }
         consumer_barrier();
-        {
+        if (kChecked && (int64_t(sn) + 1) * 16 > p.part_rows) {             // the partial's rows must lie inside the scratch
+            if (tid == 0) atomicOr(p.status, kStatusBadIndex);
+        } else {
             const int r0 = lane >> 2, c0 = warp * 64 + 2 * (lane & 3);
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
@@ -356,6 +363,8 @@ cudaError_t launch_attend_mla(const AttnLaunch& a, cudaStream_t s) {
     p.scale_log2 = a.scale * kLog2e;
     p.early = a.early_tiles;
     p.win_tail = a.win_tail;
+    for (int i = 0; i < kMaxBases; ++i) p.base_bytes[i] = a.base_bytes[i];
+    p.part_rows = a.part_rows;
     const int smem = kSmemTotal + 1024;
     static bool configured[64] = {};
     int dev = 0;

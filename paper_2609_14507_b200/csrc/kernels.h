@@ -38,6 +38,17 @@ constexpr int kMaxBases = 4;
 constexpr uint32_t kStatusNoFreeStage = 1u;     // the producer waited for the consumers to release a stage
 constexpr uint32_t kStatusNoTile = 2u;          // a consumer waited for a tile (or the end marker) to arrive
 constexpr uint32_t kStatusCopyNotLanded = 4u;   // the producer waited for its last copies before leaving
+constexpr uint32_t kStatusBadIndex = 8u;        // bounds-checked build only: a computed address left its region (the access was not made)
+
+// Bounds-checked build (-DIPKV_CHECKED; the stand-in for a memory checker): every source address the attention kernels
+// compute for a copy, every partial row they store and every window slot the append paths write is compared with the
+// extent of the region it must lie in.  A violation sets kStatusBadIndex in the status word and the access is redirected
+// to the start of the region (reads) or dropped (writes): nothing traps, nothing reads or writes out of bounds.
+#ifdef IPKV_CHECKED
+constexpr bool kChecked = true;
+#else
+constexpr bool kChecked = false;
+#endif
 
 struct AttnLaunch {
     int kind;                       // 0 = GQA, 1 = compressed latent (MLA)
@@ -60,6 +71,8 @@ struct AttnLaunch {
     uint32_t* status;               // device word, OR-ed with an error bit if a bounded wait gives up
     const void* append_k;           // fused append: [n_rows][n_kv_heads][dim_qk] bf16 new K rows (null: none)
     const void* append_v;           // [n_rows][n_kv_heads][dim_v]
+    int64_t base_bytes[kMaxBases];  // extent of the memory behind every base (0: unknown, not checked); used by the checked build
+    int64_t part_rows;              // rows of (O, LSE) partial storage behind part_o / part_lse
     int win_tail;                   // valid tokens in the last tile of the runs flagged kSegTailParam (1..64)
     int plain_launch;               // 1: the tables were written by the kernel right in front of this launch: no launch overlap
     int early_tiles;                // nonzero: no ring byte this launch reads (2: no window byte either) was written by the kernel
@@ -142,7 +155,8 @@ struct AppendRows {
     int32_t slot[kAppendRowsPerLaunch];      // token slot inside the window
 };
 // One new token per row into its D-window (TILE layout). k/v point at the first row of this launch.
+// w_bytes / status: extent of the layer's windows and the status word, for the bounds-checked build (0 / null: unchecked).
 cudaError_t launch_append(const BlockGeom& g, const void* k, const void* v, int dim_v_src, char* w_base,
-                          const AppendRows& rows, int n_rows, cudaStream_t s);
+                          const AppendRows& rows, int n_rows, cudaStream_t s, int64_t w_bytes = 0, uint32_t* status = nullptr);
 
 }  // namespace ipkvi

@@ -63,7 +63,7 @@ __global__ void tile_to_plain_kernel(BlockGeom g, const char* __restrict__ src, 
 }
 
 __global__ void append_kernel(BlockGeom g, const uint4* __restrict__ k, const uint4* __restrict__ v,
-                              char* __restrict__ w_base, AppendRows rows) {
+                              char* __restrict__ w_base, AppendRows rows, int64_t w_bytes, uint32_t* status) {
     ptx::grid_dependency_wait();       // launched so that it may come in under the previous kernel's tail (launch.cuh)
     ptx::grid_launch_dependents();
     const int row = blockIdx.x;
@@ -73,6 +73,10 @@ __global__ void append_kernel(BlockGeom g, const uint4* __restrict__ k, const ui
     const int64_t blk = slot / g.bt;
     const int toff = slot - int(blk) * g.bt;
     char* win = w_base + rows.dst_off[row] + blk * g.block_bytes();
+    if (kChecked && w_bytes > 0 && (slot < 0 || rows.dst_off[row] < 0 || rows.dst_off[row] + (blk + 1) * g.block_bytes() > w_bytes)) {
+        if (threadIdx.x == 0) atomicOr(status, kStatusBadIndex);      // the slot's block must lie inside the layer's windows
+        return;
+    }
     for (int i = threadIdx.x; i < per_token; i += blockDim.x) {
         int head, chunk;
         bool is_v;
@@ -151,9 +155,10 @@ cudaError_t launch_upload_by_value(void* dst_dev, const void* src_host, size_t b
 }
 
 cudaError_t launch_append(const BlockGeom& g, const void* k, const void* v, int /*dim_v_src*/, char* w_base,
-                          const AppendRows& rows, int n_rows, cudaStream_t s) {
+                          const AppendRows& rows, int n_rows, cudaStream_t s, int64_t w_bytes, uint32_t* status) {
     if (n_rows <= 0) return cudaSuccess;
-    return launch_overlapped(append_kernel, n_rows, 128, size_t(0), s, g, static_cast<const uint4*>(k), static_cast<const uint4*>(v), w_base, rows);
+    return launch_overlapped(append_kernel, n_rows, 128, size_t(0), s, g, static_cast<const uint4*>(k), static_cast<const uint4*>(v), w_base, rows,
+                             w_bytes, status);
 }
 
 }  // namespace ipkvi

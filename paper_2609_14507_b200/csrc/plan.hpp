@@ -40,7 +40,8 @@ inline std::string describe_device_status(uint32_t status) {
     if (status & kStatusNoFreeStage) where += " [a producer got no free stage]";
     if (status & kStatusNoTile) where += " [a consumer got no tile]";
     if (status & kStatusCopyNotLanded) where += " [a copy did not land]";
-    if (status & ~(kStatusNoFreeStage | kStatusNoTile | kStatusCopyNotLanded)) where += " [unknown bits]";
+    if (status & kStatusBadIndex) where += " [checked build: a computed address left its region]";
+    if (status & ~(kStatusNoFreeStage | kStatusNoTile | kStatusCopyNotLanded | kStatusBadIndex)) where += " [unknown bits]";
     return where;
 }
 

@@ -103,6 +103,18 @@ __device__ __forceinline__ float ex2(float x) {
     return y;
 }
 
+// Bounds-checked build: `src .. src + bytes` must lie inside [lo, lo + extent) (extent 0: unknown, not checked); if it does
+// not, `bit` goes into the status word and the region's first bytes are read instead.  Compiles to `src` otherwise.
+template <bool CHECKED>
+__device__ __forceinline__ const char* checked_src(const char* src, uint32_t bytes, const char* lo, int64_t extent, uint32_t* status,
+                                                   uint32_t bit) {
+    if (CHECKED && extent > 0 && (src < lo || src + bytes > lo + extent)) {
+        atomicOr(status, bit);
+        return lo;
+    }
+    return src;
+}
+
 // Programmatic dependent launch (see launch.cuh): wait for the previous kernel of the stream / let the next one come in.
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }

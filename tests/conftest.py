@@ -19,6 +19,7 @@ def pytest_sessionstart(session):
         from paper_2609_14507_b200 import build
         if os.path.exists(build.NVCC):
             build.build()
+            build.build(checked=True)
     except Exception as e:                                  # the tests that need the library will say so themselves
         sys.stderr.write(f"conftest: could not build libipkv.so: {e}\n")
 

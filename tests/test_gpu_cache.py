@@ -1015,3 +1015,31 @@ def test_failed_launch_behind_a_fused_append_leaves_the_window_consistent():
                 want = ref.attend(q[0], "gpu", float(np.float32(sh.scale)))
                 check_partial(o.cpu().numpy()[0], lse.cpu().numpy()[0], want[0], want[1], f"step {step}")
         assert cache.get_stats()["device_status"] == 0
+
+
+def test_checked_build_records_an_address_outside_its_declared_region():
+    """Only in the bounds-checked build (IPKV_LIB_VARIANT=checked): the resident ring is declared 64 KB long although it
+    is larger, so the attention launch computes source addresses beyond the declared extent.  Those copies are redirected
+    to the region's first bytes (nothing outside valid memory is touched, nothing traps), the status word gets the
+    bad-index bit and ipkv_get_stats returns IPKV_EINTERNAL once; with the real extent restored the same call matches the oracle."""
+    if b"bounds-checked" not in binding.lib().ipkv_version_bytes():
+        pytest.skip("ordinary build: the checks are compiled out")
+    sh = synth.SMALL_GQA
+    L = 1500
+    k, v = synth.host_kv(sh, L, seed=993)
+    q = synth.host_q(sh, 1, seed=994)
+    with make_cache(sh, 1, 1, block_tokens=64, window_tokens=256, chunk_tokens=512, max_u_tokens_per_seq=2048,
+                    max_p_tokens_per_seq=2048, resident_tokens_per_seq=2048) as cache:
+        cache.append_bulk(0, 0, synth.bits_to_torch(k, DEV), synth.bits_to_torch(v, DEV), L, 0, 1)
+        o = torch.zeros((1, sh.n_q_heads, sh.dim_v), device=DEV); lse = torch.zeros((1, sh.n_q_heads), device=DEV)
+        cache.selftest_declare_bounds(0, 65536)
+        cache.attend_gpu(0, [0], synth.bits_to_torch(q, DEV), o, lse)
+        with pytest.raises(binding.IpkvError) as err:
+            cache.get_stats()
+        assert err.value.status == 7 and "left its region" in str(err.value)       # IPKV_EINTERNAL
+        cache.selftest_declare_bounds(0, 0)
+        cache.attend_gpu(0, [0], synth.bits_to_torch(q, DEV), o, lse)
+        torch.cuda.synchronize()
+        assert cache.get_stats()["device_status"] == 0
+        o_ref, l_ref = c_oracle.attend(q[0], k, v, np.arange(L), float(np.float32(sh.scale)))
+        check_partial(o.cpu().numpy()[0], lse.cpu().numpy()[0], o_ref, l_ref, "checked build, real bounds")

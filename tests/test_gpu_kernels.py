@@ -199,6 +199,24 @@ def test_mla_tcgen05_variant_matches_oracle():
     assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
 
 
+def test_bounds_checked_build_passes_the_small_parity_cases():
+    """The -DIPKV_CHECKED build of the same kernels (every computed source address, partial row and window slot compared
+    with its region's extent; the stand-in for a memory checker) runs the small-shape parity tests of both attention
+    kernels, the handle-based decode tests and its own self-test without recording a violation where none is planted.
+    A child process, because the library variant is chosen when the library is first loaded."""
+    import os
+    import subprocess
+    import sys
+    env = dict(os.environ, IPKV_LIB_VARIANT="checked")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run([sys.executable, "-m", "pytest", "-q", "-m", "gpu", "-x", os.path.join(root, "tests", "test_gpu_kernels.py"),
+                        os.path.join(root, "tests", "test_gpu_cache.py"), "-k",
+                        "attend_runs_gqa or attend_runs_mla or peaked or config1 or decode_steps or ring_capacity or fused or checked_build_records"],
+                       env=env, cwd=root, capture_output=True, text=True, timeout=900)
+    assert r.returncode == 0, r.stdout[-3000:] + r.stderr[-2000:]
+    assert " passed" in r.stdout and "skipped" not in r.stdout.splitlines()[-1]
+
+
 def test_read_bandwidth_probe_runs():
     """The measurement aid behind `roofline.read_ceiling`: a read-only stream through the kernels' copy ring."""
     best, mean = binding.ipkv_probe_read_bandwidth(0, 256 << 20, 3)

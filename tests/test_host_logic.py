@@ -228,7 +228,7 @@ def test_device_status_word_maps_to_the_documented_messages():
     assert "no tile" in text(2) and "free stage" not in text(2)
     assert "did not land" in text(4)
     assert all(k in text(7) for k in ("free stage", "no tile", "did not land"))
-    assert "unknown" in text(8)
+    assert "left its region" in text(8) and "unknown" in text(16)
 
 
 def test_resident_ring_never_hands_a_slot_out_twice():
