@@ -594,6 +594,15 @@ def main():
     if "--cpu-engine-microbench" in sys.argv:
         cpu_engine_microbench()
         return
+    if "--umma-microbench" in sys.argv:
+        # cost of small tcgen05.mma instructions (one CTA, one issuing thread): fixed cost against throughput
+        from paper_2609_14507_b200 import binding
+        rows = binding.ipkv_probe_umma(0, 5)
+        for r in rows:
+            r["cycles_per_mma"] = r["total_cycles"] / r["n_mma"]
+        print(json.dumps({"umma_microbench": rows, "note": "SM clocks; K = 16 per instruction, bf16 operands from shared memory "
+                          "(128-byte swizzle), fp32 accumulators in tensor memory; issue = until the commit was issued, total = until it completed"}))
+        return
     if "--two-engine" in sys.argv or "--two-engine-resident" in sys.argv:
         two_engine_bench(resident="--two-engine-resident" in sys.argv)
         return

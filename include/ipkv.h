@@ -348,6 +348,15 @@ ipkv_status ipkv_profile_read(ipkv_t* h, double* attend_kernel_ms, int64_t* n_ti
  * call, runs 3 warm-up and `reps` timed launches (CUDA events), returns the best and the mean. */
 ipkv_status ipkv_probe_read_bandwidth(int32_t device, size_t bytes, int32_t reps, double* best_gbs, double* mean_gbs);
 
+/* Measurement aid (no counterpart in the paper): the cost of small fifth-generation tensor-core instructions on `device`.
+ * One CTA, one issuing thread: n_mma back-to-back tcgen05.mma of shape M x N x 16 (bf16 in, fp32 accumulate in tensor
+ * memory, operands in shared memory) and one commit.  issue_cycles: SM clocks until the last instruction and the commit
+ * were issued; total_cycles: until the commit's barrier completed; best of `reps` launches.  Shapes M 64 / 128 x N 16 /
+ * 64 / 256 with n_mma 1, 8, 36 into one accumulator, and 36 rotating over four accumulators where they fit: the fixed
+ * cost per instruction and the throughput separate.  Fills out[0 .. *n_out). */
+typedef struct { int32_t m, n, n_mma, accumulators; int64_t issue_cycles, total_cycles; } ipkv_umma_timing;
+ipkv_status ipkv_probe_umma(int32_t device, int32_t reps, ipkv_umma_timing* out, int32_t cap, int32_t* n_out);
+
 /* ---- stateless kernel entry points (no handle) ------------------------------------------------- */
 
 typedef struct {

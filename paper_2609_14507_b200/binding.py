@@ -27,7 +27,7 @@ EXPORTS = [
     "ipkv_attend_runs_noalloc", "ipkv_noalloc_scratch_limit", "ipkv_roofline_share", "ipkv_roofline_step_time",
     "ipkv_policy_create", "ipkv_policy_destroy", "ipkv_policy_observe", "ipkv_policy_update", "ipkv_policy_prefill_share",
     "ipkv_block_bytes", "ipkv_status_str", "ipkv_last_error", "ipkv_version", "ipkv_probe_read_bandwidth",
-    "ipkv_selftest_expire_wait", "ipkv_selftest_fail_next_launch", "ipkv_selftest_declare_bounds",
+    "ipkv_selftest_expire_wait", "ipkv_selftest_fail_next_launch", "ipkv_selftest_declare_bounds", "ipkv_probe_umma",
 ]
 
 
@@ -209,6 +209,23 @@ def make_config(kind, n_layers, max_seqs, n_q_heads, n_kv_heads, dim_qk, dim_v, 
         c._ring_keepalive = (C.c_int64 * max_seqs)(*[int(x) for x in resident_tokens_by_seq])
         c.resident_tokens_by_seq = C.cast(c._ring_keepalive, C.POINTER(C.c_int64))
     return c
+
+
+class UmmaTiming(C.Structure):
+    _fields_ = [("m", C.c_int32), ("n", C.c_int32), ("n_mma", C.c_int32), ("accumulators", C.c_int32),
+                ("issue_cycles", C.c_int64), ("total_cycles", C.c_int64)]
+
+
+def ipkv_probe_umma(device=0, reps=5):
+    """List of dicts: SM clocks for n back-to-back tcgen05.mma of small shapes (see ipkv.h)."""
+    out = (UmmaTiming * 64)()
+    n = C.c_int32()
+    f = lib().ipkv_probe_umma
+    f.argtypes = [C.c_int32, C.c_int32, C.POINTER(UmmaTiming), C.c_int32, C.POINTER(C.c_int32)]
+    rc = f(device, reps, out, 64, C.byref(n))
+    if rc != OK:
+        raise IpkvError(rc, "ipkv_probe_umma")
+    return [{k: getattr(out[i], k) for k, _ in UmmaTiming._fields_} for i in range(n.value)]
 
 
 def ipkv_probe_read_bandwidth(device=0, nbytes=1 << 30, reps=10):
