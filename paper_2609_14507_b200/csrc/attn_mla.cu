@@ -282,33 +282,51 @@ __global__ void __launch_bounds__(kThreads, 1) attn_mla_kernel(const MlaParams p
                     for (int nt = 0; nt < 8; ++nt) { o[nt][0] *= a0; o[nt][1] *= a0; o[nt][2] *= a1; o[nt][3] *= a1; }
                 }
                 const uint32_t vb = kb + warp * 8192;
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {
-                    uint32_t ph[4], pl[4];
+                auto load_p = [&](int kk, uint32_t (&ph)[4], uint32_t (&pl)[4]) {
                     const uint32_t poff = ((mi & 1) * 8 + r8) * kPPitch + (kk * 2 + (mi >> 1)) * 16;
                     ptx::ldmatrix_x4(s_phi + poff, ph[0], ph[1], ph[2], ph[3]);
                     ptx::ldmatrix_x4(s_plo + poff, pl[0], pl[1], pl[2], pl[3]);
+                };
+                auto load_v = [&](int kk, uint32_t (&vf)[4][4]) {
                     const int tok = kk * 16 + (mi & 1) * 8 + r8;
-                    // all value fragments first, then the p_hi products, then the p_lo products: two MMAs on the
-                    // same accumulator are eight instructions apart
-                    uint32_t vf[4][4];
 #pragma unroll
                     for (int jj = 0; jj < 4; ++jj)
                         ptx::ldmatrix_x4_trans(vb + tok * 128 + (((2 * jj + (mi >> 1)) ^ r8) << 4), vf[jj][0], vf[jj][1], vf[jj][2], vf[jj][3]);
+                };
+                auto product = [&](const uint32_t (&pw)[4], const uint32_t (&vf)[4][4]) {
 #pragma unroll
                     for (int jj = 0; jj < 4; ++jj) {
-                        ptx::mma_bf16(o[2 * jj], ph, vf[jj][0], vf[jj][1]);
-                        ptx::mma_bf16(o[2 * jj + 1], ph, vf[jj][2], vf[jj][3]);
+                        ptx::mma_bf16(o[2 * jj], pw, vf[jj][0], vf[jj][1]);
+                        ptx::mma_bf16(o[2 * jj + 1], pw, vf[jj][2], vf[jj][3]);
                     }
+                };
+                // all value fragments of a 16-token step first, then the p_hi products, then the p_lo products: two MMAs on
+                // the same accumulator are eight instructions apart
 #pragma unroll
-                    for (int jj = 0; jj < 4; ++jj) {
-                        ptx::mma_bf16(o[2 * jj], pl, vf[jj][0], vf[jj][1]);
-                        ptx::mma_bf16(o[2 * jj + 1], pl, vf[jj][2], vf[jj][3]);
-                    }
+                for (int kk = 0; kk < 2; ++kk) {
+                    uint32_t ph[4], pl[4], vf[4][4];
+                    load_p(kk, ph, pl);
+                    load_v(kk, vf);
+                    product(ph, vf);
+                    product(pl, vf);
+                }
+                // The last two steps: both steps' value fragments are fetched first and their p_hi products issued (an MMA is
+                // not issued before its operands are there, so after them the tile's last bytes have been read); the stage then
+                // goes back to the producer while the p_lo products, half of these steps' MMAs, are still to come.
+                {
+                    uint32_t ph2[4], pl2[4], ph3[4], pl3[4], vf2[4][4], vf3[4][4];
+                    load_p(2, ph2, pl2);
+                    load_v(2, vf2);
+                    load_p(3, ph3, pl3);
+                    load_v(3, vf3);
+                    product(ph2, vf2);
+                    product(ph3, vf3);
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(s_empty + 8 * st);
+                    product(pl2, vf2);
+                    product(pl3, vf3);
                 }
             }
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(s_empty + 8 * st);
         }
 
         // ---- end of span: the row owners publish m and l, every warp scales and writes its 64 columns ----
