@@ -60,8 +60,8 @@ DRAM_TRAFFIC_PER_LAUNCH = {
     "mixtral-2layers-bs16-32k-cpu25": 1615.2e6 + 5.3e6,
     "qwen3-30b-a3b-bs16-32k-cpu0": 1076.1e6 + 4.6e6,
     "qwen3-2layers-bs16-32k-cpu0": 1076.1e6 + 4.6e6,
-    "deepseek-v2-lite-mla-bs8-128k-cpu40": 725.7e6 + 5.6e6,
-    "deepseek-v2-lite-mla-2layers-bs8-128k-cpu40": 725.7e6 + 5.6e6,
+    "deepseek-v2-lite-mla-bs8-128k-cpu40": 725.7e6 + 4.1e6,
+    "deepseek-v2-lite-mla-2layers-bs8-128k-cpu40": 725.7e6 + 4.1e6,
 }
 DEFAULT_WORKLOAD = "mixtral-8x7b-bs16-32k-cpu25"
 # Short runs of the other BASELINE configurations, reported beside the default line (rank 0, one GPU): config 3 at CPU

@@ -18,7 +18,9 @@
 //      masks the ragged tail and updates the running max / sum of its rows (fp32, log2 domain); the
 //      weights are split p = p_hi + p_lo (two bf16) and written to shared memory with the rescale factor.
 //   3. output: warp w owns value columns [64w, 64w+64) (one panel): O = O*alpha + (P_hi + P_lo) V with
-//      fp32 accumulators in registers.
+//      fp32 accumulators in registers.  The stage goes back to the producer as soon as the tile's last bytes have
+//      been read into registers, before the last p_lo products: what bounds this kernel is how long a stage is
+//      held (a stage that is computed on is not being refilled), so everything that shortens the hold counts.
 // HBM traffic per KV token: 1152 bytes, read exactly once per group of 16 heads.
 #include <cuda_bf16.h>
 
