@@ -623,6 +623,8 @@ def main():
                     help="diagnostic: the kernel timed by CUDA events is the split reduce, not the attention kernel (the roofline object is then meaningless)")
     ap.add_argument("--static-schedule", action="store_true",
                     help="fixed tile assignment in the grouped-query kernel (bit-reproducible) instead of dynamic balancing")
+    ap.add_argument("--force-balance", action="store_true",
+                    help="dynamic balancing of the grouped-query kernel whatever the launch's length (the library switches it on from 64 tiles per CTA)")
     ap.add_argument("--separate-append", action="store_true",
                     help="ipkv_append as a call and a launch of its own instead of riding in ipkv_attend_gpu")
     ap.add_argument("--separate-merge", action="store_true",
@@ -695,7 +697,7 @@ def main():
     # the fused form of a layer (append riding in the call, CPU partial folded by the reduce) with its arguments marshalled once
     calls = None
     if fused and not args.separate_append:
-        calls = [cache.attend_gpu_call(l, seq_ids, q_l[l], out_l[l], out_lse, kv_splits=args.kv_splits, static_schedule=args.static_schedule,
+        calls = [cache.attend_gpu_call(l, seq_ids, q_l[l], out_l[l], out_lse, kv_splits=args.kv_splits, static_schedule=args.static_schedule, force_balance=args.force_balance,
                                        stream=cur, fold_o=oc_l[l], fold_lse=lc_l[l], **apps[l]) for l in range(NL)]
 
     def step():

@@ -713,24 +713,6 @@ void fill_launch(AttnLaunch* a, int kind, int Hq, int Hkv, int dqk, int dv, int 
 }
 
 // One group of segments for all rows: attention + split reduce, folding into (out_o, out_lse) when `fold`.
-// D-window runs that all end at the same offset inside their last tile are flagged so that their token counts travel
-// as one launch parameter (kSegTailParam); returns that offset (1..64), or 0 when the runs disagree or there are none.
-int window_tail(std::vector<std::vector<PlanSeg>>& rows) {
-    int tail = 0;
-    for (const auto& row : rows)
-        for (const PlanSeg& s : row) {
-            if (s.base_id != kSegBaseWindow || s.n_tokens <= 0) continue;
-            const int t = int((s.n_tokens - 1) % kTileTokens) + 1;
-            if (tail == 0) tail = t;
-            else if (tail != t) return 0;
-        }
-    if (tail == 0) return 0;
-    for (auto& row : rows)
-        for (PlanSeg& s : row)
-            if (s.base_id == kSegBaseWindow && s.n_tokens > 0) s.tail_param = true;
-    return tail;
-}
-
 ipkv_status run_group(ipkv* h, std::vector<std::vector<PlanSeg>>& rows, const char* const bases[kMaxBases],
                       const void* q, int kv_splits, const float* fold_o, const float* fold_lse, float* out_o, float* out_lse,
                       cudaStream_t s, int schedule_flags = 0, const void* append_k = nullptr, const void* append_v = nullptr,

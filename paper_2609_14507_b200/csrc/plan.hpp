@@ -75,6 +75,24 @@ struct Plan {
     }
 };
 
+// D-window runs that all end at the same offset inside their last tile are flagged so that their token counts travel
+// as one launch parameter (kSegTailParam); returns that offset (1..64), or 0 when the runs disagree or there are none.
+inline int window_tail(std::vector<std::vector<PlanSeg>>& rows) {
+    int tail = 0;
+    for (const auto& row : rows)
+        for (const PlanSeg& s : row) {
+            if (s.base_id != kSegBaseWindow || s.n_tokens <= 0) continue;
+            const int t = int((s.n_tokens - 1) % kTileTokens) + 1;
+            if (tail == 0) tail = t;
+            else if (tail != t) return 0;
+        }
+    if (tail == 0) return 0;
+    for (auto& row : rows)
+        for (PlanSeg& s : row)
+            if (s.base_id == kSegBaseWindow && s.n_tokens > 0) s.tail_param = true;
+    return tail;
+}
+
 // Upper bound on the number of spans build_plan can produce.  Pass 1 emits one piece per (row, head group, run), or,
 // with kv_splits, at most kv_splits + 1 pieces of it (a row's runs share the row's kv_splits pieces, each run rounds up
 // once); pass 2 then cuts a piece wherever a CTA's chunk ends inside it: one cut per CTA boundary, and there are never

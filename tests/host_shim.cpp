@@ -110,6 +110,33 @@ int64_t shim_ring_slots(int n_seqs, int64_t uniform_tokens, const int64_t* token
     return n;
 }
 
+// Two consecutive decode steps of a batch: window runs of `fill` and `fill + 1` tokens behind a resident run each.
+// Returns the launch parameter win_tail of the first step and, in *same_table, whether the two steps' serialised launch
+// tables are byte-identical (they must be, unless a window grows into a new tile, when the plan itself changes).
+int shim_window_tail(int n_rows, const int64_t* resident_tokens, const int64_t* window_fill, int n_gh, int ctas_per_sm, int* same_table,
+                     int* tail_next_out) {
+    std::vector<char> img[2];
+    int tails[2] = {0, 0};
+    for (int step = 0; step < 2; ++step) {
+        std::vector<std::vector<PlanSeg>> rows(n_rows);
+        for (int r = 0; r < n_rows; ++r) {
+            if (resident_tokens[r] > 0) rows[r].push_back(PlanSeg{0, int64_t(r) << 24, resident_tokens[r]});
+            if (window_fill[r] + step > 0) rows[r].push_back(PlanSeg{kSegBaseWindow, int64_t(r) << 16, window_fill[r] + step});
+        }
+        tails[step] = window_tail(rows);
+        Plan plan;
+        build_plan(rows, n_gh, 0, ctas_per_sm, &plan);
+        img[step].assign(plan.table_bytes(), 0);
+        plan.serialize(img[step].data());
+        int64_t want = 0;
+        for (int r = 0; r < n_rows; ++r) want += resident_tokens[r] + window_fill[r] + step;
+        if (plan.total_tokens != want) return -1;                   // the real counts stay the plan's counts
+    }
+    *same_table = img[0] == img[1] ? 1 : 0;
+    *tail_next_out = tails[1];
+    return tails[0];
+}
+
 int64_t shim_tile_chunk_offset(int32_t bt, int32_t t, int32_t chunk) { return tile_chunk_offset(bt, t, chunk); }
 int64_t shim_plain_chunk_offset(int32_t d, int32_t t, int32_t chunk) { return plain_chunk_offset(d, t, chunk); }
 int64_t shim_block_bytes(int32_t hkv, int32_t dqk, int32_t dv_stored, int32_t bt) {

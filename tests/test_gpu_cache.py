@@ -1043,3 +1043,52 @@ def test_checked_build_records_an_address_outside_its_declared_region():
         assert cache.get_stats()["device_status"] == 0
         o_ref, l_ref = c_oracle.attend(q[0], k, v, np.arange(L), float(np.float32(sh.scale)))
         check_partial(o.cpu().numpy()[0], lse.cpu().numpy()[0], o_ref, l_ref, "checked build, real bounds")
+
+
+@pytest.mark.parametrize("kind", ["gqa", "mla"])
+def test_decode_with_windows_in_and_out_of_step(kind):
+    """The D-window's fill reaches the kernels either as one launch parameter (all listed windows end at the same offset in
+    their last tile: the launch tables of consecutive steps are then identical) or in the tables (windows out of step).
+    Three sequences decode in lockstep across a tile boundary (63 -> 66 tokens in the window), then one of them alone,
+    then all three again, with the append riding in the attention call; every step's partial is checked against the oracle."""
+    if kind == "gqa":
+        sh = synth.Shape("g", "gqa", 1, 16, 2, 128, 128, 128 ** -0.5)
+    else:
+        sh = synth.Shape("m", "mla", 1, 16, 1, 576, 512, 192 ** -0.5)
+    rng = np.random.default_rng(101)
+    scale = float(np.float32(sh.scale))
+    seqs, lens = [0, 1, 2], [700, 64, 1300]
+    hq, dv = sh.n_q_heads, sh.dim_v
+    with make_cache(sh, 1, 3, block_tokens=64, window_tokens=256, chunk_tokens=256, max_u_tokens_per_seq=2048,
+                    max_p_tokens_per_seq=2048, resident_tokens_per_seq=2048, share_num=0, share_den=1) as cache:
+        refs = []
+        for s_ in seqs:
+            r = RefSeq(sh, 64, 256, 0, 1)
+            k, v = synth.host_kv(sh, lens[s_], seed=10100 + s_)
+            cache.append_bulk(0, s_, synth.bits_to_torch(k, DEV), None if v is None else synth.bits_to_torch(v, DEV), lens[s_], 0, 1)
+            r.bulk(k, v, 0, 1)
+            refs.append(r)
+
+        def step(which, what):
+            n = len(which)
+            kn = synth.normal_bf16(rng, (n, sh.n_kv_heads, sh.dim_qk))
+            vn = None if sh.kind == "mla" else synth.normal_bf16(rng, (n, sh.n_kv_heads, dv))
+            q = synth.normal_bf16(rng, (n, hq, sh.dim_qk))
+            o = torch.zeros((n, hq, dv), device=DEV); lse = torch.zeros((n, hq), device=DEV)
+            cache.attend_gpu(0, which, synth.bits_to_torch(q, DEV), o, lse, append_k=synth.bits_to_torch(kn, DEV),
+                             append_v=None if vn is None else synth.bits_to_torch(vn, DEV))
+            for i, s_ in enumerate(which):
+                refs[s_].append(kn[i:i + 1], None if vn is None else vn[i:i + 1])
+            torch.cuda.synchronize()
+            want = [refs[s_].attend(q[i], "gpu", scale) for i, s_ in enumerate(which)]
+            check_partial(o.cpu().numpy(), lse.cpu().numpy(), np.stack([w[0] for w in want]), np.stack([w[1] for w in want]), what)
+
+        for t in range(66):                      # in lockstep, across the boundary of the window's first tile
+            step(seqs, f"lockstep {t}")
+        for t in range(5):                       # one sequence runs ahead: its window is now out of step with the others
+            step([1], f"alone {t}")
+        for t in range(70):                      # all three again: exact counts in the tables, across another boundary
+            step(seqs, f"out of step {t}")
+        for s_, r in enumerate(refs):
+            check_routing(cache, 0, s_, r, sample=range(0, len(r.k), 29))
+        assert cache.get_stats()["device_status"] == 0

@@ -269,3 +269,27 @@ def test_resident_ring_never_hands_a_slot_out_twice():
                                 max_u_tokens_per_seq=64, max_p_tokens_per_seq=8192, resident_tokens_per_seq=8192,
                                 flags=binding.FLAG_NO_HOST_U | binding.FLAG_NO_HOST_P)
     assert binding.ipkv_query_sizes(cfg_u)["resident"] == 3 * 4 * 128 * 64 * 2048
+
+
+def test_window_fill_travels_as_a_launch_parameter_while_the_batch_is_in_lockstep():
+    """When every D-window run of a launch ends at the same offset inside its last 64-token tile, the runs are stored
+    rounded up to whole tiles and the offset becomes the launch parameter: two consecutive decode steps then have
+    byte-identical tables (no upload), until the windows grow into a new tile.  Windows that disagree keep their exact
+    counts in the table (parameter 0), and the tables differ from step to step."""
+    import ctypes
+    L = host_shim.lib()
+    i64 = ctypes.c_int64
+
+    def two_steps(resident, fills, n_gh=4, cps=2):
+        res = (i64 * len(resident))(*resident); fl = (i64 * len(fills))(*fills)
+        same, nxt = ctypes.c_int(), ctypes.c_int()
+        t = L.shim_window_tail(len(resident), res, fl, n_gh, cps, ctypes.byref(same), ctypes.byref(nxt))
+        return t, nxt.value, bool(same.value)
+
+    assert two_steps([8192] * 4, [5] * 4) == (5, 6, True)
+    assert two_steps([8192, 100, 33000], [63, 127, 191]) == (63, 64, True)     # different windows, same offset in the last tile
+    assert two_steps([8192] * 4, [64] * 4) == (64, 1, False)                   # the next token opens a new tile: a new plan
+    assert two_steps([8192] * 4, [0] * 4)[0] == 0                              # no window tokens yet: nothing to flag
+    t, nxt, same = two_steps([8192, 8192], [5, 6])
+    assert (t, nxt, same) == (0, 0, False)                                     # windows out of step: exact counts, tables differ
+    assert two_steps([0, 8192], [17, 17], n_gh=1, cps=1) == (17, 18, True)     # a row with nothing but its window
