@@ -138,6 +138,11 @@ struct ipkv {
     uint32_t* status_dev = nullptr;
     // scheduling words of the dynamically balanced attention kernel: two sets used by alternate launches; the
     // split reduce of one launch zeroes the set of the next
+    // the plan of the previous launch and what it was built from: a launch over the same runs (every layer of a decode step,
+    // and the next steps while the windows stay inside their tiles) reuses it without planning or serialising anything
+    Plan last_plan;
+    std::vector<int64_t> plan_sig_scratch;
+    std::vector<int64_t> last_plan_sig;
     bool fail_next_launch = false;                   // self-test: the next attention launch is refused on the host
     int32_t* steal_dev = nullptr;
     static constexpr int kStealWords = 1 << 16;     // per set
@@ -722,10 +727,32 @@ ipkv_status run_group(ipkv* h, std::vector<std::vector<PlanSeg>>& rows, const ch
         h->fail_next_launch = false;
         return fail(h, IPKV_ECUDA, "attention launch refused (ipkv_selftest_fail_next_launch)");
     }
-    Plan plan;
+    const Plan* plan_ptr = nullptr;
     const PartGeom pg = part_geom(c.kind, c.n_q_heads, c.n_kv_heads);
     const int win_tail = window_tail(rows);
-    build_plan(rows, pg.n_gh, kv_splits, pg.ctas_per_sm, &plan);
+    // signature of everything the plan depends on (the token counts as the tables will hold them)
+    std::vector<int64_t>& sig = h->plan_sig_scratch;
+    sig.clear();
+    sig.push_back(int64_t(rows.size())); sig.push_back(pg.n_gh); sig.push_back(kv_splits); sig.push_back(pg.ctas_per_sm);
+    int64_t total_tokens = 0;
+    for (const auto& row : rows) {
+        sig.push_back(int64_t(row.size()));
+        for (const PlanSeg& sg : row) {
+            total_tokens += sg.n_tokens > 0 ? sg.n_tokens : 0;
+            sig.push_back(sg.off);
+            sig.push_back(sg.tail_param ? (sg.n_tokens + kTileTokens - 1) / kTileTokens * kTileTokens : sg.n_tokens);
+            sig.push_back(int64_t(sg.base_id) | (sg.appended ? 1 << 8 : 0) | (sg.tail_param ? 1 << 9 : 0));
+        }
+    }
+    const bool same_plan = h->last_table_valid && h->last_table_stream == s && sig == h->last_plan_sig;
+    if (same_plan) {
+        plan_ptr = &h->last_plan;
+    } else {
+        build_plan(rows, pg.n_gh, kv_splits, pg.ctas_per_sm, &h->last_plan);
+        h->last_plan_sig = sig;
+        plan_ptr = &h->last_plan;
+    }
+    const Plan& plan = *plan_ptr;
     // dynamic balancing (grouped-query kernel): every CTA may fill up to kStealSlots extra partials
     const size_t n_lists = rows.size() * size_t(pg.n_gh) * (1 + kStealListCap);
     const size_t steal_words = n_lists + plan.spans.size() + 2 * size_t(plan.n_ctas());
@@ -740,8 +767,12 @@ ipkv_status run_group(ipkv* h, std::vector<std::vector<PlanSeg>>& rows, const ch
     ipkv_status rc = ensure_scratch(h, partial_bytes(plan.spans.size() + extra, pg, c.dim_v));
     if (rc != IPKV_OK) return rc;
     const char* table = nullptr;
-    rc = upload_table(h, plan, s, &table);
-    if (rc != IPKV_OK) return rc;
+    if (same_plan) {
+        table = h->table_dev + h->last_table_off;          // the tables of the previous launch, still in place
+    } else {
+        rc = upload_table(h, plan, s, &table);
+        if (rc != IPKV_OK) { h->last_plan_sig.clear(); return rc; }
+    }
     AttnLaunch a{};
     fill_launch(&a, c.kind, c.n_q_heads, c.n_kv_heads, c.dim_qk, c.dim_v, c.block_tokens, h->scale, plan, table, h->scratch, q,
                 int(rows.size()), extra);
@@ -791,7 +822,7 @@ ipkv_status run_group(ipkv* h, std::vector<std::vector<PlanSeg>>& rows, const ch
         if (timed) { CU(h, cudaEventRecord(h->prof_ev[h->prof_used + 1], s)); h->prof_used += 2; }
     }
     h->stats.reduce_kernels += 1;
-    h->stats.kv_bytes_attended += uint64_t(plan.total_tokens) * uint64_t(h->bb / c.block_tokens);
+    h->stats.kv_bytes_attended += uint64_t(total_tokens) * uint64_t(h->bb / c.block_tokens);
     return IPKV_OK;
 }
 
