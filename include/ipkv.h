@@ -304,7 +304,8 @@ ipkv_status ipkv_selftest_fail_next_launch(ipkv_t* h);
 
 /* Bounds-checked build (libipkv_checked.so, compiled with -DIPKV_CHECKED; ipkv_version() says so): every source address
  * the attention kernels compute for a copy, every partial row they store and every window slot the append paths write is
- * compared with the extent of its region.  A violation is recorded (device_status bit 3), the access is not made (a read
+ * compared with the extent of its region, and the ring destinations the host computes for the packing and ring-refresh
+ * kernels with the sequence's part of the ring.  A violation is recorded (device_status bit 3), the access is not made (a read
  * is redirected to the region's first bytes, a write is dropped), and the next ipkv_get_stats returns IPKV_EINTERNAL.
  * This self-test call (no counterpart in the paper) declares region base_id of the handle (0 resident ring of a layer,
  * 1 D-windows of a layer, 2 PP slots) to be only `bytes` long (0 restores the real extent): launches that reach

@@ -495,6 +495,16 @@ void note_kv_write(ipkv* h, int layer, bool inside_launch = false, bool window_o
     }
 }
 
+// Bounds-checked build: the host computes the destinations of the packing and ring-refresh kernels; a destination that
+// does not lie inside the part of the ring that belongs to (layer, seq) is an internal error and nothing is launched.
+ipkv_status check_ring_range(ipkv* h, int layer, int seq, const char* dst, int64_t bytes) {
+    if (!kChecked) return IPKV_OK;
+    const char* lo = h->ring_layer(layer) + h->ring_off(seq);
+    const char* hi = lo + h->ring_of(seq) * h->bb;
+    if (dst < lo || dst + bytes > hi) return fail(h, IPKV_EINTERNAL, "bounds-checked build: a ring destination left its sequence's part of the ring");
+    return IPKV_OK;
+}
+
 ipkv_status flush_layer(ipkv* h, int layer, const int* seqs_in, int n, cudaStream_t s) {
     note_kv_write(h, layer);
     const bool no_u = h->cfg.flags & IPKV_FLAG_NO_HOST_U, no_p = h->cfg.flags & IPKV_FLAG_NO_HOST_P;
@@ -574,6 +584,7 @@ ipkv_status flush_layer(ipkv* h, int layer, const int* seqs_in, int n, cudaStrea
                     while (j0 < j1) {
                         const int64_t pos = j0 % ring;
                         const int64_t cnt = std::min(j1 - j0, ring - pos);
+                        { ipkv_status crc = check_ring_range(h, layer, j.seq, base + pos * h->bb, cnt * h->bb); if (crc != IPKV_OK) return crc; }
                         spans.src[n_spans] = wsrc; spans.dst[n_spans] = base + pos * h->bb; spans.bytes[n_spans] = cnt * h->bb;
                         h->stats.d2d_bytes += uint64_t(cnt * h->bb);
                         if (++n_spans == kCopySpansPerLaunch) { ipkv_status rc = flush_spans(); if (rc != IPKV_OK) return rc; }
@@ -1058,6 +1069,8 @@ ipkv_status ipkv_append_bulk(ipkv_t* h, int32_t layer, int32_t seq, const void* 
                 const int64_t pos = (r.first_block + j) % ring;
                 j_end = std::min(nb, j + (ring - pos));
                 dst = h->ring_layer(layer) + h->ring_off(seq) + pos * h->bb;
+                rc = check_ring_range(h, layer, seq, dst, (j_end - j) * h->bb);
+                if (rc != IPKV_OK) return rc;
             } else {
                 if (!to_u && no_p) { j = first_resident; continue; }
                 rc = ensure_staging(h, stage_cap);

@@ -360,7 +360,7 @@ def test_two_engine_step_cpu_engine_plus_gpu_equals_unsplit(kind):
                       np.stack([w[0] for w in full]), np.stack([w[1] for w in full]), "two engines via ipkv_merge")
 
 
-@pytest.mark.parametrize("resident", [4096, 0, 320])
+@pytest.mark.parametrize("resident", [4096, 0, 320, (128, 2048)])
 def test_block_sparse_selection(resident):
     """Whole-block selection (Sec. 4.4): attention over the D-window plus an arbitrary set of P blocks equals the oracle
     over exactly those tokens, whether the blocks are device-resident, host-only (gathered and sent with one DMA per
@@ -371,7 +371,8 @@ def test_block_sparse_selection(resident):
     bt, D = 64, 64
     seqs, lens = [0, 1], {0: 1000, 1: 700}
     with make_cache(sh, 1, 2, block_tokens=bt, window_tokens=D, chunk_tokens=128, n_slots=2, max_u_tokens_per_seq=2000,
-                    max_p_tokens_per_seq=2000, resident_tokens_per_seq=resident, share_num=1, share_den=4) as cache:
+                    max_p_tokens_per_seq=2000, resident_tokens_per_seq=resident if isinstance(resident, int) else 64,
+                    resident_tokens_by_seq=None if isinstance(resident, int) else list(resident), share_num=1, share_den=4) as cache:
         refs = {}
         for s in seqs:
             r = RefSeq(sh, bt, D, 1, 4)
