@@ -326,6 +326,37 @@ def spawn_replicas(n, argv):
     return max(codes, key=abs) if any(codes) else 0
 
 
+def workload_config(name, wl):
+    """What the workload is, from its table entry alone: both arms print the same object for the same workload.
+    What a particular run chose (schedule, splits, timing cadence) goes under the line's "run" key instead."""
+    sh, B = wl["shape"], wl["batch"]
+    num0, den0 = wl["share"]
+    lens = seq_lens(wl)
+    n_cpu = sum(cpu_tokens(n, num0, den0) for n in lens) // B
+    n_gpu0 = sum(lens) // B - n_cpu
+    bpt = sh.bytes_per_token
+    # every layer reads its own KV, so one step sweeps all layers' bytes before a byte is read again
+    layer_bytes = sum(n - cpu_tokens(n, num0, den0) + 1 for n in lens) * bpt
+    step_bytes = layer_bytes * sh.n_layers
+    if step_bytes > 2 * (126 << 20):
+        l2_note = "inputs larger than L2 (each layer reads its own %.2f GB; %.2f GB per step)" % (layer_bytes / 1e9, step_bytes / 1e9)
+    else:
+        l2_note = "NOT flushed: the %.1f MB a step reads stay L2-resident between steps; a latency case, not a bandwidth number" % (step_bytes / 1e6)
+    gpu_share, copies = "HBM-resident", "off (benchmark)"
+    if wl.get("host_copies"):
+        copies = "on (P pinned, U unpinned); write-back on a copy stream"
+    if wl.get("grow_p"):
+        copies += "; P grown batch by batch, pinned one window ahead by a helper thread"
+    if "stream_pct" in wl:
+        gpu_share = "%d %% streamed H2D from pinned host memory each step, rest HBM-resident" % wl["stream_pct"]
+        copies = "P on (pinned), U off"
+    return {"workload": name, "layers": sh.n_layers, "batch": B,
+            "context": wl["ctx"] if "lens" not in wl else f"ragged {min(lens)}..{max(lens)} (sum {sum(lens)})",
+            "cpu_share": f"{num0}/{den0}", "gpu_share_tokens_per_seq_mean": n_gpu0 + 1, "bytes_per_kv_token": bpt,
+            "block_tokens": BLOCK, "window_tokens": wl.get("window", WINDOW), "gpu_share": gpu_share,
+            "host_copies_of_U_and_P": copies, "cpu_partial": "synthetic values", "l2": l2_note, "multi_gpu": "replicas only"}
+
+
 def run_reference(args, wl, name):
     """--impl reference: the oracle on the host cores, on the same workload and metric; each step is a bounded sample."""
     rank = int(os.environ.get("RANK", "0"))
@@ -345,7 +376,7 @@ def run_reference(args, wl, name):
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * n_tok / value, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": {"workload": name},
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": workload_config(name, wl),
         "cpu_baseline": info, "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
 
@@ -876,14 +907,6 @@ def main():
     if status != 0:
         raise RuntimeError("a kernel reported a timed-out wait; the numbers are invalid")
 
-    # every layer reads its own KV, so one step sweeps NL launches' worth of bytes before a byte is read again
-    step_bytes = bytes_attended / max(1, args.steps)
-    if step_bytes > 2 * (126 << 20):
-        l2_note = "inputs larger than L2 (each layer reads its own %.2f GB; %.2f GB per step)" % (
-            bytes_attended / max(1, n_launch) / 1e9, step_bytes / 1e9)
-    else:
-        l2_note = "NOT flushed: the %.1f MB a step reads stay L2-resident between steps; a latency case, not a bandwidth number" % (
-            step_bytes / 1e6)
     cpu = None
     others = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -899,16 +922,12 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": args.workload, "layers": NL, "batch": B,
-                       "context": ctx if "lens" not in wl else f"ragged {min(lens)}..{max(lens)} (sum {sum(lens)})",
-                       "cpu_share": f"{num0}/{den0}", "gpu_share_tokens_per_seq_mean": n_gpu0 + 1, "bytes_per_kv_token": bpt, "block_tokens": BLOCK, "window_tokens": wl.get("window", WINDOW),
-                       "gpu_share": "HBM-resident", "host_copies_of_U_and_P": "off (benchmark)", "cpu_partial": "synthetic values",
-                       "l2": l2_note,
-                       "multi_gpu": "replicas only", "kv_splits": args.kv_splits, "kernel_timing": "CUDA events around every %d%s attention launch" % (args.time_every, "th" if args.time_every != 1 else "st"), "schedule": "static" if args.static_schedule else "dynamic balancing (GQA kernel, launches long enough for it to pay: from 64 tiles per CTA)",
-                       "merge": "inside the split reduce" if fused else "separate ipkv_merge launch",
-                       "append": "separate ipkv_append" if args.separate_append else "inside ipkv_attend_gpu (written by the attention kernel for GQA)",
-                       "launch_overlap": "programmatic dependent launch; %d of %d attention launches started their copies before the previous kernel had completed"
-                                         % (st1["early_launches"] - st0["early_launches"], st1["attend_kernels"] - st0["attend_kernels"])},
+            "config": workload_config(args.workload, wl),
+            "run": {"kv_splits": args.kv_splits, "kernel_timing": "CUDA events around every %d%s attention launch" % (args.time_every, "th" if args.time_every != 1 else "st"), "schedule": "static" if args.static_schedule else "dynamic balancing (GQA kernel, launches long enough for it to pay: from 64 tiles per CTA)",
+                    "merge": "inside the split reduce" if fused else "separate ipkv_merge launch",
+                    "append": "separate ipkv_append" if args.separate_append else "inside ipkv_attend_gpu (written by the attention kernel for GQA)",
+                    "launch_overlap": "programmatic dependent launch; %d of %d attention launches started their copies before the previous kernel had completed"
+                                      % (st1["early_launches"] - st0["early_launches"], st1["attend_kernels"] - st0["attend_kernels"])},
             "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu,
             "step_gbs": bytes_all / (ms * 1e-3) / 1e9, "step_ms": step_ms,
         }
@@ -916,10 +935,7 @@ def main():
             line["step_latency"] = step_lat
         if others is not None:
             line["other_configs"] = others
-        if wl.get("host_copies"):
-            line["config"]["host_copies_of_U_and_P"] = "on (P pinned, U unpinned); write-back on a copy stream"
         if wl.get("grow_p"):
-            line["config"]["host_copies_of_U_and_P"] += "; P grown batch by batch, pinned one window ahead by a helper thread"
             line["p_growth"] = {k: st1[k] for k in ("p_segments", "p_pinned_bytes", "p_pin_us", "p_grow_waits", "p_grow_wait_us",
                                                        "p_register_us", "p_register_calls", "p_register_max_us")}
             line["p_growth"]["segments_pinned_in_timed_region"] = st1["p_segments"] - st0["p_segments"]
@@ -941,8 +957,6 @@ def main():
                                  "h2d_plateau_gbs": plateau, "attn_kernel_ms_per_step": kern_ms / args.steps,
                                  "overlap_efficiency": max(t_h2d_ideal, kern_ms) / ms,
                                  "streamed_pct_of_p_share": wl["stream_pct"], "chunk_tokens": wl.get("chunk_tokens", 512)}
-            line["config"]["gpu_share"] = "%d %% streamed H2D from pinned host memory each step, rest HBM-resident" % wl["stream_pct"]
-            line["config"]["host_copies_of_U_and_P"] = "P on (pinned), U off"
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

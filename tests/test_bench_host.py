@@ -26,6 +26,11 @@ def test_reference_arm_prints_one_json_line():
     assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] >= 1 and d["cpu_baseline"]["value"] == d["value"]
     assert d["e2e"] == {"value": d["value"], "unit": "KV-tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
     assert d["config"]["workload"] == "small-gqa-bs1-4k-cpu50" and d["vs_baseline"] is None
+    # both arms describe the workload with the same object, made from the workload's table entry alone
+    sys.path.insert(0, ROOT)
+    import bench
+    assert d["config"] == bench.workload_config("small-gqa-bs1-4k-cpu50", bench.WORKLOADS["small-gqa-bs1-4k-cpu50"])
+    assert d["config"]["layers"] >= 1 and "l2" in d["config"]
 
 
 def test_reference_arm_other_ranks_exit_quietly():
