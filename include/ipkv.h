@@ -172,7 +172,9 @@ ipkv_status ipkv_flush(ipkv_t* h, int32_t layer, int32_t seq, void* stream);
  * the library's own kernels and behind the caller's.  An attention launch whose K/V bytes the library knows to be
  * settled (nothing it enqueued since the launch before the previous one wrote them) also starts its first copies
  * before that wait.  The environment variables IPKV_NO_LAUNCH_OVERLAP and IPKV_NO_EARLY_COPIES (any value, read once
- * per process) restore plain launches / switch the early copies off. */
+ * per process) restore plain launches / switch the early copies off.  IPKV_PARTS_PER_SPAN=1 or 4 (a test hook, read
+ * once) fixes how many partials the grouped-query kernel writes per span (1: its warps join their states first), which
+ * the library otherwise chooses per launch by the length of the spans; the results agree within rounding. */
 
 typedef struct {
   int32_t kv_splits;   /* 0 = automatic; otherwise the number of sequence chunks per (sequence, KV head) */

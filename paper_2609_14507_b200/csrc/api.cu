@@ -722,7 +722,12 @@ void fill_launch(AttnLaunch* a, int kind, int Hq, int Hkv, int dqk, int dv, int 
     a->n_ctas = plan.n_ctas();
     a->n_rows = n_rows;
     a->n_gh = pg.n_gh;
-    const size_t rows = (plan.spans.size() + extra_partials) * size_t(pg.parts_per_span) * pg.rows_per_group;
+    int64_t tiles = 0;
+    for (const Span& sp : plan.spans) tiles += sp.ntiles;
+    a->parts_per_span = parts_per_span_for(kind, tiles, int64_t(plan.spans.size()));
+    static const int forced_parts = [] { const char* e = std::getenv("IPKV_PARTS_PER_SPAN"); return e ? std::atoi(e) : 0; }();
+    if (kind != 1 && (forced_parts == 1 || forced_parts == 4)) a->parts_per_span = forced_parts;     // test hook
+    const size_t rows = (plan.spans.size() + extra_partials) * size_t(a->parts_per_span) * pg.rows_per_group;
     a->part_rows = int64_t(rows);
     a->part_o = reinterpret_cast<float*>(partials);
     a->part_lse = reinterpret_cast<float*>(partials + align_up(rows * dv * sizeof(float), 256));
@@ -831,8 +836,8 @@ ipkv_status run_group(ipkv* h, std::vector<std::vector<PlanSeg>>& rows, const ch
         if (timed) CU(h, cudaEventRecord(h->prof_ev[h->prof_used], s));
         CU(h, launch_split_reduce(a, s));
         if (timed) { CU(h, cudaEventRecord(h->prof_ev[h->prof_used + 1], s)); h->prof_used += 2; }
+        h->stats.reduce_kernels += 1;
     }
-    h->stats.reduce_kernels += 1;
     h->stats.kv_bytes_attended += uint64_t(total_tokens) * uint64_t(h->bb / c.block_tokens);
     return IPKV_OK;
 }

@@ -12,9 +12,10 @@
 // Four consumer warps each own 16 tokens of every tile and run a private flash-decoding stream: query
 // fragments in registers (the G query heads that share the KV head are the M rows of the tensor-core MMA,
 // so one K/V read serves the whole group), K fragments by ldmatrix, V fragments by ldmatrix.trans, fp32
-// online softmax and fp32 output accumulators in registers.  Nothing synchronises the CTA per tile or per
-// span: at the end of a span every warp writes its own normalised partial (O, natural-log LSE) and the
-// LSE reduce joins the partials of all spans and warps of a (row, head).
+// online softmax and fp32 output accumulators in registers.  Nothing synchronises the CTA per tile.  At the
+// end of a span the four warps either write a normalised partial (O, natural-log LSE) each, or, in launches
+// whose spans are long (the host decides, plan.hpp), join their states through shared memory into one; the
+// LSE reduce joins the partials of all spans of a (row, head).
 //
 // Tiles are handed to the CTAs either in plan order or, by default for launches that are long enough, by the dynamic
 // balancing of schedule.cuh (CTAs that finish early take over tiles of the ones that are behind).
@@ -60,6 +61,7 @@ struct GqaParams {
     int early;          // nonzero: the producer may issue its first copies of ring tiles (2: of window tiles too) before the
                         // previous kernel of the stream has completed
     int Hq, G, n_hg, RG;
+    int NW;             // partials per span: 1 = the consumer warps join their states at the end of a span, 4 = each writes its own
     int bt;
     int64_t head_bytes, block_bytes;
     float scale_log2;
@@ -68,19 +70,25 @@ struct GqaParams {
     int64_t part_rows;               // bounds-checked build: rows of partial storage
 };
 
-template <int D, int STAGES>
+template <int D, int STAGES, int ROWS>
 struct SmemPlan {
     static constexpr int kPlane = D * 128;               // bytes of a 64-token K (or V) tile
     static constexpr int kStage = 2 * kPlane;
     static constexpr int kStagesBytes = STAGES * kStage;
     static constexpr int kBarOff = kStagesBytes;
     static constexpr int kMetaOff = kBarOff + 2 * STAGES * 8;     // one StageMeta (32 bytes) per stage
-    static constexpr int kTotal = kMetaOff + STAGES * 32;
+    // joining the four consumer warps' states at the end of a partial: a give-up flag, every warp's (max, sum) per
+    // query row, and one buffer of output rows (padded: rows 0..3 on distinct banks)
+    static constexpr int kFlagOff = kMetaOff + STAGES * 32;
+    static constexpr int kMlOff = kFlagOff + 16;
+    static constexpr int kRowPitch = D + 8;              // floats
+    static constexpr int kObufOff = kMlOff + 2 * kConsumerWarps * 16 * 4;
+    static constexpr int kTotal = kObufOff + ROWS * kRowPitch * 4;
 };
 
 template <int D, int STAGES, bool DUP>
 __global__ void __launch_bounds__(kThreads, 2) attn_gqa_kernel(const GqaParams p) {
-    using SP = SmemPlan<D, STAGES>;
+    using SP = SmemPlan<D, STAGES, DUP ? 8 : 16>;
     extern __shared__ unsigned char smem_dyn[];
     // align the ring to 1024 bytes so that the 128-byte chunk swizzle maps onto distinct banks
     unsigned char* smem = smem_dyn + ((1024u - (ptx::smem_addr(smem_dyn) & 1023u)) & 1023u);
@@ -88,6 +96,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_gqa_kernel(const GqaParams p
     const uint32_t s_full = s_base + SP::kBarOff;
     const uint32_t s_empty = s_full + STAGES * 8;
     volatile StageMeta* s_meta = reinterpret_cast<volatile StageMeta*>(smem + SP::kMetaOff);
+    volatile int* s_gave_up = reinterpret_cast<volatile int*>(smem + SP::kFlagOff);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int span_begin = p.cta_span_start[blockIdx.x], span_end = p.cta_span_start[blockIdx.x + 1];
@@ -98,6 +107,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_gqa_kernel(const GqaParams p
             ptx::mbar_init(s_full + 8 * s, 1);
             ptx::mbar_init(s_empty + 8 * s, kConsumerWarps);
         }
+        *s_gave_up = 0;
         ptx::mbar_fence_init();
     }
     if (p.bt < kTileTokens) {
@@ -212,7 +222,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_gqa_kernel(const GqaParams p
             sched.spans = p.spans; sched.cta_span_start = p.cta_span_start; sched.cta_tiles = p.cta_tiles;
             sched.next = p.next; sched.lists = p.lists; sched.part_lse = p.part_lse;
             sched.n_spans = p.n_spans; sched.n_ctas = p.n_ctas; sched.n_rows = p.n_rows; sched.n_gh = p.n_gh;
-            sched.lse_per_partial = kConsumerWarps * p.RG;
+            sched.lse_per_partial = p.NW * p.RG;
             sched.head_tiles = (early && dynamic) ? STAGES : 0;
             ok = produce_tiles(sched, lane, issue, [&]() { if (!waited) { ptx::grid_dependency_wait(); waited = true; } });
             if (lane == 0) {
@@ -251,8 +261,8 @@ __global__ void __launch_bounds__(kThreads, 2) attn_gqa_kernel(const GqaParams p
 
     if (dynamic) {
         // a span of this CTA's chunk may be taken over completely by other CTAs: its partial then stays empty
-        for (int sp = span_begin; sp < span_end; ++sp) {
-            const int64_t prow = (int64_t(sp) * kConsumerWarps + warp) * p.RG;
+        for (int i = (span_begin * p.NW + warp); i < span_end * p.NW; i += kConsumerWarps) {
+            const int64_t prow = int64_t(i) * p.RG;
             if ((lane & 3) == 0) {
                 if (r0 < p.RG) p.part_lse[prow + r0] = -INFINITY;
                 if (!DUP && r0 + 8 < p.RG) p.part_lse[prow + r0 + 8] = -INFINITY;
@@ -265,36 +275,133 @@ __global__ void __launch_bounds__(kThreads, 2) attn_gqa_kernel(const GqaParams p
     float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
     int cur_slot = kEndSlot, n_heads = 0;
 
-    // this warp's normalised partial of the tiles accumulated so far (rows = the group's query heads)
-    auto flush = [&]() {
+    // A barrier among the four consumer warps (they run privately otherwise).  It is a hardware barrier, which has no
+    // limit of its own; what bounds it is the order of events.  The four warps wait for the same tiles.  A warp comes here
+    // only after a tile has arrived that the others wait for as well, each with a limit that started no earlier than this
+    // warp's: they get the tile too and follow.  A warp that gave up did so before that tile arrived, and said so in shared
+    // memory before it left: whoever comes here afterwards sees the flag and leaves as well instead of waiting.
+    auto consumer_sync = [&]() -> bool {
+        __syncwarp();
+        if (*s_gave_up) return false;
+        asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory");
+        return true;
+    };
+
+    // The partial of the tiles accumulated so far: the four warps' private states (each over its 16 tokens of every tile)
+    // joined into one normalised (O, LSE) per query head (Sec. 5.1's identity, in the log2 domain), so that the split reduce
+    // reads one partial per span.  Warp w scales its accumulators by exp2(m_w - M) / L; warp 0 stores its rows into the
+    // buffer, warps 1 and 2 add theirs in turn, warp 3 adds its own to the buffer's and writes the result out.
+    auto flush = [&]() -> bool {
         l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
         l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
         if (!DUP) {
             l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
             l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
         }
-        const int64_t prow = (int64_t(cur_slot) * kConsumerWarps + warp) * p.RG;
-        if (kChecked && (prow < 0 || prow + p.RG > p.part_rows)) {    // the partial's rows must lie inside the scratch
-            if (lane == 0) atomicOr(p.status, kStatusBadIndex);
-            return;
-        }
-        if (r0 < n_heads) {
-            const float inv = l0 > 0.f ? 1.f / l0 : 0.f;
-            float* dst = p.part_o + (prow + r0) * D + c0;
-#pragma unroll
-            for (int nt = 0; nt < D / 8; ++nt) {
-                const float x = DUP ? o[nt][0] + o[nt][2] : o[nt][0], y = DUP ? o[nt][1] + o[nt][3] : o[nt][1];
-                *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(x * inv, y * inv);
+        if (p.NW != 1) {
+            // every warp writes its own normalised partial: nothing is exchanged, the reduce reads four entries per span
+            const int64_t prow = (int64_t(cur_slot) * kConsumerWarps + warp) * p.RG;
+            if (kChecked && (prow < 0 || prow + p.RG > p.part_rows)) {    // the partial's rows must lie inside the scratch
+                if (lane == 0) atomicOr(p.status, kStatusBadIndex);
+                return true;
             }
-            if ((lane & 3) == 0) p.part_lse[prow + r0] = (m0 == -INFINITY) ? -INFINITY : (m0 + log2f(l0)) * kLn2;
-        }
-        if (!DUP && r0 + 8 < n_heads) {
-            const float inv = l1 > 0.f ? 1.f / l1 : 0.f;
-            float* dst = p.part_o + (prow + r0 + 8) * D + c0;
+            if (r0 < n_heads) {
+                const float inv = l0 > 0.f ? 1.f / l0 : 0.f;
+                float* dst = p.part_o + (prow + r0) * D + c0;
 #pragma unroll
-            for (int nt = 0; nt < D / 8; ++nt) *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(o[nt][2] * inv, o[nt][3] * inv);
-            if ((lane & 3) == 0) p.part_lse[prow + r0 + 8] = (m1 == -INFINITY) ? -INFINITY : (m1 + log2f(l1)) * kLn2;
+                for (int nt = 0; nt < D / 8; ++nt) {
+                    const float x = DUP ? o[nt][0] + o[nt][2] : o[nt][0], y = DUP ? o[nt][1] + o[nt][3] : o[nt][1];
+                    *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(x * inv, y * inv);
+                }
+                if ((lane & 3) == 0) p.part_lse[prow + r0] = (m0 == -INFINITY) ? -INFINITY : (m0 + log2f(l0)) * kLn2;
+            }
+            if (!DUP && r0 + 8 < n_heads) {
+                const float inv = l1 > 0.f ? 1.f / l1 : 0.f;
+                float* dst = p.part_o + (prow + r0 + 8) * D + c0;
+#pragma unroll
+                for (int nt = 0; nt < D / 8; ++nt) *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(o[nt][2] * inv, o[nt][3] * inv);
+                if ((lane & 3) == 0) p.part_lse[prow + r0 + 8] = (m1 == -INFINITY) ? -INFINITY : (m1 + log2f(l1)) * kLn2;
+            }
+            return true;
         }
+        const uint32_t s_m = s_base + SP::kMlOff, s_l = s_m + kConsumerWarps * 16 * 4;
+        if ((lane & 3) == 0) {
+            ptx::sts_f(s_m + (warp * 16 + r0) * 4, m0); ptx::sts_f(s_l + (warp * 16 + r0) * 4, l0);
+            if (!DUP) { ptx::sts_f(s_m + (warp * 16 + r0 + 8) * 4, m1); ptx::sts_f(s_l + (warp * 16 + r0 + 8) * 4, l1); }
+        }
+        if (!consumer_sync()) return false;
+        float mw0[kConsumerWarps], lw0[kConsumerWarps], mw1[kConsumerWarps], lw1[kConsumerWarps];
+#pragma unroll
+        for (int w = 0; w < kConsumerWarps; ++w) {
+            mw0[w] = ptx::lds_f(s_m + (w * 16 + r0) * 4); lw0[w] = ptx::lds_f(s_l + (w * 16 + r0) * 4);
+            if (!DUP) { mw1[w] = ptx::lds_f(s_m + (w * 16 + r0 + 8) * 4); lw1[w] = ptx::lds_f(s_l + (w * 16 + r0 + 8) * 4); }
+        }
+        float M0 = -INFINITY, M1 = -INFINITY, L0 = 0.f, L1 = 0.f;
+#pragma unroll
+        for (int w = 0; w < kConsumerWarps; ++w) {
+            M0 = fmaxf(M0, mw0[w]);
+            if (!DUP) M1 = fmaxf(M1, mw1[w]);
+        }
+#pragma unroll
+        for (int w = 0; w < kConsumerWarps; ++w) {
+            if (mw0[w] != -INFINITY) L0 += ptx::ex2(mw0[w] - M0) * lw0[w];
+            if (!DUP && mw1[w] != -INFINITY) L1 += ptx::ex2(mw1[w] - M1) * lw1[w];
+        }
+        const float f0 = (m0 != -INFINITY && L0 > 0.f) ? ptx::ex2(m0 - M0) / L0 : 0.f;
+        const float f1 = (!DUP && m1 != -INFINITY && L1 > 0.f) ? ptx::ex2(m1 - M1) / L1 : 0.f;
+        const uint32_t buf0 = s_base + SP::kObufOff + (r0 * SP::kRowPitch + c0) * 4;
+        const uint32_t buf1 = buf0 + 8 * SP::kRowPitch * 4;
+        const int64_t prow = int64_t(cur_slot) * p.RG;
+        const bool rows_ok = !(kChecked && (prow < 0 || prow + p.RG > p.part_rows));   // the partial's rows must lie inside the scratch
+        if (!rows_ok && warp == kConsumerWarps - 1 && lane == 0) atomicOr(p.status, kStatusBadIndex);
+        const bool v0 = r0 < n_heads, v1 = !DUP && (r0 + 8 < n_heads);
+        // this warp's scaled rows (in place: the accumulators are started afresh after a flush)
+#pragma unroll
+        for (int nt = 0; nt < D / 8; ++nt) {
+            o[nt][0] = (DUP ? o[nt][0] + o[nt][2] : o[nt][0]) * f0;
+            o[nt][1] = (DUP ? o[nt][1] + o[nt][3] : o[nt][1]) * f0;
+            if (!DUP) { o[nt][2] *= f1; o[nt][3] *= f1; }
+        }
+#pragma unroll 1
+        for (int turn = 0; turn < kConsumerWarps; ++turn) {
+            if (warp == turn) {
+                if (turn > 0) {                    // the rows so far: all loads first, then the sums
+                    float2 b0[D / 8], b1[D / 8];
+#pragma unroll
+                    for (int nt = 0; nt < D / 8; ++nt) {
+                        b0[nt] = ptx::lds_f2(buf0 + nt * 32);
+                        if (!DUP) b1[nt] = ptx::lds_f2(buf1 + nt * 32);
+                    }
+#pragma unroll
+                    for (int nt = 0; nt < D / 8; ++nt) {
+                        o[nt][0] += b0[nt].x; o[nt][1] += b0[nt].y;
+                        if (!DUP) { o[nt][2] += b1[nt].x; o[nt][3] += b1[nt].y; }
+                    }
+                }
+                if (turn + 1 < kConsumerWarps) {
+#pragma unroll
+                    for (int nt = 0; nt < D / 8; ++nt) {
+                        ptx::sts_f2(buf0 + nt * 32, o[nt][0], o[nt][1]);
+                        if (!DUP) ptx::sts_f2(buf1 + nt * 32, o[nt][2], o[nt][3]);
+                    }
+                } else if (rows_ok) {
+                    if (v0) {
+                        float* dst = p.part_o + (prow + r0) * D + c0;
+#pragma unroll
+                        for (int nt = 0; nt < D / 8; ++nt) *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(o[nt][0], o[nt][1]);
+                        if ((lane & 3) == 0) p.part_lse[prow + r0] = (M0 == -INFINITY) ? -INFINITY : (M0 + log2f(L0)) * kLn2;
+                    }
+                    if (v1) {
+                        float* dst = p.part_o + (prow + r0 + 8) * D + c0;
+#pragma unroll
+                        for (int nt = 0; nt < D / 8; ++nt) *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(o[nt][2], o[nt][3]);
+                        if ((lane & 3) == 0) p.part_lse[prow + r0 + 8] = (M1 == -INFINITY) ? -INFINITY : (M1 + log2f(L1)) * kLn2;
+                    }
+                }
+            }
+            if (turn + 1 < kConsumerWarps && !consumer_sync()) return false;
+        }
+        return true;
     };
 
     // start a partial: query fragments of its head group straight from global memory (a few KB, L2-resident), empty state
@@ -328,10 +435,10 @@ __global__ void __launch_bounds__(kThreads, 2) attn_gqa_kernel(const GqaParams p
 
     for (;; ++it) {
         const int st = it % STAGES;
-        if (!ptx::mbar_wait(s_full + 8 * st, (it / STAGES) & 1)) { ok = false; break; }   // after a timeout: give up
+        if (!ptx::mbar_wait(s_full + 8 * st, (it / STAGES) & 1)) { ok = false; *s_gave_up = 1; break; }   // after a timeout: give up
         const int slot = s_meta[st].slot;
         if (slot != cur_slot) {
-            if (cur_slot != kEndSlot) flush();
+            if (cur_slot != kEndSlot && !flush()) { ok = false; break; }
             if (slot == kEndSlot) break;
             cur_slot = slot;
             begin_partial(s_meta[st].q_row, s_meta[st].n_heads);
@@ -441,12 +548,16 @@ __global__ void __launch_bounds__(kThreads, 2) attn_gqa_kernel(const GqaParams p
             if (lane == 0) ptx::mbar_arrive(s_empty + 8 * st);
         }
     }
-    if (!ok && lane == 0) atomicOr(p.status, kStatusNoTile);
+    if (!ok) {
+        *s_gave_up = 1;
+        if (lane == 0) atomicOr(p.status, kStatusNoTile);
+        return;
+    }
 }
 
 template <int D, int STAGES, bool DUP>
 cudaError_t launch_gqa(const AttnLaunch& a, cudaStream_t s) {
-    using SP = SmemPlan<D, STAGES>;
+    using SP = SmemPlan<D, STAGES, DUP ? 8 : 16>;
     GqaParams p;
     p.q = static_cast<const __nv_bfloat16*>(a.q);
     for (int i = 0; i < kMaxBases; ++i) p.bases[i] = a.bases[i];
@@ -462,6 +573,7 @@ cudaError_t launch_gqa(const AttnLaunch& a, cudaStream_t s) {
     p.Hq = a.n_q_heads; p.G = a.n_q_heads / a.n_kv_heads;
     p.n_hg = (p.G + 15) / 16;
     p.RG = part_geom(0, a.n_q_heads, a.n_kv_heads).rows_per_group;
+    p.NW = a.parts_per_span == 1 ? 1 : kConsumerWarps;
     p.bt = a.bt;
     p.head_bytes = int64_t(a.bt) * (a.dim_qk + a.dim_v) * 2;
     p.block_bytes = p.head_bytes * a.n_kv_heads;

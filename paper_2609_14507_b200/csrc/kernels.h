@@ -73,6 +73,7 @@ struct AttnLaunch {
     const void* append_v;           // [n_rows][n_kv_heads][dim_v]
     int64_t base_bytes[kMaxBases];  // extent of the memory behind every base (0: unknown, not checked); used by the checked build
     int64_t part_rows;              // rows of (O, LSE) partial storage behind part_o / part_lse
+    int parts_per_span;             // partials every span writes in this launch (plan.hpp: parts_per_span_for)
     int win_tail;                   // valid tokens in the last tile of the runs flagged kSegTailParam (1..64)
     int plain_launch;               // 1: the tables were written by the kernel right in front of this launch: no launch overlap
     int early_tiles;                // nonzero: no ring byte this launch reads (2: no window byte either) was written by the kernel
@@ -92,7 +93,7 @@ constexpr int kStealSlots = 4;      // extra partials a CTA can fill
 constexpr int kStealListCap = 16;   // extra partials a (row, head group) can take
 
 // Geometry of the partial buffers: query heads per head group (rows of one partial), head groups per row,
-// partials per span (one per consumer warp for GQA, one for MLA), resident CTAs per SM.
+// partials per span at most (sizes the scratch; one per consumer warp for GQA unless the launch joins them, one for MLA), resident CTAs per SM.
 struct PartGeom {
     int rows_per_group, n_gh, parts_per_span, ctas_per_sm;
 };
@@ -110,7 +111,7 @@ inline PartGeom part_geom(int kind, int Hq, int Hkv) {
     return g;
 }
 
-// Split-K attention: partial (O, LSE) per span (and consumer warp), rows = the query heads of the span's group.
+// Split-K attention: partial (O, LSE) per span, rows = the query heads of the span's group.
 cudaError_t launch_attend(const AttnLaunch& a, cudaStream_t s);
 // Second pass: per (row, head) LSE-reduce the partials of its head group's spans (and acc_*, if given) into out_*.
 cudaError_t launch_split_reduce(const AttnLaunch& a, cudaStream_t s);

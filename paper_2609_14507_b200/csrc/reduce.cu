@@ -237,7 +237,7 @@ cudaError_t launch_split_reduce(const AttnLaunch& a, cudaStream_t s) {
     p.Hq = a.n_q_heads; p.dv = a.dim_v;
     p.G = a.kind == 1 ? a.n_q_heads : a.n_q_heads / a.n_kv_heads;
     p.n_hg = (p.G + 15) / 16;
-    p.n_gh = pg.n_gh; p.RG = pg.rows_per_group; p.NW = pg.parts_per_span;
+    p.n_gh = pg.n_gh; p.RG = pg.rows_per_group; p.NW = a.parts_per_span;
     p.dvl = a.dim_v > 128 && a.dim_v % 128 == 0 ? 128 : a.dim_v;
     p.CS = a.dim_v / p.dvl;
     if (p.dvl % 4 != 0 || p.dvl / 4 > 128 || 128 % (p.dvl / 4) != 0) return cudaErrorInvalidValue;

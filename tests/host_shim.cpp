@@ -111,6 +111,18 @@ int64_t shim_ring_slots(int n_seqs, int64_t uniform_tokens, const int64_t* token
 }
 
 // Two consecutive decode steps of a batch: window runs of `fill` and `fill + 1` tokens behind a resident run each.
+// Partials per span of a launch whose rows hold `tokens[r]` tokens each (one run per row): the rule of plan.hpp applied to
+// the plan that is actually built.
+int shim_parts_per_span(int kind, int n_rows, const int64_t* tokens, int n_gh, int ctas_per_sm) {
+    std::vector<std::vector<PlanSeg>> rows(n_rows);
+    for (int r = 0; r < n_rows; ++r) rows[r].push_back(PlanSeg{0, int64_t(r) << 26, tokens[r]});
+    Plan plan;
+    build_plan(rows, n_gh, 0, ctas_per_sm, &plan);
+    int64_t tiles = 0;
+    for (const Span& sp : plan.spans) tiles += sp.ntiles;
+    return parts_per_span_for(kind, tiles, int64_t(plan.spans.size()));
+}
+
 // Returns the launch parameter win_tail of the first step and, in *same_table, whether the two steps' serialised launch
 // tables are byte-identical (they must be, unless a window grows into a new tile, when the plan itself changes).
 int shim_window_tail(int n_rows, const int64_t* resident_tokens, const int64_t* window_fill, int n_gh, int ctas_per_sm, int* same_table,

@@ -217,6 +217,25 @@ def test_bounds_checked_build_passes_the_small_parity_cases():
     assert " passed" in r.stdout and "skipped" not in r.stdout.splitlines()[-1]
 
 
+@pytest.mark.parametrize("parts", ["1", "4"])
+def test_both_forms_of_the_span_partial_pass_the_small_parity_cases(parts):
+    """The grouped-query kernel writes one partial per span (its four warps join their states through shared memory) in
+    launches with long spans and four otherwise; small cases would only ever see the second form.  Here each form is
+    forced in turn (IPKV_PARTS_PER_SPAN, read when the library is first used: a child process) and the small-shape parity
+    tests, ragged and balanced cases and the decode tests run against it."""
+    import os
+    import subprocess
+    import sys
+    env = dict(os.environ, IPKV_PARTS_PER_SPAN=parts)
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run([sys.executable, "-m", "pytest", "-q", "-m", "gpu", "-x", os.path.join(root, "tests", "test_gpu_kernels.py"),
+                        os.path.join(root, "tests", "test_gpu_cache.py"), "-k",
+                        "attend_runs_gqa or peaked or identical or config1 or decode_steps or fused or static_schedule or balanc or sparse"],
+                       env=env, cwd=root, capture_output=True, text=True, timeout=900)
+    assert r.returncode == 0, r.stdout[-3000:] + r.stderr[-2000:]
+    assert " passed" in r.stdout
+
+
 def test_read_bandwidth_probe_runs():
     """The measurement aid behind `roofline.read_ceiling`: a read-only stream through the kernels' copy ring."""
     best, mean = binding.ipkv_probe_read_bandwidth(0, 256 << 20, 3)

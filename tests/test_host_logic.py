@@ -293,3 +293,22 @@ def test_window_fill_travels_as_a_launch_parameter_while_the_batch_is_in_lockste
     t, nxt, same = two_steps([8192, 8192], [5, 6])
     assert (t, nxt, same) == (0, 0, False)                                     # windows out of step: exact counts, tables differ
     assert two_steps([0, 8192], [17, 17], n_gh=1, cps=1) == (17, 18, True)     # a row with nothing but its window
+
+
+def test_consumer_warps_join_their_partials_only_in_launches_with_long_spans():
+    """The grouped-query kernel writes one partial per span (its four warps join their states first) when the launch's
+    spans are long, four when they are short; the compressed-latent kernel always writes one."""
+    L = host_shim.lib()
+    i64 = C.c_int64
+    L.shim_parts_per_span.restype = C.c_int
+    L.shim_parts_per_span.argtypes = [C.c_int, C.c_int, C.POINTER(i64), C.c_int, C.c_int]
+
+    def parts(kind, tokens, n_gh, cps):
+        return L.shim_parts_per_span(kind, len(tokens), (i64 * len(tokens))(*tokens), n_gh, cps)
+
+    assert parts(0, [24577] * 16, 8, 2) == 1            # Mixtral shape at a quarter on the CPU: 116 tiles per span
+    assert parts(0, [32769] * 16, 4, 2) == 1            # Qwen3 shape, everything on the GPU
+    assert parts(0, [9831] * 16, 4, 2) == 4             # the same at 70 % on the CPU: 24 tiles per span
+    assert parts(0, [4097], 4, 2) == 4                  # one short sequence: one tile per CTA
+    assert parts(0, [100, 1], 4, 2) == 4
+    assert parts(1, [78644] * 8, 1, 1) == 1 and parts(1, [100], 1, 1) == 1
