@@ -56,10 +56,10 @@ WORKLOADS = {
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention-kernel launch, read from one ncu capture per kernel
 # (taken on the 2-layer case of each shape, whose per-layer launch is the full-size workload's launch): read + write bytes.
 DRAM_TRAFFIC_PER_LAUNCH = {
-    "mixtral-8x7b-bs16-32k-cpu25": 1615.2e6 + 5.3e6,
-    "mixtral-2layers-bs16-32k-cpu25": 1615.2e6 + 5.3e6,
-    "qwen3-30b-a3b-bs16-32k-cpu0": 1076.1e6 + 4.6e6,
-    "qwen3-2layers-bs16-32k-cpu0": 1076.1e6 + 4.6e6,
+    "mixtral-8x7b-bs16-32k-cpu25": 1615.2e6 + 4.5e6,
+    "mixtral-2layers-bs16-32k-cpu25": 1615.2e6 + 4.5e6,
+    "qwen3-30b-a3b-bs16-32k-cpu0": 1076.1e6 + 3.9e6,
+    "qwen3-2layers-bs16-32k-cpu0": 1076.1e6 + 3.9e6,
     "deepseek-v2-lite-mla-bs8-128k-cpu40": 725.7e6 + 4.1e6,
     "deepseek-v2-lite-mla-2layers-bs8-128k-cpu40": 725.7e6 + 4.1e6,
 }
