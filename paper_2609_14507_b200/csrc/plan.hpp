@@ -79,10 +79,11 @@ struct Plan {
 // as one launch parameter (kSegTailParam); returns that offset (1..64), or 0 when the runs disagree or there are none.
 // How many partials a span writes.  The grouped-query kernel's four consumer warps run privately; at the end of a span they
 // either write a partial each, or join their states first (about a microsecond in which the CTA streams nothing, for a
-// reduce that reads a quarter of the entries).  Joining pays when spans are long.  Measured per layer: +0.9 % on spans of
-// 116 tiles (Mixtral shape, batch 16, 24K tokens), nothing on 24 (Qwen3 shape, 9.8K tokens), -2.3 % on 17 (ragged batch of
-// 64 at a tenth of its tokens).  The compressed-latent kernel's consumer warps share one state: one partial.
-constexpr int64_t kJoinWarpsFromTilesPerSpan = 32;
+// reduce that reads a quarter of the entries).  Joining pays when spans are long.  Measured per step, joined against not,
+// by mean tiles per span: 116 (Mixtral shape, batch 16, 24K tokens) +0.7 %; 91 / 64 / 45 / 24 (Qwen3 shape, 32K tokens at CPU
+// shares 0 / 30 / 50 / 70 %) +1.5 / +1.4 / +0.5 / 0 %; 81 / 57 / 40 / 24 / 17 (ragged batch of 64 at shares 0 / 30 / 50 / 70 /
+// 90 %) +1.5 / +1.5 / -0.4 / -0.5 / -2.3 %.  The compressed-latent kernel's consumer warps share one state: one partial.
+constexpr int64_t kJoinWarpsFromTilesPerSpan = 48;
 inline int parts_per_span_for(int kind, int64_t tiles, int64_t spans) {
     if (kind == 1) return 1;
     return (spans > 0 && tiles >= kJoinWarpsFromTilesPerSpan * spans) ? 1 : 4;
