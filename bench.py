@@ -771,7 +771,12 @@ def main():
     cache.profile_enable(not args.no_kernel_timing, reduce=args.profile_reduce, every=args.time_every)
     cache.profile_read()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]       # one event per step: medians and tails
+    # One event per step gives medians and tails.  An event between two launches keeps the second from starting under the
+    # first one's tail, which a step of a few hundred microseconds does not notice; a step of a dozen (the small L2-resident
+    # case: 12 us back to back, 18 with a mark per step) is timed without them unless --latency asks for the distribution.
+    step_bytes_static = sum(n - cpu_tokens(n, num0, den0) + 1 for n in lens) * bpt * NL
+    with_marks = args.latency or step_bytes_static > 2 * (126 << 20)
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)] if with_marks else []
     e0.record()
     for i in range(args.steps):
         if marks:
@@ -782,9 +787,9 @@ def main():
     e1.record()
     barrier()
     ms = max_over_ranks(e0.elapsed_time(e1))
-    raw = [marks[i].elapsed_time(marks[i + 1]) for i in range(args.steps)]
+    raw = [marks[i].elapsed_time(marks[i + 1]) for i in range(args.steps)] if marks else [ms / args.steps]
     lat = sorted(raw)
-    step_ms = {"median": lat[len(lat) // 2], "best": lat[0]}
+    step_ms = {"median": lat[len(lat) // 2], "best": lat[0]} if marks else {"median": None, "best": None, "note": "no per-step events on a step this short"}
     step_lat = None
     if args.latency:
         slowest = sorted(range(args.steps), key=lambda i: -raw[i])[:4]
