@@ -645,7 +645,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--kv-splits", type=int, default=0)
     ap.add_argument("--no-read-ceiling", action="store_true", help="skip the read-only bandwidth probe reported in roofline.read_ceiling")
-    ap.add_argument("--time-every", type=int, default=13,
+    ap.add_argument("--time-every", type=int, default=53,
                     help="CUDA events around every N-th attention launch of the timed region (every launch does the same work; an event "
                          "between two kernels costs the step several microseconds, so bracketing all of them would slow what is measured)")
     ap.add_argument("--no-kernel-timing", action="store_true",
