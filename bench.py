@@ -766,8 +766,8 @@ def main():
         step()
     barrier()
     st0 = cache.get_stats()
-    # short runs bracket more of their launches, so that at least about two dozen are timed
-    args.time_every = max(1, min(args.time_every, args.steps * sh.n_layers // 24))
+    # short runs bracket more of their launches, so that at least a dozen are timed
+    args.time_every = max(1, min(args.time_every, args.steps * sh.n_layers // 12))
     cache.profile_enable(not args.no_kernel_timing, reduce=args.profile_reduce, every=args.time_every)
     cache.profile_read()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
