@@ -44,9 +44,9 @@ struct ReduceParams {
 // EXTRAS: the launch was dynamically balanced and may have extra partials (kept out of the plain instantiation, which
 // then needs few enough registers for five CTAs per SM: launches with thousands of (row, head) pairs run in fewer waves).
 // THREADS: 256, or 128 for launches with so many (row, head) pairs that 256-thread CTAs would need several waves (a
-// ragged batch of 64 sequences x 32 heads: 2048 CTAs, at five per SM 2.8 waves, measured 10.4 us; with 128 threads all
-// of them are resident at once; squeezing them to 32 registers so that 14 or 16 fit an SM spills, and was slower: 2.225 ->
-// 2.269 ms per step).
+// ragged batch of 64 sequences x 32 heads: 2048 CTAs, at five per SM 2.8 waves, measured 10.4 us; with 128 threads ten
+// fit an SM, 1.4 waves, 7.3 us; squeezing them to 32 registers so that 14 or 16 fit, one wave, spills, and was slower:
+// 2.225 -> 2.269 ms per step).
 template <bool EXTRAS, int THREADS>
 __global__ void __launch_bounds__(THREADS, THREADS == 256 ? (EXTRAS ? 4 : 5) : 10) split_reduce_kernel(const ReduceParams p) {
     constexpr int kReduceThreads = THREADS;
