@@ -928,7 +928,7 @@ def main():
             "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
             "config": workload_config(args.workload, wl),
-            "run": {"kv_splits": args.kv_splits, "kernel_timing": "CUDA events around every %d%s attention launch" % (args.time_every, "th" if args.time_every != 1 else "st"), "schedule": "static" if args.static_schedule else "dynamic balancing (GQA kernel, launches long enough for it to pay: from 64 tiles per CTA)",
+            "run": {"kv_splits": args.kv_splits, "kernel_timing": "CUDA events around every %d%s attention launch" % (args.time_every, "th" if 10 <= args.time_every % 100 <= 20 else {1: "st", 2: "nd", 3: "rd"}.get(args.time_every % 10, "th")), "schedule": "static" if args.static_schedule else "dynamic balancing (GQA kernel, launches long enough for it to pay: from 64 tiles per CTA)",
                     "merge": "inside the split reduce" if fused else "separate ipkv_merge launch",
                     "append": "separate ipkv_append" if args.separate_append else "inside ipkv_attend_gpu (written by the attention kernel for GQA)",
                     "launch_overlap": "programmatic dependent launch; %d of %d attention launches started their copies before the previous kernel had completed"
