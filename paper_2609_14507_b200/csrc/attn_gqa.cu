@@ -404,11 +404,12 @@ __global__ void __launch_bounds__(kThreads, 2) attn_gqa_kernel(const GqaParams p
         return true;
     };
 
-    // start a partial: query fragments of its head group straight from global memory (a few KB, L2-resident), empty state
-    auto begin_partial = [&](int q_row, int nh) {
-        n_heads = nh;
+    // start a partial: query fragments of its head group straight from global memory (a few KB, L2-resident), then an empty
+    // state.  The two are separate because the fragments of the partial before are dead once its last scores are taken: at a
+    // change of partial the next one's loads are issued before the flush, so that their latency passes under it.
+    auto load_queries = [&](int q_row, int nh) {
         const __nv_bfloat16* qrow0 = p.q + (int64_t(q_row) + r0) * D + c0;
-        const bool v0 = r0 < n_heads, v1 = !DUP && (r0 + 8 < n_heads);
+        const bool v0 = r0 < nh, v1 = !DUP && (r0 + 8 < nh);
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks) {
             const uint32_t x0 = v0 ? __ldg(reinterpret_cast<const uint32_t*>(qrow0 + ks * 16)) : 0u;
@@ -420,6 +421,9 @@ __global__ void __launch_bounds__(kThreads, 2) attn_gqa_kernel(const GqaParams p
                 qa[ks][3] = v1 ? __ldg(reinterpret_cast<const uint32_t*>(qrow0 + 8 * D + ks * 16 + 8)) : 0u;
             }
         }
+    };
+    auto empty_state = [&](int nh) {
+        n_heads = nh;
 #pragma unroll
         for (int nt = 0; nt < D / 8; ++nt) { o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f; }
         m0 = m1 = -INFINITY; l0 = l1 = 0.f;
@@ -430,7 +434,8 @@ __global__ void __launch_bounds__(kThreads, 2) attn_gqa_kernel(const GqaParams p
         const Span first = p.spans[span_begin];
         const int g = first.gh / p.n_hg, hg = first.gh - g * p.n_hg;
         cur_slot = span_begin;
-        begin_partial(first.row * p.Hq + g * p.G + hg * 16, min(16, p.G - hg * 16));
+        load_queries(first.row * p.Hq + g * p.G + hg * 16, min(16, p.G - hg * 16));
+        empty_state(min(16, p.G - hg * 16));
     }
 
     for (;; ++it) {
@@ -438,10 +443,12 @@ __global__ void __launch_bounds__(kThreads, 2) attn_gqa_kernel(const GqaParams p
         if (!ptx::mbar_wait(s_full + 8 * st, (it / STAGES) & 1)) { ok = false; *s_gave_up = 1; break; }   // after a timeout: give up
         const int slot = s_meta[st].slot;
         if (slot != cur_slot) {
+            const int nh_next = s_meta[st].n_heads;
+            if (slot != kEndSlot) load_queries(s_meta[st].q_row, nh_next);
             if (cur_slot != kEndSlot && !flush()) { ok = false; break; }
             if (slot == kEndSlot) break;
             cur_slot = slot;
-            begin_partial(s_meta[st].q_row, s_meta[st].n_heads);
+            empty_state(nh_next);
         }
         const int n_valid = s_meta[st].n_valid;
         {
