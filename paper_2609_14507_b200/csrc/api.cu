@@ -724,7 +724,7 @@ void fill_launch(AttnLaunch* a, int kind, int Hq, int Hkv, int dqk, int dv, int 
     a->n_gh = pg.n_gh;
     int64_t tiles = 0;
     for (const Span& sp : plan.spans) tiles += sp.ntiles;
-    a->parts_per_span = parts_per_span_for(kind, tiles, int64_t(plan.spans.size()));
+    a->parts_per_span = parts_per_span_for(kind, tiles, int64_t(plan.spans.size()), int64_t(plan.n_ctas()));
     static const int forced_parts = [] { const char* e = std::getenv("IPKV_PARTS_PER_SPAN"); return e ? std::atoi(e) : 0; }();
     if (kind != 1 && (forced_parts == 1 || forced_parts == 4)) a->parts_per_span = forced_parts;     // test hook
     const size_t rows = (plan.spans.size() + extra_partials) * size_t(a->parts_per_span) * pg.rows_per_group;

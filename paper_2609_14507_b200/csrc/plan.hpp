@@ -79,14 +79,20 @@ struct Plan {
 // as one launch parameter (kSegTailParam); returns that offset (1..64), or 0 when the runs disagree or there are none.
 // How many partials a span writes.  The grouped-query kernel's four consumer warps run privately; at the end of a span they
 // either write a partial each, or join their states first (about a microsecond in which the CTA streams nothing, for a
-// reduce that reads a quarter of the entries).  Joining pays when spans are long.  Measured per step, joined against not,
-// by mean tiles per span: 116 (Mixtral shape, batch 16, 24K tokens) +0.7 %; 91 / 64 / 45 / 24 (Qwen3 shape, 32K tokens at CPU
-// shares 0 / 30 / 50 / 70 %) +1.5 / +1.4 / +0.5 / 0 %; 81 / 57 / 40 / 24 / 17 (ragged batch of 64 at shares 0 / 30 / 50 / 70 /
-// 90 %) +1.5 / +1.5 / -0.4 / -0.5 / -2.3 %.  The compressed-latent kernel's consumer warps share one state: one partial.
-constexpr int64_t kJoinWarpsFromTilesPerSpan = 48;
-inline int parts_per_span_for(int kind, int64_t tiles, int64_t spans) {
+// reduce that reads a quarter of the entries and ends about two microseconds sooner).  Joining pays when spans are long, or
+// when a CTA has few of them and they are not tiny.  Measured per step, joined against not, by mean tiles per span (and
+// spans per CTA): 116 (1.9; Mixtral shape, batch 16, 24K tokens) +0.7 %; 91 / 64 / 45 / 24 (1.4; Qwen3 shape, 32K tokens at
+// CPU shares 0 / 30 / 50 / 70 %) +1.5 / +1.4 / +0.5 / +0.3 %; 81 / 57 / 40 / 24 / 17 (2.7; ragged batch of 64 at shares 0 / 30 /
+// 50 / 70 / 90 %) +1.5 / +1.5 / -0.4 / -0.6 / -2.3 %; 1 (1.0; one sequence of 4K tokens) a kernel of 10.4 instead of 9.0 us.
+// The compressed-latent kernel's consumer warps share one state: one partial.
+constexpr int64_t kJoinWarpsFromTilesPerSpan = 48;        // long spans: always
+constexpr int64_t kJoinWarpsFromTilesPerSpanIfFew = 16;   // shorter ones: if a CTA has at most 1.6 spans on average
+inline int parts_per_span_for(int kind, int64_t tiles, int64_t spans, int64_t ctas) {
     if (kind == 1) return 1;
-    return (spans > 0 && tiles >= kJoinWarpsFromTilesPerSpan * spans) ? 1 : 4;
+    if (spans <= 0) return 4;
+    if (tiles >= kJoinWarpsFromTilesPerSpan * spans) return 1;
+    if (tiles >= kJoinWarpsFromTilesPerSpanIfFew * spans && 5 * spans <= 8 * ctas) return 1;
+    return 4;
 }
 
 inline int window_tail(std::vector<std::vector<PlanSeg>>& rows) {

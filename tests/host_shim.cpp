@@ -120,8 +120,10 @@ int shim_parts_per_span(int kind, int n_rows, const int64_t* tokens, int n_gh, i
     build_plan(rows, n_gh, 0, ctas_per_sm, &plan);
     int64_t tiles = 0;
     for (const Span& sp : plan.spans) tiles += sp.ntiles;
-    return parts_per_span_for(kind, tiles, int64_t(plan.spans.size()));
+    return parts_per_span_for(kind, tiles, int64_t(plan.spans.size()), int64_t(plan.n_ctas()));
 }
+
+int shim_parts_rule(int kind, int64_t tiles, int64_t spans, int64_t ctas) { return parts_per_span_for(kind, tiles, spans, ctas); }
 
 // Returns the launch parameter win_tail of the first step and, in *same_table, whether the two steps' serialised launch
 // tables are byte-identical (they must be, unless a window grows into a new tile, when the plan itself changes).

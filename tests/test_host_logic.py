@@ -308,7 +308,17 @@ def test_consumer_warps_join_their_partials_only_in_launches_with_long_spans():
 
     assert parts(0, [24577] * 16, 8, 2) == 1            # Mixtral shape at a quarter on the CPU: 116 tiles per span
     assert parts(0, [32769] * 16, 4, 2) == 1            # Qwen3 shape, everything on the GPU
-    assert parts(0, [9831] * 16, 4, 2) == 4             # the same at 70 % on the CPU: 24 tiles per span
+    assert parts(0, [9831] * 16, 4, 2) == 1             # the same at 70 % on the CPU: 24 tiles per span, but 1.2 spans per CTA
     assert parts(0, [4097], 4, 2) == 4                  # one short sequence: one tile per CTA
     assert parts(0, [100, 1], 4, 2) == 4
     assert parts(1, [78644] * 8, 1, 1) == 1 and parts(1, [100], 1, 1) == 1
+    # the rule itself on the launches it was measured on: (tiles, spans, CTAs)
+    L.shim_parts_rule.restype = C.c_int
+    L.shim_parts_rule.argtypes = [C.c_int, i64, i64, i64]
+    rule = lambda tiles, spans, ctas: L.shim_parts_rule(0, tiles, spans, ctas)
+    assert rule(65600, 808, 296) == 1 and rule(46000, 808, 296) == 1        # ragged batch of 64, CPU share 0 and 30 %: long spans
+    assert rule(32800, 808, 296) == 4 and rule(19700, 808, 296) == 4        # at 50 and 70 %: 41 and 24 tiles per span, 2.7 spans per CTA
+    assert rule(6600, 808, 296) == 4                                        # at 90 %
+    assert rule(9856, 424, 296) == 1                                        # Qwen3 shape at 70 %: 23 tiles per span, 1.4 spans per CTA
+    assert rule(260, 264, 260) == 4                                         # one 4K sequence: single-tile spans
+    assert rule(0, 0, 0) == 4
