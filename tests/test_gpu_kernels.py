@@ -217,16 +217,18 @@ def test_bounds_checked_build_passes_the_small_parity_cases():
     assert " passed" in r.stdout and "skipped" not in r.stdout.splitlines()[-1]
 
 
-@pytest.mark.parametrize("parts", ["1", "4"])
-def test_both_forms_of_the_span_partial_pass_the_small_parity_cases(parts):
+@pytest.mark.parametrize("parts,variant", [("1", ""), ("4", ""), ("1", "checked")])
+def test_both_forms_of_the_span_partial_pass_the_small_parity_cases(parts, variant):
     """The grouped-query kernel writes one partial per span (its four warps join their states through shared memory) in
     launches with long spans and four otherwise; small cases would only ever see the second form.  Here each form is
     forced in turn (IPKV_PARTS_PER_SPAN, read when the library is first used: a child process) and the small-shape parity
-    tests, ragged and balanced cases and the decode tests run against it."""
+    tests, ragged and balanced cases and the decode tests run against it; the joined form also in the bounds-checked build."""
     import os
     import subprocess
     import sys
     env = dict(os.environ, IPKV_PARTS_PER_SPAN=parts)
+    if variant:
+        env["IPKV_LIB_VARIANT"] = variant
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
     r = subprocess.run([sys.executable, "-m", "pytest", "-q", "-m", "gpu", "-x", os.path.join(root, "tests", "test_gpu_kernels.py"),
                         os.path.join(root, "tests", "test_gpu_cache.py"), "-k",
