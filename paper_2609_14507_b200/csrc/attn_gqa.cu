@@ -287,10 +287,11 @@ __global__ void __launch_bounds__(kThreads, 2) attn_gqa_kernel(const GqaParams p
         return true;
     };
 
-    // The partial of the tiles accumulated so far: the four warps' private states (each over its 16 tokens of every tile)
-    // joined into one normalised (O, LSE) per query head (Sec. 5.1's identity, in the log2 domain), so that the split reduce
-    // reads one partial per span.  Warp w scales its accumulators by exp2(m_w - M) / L; warp 0 stores its rows into the
-    // buffer, warps 1 and 2 add theirs in turn, warp 3 adds its own to the buffer's and writes the result out.
+    // The partial of the tiles accumulated so far.  Either every warp writes its own (p.NW == 4), or the four warps' private
+    // states (each over its 16 tokens of every tile) are joined into one normalised (O, LSE) per query head (Sec. 5.1's
+    // identity, in the log2 domain), so that the split reduce reads one partial per span: warp w scales its accumulators by
+    // exp2(m_w - M) / L; warp 0 stores its rows into the buffer, warps 1 and 2 add theirs in turn, warp 3 adds its own to
+    // the buffer's and writes the result out.
     auto flush = [&]() -> bool {
         l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
         l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
