@@ -33,7 +33,10 @@ def cpu_engine_commands(obj_dir):
     base = ["g++", "-std=c++17", "-O3", "-fopenmp", "-fPIC", "-Wno-psabi"]
     for src in sorted(glob.glob(os.path.join(CSRC, "*.cpp"))):
         name = os.path.basename(src)[:-4]
-        if name == "cpu_engine_kernel":
+        if name == "cpu_engine_amx":
+            obj = os.path.join(obj_dir, name + ".o")
+            out.append((base + ["-march=x86-64-v4", "-mamx-tile", "-mamx-bf16", "-c", src, "-o", obj], obj))
+        elif name == "cpu_engine_kernel":
             for level, flags in CPU_KERNEL_LEVELS:
                 obj = os.path.join(obj_dir, f"{name}_{level}.o")
                 out.append((base + flags + [f"-DIPKV_CPU_KERNEL=attend_chunk_{level}", "-c", src, "-o", obj], obj))

@@ -1,8 +1,9 @@
 // CPU-side in-place attention over the unpinned compute region (Sec. 6.1): the engine that produces the
 // CPU partial (O, LSE) which ipkv_merge joins with the GPU partial.
 //
-// Follows the paper's CPU kernel in spirit, written for whatever vector width the host has (the tile kernel,
-// cpu_engine_kernel.cpp, is compiled for AVX-512, AVX2 + FMA and baseline x86-64; one is picked at first use):
+// Follows the paper's CPU kernel in spirit, written for whatever the host has (the tile kernel, cpu_engine_kernel.cpp, is
+// compiled for AVX-512, AVX2 + FMA and baseline x86-64; cpu_engine_amx.cpp does the two contractions on the AMX tile unit
+// where there is one; the best available is picked at first use, IPKV_CPU_KERNEL=amx|v4|v3|base overrides for tests):
 //   * zero-copy: K/V are read where write-time routing put them — PLAIN blocks of region U, per KV head
 //     K[bt][dqk] then V[bt][dv], addressed with strides, never gathered into a contiguous copy;
 //   * scores are never materialised beyond a 16-token tile; online softmax keeps a running max and sum per
@@ -22,28 +23,73 @@
 #include <omp.h>
 #endif
 
+#if defined(__x86_64__) && defined(__linux__)
+#include <cpuid.h>
+#include <sys/syscall.h>
+#include <unistd.h>
+#endif
+#include <cstdlib>
+
 #include "cpu_engine.h"
 
 namespace ipkvi {
 
-// cpu_engine_kernel.cpp, compiled per instruction-set level
-void attend_chunk_v4(const CpuShape&, const float*, int, int, const CpuRun*, int, int64_t, int64_t, float*, float*, float*);
-void attend_chunk_v3(const CpuShape&, const float*, int, int, const CpuRun*, int, int64_t, int64_t, float*, float*, float*);
-void attend_chunk_base(const CpuShape&, const float*, int, int, const CpuRun*, int, int64_t, int64_t, float*, float*, float*);
+// cpu_engine_kernel.cpp, compiled per instruction-set level, and cpu_engine_amx.cpp: one item each; the queries come
+// widened and pre-scaled (fp32) and as their bf16 bits
+#define IPKV_CHUNK_ARGS const CpuShape&, const float*, const uint16_t*, int, int, const CpuRun*, int, int64_t, int64_t, float*, float*, float*
+void attend_chunk_amx(IPKV_CHUNK_ARGS);
+void attend_chunk_v4(IPKV_CHUNK_ARGS);
+void attend_chunk_v3(IPKV_CHUNK_ARGS);
+void attend_chunk_base(IPKV_CHUNK_ARGS);
 
 namespace {
 
-using ChunkFn = void (*)(const CpuShape&, const float*, int, int, const CpuRun*, int, int64_t, int64_t, float*, float*, float*);
+using ChunkFn = void (*)(IPKV_CHUNK_ARGS);
 
-ChunkFn pick_kernel() {
+bool cpu_has_avx512() {
 #if defined(__x86_64__) && defined(__GNUC__)
     __builtin_cpu_init();
-    if (__builtin_cpu_supports("avx512f") && __builtin_cpu_supports("avx512bw") && __builtin_cpu_supports("avx512dq") &&
-        __builtin_cpu_supports("avx512vl"))
-        return attend_chunk_v4;
-    if (__builtin_cpu_supports("avx2") && __builtin_cpu_supports("fma")) return attend_chunk_v3;
+    return __builtin_cpu_supports("avx512f") && __builtin_cpu_supports("avx512bw") && __builtin_cpu_supports("avx512dq") &&
+           __builtin_cpu_supports("avx512vl");
+#else
+    return false;
 #endif
-    return attend_chunk_base;
+}
+
+// AMX: the CPU must have the tile unit with bf16 products, and the kernel must grant this process the tile state.
+bool amx_usable() {
+#if defined(__x86_64__) && defined(__linux__)
+    if (!cpu_has_avx512()) return false;
+    unsigned a = 0, b = 0, c = 0, d = 0;
+    if (!__get_cpuid_count(7, 0, &a, &b, &c, &d)) return false;
+    if (!((d >> 22) & 1u) || !((d >> 24) & 1u)) return false;                 // AMX-BF16, AMX-TILE
+    constexpr long kArchReqXcompPerm = 0x1023, kXfeatureXtiledata = 18;
+    return syscall(SYS_arch_prctl, kArchReqXcompPerm, kXfeatureXtiledata) == 0;
+#else
+    return false;
+#endif
+}
+
+struct Kernels {
+    ChunkFn vec;        // the vector kernel for this host: any shape
+    ChunkFn amx;        // null where there is no tile unit: groups of at most 16 heads, dimensions in multiples of 32
+};
+
+Kernels pick_kernels() {
+    Kernels k{attend_chunk_base, nullptr};
+#if defined(__x86_64__) && defined(__GNUC__)
+    __builtin_cpu_init();
+    if (cpu_has_avx512()) k.vec = attend_chunk_v4;
+    else if (__builtin_cpu_supports("avx2") && __builtin_cpu_supports("fma")) k.vec = attend_chunk_v3;
+    if (amx_usable()) k.amx = attend_chunk_amx;
+    if (const char* want = std::getenv("IPKV_CPU_KERNEL")) {                  // tests: a lower level than the host's best
+        const bool avx512 = cpu_has_avx512(), avx2 = __builtin_cpu_supports("avx2") && __builtin_cpu_supports("fma");
+        if (!std::strcmp(want, "v4") && avx512) { k.vec = attend_chunk_v4; k.amx = nullptr; }
+        else if (!std::strcmp(want, "v3") && avx2) { k.vec = attend_chunk_v3; k.amx = nullptr; }
+        else if (!std::strcmp(want, "base")) { k.vec = attend_chunk_base; k.amx = nullptr; }
+    }
+#endif
+    return k;
 }
 
 struct Partial {            // online-softmax state of one (row, KV head, chunk): per head m, l; O is unnormalised
@@ -56,7 +102,8 @@ int cpu_attend_batch(const CpuShape& sh, int n_rows, const uint16_t* q, const Cp
                      float* o_out, float* lse_out, int n_threads) {
     const int G = sh.n_q_heads / sh.n_kv_heads;
     if (G > kCpuMaxGroup || sh.dim_qk > kCpuMaxDim || sh.dim_v > kCpuMaxDim || sh.dim_qk % 16 != 0 || sh.dim_v % 16 != 0) return -1;
-    static const ChunkFn attend = pick_kernel();
+    static const Kernels kernels = pick_kernels();
+    const ChunkFn attend = (kernels.amx && G <= 16 && sh.dim_qk % 32 == 0 && sh.dim_v % 32 == 0) ? kernels.amx : kernels.vec;
     struct Item { int row, g; int64_t t0, t1; };
     std::vector<Item> items;
     std::vector<int> first_item(size_t(n_rows) * sh.n_kv_heads + 1, 0);
@@ -89,7 +136,8 @@ int cpu_attend_batch(const CpuShape& sh, int n_rows, const uint16_t* q, const Cp
         const Item& it = items[size_t(i)];
         Partial& p = parts[size_t(i)];
         p.m.resize(G); p.l.resize(G); p.o.resize(size_t(G) * sh.dim_v);
-        attend(sh, qf.data() + (size_t(it.row) * sh.n_q_heads + size_t(it.g) * G) * sh.dim_qk, G, it.g,
+        const size_t q_off = (size_t(it.row) * sh.n_q_heads + size_t(it.g) * G) * sh.dim_qk;
+        attend(sh, qf.data() + q_off, q + q_off, G, it.g,
                      runs + row_run_start[it.row], row_run_start[it.row + 1] - row_run_start[it.row], it.t0, it.t1,
                      p.m.data(), p.l.data(), p.o.data());
     }
@@ -118,6 +166,13 @@ int cpu_attend_batch(const CpuShape& sh, int n_rows, const uint16_t* q, const Cp
             }
         }
     return 0;
+}
+
+const char* cpu_engine_kernel_name(const CpuShape& sh) {
+    static const Kernels kernels = pick_kernels();
+    const int G = sh.n_q_heads / sh.n_kv_heads;
+    if (kernels.amx && G <= 16 && sh.dim_qk % 32 == 0 && sh.dim_v % 32 == 0) return "amx";
+    return kernels.vec == attend_chunk_v4 ? "v4" : kernels.vec == attend_chunk_v3 ? "v3" : "base";
 }
 
 int cpu_engine_threads() {

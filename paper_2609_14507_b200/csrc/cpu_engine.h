@@ -24,5 +24,7 @@ struct CpuRun {
 int cpu_attend_batch(const CpuShape& sh, int n_rows, const uint16_t* q, const CpuRun* runs, const int32_t* row_run_start,
                      float* o_out, float* lse_out, int n_threads);
 int cpu_engine_threads();
+// Which tile kernel cpu_attend_batch uses for this shape on this host: "amx", "v4", "v3" or "base".
+const char* cpu_engine_kernel_name(const CpuShape& sh);
 
 }  // namespace ipkvi

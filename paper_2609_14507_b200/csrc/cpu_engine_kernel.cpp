@@ -100,7 +100,7 @@ __attribute__((always_inline)) inline void prefetch_rows(const char* p, int byte
 // widened K/V value loaded from L1 feeds several multiply-adds.
 }  // namespace
 
-void IPKV_CPU_KERNEL(const CpuShape& sh, const float* qf /*[G][dqk], pre-scaled*/, int G, int g,
+void IPKV_CPU_KERNEL(const CpuShape& sh, const float* qf /*[G][dqk], pre-scaled*/, const uint16_t* /*bf16 bits: not used here*/, int G, int g,
                   const CpuRun* runs, int n_runs, int64_t t_begin, int64_t t_end, float* m, float* l, float* o) {
     const int dqk = sh.dim_qk, dv = sh.dim_v;
     const bool alias_v = sh.dim_v_stored == 0;

@@ -21,7 +21,7 @@ def _lib():
     os.makedirs(obj_dir, exist_ok=True)
     cmds = lib_build.cpu_engine_commands(obj_dir)
     deps = [os.path.join(HERE, "cpu_engine_shim.cpp"), os.path.join(CSRC, "cpu_engine.h"), os.path.join(CSRC, "cpu_engine.cpp"),
-            os.path.join(CSRC, "cpu_engine_kernel.cpp")]
+            os.path.join(CSRC, "cpu_engine_kernel.cpp"), os.path.join(CSRC, "cpu_engine_amx.cpp")]
     if not os.path.exists(LIB) or os.path.getmtime(LIB) < max(os.path.getmtime(d) for d in deps):
         for cmd, _ in cmds:
             subprocess.run(cmd, check=True)
@@ -86,3 +86,35 @@ def test_cpu_engine_extremes():
     o, lse = run_engine(sh, kb, v, qb, [300], 64)
     o_ref, l_ref = c_oracle.attend(qb, kb, v, np.arange(300), float(np.float32(sh.scale)))
     assert np.abs(o - o_ref).max() < 1e-4 and np.abs(lse - l_ref).max() / abs(l_ref).max() < 1e-6
+
+
+@pytest.mark.parametrize("level", ["v4", "v3", "base"])
+def test_every_kernel_level_matches_the_oracle(level):
+    """The engine picks the best tile kernel the host has (the AMX one where there is a tile unit), so on such a host the
+    vector kernels would go untested: the same parity cases run once more with each level forced (IPKV_CPU_KERNEL, read
+    when the engine is first used: a child process).  A level the host cannot run falls back to the host's best."""
+    import sys
+    _lib()          # built once, here, not by the children at the same time
+    root = os.path.dirname(HERE)
+    env = dict(os.environ, IPKV_CPU_KERNEL=level)
+    r = subprocess.run([sys.executable, "-m", "pytest", "-q", "-x", os.path.join(HERE, "test_cpu_engine.py"), "-k",
+                        "matches_oracle or extremes or ragged_steps" ], env=env, cwd=root, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stdout[-3000:] + r.stderr[-2000:]
+
+
+@pytest.mark.parametrize("shape,bt,runs", [
+    (synth.Shape("g8", "gqa", 1, 32, 4, 128, 128, 128 ** -0.5), 64, [64, 31, 33, 1, 95, 2048 + 7]),     # steps straddle blocks and runs
+    (synth.Shape("g2d64", "gqa", 1, 4, 2, 64, 64, 64 ** -0.5), 32, [32, 32, 5, 64]),
+    (synth.Shape("g16", "gqa", 1, 16, 1, 128, 128, 128 ** -0.5), 128, [4096 + 40]),                     # several items of 2048 tokens
+    (synth.Shape("mla16", "mla", 1, 16, 1, 576, 512, 192 ** -0.5), 32, [31, 2049]),
+    (synth.Shape("g32", "gqa", 1, 32, 1, 128, 128, 128 ** -0.5), 64, [200]),                            # more heads than one tile holds
+])
+def test_cpu_engine_ragged_steps_and_wide_groups(shape, bt, runs):
+    """Shapes around the 32-token steps of the tile-unit kernel: runs that end inside a step, blocks smaller than a step,
+    steps that straddle a block boundary, groups that fill all 16 tile rows, and a group too wide for it."""
+    n = sum(runs)
+    k, v = synth.host_kv(shape, n, seed=77 + n)
+    q = synth.host_q(shape, 1, seed=78 + n)[0]
+    o, lse = run_engine(shape, k, v, q, runs, bt)
+    o_ref, l_ref = c_oracle.attend(q, k, shape.dim_v if v is None else v, np.arange(n), float(np.float32(shape.scale)))
+    assert np.abs(o - o_ref).max() < 2e-5 and np.abs(lse - l_ref).max() < 2e-5
