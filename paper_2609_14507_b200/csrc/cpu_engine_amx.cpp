@@ -135,42 +135,44 @@ void attend_chunk_amx(const CpuShape& sh, const float* /*qf*/, const uint16_t* q
     for (int r = 0; r < n_runs; ++r) {
         const int64_t run_last = run_first + runs[r].n_tokens;
         const int64_t lo = std::max(t_begin, run_first), hi = std::min(t_end, run_last);
-        auto head_of = [&](int64_t rel, int64_t* off) {
+        // where the K and V rows of `count` consecutive tokens of this run are (one division, then steps)
+        auto rows_of = [&](int64_t rel, int count, const char** kr, const char** vr) {
             const int64_t blk = rel / sh.bt;
-            *off = rel - blk * sh.bt;
-            return runs[r].blocks + blk * block_bytes + int64_t(g) * head_bytes;
+            int64_t off = rel - blk * sh.bt;
+            const char* head = runs[r].blocks + blk * block_bytes + int64_t(g) * head_bytes;
+            for (int j = 0; j < count; ++j) {
+                kr[j] = head + off * kpitch;
+                vr[j] = alias_v ? kr[j] : head + int64_t(sh.bt) * kpitch + off * vpitch;
+                if (++off == sh.bt) { off = 0; head += block_bytes; }
+            }
         };
         for (int64_t t0 = lo; t0 < hi; t0 += kStep) {
             const int nt = int(std::min<int64_t>(kStep, hi - t0));
             const int64_t rel0 = t0 - run_first;
+            const char* krow[kStep];
+            const char* vrow[kStep];
             // the rows two steps ahead, wherever their block is
-            for (int j = 0; j < kStep; j += 1) {
-                const int64_t rel = rel0 + 2 * kStep + j;
-                if (rel >= runs[r].n_tokens) break;
-                int64_t off;
-                const char* head = head_of(rel, &off);
-                const char* krow = head + off * kpitch;
-                for (int b = 0; b < kpitch; b += 64) _mm_prefetch(krow + b, _MM_HINT_T0);
-                if (!alias_v) {
-                    const char* vrow = head + int64_t(sh.bt) * kpitch + off * vpitch;
-                    for (int b = 0; b < vpitch; b += 64) _mm_prefetch(vrow + b, _MM_HINT_T0);
+            {
+                const int64_t rel = rel0 + 2 * kStep;
+                const int ahead = int(std::min<int64_t>(kStep, runs[r].n_tokens - rel));
+                if (ahead > 0) {
+                    rows_of(rel, ahead, krow, vrow);
+                    for (int j = 0; j < ahead; ++j) {
+                        for (int b = 0; b < kpitch; b += 64) _mm_prefetch(krow[j] + b, _MM_HINT_T0);
+                        if (!alias_v)
+                            for (int b = 0; b < vpitch; b += 64) _mm_prefetch(vrow[j] + b, _MM_HINT_T0);
+                    }
                 }
             }
-            int64_t off0;
-            const char* head0 = head_of(rel0, &off0);
-            const bool contiguous = nt == kStep && off0 + kStep <= sh.bt;
+            rows_of(rel0, nt, krow, vrow);
+            const bool contiguous = nt == kStep && krow[kStep - 1] == krow[0] + int64_t(kStep - 1) * kpitch;
             const char* kbase;
             if (contiguous) {
-                kbase = head0 + off0 * kpitch;
+                kbase = krow[0];
             } else {
                 for (int j = 0; j < kStep; ++j) {
-                    if (j < nt) {
-                        int64_t off;
-                        const char* head = head_of(rel0 + j, &off);
-                        std::memcpy(kstage + size_t(j) * dqk, head + off * kpitch, size_t(kpitch));
-                    } else {
-                        std::memset(kstage + size_t(j) * dqk, 0, size_t(kpitch));
-                    }
+                    if (j < nt) std::memcpy(kstage + size_t(j) * dqk, krow[j], size_t(kpitch));
+                    else std::memset(kstage + size_t(j) * dqk, 0, size_t(kpitch));
                 }
                 kbase = reinterpret_cast<const char*>(kstage);
             }
@@ -218,10 +220,8 @@ void attend_chunk_amx(const CpuShape& sh, const float* /*qf*/, const uint16_t* q
             // ---- V rows of every token pair, interleaved column by column ----
             for (int pr = 0; pr < kStep / 2; ++pr) {
                 const int j0 = 2 * pr, j1 = 2 * pr + 1;
-                const char* v0 = nullptr;
-                const char* v1 = nullptr;
-                if (j0 < nt) { int64_t off; const char* head = head_of(rel0 + j0, &off); v0 = alias_v ? head + off * kpitch : head + int64_t(sh.bt) * kpitch + off * vpitch; }
-                if (j1 < nt) { int64_t off; const char* head = head_of(rel0 + j1, &off); v1 = alias_v ? head + off * kpitch : head + int64_t(sh.bt) * kpitch + off * vpitch; }
+                const char* v0 = j0 < nt ? vrow[j0] : nullptr;
+                const char* v1 = j1 < nt ? vrow[j1] : nullptr;
                 for (int c = 0; c < dv; c += 32) {
                     const __m512i a = v0 ? _mm512_loadu_si512(v0 + c * 2) : _mm512_setzero_si512();
                     const __m512i b = v1 ? _mm512_loadu_si512(v1 + c * 2) : _mm512_setzero_si512();
