@@ -72,7 +72,7 @@ bool amx_usable() {
 
 struct Kernels {
     ChunkFn vec;        // the vector kernel for this host: any shape
-    ChunkFn amx;        // null where there is no tile unit: groups of at most 16 heads, dimensions in multiples of 32
+    ChunkFn amx;        // null where there is no tile unit: at most 16 heads a call, dimensions in multiples of 32
 };
 
 Kernels pick_kernels() {
@@ -103,7 +103,11 @@ int cpu_attend_batch(const CpuShape& sh, int n_rows, const uint16_t* q, const Cp
     const int G = sh.n_q_heads / sh.n_kv_heads;
     if (G > kCpuMaxGroup || sh.dim_qk > kCpuMaxDim || sh.dim_v > kCpuMaxDim || sh.dim_qk % 16 != 0 || sh.dim_v % 16 != 0) return -1;
     static const Kernels kernels = pick_kernels();
-    const ChunkFn attend = (kernels.amx && G <= 16 && sh.dim_qk % 32 == 0 && sh.dim_v % 32 == 0) ? kernels.amx : kernels.vec;
+    // the tile-unit kernel takes 16 query heads at a time: a wider group is done in slices (its rows are then read once per
+    // slice, the later times from cache)
+    const bool use_amx = kernels.amx && sh.dim_qk % 32 == 0 && sh.dim_v % 32 == 0;
+    const ChunkFn attend = use_amx ? kernels.amx : kernels.vec;
+    const int slice = use_amx ? 16 : G;
     struct Item { int row, g; int64_t t0, t1; };
     std::vector<Item> items;
     std::vector<int> first_item(size_t(n_rows) * sh.n_kv_heads + 1, 0);
@@ -137,9 +141,10 @@ int cpu_attend_batch(const CpuShape& sh, int n_rows, const uint16_t* q, const Cp
         Partial& p = parts[size_t(i)];
         p.m.resize(G); p.l.resize(G); p.o.resize(size_t(G) * sh.dim_v);
         const size_t q_off = (size_t(it.row) * sh.n_q_heads + size_t(it.g) * G) * sh.dim_qk;
-        attend(sh, qf.data() + q_off, q + q_off, G, it.g,
-                     runs + row_run_start[it.row], row_run_start[it.row + 1] - row_run_start[it.row], it.t0, it.t1,
-                     p.m.data(), p.l.data(), p.o.data());
+        for (int h0 = 0; h0 < G; h0 += slice)
+            attend(sh, qf.data() + q_off + size_t(h0) * sh.dim_qk, q + q_off + size_t(h0) * sh.dim_qk, std::min(slice, G - h0), it.g,
+                   runs + row_run_start[it.row], row_run_start[it.row + 1] - row_run_start[it.row], it.t0, it.t1,
+                   p.m.data() + h0, p.l.data() + h0, p.o.data() + size_t(h0) * sh.dim_v);
     }
     // join the chunk partials of every (row, head): exact LSE merge, natural-log LSE out
     for (int r = 0; r < n_rows; ++r)
@@ -170,8 +175,7 @@ int cpu_attend_batch(const CpuShape& sh, int n_rows, const uint16_t* q, const Cp
 
 const char* cpu_engine_kernel_name(const CpuShape& sh) {
     static const Kernels kernels = pick_kernels();
-    const int G = sh.n_q_heads / sh.n_kv_heads;
-    if (kernels.amx && G <= 16 && sh.dim_qk % 32 == 0 && sh.dim_v % 32 == 0) return "amx";
+    if (kernels.amx && sh.dim_qk % 32 == 0 && sh.dim_v % 32 == 0) return "amx";
     return kernels.vec == attend_chunk_v4 ? "v4" : kernels.vec == attend_chunk_v3 ? "v3" : "base";
 }
 

@@ -16,7 +16,8 @@
 // they are requested two steps ahead, across block boundaries.
 //
 // Compiled with -march=x86-64-v4 -mamx-tile -mamx-bf16; cpu_engine.cpp uses it only where the CPU has AMX and the kernel
-// grants the tile state (arch_prctl), for groups of at most 16 query heads and head dimensions that are multiples of 32.
+// grants the tile state (arch_prctl), for head dimensions that are multiples of 32; at most 16 query heads a call (a wider
+// group is done in slices).
 #include <immintrin.h>
 
 #include <algorithm>

@@ -107,11 +107,11 @@ def test_every_kernel_level_matches_the_oracle(level):
     (synth.Shape("g2d64", "gqa", 1, 4, 2, 64, 64, 64 ** -0.5), 32, [32, 32, 5, 64]),
     (synth.Shape("g16", "gqa", 1, 16, 1, 128, 128, 128 ** -0.5), 128, [4096 + 40]),                     # several items of 2048 tokens
     (synth.Shape("mla16", "mla", 1, 16, 1, 576, 512, 192 ** -0.5), 32, [31, 2049]),
-    (synth.Shape("g32", "gqa", 1, 32, 1, 128, 128, 128 ** -0.5), 64, [200]),                            # more heads than one tile holds
+    (synth.Shape("g32", "gqa", 1, 32, 1, 128, 128, 128 ** -0.5), 64, [200]),                            # more heads than one tile holds: done in slices of 16
 ])
 def test_cpu_engine_ragged_steps_and_wide_groups(shape, bt, runs):
     """Shapes around the 32-token steps of the tile-unit kernel: runs that end inside a step, blocks smaller than a step,
-    steps that straddle a block boundary, groups that fill all 16 tile rows, and a group too wide for it."""
+    steps that straddle a block boundary, groups that fill all 16 tile rows, and a group wider than that."""
     n = sum(runs)
     k, v = synth.host_kv(shape, n, seed=77 + n)
     q = synth.host_q(shape, 1, seed=78 + n)[0]
