@@ -233,10 +233,11 @@ ipkv_status ipkv_attend_cpu(ipkv_t* h, int32_t layer, const int32_t* seq_ids, in
 /* Exact n-way log-sum-exp join (Sec. 4.2, 5.1) of row-aligned partials over disjoint token sets:
  *   LSE = m + ln sum_i exp(LSE_i - m), m = max_i LSE_i;  O = sum_i exp(LSE_i - LSE) * O_i.
  * o_parts[i] [n_rows][dim_v] fp32, lse_parts[i] [n_rows] fp32; the pointer arrays are host memory;
- * each part may be device memory or host memory (host parts are copied on `stream` first; pinned host
- * memory keeps that copy asynchronous).  1 <= n_parts <= 8.  o_out_dev is fp32, or bf16 (round to
- * nearest even) when o_out_is_bf16 != 0.  lse_out_dev may be NULL.  h may be NULL only if every part is
- * device memory. */
+ * each part may be device memory or host memory.  A part in pinned (page-locked or registered) host memory is
+ * read by the kernel where it is, in stream order: it must stay unchanged until the call's work on `stream`
+ * has completed.  A part in pageable host memory is copied on `stream` first.  1 <= n_parts <= 8.
+ * o_out_dev is fp32, or bf16 (round to nearest even) when o_out_is_bf16 != 0.  lse_out_dev may be NULL.
+ * h may be NULL only if no part is pageable host memory. */
 ipkv_status ipkv_merge(ipkv_t* h, int32_t n_rows, int32_t dim_v, int32_t n_parts,
                        const float* const* o_parts, const float* const* lse_parts,
                        void* o_out_dev, int32_t o_out_is_bf16, float* lse_out_dev, void* stream);
