@@ -152,19 +152,28 @@ void attend_chunk_amx(const CpuShape& sh, const float* /*qf*/, const uint16_t* q
             const int64_t rel0 = t0 - run_first;
             const char* krow[kStep];
             const char* vrow[kStep];
-            // the rows two steps ahead, wherever their block is
+            // The rows two steps ahead, wherever their block is.  They are requested a few lines at a time between the phases
+            // below: a core has a dozen line-fill buffers, and hundreds of requests issued in one go would wait for them
+            // while nothing else runs.
+            const char* pf_k[kStep];
+            const char* pf_v[kStep];
+            int pf_rows = 0, pf_row = 0, pf_byte = 0;
             {
                 const int64_t rel = rel0 + 2 * kStep;
-                const int ahead = int(std::min<int64_t>(kStep, runs[r].n_tokens - rel));
-                if (ahead > 0) {
-                    rows_of(rel, ahead, krow, vrow);
-                    for (int j = 0; j < ahead; ++j) {
-                        for (int b = 0; b < kpitch; b += 64) _mm_prefetch(krow[j] + b, _MM_HINT_T0);
-                        if (!alias_v)
-                            for (int b = 0; b < vpitch; b += 64) _mm_prefetch(vrow[j] + b, _MM_HINT_T0);
-                    }
-                }
+                pf_rows = int(std::max<int64_t>(0, std::min<int64_t>(kStep, runs[r].n_tokens - rel)));
+                if (pf_rows > 0) rows_of(rel, pf_rows, pf_k, pf_v);
             }
+            const int pf_row_bytes = kpitch + (alias_v ? 0 : vpitch);
+            const int pf_slots = n_kc + kStep / 2 + (n_cb + 3) / 4;
+            const int pf_lines = (pf_rows * pf_row_bytes / 64 + pf_slots - 1) / pf_slots;
+            auto prefetch_some = [&]() {
+                for (int i = 0; i < pf_lines && pf_row < pf_rows; ++i) {
+                    const char* p = pf_byte < kpitch ? pf_k[pf_row] + pf_byte : pf_v[pf_row] + (pf_byte - kpitch);
+                    _mm_prefetch(p, _MM_HINT_T0);
+                    pf_byte += 64;
+                    if (pf_byte >= pf_row_bytes) { pf_byte = 0; ++pf_row; }
+                }
+            };
             rows_of(rel0, nt, krow, vrow);
             const bool contiguous = nt == kStep && krow[kStep - 1] == krow[0] + int64_t(kStep - 1) * kpitch;
             const char* kbase;
@@ -186,6 +195,7 @@ void attend_chunk_amx(const CpuShape& sh, const float* /*qf*/, const uint16_t* q
                 _tile_dpbf16ps(0, 6, 7);
                 _tile_loadd(5, kbase + 16 * kpitch + kc * 64, kpitch);
                 _tile_dpbf16ps(1, 5, 7);
+                prefetch_some();
             }
             _tile_stored(0, sbuf[0], 64);
             _tile_stored(1, sbuf[16], 64);
@@ -223,6 +233,7 @@ void attend_chunk_amx(const CpuShape& sh, const float* /*qf*/, const uint16_t* q
                 const int j0 = 2 * pr, j1 = 2 * pr + 1;
                 const char* v0 = j0 < nt ? vrow[j0] : nullptr;
                 const char* v1 = j1 < nt ? vrow[j1] : nullptr;
+                prefetch_some();
                 for (int c = 0; c < dv; c += 32) {
                     const __m512i a = v0 ? _mm512_loadu_si512(v0 + c * 2) : _mm512_setzero_si512();
                     const __m512i b = v1 ? _mm512_loadu_si512(v1 + c * 2) : _mm512_setzero_si512();
@@ -245,6 +256,7 @@ void attend_chunk_amx(const CpuShape& sh, const float* /*qf*/, const uint16_t* q
             _tile_loadd(5, p_lo, 64);
             for (int cb0 = 0; cb0 < n_cb; cb0 += 4) {
                 const int nb = std::min(4, n_cb - cb0);
+                prefetch_some();
                 // (tile numbers are immediates: the four column blocks are written out)
                 _tile_loadd(0, obuf + (cb0 + 0) * 16, dv * 4);
                 _tile_loadd(6, vn + size_t(cb0 + 0) * 16 * 32, 64);
