@@ -220,8 +220,11 @@ ipkv_status ipkv_attend_gpu_sparse(ipkv_t* h, int32_t layer, const int32_t* seq_
  * read where they lie (PLAIN blocks, no copy).  This is the paper's second engine, not a fallback for the GPU
  * path: it attends a disjoint token range and its partial is joined by ipkv_merge / the fold option.
  * q_host [n_seq][n_q_heads][dim_qk] bf16 in host memory; o_part_host [n_seq][n_q_heads][dim_v] and
- * lse_part_host [n_seq][n_q_heads] fp32 in host memory (pinned memory lets the later copy to the GPU overlap).
- * The call runs synchronously on the calling thread plus OpenMP workers (n_threads <= 0: all cores).
+ * lse_part_host [n_seq][n_q_heads] fp32 in host memory (in pinned memory ipkv_merge reads them where they are).
+ * The call runs synchronously on the calling thread plus OpenMP workers (n_threads <= 0: all cores).  The tile
+ * kernel is chosen at first use: the AMX tile unit where the CPU has one and the operating system grants its state,
+ * else AVX-512, AVX2 or baseline vector code; the environment variable IPKV_CPU_KERNEL=v4|v3|base forces a lower
+ * level (tests).  The levels agree within fp32 rounding.
  * U is filled by device-to-host copies queued by the append / flush calls: synchronise their stream first.
  * This call may run on a second host thread while ipkv_attend_gpu / ipkv_merge of the same handle run on the first
  * (the paper's step: both engines at once, one join): it only reads the routing state.  No call that changes routing
